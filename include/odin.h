@@ -1,0 +1,184 @@
+/* odin.h -- C ABI of the per-view training step of point-based (3D Gaussian) neural rendering on one B200.
+ *
+ * The paper schedules "training views": render one camera, compute an image loss, back-propagate, and update only the
+ * primitives that take part in the view (Sec. 2.1), in the phase order preprocessing / rendering / backward / optimizer
+ * update (Sec. 4.1 phase task graph, Fig. 7 labels P/R/B/U).  Its runtime publishes and checks, per view, the
+ * primitive-index scope the view may read and update (Sec. 2.1 scopes G_i, R_i^+, W_i^+; Sec. 4.3 hazard sets).  This
+ * library is that view step and that scope state as CUDA kernels for sm_100a; the paper leaves the renderer arithmetic to
+ * the 3D Gaussian Splatting method it builds on (Sec. 1), which is restated beside each call below.
+ *
+ * Conventions
+ *  - Pointers named d_* and every pointer inside odin_scene / odin_projected are DEVICE pointers owned by the caller.
+ *    Structs themselves (odin_scene, odin_projected, odin_camera, odin_config) are HOST structs read at call time.
+ *  - Every call enqueues its kernels on `stream` (a cudaStream_t passed as void*, NULL = default stream) and returns
+ *    without synchronising the host, except odin_create / odin_destroy / odin_poll.
+ *  - The library allocates device memory only inside odin_create (a few hundred bytes).  Scratch comes from the
+ *    caller's workspace `ws` (>= odin_workspace_bytes(), 256-byte aligned).  Calls on one context must not overlap on
+ *    the GPU when they share a workspace.
+ *  - Return value: ODIN_OK (0) or a negative odin_status.  Arguments are validated on the host before any launch.
+ *    Data-dependent failures (more rows or instances than the caller's capacity, a bounded device-side wait that ran
+ *    out) are recorded on the device, never write out of bounds, and are returned by the next odin_poll.
+ *  - Counts that are only known on the device (number of touched primitives V, number of (tile, primitive) instances
+ *    M) stay on the device: later calls take the device pointers and size their work from them.
+ *  - Row-major arrays; "row r" of a compact array belongs to primitive prim_id[r]; rows ascend with the primitive id.
+ *  - No call spins without a bound, traps, or aborts.
+ */
+#ifndef ODIN_H_
+#define ODIN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ODIN_OK = 0,
+  ODIN_ERR_NULL = -1,        /* a required pointer is NULL */
+  ODIN_ERR_INVALID_ARG = -2, /* bad size, degree, alignment, tile size ... */
+  ODIN_ERR_CAPACITY = -3,    /* deferred: V > row capacity or M > instance capacity; outputs are truncated */
+  ODIN_ERR_WORKSPACE = -4,   /* workspace missing, misaligned or too small */
+  ODIN_ERR_CUDA = -5,        /* a CUDA runtime call failed */
+  ODIN_ERR_TIMEOUT = -6,     /* deferred: a bounded device-side wait gave up; outputs of that call are invalid */
+  ODIN_ERR_UNSUPPORTED = -7
+} odin_status;
+
+typedef struct odin_ctx odin_ctx; /* opaque: device ordinal, configuration, deferred-status word */
+
+/* Renderer constants.  Defaults (pass NULL to odin_create): 1/255, 0.99, 1e-4, 0.3, 3, 1.3, 16. */
+typedef struct {
+  float alpha_min;     /* a contribution with alpha below this is skipped */
+  float alpha_max;     /* alpha clamp */
+  float t_min;         /* a pixel stops before the splat that would push its transmittance below this */
+  float dilation;      /* low-pass term added to both diagonal entries of the 2D covariance */
+  float radius_sigmas; /* screen extent in standard deviations of the major axis */
+  float jac_clamp;     /* t_x/t_z and t_y/t_z are clamped to +-jac_clamp * (half image / focal) inside the Jacobian */
+  int tile;            /* tile edge in pixels; only 16 is supported */
+} odin_config;
+
+/* Pinhole camera (host struct).  w2c is the row-major 3x4 world-to-camera matrix [R|t]; camera axes are x right,
+ * y down, z forward; pixel (i,j) is sampled at (i+0.5, j+0.5).  bg is the colour behind everything. */
+typedef struct {
+  int width, height;
+  float fx, fy, cx, cy, znear, zfar;
+  float w2c[12];
+  float bg[3];
+} odin_camera;
+
+/* The primitive pool as aligned per-attribute tensors indexed by primitive id (Sec. 2.1, Fig. 4).  The same struct
+ * shape holds the parameters, the two Adam moments, and a compact block of gradient rows (n = row capacity).
+ *   means [n][3], log_scales [n][3], quats [n][4] (w,x,y,z; normalised inside the step), opacity_logit [n],
+ *   sh [n][(sh_degree+1)^2][3].  All float32, each array 16-byte aligned. */
+typedef struct {
+  uint32_t n;
+  int sh_degree; /* 0..3 */
+  float* means;
+  float* log_scales;
+  float* quats;
+  float* opacity_logit;
+  float* sh;
+} odin_scene;
+
+/* Output of the preprocessing phase.  tiles_touched is dense (one entry per primitive, 0 = culled); everything else
+ * is compact: one row per visible primitive, rows in ascending primitive order, at most `capacity` rows. */
+typedef struct {
+  uint32_t capacity;        /* rows the compact arrays can hold */
+  uint32_t* tiles_touched;  /* [n]       number of 16x16 tiles the splat's rectangle covers (0 = not visible) */
+  uint32_t* prim_id;        /* [capacity] primitive id of the row */
+  float* xy;                /* [capacity][2] pixel-space centre (u, v) */
+  float* depth;             /* [capacity] camera-space z */
+  float* conic_opacity;     /* [capacity][4] inverse 2D covariance (A, B, C) and opacity */
+  float* rgb;               /* [capacity][3] view-dependent colour, clamped at 0 */
+  int32_t* radius;          /* [capacity] screen radius in pixels */
+  uint16_t* rect;           /* [capacity][4] tile rectangle x0,y0,x1,y1 (half open, tile units) */
+  uint32_t* tile_offset;    /* [capacity] exclusive prefix sum of tiles_touched over the rows */
+  uint8_t* clamp_flags;     /* [capacity] bit c set when colour channel c was clamped at 0 */
+  uint32_t* num_rows;       /* [1] V: number of rows written (device) */
+  uint64_t* num_instances;  /* [1] M: sum of tiles_touched (device) */
+} odin_projected;
+
+/* ---- context ------------------------------------------------------------------------------------------------- */
+
+/* Creates a context on CUDA device `device` (made current for the call).  cfg == NULL selects the defaults. */
+int odin_create(odin_ctx** ctx, int device, const odin_config* cfg);
+int odin_destroy(odin_ctx* ctx);
+const char* odin_status_string(int status);
+
+/* Synchronises `stream`, returns the first deferred device-side status since the last poll (ODIN_OK if none) and
+ * clears it. */
+int odin_poll(odin_ctx* ctx, void* stream);
+
+/* Workspace size sufficient for every call below with at most n primitives and `max_instances` instance capacity. */
+int odin_workspace_bytes(const odin_ctx* ctx, uint32_t n, uint64_t max_instances, size_t* bytes);
+
+/* ---- the seven calls of the view step ------------------------------------------------------------------------ */
+
+/* Preprocessing (phase P).  For every primitive: camera-space mean t = R mu + t_c; cull unless znear < t_z < zfar;
+ * Sigma = R(q) diag(exp(ls))^2 R(q)^T; Sigma' = J R_c Sigma R_c^T J^T + dilation I with the pinhole Jacobian J
+ * (ratio t_x/t_z, t_y/t_z clamped inside J only); conic = inverse of Sigma'; radius = ceil(radius_sigmas *
+ * sqrt(larger eigenvalue)); tile rectangle = floor/ceil of (centre -+ radius)/16 clamped to the grid, cull if empty;
+ * opacity = sigmoid(logit); colour = max(0, 0.5 + sum_k Y_k(dir) sh[k]) with the real SH basis up to degree 3 and
+ * dir the unit vector from the camera centre to the mean.  Writes `out` as described at odin_projected.  Rows beyond
+ * out->capacity are dropped and ODIN_ERR_CAPACITY is deferred; so is M >= 2^32. */
+int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_camera* cam, odin_projected* out, void* ws,
+                 size_t ws_bytes, void* stream);
+
+/* Touched set: the view's candidate scope G_i = R_i^+ = W_i^+ (Sec. 2.1), i.e. every primitive with tiles_touched > 0.
+ * d_mask [ceil(n/32)]: bit (p & 31) of word (p >> 5); d_idx: the ascending list of those primitive ids (first
+ * idx_capacity of them; more defers ODIN_ERR_CAPACITY); d_count [1]: their number V. */
+int odin_touched_set(odin_ctx* ctx, const uint32_t* d_tiles_touched, uint32_t n, uint32_t* d_mask, uint32_t* d_idx,
+                     uint32_t idx_capacity, uint32_t* d_count, void* ws, size_t ws_bytes, void* stream);
+
+/* Binning and sort.  Emits one (key, value) per (tile, row) pair of the rectangles: key = tile_id << 32 | bit pattern
+ * of the float32 depth, tile_id = ty * ceil(width/16) + tx; value = ROW index r (the primitive is proj->prim_id[r]).
+ * Sorts by key with a least-significant-digit radix sort (stable: equal keys keep ascending row order) and writes
+ * d_tile_ranges [tiles][2] = [first, one past last) position of each tile (an empty tile has first == last).
+ * Only the first `capacity` instances are produced when M > capacity (ODIN_ERR_CAPACITY deferred). */
+int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int width, int height, uint64_t* d_keys, uint32_t* d_vals,
+                  uint64_t capacity, uint32_t* d_tile_ranges, void* ws, size_t ws_bytes, void* stream);
+
+/* Rendering (phase R).  Per pixel, front to back over its tile's sorted rows: dx = u - x, dy = v - y,
+ * power = -(A dx^2 + C dy^2)/2 - B dx dy; skip if power > 0; alpha = min(alpha_max, opacity * exp(power)); skip if
+ * alpha < alpha_min; stop if T (1 - alpha) < t_min; colour += rgb * alpha * T; T *= 1 - alpha.
+ * d_rgb [3][H][W] = colour + T * bg (planar, not clamped); d_final_T [H][W]; d_n_contrib [H][W] = 1 + list offset of the
+ * last row that contributed (0 if none). */
+int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const uint32_t* d_vals, const uint32_t* d_tile_ranges,
+                    const odin_camera* cam, float* d_rgb, float* d_final_T, uint32_t* d_n_contrib, void* stream);
+
+/* Image loss of the view (Sec. 2.1): d_loss [1] = mean |rgb - target| over 3*H*W values;
+ * d_dL_drgb [3][H][W] = sign(rgb - target) / (3 H W). */
+int odin_l1_loss(odin_ctx* ctx, const float* d_rgb, const float* d_target, int width, int height, float* d_loss,
+                 float* d_dL_drgb, void* stream);
+
+/* Backward (phase B).  (a) Per pixel, back to front over the rows that contributed: gradients of the loss with
+ * respect to each row's colour, opacity, conic and centre (a clamped alpha passes no gradient), summed over pixels
+ * into d_grad2d [capacity][9] = (u, v, A, B, C, opacity, r, g, b).  (b) Per row: chain rule through the conic
+ * inverse, the EWA projection, the Jacobian (clamp frozen), Sigma = M M^T, scale = exp(log scale), the rotation and
+ * the quaternion normalisation, the pixel centre, the SH colour (clamped channels pass nothing; the direction term
+ * reaches the mean) and the sigmoid.  grad_rows: compact rows (row r <-> proj->prim_id[r]) in the layout of
+ * odin_scene with n >= V. */
+int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odin_camera* cam, const odin_projected* proj,
+                    const uint32_t* d_vals, const uint32_t* d_tile_ranges, const float* d_final_T,
+                    const uint32_t* d_n_contrib, const float* d_dL_drgb, float* d_grad2d, odin_scene* grad_rows,
+                    void* stream);
+
+/* Optimizer update (phase U) restricted to the touched rows: for every r < *d_count and every scalar theta of
+ * primitive d_idx[r] with gradient g: m = b1 m + (1-b1) g; v = b2 v + (1-b2) g^2;
+ * theta -= lr_group / (1 - b1^step) * m / (sqrt(v) / sqrt(1 - b2^step) + eps).  step is the global 1-based step.
+ * lr: mean, log scale, quaternion, opacity, SH degree 0, SH degrees >= 1.  Rows that are not listed are neither read
+ * nor written.  d_idx must be strictly ascending (as produced by odin_touched_set / odin_project). */
+int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m, odin_scene* v, const odin_scene* grad_rows,
+                     const uint32_t* d_idx, const uint32_t* d_count, const float lr[6], float beta1, float beta2,
+                     float eps, uint32_t step, void* stream);
+
+/* Conflict counts (Sec. 4.3): for each listed pair (a, b) of views, |W^+(a) & W^+(b)| = popcount of the AND of their
+ * touched bitmasks, the size of C_WAW^+ (C_RAW^+ and C_WAR^+ are empty because R^+ = W^+ here).
+ * d_masks [n_masks][mask_stride_words]; d_pairs [n_pairs][2] view slots; d_counts [n_pairs] (overwritten). */
+int odin_conflict_count(odin_ctx* ctx, const uint32_t* d_masks, uint32_t n_masks, uint32_t mask_stride_words,
+                        uint32_t n_prims, const uint32_t* d_pairs, uint32_t n_pairs, uint64_t* d_counts, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ODIN_H_ */

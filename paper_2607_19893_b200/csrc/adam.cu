@@ -1,0 +1,139 @@
+// Optimizer update restricted to the touched rows: bandwidth-bound gather / scatter Adam.
+// The gradient side is read fully coalesced (consecutive threads, consecutive floats of the compact rows); the
+// parameter side touches, per row, one contiguous span per attribute array (192 B for degree-3 SH = six full sectors).
+#include "common.cuh"
+
+namespace {
+
+struct AdamK {
+  float beta1, beta2, omb1, omb2, eps;
+  float step_size[6];  // lr_g / (1 - beta1^t)
+  float inv_bc2s;      // 1 / sqrt(1 - beta2^t)
+};
+
+__device__ __forceinline__ void adam_one(float& th, float& m, float& v, float g, float step_size, const AdamK& k) {
+  m = k.beta1 * m + k.omb1 * g;
+  v = k.beta2 * v + k.omb2 * g * g;
+  th = th - step_size * m / (sqrtf(v) * k.inv_bc2s + k.eps);
+}
+
+// SH block: ROWF floats per row (3, 12, 27 or 48), processed as VEC-wide elements; element e of the compact
+// gradient block belongs to row e / (ROWF / VEC).
+template <int ROWF, int VEC>
+__global__ void __launch_bounds__(256)
+adam_sh_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v, const float* __restrict__ g,
+               const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count, uint32_t cap, AdamK k) {
+  constexpr int EPR = ROWF / VEC;  // elements per row
+  const uint32_t V = min(*count, cap);
+  const size_t total = (size_t)V * EPR;
+  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+    const uint32_t r = (uint32_t)(e / EPR);
+    const uint32_t j = (uint32_t)(e - (size_t)r * EPR);
+    const size_t dst = (size_t)idx[r] * ROWF + (size_t)j * VEC;
+    if (VEC == 4) {
+      const float4 gg = reinterpret_cast<const float4*>(g)[e];
+      float4 pp = *reinterpret_cast<float4*>(p + dst), mm = *reinterpret_cast<float4*>(m + dst),
+             vv = *reinterpret_cast<float4*>(v + dst);
+      // floats 0..2 of a row are the degree-0 coefficients (group 4); the rest group 5
+      const int f0 = j * 4;
+      adam_one(pp.x, mm.x, vv.x, gg.x, k.step_size[f0 + 0 < 3 ? 4 : 5], k);
+      adam_one(pp.y, mm.y, vv.y, gg.y, k.step_size[f0 + 1 < 3 ? 4 : 5], k);
+      adam_one(pp.z, mm.z, vv.z, gg.z, k.step_size[f0 + 2 < 3 ? 4 : 5], k);
+      adam_one(pp.w, mm.w, vv.w, gg.w, k.step_size[5], k);
+      *reinterpret_cast<float4*>(p + dst) = pp;
+      *reinterpret_cast<float4*>(m + dst) = mm;
+      *reinterpret_cast<float4*>(v + dst) = vv;
+    } else {
+      float pp = p[dst], mm = m[dst], vv = v[dst];
+      adam_one(pp, mm, vv, g[e], k.step_size[j < 3 ? 4 : 5], k);
+      p[dst] = pp; m[dst] = mm; v[dst] = vv;
+    }
+  }
+}
+
+// Geometry block: one thread per row handles mean(3), log scale(3), quaternion(4), opacity(1).
+__global__ void __launch_bounds__(256)
+adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* __restrict__ p_q, float* __restrict__ p_o,
+                 float* __restrict__ m_mean, float* __restrict__ m_ls, float4* __restrict__ m_q, float* __restrict__ m_o,
+                 float* __restrict__ v_mean, float* __restrict__ v_ls, float4* __restrict__ v_q, float* __restrict__ v_o,
+                 const float* __restrict__ g_mean, const float* __restrict__ g_ls, const float4* __restrict__ g_q,
+                 const float* __restrict__ g_o, const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count,
+                 uint32_t cap, AdamK k) {
+  const uint32_t V = min(*count, cap);
+  for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
+    const size_t d = idx[r];
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+      float pp = p_mean[3 * d + i], mm = m_mean[3 * d + i], vv = v_mean[3 * d + i];
+      adam_one(pp, mm, vv, g_mean[3 * (size_t)r + i], k.step_size[0], k);
+      p_mean[3 * d + i] = pp; m_mean[3 * d + i] = mm; v_mean[3 * d + i] = vv;
+    }
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+      float pp = p_ls[3 * d + i], mm = m_ls[3 * d + i], vv = v_ls[3 * d + i];
+      adam_one(pp, mm, vv, g_ls[3 * (size_t)r + i], k.step_size[1], k);
+      p_ls[3 * d + i] = pp; m_ls[3 * d + i] = mm; v_ls[3 * d + i] = vv;
+    }
+    {
+      float4 pp = p_q[d], mm = m_q[d], vv = v_q[d];
+      const float4 gg = g_q[r];
+      adam_one(pp.x, mm.x, vv.x, gg.x, k.step_size[2], k);
+      adam_one(pp.y, mm.y, vv.y, gg.y, k.step_size[2], k);
+      adam_one(pp.z, mm.z, vv.z, gg.z, k.step_size[2], k);
+      adam_one(pp.w, mm.w, vv.w, gg.w, k.step_size[2], k);
+      p_q[d] = pp; m_q[d] = mm; v_q[d] = vv;
+    }
+    {
+      float pp = p_o[d], mm = m_o[d], vv = v_o[d];
+      adam_one(pp, mm, vv, g_o[r], k.step_size[3], k);
+      p_o[d] = pp; m_o[d] = mm; v_o[d] = vv;
+    }
+  }
+}
+
+}  // namespace
+
+extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m, odin_scene* v,
+                                const odin_scene* grad_rows, const uint32_t* d_idx, const uint32_t* d_count,
+                                const float lr[6], float beta1, float beta2, float eps, uint32_t step, void* stream) {
+  if (!ctx || !lr || !d_count) return ODIN_ERR_NULL;
+  int rc = odin_check_scene(params);
+  if (rc == ODIN_OK) rc = odin_check_scene(m);
+  if (rc == ODIN_OK) rc = odin_check_scene(v);
+  if (rc == ODIN_OK) rc = odin_check_scene(grad_rows);
+  if (rc != ODIN_OK) return rc;
+  if (m->n != params->n || v->n != params->n || m->sh_degree != params->sh_degree || v->sh_degree != params->sh_degree ||
+      grad_rows->sh_degree != params->sh_degree)
+    return ODIN_ERR_INVALID_ARG;
+  if (step == 0 || !(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f))
+    return ODIN_ERR_INVALID_ARG;
+  if (params->n == 0 || grad_rows->n == 0) return ODIN_OK;
+  if (!d_idx) return ODIN_ERR_NULL;
+  AdamK k;
+  k.beta1 = beta1; k.beta2 = beta2; k.omb1 = 1.f - beta1; k.omb2 = 1.f - beta2; k.eps = eps;
+  const float bc1 = 1.f - (float)pow((double)beta1, (double)step);
+  const float bc2s = (float)sqrt(1.0 - pow((double)beta2, (double)step));
+  for (int i = 0; i < 6; ++i) k.step_size[i] = lr[i] / bc1;
+  k.inv_bc2s = 1.f / bc2s;
+  cudaStream_t st = (cudaStream_t)stream;
+  const uint32_t cap = grad_rows->n;
+  const int K = (params->sh_degree + 1) * (params->sh_degree + 1);
+  const size_t max_elems = (size_t)cap * (K == 9 ? 27 : (K == 1 ? 3 : 3 * K / 4));
+  size_t blocks = (max_elems + 255) / 256;
+  if (blocks > (size_t)ctx->sm_count * 16) blocks = (size_t)ctx->sm_count * 16;
+  const unsigned gsh = (unsigned)blocks;
+  switch (params->sh_degree) {
+    case 0: adam_sh_kernel<3, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
+    case 1: adam_sh_kernel<12, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
+    case 2: adam_sh_kernel<27, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
+    default: adam_sh_kernel<48, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
+  }
+  size_t gb = ((size_t)cap + 255) / 256;
+  if (gb > (size_t)ctx->sm_count * 16) gb = (size_t)ctx->sm_count * 16;
+  adam_geom_kernel<<<(unsigned)gb, 256, 0, st>>>(
+      params->means, params->log_scales, reinterpret_cast<float4*>(params->quats), params->opacity_logit, m->means,
+      m->log_scales, reinterpret_cast<float4*>(m->quats), m->opacity_logit, v->means, v->log_scales,
+      reinterpret_cast<float4*>(v->quats), v->opacity_logit, grad_rows->means, grad_rows->log_scales,
+      reinterpret_cast<const float4*>(grad_rows->quats), grad_rows->opacity_logit, d_idx, d_count, cap, k);
+  return odin_launch_status();
+}

@@ -1,0 +1,79 @@
+// Context management, deferred status and workspace sizing of the C ABI.
+#include <new>
+
+#include "common.cuh"
+#include "layout.cuh"
+
+extern "C" int odin_create(odin_ctx** out, int device, const odin_config* cfg) {
+  if (!out) return ODIN_ERR_NULL;
+  *out = nullptr;
+  odin_config c = {1.0f / 255.0f, 0.99f, 1e-4f, 0.3f, 3.0f, 1.3f, 16};
+  if (cfg) c = *cfg;
+  if (c.tile != 16) return ODIN_ERR_UNSUPPORTED;
+  if (!(c.alpha_min > 0) || !(c.alpha_max < 1) || !(c.alpha_max > c.alpha_min) || !(c.t_min > 0) || !(c.dilation >= 0) ||
+      !(c.radius_sigmas > 0) || !(c.jac_clamp > 0))
+    return ODIN_ERR_INVALID_ARG;
+  ODIN_CUDA(cudaSetDevice(device));
+  odin_ctx* ctx = new (std::nothrow) odin_ctx();
+  if (!ctx) return ODIN_ERR_CUDA;
+  ctx->device = device;
+  ctx->cfg = c;
+  ctx->d_status = nullptr;
+  ctx->h_status = nullptr;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess || cudaMalloc(&ctx->d_status, 256) != cudaSuccess ||
+      cudaMallocHost(&ctx->h_status, sizeof(int)) != cudaSuccess || cudaMemset(ctx->d_status, 0, 256) != cudaSuccess) {
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->h_status) cudaFreeHost(ctx->h_status);
+    delete ctx;
+    return ODIN_ERR_CUDA;
+  }
+  ctx->sm_count = prop.multiProcessorCount;
+  *ctx->h_status = 0;
+  *out = ctx;
+  return ODIN_OK;
+}
+
+extern "C" int odin_destroy(odin_ctx* ctx) {
+  if (!ctx) return ODIN_ERR_NULL;
+  cudaFree(ctx->d_status);
+  cudaFreeHost(ctx->h_status);
+  delete ctx;
+  return ODIN_OK;
+}
+
+extern "C" const char* odin_status_string(int s) {
+  switch (s) {
+    case ODIN_OK: return "ok";
+    case ODIN_ERR_NULL: return "null pointer";
+    case ODIN_ERR_INVALID_ARG: return "invalid argument";
+    case ODIN_ERR_CAPACITY: return "capacity exceeded (outputs truncated)";
+    case ODIN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case ODIN_ERR_CUDA: return "CUDA runtime error";
+    case ODIN_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    case ODIN_ERR_UNSUPPORTED: return "unsupported";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int odin_poll(odin_ctx* ctx, void* stream) {
+  if (!ctx) return ODIN_ERR_NULL;
+  cudaStream_t st = (cudaStream_t)stream;
+  ODIN_CUDA(cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  ODIN_CUDA(cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st));
+  ODIN_CUDA(cudaStreamSynchronize(st));
+  const int s = *ctx->h_status;
+  *ctx->h_status = 0;
+  return s;
+}
+
+extern "C" int odin_workspace_bytes(const odin_ctx* ctx, uint32_t n, uint64_t max_instances, size_t* bytes) {
+  if (!ctx || !bytes) return ODIN_ERR_NULL;
+  size_t b = project_ws_bytes(n);
+  const size_t t = touched_ws_bytes(n);
+  const size_t s = binsort_ws_bytes(max_instances);
+  if (t > b) b = t;
+  if (s > b) b = s;
+  *bytes = b;
+  return ODIN_OK;
+}

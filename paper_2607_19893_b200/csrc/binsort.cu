@@ -1,0 +1,319 @@
+// Tile binning and sort: instance emission (load balanced over instances), digit histograms, a onesweep
+// least-significant-digit radix sort with decoupled look-back (no library sort), and the per-tile ranges.
+#include "common.cuh"
+#include "layout.cuh"
+
+namespace {
+
+// ------------------------------------------------------------------------------------------------ emission
+constexpr int DUP_THREADS = 256;
+constexpr int DUP_ITEMS = 8;
+constexpr int DUP_CHUNK = DUP_THREADS * DUP_ITEMS;  // instances per chunk; a chunk spans at most DUP_CHUNK rows
+
+// Cooperative 256-ary upper bound: first r in [0, V) with off[r] > x (V if none).  All threads must call.
+__device__ __forceinline__ uint32_t block_upper_bound(const uint32_t* __restrict__ off, uint32_t V, uint32_t x) {
+  uint32_t lo = 0, hi = V;
+  while (lo < hi) {
+    const uint32_t span = hi - lo;
+    const uint32_t step = (span + DUP_THREADS - 1) / DUP_THREADS;
+    const uint32_t probe = lo + threadIdx.x * step;
+    const int below = (probe < hi) && (off[probe] <= x);
+    const uint32_t cnt = (uint32_t)__syncthreads_count(below);  // monotone predicate: the first cnt probes are <= x
+    if (cnt == 0) { hi = lo; break; }
+    const uint32_t new_lo = lo + (cnt - 1) * step + 1;
+    const uint32_t new_hi = min(hi, lo + cnt * step);
+    lo = new_lo; hi = new_hi;
+  }
+  return lo;
+}
+
+// Each chunk of DUP_CHUNK consecutive instance slots finds the rows it overlaps, stages their offsets, rectangles and
+// depths in shared memory, and every thread expands its slots: slot i of row r is tile (y0 + k / w, x0 + k % w) with
+// k = i - offset[r], w = x1 - x0.  Keys and values are written fully coalesced.  Digit histograms for the sort are
+// accumulated on the way: depth digits once per row (weighted by the row's slots in the chunk), tile digits per
+// slot with warp aggregation.
+__global__ void __launch_bounds__(DUP_THREADS)
+emit_instances_kernel(const uint32_t* __restrict__ tile_offset, const ushort4* __restrict__ rect,
+                      const float* __restrict__ depth, const uint32_t* __restrict__ num_rows,
+                      const uint64_t* __restrict__ num_instances, uint64_t capacity, int TX, int passes,
+                      uint64_t* __restrict__ keys, uint32_t* __restrict__ vals, uint32_t* __restrict__ hist, int* status) {
+  __shared__ uint32_t s_off[DUP_CHUNK + 1];
+  __shared__ ushort4 s_rect[DUP_CHUNK];
+  __shared__ uint32_t s_depth[DUP_CHUNK];
+  __shared__ uint32_t s_hist[SORT_MAX_PASSES][SORT_RADIX];
+  const uint32_t V = *num_rows;
+  const uint64_t M_all = *num_instances;
+  const uint64_t M64 = M_all < capacity ? M_all : capacity;
+  if (blockIdx.x == 0 && threadIdx.x == 0 && M_all > capacity) odin_set_error(status, ODIN_ERR_CAPACITY);
+  const uint32_t M = (uint32_t)(M64 < 0xffffffffull ? M64 : 0xffffffffull);
+  for (int i = threadIdx.x; i < SORT_MAX_PASSES * (int)SORT_RADIX; i += DUP_THREADS) (&s_hist[0][0])[i] = 0;
+  __syncthreads();
+  const uint32_t chunks = V == 0 ? 0u : (M + DUP_CHUNK - 1) / DUP_CHUNK;
+  const unsigned lane = threadIdx.x & 31;
+  for (uint32_t chunk = blockIdx.x; chunk < chunks; chunk += gridDim.x) {
+    const uint32_t c0 = chunk * DUP_CHUNK;
+    const uint32_t c1 = (M - c0 < (uint32_t)DUP_CHUNK) ? M : c0 + DUP_CHUNK;
+    const uint32_t row_lo = block_upper_bound(tile_offset, V, c0) - 1;  // offset[0] = 0 <= c0, so the bound is >= 1
+    const uint32_t row_hi = block_upper_bound(tile_offset, V, c1 - 1) - 1;
+    const uint32_t nrows = row_hi - row_lo + 1;  // <= DUP_CHUNK: every row owns at least one slot
+    for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS) {
+      s_off[i] = tile_offset[row_lo + i];
+      s_rect[i] = rect[row_lo + i];
+      s_depth[i] = __float_as_uint(depth[row_lo + i]);
+    }
+    if (threadIdx.x == 0) s_off[nrows] = (row_hi + 1 < V) ? tile_offset[row_hi + 1] : (uint32_t)M_all;
+    __syncthreads();
+    // depth digits, once per row
+    for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS) {
+      const uint32_t b = max(s_off[i], c0), e = min(s_off[i + 1], c1);
+      const uint32_t wgt = e - b, bits = s_depth[i];
+#pragma unroll
+      for (int d = 0; d < 4; ++d) atomicAdd(&s_hist[d][(bits >> (8 * d)) & 255u], wgt);
+    }
+#pragma unroll
+    for (int k = 0; k < DUP_ITEMS; ++k) {
+      const uint32_t i = c0 + k * DUP_THREADS + threadIdx.x;
+      const bool valid = i < c1;
+      uint32_t tile = 0xffffffffu;
+      if (valid) {
+        uint32_t lo = 0, hi = nrows;  // last j with s_off[j] <= i
+        while (hi - lo > 1) {
+          const uint32_t mid = (lo + hi) >> 1;
+          if (s_off[mid] <= i) lo = mid; else hi = mid;
+        }
+        const ushort4 rc = s_rect[lo];
+        const uint32_t local = i - s_off[lo];
+        const uint32_t w = (uint32_t)rc.z - (uint32_t)rc.x;
+        const uint32_t dy = local / w, dx = local - dy * w;
+        tile = ((uint32_t)rc.y + dy) * (uint32_t)TX + (uint32_t)rc.x + dx;
+        keys[i] = ((uint64_t)tile << 32) | (uint64_t)s_depth[lo];
+        vals[i] = row_lo + lo;
+      }
+      for (int d = 4; d < passes; ++d) {
+        const uint32_t digit = valid ? ((tile >> (8 * (d - 4))) & 255u) : (256u + lane);
+        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+        if (valid && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&s_hist[d][digit], (uint32_t)__popc(peers));
+      }
+    }
+    __syncthreads();
+  }
+  for (int i = threadIdx.x; i < passes * (int)SORT_RADIX; i += DUP_THREADS) {
+    const uint32_t c = (&s_hist[0][0])[i];
+    if (c) atomicAdd(&hist[i], c);
+  }
+}
+
+// exclusive scan of each pass's 256-bin histogram (one block per pass)
+__global__ void __launch_bounds__(SORT_RADIX) digit_base_kernel(const uint32_t* __restrict__ hist, uint32_t* __restrict__ base) {
+  __shared__ uint32_t s_warp[33];
+  uint32_t total;
+  const uint32_t h = hist[blockIdx.x * SORT_RADIX + threadIdx.x];
+  base[blockIdx.x * SORT_RADIX + threadIdx.x] = odin_block_exclusive_sum(h, s_warp, &total);
+}
+
+// ------------------------------------------------------------------------------------------------ onesweep pass
+constexpr int OS_THREADS = 256;
+constexpr int OS_WARPS = OS_THREADS / 32;
+constexpr int OS_ITEMS = SORT_TILE / OS_THREADS;  // 16 keys per thread
+constexpr uint32_t OS_FLAG_AGG = 1u << 30, OS_FLAG_INC = 2u << 30, OS_VALUE = (1u << 30) - 1;
+constexpr size_t OS_SMEM = (size_t)SORT_TILE * 8 + (size_t)SORT_TILE * 4 + (size_t)OS_WARPS * SORT_RADIX * 4 + 2 * SORT_RADIX * 4 + 16;
+
+// One pass over one 8-bit digit.  Persistent blocks take 4096-key tiles by ticket.  Per tile: warp-striped loads,
+// per-warp digit ranking with match.any (stable), block digit counts published for look-back, exclusive global digit
+// offsets by a per-digit look-back walk (thread d walks digit d), keys and values exchanged through shared memory so
+// that the global scatter writes runs of consecutive addresses.
+__global__ void __launch_bounds__(OS_THREADS)
+onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in, uint64_t* __restrict__ keys_out,
+                uint32_t* __restrict__ vals_out, const uint64_t* __restrict__ num_instances, uint64_t capacity, int shift,
+                const uint32_t* __restrict__ digit_base, uint32_t* states, uint32_t* ticket, int* status) {
+  extern __shared__ __align__(16) unsigned char os_smem[];
+  uint64_t* s_keys = reinterpret_cast<uint64_t*>(os_smem);
+  uint32_t* s_vals = reinterpret_cast<uint32_t*>(os_smem + (size_t)SORT_TILE * 8);
+  uint32_t(*s_warp_hist)[SORT_RADIX] = reinterpret_cast<uint32_t(*)[SORT_RADIX]>(os_smem + (size_t)SORT_TILE * 12);
+  uint32_t* s_digit_start = reinterpret_cast<uint32_t*>(os_smem + (size_t)SORT_TILE * 12 + (size_t)OS_WARPS * SORT_RADIX * 4);
+  uint32_t* s_global = s_digit_start + SORT_RADIX;
+  uint32_t* s_misc = s_global + SORT_RADIX;  // [0] tile ticket
+  __shared__ uint32_t s_scan[33];
+
+  const uint64_t M_all = *num_instances;
+  const uint64_t M64 = M_all < capacity ? M_all : capacity;
+  const uint32_t M = (uint32_t)(M64 < (uint64_t)OS_VALUE ? M64 : (uint64_t)OS_VALUE);
+  const uint32_t ntiles = (M + SORT_TILE - 1) / SORT_TILE;
+  const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t lt_mask = (1u << lane) - 1u;
+
+  while (true) {
+    if (threadIdx.x == 0) s_misc[0] = atomicAdd(ticket, 1u);
+    for (int i = threadIdx.x; i < OS_WARPS * (int)SORT_RADIX; i += OS_THREADS) (&s_warp_hist[0][0])[i] = 0;
+    __syncthreads();
+    const uint32_t tile = s_misc[0];
+    if (tile >= ntiles) break;
+    const uint32_t tile_base = tile * SORT_TILE;
+    const uint32_t tile_count = min((uint32_t)SORT_TILE, M - tile_base);
+    const uint32_t warp_base = tile_base + warp * (32 * OS_ITEMS);
+
+    uint64_t key[OS_ITEMS];
+    uint32_t val[OS_ITEMS];
+    uint32_t pos[OS_ITEMS];
+#pragma unroll
+    for (int j = 0; j < OS_ITEMS; ++j) {
+      const uint32_t i = warp_base + 32 * j + lane;
+      key[j] = (i < M) ? keys_in[i] : ~0ull;  // padding sorts to the end of the tile and is never written
+      val[j] = (i < M) ? vals_in[i] : 0u;
+    }
+#pragma unroll
+    for (int j = 0; j < OS_ITEMS; ++j) {
+      const uint32_t d = (uint32_t)(key[j] >> shift) & (SORT_RADIX - 1);
+      const uint32_t peers = __match_any_sync(0xffffffffu, d);
+      const int leader = __ffs(peers) - 1;
+      uint32_t old = 0;
+      if ((int)lane == leader) {
+        old = s_warp_hist[warp][d];
+        s_warp_hist[warp][d] = old + __popc(peers);
+      }
+      old = __shfl_sync(0xffffffffu, old, leader);
+      pos[j] = old + __popc(peers & lt_mask);
+      __syncwarp();
+    }
+    __syncthreads();
+
+    // thread d owns digit d
+    const uint32_t d = threadIdx.x;
+    uint32_t cta_count = 0;
+#pragma unroll
+    for (int w = 0; w < OS_WARPS; ++w) {
+      const uint32_t t = s_warp_hist[w][d];
+      s_warp_hist[w][d] = cta_count;  // exclusive offset of warp w inside digit d
+      cta_count += t;
+    }
+    uint32_t* my_state = states + (size_t)tile * SORT_RADIX + d;
+    st_volatile_u32(my_state, (tile == 0 ? OS_FLAG_INC : OS_FLAG_AGG) | cta_count);
+    uint32_t total;
+    const uint32_t digit_start = odin_block_exclusive_sum(cta_count, s_scan, &total);
+    s_digit_start[d] = digit_start;
+    uint32_t exclusive = 0;
+    if (tile > 0) {
+      int64_t t = (int64_t)tile - 1;
+      int spins = 0;
+      while (t >= 0) {
+        const uint32_t s = ld_volatile_u32(states + (size_t)t * SORT_RADIX + d);
+        const uint32_t flag = s >> 30;
+        if (flag == 0) {
+          __nanosleep(64);
+          if (++spins > ODIN_SPIN_LIMIT) { odin_set_error(status, ODIN_ERR_TIMEOUT); break; }
+          continue;
+        }
+        exclusive += s & OS_VALUE;
+        if (flag == 2) break;
+        --t;
+      }
+      st_volatile_u32(my_state, OS_FLAG_INC | ((exclusive + cta_count) & OS_VALUE));
+    }
+    s_global[d] = digit_base[d] + exclusive - digit_start;  // add the slot index inside the tile to get the address
+    __syncthreads();
+
+#pragma unroll
+    for (int j = 0; j < OS_ITEMS; ++j) {
+      const uint32_t dg = (uint32_t)(key[j] >> shift) & (SORT_RADIX - 1);
+      const uint32_t slot = s_digit_start[dg] + s_warp_hist[warp][dg] + pos[j];
+      s_keys[slot] = key[j];
+      s_vals[slot] = val[j];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < OS_ITEMS; ++j) {
+      const uint32_t slot = j * OS_THREADS + threadIdx.x;
+      if (slot < tile_count) {
+        const uint64_t k = s_keys[slot];
+        const uint32_t dst = s_global[(uint32_t)(k >> shift) & (SORT_RADIX - 1)] + slot;
+        if (dst < M) {
+          keys_out[dst] = k;
+          vals_out[dst] = s_vals[slot];
+        }
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ ranges
+__global__ void __launch_bounds__(256)
+tile_ranges_kernel(const uint64_t* __restrict__ keys, const uint64_t* __restrict__ num_instances, uint64_t capacity,
+                   uint32_t n_tiles, uint32_t* __restrict__ ranges) {
+  const uint64_t M_all = *num_instances;
+  const uint64_t M = M_all < capacity ? M_all : capacity;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < M; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint32_t t = (uint32_t)(keys[i] >> 32);
+    if (t >= n_tiles) continue;
+    if (i == 0) ranges[2 * t] = 0;
+    else {
+      const uint32_t tp = (uint32_t)(keys[i - 1] >> 32);
+      if (tp != t) {
+        ranges[2 * t] = (uint32_t)i;
+        if (tp < n_tiles) ranges[2 * tp + 1] = (uint32_t)i;
+      }
+    }
+    if (i == M - 1) ranges[2 * t + 1] = (uint32_t)M;
+  }
+}
+
+int sort_passes(int n_tiles) {
+  int tile_bits = 0;
+  while ((1ll << tile_bits) < (long long)n_tiles) ++tile_bits;
+  return (32 + tile_bits + (int)SORT_RADIX_BITS - 1) / (int)SORT_RADIX_BITS;
+}
+
+}  // namespace
+
+extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int width, int height, uint64_t* d_keys,
+                             uint32_t* d_vals, uint64_t capacity, uint32_t* d_tile_ranges, void* ws, size_t ws_bytes,
+                             void* stream) {
+  if (!ctx || !proj || !d_tile_ranges) return ODIN_ERR_NULL;
+  if (width <= 0 || height <= 0 || width > 16384 || height > 16384) return ODIN_ERR_INVALID_ARG;
+  if (!proj->num_rows || !proj->num_instances) return ODIN_ERR_NULL;
+  if (capacity >= (1ull << 30)) return ODIN_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int TX = (width + 15) / 16, TY = (height + 15) / 16;
+  const uint32_t n_tiles = (uint32_t)TX * (uint32_t)TY;
+  ODIN_CUDA(cudaMemsetAsync(d_tile_ranges, 0, (size_t)n_tiles * 8, st));
+  if (capacity == 0 || proj->capacity == 0) return ODIN_OK;
+  if (!d_keys || !d_vals || !proj->tile_offset || !proj->rect || !proj->depth) return ODIN_ERR_NULL;
+  if (!odin_aligned(d_keys, 16) || !odin_aligned(d_vals, 16) || !odin_aligned(proj->rect, 8)) return ODIN_ERR_INVALID_ARG;
+  const BinSortLayout L = binsort_layout(capacity);
+  if (!ws || !odin_aligned(ws, 256) || ws_bytes < L.total) return ODIN_ERR_WORKSPACE;
+  char* base = reinterpret_cast<char*>(ws);
+  const int passes = sort_passes((int)n_tiles);
+  // zero tickets, histograms and the look-back words of the passes that will run
+  const size_t zero = L.states + (size_t)passes * L.tiles * SORT_RADIX * 4;
+  ODIN_CUDA(cudaMemsetAsync(base, 0, zero, st));
+  uint32_t* tickets = reinterpret_cast<uint32_t*>(base + L.header);
+  uint32_t* hist = reinterpret_cast<uint32_t*>(base + L.hist);
+  uint32_t* dbase = reinterpret_cast<uint32_t*>(base + L.digit_base);
+  uint32_t* states = reinterpret_cast<uint32_t*>(base + L.states);
+  uint64_t* alt_keys = reinterpret_cast<uint64_t*>(base + L.alt_keys);
+  uint32_t* alt_vals = reinterpret_cast<uint32_t*>(base + L.alt_vals);
+  // with an odd number of passes the emission goes to the alternate buffers so that the last pass lands in d_keys
+  uint64_t* kbuf[2] = {d_keys, alt_keys};
+  uint32_t* vbuf[2] = {d_vals, alt_vals};
+  int cur = passes & 1;
+
+  const uint64_t chunks_cap = (capacity + DUP_CHUNK - 1) / DUP_CHUNK;
+  uint32_t grid = (uint32_t)(chunks_cap < (uint64_t)ctx->sm_count * 6 ? chunks_cap : (uint64_t)ctx->sm_count * 6);
+  emit_instances_kernel<<<grid, DUP_THREADS, 0, st>>>(proj->tile_offset, reinterpret_cast<const ushort4*>(proj->rect),
+                                                      proj->depth, proj->num_rows, proj->num_instances, capacity, TX,
+                                                      passes, kbuf[cur], vbuf[cur], hist, ctx->d_status);
+  digit_base_kernel<<<passes, SORT_RADIX, 0, st>>>(hist, dbase);
+  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OS_SMEM));
+  uint32_t os_grid = L.tiles < (uint32_t)ctx->sm_count * 3 ? L.tiles : (uint32_t)ctx->sm_count * 3;
+  for (int p = 0; p < passes; ++p) {
+    onesweep_kernel<<<os_grid, OS_THREADS, OS_SMEM, st>>>(kbuf[cur], vbuf[cur], kbuf[cur ^ 1], vbuf[cur ^ 1],
+                                                          proj->num_instances, capacity, p * (int)SORT_RADIX_BITS,
+                                                          dbase + p * SORT_RADIX, states + (size_t)p * L.tiles * SORT_RADIX,
+                                                          tickets + p, ctx->d_status);
+    cur ^= 1;
+  }
+  const uint64_t rblocks = (capacity + 255) / 256;
+  const uint32_t rgrid = (uint32_t)(rblocks < (uint64_t)ctx->sm_count * 8 ? rblocks : (uint64_t)ctx->sm_count * 8);
+  tile_ranges_kernel<<<rgrid, 256, 0, st>>>(d_keys, proj->num_instances, capacity, n_tiles, d_tile_ranges);
+  return odin_launch_status();
+}

@@ -1,0 +1,294 @@
+// Backward phase: (a) per-tile back-to-front replay of the compositing with warp-transposed reductions of the nine
+// per-row gradient words, block-level accumulation in shared memory and one global atomic per (tile, row, word);
+// (b) per-row chain rule through the projection into compact gradient rows.
+#include "geom.cuh"
+
+namespace {
+
+constexpr int BB = 256;  // threads per block = pixels per tile = rows per batch
+
+__global__ void zero_rows_kernel(float* __restrict__ g2d, const uint32_t* __restrict__ num_rows, uint32_t capacity) {
+  const uint32_t V = min(*num_rows, capacity);
+  const size_t count = (size_t)V * 9;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x) g2d[i] = 0.f;
+}
+
+// Sums eight values across the warp with 9 shuffles: at each of the first three steps a lane hands half of its
+// values to its partner and keeps the other half, so after offsets 16, 8, 4 every lane holds one value summed over
+// 8 lanes; offsets 2 and 1 finish it.  On return lane 4*v holds the warp total of value v.
+__device__ __forceinline__ float warp_transpose_sum8(float a0, float a1, float a2, float a3, float a4, float a5, float a6,
+                                                     float a7, unsigned lane) {
+  const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4;
+  float b0 = (h16 ? a4 : a0) + __shfl_xor_sync(0xffffffffu, h16 ? a0 : a4, 16);
+  float b1 = (h16 ? a5 : a1) + __shfl_xor_sync(0xffffffffu, h16 ? a1 : a5, 16);
+  float b2 = (h16 ? a6 : a2) + __shfl_xor_sync(0xffffffffu, h16 ? a2 : a6, 16);
+  float b3 = (h16 ? a7 : a3) + __shfl_xor_sync(0xffffffffu, h16 ? a3 : a7, 16);
+  float c0 = (h8 ? b2 : b0) + __shfl_xor_sync(0xffffffffu, h8 ? b0 : b2, 8);
+  float c1 = (h8 ? b3 : b1) + __shfl_xor_sync(0xffffffffu, h8 ? b1 : b3, 8);
+  float d = (h4 ? c1 : c0) + __shfl_xor_sync(0xffffffffu, h4 ? c0 : c1, 4);
+  d += __shfl_xor_sync(0xffffffffu, d, 2);
+  d += __shfl_xor_sync(0xffffffffu, d, 1);
+  return d;
+}
+
+__global__ void __launch_bounds__(BB)
+render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
+                        const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
+                        float bg0, float bg1, float bg2, float alpha_min, float alpha_max,
+                        const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
+                        const float* __restrict__ dL, float* __restrict__ g2d) {
+  __shared__ float2 s_xy[BB];
+  __shared__ float4 s_co[BB];
+  __shared__ float s_rgb[BB][3];
+  __shared__ uint32_t s_row[BB];
+  __shared__ float s_acc[BB * 9];
+  __shared__ uint32_t s_max;
+  const int tile = blockIdx.x;
+  const int tx = tile % TX, ty = tile / TX;
+  const int lx = threadIdx.x & 15, ly = threadIdx.x >> 4;
+  const int px = tx * 16 + lx, py = ty * 16 + ly;
+  const bool inside = px < W && py < H;
+  const unsigned lane = threadIdx.x & 31;
+  const float fx = (float)px + 0.5f, fy = (float)py + 0.5f;
+  const uint32_t start = ranges[tile].x;
+  const size_t pix = (size_t)py * W + px, plane = (size_t)W * H;
+  float T = 1.f, g0 = 0.f, g1 = 0.f, g2 = 0.f;
+  uint32_t last = 0;
+  if (inside) {
+    T = final_T[pix];
+    last = n_contrib[pix];
+    g0 = dL[pix]; g1 = dL[plane + pix]; g2 = dL[2 * plane + pix];
+  }
+  if (threadIdx.x == 0) s_max = 0;
+  for (int i = threadIdx.x; i < BB * 9; i += BB) s_acc[i] = 0.f;
+  __syncthreads();
+  {
+    uint32_t m = last;
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0 && m) atomicMax(&s_max, m);
+  }
+  __syncthreads();
+  const uint32_t total = s_max;  // list entries any pixel of the tile used
+  float S0 = T * bg0, S1 = T * bg1, S2 = T * bg2;
+  const int nb = (int)((total + BB - 1) / BB);
+  for (int bi = nb - 1; bi >= 0; --bi) {
+    const uint32_t b = (uint32_t)bi * BB;
+    const int cnt = (int)min((uint32_t)BB, total - b);
+    if ((int)threadIdx.x < cnt) {
+      const uint32_t r = vals[start + b + threadIdx.x];
+      s_row[threadIdx.x] = r;
+      s_xy[threadIdx.x] = xy[r];
+      s_co[threadIdx.x] = conic_o[r];
+      s_rgb[threadIdx.x][0] = rgb[3 * (size_t)r];
+      s_rgb[threadIdx.x][1] = rgb[3 * (size_t)r + 1];
+      s_rgb[threadIdx.x][2] = rgb[3 * (size_t)r + 2];
+    }
+    __syncthreads();
+    for (int j = cnt - 1; j >= 0; --j) {
+      const float2 c = s_xy[j];
+      const float4 co = s_co[j];
+      const float dx = c.x - fx, dy = c.y - fy;
+      const float power = -0.5f * (co.x * dx * dx + co.z * dy * dy) - co.y * dx * dy;
+      const float G = __expf(power);
+      const float og = co.w * G;
+      const float alpha = fminf(alpha_max, og);
+      const bool on = (b + j < last) && (power <= 0.f) && (alpha >= alpha_min);
+      if (__ballot_sync(0xffffffffu, on) == 0) continue;
+      float vu = 0.f, vv = 0.f, vA = 0.f, vB = 0.f, vC = 0.f, vo = 0.f, vr = 0.f, vg = 0.f, vb = 0.f;
+      if (on) {
+        const float inv = 1.f / (1.f - alpha);
+        const float Tb = T * inv;  // transmittance in front of this row
+        const float w = alpha * Tb;
+        const float c0 = s_rgb[j][0], c1 = s_rgb[j][1], c2 = s_rgb[j][2];
+        vr = w * g0; vg = w * g1; vb = w * g2;
+        const float dLda = (c0 * Tb - S0 * inv) * g0 + (c1 * Tb - S1 * inv) * g1 + (c2 * Tb - S2 * inv) * g2;
+        S0 += c0 * w; S1 += c1 * w; S2 += c2 * w;
+        T = Tb;
+        if (og <= alpha_max) {
+          const float gp = G * co.w * dLda;
+          vu = (-co.x * dx - co.y * dy) * gp;
+          vv = (-co.z * dy - co.y * dx) * gp;
+          vA = -0.5f * dx * dx * gp;
+          vB = -dx * dy * gp;
+          vC = -0.5f * dy * dy * gp;
+          vo = G * dLda;
+        }
+      }
+      const float t8 = warp_transpose_sum8(vu, vv, vA, vB, vC, vo, vr, vg, lane);
+      for (int o = 16; o > 0; o >>= 1) vb += __shfl_xor_sync(0xffffffffu, vb, o);
+      if ((lane & 3) == 0) atomicAdd(&s_acc[j * 9 + (lane >> 2)], t8);
+      if (lane == 1) atomicAdd(&s_acc[j * 9 + 8], vb);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < cnt * 9; i += BB) {
+      const float v = s_acc[i];
+      if (v != 0.f) {
+        atomicAdd(&g2d[(size_t)s_row[i / 9] * 9 + (i % 9)], v);
+        s_acc[i] = 0.f;
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// ----------------------------------------------------------------------------------------------------------------
+template <int DEG>
+__global__ void __launch_bounds__(128)
+render_bwd_project_kernel(const float* __restrict__ means, const float* __restrict__ log_scales,
+                          const float4* __restrict__ quats, const float* __restrict__ opacity_logit,
+                          const float* __restrict__ sh, CamParams cam, float dilation, const uint32_t* __restrict__ prim_id,
+                          const uint8_t* __restrict__ clamp_flags, const uint32_t* __restrict__ num_rows, uint32_t capacity,
+                          const float* __restrict__ g2d, float* __restrict__ g_means, float* __restrict__ g_ls,
+                          float4* __restrict__ g_quats, float* __restrict__ g_opac, float* __restrict__ g_sh) {
+  constexpr int K = (DEG + 1) * (DEG + 1);
+  const uint32_t V = min(*num_rows, capacity);
+  for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
+    const size_t p = prim_id[r];
+    const float* gg = g2d + (size_t)r * 9;
+    const float gu = gg[0], gv = gg[1], gA = gg[2], gB = gg[3], gC = gg[4], go = gg[5];
+    const float grgb[3] = {gg[6], gg[7], gg[8]};
+    const float mx = means[3 * p], my = means[3 * p + 1], mz = means[3 * p + 2];
+    SplatGeom g;
+    odin_camera_space(cam, mx, my, mz, g.t);
+    const float ls[3] = {log_scales[3 * p], log_scales[3 * p + 1], log_scales[3 * p + 2]};
+    odin_splat_geometry(cam, dilation, ls, quats[p], g);
+    // conic -> 2D covariance
+    const float a = g.a, b = g.b, c = g.c, D = g.det * g.det;
+    const float ga = (-c * c * gA + b * c * gB - b * b * gC) / D;
+    const float gb = (2.f * b * c * gA - (a * c + b * b) * gB + 2.f * a * b * gC) / D;
+    const float gc = (-b * b * gA + a * b * gB - a * a * gC) / D;
+    const float Gs[4] = {ga, 0.5f * gb, 0.5f * gb, gc};
+    float GT[6];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 3; ++j) GT[3 * i + j] = Gs[2 * i] * g.Tm[j] + Gs[2 * i + 1] * g.Tm[3 + j];
+    const float S[9] = {g.Sig[0], g.Sig[1], g.Sig[2], g.Sig[1], g.Sig[3], g.Sig[4], g.Sig[2], g.Sig[4], g.Sig[5]};
+    float gSig[9], gTm[6];
+#pragma unroll
+    for (int i = 0; i < 3; ++i)
+#pragma unroll
+      for (int j = 0; j < 3; ++j) gSig[3 * i + j] = g.Tm[i] * GT[j] + g.Tm[3 + i] * GT[3 + j];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 3; ++j) gTm[3 * i + j] = 2.f * (GT[3 * i] * S[j] + GT[3 * i + 1] * S[3 + j] + GT[3 * i + 2] * S[6 + j]);
+    // dL/dJ = dL/dTm R_c^T; only J00, J02, J11, J12 depend on t
+    const float gJ00 = gTm[0] * cam.R[0] + gTm[1] * cam.R[1] + gTm[2] * cam.R[2];
+    const float gJ02 = gTm[0] * cam.R[6] + gTm[1] * cam.R[7] + gTm[2] * cam.R[8];
+    const float gJ11 = gTm[3] * cam.R[3] + gTm[4] * cam.R[4] + gTm[5] * cam.R[5];
+    const float gJ12 = gTm[3] * cam.R[6] + gTm[4] * cam.R[7] + gTm[5] * cam.R[8];
+    const float tx = g.t[0], ty = g.t[1], tz = g.t[2];
+    const float iz = 1.f / tz, iz2 = iz * iz, iz3 = iz2 * iz;
+    float gt0 = 0.f, gt1 = 0.f, gt2 = -(gJ00 * cam.fx + gJ11 * cam.fy) * iz2;
+    if (g.clampx) gt2 += gJ02 * cam.fx * g.Lx * iz2;
+    else { gt0 += -gJ02 * cam.fx * iz2; gt2 += 2.f * gJ02 * cam.fx * tx * iz3; }
+    if (g.clampy) gt2 += gJ12 * cam.fy * g.Ly * iz2;
+    else { gt1 += -gJ12 * cam.fy * iz2; gt2 += 2.f * gJ12 * cam.fy * ty * iz3; }
+    gt0 += gu * cam.fx * iz; gt2 += -gu * cam.fx * tx * iz2;
+    gt1 += gv * cam.fy * iz; gt2 += -gv * cam.fy * ty * iz2;
+    float gmu[3];
+#pragma unroll
+    for (int j = 0; j < 3; ++j) gmu[j] = cam.R[j] * gt0 + cam.R[3 + j] * gt1 + cam.R[6 + j] * gt2;
+    // Sigma = M M^T
+    float gM[9], gR[9], gls[3];
+#pragma unroll
+    for (int i = 0; i < 3; ++i)
+#pragma unroll
+      for (int j = 0; j < 3; ++j)
+        gM[3 * i + j] = 2.f * (gSig[3 * i] * g.M[j] + gSig[3 * i + 1] * g.M[3 + j] + gSig[3 * i + 2] * g.M[6 + j]);
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+      float gs = 0.f;
+#pragma unroll
+      for (int i = 0; i < 3; ++i) { gs += g.Rm[3 * i + j] * gM[3 * i + j]; gR[3 * i + j] = gM[3 * i + j] * g.s[j]; }
+      gls[j] = g.s[j] * gs;
+    }
+    const float w = g.qn[0], x = g.qn[1], y = g.qn[2], z = g.qn[3];
+    float gq[4];
+    gq[0] = 2.f * (-z * gR[1] + y * gR[2] + z * gR[3] - x * gR[5] - y * gR[6] + x * gR[7]);
+    gq[1] = 2.f * (y * gR[1] + z * gR[2] + y * gR[3] - 2.f * x * gR[4] - w * gR[5] + z * gR[6] + w * gR[7] - 2.f * x * gR[8]);
+    gq[2] = 2.f * (-2.f * y * gR[0] + x * gR[1] + w * gR[2] + x * gR[3] + z * gR[5] - w * gR[6] + z * gR[7] - 2.f * y * gR[8]);
+    gq[3] = 2.f * (-2.f * z * gR[0] - w * gR[1] + x * gR[2] + w * gR[3] - 2.f * z * gR[4] + y * gR[5] + x * gR[6] + y * gR[7]);
+    const float qd = w * gq[0] + x * gq[1] + y * gq[2] + z * gq[3];
+    const float iq = 1.f / g.qlen;
+    // colour
+    float dvx = mx - cam.pos[0], dvy = my - cam.pos[1], dvz = mz - cam.pos[2];
+    const float len = sqrtf(dvx * dvx + dvy * dvy + dvz * dvz);
+    const float d0 = dvx / len, d1 = dvy / len, d2 = dvz / len;
+    float Y[16], dY[16][3];
+    odin_sh_basis<DEG>(d0, d1, d2, Y);
+    odin_sh_basis_grad<DEG>(d0, d1, d2, dY);
+    const uint8_t flags = clamp_flags[r];
+    float gch[3];
+#pragma unroll
+    for (int ch = 0; ch < 3; ++ch) gch[ch] = (flags & (1u << ch)) ? 0.f : grgb[ch];
+    float gd[3] = {0.f, 0.f, 0.f};
+    const float* shrow = sh + p * (3 * K);
+    float* gshrow = g_sh + (size_t)r * (3 * K);
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+#pragma unroll
+      for (int ch = 0; ch < 3; ++ch) {
+        gshrow[3 * k + ch] = Y[k] * gch[ch];
+        if (k > 0) {
+          const float wgt = shrow[3 * k + ch] * gch[ch];
+          gd[0] += dY[k][0] * wgt; gd[1] += dY[k][1] * wgt; gd[2] += dY[k][2] * wgt;
+        }
+      }
+    }
+    const float dd = d0 * gd[0] + d1 * gd[1] + d2 * gd[2];
+    gmu[0] += (gd[0] - d0 * dd) / len; gmu[1] += (gd[1] - d1 * dd) / len; gmu[2] += (gd[2] - d2 * dd) / len;
+    g_means[3 * (size_t)r] = gmu[0]; g_means[3 * (size_t)r + 1] = gmu[1]; g_means[3 * (size_t)r + 2] = gmu[2];
+    g_ls[3 * (size_t)r] = gls[0]; g_ls[3 * (size_t)r + 1] = gls[1]; g_ls[3 * (size_t)r + 2] = gls[2];
+    g_quats[r] = make_float4((gq[0] - w * qd) * iq, (gq[1] - x * qd) * iq, (gq[2] - y * qd) * iq, (gq[3] - z * qd) * iq);
+    const float o = 1.f / (1.f + expf(-opacity_logit[p]));
+    g_opac[r] = o * (1.f - o) * go;
+  }
+}
+
+}  // namespace
+
+extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odin_camera* cam, const odin_projected* proj,
+                               const uint32_t* d_vals, const uint32_t* d_tile_ranges, const float* d_final_T,
+                               const uint32_t* d_n_contrib, const float* d_dL_drgb, float* d_grad2d, odin_scene* grad_rows,
+                               void* stream) {
+  if (!ctx || !proj || !grad_rows) return ODIN_ERR_NULL;
+  int rc = odin_check_scene(scene);
+  if (rc != ODIN_OK) return rc;
+  rc = odin_check_camera(cam);
+  if (rc != ODIN_OK) return rc;
+  rc = odin_check_scene(grad_rows);
+  if (rc != ODIN_OK) return rc;
+  if (grad_rows->sh_degree != scene->sh_degree) return ODIN_ERR_INVALID_ARG;
+  if (proj->capacity == 0 || scene->n == 0) return ODIN_OK;
+  if (grad_rows->n < proj->capacity) return ODIN_ERR_INVALID_ARG;
+  if (!d_vals || !d_tile_ranges || !d_final_T || !d_n_contrib || !d_dL_drgb || !d_grad2d || !proj->xy ||
+      !proj->conic_opacity || !proj->rgb || !proj->prim_id || !proj->clamp_flags || !proj->num_rows)
+    return ODIN_ERR_NULL;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int TX = (cam->width + 15) / 16, TY = (cam->height + 15) / 16;
+  const uint32_t zgrid = (uint32_t)ctx->sm_count * 8;
+  zero_rows_kernel<<<zgrid, 256, 0, st>>>(d_grad2d, proj->num_rows, proj->capacity);
+  render_bwd_blend_kernel<<<TX * TY, BB, 0, st>>>(
+      reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
+      reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
+      ctx->cfg.alpha_min, ctx->cfg.alpha_max, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d);
+  const CamParams cp = odin_cam_params(cam, ctx->cfg);
+  const uint32_t blocks_cap = (proj->capacity + 127) / 128;
+  const uint32_t pgrid = blocks_cap < (uint32_t)ctx->sm_count * 16 ? blocks_cap : (uint32_t)ctx->sm_count * 16;
+#define LAUNCH(D)                                                                                                       \
+  render_bwd_project_kernel<D><<<pgrid, 128, 0, st>>>(                                                                  \
+      scene->means, scene->log_scales, reinterpret_cast<const float4*>(scene->quats), scene->opacity_logit, scene->sh,  \
+      cp, ctx->cfg.dilation, proj->prim_id, proj->clamp_flags, proj->num_rows, proj->capacity, d_grad2d,                \
+      grad_rows->means, grad_rows->log_scales, reinterpret_cast<float4*>(grad_rows->quats), grad_rows->opacity_logit,    \
+      grad_rows->sh)
+  switch (scene->sh_degree) {
+    case 0: LAUNCH(0); break;
+    case 1: LAUNCH(1); break;
+    case 2: LAUNCH(2); break;
+    default: LAUNCH(3); break;
+  }
+#undef LAUNCH
+  return odin_launch_status();
+}

@@ -1,0 +1,154 @@
+// Touched-set bitmask + ascending index list (single pass, decoupled look-back) and pairwise intersection counts.
+#include "common.cuh"
+#include "layout.cuh"
+
+namespace {
+
+constexpr int TS_THREADS = 256;
+constexpr int TS_ITEMS = TOUCHED_TILE / TS_THREADS;  // 8 words of 32 primitives per warp
+
+// Each warp owns 256 consecutive primitives = 8 mask words; load j of lane l is primitive warp_base + 32 j + l, so one
+// ballot is one mask word and ranks inside the warp follow the primitive order.
+__global__ void __launch_bounds__(TS_THREADS)
+touched_set_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint32_t* __restrict__ mask,
+                   uint32_t* __restrict__ idx, uint32_t idx_capacity, uint32_t* __restrict__ count, uint32_t* ticket,
+                   uint64_t* state, int* status) {
+  __shared__ uint32_t s_tile;
+  __shared__ uint32_t s_warp[33];
+  __shared__ uint64_t s_base;
+  if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
+  __syncthreads();
+  const uint32_t tile = s_tile;
+  const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t warp_base = tile * TOUCHED_TILE + warp * (32 * TS_ITEMS);
+  uint32_t t[TS_ITEMS];
+#pragma unroll
+  for (int j = 0; j < TS_ITEMS; ++j) {
+    const uint32_t p = warp_base + 32 * j + lane;
+    t[j] = (p < n) ? tiles_touched[p] : 0u;
+  }
+  uint32_t ballots[TS_ITEMS];
+  uint32_t warp_count = 0;
+#pragma unroll
+  for (int j = 0; j < TS_ITEMS; ++j) {
+    ballots[j] = __ballot_sync(0xffffffffu, t[j] > 0);
+    warp_count += __popc(ballots[j]);
+  }
+  // mask words (lane j writes word j of the warp)
+  if (lane < TS_ITEMS) {
+    uint32_t w = 0;
+#pragma unroll
+    for (int j = 0; j < TS_ITEMS; ++j)
+      if (lane == (unsigned)j) w = ballots[j];
+    const uint32_t word = warp_base / 32 + lane;
+    if (word < (n + 31) / 32) mask[word] = w;
+  }
+  // exclusive offsets of the warps inside the block
+  uint32_t total;
+  const uint32_t scan = odin_block_exclusive_sum(lane == 0 ? warp_count : 0u, s_warp, &total);
+  const uint32_t warp_off = __shfl_sync(0xffffffffu, scan, 0);
+  if (threadIdx.x < 32) {
+    const uint64_t ex = odin_lookback_u64(state, tile, (uint64_t)total, status);
+    if (threadIdx.x == 0) s_base = ex;
+  }
+  __syncthreads();
+  const uint64_t base = s_base;
+  if (tile == (n + TOUCHED_TILE - 1) / TOUCHED_TILE - 1 && threadIdx.x == 0) {
+    const uint64_t v = base + total;
+    *count = (uint32_t)(v < idx_capacity ? v : idx_capacity);
+    if (v > idx_capacity) odin_set_error(status, ODIN_ERR_CAPACITY);
+  }
+  uint64_t pos = base + warp_off;
+#pragma unroll
+  for (int j = 0; j < TS_ITEMS; ++j) {
+    if (t[j] > 0) {
+      const uint64_t dst = pos + __popc(ballots[j] & ((1u << lane) - 1u));
+      if (dst < idx_capacity) idx[dst] = warp_base + 32 * j + lane;
+    }
+    pos += __popc(ballots[j]);
+  }
+}
+
+constexpr int CC_THREADS = 256;
+
+// One block column per pair (blockIdx.y); blocks of a column stride over the mask words four at a time.
+__global__ void __launch_bounds__(CC_THREADS)
+conflict_count_kernel(const uint32_t* __restrict__ masks, uint32_t stride_words, uint32_t words,
+                      const uint32_t* __restrict__ pairs, uint32_t n_masks, unsigned long long* __restrict__ counts,
+                      int* status) {
+  const uint32_t pair = blockIdx.y;
+  const uint32_t va = pairs[2 * pair], vb = pairs[2 * pair + 1];
+  if (va >= n_masks || vb >= n_masks) {  // uniform over the block: a pair naming a missing view counts 0
+    if (threadIdx.x == 0) odin_set_error(status, ODIN_ERR_INVALID_ARG);
+    return;
+  }
+  const uint32_t* a = masks + (size_t)va * stride_words;
+  const uint32_t* b = masks + (size_t)vb * stride_words;
+  uint32_t c = 0;
+  const uint32_t vec = words / 4;
+  const uint4* a4 = reinterpret_cast<const uint4*>(a);
+  const uint4* b4 = reinterpret_cast<const uint4*>(b);
+  for (uint32_t i = blockIdx.x * CC_THREADS + threadIdx.x; i < vec; i += gridDim.x * CC_THREADS) {
+    const uint4 x = a4[i], y = b4[i];
+    c += __popc(x.x & y.x) + __popc(x.y & y.y) + __popc(x.z & y.z) + __popc(x.w & y.w);
+  }
+  if (blockIdx.x == 0)
+    for (uint32_t i = vec * 4 + threadIdx.x; i < words; i += CC_THREADS) c += __popc(a[i] & b[i]);
+  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+  __shared__ uint32_t s[CC_THREADS / 32];
+  if ((threadIdx.x & 31) == 0) s[threadIdx.x >> 5] = c;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t tot = 0;
+    for (int i = 0; i < CC_THREADS / 32; ++i) tot += s[i];
+    if (tot) atomicAdd(&counts[pair], (unsigned long long)tot);
+  }
+}
+
+}  // namespace
+
+extern "C" int odin_touched_set(odin_ctx* ctx, const uint32_t* d_tiles_touched, uint32_t n, uint32_t* d_mask,
+                                uint32_t* d_idx, uint32_t idx_capacity, uint32_t* d_count, void* ws, size_t ws_bytes,
+                                void* stream) {
+  if (!ctx || !d_count) return ODIN_ERR_NULL;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (n >= (1u << 28)) return ODIN_ERR_INVALID_ARG;
+  if (n == 0) {
+    ODIN_CUDA(cudaMemsetAsync(d_count, 0, 4, st));
+    return ODIN_OK;
+  }
+  if (!d_tiles_touched || !d_mask || (idx_capacity > 0 && !d_idx)) return ODIN_ERR_NULL;
+  const size_t need = touched_ws_bytes(n);
+  if (!ws || !odin_aligned(ws, 256) || ws_bytes < need) return ODIN_ERR_WORKSPACE;
+  ODIN_CUDA(cudaMemsetAsync(ws, 0, need, st));
+  uint32_t* ticket = reinterpret_cast<uint32_t*>(ws);
+  uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + 256);
+  const uint32_t grid = (n + TOUCHED_TILE - 1) / TOUCHED_TILE;
+  touched_set_kernel<<<grid, TS_THREADS, 0, st>>>(d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket, state,
+                                                  ctx->d_status);
+  return odin_launch_status();
+}
+
+extern "C" int odin_conflict_count(odin_ctx* ctx, const uint32_t* d_masks, uint32_t n_masks, uint32_t mask_stride_words,
+                                   uint32_t n_prims, const uint32_t* d_pairs, uint32_t n_pairs, uint64_t* d_counts,
+                                   void* stream) {
+  if (!ctx) return ODIN_ERR_NULL;
+  if (n_pairs == 0) return ODIN_OK;
+  if (!d_pairs || !d_counts) return ODIN_ERR_NULL;
+  if (n_pairs > 65535) return ODIN_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  ODIN_CUDA(cudaMemsetAsync(d_counts, 0, (size_t)n_pairs * 8, st));
+  const uint32_t words = (n_prims + 31) / 32;
+  if (words == 0) return ODIN_OK;
+  if (!d_masks) return ODIN_ERR_NULL;
+  if (n_masks == 0 || mask_stride_words < words || (mask_stride_words % 4) != 0 || !odin_aligned(d_masks, 16))
+    return ODIN_ERR_INVALID_ARG;
+  uint32_t gx = (words / 4 + CC_THREADS - 1) / CC_THREADS;
+  const uint32_t cap = (uint32_t)(ctx->sm_count * 8 + n_pairs - 1) / n_pairs;
+  if (gx > cap) gx = cap;
+  if (gx == 0) gx = 1;
+  conflict_count_kernel<<<dim3(gx, n_pairs), CC_THREADS, 0, st>>>(d_masks, mask_stride_words, words, d_pairs, n_masks,
+                                                                 reinterpret_cast<unsigned long long*>(d_counts),
+                                                                 ctx->d_status);
+  return odin_launch_status();
+}

@@ -1,0 +1,179 @@
+"""Device buffers (through PyTorch) and the call sequence of one training view.
+
+This file only allocates memory and marshals arguments; all arithmetic happens inside libodin.so.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+def _dev(a: np.ndarray, device) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+
+
+class DeviceScene:
+    """Five aligned attribute tensors on the device + the odin_scene struct that points at them."""
+
+    def __init__(self, n: int, sh_degree: int, device, tensors=None):
+        k = (sh_degree + 1) ** 2
+        self.n, self.sh_degree, self.k = int(n), int(sh_degree), k
+        if tensors is None:
+            z = lambda *s: torch.zeros(*s, dtype=torch.float32, device=device)  # noqa: E731
+            tensors = (z(max(n, 1), 3), z(max(n, 1), 3), z(max(n, 1), 4), z(max(n, 1)), z(max(n, 1), k, 3))
+        self.means, self.log_scales, self.quats, self.opacity_logit, self.sh = tensors
+        self.struct = B.make_scene(n, sh_degree, self.means, self.log_scales, self.quats, self.opacity_logit, self.sh)
+
+    @classmethod
+    def from_host(cls, scene, device) -> "DeviceScene":
+        t = tuple(_dev(np.asarray(a, dtype=np.float32), device)
+                  for a in (scene.means, scene.log_scales, scene.quats, scene.opacity_logit, scene.sh))
+        return cls(scene.means.shape[0], scene.sh_degree, device, t)
+
+    def tensors(self):
+        return (self.means, self.log_scales, self.quats, self.opacity_logit, self.sh)
+
+    def to_host(self):
+        return tuple(t[: self.n].cpu().numpy() for t in self.tensors())
+
+    def rows_as_matrix(self, v: int) -> np.ndarray:
+        """First v rows as one [v, 11+3K] matrix in the order mean, log scale, quaternion, opacity, SH."""
+        m, ls, q, o, sh = (t[:v].cpu().numpy() for t in self.tensors())
+        return np.concatenate([m, ls, q, o[:, None], sh.reshape(v, -1)], axis=1)
+
+
+class ProjectedBuffers:
+    def __init__(self, n: int, capacity: int, device):
+        cap = max(int(capacity), 1)
+        self.n, self.capacity = int(n), int(capacity)
+        i32, u8, f32 = torch.int32, torch.uint8, torch.float32
+        z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=device)  # noqa: E731
+        self.tiles_touched = z(max(n, 1), i32)
+        self.prim_id = z(cap, i32)
+        self.xy = z((cap, 2), f32)
+        self.depth = z(cap, f32)
+        self.conic_opacity = z((cap, 4), f32)
+        self.rgb = z((cap, 3), f32)
+        self.radius = z(cap, i32)
+        self.rect = z((cap, 4), torch.int16)
+        self.tile_offset = z(cap, i32)
+        self.clamp_flags = z(cap, u8)
+        self.num_rows = z(1, i32)
+        self.num_instances = z(1, torch.int64)
+        self.struct = B.odin_projected(
+            self.capacity, *(t.data_ptr() for t in (self.tiles_touched, self.prim_id, self.xy, self.depth,
+                                                    self.conic_opacity, self.rgb, self.radius, self.rect, self.tile_offset,
+                                                    self.clamp_flags, self.num_rows, self.num_instances)))
+
+    def load_rows(self, **arrays) -> None:
+        """Overwrite compact arrays from host data (used by stage-isolated tests)."""
+        for name, a in arrays.items():
+            t = getattr(self, name)
+            src = torch.from_numpy(np.ascontiguousarray(a))
+            if src.dtype == torch.uint32:
+                src = src.view(torch.int32)
+            if src.dtype == torch.uint16:
+                src = src.view(torch.int16)
+            if src.dtype == torch.uint64:
+                src = src.view(torch.int64)
+            t.view(-1)[: src.numel()].copy_(src.view(-1).to(t.device))
+
+
+class ViewTrainer:
+    """Owns every device buffer of the view step and enqueues the seven calls (plus the loss) on one stream."""
+
+    def __init__(self, scene, width: int, height: int, row_capacity: int, instance_capacity: int, mask_slots: int = 1,
+                 device: int = 0):
+        self.device = torch.device("cuda", device)
+        torch.cuda.set_device(self.device)
+        self.ctx = B.odin_create(device)
+        self.n, self.sh_degree = scene.means.shape[0], scene.sh_degree
+        self.width, self.height = int(width), int(height)
+        self.tx, self.ty = (width + 15) // 16, (height + 15) // 16
+        self.row_capacity, self.instance_capacity = int(row_capacity), int(instance_capacity)
+        dev = self.device
+        self.params = DeviceScene.from_host(scene, dev)
+        self.m = DeviceScene(self.n, self.sh_degree, dev)
+        self.v = DeviceScene(self.n, self.sh_degree, dev)
+        self.grads = DeviceScene(self.row_capacity, self.sh_degree, dev)
+        self.proj = ProjectedBuffers(self.n, self.row_capacity, dev)
+        z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=dev)  # noqa: E731
+        self.keys = z(max(self.instance_capacity, 1), torch.int64)
+        self.vals = z(max(self.instance_capacity, 1), torch.int32)
+        self.ranges = z((self.tx * self.ty, 2), torch.int32)
+        self.out = z((3, height, width), torch.float32)
+        self.final_T = z((height, width), torch.float32)
+        self.n_contrib = z((height, width), torch.int32)
+        self.target = z((3, height, width), torch.float32)
+        self.dL = z((3, height, width), torch.float32)
+        self.loss = z(1, torch.float32)
+        self.grad2d = z((max(self.row_capacity, 1), 9), torch.float32)
+        self.mask_words = (self.n + 31) // 32
+        self.mask_stride = (self.mask_words + 3) // 4 * 4
+        self.mask_slots = int(mask_slots)
+        self.masks = z((self.mask_slots, max(self.mask_stride, 4)), torch.int32)
+        self.idx = z(max(self.row_capacity, 1), torch.int32)
+        self.count = z(1, torch.int32)
+        ws_bytes = B.odin_workspace_bytes(self.ctx, self.n, self.instance_capacity)
+        self.ws = z(ws_bytes, torch.uint8)
+        self.kernel_launches_per_step = 0
+
+    def close(self) -> None:
+        if self.ctx is not None:
+            B.odin_destroy(self.ctx)
+            self.ctx = None
+
+    # -------------------------------------------------------------------------------------------- stages
+    def project(self, cam: B.odin_camera, stream=None) -> None:
+        B.odin_project(self.ctx, self.params.struct, cam, self.proj.struct, self.ws, stream)
+
+    def touched_set(self, slot: int = 0, stream=None) -> None:
+        B.odin_touched_set(self.ctx, self.proj.tiles_touched, self.n, self.masks[slot], self.idx, self.row_capacity,
+                           self.count, self.ws, stream)
+
+    def bin_sort(self, stream=None) -> None:
+        B.odin_bin_sort(self.ctx, self.proj.struct, self.width, self.height, self.keys, self.vals, self.instance_capacity,
+                        self.ranges, self.ws, stream)
+
+    def render_fwd(self, cam: B.odin_camera, stream=None) -> None:
+        B.odin_render_fwd(self.ctx, self.proj.struct, self.vals, self.ranges, cam, self.out, self.final_T, self.n_contrib,
+                          stream)
+
+    def l1_loss(self, stream=None) -> None:
+        B.odin_l1_loss(self.ctx, self.out, self.target, self.width, self.height, self.loss, self.dL, stream)
+
+    def render_bwd(self, cam: B.odin_camera, stream=None) -> None:
+        B.odin_render_bwd(self.ctx, self.params.struct, cam, self.proj.struct, self.vals, self.ranges, self.final_T,
+                          self.n_contrib, self.dL, self.grad2d, self.grads.struct, stream)
+
+    def sparse_adam(self, lr, beta1, beta2, eps, step: int, stream=None) -> None:
+        B.odin_sparse_adam(self.ctx, self.params.struct, self.m.struct, self.v.struct, self.grads.struct, self.idx,
+                           self.count, lr, beta1, beta2, eps, step, stream)
+
+    def conflict_count(self, d_pairs, n_pairs: int, d_counts, stream=None) -> None:
+        B.odin_conflict_count(self.ctx, self.masks, self.mask_slots, self.masks.shape[1], self.n, d_pairs, n_pairs,
+                              d_counts, stream)
+
+    # -------------------------------------------------------------------------------------------- whole view
+    def view_step(self, cam: B.odin_camera, step: int, lr, beta1: float, beta2: float, eps: float, slot: int = 0,
+                  d_pairs=None, n_pairs: int = 0, d_counts=None, update: bool = True, stream=None) -> None:
+        """project -> touched set -> bin/sort -> composite -> L1 loss -> backward -> sparse Adam -> conflict counts.
+        The target image must already be in self.target.  Nothing here synchronises the host."""
+        self.project(cam, stream)
+        self.touched_set(slot, stream)
+        self.bin_sort(stream)
+        self.render_fwd(cam, stream)
+        self.l1_loss(stream)
+        self.render_bwd(cam, stream)
+        if update:
+            self.sparse_adam(lr, beta1, beta2, eps, step, stream)
+        if n_pairs:
+            self.conflict_count(d_pairs, n_pairs, d_counts, stream)
+
+    def poll(self, stream=None) -> int:
+        return B.odin_poll(self.ctx, stream)

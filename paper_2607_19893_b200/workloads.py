@@ -164,14 +164,15 @@ def _attributes(rng, n, sh_degree, ls_mu, ls_sigma):
     q /= np.linalg.norm(q, axis=1, keepdims=True)
     logits = rng.standard_normal(n, dtype=np.float32)
     sh = np.empty((n, k, 3), dtype=np.float32)
-    rgb = rng.random((n, 3), dtype=np.float32)
-    sh[:, 0, :] = (rgb - 0.5) / np.float32(SH_DC)
     if k > 1:
-        # fill in slabs to bound peak memory on the 20M preset
+        # drawn in place, slab by slab, to bound peak memory and time on the 20M preset
         step = 1 << 20
         for s in range(0, n, step):
-            e = min(n, s + step)
-            sh[s:e, 1:, :] = 0.1 * rng.standard_normal((e - s, k - 1, 3), dtype=np.float32)
+            slab = sh[s:min(n, s + step)]
+            rng.standard_normal(out=slab, dtype=np.float32)
+            slab *= np.float32(0.1)
+    rgb = rng.random((n, 3), dtype=np.float32)
+    sh[:, 0, :] = (rgb - 0.5) / np.float32(SH_DC)
     return log_scales, q.astype(np.float32), logits, sh
 
 

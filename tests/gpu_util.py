@@ -1,0 +1,53 @@
+"""Helpers shared by the GPU parity tests: build a trainer, feed oracle stage outputs to the device, read back."""
+import numpy as np
+import torch
+
+from paper_2607_19893_b200 import binding as B
+from paper_2607_19893_b200.engine import ViewTrainer
+
+
+def trainer_for(scene, cam, row_capacity=None, instance_capacity=None, mask_slots=1):
+    n = scene.means.shape[0]
+    return ViewTrainer(scene, cam.width, cam.height, row_capacity if row_capacity is not None else n,
+                       instance_capacity if instance_capacity is not None else max(64 * n, 1 << 16), mask_slots)
+
+
+def compact_from_oracle(proj, idx):
+    """Oracle's dense projection -> the compact arrays of odin_projected (row r <-> primitive idx[r])."""
+    idx = idx.astype(np.int64)
+    tt = proj.tiles_touched[idx].astype(np.uint64)
+    off = np.concatenate([[0], np.cumsum(tt)[:-1]]).astype(np.uint32) if len(idx) else np.zeros(0, np.uint32)
+    return dict(
+        prim_id=idx.astype(np.uint32), xy=proj.xy[idx].astype(np.float32), depth=proj.depth[idx].astype(np.float32),
+        conic_opacity=proj.conic_o[idx].astype(np.float32), rgb=proj.rgb[idx].astype(np.float32),
+        radius=proj.radius[idx].astype(np.int32), rect=proj.rect[idx].astype(np.uint16), tile_offset=off,
+        clamp_flags=proj.clamp_flags[idx].astype(np.uint8),
+    )
+
+
+def load_oracle_projection(tr, proj, idx):
+    rows = compact_from_oracle(proj, idx)
+    tr.proj.load_rows(**rows)
+    tr.proj.tiles_touched[: len(proj.tiles_touched)].copy_(
+        torch.from_numpy(proj.tiles_touched.view(np.int32)).to(tr.device))
+    tr.proj.num_rows.fill_(len(idx))
+    tr.proj.num_instances.fill_(int(proj.tiles_touched.astype(np.int64).sum()))
+    return rows
+
+
+def u32(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def u64(t):
+    return t.cpu().numpy().view(np.uint64)
+
+
+def rows_of(inv_idx, vals):
+    """Map oracle values (primitive ids) to compact row ids."""
+    return inv_idx[vals.astype(np.int64)]
+
+
+def poll_ok(tr):
+    st = tr.poll()
+    assert st == B.ODIN_OK, B.status_string(st)

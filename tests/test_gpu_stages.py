@@ -1,0 +1,409 @@
+"""Stage-isolated parity of the CUDA library against the CPU oracle (needs a GPU).
+
+Every stage is fed the ORACLE's outputs of the previous stages, so integer stages must agree bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_19893_b200 import binding as B
+from paper_2607_19893_b200 import workloads as wl
+from paper_2607_19893_b200.engine import DeviceScene
+
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+PIX_TOL = 1e-4          # absolute, rendered pixels
+GRAD_RTOL, GRAD_ATOL = 1e-3, 1e-5  # gradients and updated parameters
+
+
+# ------------------------------------------------------------------------------------------------ touched set
+@pytest.mark.parametrize("n", [1, 31, 32, 33, 2047, 2048, 2049, 100_003, 3_000_001])
+def test_touched_set_bit_exact(oracle32, n):
+    rng = np.random.default_rng(n)
+    tt = ((rng.random(n) < 0.3) * rng.integers(1, 50, n)).astype(np.uint32)
+    if n > 5000:
+        tt[1000:4000] = 0          # a long empty run and a long full run
+        tt[4000:9000] = 3
+    mask_o, idx_o = oracle32.touched_set(tt)
+    dev = torch.device("cuda", 0)
+    ctx = B.odin_create(0)
+    d_tt = torch.from_numpy(tt.view(np.int32)).to(dev)
+    words = (n + 31) // 32
+    d_mask = torch.full((words,), -1, dtype=torch.int32, device=dev)
+    d_idx = torch.full((n,), -1, dtype=torch.int32, device=dev)
+    d_count = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = torch.zeros(B.odin_workspace_bytes(ctx, n, 0), dtype=torch.uint8, device=dev)
+    for _ in range(2):  # twice: the workspace is reused
+        B.odin_touched_set(ctx, d_tt, n, d_mask, d_idx, n, d_count, ws)
+        assert B.odin_poll(ctx) == B.ODIN_OK
+        v = int(d_count.item())
+        assert v == len(idx_o)
+        assert np.array_equal(G.u32(d_mask), mask_o)
+        assert np.array_equal(G.u32(d_idx[:v]), idx_o)
+    # capacity smaller than V: truncated list, deferred error, nothing written past the capacity
+    if len(idx_o) > 4:
+        cap = len(idx_o) // 2
+        d_idx.fill_(-1)
+        B.odin_touched_set(ctx, d_tt, n, d_mask, d_idx, cap, d_count, ws)
+        assert B.odin_poll(ctx) == B.ODIN_ERR_CAPACITY
+        assert int(d_count.item()) == cap
+        assert np.array_equal(G.u32(d_idx[:cap]), idx_o[:cap]) and bool((d_idx[cap:] == -1).all())
+        assert B.odin_poll(ctx) == B.ODIN_OK  # cleared
+    B.odin_destroy(ctx)
+
+
+def test_touched_set_empty(oracle32):
+    dev = torch.device("cuda", 0)
+    ctx = B.odin_create(0)
+    d_count = torch.full((1,), 7, dtype=torch.int32, device=dev)
+    B.odin_touched_set(ctx, None, 0, None, None, 0, d_count, None)
+    assert B.odin_poll(ctx) == B.ODIN_OK and int(d_count.item()) == 0
+    B.odin_destroy(ctx)
+
+
+# ------------------------------------------------------------------------------------------------ conflict count
+@pytest.mark.parametrize("n", [1, 127, 128, 129, 100_000, 5_000_001])
+def test_conflict_count_bit_exact(oracle32, n):
+    rng = np.random.default_rng(n + 1)
+    views = 6
+    dens = [0.0, 0.02, 0.3, 0.5, 0.97, 1.0]
+    sets = [np.nonzero(rng.random(n) < d)[0].astype(np.uint32) for d in dens]
+    words = (n + 31) // 32
+    stride = (words + 3) // 4 * 4
+    masks = np.zeros((views, stride), np.uint32)
+    for i, s in enumerate(sets):
+        np.bitwise_or.at(masks[i], s >> 5, np.uint32(1) << (s & 31))
+    pairs = np.array([(a, b) for a in range(views) for b in range(views)], np.uint32)
+    want = np.array([oracle32.conflict_count(sets[a], sets[b]) for a, b in pairs], np.uint64)
+    dev = torch.device("cuda", 0)
+    ctx = B.odin_create(0)
+    d_masks = torch.from_numpy(masks.view(np.int32)).to(dev)
+    d_pairs = torch.from_numpy(pairs.view(np.int32)).to(dev)
+    d_counts = torch.full((len(pairs),), -1, dtype=torch.int64, device=dev)
+    B.odin_conflict_count(ctx, d_masks, views, stride, n, d_pairs, len(pairs), d_counts)
+    assert B.odin_poll(ctx) == B.ODIN_OK
+    assert np.array_equal(G.u64(d_counts), want)
+    # a pair naming a missing view: deferred error, count 0
+    bad = torch.tensor([[0, views]], dtype=torch.int32, device=dev)
+    B.odin_conflict_count(ctx, d_masks, views, stride, n, bad, 1, d_counts)
+    assert B.odin_poll(ctx) == B.ODIN_ERR_INVALID_ARG and int(d_counts[0].item()) == 0
+    B.odin_destroy(ctx)
+
+
+# ------------------------------------------------------------------------------------------------ Adam
+@pytest.mark.parametrize("sh_degree,n,v", [(3, 5000, 1700), (0, 1024, 1024), (1, 999, 10), (2, 4001, 4001), (3, 300_000, 90_000)])
+def test_sparse_adam_stage(oracle32, sh_degree, n, v):
+    rng = np.random.default_rng(v)
+    k = (sh_degree + 1) ** 2
+    f = 11 + 3 * k
+
+    def rand_scene(scale=1.0, positive=False):
+        a = [rng.standard_normal(s).astype(np.float32) * np.float32(scale) for s in ((n, 3), (n, 3), (n, 4), (n,), (n, k, 3))]
+        if positive:
+            a = [np.abs(x) for x in a]
+        return wl.Scene(sh_degree, *a)
+
+    p, m, vv = rand_scene(), rand_scene(0.1), rand_scene(0.01, True)
+    idx = np.sort(rng.choice(n, v, replace=False)).astype(np.uint32)
+    rows = rng.standard_normal((v, f)).astype(np.float32)
+    rows[rng.random((v, f)) < 0.1] = 0
+    lr = np.array([1e-3, 2e-3, 5e-4, 1e-2, 3e-3, 1e-4], np.float32)
+    dev = torch.device("cuda", 0)
+    ctx = B.odin_create(0)
+    dp, dm, dv = (DeviceScene.from_host(s, dev) for s in (p, m, vv))
+    g = wl.Scene(sh_degree, rows[:, 0:3], rows[:, 3:6], rows[:, 6:10], rows[:, 10], rows[:, 11:].reshape(v, k, 3))
+    dg = DeviceScene.from_host(g, dev)
+    d_idx = torch.from_numpy(idx.view(np.int32)).to(dev)
+    d_count = torch.tensor([v], dtype=torch.int32, device=dev)
+    before = [t.clone() for s in (dp, dm, dv) for t in s.tensors()]
+    for step in (1, 2, 7):
+        oracle32.sparse_adam(p, m, vv, rows, idx, lr, 0.9, 0.999, 1e-15, step)
+        B.odin_sparse_adam(ctx, dp.struct, dm.struct, dv.struct, dg.struct, d_idx, d_count, lr, 0.9, 0.999, 1e-15, step)
+    assert B.odin_poll(ctx) == B.ODIN_OK
+    after = [t for s in (dp, dm, dv) for t in s.tensors()]
+    host = [a for s in (p, m, vv) for a in (s.means, s.log_scales, s.quats, s.opacity_logit, s.sh)]
+    un = np.setdiff1d(np.arange(n), idx)
+    for b, a, h in zip(before, after, host):
+        a = a.cpu().numpy()
+        assert np.allclose(a, h, rtol=2e-5, atol=1e-7)
+        # untouched rows: bitwise identical
+        assert np.array_equal(b.cpu().numpy()[un].view(np.uint32), a[un].view(np.uint32))
+    # count = 0 on the device: nothing moves
+    d_count.zero_()
+    snap = [t.clone() for t in after]
+    B.odin_sparse_adam(ctx, dp.struct, dm.struct, dv.struct, dg.struct, d_idx, d_count, lr, 0.9, 0.999, 1e-15, 8)
+    assert B.odin_poll(ctx) == B.ODIN_OK
+    for s, a in zip(snap, after):
+        assert torch.equal(s, a)
+    B.odin_destroy(ctx)
+
+
+# ------------------------------------------------------------------------------------------------ projection
+def check_projection(oracle32, scene, cam, row_capacity=None):
+    tr = G.trainer_for(scene, cam, row_capacity=row_capacity)
+    ccam = B.make_camera(cam)
+    po = oracle32.project(scene, cam)
+    for _ in range(2):
+        tr.project(ccam)
+        G.poll_ok(tr)
+    tt = G.u32(tr.proj.tiles_touched)[: scene.n]
+    safe = po.margin > 1e-4
+    assert safe.mean() > 0.98
+    assert np.array_equal(tt[safe], po.tiles_touched[safe])
+    v = int(tr.proj.num_rows.item())
+    prim = G.u32(tr.proj.prim_id)[:v]
+    assert np.array_equal(prim, np.nonzero(tt)[0])  # rows ascend with the primitive id and match tiles_touched
+    assert int(tr.proj.num_instances.item()) == int(tt.astype(np.int64).sum())
+    off = G.u32(tr.proj.tile_offset)[:v]
+    assert np.array_equal(off, np.concatenate([[0], np.cumsum(tt[prim].astype(np.int64))[:-1]]).astype(np.uint32)[:v])
+    ok = safe[prim] & (po.tiles_touched[prim] > 0)
+    pp = prim[ok]
+    rect = tr.proj.rect.cpu().numpy().view(np.uint16)[:v][ok]
+    assert np.array_equal(rect.astype(np.int32), po.rect[pp])
+    assert np.array_equal(tr.proj.radius.cpu().numpy()[:v][ok], po.radius[pp])
+    assert np.array_equal(tr.proj.clamp_flags.cpu().numpy()[:v][ok], po.clamp_flags[pp])
+    assert np.allclose(tr.proj.xy.cpu().numpy()[:v][ok], po.xy[pp], rtol=1e-5, atol=2e-3)
+    assert np.allclose(tr.proj.depth.cpu().numpy()[:v][ok], po.depth[pp], rtol=1e-6)
+    assert np.allclose(tr.proj.conic_opacity.cpu().numpy()[:v][ok], po.conic_o[pp], rtol=5e-4, atol=1e-7)
+    assert np.allclose(tr.proj.rgb.cpu().numpy()[:v][ok], po.rgb[pp], rtol=1e-5, atol=2e-6)
+    tr.close()
+    return v
+
+
+def test_project_cfg1(oracle32):
+    w = wl.make_workload(1)
+    assert check_projection(oracle32, w.scene, w.cameras[0]) == 1024
+
+
+@pytest.mark.parametrize("view", [0, 5])
+def test_project_cfg2(oracle32, view):
+    w = wl.make_workload(2)
+    check_projection(oracle32, w.scene, w.cameras[view])
+
+
+def test_project_unbounded_ragged(oracle32):
+    w = wl.make_workload(3, n=300_007, resolution=(800, 533))
+    check_projection(oracle32, w.scene, w.cameras[3])
+
+
+def test_project_city_low_visibility(oracle32):
+    w = wl.make_workload(5, n=400_000, n_cameras=4)
+    for c in (0, 1):
+        v = check_projection(oracle32, w.scene, w.cameras[c])
+        assert 0 < v < 0.1 * w.scene.n
+
+
+@pytest.mark.parametrize("deg", [1, 2])
+def test_project_other_sh_degrees(oracle32, deg):
+    w = wl.make_workload(2, n=20_000)
+    s = w.scene
+    k = (deg + 1) ** 2
+    s2 = wl.Scene(deg, s.means, s.log_scales, s.quats, s.opacity_logit, np.ascontiguousarray(s.sh[:, :k]))
+    check_projection(oracle32, s2, w.cameras[1])
+
+
+def test_project_row_capacity_overflow(oracle32):
+    w = wl.make_workload(1)
+    tr = G.trainer_for(w.scene, w.cameras[0], row_capacity=100)
+    tr.proj.prim_id.fill_(-1)
+    tr.project(B.make_camera(w.cameras[0]))
+    assert tr.poll() == B.ODIN_ERR_CAPACITY
+    assert int(tr.proj.num_rows.item()) == 100
+    assert np.array_equal(G.u32(tr.proj.prim_id), np.arange(100))  # the first 100 rows, nothing beyond
+    tr.close()
+
+
+# ------------------------------------------------------------------------------------------------ bin / sort
+def check_bin_sort(oracle32, scene, cam, instance_capacity=None):
+    po = oracle32.project(scene, cam)
+    mask, idx = oracle32.touched_set(po.tiles_touched)
+    keys_o, vals_o, ranges_o = oracle32.bin_sort(po, cam)
+    m = len(keys_o)
+    tr = G.trainer_for(scene, cam, row_capacity=max(len(idx), 1),
+                       instance_capacity=instance_capacity if instance_capacity is not None else m + 17)
+    G.load_oracle_projection(tr, po, idx)
+    inv = np.full(scene.n, -1, np.int64)
+    inv[idx] = np.arange(len(idx))
+    for _ in range(2):
+        tr.keys.fill_(-1)
+        tr.bin_sort()
+        G.poll_ok(tr)
+        assert np.array_equal(G.u64(tr.keys)[:m], keys_o)
+        assert np.array_equal(G.u32(tr.vals)[:m], G.rows_of(inv, vals_o).astype(np.uint32))
+        rg = G.u32(tr.ranges)
+        assert np.array_equal(rg[:, 1] - rg[:, 0], ranges_o[:, 1] - ranges_o[:, 0])
+        ne = ranges_o[:, 1] > ranges_o[:, 0]
+        assert np.array_equal(rg[ne], ranges_o[ne])
+    tr.close()
+    return m
+
+
+def test_bin_sort_cfg1(oracle32):
+    w = wl.make_workload(1)
+    check_bin_sort(oracle32, w.scene, w.cameras[0])
+
+
+def test_bin_sort_cfg2(oracle32):
+    w = wl.make_workload(2)
+    m = check_bin_sort(oracle32, w.scene, w.cameras[2])
+    assert m > 3 * 4096  # several sort tiles and a ragged tail
+
+
+def test_bin_sort_many_tiles_six_passes(oracle32):
+    w = wl.make_workload(3, n=120_000)  # 6700 tiles -> 13 tile bits -> 6 digit passes, ~1.2M instances
+    m = check_bin_sort(oracle32, w.scene, w.cameras[7])
+    assert m > 500_000
+
+
+def test_bin_sort_equal_depth_ties(oracle32):
+    # many identical splats: identical keys, order decided by the row index alone
+    w = wl.make_workload(1)
+    s = w.scene
+    rep = lambda a: np.ascontiguousarray(np.repeat(a[:3], 3000, axis=0))  # noqa: E731
+    s2 = wl.Scene(0, rep(s.means), rep(s.log_scales), rep(s.quats), rep(s.opacity_logit), rep(s.sh))
+    check_bin_sort(oracle32, s2, w.cameras[0])
+
+
+def test_bin_sort_empty_view(oracle32):
+    w = wl.make_workload(1)
+    s = w.scene.copy()
+    s.means[:, 2] = -5.0  # everything behind the camera
+    check_bin_sort(oracle32, s, w.cameras[0])
+
+
+def test_bin_sort_instance_capacity_overflow(oracle32):
+    w = wl.make_workload(1)
+    cam = w.cameras[0]
+    po = oracle32.project(w.scene, cam)
+    mask, idx = oracle32.touched_set(po.tiles_touched)
+    tr = G.trainer_for(w.scene, cam, instance_capacity=1000)
+    G.load_oracle_projection(tr, po, idx)
+    tr.bin_sort()
+    assert tr.poll() == B.ODIN_ERR_CAPACITY
+    keys = G.u64(tr.keys)[:1000]
+    assert np.all(np.diff(keys.astype(np.int64)) >= 0)  # the first 1000 instances, sorted; nothing out of bounds
+    tr.close()
+
+
+# ------------------------------------------------------------------------------------------------ forward
+def oracle_view(oracle32, scene, cam):
+    f = oracle32.view_forward(scene, cam)
+    inv = np.full(scene.n, -1, np.int64)
+    inv[f["idx"]] = np.arange(len(f["idx"]))
+    return f, inv
+
+
+def load_sorted(tr, f, inv):
+    G.load_oracle_projection(tr, f["proj"], f["idx"])
+    m = len(f["vals"])
+    tr.vals[:m].copy_(torch.from_numpy(G.rows_of(inv, f["vals"]).astype(np.int32)).to(tr.device))
+    tr.ranges.copy_(torch.from_numpy(f["ranges"].view(np.int32)).to(tr.device))
+
+
+def check_forward(oracle32, scene, cam):
+    f, inv = oracle_view(oracle32, scene, cam)
+    tr = G.trainer_for(scene, cam, row_capacity=max(len(f["idx"]), 1), instance_capacity=len(f["vals"]) + 1)
+    load_sorted(tr, f, inv)
+    tr.render_fwd(B.make_camera(cam))
+    G.poll_ok(tr)
+    out = tr.out.cpu().numpy()
+    ft = tr.final_T.cpu().numpy()
+    nc = G.u32(tr.n_contrib)
+    robust = f["pix_margin"] > 1e-4
+    assert robust.mean() > 1 - 2e-3
+    assert np.abs(out - f["out"])[:, robust].max() < PIX_TOL
+    assert np.abs(ft - f["final_T"])[robust].max() < PIX_TOL
+    assert np.array_equal(nc[robust], f["n_contrib"][robust])
+    # fragile pixels (a decision within 1e-4 of its threshold) may flip one contribution: bounded by alpha * T <= 1/255
+    # for the skip test and by 1e-4 for termination; they still have to stay close
+    assert np.abs(out - f["out"]).max() < 5e-3
+    tr.close()
+    return f
+
+
+def test_render_fwd_cfg1(oracle32):
+    w = wl.make_workload(1)
+    check_forward(oracle32, w.scene, w.cameras[0])
+
+
+def test_render_fwd_cfg2(oracle32):
+    w = wl.make_workload(2)
+    cam = w.cameras[4]
+    cam.bg = np.array([0.2, 0.5, 0.9])
+    check_forward(oracle32, w.scene, cam)
+
+
+def test_render_fwd_ragged_image_long_lists(oracle32):
+    w = wl.make_workload(3, n=150_000, resolution=(410, 275))  # edge tiles, lists of several batches
+    f = check_forward(oracle32, w.scene, w.cameras[1])
+    assert (f["ranges"][:, 1] - f["ranges"][:, 0]).max() > 600
+
+
+# ------------------------------------------------------------------------------------------------ loss
+def test_l1_loss(oracle32):
+    rng = np.random.default_rng(0)
+    w_, h_ = 333, 77
+    out = rng.random((3, h_, w_), dtype=np.float32)
+    tgt = rng.random((3, h_, w_), dtype=np.float32)
+    tgt[0, :5] = out[0, :5]  # exact zeros
+    loss_o, g_o = oracle32.l1_loss(out, tgt)
+    dev = torch.device("cuda", 0)
+    ctx = B.odin_create(0)
+    d_out, d_tgt = torch.from_numpy(out).to(dev), torch.from_numpy(tgt).to(dev)
+    d_loss = torch.zeros(1, device=dev)
+    d_g = torch.zeros_like(d_out)
+    B.odin_l1_loss(ctx, d_out, d_tgt, w_, h_, d_loss, d_g)
+    assert B.odin_poll(ctx) == B.ODIN_OK
+    assert abs(float(d_loss.item()) - loss_o) < 1e-6 * max(1.0, loss_o)
+    assert np.array_equal(d_g.cpu().numpy(), g_o)
+    B.odin_destroy(ctx)
+
+
+# ------------------------------------------------------------------------------------------------ backward
+def check_backward(oracle32, scene, cam, seed=0):
+    f, inv = oracle_view(oracle32, scene, cam)
+    rng = np.random.default_rng(seed)
+    dl = (rng.uniform(-1, 1, f["out"].shape) / f["out"].size).astype(np.float32)
+    g2d_o = oracle32.render_bwd_blend(f["proj"], f["vals"], f["ranges"], cam, f["final_T"], f["n_contrib"], dl)
+    rows_o = oracle32.render_bwd_project(scene, cam, f["idx"], g2d_o, f["proj"].clamp_flags)
+    v = len(f["idx"])
+    tr = G.trainer_for(scene, cam, row_capacity=max(v, 1), instance_capacity=len(f["vals"]) + 1)
+    load_sorted(tr, f, inv)
+    tr.final_T.copy_(torch.from_numpy(f["final_T"]).to(tr.device))
+    tr.n_contrib.copy_(torch.from_numpy(f["n_contrib"].view(np.int32)).to(tr.device))
+    tr.dL.copy_(torch.from_numpy(dl).to(tr.device))
+    for _ in range(2):
+        tr.render_bwd(B.make_camera(cam))
+        G.poll_ok(tr)
+    g2d = tr.grad2d.cpu().numpy()[:v].astype(np.float64)
+    want2d = g2d_o[f["idx"]]
+    # per column scale: sums of many signed terms are compared relative to the column's typical size
+    for c in range(9):
+        scale = np.abs(want2d[:, c]).mean() + 1e-30
+        err = np.abs(g2d[:, c] - want2d[:, c])
+        assert np.all(err <= GRAD_RTOL * np.abs(want2d[:, c]) + GRAD_RTOL * scale + 1e-12), (c, err.max(), scale)
+    rows = tr.grads.rows_as_matrix(v).astype(np.float64)
+    scale = np.abs(rows_o).mean(axis=0) + 1e-30
+    err = np.abs(rows - rows_o)
+    assert np.all(err <= GRAD_RTOL * np.abs(rows_o) + GRAD_RTOL * scale[None, :] + 1e-12), err.max()
+    tr.close()
+
+
+def test_render_bwd_cfg1(oracle32):
+    w = wl.make_workload(1)
+    check_backward(oracle32, w.scene, w.cameras[0])
+
+
+def test_render_bwd_cfg2(oracle32):
+    w = wl.make_workload(2, n=30_000)
+    cam = w.cameras[6]
+    cam.bg = np.array([0.3, 0.1, 0.7])
+    check_backward(oracle32, w.scene, cam, seed=3)
+
+
+def test_render_bwd_ragged_image_other_degree(oracle32):
+    w = wl.make_workload(3, n=60_000, resolution=(410, 275))
+    s = w.scene
+    s2 = wl.Scene(1, s.means, s.log_scales, s.quats, s.opacity_logit, np.ascontiguousarray(s.sh[:, :4]))
+    check_backward(oracle32, s2, w.cameras[2], seed=5)
