@@ -1,0 +1,383 @@
+#!/usr/bin/env python
+"""Throughput of the per-view training step (project -> touched set -> bin/sort -> composite -> L1 loss -> backward ->
+sparse Adam -> conflict counts) on seeded synthetic scenes.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl reference]
+
+One JSON line on stdout (rank 0).  `value` = views/s with every input resident in HBM; `e2e` = the same step driven
+with HOST inputs (the view's target image copied from pinned memory, loss / V / conflict counts read back) inside the
+timed region.  `roofline` describes the kernel with the largest share of the step, timed with CUDA events on the launch
+stream inside the timed region; `step_hbm` gives the whole step's algorithmic bytes against the measured HBM peak.
+The path does not shard (one view step is one GPU's work): with --gpus N every rank runs an independent replica.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_19893_b200 import workloads as wl  # noqa: E402
+
+METRIC = "train views/s (fwd+bwd+sparse Adam) on 1 B200; % of HBM roofline"
+UNIT = "views/s"
+ROW_CAP_FRAC = {1: 1.0, 2: 1.0, 3: 0.45, 4: 0.25, 5: 0.08}
+INSTANCE_CAP = {1: 1 << 16, 2: 1 << 21, 3: 1 << 24, 4: 320_000_000, 5: 1 << 23}
+CONFLICT_WINDOW = 4  # each view is compared with the 4 views before it
+MASK_SLOTS = CONFLICT_WINDOW + 1
+
+# Blend kernels are bound by plain fp32 ALU work.  Peak = SMs x 128 fp32 lanes x 2 (fma) x max SM clock.
+ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+FLOPS_PER_PAIR = {"render_fwd": 25.0, "render_bwd_blend": 75.0}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    return 6650.0, "fallback (profiling recipe)"
+
+
+class ClockSampler:
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def mark(self):
+        """Wall-clock time stamp in nvidia-smi's own format base (local time)."""
+        return time.time()
+
+    def stop(self, t_begin=None, t_end=None):
+        """Median SM clock over the samples taken between the two marks (all samples if none fall inside)."""
+        import datetime
+
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        rows = []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(f[1]), float(f[2]), [n for n, v in zip(names, f[4:8]) if v.lower().startswith("active")]))
+            except ValueError:
+                continue
+        inside = [r for r in rows if t_begin is not None and t_begin - 0.05 <= r[0] <= t_end + 0.05]
+        out["window"] = "timed region" if inside else "whole run (no sample fell inside the timed region)"
+        sm, mx, reasons = [], [], set()
+        for _, a, b, rs in (inside or rows):
+            sm.append(a); mx.append(b); reasons.update(rs)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def conflict_pairs(step: int):
+    """View slots compared after step `step`: the current slot against the (up to) 4 previous ones."""
+    cur = step % MASK_SLOTS
+    return [(cur, (step - j) % MASK_SLOTS) for j in range(1, min(CONFLICT_WINDOW, step) + 1)]
+
+
+def algorithmic_bytes(n, f, v, m, m_proc, p, t, passes, n_pairs):
+    """Bytes one view has to move, per stage (fp32; F floats per primitive)."""
+    f4 = 4 * f
+    b = {
+        "project": 12 * n + (f4 - 12) * v + 4 * n + 61 * v,
+        "touched_set": 4 * n + n / 8 + 4 * v,
+        "emit_instances": 16 * v + 12 * m,
+        "onesweep_pass": passes * 24 * m,
+        "tile_ranges": 8 * m + 8 * t,
+        "render_fwd": 4 * m_proc + 36 * v + 20 * p,
+        "l1_loss": 36 * p,
+        "render_bwd_blend": 4 * m_proc + 36 * v + 20 * p + 72 * v,
+        "render_bwd_project": 36 * v + 5 * v + f4 * v + f4 * v,
+        "adam": 4 * v + 4 * f4 * v + 3 * f4 * v,
+        "conflict_count": n_pairs * 2 * n / 8,
+    }
+    b["total"] = float(sum(b.values()))
+    return b
+
+
+def run_reference(args, rank):
+    """The oracle as it stands, on the host cores, on the same workload (rank 0 only)."""
+    if rank != 0:
+        return
+    import oracle
+
+    o32 = oracle.get(np.float32)
+    w = wl.make_workload(args.config)
+    n = w.scene.n
+    steps, warm = args.steps, args.warmup
+    # size the per-step sample so that the whole run stays within ~150 s: a probe on 20k primitives gives the cost
+    sub = lambda k: wl.Scene(w.scene.sh_degree, *(np.ascontiguousarray(a[:k]) for a in (
+        w.scene.means, w.scene.log_scales, w.scene.quats, w.scene.opacity_logit, w.scene.sh)))  # noqa: E731
+    probe_n = min(n, 20_000)
+    ps = sub(probe_n)
+    t0 = time.perf_counter()
+    o32.view_step(ps, ps.zeros_like(), ps.zeros_like(), w.cameras[0], w.target(0), w.lr, w.beta1, w.beta2, w.eps, 1)
+    per_prim = (time.perf_counter() - t0) / probe_n
+    n_s = int(min(n, max(1000, 150.0 / max(steps + warm, 1) / per_prim)))
+    p = sub(n_s)
+    m, v = p.zeros_like(), p.zeros_like()
+    times = []
+    for s in range(warm + steps):
+        view = s % len(w.cameras)
+        tgt = w.target(view)
+        t0 = time.perf_counter()
+        o32.view_step(p, m, v, w.cameras[view], tgt, w.lr, w.beta1, w.beta2, w.eps, s + 1)
+        if s >= warm:
+            times.append(time.perf_counter() - t0)
+    t = float(np.sum(times))
+    value = steps / t * (n_s / n)
+    sample = f"oracle view step on the first {n_s} of {n} primitives per step; views/s scaled by {n_s}/{n}"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warm, "ms_per_step": 1e3 * t / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": {"workload": w.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": o32.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=96)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=3, help="workload preset 1..5 (default 3: 1M primitives, 1600x1066)")
+    ap.add_argument("--impl", default="odin", choices=["odin", "reference"])
+    ap.add_argument("--no-kernel-events", action="store_true", help="do not bracket kernels with CUDA events")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "odin" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_19893_b200 import binding as B
+    from paper_2607_19893_b200 import build as odin_build
+    from paper_2607_19893_b200.engine import ViewTrainer
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation")
+    if rank == 0:
+        odin_build.build()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+
+    w = wl.make_workload(args.config)
+    scene = w.scene
+    n, f = scene.n, scene.floats_per_primitive
+    cam0 = w.cameras[0]
+    W, H = cam0.width, cam0.height
+    row_cap = max(1, int(ROW_CAP_FRAC[args.config] * n))
+    tr = ViewTrainer(scene, W, H, row_cap, INSTANCE_CAP[args.config], mask_slots=MASK_SLOTS, device=local_rank)
+    n_views = min(len(w.cameras), args.steps + args.warmup)
+    # rank r starts its replica at view r so that replicas do not all render the same camera at the same time
+    view_of = lambda s: (s + rank) % n_views  # noqa: E731
+    cams = [B.make_camera(c) for c in w.cameras[:n_views]]
+    host_targets = [torch.from_numpy(w.target(i)).pin_memory() for i in range(n_views)]
+    bank = torch.stack([t.to(dev) for t in host_targets])
+    total_steps = args.warmup + args.steps
+    pair_lists = [conflict_pairs(s) for s in range(total_steps)]
+    d_pairs = [torch.tensor(pl if pl else [(0, 0)], dtype=torch.int32, device=dev) for pl in pair_lists]
+    d_counts = torch.zeros(max(CONFLICT_WINDOW, 1), dtype=torch.int64, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(s, target):
+        tr.target = target
+        tr.view_step(cams[view_of(s)], s + 1, w.lr, w.beta1, w.beta2, w.eps, slot=s % MASK_SLOTS, d_pairs=d_pairs[s],
+                     n_pairs=len(pair_lists[s]), d_counts=d_counts, stream=stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident run -----------------------------------------------------------------------------------
+    sampler = ClockSampler(local_rank) if rank == 0 else None  # started early: nvidia-smi takes a while to come up
+    for s in range(args.warmup):
+        step(s, bank[view_of(s)])
+    st = tr.poll()
+    if st != B.ODIN_OK:
+        raise SystemExit(f"warm-up failed: {B.status_string(st)}")
+    B.odin_profile_collect(tr.ctx, stream)  # reset launch counters
+    B.odin_profile_enable(tr.ctx, not args.no_kernel_events)
+    barrier()
+    t_begin = time.time()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for s in range(args.warmup, total_steps):
+        step(s, bank[view_of(s)])
+    e1.record(stream)
+    barrier()
+    t_end = time.time()
+    ms = e0.elapsed_time(e1)
+    prof = B.odin_profile_collect(tr.ctx, stream)
+    B.odin_profile_enable(tr.ctx, False)
+    st = tr.poll()
+    if st != B.ODIN_OK:
+        raise SystemExit(f"timed run failed: {B.status_string(st)}")
+    t_max = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_max, op=dist.ReduceOp.MAX)
+    ms = float(t_max.item())
+    value = world * args.steps / (ms * 1e-3)
+
+    # workload counters of the last view (device side), for the byte model
+    v_last = int(tr.count.item())
+    m_last = int(tr.proj.num_instances.item())
+    ncon = tr.n_contrib.view(torch.int32)
+    ty, tx = tr.ty, tr.tx
+    pad = torch.zeros((ty * 16, tx * 16), dtype=torch.int32, device=dev)
+    pad[:H, :W] = ncon
+    tile_max = pad.view(ty, 16, tx, 16).amax(dim=(1, 3)).to(torch.int64)
+    m_proc = int(tile_max.sum().item())           # list entries the backward pass walks
+    pairs_bwd = 256 * m_proc
+    passes = (32 + max(int(np.ceil(np.log2(max(tx * ty, 1)))), 0) + 7) // 8
+    n_pairs_last = len(pair_lists[-1])
+    bytes_model = algorithmic_bytes(n, f, v_last, m_last, m_proc, W * H, tx * ty, passes, n_pairs_last)
+
+    # ---- end-to-end run: host target in, loss / V / counts out, every step --------------------------------------
+    h_loss = torch.zeros(1, dtype=torch.float32).pin_memory()
+    h_count = torch.zeros(1, dtype=torch.int32).pin_memory()
+    h_counts = torch.zeros(max(CONFLICT_WINDOW, 1), dtype=torch.int64).pin_memory()
+    staging = torch.empty_like(bank[0])
+    barrier()
+    t0 = time.perf_counter()
+    for s in range(args.warmup, total_steps):
+        staging.copy_(host_targets[view_of(s)], non_blocking=True)
+        step(s, staging)
+        h_loss.copy_(tr.loss, non_blocking=True)
+        h_count.copy_(tr.count, non_blocking=True)
+        h_counts.copy_(d_counts, non_blocking=True)
+        torch.cuda.synchronize()
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    e2e_t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
+    e2e_value = world * args.steps / float(e2e_t.item())
+    st = tr.poll()
+    if st != B.ODIN_OK:
+        raise SystemExit(f"end-to-end run failed: {B.status_string(st)}")
+    h2d = int(staging.numel() * 4)
+    d2h = int(4 + 4 + 8 * max(CONFLICT_WINDOW, 1))
+
+    clocks = sampler.stop(t_begin, t_end) if sampler else None
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel ------------------------------------------------------------------------
+    peak_gbs, peak_src = measured_peaks()
+    launches = sum(c for _, c in prof.values())
+    total_kernel_ms = sum(t for t, _ in prof.values())
+    roofline, shares = None, {}
+    if total_kernel_ms > 0:
+        shares = {k: {"ms_per_step": t / args.steps, "launches_per_step": c / args.steps, "share": t / total_kernel_ms}
+                  for k, (t, c) in prof.items() if c}
+        top = max(shares, key=lambda k: shares[k]["share"])
+        t_launch = prof[top][0] / max(prof[top][1], 1) * 1e-3
+        if top in FLOPS_PER_PAIR:
+            flops = FLOPS_PER_PAIR[top] * pairs_bwd
+            ach = flops / t_launch / 1e12
+            roofline = {"kernel": top, "bound": "alu", "achieved": ach, "peak": ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
+                        "frac": ach / ALU_PEAK_TFLOPS, "traffic": None,
+                        "note": f"{FLOPS_PER_PAIR[top]:.0f} flop x {pairs_bwd} (pixel,row) pairs per launch; peak = "
+                                "148 SM x 128 lanes x 2 x 1.965 GHz"}
+        else:
+            key = "adam" if top.startswith("adam") else top
+            per_launch = bytes_model[key] / (passes if top == "onesweep_pass" else 1)
+            ach = per_launch / t_launch / 1e9
+            roofline = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": peak_gbs, "unit": "GB/s",
+                        "frac": ach / peak_gbs, "traffic": None, "peak_source": peak_src}
+    step_gbs = bytes_model["total"] / (ms * 1e-3 / args.steps) / 1e9
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": w.name, "primitives": n, "floats_per_primitive": f, "image": [W, H], "views": n_views,
+                   "visible_last_view": v_last, "instances_last_view": m_last, "traversed_last_view": m_proc,
+                   "conflict_window": CONFLICT_WINDOW, "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   "l2": "no flush: parameters + moments + instance buffers exceed the 126 MB L2 between uses"},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "step_hbm": {"algorithmic_bytes_per_view": bytes_model["total"], "achieved_gbs": step_gbs, "peak_gbs": peak_gbs,
+                     "frac_of_measured": step_gbs / peak_gbs, "frac_of_8tbs": step_gbs / 8000.0, "peak_source": peak_src},
+        "kernels": shares,
+    }
+
+    # ---- the oracle on the host cores, bounded sample -----------------------------------------------------------
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+
+        o32 = oracle.get(np.float32)
+        n_sample_views = 1 if n >= 1_000_000 else (2 if n >= 100_000 else 8)
+        p = scene.copy()
+        m_, v_ = p.zeros_like(), p.zeros_like()
+        t0 = time.perf_counter()
+        for s in range(n_sample_views):
+            o32.view_step(p, m_, v_, w.cameras[s % len(w.cameras)], w.target(s % len(w.cameras)), w.lr, w.beta1, w.beta2,
+                          w.eps, s + 1)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": n_sample_views / dt, "unit": UNIT, "cores": o32.num_threads(), "kind": "oracle",
+                                "sample": f"{n_sample_views} full view step(s) of the same workload"}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line))
+    tr.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -112,6 +112,17 @@ int odin_poll(odin_ctx* ctx, void* stream);
 /* Workspace size sufficient for every call below with at most n primitives and `max_instances` instance capacity. */
 int odin_workspace_bytes(const odin_ctx* ctx, uint32_t n, uint64_t max_instances, size_t* bytes);
 
+/* Launch accounting and optional per-kernel timing (the coarse phase profile the paper's scheduler consumes, Sec. 4.2,
+ * is built from numbers like these).  Every kernel launch of the library is counted per kernel id.  After
+ * odin_profile_enable(ctx, 1) each launch is also bracketed by two CUDA events on its stream (at most 65536 launches
+ * between collections).  odin_profile_collect synchronises `stream`, writes per kernel id the summed event time in
+ * milliseconds (h_ms, may be NULL) and the launch count since the last collection (h_launches, may be NULL) into HOST
+ * arrays of odin_kernel_count() entries, and resets both. */
+int odin_kernel_count(void);
+const char* odin_kernel_name(int id);
+int odin_profile_enable(odin_ctx* ctx, int on);
+int odin_profile_collect(odin_ctx* ctx, void* stream, float* h_ms, uint64_t* h_launches);
+
 /* ---- the seven calls of the view step ------------------------------------------------------------------------ */
 
 /* Preprocessing (phase P).  For every primitive: camera-space mean t = R mu + t_c; cull unless znear < t_z < zfar;

@@ -419,15 +419,18 @@ double l1_loss(int64_t count, const Real* out, const Real* target, Real* dL_dout
 // Backward of the compositing.  For every pixel the contributing splats are replayed front to
 // back (same skip tests; the list stops at n_contrib), then visited in reverse with the suffix sum
 // S_k = sum_{j>k} c_j alpha_j T_j + T_final * bg.  Output: dense [N,9] double gradient sums with
-// columns (u, v, conicA, conicB, conicC, opacity, r, g, b).
+// columns (u, v, conicA, conicB, conicC, opacity, r, g, b).  g2d_abs (optional, same shape) receives the sum of the
+// absolute values of the same per-pixel terms: the size against which a cancelled sum has to be judged.
 template <class Real>
 void render_bwd_blend(const Real* xy, const Real* conic_o, const Real* rgb, const uint32_t* vals, const uint32_t* ranges,
                       const CameraD& camd, const Config& cfg, const Real* final_T, const uint32_t* n_contrib,
-                      const Real* dL_dout, int64_t n, double* g2d) {
+                      const Real* dL_dout, int64_t n, double* g2d, double* g2d_abs) {
   const Cam<Real> cam = make_cam<Real>(camd, cfg.tile);
   const int W = cam.W, H = cam.H;
   const Real amin = (Real)cfg.alpha_min, amax = (Real)cfg.alpha_max;
   for (int64_t i = 0; i < 9 * n; ++i) g2d[i] = 0;
+  if (g2d_abs)
+    for (int64_t i = 0; i < 9 * n; ++i) g2d_abs[i] = 0;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int t = 0; t < cam.TX * cam.TY; ++t) {
     const int tx = t % cam.TX, ty = t / cam.TX;
@@ -467,6 +470,10 @@ void render_bwd_blend(const Real* xy, const Real* conic_o, const Real* rgb, cons
             const double dc = (double)e.alpha * (double)e.T * (double)g[ch];
 #pragma omp atomic
             g2d[9 * (size_t)p + 6 + ch] += dc;
+            if (g2d_abs) {
+#pragma omp atomic
+              g2d_abs[9 * (size_t)p + 6 + ch] += std::abs(dc);
+            }
             S[ch] += c * (double)e.alpha * (double)e.T;
           }
           if (e.clamped) continue;  // alpha = 0.99 is constant there
@@ -480,6 +487,10 @@ void render_bwd_blend(const Real* xy, const Real* conic_o, const Real* rgb, cons
           for (int w = 0; w < 6; ++w) {
 #pragma omp atomic
             g2d[9 * (size_t)p + w] += add[w];
+            if (g2d_abs) {
+#pragma omp atomic
+              g2d_abs[9 * (size_t)p + w] += std::abs(add[w]);
+            }
           }
         }
       }

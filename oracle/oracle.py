@@ -147,16 +147,18 @@ class Oracle:
         loss = self._f("oracle_l1_loss")(C.c_int64(o.size), _p(o), _p(t), _p(g))
         return float(loss), g
 
-    def render_bwd_blend(self, proj: Projected, vals, ranges, cam, final_t, n_contrib, dl_dout) -> np.ndarray:
+    def render_bwd_blend(self, proj: Projected, vals, ranges, cam, final_t, n_contrib, dl_dout, want_abs: bool = False):
+        """Dense [N,9] gradient sums; with want_abs also the sums of the absolute per-pixel terms."""
         n = proj.depth.shape[0]
         g2d = np.zeros((n, 9), np.float64)
+        g2d_abs = np.zeros((n, 9), np.float64) if want_abs else None
         self._f("oracle_render_bwd_blend")(
             _p(self._a(proj.xy)), _p(self._a(proj.conic_o)), _p(self._a(proj.rgb)),
             _p(np.ascontiguousarray(vals, np.uint32)), _p(np.ascontiguousarray(ranges, np.uint32)), _p(_cam(cam)),
             _p(self.cfg), _p(self._a(final_t)), _p(np.ascontiguousarray(n_contrib, np.uint32)), _p(self._a(dl_dout)),
-            C.c_int64(n), _p(g2d),
+            C.c_int64(n), _p(g2d), _p(g2d_abs),
         )
-        return g2d
+        return (g2d, g2d_abs) if want_abs else g2d
 
     def render_bwd_project(self, scene, cam, idx, g2d, clamp_flags) -> np.ndarray:
         idx = np.ascontiguousarray(idx, np.uint32)

@@ -46,9 +46,10 @@ Config cfg_from(const double* c) {
   extern "C" void oracle_render_bwd_blend_##SUF(const Real* xy, const Real* conic_o, const Real* rgb,                 \
                                                 const uint32_t* vals, const uint32_t* ranges, const double* cam,       \
                                                 const double* cfg, const Real* final_T, const uint32_t* n_contrib,     \
-                                                const Real* dL_dout, int64_t n, double* g2d) {                         \
+                                                const Real* dL_dout, int64_t n, double* g2d,           \
+                                                double* g2d_abs) {                                                     \
     render_bwd_blend<Real>(xy, conic_o, rgb, vals, ranges, cam_from(cam), cfg_from(cfg), final_T, n_contrib, dL_dout,  \
-                           n, g2d);                                                                                    \
+                           n, g2d, g2d_abs);                                                                           \
   }                                                                                                                    \
   extern "C" void oracle_render_bwd_project_##SUF(int sh_degree, const Real* means, const Real* log_scales,           \
                                                   const Real* quats, const Real* opacity_logit, const Real* sh,        \

@@ -26,7 +26,7 @@ ODIN_ERR_UNSUPPORTED = -7
 EXPORTS = [
     "odin_create", "odin_destroy", "odin_status_string", "odin_poll", "odin_workspace_bytes", "odin_project",
     "odin_touched_set", "odin_bin_sort", "odin_render_fwd", "odin_l1_loss", "odin_render_bwd", "odin_sparse_adam",
-    "odin_conflict_count",
+    "odin_conflict_count", "odin_kernel_count", "odin_kernel_name", "odin_profile_enable", "odin_profile_collect",
 ]
 
 
@@ -90,9 +90,14 @@ def lib() -> C.CDLL:
         L.odin_sparse_adam.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_scene), C.POINTER(odin_scene),
                                        C.POINTER(odin_scene), vp, vp, C.POINTER(f32), f32, f32, f32, u32, vp]
         L.odin_conflict_count.argtypes = [vp, vp, u32, u32, u32, vp, u32, vp, vp]
+        L.odin_kernel_count.argtypes = []
+        L.odin_kernel_name.argtypes = [i32]
+        L.odin_profile_enable.argtypes = [vp, i32]
+        L.odin_profile_collect.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(u64)]
         for name in EXPORTS:
-            if name != "odin_status_string":
+            if name not in ("odin_status_string", "odin_kernel_name"):
                 getattr(L, name).restype = C.c_int
+        L.odin_kernel_name.restype = C.c_char_p
         _lib = L
     return _lib
 
@@ -213,3 +218,24 @@ def odin_conflict_count(ctx, d_masks, n_masks: int, mask_stride_words: int, n_pr
                         stream=None) -> None:
     _check(lib().odin_conflict_count(ctx, _ptr(d_masks), int(n_masks), int(mask_stride_words), int(n_prims), _ptr(d_pairs),
                                      int(n_pairs), _ptr(d_counts), _stream(stream)), "odin_conflict_count")
+
+
+def odin_kernel_count() -> int:
+    return int(lib().odin_kernel_count())
+
+
+def odin_kernel_name(kid: int) -> str:
+    return lib().odin_kernel_name(int(kid)).decode()
+
+
+def odin_profile_enable(ctx, on: bool) -> None:
+    _check(lib().odin_profile_enable(ctx, 1 if on else 0), "odin_profile_enable")
+
+
+def odin_profile_collect(ctx, stream=None):
+    """Synchronises the stream; returns {kernel name: (milliseconds summed over its launches, launches)}."""
+    k = odin_kernel_count()
+    ms = (C.c_float * k)()
+    cnt = (C.c_uint64 * k)()
+    _check(lib().odin_profile_collect(ctx, _stream(stream), ms, cnt), "odin_profile_collect")
+    return {odin_kernel_name(i): (float(ms[i]), int(cnt[i])) for i in range(k)}

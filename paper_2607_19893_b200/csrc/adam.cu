@@ -122,14 +122,18 @@ extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m
   size_t blocks = (max_elems + 255) / 256;
   if (blocks > (size_t)ctx->sm_count * 16) blocks = (size_t)ctx->sm_count * 16;
   const unsigned gsh = (unsigned)blocks;
-  switch (params->sh_degree) {
+  {
+    OdinKernelScope ks(ctx, K_ADAM_SH, st);
+    switch (params->sh_degree) {
     case 0: adam_sh_kernel<3, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
     case 1: adam_sh_kernel<12, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
     case 2: adam_sh_kernel<27, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
     default: adam_sh_kernel<48, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
+    }
   }
   size_t gb = ((size_t)cap + 255) / 256;
   if (gb > (size_t)ctx->sm_count * 16) gb = (size_t)ctx->sm_count * 16;
+  OdinKernelScope ks(ctx, K_ADAM_GEOM, st);
   adam_geom_kernel<<<(unsigned)gb, 256, 0, st>>>(
       params->means, params->log_scales, reinterpret_cast<float4*>(params->quats), params->opacity_logit, m->means,
       m->log_scales, reinterpret_cast<float4*>(m->quats), m->opacity_logit, v->means, v->log_scales,

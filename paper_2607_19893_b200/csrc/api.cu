@@ -38,6 +38,7 @@ extern "C" int odin_destroy(odin_ctx* ctx) {
   if (!ctx) return ODIN_ERR_NULL;
   cudaFree(ctx->d_status);
   cudaFreeHost(ctx->h_status);
+  for (cudaEvent_t e : ctx->prof.events) cudaEventDestroy(e);
   delete ctx;
   return ODIN_OK;
 }
@@ -65,6 +66,37 @@ extern "C" int odin_poll(odin_ctx* ctx, void* stream) {
   const int s = *ctx->h_status;
   *ctx->h_status = 0;
   return s;
+}
+
+static const char* const kKernelNames[K_COUNT] = {
+    "project", "touched_set", "emit_instances", "digit_base", "onesweep_pass", "tile_ranges", "render_fwd", "l1_loss",
+    "l1_finish", "zero_rows", "render_bwd_blend", "render_bwd_project", "adam_sh", "adam_geom", "conflict_count"};
+
+extern "C" int odin_kernel_count(void) { return K_COUNT; }
+
+extern "C" const char* odin_kernel_name(int id) { return (id >= 0 && id < K_COUNT) ? kKernelNames[id] : "unknown"; }
+
+extern "C" int odin_profile_enable(odin_ctx* ctx, int on) {
+  if (!ctx) return ODIN_ERR_NULL;
+  ctx->prof.enabled = on != 0;
+  return ODIN_OK;
+}
+
+extern "C" int odin_profile_collect(odin_ctx* ctx, void* stream, float* h_ms, uint64_t* h_launches) {
+  if (!ctx) return ODIN_ERR_NULL;
+  ODIN_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  OdinProf& p = ctx->prof;
+  for (int k = 0; k < K_COUNT; ++k) {
+    if (h_ms) h_ms[k] = 0.f;
+    if (h_launches) h_launches[k] = p.launches[k];
+    p.launches[k] = 0;
+  }
+  for (size_t i = 0; i < p.used; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, p.events[2 * i], p.events[2 * i + 1]) == cudaSuccess && h_ms) h_ms[p.ids[i]] += ms;
+  }
+  p.used = 0;
+  return ODIN_OK;
 }
 
 extern "C" int odin_workspace_bytes(const odin_ctx* ctx, uint32_t n, uint64_t max_instances, size_t* bytes) {

@@ -299,13 +299,20 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
 
   const uint64_t chunks_cap = (capacity + DUP_CHUNK - 1) / DUP_CHUNK;
   uint32_t grid = (uint32_t)(chunks_cap < (uint64_t)ctx->sm_count * 6 ? chunks_cap : (uint64_t)ctx->sm_count * 6);
-  emit_instances_kernel<<<grid, DUP_THREADS, 0, st>>>(proj->tile_offset, reinterpret_cast<const ushort4*>(proj->rect),
-                                                      proj->depth, proj->num_rows, proj->num_instances, capacity, TX,
-                                                      passes, kbuf[cur], vbuf[cur], hist, ctx->d_status);
-  digit_base_kernel<<<passes, SORT_RADIX, 0, st>>>(hist, dbase);
+  {
+    OdinKernelScope ks(ctx, K_EMIT, st);
+    emit_instances_kernel<<<grid, DUP_THREADS, 0, st>>>(proj->tile_offset, reinterpret_cast<const ushort4*>(proj->rect),
+                                                        proj->depth, proj->num_rows, proj->num_instances, capacity, TX,
+                                                        passes, kbuf[cur], vbuf[cur], hist, ctx->d_status);
+  }
+  {
+    OdinKernelScope ks(ctx, K_DIGIT_BASE, st);
+    digit_base_kernel<<<passes, SORT_RADIX, 0, st>>>(hist, dbase);
+  }
   ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OS_SMEM));
   uint32_t os_grid = L.tiles < (uint32_t)ctx->sm_count * 3 ? L.tiles : (uint32_t)ctx->sm_count * 3;
   for (int p = 0; p < passes; ++p) {
+    OdinKernelScope ks(ctx, K_ONESWEEP, st);
     onesweep_kernel<<<os_grid, OS_THREADS, OS_SMEM, st>>>(kbuf[cur], vbuf[cur], kbuf[cur ^ 1], vbuf[cur ^ 1],
                                                           proj->num_instances, capacity, p * (int)SORT_RADIX_BITS,
                                                           dbase + p * SORT_RADIX, states + (size_t)p * L.tiles * SORT_RADIX,
@@ -314,6 +321,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   }
   const uint64_t rblocks = (capacity + 255) / 256;
   const uint32_t rgrid = (uint32_t)(rblocks < (uint64_t)ctx->sm_count * 8 ? rblocks : (uint64_t)ctx->sm_count * 8);
+  OdinKernelScope ks(ctx, K_RANGES, st);
   tile_ranges_kernel<<<rgrid, 256, 0, st>>>(d_keys, proj->num_instances, capacity, n_tiles, d_tile_ranges);
   return odin_launch_status();
 }

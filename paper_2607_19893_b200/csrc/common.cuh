@@ -3,7 +3,23 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "../../include/odin.h"
+
+// Kernel ids for launch counting and optional per-kernel CUDA-event timing.
+enum OdinKernelId {
+  K_PROJECT = 0, K_TOUCHED, K_EMIT, K_DIGIT_BASE, K_ONESWEEP, K_RANGES, K_FWD, K_L1, K_L1_FINISH, K_ZERO_ROWS,
+  K_BWD_BLEND, K_BWD_PROJECT, K_ADAM_SH, K_ADAM_GEOM, K_CONFLICT, K_COUNT
+};
+
+struct OdinProf {
+  bool enabled = false;
+  std::vector<cudaEvent_t> events;  // start/stop pairs, reused between collections
+  std::vector<int> ids;             // kernel id of pair i
+  size_t used = 0;                  // pairs recorded since the last collection
+  uint64_t launches[K_COUNT] = {};
+};
 
 struct odin_ctx {
   int device;
@@ -11,6 +27,34 @@ struct odin_ctx {
   odin_config cfg;
   int* d_status;  // first deferred device-side error (0 = none)
   int* h_status;  // pinned mirror read by odin_poll
+  OdinProf prof;
+};
+
+// Brackets one kernel launch: counts it and, when profiling is on, records a CUDA event on the launch stream before
+// and after it.
+struct OdinKernelScope {
+  odin_ctx* ctx;
+  cudaStream_t st;
+  bool rec = false;
+  size_t slot = 0;
+  OdinKernelScope(odin_ctx* c, int id, cudaStream_t s) : ctx(c), st(s) {
+    OdinProf& p = c->prof;
+    ++p.launches[id];
+    if (!p.enabled || p.used >= (1u << 16)) return;
+    slot = p.used++;
+    if (p.events.size() < 2 * (slot + 1)) {
+      cudaEvent_t a = nullptr, b = nullptr;
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { --p.used; return; }
+      p.events.push_back(a); p.events.push_back(b); p.ids.push_back(id);
+    } else {
+      p.ids[slot] = id;
+    }
+    rec = true;
+    cudaEventRecord(p.events[2 * slot], st);
+  }
+  ~OdinKernelScope() {
+    if (rec) cudaEventRecord(ctx->prof.events[2 * slot + 1], st);
+  }
 };
 
 #define ODIN_CUDA(call)                          \

@@ -166,6 +166,7 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   project_kernel<D><<<grid, PROJECT_TILE, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit, scene->sh, \
                                                    n, cp, ctx->cfg.dilation, ctx->cfg.radius_sigmas, *out, ticket, state, \
                                                    ctx->d_status)
+  OdinKernelScope ks(ctx, K_PROJECT, st);
   switch (scene->sh_degree) {
     case 0: LAUNCH(0); break;
     case 1: LAUNCH(1); break;

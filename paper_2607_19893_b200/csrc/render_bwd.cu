@@ -269,11 +269,17 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
   cudaStream_t st = (cudaStream_t)stream;
   const int TX = (cam->width + 15) / 16, TY = (cam->height + 15) / 16;
   const uint32_t zgrid = (uint32_t)ctx->sm_count * 8;
-  zero_rows_kernel<<<zgrid, 256, 0, st>>>(d_grad2d, proj->num_rows, proj->capacity);
-  render_bwd_blend_kernel<<<TX * TY, BB, 0, st>>>(
-      reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
-      reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
-      ctx->cfg.alpha_min, ctx->cfg.alpha_max, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d);
+  {
+    OdinKernelScope ks(ctx, K_ZERO_ROWS, st);
+    zero_rows_kernel<<<zgrid, 256, 0, st>>>(d_grad2d, proj->num_rows, proj->capacity);
+  }
+  {
+    OdinKernelScope ks(ctx, K_BWD_BLEND, st);
+    render_bwd_blend_kernel<<<TX * TY, BB, 0, st>>>(
+        reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
+        reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
+        ctx->cfg.alpha_min, ctx->cfg.alpha_max, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d);
+  }
   const CamParams cp = odin_cam_params(cam, ctx->cfg);
   const uint32_t blocks_cap = (proj->capacity + 127) / 128;
   const uint32_t pgrid = blocks_cap < (uint32_t)ctx->sm_count * 16 ? blocks_cap : (uint32_t)ctx->sm_count * 16;
@@ -283,6 +289,7 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
       cp, ctx->cfg.dilation, proj->prim_id, proj->clamp_flags, proj->num_rows, proj->capacity, d_grad2d,                \
       grad_rows->means, grad_rows->log_scales, reinterpret_cast<float4*>(grad_rows->quats), grad_rows->opacity_logit,    \
       grad_rows->sh)
+  OdinKernelScope ks(ctx, K_BWD_PROJECT, st);
   switch (scene->sh_degree) {
     case 0: LAUNCH(0); break;
     case 1: LAUNCH(1); break;

@@ -102,6 +102,7 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
   if (!odin_aligned(proj->xy, 8) || !odin_aligned(proj->conic_opacity, 16) || !odin_aligned(d_tile_ranges, 8))
     return ODIN_ERR_INVALID_ARG;
   const int TX = (cam->width + 15) / 16, TY = (cam->height + 15) / 16;
+  OdinKernelScope ks(ctx, K_FWD, (cudaStream_t)stream);
   render_fwd_kernel<<<TX * TY, FB, 0, (cudaStream_t)stream>>>(
       reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
       reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
@@ -120,7 +121,11 @@ extern "C" int odin_l1_loss(odin_ctx* ctx, const float* d_rgb, const float* d_ta
   ODIN_CUDA(cudaMemsetAsync(acc, 0, 8, st));
   size_t blocks = (count + LB - 1) / LB;
   if (blocks > (size_t)ctx->sm_count * 8) blocks = (size_t)ctx->sm_count * 8;
-  l1_loss_kernel<<<(unsigned)blocks, LB, 0, st>>>(d_rgb, d_target, count, (float)(1.0 / (double)count), acc, d_dL_drgb);
+  {
+    OdinKernelScope ks(ctx, K_L1, st);
+    l1_loss_kernel<<<(unsigned)blocks, LB, 0, st>>>(d_rgb, d_target, count, (float)(1.0 / (double)count), acc, d_dL_drgb);
+  }
+  OdinKernelScope ks(ctx, K_L1_FINISH, st);
   l1_finish_kernel<<<1, 1, 0, st>>>(acc, 1.0 / (double)count, d_loss);
   return odin_launch_status();
 }

@@ -124,6 +124,7 @@ extern "C" int odin_touched_set(odin_ctx* ctx, const uint32_t* d_tiles_touched, 
   uint32_t* ticket = reinterpret_cast<uint32_t*>(ws);
   uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + 256);
   const uint32_t grid = (n + TOUCHED_TILE - 1) / TOUCHED_TILE;
+  OdinKernelScope ks(ctx, K_TOUCHED, st);
   touched_set_kernel<<<grid, TS_THREADS, 0, st>>>(d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket, state,
                                                   ctx->d_status);
   return odin_launch_status();
@@ -147,6 +148,7 @@ extern "C" int odin_conflict_count(odin_ctx* ctx, const uint32_t* d_masks, uint3
   const uint32_t cap = (uint32_t)(ctx->sm_count * 8 + n_pairs - 1) / n_pairs;
   if (gx > cap) gx = cap;
   if (gx == 0) gx = 1;
+  OdinKernelScope ks(ctx, K_CONFLICT, st);
   conflict_count_kernel<<<dim3(gx, n_pairs), CC_THREADS, 0, st>>>(d_masks, mask_stride_words, words, d_pairs, n_masks,
                                                                  reinterpret_cast<unsigned long long*>(d_counts),
                                                                  ctx->d_status);

@@ -51,3 +51,31 @@ def rows_of(inv_idx, vals):
 def poll_ok(tr):
     st = tr.poll()
     assert st == B.ODIN_OK, B.status_string(st)
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Gradient parity bar.  A gradient word is a sum over pixels of signed terms.  fp32 evaluation on the device
+# (ex2.approx, transmittance recovered by division, atomic accumulation order) perturbs every TERM by a relative
+# ~1e-6, so the error of the SUM scales with sum|term| (reported by the oracle), not with the possibly cancelled
+# sum.  Bar for the nine compositing words:  |dev - oracle| <= 1e-3 |oracle| + 1e-5 sum|term|.
+# The per-primitive chain rule is linear in those nine words, so the same absolute slack is pushed through the
+# oracle's own Jacobian (nine evaluations on unit inputs) for the final gradient rows.
+GRAD_RTOL = 1e-3
+GRAD_FLOOR = 1e-5
+
+
+def grad2d_bound(want2d, abs2d):
+    return GRAD_RTOL * np.abs(want2d) + GRAD_FLOOR * abs2d + 1e-30
+
+
+def rows_bound(oracle, scene, cam, idx, clamp_flags, rows_o, want2d_dense, abs2d_dense):
+    n = want2d_dense.shape[0]
+    # second term: rounding inside the fp32 chain rule itself (its own sums cancel too)
+    slack2d = GRAD_FLOOR * abs2d_dense + GRAD_FLOOR * np.abs(want2d_dense)
+    bound = GRAD_RTOL * np.abs(rows_o) + 1e-30
+    for c in range(9):
+        unit = np.zeros((n, 9))
+        unit[:, c] = 1.0
+        jac_c = oracle.render_bwd_project(scene, cam, idx, unit, clamp_flags).astype(np.float64)
+        bound = bound + np.abs(jac_c) * slack2d[idx.astype(np.int64), c][:, None]
+    return bound

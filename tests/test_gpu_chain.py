@@ -28,15 +28,21 @@ def run_chain(oracle32, w, steps, views, window=None):
         view = views[s % len(views)]
         cam = w.cameras[view]
         tgt = w.target(view)
+        pre = p.copy()  # parameters this view was rendered with
         o = oracle32.view_step(p, m, v, cam, tgt, w.lr, w.beta1, w.beta2, w.eps, s + 1)
         tr.target.copy_(torch.from_numpy(tgt).to(dev))
         slot = s % len(views)
         tr.view_step(B.make_camera(cam), s + 1, w.lr, w.beta1, w.beta2, w.eps, slot=slot)
         G.poll_ok(tr)
-        fragile_prims = o["proj"].margin < 1e-4
-        n_fragile += int(fragile_prims.sum())
+        # integer decisions of the projection may legitimately differ only on primitives that sit within a few
+        # float ulps of a threshold; when none differs, every integer output of the chain must be bit exact
+        fragile_prims = o["proj"].margin < 2e-6
+        tt_dev = G.u32(tr.proj.tiles_touched)[:n]
+        differs = tt_dev != o["proj"].tiles_touched
+        assert not (differs & ~fragile_prims).any()
+        n_fragile += int(differs.sum())
         vdev = int(tr.count.item())
-        if not fragile_prims.any():
+        if not differs.any():
             # identical projected decisions: integer outputs are bit exact through the whole chain
             assert vdev == len(o["idx"])
             assert np.array_equal(G.u32(tr.idx)[:vdev], o["idx"])
@@ -57,23 +63,35 @@ def run_chain(oracle32, w, steps, views, window=None):
         dev_state = [t.cpu().numpy() for s_ in (tr.params, tr.m, tr.v) for t in s_.tensors()]
         host_state = [a for s_ in (p, m, v) for a in (s_.means, s_.log_scales, s_.quats, s_.opacity_logit, s_.sh)]
         un = np.setdiff1d(np.arange(n), idx)
-        for i, (d, h) in enumerate(zip(dev_state, host_state)):
+        for d, h in zip(dev_state, host_state):
             # untouched rows identical to the oracle's (which never changed them)
             assert np.array_equal(d[un].view(np.uint32), h[un].view(np.uint32))
-            if i >= 5:  # m and v are direct functions of the gradient
-                scale = np.abs(h[idx]).mean() + 1e-30
-                assert np.all(np.abs(d[idx] - h[idx]) <= 1e-3 * np.abs(h[idx]) + 1e-3 * scale + 1e-12), i
-        # parameters: with eps = 1e-15 the first steps move every touched scalar by ~lr * sign(g); a gradient that is
-        # pure rounding noise may flip, so compare where the oracle's gradient is not negligible
-        rows = o["rows"]
-        gsc = np.abs(rows).mean(axis=0, keepdims=True) + 1e-30
-        sig = np.abs(rows) > 1e-3 * gsc
-        devp = np.concatenate([dev_state[0][idx], dev_state[1][idx], dev_state[2][idx], dev_state[3][idx][:, None],
-                               dev_state[4][idx].reshape(len(idx), -1)], axis=1)
-        hostp = np.concatenate([p.means[idx], p.log_scales[idx], p.quats[idx], p.opacity_logit[idx][:, None],
-                                p.sh[idx].reshape(len(idx), -1)], axis=1)
-        assert np.all(np.abs(devp - hostp)[sig] <= 1e-3 * np.abs(hostp)[sig] + 1e-5)
-        assert sig.mean() > 0.9
+        # gradient rows: every word inside the bar derived from the un-cancelled term sums (see gpu_util)
+        _, g2d_abs = oracle32.render_bwd_blend(o["proj"], o["vals"], o["ranges"], cam, o["final_T"], o["n_contrib"],
+                                               o["dL_dout"], want_abs=True)
+        rows = o["rows"].astype(np.float64)
+        rows_dev = tr.grads.rows_as_matrix(len(idx)).astype(np.float64)
+        if not differs.any():
+            bound = G.rows_bound(oracle32, pre, cam, o["idx"], o["proj"].clamp_flags, rows, o["g2d"], g2d_abs)
+            # the chained run also carries the device's own projection and pixel rounding into the gradients
+            assert (np.abs(rows_dev - rows) <= 4 * bound).mean() > 0.9999
+        # Adam state and parameters.  With eps = 1e-15 a first Adam step is ~ lr * sign(g), so a gradient word that is
+        # rounding noise (a cancelled sum) can legitimately move its parameter the other way: compare m, v and the
+        # parameters wherever the two gradients agree to 1e-3 relative, and require that to be the bulk of the words.
+        agree = np.abs(rows_dev - rows) <= 1e-3 * np.abs(rows)
+        assert agree.mean() > 0.9, agree.mean()
+
+        def as_rows(st):
+            return np.concatenate([st[0][idx], st[1][idx], st[2][idx], st[3][idx][:, None],
+                                   st[4][idx].reshape(len(idx), -1)], axis=1).astype(np.float64)
+
+        g_abs = np.abs(rows)
+        dp, hp = as_rows(dev_state[0:5]), as_rows(host_state[0:5])
+        dm, hm = as_rows(dev_state[5:10]), as_rows(host_state[5:10])
+        dv, hv = as_rows(dev_state[10:15]), as_rows(host_state[10:15])
+        assert np.all(np.abs(dm - hm)[agree] <= (1e-3 * (1 - w.beta1) * g_abs + 1e-6 * np.abs(hm) + 1e-30)[agree])
+        assert np.all(np.abs(dv - hv)[agree] <= (2.1e-3 * (1 - w.beta2) * g_abs ** 2 + 1e-6 * np.abs(hv) + 1e-30)[agree])
+        assert np.all(np.abs(dp - hp)[agree] <= 1e-3 * np.abs(hp)[agree] + 1e-5)
         masks_o[slot] = o["idx"]
         # re-synchronise the oracle's state from the device
         for s_dev, s_host in ((tr.params, p), (tr.m, m), (tr.v, v)):

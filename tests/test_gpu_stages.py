@@ -14,7 +14,6 @@ import gpu_util as G
 pytestmark = pytest.mark.gpu
 
 PIX_TOL = 1e-4          # absolute, rendered pixels
-GRAD_RTOL, GRAD_ATOL = 1e-3, 1e-5  # gradients and updated parameters
 
 
 # ------------------------------------------------------------------------------------------------ touched set
@@ -148,8 +147,9 @@ def check_projection(oracle32, scene, cam, row_capacity=None):
         tr.project(ccam)
         G.poll_ok(tr)
     tt = G.u32(tr.proj.tiles_touched)[: scene.n]
-    safe = po.margin > 1e-4
-    assert safe.mean() > 0.98
+    # a primitive is "safe" when none of its integer decisions sits within ~30 float ulps of its threshold
+    safe = po.margin > 2e-6
+    assert safe.mean() > 0.995
     assert np.array_equal(tt[safe], po.tiles_touched[safe])
     v = int(tr.proj.num_rows.item())
     prim = G.u32(tr.proj.prim_id)[:v]
@@ -310,7 +310,8 @@ def check_forward(oracle32, scene, cam):
     out = tr.out.cpu().numpy()
     ft = tr.final_T.cpu().numpy()
     nc = G.u32(tr.n_contrib)
-    robust = f["pix_margin"] > 1e-4
+    # the device evaluates exp with ex2.approx (relative error ~1e-6): a threshold test within 2e-5 may flip
+    robust = f["pix_margin"] > 2e-5
     assert robust.mean() > 1 - 2e-3
     assert np.abs(out - f["out"])[:, robust].max() < PIX_TOL
     assert np.abs(ft - f["final_T"])[robust].max() < PIX_TOL
@@ -364,29 +365,36 @@ def test_l1_loss(oracle32):
 def check_backward(oracle32, scene, cam, seed=0):
     f, inv = oracle_view(oracle32, scene, cam)
     rng = np.random.default_rng(seed)
-    dl = (rng.uniform(-1, 1, f["out"].shape) / f["out"].size).astype(np.float32)
-    g2d_o = oracle32.render_bwd_blend(f["proj"], f["vals"], f["ranges"], cam, f["final_T"], f["n_contrib"], dl)
-    rows_o = oracle32.render_bwd_project(scene, cam, f["idx"], g2d_o, f["proj"].clamp_flags)
+    dl = rng.uniform(-1, 1, f["out"].shape).astype(np.float32)
+    g2d_o, g2d_abs = oracle32.render_bwd_blend(f["proj"], f["vals"], f["ranges"], cam, f["final_T"], f["n_contrib"], dl,
+                                               want_abs=True)
+    rows_o = oracle32.render_bwd_project(scene, cam, f["idx"], g2d_o, f["proj"].clamp_flags).astype(np.float64)
     v = len(f["idx"])
     tr = G.trainer_for(scene, cam, row_capacity=max(v, 1), instance_capacity=len(f["vals"]) + 1)
     load_sorted(tr, f, inv)
     tr.final_T.copy_(torch.from_numpy(f["final_T"]).to(tr.device))
     tr.n_contrib.copy_(torch.from_numpy(f["n_contrib"].view(np.int32)).to(tr.device))
     tr.dL.copy_(torch.from_numpy(dl).to(tr.device))
-    for _ in range(2):
+    for _ in range(2):  # twice: accumulators are re-zeroed, atomics order changes
         tr.render_bwd(B.make_camera(cam))
         G.poll_ok(tr)
-    g2d = tr.grad2d.cpu().numpy()[:v].astype(np.float64)
-    want2d = g2d_o[f["idx"]]
-    # per column scale: sums of many signed terms are compared relative to the column's typical size
-    for c in range(9):
-        scale = np.abs(want2d[:, c]).mean() + 1e-30
-        err = np.abs(g2d[:, c] - want2d[:, c])
-        assert np.all(err <= GRAD_RTOL * np.abs(want2d[:, c]) + GRAD_RTOL * scale + 1e-12), (c, err.max(), scale)
-    rows = tr.grads.rows_as_matrix(v).astype(np.float64)
-    scale = np.abs(rows_o).mean(axis=0) + 1e-30
-    err = np.abs(rows - rows_o)
-    assert np.all(err <= GRAD_RTOL * np.abs(rows_o) + GRAD_RTOL * scale[None, :] + 1e-12), err.max()
+        g2d = tr.grad2d.cpu().numpy()[:v].astype(np.float64)
+        want2d, abs2d = g2d_o[f["idx"]], g2d_abs[f["idx"]]
+        err = np.abs(g2d - want2d)
+        bad = err > G.grad2d_bound(want2d, abs2d)
+        assert not bad.any(), (int(bad.sum()), np.argwhere(bad)[:5], err[bad][:5], want2d[bad][:5], abs2d[bad][:5])
+        assert np.abs(want2d).max() > 1e-3
+        rows = tr.grads.rows_as_matrix(v).astype(np.float64)
+        bound = G.rows_bound(oracle32, scene, cam, f["idx"], f["proj"].clamp_flags, rows_o, g2d_o, g2d_abs)
+        err = np.abs(rows - rows_o)
+        bad = err > bound
+        # the bound does not see cancellation INSIDE a Jacobian entry (e.g. the conic-to-covariance step of a nearly
+        # degenerate conic), where oracle and device both round in fp32: allow 1e-4 of the words up to 10x the bound
+        assert bad.mean() < 1e-4 and not (err > 10 * bound).any(), (
+            int(bad.sum()), np.argwhere(bad)[:5], err[bad][:5], rows_o[bad][:5], bound[bad][:5])
+        # most words are not cancelled sums and meet the plain bar: 1e-3 relative with a 1e-5 absolute floor
+        plain = err <= 1e-3 * np.abs(rows_o) + 1e-5
+        assert plain.mean() > 0.999, plain.mean()
     tr.close()
 
 
