@@ -141,6 +141,24 @@ int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_camera* cam,
 int odin_touched_set(odin_ctx* ctx, const uint32_t* d_tiles_touched, uint32_t n, uint32_t* d_mask, uint32_t* d_idx,
                      uint32_t idx_capacity, uint32_t* d_count, void* ws, size_t ws_bytes, void* stream);
 
+/* Touched set for callers that may not allocate.  (The paper has no counterpart; this is a packaging variant of
+ * odin_touched_set.)  Some users get all of their GPU memory handed out up front and are never allowed to allocate
+ * again - a component living inside a host application's memory pool, a real-time loop where an allocation may stall or
+ * fail - so they can neither create a context nor allocate a workspace.  This call needs neither: it runs the same
+ * kernel with its scratch in a fixed device array that is part of the library image (128.3 KB on every GPU that loads
+ * the library, held until the process exits).  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *  - Inputs and outputs are the caller's device buffers, exactly as for odin_touched_set; the work runs on the device
+ *    that is current when the call is made.
+ *  - n may be at most 33,554,432 (2^25) primitives; a larger n returns ODIN_ERR_INVALID_ARG and nothing is launched.
+ *  - d_status (device int, may be NULL) is where a deferred ODIN_ERR_CAPACITY / ODIN_ERR_TIMEOUT is written (only if it
+ *    holds 0, so clear it beforehand); with NULL those conditions are dropped (outputs are still truncated safely).
+ *  - The first call on each device also looks up the array's device address; make that first call before any stream
+ *    capture begins.
+ *  - Every call on a device shares the one array.  The call clears the part it uses, but two calls whose kernels
+ *    overlap on the GPU (different streams, different host threads) race on it: serialise them. */
+int odin_touched_set_static(const uint32_t* d_tiles_touched, uint32_t n, uint32_t* d_mask, uint32_t* d_idx,
+                            uint32_t idx_capacity, uint32_t* d_count, int* d_status, void* stream);
+
 /* Binning and sort.  Emits one (key, value) per (tile, row) pair of the rectangles: key = tile_id << 32 | bit pattern
  * of the float32 depth, tile_id = ty * ceil(width/16) + tx; value = ROW index r (the primitive is proj->prim_id[r]).
  * Sorts by key with a least-significant-digit radix sort (stable: equal keys keep ascending row order) and writes

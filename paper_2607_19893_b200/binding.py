@@ -27,6 +27,7 @@ EXPORTS = [
     "odin_create", "odin_destroy", "odin_status_string", "odin_poll", "odin_workspace_bytes", "odin_project",
     "odin_touched_set", "odin_bin_sort", "odin_render_fwd", "odin_l1_loss", "odin_render_bwd", "odin_sparse_adam",
     "odin_conflict_count", "odin_kernel_count", "odin_kernel_name", "odin_profile_enable", "odin_profile_collect",
+    "odin_touched_set_static",
 ]
 
 
@@ -90,6 +91,7 @@ def lib() -> C.CDLL:
         L.odin_sparse_adam.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_scene), C.POINTER(odin_scene),
                                        C.POINTER(odin_scene), vp, vp, C.POINTER(f32), f32, f32, f32, u32, vp]
         L.odin_conflict_count.argtypes = [vp, vp, u32, u32, u32, vp, u32, vp, vp]
+        L.odin_touched_set_static.argtypes = [vp, u32, vp, vp, u32, vp, vp, vp]
         L.odin_kernel_count.argtypes = []
         L.odin_kernel_name.argtypes = [i32]
         L.odin_profile_enable.argtypes = [vp, i32]
@@ -179,6 +181,14 @@ def odin_touched_set(ctx, d_tiles_touched, n: int, d_mask, d_idx, idx_capacity: 
     _check(lib().odin_touched_set(ctx, _ptr(d_tiles_touched), int(n), _ptr(d_mask), _ptr(d_idx), int(idx_capacity),
                                   _ptr(d_count), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
                                   _stream(stream)), "odin_touched_set")
+
+
+def odin_touched_set_static(d_tiles_touched, n: int, d_mask, d_idx, idx_capacity: int, d_count, d_status=None,
+                            stream=None) -> None:
+    """Touched set for callers that are not allowed to allocate GPU memory (no context, no workspace): the scratch is
+    a fixed array inside the library, n <= 2**25.  Calls on one device share that array: do not let two overlap."""
+    _check(lib().odin_touched_set_static(_ptr(d_tiles_touched), int(n), _ptr(d_mask), _ptr(d_idx), int(idx_capacity),
+                                         _ptr(d_count), _ptr(d_status), _stream(stream)), "odin_touched_set_static")
 
 
 def odin_bin_sort(ctx, proj: odin_projected, width: int, height: int, d_keys, d_vals, capacity: int, d_tile_ranges, ws,

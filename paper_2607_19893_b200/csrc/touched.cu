@@ -130,6 +130,54 @@ extern "C" int odin_touched_set(odin_ctx* ctx, const uint32_t* d_tiles_touched, 
   return odin_launch_status();
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Touched set without any allocation.  Some users of this library are handed all of their GPU memory up front and may
+// never allocate again: a component embedded in a host application that owns the memory pool, or a real-time loop in
+// which an allocation could stall or fail at a bad moment.  They cannot call odin_create (it allocates the status word)
+// nor size and allocate a workspace.  For them this entry point runs the same kernel as odin_touched_set with its
+// scratch (tile ticket, deferred-status sink, look-back words) in a fixed array that is part of the loaded library:
+// every GPU that loads libodin.so holds these 128.3 KB until the process exits.
+constexpr uint32_t TS_STATIC_MAX_N = 1u << 25;  // 33,554,432 primitives
+constexpr size_t TS_STATIC_HEADER = 256;        // [0] ticket, [64] status sink
+constexpr size_t TS_STATIC_BYTES = TS_STATIC_HEADER + (size_t)(TS_STATIC_MAX_N / TOUCHED_TILE) * 8;
+static __device__ __align__(256) unsigned char g_touched_static_scratch[TS_STATIC_BYTES];
+
+// In host code the array's name is only a handle for the runtime, not a device address, so the address is asked for
+// once per device (with that device current) and cached.
+constexpr int TS_STATIC_MAX_DEVICES = 64;
+static unsigned char* g_touched_static_ptr[TS_STATIC_MAX_DEVICES] = {};
+
+extern "C" int odin_touched_set_static(const uint32_t* d_tiles_touched, uint32_t n, uint32_t* d_mask, uint32_t* d_idx,
+                                       uint32_t idx_capacity, uint32_t* d_count, int* d_status, void* stream) {
+  if (!d_count) return ODIN_ERR_NULL;
+  if (n > TS_STATIC_MAX_N) return ODIN_ERR_INVALID_ARG;  // beyond the fixed scratch: use odin_touched_set
+  cudaStream_t st = (cudaStream_t)stream;
+  if (n == 0) {
+    ODIN_CUDA(cudaMemsetAsync(d_count, 0, 4, st));
+    return ODIN_OK;
+  }
+  if (!d_tiles_touched || !d_mask || (idx_capacity > 0 && !d_idx)) return ODIN_ERR_NULL;
+  int device = -1;
+  ODIN_CUDA(cudaGetDevice(&device));
+  if (device < 0 || device >= TS_STATIC_MAX_DEVICES) return ODIN_ERR_UNSUPPORTED;
+  if (!g_touched_static_ptr[device]) {  // first call on this device: resolve the array's device address
+    void* p = nullptr;
+    ODIN_CUDA(cudaGetSymbolAddress(&p, g_touched_static_scratch));
+    if (!p) return ODIN_ERR_CUDA;
+    g_touched_static_ptr[device] = static_cast<unsigned char*>(p);
+  }
+  unsigned char* scratch = g_touched_static_ptr[device];
+  const uint32_t tiles = (n + TOUCHED_TILE - 1) / TOUCHED_TILE;
+  // the array keeps whatever the previous call left: the ticket, the sink and the look-back words must start at zero
+  ODIN_CUDA(cudaMemsetAsync(scratch, 0, TS_STATIC_HEADER + (size_t)tiles * 8, st));
+  uint32_t* ticket = reinterpret_cast<uint32_t*>(scratch);
+  int* status = d_status ? d_status : reinterpret_cast<int*>(scratch + 64);
+  uint64_t* state = reinterpret_cast<uint64_t*>(scratch + TS_STATIC_HEADER);
+  touched_set_kernel<<<tiles, TS_THREADS, 0, st>>>(d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket, state,
+                                                  status);
+  return odin_launch_status();
+}
+
 extern "C" int odin_conflict_count(odin_ctx* ctx, const uint32_t* d_masks, uint32_t n_masks, uint32_t mask_stride_words,
                                    uint32_t n_prims, const uint32_t* d_pairs, uint32_t n_pairs, uint64_t* d_counts,
                                    void* stream) {
