@@ -109,8 +109,14 @@ const char* odin_status_string(int status);
  * clears it. */
 int odin_poll(odin_ctx* ctx, void* stream);
 
-/* Workspace size sufficient for every call below with at most n primitives and `max_instances` instance capacity. */
+/* Workspace size sufficient for odin_project, odin_touched_set and odin_bin_sort with at most n primitives and
+ * `max_instances` instance capacity. */
 int odin_workspace_bytes(const odin_ctx* ctx, uint32_t n, uint64_t max_instances, size_t* bytes);
+
+/* Workspace size for odin_render_fwd / odin_render_bwd on a width x height image (per-tile flags and 16 bytes per
+ * pixel of hand-over state for tiles with long lists).  The same workspace may serve all five calls if it is at least
+ * as large as both sizes. */
+int odin_render_workspace_bytes(const odin_ctx* ctx, int width, int height, size_t* bytes);
 
 /* Launch accounting and optional per-kernel timing (the coarse phase profile the paper's scheduler consumes, Sec. 4.2,
  * is built from numbers like these).  Every kernel launch of the library is counted per kernel id.  After
@@ -173,7 +179,8 @@ int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int width, int heig
  * d_rgb [3][H][W] = colour + T * bg (planar, not clamped); d_final_T [H][W]; d_n_contrib [H][W] = 1 + list offset of the
  * last row that contributed (0 if none). */
 int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const uint32_t* d_vals, const uint32_t* d_tile_ranges,
-                    const odin_camera* cam, float* d_rgb, float* d_final_T, uint32_t* d_n_contrib, void* stream);
+                    const odin_camera* cam, float* d_rgb, float* d_final_T, uint32_t* d_n_contrib, void* ws, size_t ws_bytes,
+                    void* stream);
 
 /* Image loss of the view (Sec. 2.1): d_loss [1] = mean |rgb - target| over 3*H*W values;
  * d_dL_drgb [3][H][W] = sign(rgb - target) / (3 H W). */
@@ -190,7 +197,7 @@ int odin_l1_loss(odin_ctx* ctx, const float* d_rgb, const float* d_target, int w
 int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odin_camera* cam, const odin_projected* proj,
                     const uint32_t* d_vals, const uint32_t* d_tile_ranges, const float* d_final_T,
                     const uint32_t* d_n_contrib, const float* d_dL_drgb, float* d_grad2d, odin_scene* grad_rows,
-                    void* stream);
+                    void* ws, size_t ws_bytes, void* stream);
 
 /* Optimizer update (phase U) restricted to the touched rows: for every r < *d_count and every scalar theta of
  * primitive d_idx[r] with gradient g: m = b1 m + (1-b1) g; v = b2 v + (1-b2) g^2;

@@ -27,7 +27,7 @@ EXPORTS = [
     "odin_create", "odin_destroy", "odin_status_string", "odin_poll", "odin_workspace_bytes", "odin_project",
     "odin_touched_set", "odin_bin_sort", "odin_render_fwd", "odin_l1_loss", "odin_render_bwd", "odin_sparse_adam",
     "odin_conflict_count", "odin_kernel_count", "odin_kernel_name", "odin_profile_enable", "odin_profile_collect",
-    "odin_touched_set_static",
+    "odin_touched_set_static", "odin_render_workspace_bytes",
 ]
 
 
@@ -84,10 +84,12 @@ def lib() -> C.CDLL:
                                    C.c_size_t, vp]
         L.odin_touched_set.argtypes = [vp, vp, u32, vp, vp, u32, vp, vp, C.c_size_t, vp]
         L.odin_bin_sort.argtypes = [vp, C.POINTER(odin_projected), i32, i32, vp, vp, u64, vp, vp, C.c_size_t, vp]
-        L.odin_render_fwd.argtypes = [vp, C.POINTER(odin_projected), vp, vp, C.POINTER(odin_camera), vp, vp, vp, vp]
+        L.odin_render_workspace_bytes.argtypes = [vp, i32, i32, C.POINTER(C.c_size_t)]
+        L.odin_render_fwd.argtypes = [vp, C.POINTER(odin_projected), vp, vp, C.POINTER(odin_camera), vp, vp, vp, vp,
+                                      C.c_size_t, vp]
         L.odin_l1_loss.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
         L.odin_render_bwd.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_camera), C.POINTER(odin_projected), vp, vp,
-                                      vp, vp, vp, vp, C.POINTER(odin_scene), vp]
+                                      vp, vp, vp, vp, C.POINTER(odin_scene), vp, C.c_size_t, vp]
         L.odin_sparse_adam.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_scene), C.POINTER(odin_scene),
                                        C.POINTER(odin_scene), vp, vp, C.POINTER(f32), f32, f32, f32, u32, vp]
         L.odin_conflict_count.argtypes = [vp, vp, u32, u32, u32, vp, u32, vp, vp]
@@ -199,9 +201,16 @@ def odin_bin_sort(ctx, proj: odin_projected, width: int, height: int, d_keys, d_
 
 
 def odin_render_fwd(ctx, proj: odin_projected, d_vals, d_tile_ranges, cam: odin_camera, d_rgb, d_final_T, d_n_contrib,
-                    stream=None) -> None:
+                    ws, stream=None) -> None:
     _check(lib().odin_render_fwd(ctx, C.byref(proj), _ptr(d_vals), _ptr(d_tile_ranges), C.byref(cam), _ptr(d_rgb),
-                                 _ptr(d_final_T), _ptr(d_n_contrib), _stream(stream)), "odin_render_fwd")
+                                 _ptr(d_final_T), _ptr(d_n_contrib), _ptr(ws),
+                                 0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)), "odin_render_fwd")
+
+
+def odin_render_workspace_bytes(ctx, width: int, height: int) -> int:
+    b = C.c_size_t(0)
+    _check(lib().odin_render_workspace_bytes(ctx, int(width), int(height), C.byref(b)), "odin_render_workspace_bytes")
+    return int(b.value)
 
 
 def odin_l1_loss(ctx, d_rgb, d_target, width: int, height: int, d_loss, d_dL_drgb, stream=None) -> None:
@@ -210,10 +219,11 @@ def odin_l1_loss(ctx, d_rgb, d_target, width: int, height: int, d_loss, d_dL_drg
 
 
 def odin_render_bwd(ctx, scene: odin_scene, cam: odin_camera, proj: odin_projected, d_vals, d_tile_ranges, d_final_T,
-                    d_n_contrib, d_dL_drgb, d_grad2d, grad_rows: odin_scene, stream=None) -> None:
+                    d_n_contrib, d_dL_drgb, d_grad2d, grad_rows: odin_scene, ws, stream=None) -> None:
     _check(lib().odin_render_bwd(ctx, C.byref(scene), C.byref(cam), C.byref(proj), _ptr(d_vals), _ptr(d_tile_ranges),
                                  _ptr(d_final_T), _ptr(d_n_contrib), _ptr(d_dL_drgb), _ptr(d_grad2d), C.byref(grad_rows),
-                                 _stream(stream)), "odin_render_bwd")
+                                 _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "odin_render_bwd")
 
 
 def odin_sparse_adam(ctx, params: odin_scene, m: odin_scene, v: odin_scene, grad_rows: odin_scene, d_idx, d_count,

@@ -70,7 +70,7 @@ extern "C" int odin_poll(odin_ctx* ctx, void* stream) {
 
 static const char* const kKernelNames[K_COUNT] = {
     "project", "touched_set", "emit_instances", "digit_base", "onesweep_pass", "tile_ranges", "render_fwd", "l1_loss",
-    "l1_finish", "zero_rows", "render_bwd_blend", "render_bwd_project", "adam_sh", "adam_geom", "conflict_count"};
+    "l1_finish", "zero_rows", "render_bwd_blend", "render_bwd_project", "adam_sh", "adam_geom", "conflict_count", "render_fwd_tail", "render_bwd_tail"};
 
 extern "C" int odin_kernel_count(void) { return K_COUNT; }
 

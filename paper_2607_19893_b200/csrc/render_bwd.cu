@@ -1,11 +1,10 @@
-// Backward phase: (a) per-tile back-to-front replay of the compositing with warp-transposed reductions of the nine
-// per-row gradient words, block-level accumulation in shared memory and one global atomic per (tile, row, word);
+// Backward phase: (a) per-tile back-to-front replay of the compositing, one warp per tile, per-lane accumulation over
+// eight pixels, one transposing warp reduction and one global atomic per (tile, row, word);
 // (b) per-row chain rule through the projection into compact gradient rows.
+#include "blend.cuh"
 #include "geom.cuh"
 
 namespace {
-
-constexpr int BB = 256;  // threads per block = pixels per tile = rows per batch
 
 __global__ void zero_rows_kernel(float* __restrict__ g2d, const uint32_t* __restrict__ num_rows, uint32_t capacity) {
   const uint32_t V = min(*num_rows, capacity);
@@ -31,16 +30,20 @@ __device__ __forceinline__ float warp_transpose_sum8(float a0, float a1, float a
   return d;
 }
 
-__global__ void __launch_bounds__(BB)
-render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
-                        const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
-                        float bg0, float bg1, float bg2, float alpha_min, float alpha_max,
-                        const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
-                        const float* __restrict__ dL, float* __restrict__ g2d) {
-  __shared__ float2 s_xy[BB];
-  __shared__ float4 s_co[BB];
-  __shared__ float s_rgb[BB][3];
-  __shared__ uint32_t s_row[BB];
+// Tail of long lists (runs first): tiles in which some pixel used more than BLEND_HEAD entries get a block of 256
+// threads, one pixel per thread, that walks entries [BLEND_HEAD, total) back to front, 256 at a time, reduces the
+// nine words over each warp and over the block in shared memory, issues one global atomic per (tile, row, word) and
+// leaves every pixel's transmittance and suffix colour in `state` for the head kernel.
+__global__ void __launch_bounds__(BLEND_TAIL_THREADS)
+render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
+                       const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
+                       float bg0, float bg1, float bg2, float alpha_min, float alpha_max,
+                       const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
+                       const float* __restrict__ dL, float* __restrict__ g2d, float* __restrict__ state) {
+  constexpr int BB = BLEND_TAIL_THREADS;
+  __shared__ BlendRow s_rowdata[BB];
+  __shared__ float s_blue[BB];
+  __shared__ uint32_t s_rowid[BB];
   __shared__ float s_acc[BB * 9];
   __shared__ uint32_t s_max;
   const int tile = blockIdx.x;
@@ -49,7 +52,9 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
   const int px = tx * 16 + lx, py = ty * 16 + ly;
   const bool inside = px < W && py < H;
   const unsigned lane = threadIdx.x & 31;
-  const float fx = (float)px + 0.5f, fy = (float)py + 0.5f;
+  const float fx = (float)px + 0.5f;
+  const float fy0 = (float)(ty * 16 + (ly & 1)) + 0.5f;
+  const float slot2 = (float)(2 * (ly >> 1));
   const uint32_t start = ranges[tile].x;
   const size_t pix = (size_t)py * W + px, plane = (size_t)W * H;
   float T = 1.f, g0 = 0.f, g1 = 0.f, g2 = 0.f;
@@ -60,7 +65,6 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
     g0 = dL[pix]; g1 = dL[plane + pix]; g2 = dL[2 * plane + pix];
   }
   if (threadIdx.x == 0) s_max = 0;
-  for (int i = threadIdx.x; i < BB * 9; i += BB) s_acc[i] = 0.f;
   __syncthreads();
   {
     uint32_t m = last;
@@ -68,50 +72,57 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
     if (lane == 0 && m) atomicMax(&s_max, m);
   }
   __syncthreads();
-  const uint32_t total = s_max;  // list entries any pixel of the tile used
+  const uint32_t total = s_max;
+  if (total <= BLEND_HEAD) return;  // uniform over the block: the head kernel does the whole tile
+  for (int i = threadIdx.x; i < BB * 9; i += BB) s_acc[i] = 0.f;
   float S0 = T * bg0, S1 = T * bg1, S2 = T * bg2;
-  const int nb = (int)((total + BB - 1) / BB);
+  const uint32_t span = total - BLEND_HEAD;
+  const int nb = (int)((span + BB - 1) / BB);
   for (int bi = nb - 1; bi >= 0; --bi) {
-    const uint32_t b = (uint32_t)bi * BB;
+    const uint32_t b = BLEND_HEAD + (uint32_t)bi * BB;
     const int cnt = (int)min((uint32_t)BB, total - b);
+    __syncthreads();
     if ((int)threadIdx.x < cnt) {
       const uint32_t r = vals[start + b + threadIdx.x];
-      s_row[threadIdx.x] = r;
-      s_xy[threadIdx.x] = xy[r];
-      s_co[threadIdx.x] = conic_o[r];
-      s_rgb[threadIdx.x][0] = rgb[3 * (size_t)r];
-      s_rgb[threadIdx.x][1] = rgb[3 * (size_t)r + 1];
-      s_rgb[threadIdx.x][2] = rgb[3 * (size_t)r + 2];
+      const float2 c = xy[r];
+      BlendRow row;
+      row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
+      row.q1 = conic_o[r];
+      s_rowdata[threadIdx.x] = row;
+      s_blue[threadIdx.x] = rgb[3 * (size_t)r + 2];
+      s_rowid[threadIdx.x] = r;
     }
     __syncthreads();
     for (int j = cnt - 1; j >= 0; --j) {
-      const float2 c = s_xy[j];
-      const float4 co = s_co[j];
-      const float dx = c.x - fx, dy = c.y - fy;
-      const float power = -0.5f * (co.x * dx * dx + co.z * dy * dy) - co.y * dx * dy;
+      const float4 q0 = s_rowdata[j].q0, q1 = s_rowdata[j].q1;
+      const float dx = q0.x - fx;
+      const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
+      const float dy = (q0.y - fy0) - slot2;
+      const float power = blend_power(h0, h1, h2, dy);
       const float G = __expf(power);
-      const float og = co.w * G;
+      const float og = q1.w * G;
       const float alpha = fminf(alpha_max, og);
       const bool on = (b + j < last) && (power <= 0.f) && (alpha >= alpha_min);
       if (__ballot_sync(0xffffffffu, on) == 0) continue;
       float vu = 0.f, vv = 0.f, vA = 0.f, vB = 0.f, vC = 0.f, vo = 0.f, vr = 0.f, vg = 0.f, vb = 0.f;
       if (on) {
-        const float inv = 1.f / (1.f - alpha);
+        const float inv = __fdividef(1.f, 1.f - alpha);
         const float Tb = T * inv;  // transmittance in front of this row
         const float w = alpha * Tb;
-        const float c0 = s_rgb[j][0], c1 = s_rgb[j][1], c2 = s_rgb[j][2];
+        const float c0 = q0.z, c1 = q0.w, c2 = s_blue[j];
         vr = w * g0; vg = w * g1; vb = w * g2;
         const float dLda = (c0 * Tb - S0 * inv) * g0 + (c1 * Tb - S1 * inv) * g1 + (c2 * Tb - S2 * inv) * g2;
-        S0 += c0 * w; S1 += c1 * w; S2 += c2 * w;
+        S0 = fmaf(c0, w, S0); S1 = fmaf(c1, w, S1); S2 = fmaf(c2, w, S2);
         T = Tb;
         if (og <= alpha_max) {
-          const float gp = G * co.w * dLda;
-          vu = (-co.x * dx - co.y * dy) * gp;
-          vv = (-co.z * dy - co.y * dx) * gp;
+          const float t = G * dLda;
+          const float gp = q1.w * t;
+          vu = -(q1.x * dx + q1.y * dy) * gp;
+          vv = -(q1.z * dy + q1.y * dx) * gp;
           vA = -0.5f * dx * dx * gp;
           vB = -dx * dy * gp;
           vC = -0.5f * dy * dy * gp;
-          vo = G * dLda;
+          vo = t;
         }
       }
       const float t8 = warp_transpose_sum8(vu, vv, vA, vB, vC, vo, vr, vg, lane);
@@ -123,11 +134,140 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
     for (int i = threadIdx.x; i < cnt * 9; i += BB) {
       const float v = s_acc[i];
       if (v != 0.f) {
-        atomicAdd(&g2d[(size_t)s_row[i / 9] * 9 + (i % 9)], v);
+        atomicAdd(&g2d[(size_t)s_rowid[i / 9] * 9 + (i % 9)], v);
         s_acc[i] = 0.f;
       }
     }
-    __syncthreads();
+  }
+  if (inside) {
+    state[pix] = T; state[plane + pix] = S0; state[2 * plane + pix] = S1; state[3 * plane + pix] = S2;
+  }
+}
+
+// One warp per tile, eight pixels per lane (blend.cuh).  For every row of the list the lane accumulates, over its own
+// pixels, the colour and opacity gradients and three moments of dL/dpower (sum, sum*dy, sum*dy^2); dx is constant per
+// lane, so the conic / centre gradients follow from the moments with a handful of operations per row instead of per
+// pixel.  One transposing warp reduction and nine global atomics per (tile, row) that contributed.
+__global__ void __launch_bounds__(BLEND_THREADS)
+render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
+                        const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
+                        int n_tiles, float bg0, float bg1, float bg2, float alpha_min, float alpha_max,
+                        const float* __restrict__ state,
+                        const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
+                        const float* __restrict__ dL, float* __restrict__ g2d) {
+  __shared__ BlendRow s_rowdata[BLEND_WARPS][32];
+  __shared__ float s_blue[BLEND_WARPS][32];
+  __shared__ uint32_t s_rowid[BLEND_WARPS][32];
+  const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int tile = blockIdx.x * BLEND_WARPS + warp;
+  if (tile >= n_tiles) return;  // warps never synchronise with each other
+  const int tx = tile % TX, ty = tile / TX;
+  const int px = tx * 16 + (int)(lane & 15);
+  const int py0 = ty * 16 + (int)(lane >> 4);
+  const float fx = (float)px + 0.5f, fy0 = (float)py0 + 0.5f;
+  const uint32_t start = ranges[tile].x;
+  const size_t plane = (size_t)W * H;
+
+  float T[BLEND_SLOTS], S0[BLEND_SLOTS], S1[BLEND_SLOTS], S2[BLEND_SLOTS];
+  float g0[BLEND_SLOTS], g1[BLEND_SLOTS], g2[BLEND_SLOTS];
+  uint32_t last[BLEND_SLOTS];
+  uint32_t total = 0;
+#pragma unroll
+  for (int s = 0; s < BLEND_SLOTS; ++s) {
+    const int py = py0 + 2 * s;
+    T[s] = 1.f; g0[s] = g1[s] = g2[s] = 0.f; last[s] = 0;
+    if (px < W && py < H) {
+      const size_t pix = (size_t)py * W + px;
+      T[s] = final_T[pix];
+      last[s] = n_contrib[pix];
+      g0[s] = dL[pix]; g1[s] = dL[plane + pix]; g2[s] = dL[2 * plane + pix];
+    }
+    S0[s] = T[s] * bg0; S1[s] = T[s] * bg1; S2[s] = T[s] * bg2;
+    total = max(total, last[s]);
+  }
+  for (int o = 16; o > 0; o >>= 1) total = max(total, __shfl_xor_sync(0xffffffffu, total, o));
+  // `total` = list entries any pixel of the tile used.  Entries beyond BLEND_HEAD were already walked by the tail
+  // kernel, which left every pixel's transmittance and suffix colour in the workspace.
+  if (total > BLEND_HEAD) {
+    total = BLEND_HEAD;
+#pragma unroll
+    for (int s = 0; s < BLEND_SLOTS; ++s) {
+      const int py = py0 + 2 * s;
+      if (px < W && py < H) {
+        const size_t pix = (size_t)py * W + px;
+        T[s] = state[pix]; S0[s] = state[plane + pix]; S1[s] = state[2 * plane + pix]; S2[s] = state[3 * plane + pix];
+      }
+    }
+  }
+  // walk the remaining entries back to front, 32 at a time
+  const int nb = (int)((total + 31) / 32);
+  for (int bi = nb - 1; bi >= 0; --bi) {
+    const uint32_t b = (uint32_t)bi * 32;
+    const int cnt = (int)min(32u, total - b);
+    if ((int)lane < cnt) {
+      const uint32_t r = vals[start + b + lane];
+      const float2 c = xy[r];
+      BlendRow row;
+      row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
+      row.q1 = conic_o[r];
+      s_rowdata[warp][lane] = row;
+      s_blue[warp][lane] = rgb[3 * (size_t)r + 2];
+      s_rowid[warp][lane] = r;
+    }
+    __syncwarp();
+    for (int j = cnt - 1; j >= 0; --j) {
+      const float4 q0 = s_rowdata[warp][j].q0, q1 = s_rowdata[warp][j].q1;
+      const float blue = s_blue[warp][j];
+      const float dx = q0.x - fx;
+      const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
+      const float dy0 = q0.y - fy0;
+      const uint32_t k = b + j;
+      // per-lane sums over its eight pixels; the x-dependent factors are applied once at the end
+      float ar = 0.f, ag = 0.f, ab = 0.f, ao = 0.f, gpsum = 0.f, m1y = 0.f, m2yy = 0.f;
+      bool any = false;
+#pragma unroll
+      for (int s = 0; s < BLEND_SLOTS; ++s) {
+        const float dy = dy0 - (float)(2 * s);
+        const float power = blend_power(h0, h1, h2, dy);
+        const float G = __expf(power);
+        const float og = q1.w * G;
+        const float alpha = fminf(alpha_max, og);
+        const bool on = (k < last[s]) && (power <= 0.f) && (alpha >= alpha_min);
+        if (__any_sync(0xffffffffu, on)) {
+          any = true;
+          if (on) {
+            const float inv = __fdividef(1.f, 1.f - alpha);
+            const float Tb = T[s] * inv;  // transmittance in front of this row
+            const float w = alpha * Tb;
+            ar = fmaf(w, g0[s], ar); ag = fmaf(w, g1[s], ag); ab = fmaf(w, g2[s], ab);
+            const float dLda = (q0.z * Tb - S0[s] * inv) * g0[s] + (q0.w * Tb - S1[s] * inv) * g1[s] +
+                               (blue * Tb - S2[s] * inv) * g2[s];
+            S0[s] = fmaf(q0.z, w, S0[s]); S1[s] = fmaf(q0.w, w, S1[s]); S2[s] = fmaf(blue, w, S2[s]);
+            T[s] = Tb;
+            if (og <= alpha_max) {  // a clamped alpha passes no gradient to opacity or geometry
+              const float t = G * dLda;
+              ao += t;
+              const float gp = q1.w * t;  // dL/dpower
+              gpsum += gp;
+              const float gy = gp * dy;
+              m1y += gy;
+              m2yy = fmaf(gy, dy, m2yy);
+            }
+          }
+        }
+      }
+      if (!any) continue;  // warp-uniform: `any` was set from warp votes
+      const float gd = dx * gpsum;  // sum of dL/dpower * dx
+      const float vu = -(q1.x * gd + q1.y * m1y);
+      const float vv = -(q1.z * m1y + q1.y * gd);
+      const float vA = -0.5f * dx * gd, vB = -dx * m1y, vC = -0.5f * m2yy;
+      const float t8 = warp_transpose_sum8(vu, vv, vA, vB, vC, ao, ar, ag, lane);
+      for (int o = 16; o > 0; o >>= 1) ab += __shfl_xor_sync(0xffffffffu, ab, o);
+      float* dst = g2d + (size_t)s_rowid[warp][j] * 9;
+      if ((lane & 3) == 0) atomicAdd(dst + (lane >> 2), t8);
+      if (lane == 1) atomicAdd(dst + 8, ab);
+    }
+    __syncwarp();
   }
 }
 
@@ -252,7 +392,7 @@ render_bwd_project_kernel(const float* __restrict__ means, const float* __restri
 extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odin_camera* cam, const odin_projected* proj,
                                const uint32_t* d_vals, const uint32_t* d_tile_ranges, const float* d_final_T,
                                const uint32_t* d_n_contrib, const float* d_dL_drgb, float* d_grad2d, odin_scene* grad_rows,
-                               void* stream) {
+                               void* ws, size_t ws_bytes, void* stream) {
   if (!ctx || !proj || !grad_rows) return ODIN_ERR_NULL;
   int rc = odin_check_scene(scene);
   if (rc != ODIN_OK) return rc;
@@ -268,17 +408,27 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
     return ODIN_ERR_NULL;
   cudaStream_t st = (cudaStream_t)stream;
   const int TX = (cam->width + 15) / 16, TY = (cam->height + 15) / 16;
+  if (!ws || !odin_aligned(ws, 256) || ws_bytes < blend_ws_bytes(cam->width, cam->height)) return ODIN_ERR_WORKSPACE;
   const uint32_t zgrid = (uint32_t)ctx->sm_count * 8;
   {
     OdinKernelScope ks(ctx, K_ZERO_ROWS, st);
     zero_rows_kernel<<<zgrid, 256, 0, st>>>(d_grad2d, proj->num_rows, proj->capacity);
   }
+  const int n_tiles = TX * TY;
+  float* state = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + blend_ws_flags_bytes(n_tiles));
   {
-    OdinKernelScope ks(ctx, K_BWD_BLEND, st);
-    render_bwd_blend_kernel<<<TX * TY, BB, 0, st>>>(
+    OdinKernelScope ks(ctx, K_BWD_TAIL, st);
+    render_bwd_tail_kernel<<<n_tiles, BLEND_TAIL_THREADS, 0, st>>>(
         reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
         reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
-        ctx->cfg.alpha_min, ctx->cfg.alpha_max, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d);
+        ctx->cfg.alpha_min, ctx->cfg.alpha_max, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d, state);
+  }
+  {
+    OdinKernelScope ks(ctx, K_BWD_BLEND, st);
+    render_bwd_blend_kernel<<<(n_tiles + BLEND_WARPS - 1) / BLEND_WARPS, BLEND_THREADS, 0, st>>>(
+        reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
+        reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0], cam->bg[1],
+        cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, state, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d);
   }
   const CamParams cp = odin_cam_params(cam, ctx->cfg);
   const uint32_t blocks_cap = (proj->capacity + 127) / 128;

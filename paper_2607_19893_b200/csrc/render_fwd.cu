@@ -1,63 +1,166 @@
-// Rendering phase: front-to-back alpha compositing, one 16x16 block per tile, the tile's sorted rows staged through
-// shared memory in batches of 256, early exit once every pixel of the tile has terminated.  Also the L1 image loss.
-#include "common.cuh"
+// Rendering phase: front-to-back alpha compositing.  Head kernel: one WARP per 16x16 tile, eight pixels per lane (see
+// blend.cuh), the tile's sorted rows staged 32 at a time through shared memory, warp-ballot early exit once every
+// pixel of the tile has terminated; per row and lane the x-dependent terms are computed once, each pixel costs two
+// fused multiply-adds, one ex2 and the blend.  Tiles still live after BLEND_HEAD entries are finished by the tail
+// kernel (eight warps per tile, rows staged 256 at a time).  Also the L1 image loss.
+#include "blend.cuh"
 
 namespace {
 
-constexpr int FB = 256;  // threads per block = pixels per tile = rows per batch
-
-__global__ void __launch_bounds__(FB)
+__global__ void __launch_bounds__(BLEND_THREADS)
 render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
-                  const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX, float bg0,
-                  float bg1, float bg2, float alpha_min, float alpha_max, float t_min, float* __restrict__ out,
-                  float* __restrict__ final_T, uint32_t* __restrict__ n_contrib) {
-  __shared__ float2 s_xy[FB];
-  __shared__ float4 s_co[FB];
-  __shared__ float s_rgb[FB][3];
+                  const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX, int n_tiles,
+                  float bg0, float bg1, float bg2, float alpha_min, float alpha_max, float t_min, float* __restrict__ out,
+                  float* __restrict__ final_T, uint32_t* __restrict__ n_contrib, uint32_t* __restrict__ tile_more) {
+  __shared__ BlendRow s_row[BLEND_WARPS][32];
+  __shared__ float s_blue[BLEND_WARPS][32];
+  const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int tile = blockIdx.x * BLEND_WARPS + warp;
+  if (tile >= n_tiles) return;  // warps never synchronise with each other
+  const int tx = tile % TX, ty = tile / TX;
+  const int px = tx * 16 + (int)(lane & 15);
+  const int py0 = ty * 16 + (int)(lane >> 4);
+  const float fx = (float)px + 0.5f, fy0 = (float)py0 + 0.5f;
+  const uint2 rg = ranges[tile];
+  const uint32_t start = rg.x;
+  const uint32_t end = min(rg.y, rg.x + BLEND_HEAD);
+
+  float T[BLEND_SLOTS], C0[BLEND_SLOTS], C1[BLEND_SLOTS], C2[BLEND_SLOTS];
+  uint32_t last[BLEND_SLOTS];
+  uint32_t live = 0;  // bit s: pixel of slot s still accumulating
+#pragma unroll
+  for (int s = 0; s < BLEND_SLOTS; ++s) {
+    T[s] = 1.f; C0[s] = C1[s] = C2[s] = 0.f; last[s] = 0;
+    if (px < W && py0 + 2 * s < H) live |= 1u << s;
+  }
+  const uint32_t inside = live;
+
+  for (uint32_t b = start; b < end; b += 32) {
+    if (!__any_sync(0xffffffffu, live != 0)) break;
+    const uint32_t i = b + lane;
+    if (i < end) {
+      const uint32_t r = vals[i];
+      const float2 c = xy[r];
+      BlendRow row;
+      row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
+      row.q1 = conic_o[r];
+      s_row[warp][lane] = row;
+      s_blue[warp][lane] = rgb[3 * (size_t)r + 2];
+    }
+    __syncwarp();
+    const int cnt = (int)min(32u, end - b);
+    for (int j = 0; j < cnt; ++j) {
+      const float4 q0 = s_row[warp][j].q0, q1 = s_row[warp][j].q1;
+      const float blue = s_blue[warp][j];
+      const float dx = q0.x - fx;
+      const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
+      const float dy0 = q0.y - fy0;
+      const uint32_t ord = (b - start) + j + 1;
+#pragma unroll
+      for (int s = 0; s < BLEND_SLOTS; ++s) {
+        const float dy = dy0 - (float)(2 * s);
+        const float power = blend_power(h0, h1, h2, dy);
+        const float alpha = fminf(alpha_max, q1.w * __expf(power));
+        if ((live >> s & 1u) && power <= 0.f && alpha >= alpha_min) {
+          const float Tn = T[s] * (1.f - alpha);
+          if (Tn < t_min) {
+            live &= ~(1u << s);
+          } else {
+            const float w = alpha * T[s];
+            C0[s] = fmaf(q0.z, w, C0[s]); C1[s] = fmaf(q0.w, w, C1[s]); C2[s] = fmaf(blue, w, C2[s]);
+            T[s] = Tn;
+            last[s] = ord;
+          }
+        }
+      }
+    }
+    __syncwarp();
+  }
+  // the tail kernel takes over when entries remain and some pixel is still live
+  const bool more = (rg.y > end) && __any_sync(0xffffffffu, live != 0);
+  if (lane == 0) tile_more[tile] = more ? 1u : 0u;
+  const size_t plane = (size_t)W * H;
+#pragma unroll
+  for (int s = 0; s < BLEND_SLOTS; ++s) {
+    const int py = py0 + 2 * s;
+    if (inside >> s & 1u) {
+      const size_t pix = (size_t)py * W + px;
+      const float tb = more ? 0.f : T[s];  // the background is added by whoever finishes the pixel
+      out[pix] = C0[s] + tb * bg0;
+      out[plane + pix] = C1[s] + tb * bg1;
+      out[2 * plane + pix] = C2[s] + tb * bg2;
+      final_T[pix] = T[s];
+      n_contrib[pix] = last[s] | ((more && !(live >> s & 1u)) ? BLEND_DONE_BIT : 0u);
+    }
+  }
+}
+
+// Tail: one block of 256 threads per tile that the head kernel left unfinished, one pixel per thread, rows staged 256
+// at a time.  Thread t handles column t % 16 and row t / 16 = 2 s + (row inside the slot pair), as in the head kernel.
+__global__ void __launch_bounds__(BLEND_TAIL_THREADS)
+render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
+                       const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
+                       float bg0, float bg1, float bg2, float alpha_min, float alpha_max, float t_min,
+                       float* __restrict__ out, float* __restrict__ final_T, uint32_t* __restrict__ n_contrib,
+                       const uint32_t* __restrict__ tile_more) {
   const int tile = blockIdx.x;
+  if (!tile_more[tile]) return;
+  __shared__ BlendRow s_row[BLEND_TAIL_THREADS];
+  __shared__ float s_blue[BLEND_TAIL_THREADS];
   const int tx = tile % TX, ty = tile / TX;
   const int lx = threadIdx.x & 15, ly = threadIdx.x >> 4;
   const int px = tx * 16 + lx, py = ty * 16 + ly;
   const bool inside = px < W && py < H;
-  const float fx = (float)px + 0.5f, fy = (float)py + 0.5f;
+  const float fx = (float)px + 0.5f;
+  const float fy0 = (float)(ty * 16 + (ly & 1)) + 0.5f;
+  const float slot2 = (float)(2 * (ly >> 1));
   const uint2 rg = ranges[tile];
   const uint32_t start = rg.x, end = rg.y;
+  const size_t pix = (size_t)py * W + px, plane = (size_t)W * H;
   float T = 1.f, C0 = 0.f, C1 = 0.f, C2 = 0.f;
   uint32_t last = 0;
-  bool done = !inside;
-  for (uint32_t b = start; b < end; b += FB) {
-    if (__syncthreads_count(done) == FB) break;
+  bool done = true;
+  if (inside) {
+    T = final_T[pix];
+    C0 = out[pix]; C1 = out[plane + pix]; C2 = out[2 * plane + pix];
+    const uint32_t nc = n_contrib[pix];
+    last = nc & ~BLEND_DONE_BIT;
+    done = (nc & BLEND_DONE_BIT) != 0;
+  }
+  for (uint32_t b = start + BLEND_HEAD; b < end; b += BLEND_TAIL_THREADS) {
+    if (__syncthreads_count(done) == BLEND_TAIL_THREADS) break;
     const uint32_t i = b + threadIdx.x;
     if (i < end) {
       const uint32_t r = vals[i];
-      s_xy[threadIdx.x] = xy[r];
-      s_co[threadIdx.x] = conic_o[r];
-      s_rgb[threadIdx.x][0] = rgb[3 * (size_t)r];
-      s_rgb[threadIdx.x][1] = rgb[3 * (size_t)r + 1];
-      s_rgb[threadIdx.x][2] = rgb[3 * (size_t)r + 2];
+      const float2 c = xy[r];
+      BlendRow row;
+      row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
+      row.q1 = conic_o[r];
+      s_row[threadIdx.x] = row;
+      s_blue[threadIdx.x] = rgb[3 * (size_t)r + 2];
     }
     __syncthreads();
-    const int cnt = (int)min((uint32_t)FB, end - b);
+    const int cnt = (int)min((uint32_t)BLEND_TAIL_THREADS, end - b);
     if (!done) {
       for (int j = 0; j < cnt; ++j) {
-        const float2 c = s_xy[j];
-        const float4 co = s_co[j];
-        const float dx = c.x - fx, dy = c.y - fy;
-        const float power = -0.5f * (co.x * dx * dx + co.z * dy * dy) - co.y * dx * dy;
+        const float4 q0 = s_row[j].q0, q1 = s_row[j].q1;
+        const float dx = q0.x - fx;
+        const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
+        const float dy = (q0.y - fy0) - slot2;
+        const float power = blend_power(h0, h1, h2, dy);
         if (power > 0.f) continue;
-        const float alpha = fminf(alpha_max, co.w * __expf(power));
+        const float alpha = fminf(alpha_max, q1.w * __expf(power));
         if (alpha < alpha_min) continue;
         const float Tn = T * (1.f - alpha);
         if (Tn < t_min) { done = true; break; }
         const float w = alpha * T;
-        C0 += s_rgb[j][0] * w; C1 += s_rgb[j][1] * w; C2 += s_rgb[j][2] * w;
+        C0 = fmaf(q0.z, w, C0); C1 = fmaf(q0.w, w, C1); C2 = fmaf(s_blue[j], w, C2);
         T = Tn;
         last = (b - start) + j + 1;
       }
     }
   }
   if (inside) {
-    const size_t pix = (size_t)py * W + px, plane = (size_t)W * H;
     out[pix] = C0 + T * bg0;
     out[plane + pix] = C1 + T * bg1;
     out[2 * plane + pix] = C2 + T * bg2;
@@ -92,9 +195,16 @@ __global__ void l1_finish_kernel(const double* acc, double inv, float* loss) { *
 
 }  // namespace
 
+extern "C" int odin_render_workspace_bytes(const odin_ctx* ctx, int width, int height, size_t* bytes) {
+  if (!ctx || !bytes) return ODIN_ERR_NULL;
+  if (width <= 0 || height <= 0 || width > 16384 || height > 16384) return ODIN_ERR_INVALID_ARG;
+  *bytes = blend_ws_bytes(width, height);
+  return ODIN_OK;
+}
+
 extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const uint32_t* d_vals,
                                const uint32_t* d_tile_ranges, const odin_camera* cam, float* d_rgb, float* d_final_T,
-                               uint32_t* d_n_contrib, void* stream) {
+                               uint32_t* d_n_contrib, void* ws, size_t ws_bytes, void* stream) {
   if (!ctx || !proj || !d_tile_ranges || !d_rgb || !d_final_T || !d_n_contrib) return ODIN_ERR_NULL;
   const int rc = odin_check_camera(cam);
   if (rc != ODIN_OK) return rc;
@@ -102,11 +212,22 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
   if (!odin_aligned(proj->xy, 8) || !odin_aligned(proj->conic_opacity, 16) || !odin_aligned(d_tile_ranges, 8))
     return ODIN_ERR_INVALID_ARG;
   const int TX = (cam->width + 15) / 16, TY = (cam->height + 15) / 16;
-  OdinKernelScope ks(ctx, K_FWD, (cudaStream_t)stream);
-  render_fwd_kernel<<<TX * TY, FB, 0, (cudaStream_t)stream>>>(
+  const int n_tiles = TX * TY;
+  if (!ws || !odin_aligned(ws, 256) || ws_bytes < blend_ws_flags_bytes(n_tiles)) return ODIN_ERR_WORKSPACE;
+  uint32_t* tile_more = reinterpret_cast<uint32_t*>(ws);
+  cudaStream_t st = (cudaStream_t)stream;
+  {
+    OdinKernelScope ks(ctx, K_FWD, st);
+    render_fwd_kernel<<<(n_tiles + BLEND_WARPS - 1) / BLEND_WARPS, BLEND_THREADS, 0, st>>>(
+        reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
+        reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0], cam->bg[1],
+        cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_more);
+  }
+  OdinKernelScope ks(ctx, K_FWD_TAIL, st);
+  render_fwd_tail_kernel<<<n_tiles, BLEND_TAIL_THREADS, 0, st>>>(
       reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
       reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
-      ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib);
+      ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_more);
   return odin_launch_status();
 }
 

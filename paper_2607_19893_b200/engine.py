@@ -119,7 +119,8 @@ class ViewTrainer:
         self.masks = z((self.mask_slots, max(self.mask_stride, 4)), torch.int32)
         self.idx = z(max(self.row_capacity, 1), torch.int32)
         self.count = z(1, torch.int32)
-        ws_bytes = B.odin_workspace_bytes(self.ctx, self.n, self.instance_capacity)
+        ws_bytes = max(B.odin_workspace_bytes(self.ctx, self.n, self.instance_capacity),
+                       B.odin_render_workspace_bytes(self.ctx, self.width, self.height))
         self.ws = z(ws_bytes, torch.uint8)
         self.kernel_launches_per_step = 0
 
@@ -142,14 +143,14 @@ class ViewTrainer:
 
     def render_fwd(self, cam: B.odin_camera, stream=None) -> None:
         B.odin_render_fwd(self.ctx, self.proj.struct, self.vals, self.ranges, cam, self.out, self.final_T, self.n_contrib,
-                          stream)
+                          self.ws, stream)
 
     def l1_loss(self, stream=None) -> None:
         B.odin_l1_loss(self.ctx, self.out, self.target, self.width, self.height, self.loss, self.dL, stream)
 
     def render_bwd(self, cam: B.odin_camera, stream=None) -> None:
         B.odin_render_bwd(self.ctx, self.params.struct, cam, self.proj.struct, self.vals, self.ranges, self.final_T,
-                          self.n_contrib, self.dL, self.grad2d, self.grads.struct, stream)
+                          self.n_contrib, self.dL, self.grad2d, self.grads.struct, self.ws, stream)
 
     def sparse_adam(self, lr, beta1, beta2, eps, step: int, stream=None) -> None:
         B.odin_sparse_adam(self.ctx, self.params.struct, self.m.struct, self.v.struct, self.grads.struct, self.idx,

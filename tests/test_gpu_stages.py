@@ -301,7 +301,7 @@ def load_sorted(tr, f, inv):
     tr.ranges.copy_(torch.from_numpy(f["ranges"].view(np.int32)).to(tr.device))
 
 
-def check_forward(oracle32, scene, cam):
+def check_forward(oracle32, scene, cam, min_robust=1 - 2e-3):
     f, inv = oracle_view(oracle32, scene, cam)
     tr = G.trainer_for(scene, cam, row_capacity=max(len(f["idx"]), 1), instance_capacity=len(f["vals"]) + 1)
     load_sorted(tr, f, inv)
@@ -312,7 +312,7 @@ def check_forward(oracle32, scene, cam):
     nc = G.u32(tr.n_contrib)
     # the device evaluates exp with ex2.approx (relative error ~1e-6): a threshold test within 2e-5 may flip
     robust = f["pix_margin"] > 2e-5
-    assert robust.mean() > 1 - 2e-3
+    assert robust.mean() > min_robust
     assert np.abs(out - f["out"])[:, robust].max() < PIX_TOL
     assert np.abs(ft - f["final_T"])[robust].max() < PIX_TOL
     assert np.array_equal(nc[robust], f["n_contrib"][robust])
@@ -362,10 +362,16 @@ def test_l1_loss(oracle32):
 
 
 # ------------------------------------------------------------------------------------------------ backward
-def check_backward(oracle32, scene, cam, seed=0):
+def check_backward(oracle32, scene, cam, seed=0, min_robust=1 - 2e-3):
     f, inv = oracle_view(oracle32, scene, cam)
     rng = np.random.default_rng(seed)
     dl = rng.uniform(-1, 1, f["out"].shape).astype(np.float32)
+    # The backward pass re-takes the skip decisions of every (pixel, row) pair.  On a pixel where one of them sits
+    # within float rounding of its threshold the two sides may replay a different set of rows, which is a different
+    # (equally valid) function: such pixels (a fraction < 2e-3) get no incoming gradient here.
+    robust = f["pix_margin"] > 2e-5
+    assert robust.mean() > min_robust
+    dl[:, ~robust] = 0
     g2d_o, g2d_abs = oracle32.render_bwd_blend(f["proj"], f["vals"], f["ranges"], cam, f["final_T"], f["n_contrib"], dl,
                                                want_abs=True)
     rows_o = oracle32.render_bwd_project(scene, cam, f["idx"], g2d_o, f["proj"].clamp_flags).astype(np.float64)
@@ -415,3 +421,39 @@ def test_render_bwd_ragged_image_other_degree(oracle32):
     s = w.scene
     s2 = wl.Scene(1, s.means, s.log_scales, s.quats, s.opacity_logit, np.ascontiguousarray(s.sh[:, :4]))
     check_backward(oracle32, s2, w.cameras[2], seed=5)
+
+
+# ------------------------------------------------------------------------------------------------ long lists
+def faint_scene(n=20_000, seed=9):
+    """Many faint splats on a small image: no pixel saturates, so every tile walks thousands of list entries and
+    both the one-warp head kernels and the eight-warp tail kernels are exercised."""
+    w = wl.make_workload(1, n=n)
+    s = w.scene.copy()
+    rng = np.random.default_rng(seed)
+    s.opacity_logit[:] = rng.uniform(-5.2, -3.5, n).astype(np.float32)
+    s.log_scales[:] = (-2.6 + 0.3 * rng.standard_normal((n, 3))).astype(np.float32)
+    cam = w.cameras[0]
+    cam.bg = np.array([0.4, 0.2, 0.6])
+    return s, cam
+
+
+def test_render_fwd_lists_longer_than_the_head(oracle32):
+    s, cam = faint_scene()
+    # thousands of pairs per pixel: proportionally more pixels have one pair near a threshold
+    f = check_forward(oracle32, s, cam, min_robust=0.98)
+    assert f["n_contrib"].max() > 1500 and (f["ranges"][:, 1] - f["ranges"][:, 0]).min() > 512
+
+
+def test_render_bwd_lists_longer_than_the_head(oracle32):
+    s, cam = faint_scene(n=12_000, seed=10)
+    check_backward(oracle32, s, cam, seed=11, min_robust=0.98)
+
+
+def test_render_fwd_mixed_short_and_long_lists(oracle32):
+    # half of the image crowded with faint splats (tail kernel), the other half nearly empty (head kernel only)
+    s, cam = faint_scene(n=16_000, seed=12)
+    s.means[:, 0] = np.abs(s.means[:, 0])
+    f = check_forward(oracle32, s, cam, min_robust=0.98)
+    lens = f["ranges"][:, 1] - f["ranges"][:, 0]
+    assert lens.min() < 512 < lens.max()
+    check_backward(oracle32, s, cam, seed=13, min_robust=0.98)
