@@ -3,7 +3,7 @@
 #include <stddef.h>
 #include <stdint.h>
 
-constexpr uint32_t PROJECT_TILE = 256;    // primitives per look-back tile of the projection kernel
+constexpr uint32_t PROJECT_TILE = 2048;   // primitives per look-back tile of the projection scan
 constexpr uint32_t TOUCHED_TILE = 2048;   // primitives per look-back tile of the touched-set kernel
 constexpr uint32_t SORT_TILE = 4096;      // keys per onesweep tile
 constexpr uint32_t SORT_RADIX_BITS = 8;

@@ -1,109 +1,168 @@
-// Preprocessing phase: cull, EWA projection, tile rectangle, SH colour; compaction of the visible rows and the
-// exclusive scan of their tile counts in the same pass (decoupled look-back over 256-primitive tiles).
+// Preprocessing phase in three streaming kernels:
+//   1. cull + count: every primitive -> number of tiles its rectangle covers (0 = culled); no synchronisation at all,
+//      the attributes beyond the mean are only loaded for primitives that pass the depth test;
+//   2. scan: single-pass decoupled look-back over the counts -> ascending list of visible primitives (the row map) and
+//      the exclusive prefix of their tile counts (instance offsets), totals V and M;
+//   3. rows: one thread per VISIBLE primitive recomputes the (deterministic) geometry and writes the compact record,
+//      evaluates the SH colour and the opacity.
+// At 2-30 % visibility recomputing the geometry of the visible rows is far cheaper than carrying per-primitive state
+// through a block-wide scan in the first kernel.
 #include "geom.cuh"
 #include "layout.cuh"
 
 namespace {
 
+struct Footprint {
+  float u, v, depth, cA, cB, cC;
+  int rad, x0, y0, x1, y1;
+  uint32_t tiles;
+};
+
+// Conic, radius and tile rectangle of one primitive.  Plain IEEE arithmetic (this file is compiled without fused
+// multiply-add contraction): the integer results must not depend on which kernel evaluates them.
+__device__ __forceinline__ Footprint project_footprint(const CamParams& cam, float dilation, float radius_sigmas,
+                                                      const float* __restrict__ means,
+                                                      const float* __restrict__ log_scales,
+                                                      const float4* __restrict__ quats, size_t p) {
+  Footprint f;
+  f.tiles = 0; f.u = f.v = f.depth = f.cA = f.cB = f.cC = 0.f; f.rad = f.x0 = f.y0 = f.x1 = f.y1 = 0;
+  SplatGeom g;
+  odin_camera_space(cam, means[3 * p], means[3 * p + 1], means[3 * p + 2], g.t);
+  if (!(g.t[2] > cam.znear && g.t[2] < cam.zfar)) return f;
+  const float ls[3] = {log_scales[3 * p], log_scales[3 * p + 1], log_scales[3 * p + 2]};
+  odin_splat_geometry(cam, dilation, ls, quats[p], g);
+  if (!(g.det > 0.f)) return f;
+  f.cA = g.c / g.det; f.cB = -g.b / g.det; f.cC = g.a / g.det;
+  const float mid = (g.a + g.c) / 2.f;
+  const float lam = mid + sqrtf(fmaxf(0.1f, mid * mid - g.det));
+  const float radf = ceilf(radius_sigmas * sqrtf(lam));
+  f.u = cam.fx * g.t[0] / g.t[2] + cam.cx;
+  f.v = cam.fy * g.t[1] / g.t[2] + cam.cy;
+  f.depth = g.t[2];
+  const float ftx = (float)cam.TX, fty = (float)cam.TY;
+  f.x0 = (int)fminf(ftx, fmaxf(0.f, floorf((f.u - radf) / 16.f)));
+  f.x1 = (int)fminf(ftx, fmaxf(0.f, ceilf((f.u + radf) / 16.f)));
+  f.y0 = (int)fminf(fty, fmaxf(0.f, floorf((f.v - radf) / 16.f)));
+  f.y1 = (int)fminf(fty, fmaxf(0.f, ceilf((f.v + radf) / 16.f)));
+  f.tiles = (uint32_t)(f.x1 - f.x0) * (uint32_t)(f.y1 - f.y0);
+  f.rad = (int)fminf(radf, 2.0e9f);
+  return f;
+}
+
+__global__ void __launch_bounds__(256)
+project_cull_kernel(const float* __restrict__ means, const float* __restrict__ log_scales, const float4* __restrict__ quats,
+                    uint32_t n, CamParams cam, float dilation, float radius_sigmas, uint32_t* __restrict__ tiles_touched) {
+  const uint32_t p = blockIdx.x * 256u + threadIdx.x;
+  if (p >= n) return;
+  tiles_touched[p] = project_footprint(cam, dilation, radius_sigmas, means, log_scales, quats, p).tiles;
+}
+
 // packed look-back value: rows in the upper 28 bits, tile instances in the lower 34 bits
 constexpr int PACK_SHIFT = 34;
 constexpr uint64_t PACK_LOW = (1ull << PACK_SHIFT) - 1;
+constexpr int SCAN_THREADS = 256;
+constexpr int SCAN_ITEMS = PROJECT_TILE / SCAN_THREADS;
 
-template <int DEG>
-__global__ void __launch_bounds__(PROJECT_TILE)
-project_kernel(const float* __restrict__ means, const float* __restrict__ log_scales, const float4* __restrict__ quats,
-               const float* __restrict__ opacity_logit, const float* __restrict__ sh, uint32_t n, CamParams cam,
-               float dilation, float radius_sigmas, odin_projected out, uint32_t* ticket, uint64_t* state, int* status) {
-  constexpr int K = (DEG + 1) * (DEG + 1);
+// Each warp owns 32 * SCAN_ITEMS consecutive primitives; load j of lane l is primitive warp_base + 32 j + l, so ranks
+// inside the warp follow the primitive order.  Row index and instance offset come from one 64-bit look-back.
+__global__ void __launch_bounds__(SCAN_THREADS)
+project_scan_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint32_t capacity,
+                    uint32_t* __restrict__ prim_id, uint32_t* __restrict__ tile_offset, uint32_t* __restrict__ num_rows,
+                    uint64_t* __restrict__ num_instances, uint32_t* ticket, uint64_t* state, int* status) {
   __shared__ uint32_t s_tile;
-  __shared__ uint32_t s_warp[33];
-  __shared__ uint32_t s_warp2[33];
+  __shared__ uint64_t s_warp[SCAN_THREADS / 32 + 1];
   __shared__ uint64_t s_base;
   if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
   __syncthreads();
   const uint32_t tile = s_tile;
-  const uint32_t p = tile * PROJECT_TILE + threadIdx.x;
-
-  uint32_t tiles = 0;
-  float u = 0.f, v = 0.f, depth = 0.f, cA = 0.f, cB = 0.f, cC = 0.f;
-  int rad = 0;
-  int x0 = 0, y0 = 0, x1 = 0, y1 = 0;
-  float mx = 0.f, my = 0.f, mz = 0.f;
-  if (p < n) {
-    mx = means[3 * (size_t)p]; my = means[3 * (size_t)p + 1]; mz = means[3 * (size_t)p + 2];
-    SplatGeom g;
-    odin_camera_space(cam, mx, my, mz, g.t);
-    if (g.t[2] > cam.znear && g.t[2] < cam.zfar) {
-      const float ls[3] = {log_scales[3 * (size_t)p], log_scales[3 * (size_t)p + 1], log_scales[3 * (size_t)p + 2]};
-      odin_splat_geometry(cam, dilation, ls, quats[p], g);
-      if (g.det > 0.f) {
-        cA = g.c / g.det; cB = -g.b / g.det; cC = g.a / g.det;
-        const float mid = (g.a + g.c) / 2.f;
-        const float lam = mid + sqrtf(fmaxf(0.1f, mid * mid - g.det));
-        const float radf = ceilf(radius_sigmas * sqrtf(lam));
-        u = cam.fx * g.t[0] / g.t[2] + cam.cx;
-        v = cam.fy * g.t[1] / g.t[2] + cam.cy;
-        depth = g.t[2];
-        const float ftx = (float)cam.TX, fty = (float)cam.TY;
-        x0 = (int)fminf(ftx, fmaxf(0.f, floorf((u - radf) / 16.f)));
-        x1 = (int)fminf(ftx, fmaxf(0.f, ceilf((u + radf) / 16.f)));
-        y0 = (int)fminf(fty, fmaxf(0.f, floorf((v - radf) / 16.f)));
-        y1 = (int)fminf(fty, fmaxf(0.f, ceilf((v + radf) / 16.f)));
-        tiles = (uint32_t)(x1 - x0) * (uint32_t)(y1 - y0);
-        rad = (int)fminf(radf, 2.0e9f);
+  const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t warp_base = tile * PROJECT_TILE + warp * (32 * SCAN_ITEMS);
+  uint32_t t[SCAN_ITEMS];
+#pragma unroll
+  for (int j = 0; j < SCAN_ITEMS; ++j) {
+    const uint32_t p = warp_base + 32 * j + lane;
+    t[j] = (p < n) ? tiles_touched[p] : 0u;
+  }
+  // per item: packed (1 row, t tiles) exclusive prefix inside the warp, in primitive order
+  uint64_t ex[SCAN_ITEMS];
+  uint64_t run = 0;
+#pragma unroll
+  for (int j = 0; j < SCAN_ITEMS; ++j) {
+    const uint64_t v = t[j] ? ((1ull << PACK_SHIFT) | (uint64_t)t[j]) : 0ull;
+    uint64_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint64_t y = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= (unsigned)o) inc += y;
+    }
+    ex[j] = run + inc - v;
+    run += __shfl_sync(0xffffffffu, inc, 31);
+  }
+  if (lane == 0) s_warp[warp] = run;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    uint64_t w = (lane < SCAN_THREADS / 32) ? s_warp[lane] : 0ull;
+    uint64_t inc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint64_t y = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= (unsigned)o) inc += y;
+    }
+    const uint64_t total = __shfl_sync(0xffffffffu, inc, 31);
+    if (lane < SCAN_THREADS / 32) s_warp[lane] = inc - w;
+    const uint64_t base = odin_lookback_u64(state, tile, total, status);
+    if (lane == 0) {
+      s_base = base;
+      if (tile == (n + PROJECT_TILE - 1) / PROJECT_TILE - 1) {  // last tile: totals
+        const uint64_t all = base + total;
+        const uint64_t rows = all >> PACK_SHIFT, inst = all & PACK_LOW;
+        *num_rows = (uint32_t)(rows < capacity ? rows : capacity);
+        *num_instances = inst;
+        if (rows > capacity || inst >= (1ull << 32)) odin_set_error(status, ODIN_ERR_CAPACITY);
       }
     }
-    out.tiles_touched[p] = tiles;
-  }
-
-  // block scan of (visible, tiles) and look-back for the global row / instance offsets
-  uint32_t total_rows, total_tiles;
-  const uint32_t vis = tiles > 0 ? 1u : 0u;
-  const uint32_t row_local = odin_block_exclusive_sum(vis, s_warp, &total_rows);
-  // images are limited to 16384^2 pixels = 2^20 tiles, so 256 rectangles sum to < 2^32
-  const uint32_t off_local = odin_block_exclusive_sum(tiles, s_warp2, &total_tiles);
-  if (threadIdx.x < 32) {
-    const uint64_t agg = ((uint64_t)total_rows << PACK_SHIFT) | (uint64_t)total_tiles;
-    const uint64_t ex = odin_lookback_u64(state, tile, agg, status);
-    if (threadIdx.x == 0) s_base = ex;
   }
   __syncthreads();
-  const uint64_t base = s_base;
-  const uint64_t row_base = base >> PACK_SHIFT, inst_base = base & PACK_LOW;
-
-  if (tile == (n + PROJECT_TILE - 1) / PROJECT_TILE - 1 && threadIdx.x == 0) {  // last tile: totals
-    const uint64_t rows = row_base + total_rows, inst = inst_base + total_tiles;
-    *out.num_rows = (uint32_t)(rows < out.capacity ? rows : out.capacity);
-    *out.num_instances = inst;
-    if (rows > out.capacity || inst >= (1ull << 32)) odin_set_error(status, ODIN_ERR_CAPACITY);
+  const uint64_t base = s_base + s_warp[warp];
+#pragma unroll
+  for (int j = 0; j < SCAN_ITEMS; ++j) {
+    if (t[j]) {
+      const uint64_t e = base + ex[j];
+      const uint64_t r = e >> PACK_SHIFT;
+      if (r < capacity) {
+        prim_id[r] = warp_base + 32 * j + lane;
+        tile_offset[r] = (uint32_t)(e & PACK_LOW);
+      }
+    }
   }
-  if (!vis) return;
-  const uint64_t r64 = row_base + row_local;
-  if (r64 >= out.capacity) return;
-  const size_t r = (size_t)r64;
-  out.prim_id[r] = p;
-  reinterpret_cast<float2*>(out.xy)[r] = make_float2(u, v);
-  out.depth[r] = depth;
-  const float o = 1.f / (1.f + expf(-opacity_logit[p]));
-  reinterpret_cast<float4*>(out.conic_opacity)[r] = make_float4(cA, cB, cC, o);
-  out.radius[r] = rad;
-  reinterpret_cast<ushort4*>(out.rect)[r] = make_ushort4((unsigned short)x0, (unsigned short)y0, (unsigned short)x1,
-                                                         (unsigned short)y1);
-  out.tile_offset[r] = (uint32_t)(inst_base + off_local);
+}
 
-  // colour
-  float dx = mx - cam.pos[0], dy = my - cam.pos[1], dz = mz - cam.pos[2];
-  const float len = sqrtf(dx * dx + dy * dy + dz * dz);
-  dx /= len; dy /= len; dz /= len;
-  float Y[16];
-  odin_sh_basis<DEG>(dx, dy, dz, Y);
-  float acc[3] = {0.f, 0.f, 0.f};
-  const float* row = sh + (size_t)p * (3 * K);
-  if (K == 1) {
-    acc[0] = Y[0] * row[0]; acc[1] = Y[0] * row[1]; acc[2] = Y[0] * row[2];
-  } else {
-    // 3K floats are a multiple of 4 for K = 4, 16 (and 27 = 3*9 for K = 9 is not): use scalar loads there
-    if ((3 * K) % 4 == 0) {
+template <int DEG>
+__global__ void __launch_bounds__(128)
+project_rows_kernel(const float* __restrict__ means, const float* __restrict__ log_scales, const float4* __restrict__ quats,
+                    const float* __restrict__ opacity_logit, const float* __restrict__ sh, CamParams cam, float dilation,
+                    float radius_sigmas, odin_projected out) {
+  constexpr int K = (DEG + 1) * (DEG + 1);
+  const uint32_t V = min(*out.num_rows, out.capacity);
+  for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
+    const size_t p = out.prim_id[r];
+    const Footprint f = project_footprint(cam, dilation, radius_sigmas, means, log_scales, quats, p);
+    reinterpret_cast<float2*>(out.xy)[r] = make_float2(f.u, f.v);
+    out.depth[r] = f.depth;
+    const float o = 1.f / (1.f + expf(-opacity_logit[p]));
+    reinterpret_cast<float4*>(out.conic_opacity)[r] = make_float4(f.cA, f.cB, f.cC, o);
+    out.radius[r] = f.rad;
+    reinterpret_cast<ushort4*>(out.rect)[r] =
+        make_ushort4((unsigned short)f.x0, (unsigned short)f.y0, (unsigned short)f.x1, (unsigned short)f.y1);
+    // colour
+    float dx = means[3 * p] - cam.pos[0], dy = means[3 * p + 1] - cam.pos[1], dz = means[3 * p + 2] - cam.pos[2];
+    const float len = sqrtf(dx * dx + dy * dy + dz * dz);
+    dx /= len; dy /= len; dz /= len;
+    float Y[16];
+    odin_sh_basis<DEG>(dx, dy, dz, Y);
+    float acc[3] = {0.f, 0.f, 0.f};
+    const float* row = sh + p * (3 * K);
+    if ((3 * K) % 4 == 0) {  // 12 or 48 floats: 16-byte loads
       const float4* row4 = reinterpret_cast<const float4*>(row);
 #pragma unroll
       for (int i = 0; i < 3 * K / 4; ++i) {
@@ -111,23 +170,23 @@ project_kernel(const float* __restrict__ means, const float* __restrict__ log_sc
         const float e[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const int f = 4 * i + j;
-          acc[f % 3] += Y[f / 3] * e[j];
+          const int w = 4 * i + j;
+          acc[w % 3] += Y[w / 3] * e[j];
         }
       }
     } else {
 #pragma unroll
-      for (int f = 0; f < 3 * K; ++f) acc[f % 3] += Y[f / 3] * row[f];
+      for (int w = 0; w < 3 * K; ++w) acc[w % 3] += Y[w / 3] * row[w];
     }
-  }
-  uint8_t flags = 0;
+    uint8_t flags = 0;
 #pragma unroll
-  for (int ch = 0; ch < 3; ++ch) {
-    acc[ch] += 0.5f;
-    if (acc[ch] < 0.f) { acc[ch] = 0.f; flags |= (uint8_t)(1u << ch); }
+    for (int ch = 0; ch < 3; ++ch) {
+      acc[ch] += 0.5f;
+      if (acc[ch] < 0.f) { acc[ch] = 0.f; flags |= (uint8_t)(1u << ch); }
+    }
+    out.rgb[3 * (size_t)r] = acc[0]; out.rgb[3 * (size_t)r + 1] = acc[1]; out.rgb[3 * (size_t)r + 2] = acc[2];
+    out.clamp_flags[r] = flags;
   }
-  out.rgb[3 * r] = acc[0]; out.rgb[3 * r + 1] = acc[1]; out.rgb[3 * r + 2] = acc[2];
-  out.clamp_flags[r] = flags;
 }
 
 }  // namespace
@@ -160,13 +219,25 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   uint32_t* ticket = reinterpret_cast<uint32_t*>(ws);
   uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + 256);
   const CamParams cp = odin_cam_params(cam, ctx->cfg);
-  const uint32_t grid = (n + PROJECT_TILE - 1) / PROJECT_TILE;
   const float4* q4 = reinterpret_cast<const float4*>(scene->quats);
-#define LAUNCH(D)                                                                                                    \
-  project_kernel<D><<<grid, PROJECT_TILE, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit, scene->sh, \
-                                                   n, cp, ctx->cfg.dilation, ctx->cfg.radius_sigmas, *out, ticket, state, \
-                                                   ctx->d_status)
-  OdinKernelScope ks(ctx, K_PROJECT, st);
+  {
+    OdinKernelScope ks(ctx, K_PROJECT, st);
+    project_cull_kernel<<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4, n, cp, ctx->cfg.dilation,
+                                                         ctx->cfg.radius_sigmas, out->tiles_touched);
+  }
+  {
+    OdinKernelScope ks(ctx, K_PROJECT_SCAN, st);
+    project_scan_kernel<<<(n + PROJECT_TILE - 1) / PROJECT_TILE, SCAN_THREADS, 0, st>>>(
+        out->tiles_touched, n, out->capacity, out->prim_id, out->tile_offset, out->num_rows, out->num_instances, ticket,
+        state, ctx->d_status);
+  }
+  if (out->capacity == 0) return odin_launch_status();
+  const uint32_t blocks_cap = (out->capacity + 127) / 128;
+  const uint32_t grid = blocks_cap < (uint32_t)ctx->sm_count * 16 ? blocks_cap : (uint32_t)ctx->sm_count * 16;
+  OdinKernelScope ks(ctx, K_PROJECT_ROWS, st);
+#define LAUNCH(D)                                                                                                      \
+  project_rows_kernel<D><<<grid, 128, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit, scene->sh, cp, \
+                                               ctx->cfg.dilation, ctx->cfg.radius_sigmas, *out)
   switch (scene->sh_degree) {
     case 0: LAUNCH(0); break;
     case 1: LAUNCH(1); break;
