@@ -32,8 +32,23 @@ __device__ __forceinline__ uint32_t block_upper_bound(const uint32_t* __restrict
 // k = i - offset[r], w = x1 - x0.  Keys and values are written fully coalesced.  Digit histograms for the sort are
 // accumulated on the way: depth digits once per row (weighted by the row's slots in the chunk), tile digits per
 // slot with warp aggregation.
+// chunk_row[c] = the row whose slots contain slot c * DUP_CHUNK (one thread per row; a row writes an entry for every
+// chunk boundary that falls inside its slot range, usually none or one).
+__global__ void __launch_bounds__(256)
+chunk_rows_kernel(const uint32_t* __restrict__ tile_offset, const uint32_t* __restrict__ num_rows,
+                  const uint64_t* __restrict__ num_instances, uint32_t chunks_cap, uint32_t* __restrict__ chunk_row) {
+  const uint32_t V = *num_rows;
+  const uint64_t M_all = *num_instances;
+  for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
+    const uint64_t lo = tile_offset[r];
+    const uint64_t hi = (r + 1 < V) ? (uint64_t)tile_offset[r + 1] : M_all;
+    for (uint64_t c = (lo + DUP_CHUNK - 1) / DUP_CHUNK; c * DUP_CHUNK < hi && c < chunks_cap; ++c) chunk_row[c] = r;
+  }
+}
+
 __global__ void __launch_bounds__(DUP_THREADS)
-emit_instances_kernel(const uint32_t* __restrict__ tile_offset, const ushort4* __restrict__ rect,
+emit_instances_kernel(const uint32_t* __restrict__ tile_offset, const uint32_t* __restrict__ chunk_row,
+                      const ushort4* __restrict__ rect,
                       const float* __restrict__ depth, const uint32_t* __restrict__ num_rows,
                       const uint64_t* __restrict__ num_instances, uint64_t capacity, int TX, int passes,
                       uint64_t* __restrict__ keys, uint32_t* __restrict__ vals, uint32_t* __restrict__ hist, int* status) {
@@ -53,8 +68,15 @@ emit_instances_kernel(const uint32_t* __restrict__ tile_offset, const ushort4* _
   for (uint32_t chunk = blockIdx.x; chunk < chunks; chunk += gridDim.x) {
     const uint32_t c0 = chunk * DUP_CHUNK;
     const uint32_t c1 = (M - c0 < (uint32_t)DUP_CHUNK) ? M : c0 + DUP_CHUNK;
-    const uint32_t row_lo = block_upper_bound(tile_offset, V, c0) - 1;  // offset[0] = 0 <= c0, so the bound is >= 1
-    const uint32_t row_hi = block_upper_bound(tile_offset, V, c1 - 1) - 1;
+    // first and last row of the chunk from the chunk -> row table; only the last chunk has to search for its end
+    const uint32_t row_lo = chunk_row[chunk];
+    uint32_t row_hi;
+    if (chunk + 1 < chunks) {
+      const uint32_t rn = chunk_row[chunk + 1];  // row that holds slot c1
+      row_hi = (tile_offset[rn] == c1) ? rn - 1 : rn;
+    } else {
+      row_hi = block_upper_bound(tile_offset, V, c1 - 1) - 1;  // offset[0] = 0, so the bound is >= 1
+    }
     const uint32_t nrows = row_hi - row_lo + 1;  // <= DUP_CHUNK: every row owns at least one slot
     for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS) {
       s_off[i] = tile_offset[row_lo + i];
@@ -68,13 +90,15 @@ emit_instances_kernel(const uint32_t* __restrict__ tile_offset, const ushort4* _
       const uint32_t b = max(s_off[i], c0), e = min(s_off[i + 1], c1);
       const uint32_t wgt = e - b, bits = s_depth[i];
 #pragma unroll
-      for (int d = 0; d < 4; ++d) atomicAdd(&s_hist[d][(bits >> (8 * d)) & 255u], wgt);
+      for (int d = 0; d < SORT_DEPTH_DIGITS; ++d)
+        atomicAdd(&s_hist[d][(bits >> (SORT_RADIX_BITS * d)) & (SORT_RADIX - 1)], wgt);
     }
 #pragma unroll
     for (int k = 0; k < DUP_ITEMS; ++k) {
       const uint32_t i = c0 + k * DUP_THREADS + threadIdx.x;
       const bool valid = i < c1;
       uint32_t tile = 0xffffffffu;
+      uint64_t key = 0;
       if (valid) {
         uint32_t lo = 0, hi = nrows;  // last j with s_off[j] <= i
         while (hi - lo > 1) {
@@ -86,11 +110,13 @@ emit_instances_kernel(const uint32_t* __restrict__ tile_offset, const ushort4* _
         const uint32_t w = (uint32_t)rc.z - (uint32_t)rc.x;
         const uint32_t dy = local / w, dx = local - dy * w;
         tile = ((uint32_t)rc.y + dy) * (uint32_t)TX + (uint32_t)rc.x + dx;
-        keys[i] = ((uint64_t)tile << 32) | (uint64_t)s_depth[lo];
+        key = ((uint64_t)tile << 32) | (uint64_t)s_depth[lo];
+        keys[i] = key;
         vals[i] = row_lo + lo;
       }
-      for (int d = 4; d < passes; ++d) {
-        const uint32_t digit = valid ? ((tile >> (8 * (d - 4))) & 255u) : (256u + lane);
+      // digits that contain tile bits differ from slot to slot of a row: count them per slot, aggregated per warp
+      for (int d = SORT_DEPTH_DIGITS; d < passes; ++d) {
+        const uint32_t digit = valid ? ((uint32_t)(key >> (SORT_RADIX_BITS * d)) & (SORT_RADIX - 1)) : (SORT_RADIX + lane);
         const uint32_t peers = __match_any_sync(0xffffffffu, digit);
         if (valid && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&s_hist[d][digit], (uint32_t)__popc(peers));
       }
@@ -115,6 +141,8 @@ __global__ void __launch_bounds__(SORT_RADIX) digit_base_kernel(const uint32_t* 
 constexpr int OS_THREADS = 256;
 constexpr int OS_WARPS = OS_THREADS / 32;
 constexpr int OS_ITEMS = SORT_TILE / OS_THREADS;  // 16 keys per thread
+constexpr int OS_DPT = SORT_RADIX / OS_THREADS;   // digits owned by a thread
+constexpr int OS_WINDOW = 2;                      // predecessors fetched per look-back step and digit
 constexpr uint32_t OS_FLAG_AGG = 1u << 30, OS_FLAG_INC = 2u << 30, OS_VALUE = (1u << 30) - 1;
 constexpr size_t OS_SMEM = (size_t)SORT_TILE * 8 + (size_t)SORT_TILE * 4 + (size_t)OS_WARPS * SORT_RADIX * 4 + 2 * SORT_RADIX * 4 + 16;
 
@@ -122,7 +150,7 @@ constexpr size_t OS_SMEM = (size_t)SORT_TILE * 8 + (size_t)SORT_TILE * 4 + (size
 // per-warp digit ranking with match.any (stable), block digit counts published for look-back, exclusive global digit
 // offsets by a per-digit look-back walk (thread d walks digit d), keys and values exchanged through shared memory so
 // that the global scatter writes runs of consecutive addresses.
-__global__ void __launch_bounds__(OS_THREADS)
+__global__ void __launch_bounds__(OS_THREADS, 3)
 onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in, uint64_t* __restrict__ keys_out,
                 uint32_t* __restrict__ vals_out, const uint64_t* __restrict__ num_instances, uint64_t capacity, int shift,
                 const uint32_t* __restrict__ digit_base, uint32_t* states, uint32_t* ticket, int* status) {
@@ -142,25 +170,32 @@ onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t lt_mask = (1u << lane) - 1u;
 
-  while (true) {
-    if (threadIdx.x == 0) s_misc[0] = atomicAdd(ticket, 1u);
-    for (int i = threadIdx.x; i < OS_WARPS * (int)SORT_RADIX; i += OS_THREADS) (&s_warp_hist[0][0])[i] = 0;
-    __syncthreads();
-    const uint32_t tile = s_misc[0];
-    if (tile >= ntiles) break;
-    const uint32_t tile_base = tile * SORT_TILE;
-    const uint32_t tile_count = min((uint32_t)SORT_TILE, M - tile_base);
-    const uint32_t warp_base = tile_base + warp * (32 * OS_ITEMS);
-
-    uint64_t key[OS_ITEMS];
-    uint32_t val[OS_ITEMS];
-    uint32_t pos[OS_ITEMS];
+  // The keys and values of the NEXT tile are requested as soon as the registers of the current one are free (after
+  // the exchange through shared memory), so that their latency overlaps the global scatter of the current tile.
+  uint64_t key[OS_ITEMS];
+  uint32_t val[OS_ITEMS];
+  auto load_tile = [&](uint32_t t) {
+    const uint32_t wb = t * SORT_TILE + warp * (32 * OS_ITEMS);
 #pragma unroll
     for (int j = 0; j < OS_ITEMS; ++j) {
-      const uint32_t i = warp_base + 32 * j + lane;
-      key[j] = (i < M) ? keys_in[i] : ~0ull;  // padding sorts to the end of the tile and is never written
-      val[j] = (i < M) ? vals_in[i] : 0u;
+      const uint32_t i = wb + 32 * j + lane;
+      const bool in = t < ntiles && i < M;
+      key[j] = in ? keys_in[i] : ~0ull;  // padding sorts to the end of the tile and is never written
+      val[j] = in ? vals_in[i] : 0u;
     }
+  };
+  if (threadIdx.x == 0) s_misc[0] = atomicAdd(ticket, 1u);
+  __syncthreads();
+  uint32_t tile = s_misc[0];
+  load_tile(tile);
+
+  while (tile < ntiles) {
+    for (int i = threadIdx.x; i < OS_WARPS * (int)SORT_RADIX; i += OS_THREADS) (&s_warp_hist[0][0])[i] = 0;
+    __syncthreads();
+    const uint32_t tile_base = tile * SORT_TILE;
+    const uint32_t tile_count = min((uint32_t)SORT_TILE, M - tile_base);
+
+    uint32_t pos[OS_ITEMS];
 #pragma unroll
     for (int j = 0; j < OS_ITEMS; ++j) {
       const uint32_t d = (uint32_t)(key[j] >> shift) & (SORT_RADIX - 1);
@@ -177,39 +212,84 @@ onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict
     }
     __syncthreads();
 
-    // thread d owns digit d
-    const uint32_t d = threadIdx.x;
-    uint32_t cta_count = 0;
+    // thread t owns digits t, t + 256, ...: exclusive offsets of the warps inside each digit, block totals published
+    uint32_t cta_count[OS_DPT];
 #pragma unroll
-    for (int w = 0; w < OS_WARPS; ++w) {
-      const uint32_t t = s_warp_hist[w][d];
-      s_warp_hist[w][d] = cta_count;  // exclusive offset of warp w inside digit d
-      cta_count += t;
-    }
-    uint32_t* my_state = states + (size_t)tile * SORT_RADIX + d;
-    st_volatile_u32(my_state, (tile == 0 ? OS_FLAG_INC : OS_FLAG_AGG) | cta_count);
-    uint32_t total;
-    const uint32_t digit_start = odin_block_exclusive_sum(cta_count, s_scan, &total);
-    s_digit_start[d] = digit_start;
-    uint32_t exclusive = 0;
-    if (tile > 0) {
-      int64_t t = (int64_t)tile - 1;
-      int spins = 0;
-      while (t >= 0) {
-        const uint32_t s = ld_volatile_u32(states + (size_t)t * SORT_RADIX + d);
-        const uint32_t flag = s >> 30;
-        if (flag == 0) {
-          __nanosleep(64);
-          if (++spins > ODIN_SPIN_LIMIT) { odin_set_error(status, ODIN_ERR_TIMEOUT); break; }
-          continue;
-        }
-        exclusive += s & OS_VALUE;
-        if (flag == 2) break;
-        --t;
+    for (int q = 0; q < OS_DPT; ++q) {
+      const uint32_t d = threadIdx.x + q * OS_THREADS;
+      uint32_t c = 0;
+#pragma unroll
+      for (int w = 0; w < OS_WARPS; ++w) {
+        const uint32_t t = s_warp_hist[w][d];
+        s_warp_hist[w][d] = c;
+        c += t;
       }
-      st_volatile_u32(my_state, OS_FLAG_INC | ((exclusive + cta_count) & OS_VALUE));
+      cta_count[q] = c;
+      st_volatile_u32(states + (size_t)tile * SORT_RADIX + d, (tile == 0 ? OS_FLAG_INC : OS_FLAG_AGG) | c);
     }
-    s_global[d] = digit_base[d] + exclusive - digit_start;  // add the slot index inside the tile to get the address
+    uint32_t digit_start[OS_DPT];
+    {
+      uint32_t carry = 0;
+#pragma unroll
+      for (int q = 0; q < OS_DPT; ++q) {  // digits ascend with q first, so the scans chain
+        uint32_t total;
+        digit_start[q] = carry + odin_block_exclusive_sum(cta_count[q], s_scan, &total);
+        s_digit_start[threadIdx.x + q * OS_THREADS] = digit_start[q];
+        carry += total;
+      }
+    }
+    uint32_t exclusive[OS_DPT];
+#pragma unroll
+    for (int q = 0; q < OS_DPT; ++q) exclusive[q] = 0;
+    if (tile > 0) {
+      // walk back over the predecessors for all owned digits at once
+      int64_t t[OS_DPT];
+#pragma unroll
+      for (int q = 0; q < OS_DPT; ++q) t[q] = (int64_t)tile - 1;
+      int spins = 0;
+      bool busy = true;
+      while (busy) {
+        busy = false;
+        bool stalled = true;  // cleared as soon as any predecessor word is consumed
+        // a window of OS_WINDOW predecessors per digit is fetched at once: the walk is a chain of dependent L2 round
+        // trips, and when a launch starts every resident tile has hundreds of aggregates in front of it
+        uint32_t s[OS_DPT][OS_WINDOW];
+#pragma unroll
+        for (int q = 0; q < OS_DPT; ++q)
+#pragma unroll
+          for (int k = 0; k < OS_WINDOW; ++k)
+            s[q][k] = (t[q] - k >= 0)
+                          ? ld_volatile_u32(states + (size_t)(t[q] - k) * SORT_RADIX + threadIdx.x + q * OS_THREADS)
+                          : 0u;
+#pragma unroll
+        for (int q = 0; q < OS_DPT; ++q) {
+          if (t[q] < 0) continue;
+#pragma unroll
+          for (int k = 0; k < OS_WINDOW; ++k) {
+            if (t[q] < 0) break;
+            const uint32_t flag = s[q][k] >> 30;
+            if (flag == 0) break;  // not published yet: use what precedes it, come back
+            exclusive[q] += s[q][k] & OS_VALUE;
+            t[q] = (flag == 2) ? -1 : t[q] - 1;
+            stalled = false;
+          }
+          if (t[q] >= 0) busy = true;
+        }
+        if (busy && stalled) {
+          __nanosleep(32);
+          if (++spins > ODIN_SPIN_LIMIT) { odin_set_error(status, ODIN_ERR_TIMEOUT); break; }
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < OS_DPT; ++q)
+        st_volatile_u32(states + (size_t)tile * SORT_RADIX + threadIdx.x + q * OS_THREADS,
+                        OS_FLAG_INC | ((exclusive[q] + cta_count[q]) & OS_VALUE));
+    }
+#pragma unroll
+    for (int q = 0; q < OS_DPT; ++q) {
+      const uint32_t d = threadIdx.x + q * OS_THREADS;
+      s_global[d] = digit_base[d] + exclusive[q] - digit_start[q];  // + slot index inside the tile = address
+    }
     __syncthreads();
 
 #pragma unroll
@@ -219,7 +299,10 @@ onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict
       s_keys[slot] = key[j];
       s_vals[slot] = val[j];
     }
+    if (threadIdx.x == 0) s_misc[0] = atomicAdd(ticket, 1u);
     __syncthreads();
+    const uint32_t next = s_misc[0];
+    load_tile(next);  // in flight while the current tile is written out
 #pragma unroll
     for (int j = 0; j < OS_ITEMS; ++j) {
       const uint32_t slot = j * OS_THREADS + threadIdx.x;
@@ -232,6 +315,7 @@ onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict
         }
       }
     }
+    tile = next;
     __syncthreads();
   }
 }
@@ -299,9 +383,17 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
 
   const uint64_t chunks_cap = (capacity + DUP_CHUNK - 1) / DUP_CHUNK;
   uint32_t grid = (uint32_t)(chunks_cap < (uint64_t)ctx->sm_count * 6 ? chunks_cap : (uint64_t)ctx->sm_count * 6);
+  uint32_t* chunk_row = reinterpret_cast<uint32_t*>(base + L.chunk_row);
+  {
+    OdinKernelScope ks(ctx, K_CHUNK_ROWS, st);
+    const uint32_t rb = (proj->capacity + 255) / 256;
+    chunk_rows_kernel<<<rb < (uint32_t)ctx->sm_count * 8 ? rb : (uint32_t)ctx->sm_count * 8, 256, 0, st>>>(
+        proj->tile_offset, proj->num_rows, proj->num_instances, (uint32_t)chunks_cap, chunk_row);
+  }
   {
     OdinKernelScope ks(ctx, K_EMIT, st);
-    emit_instances_kernel<<<grid, DUP_THREADS, 0, st>>>(proj->tile_offset, reinterpret_cast<const ushort4*>(proj->rect),
+    emit_instances_kernel<<<grid, DUP_THREADS, 0, st>>>(proj->tile_offset, chunk_row,
+                                                        reinterpret_cast<const ushort4*>(proj->rect),
                                                         proj->depth, proj->num_rows, proj->num_instances, capacity, TX,
                                                         passes, kbuf[cur], vbuf[cur], hist, ctx->d_status);
   }

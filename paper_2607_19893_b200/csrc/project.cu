@@ -68,7 +68,9 @@ constexpr int SCAN_ITEMS = PROJECT_TILE / SCAN_THREADS;
 __global__ void __launch_bounds__(SCAN_THREADS)
 project_scan_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint32_t capacity,
                     uint32_t* __restrict__ prim_id, uint32_t* __restrict__ tile_offset, uint32_t* __restrict__ num_rows,
-                    uint64_t* __restrict__ num_instances, uint32_t* ticket, uint64_t* state, int* status) {
+                    uint64_t* __restrict__ num_instances, uint32_t* ticket, uint64_t* state, int* status,
+                    int scan_rounds) {
+  const uint32_t scan_chunk = PROJECT_TILE * (uint32_t)scan_rounds;
   __shared__ uint32_t s_tile;
   __shared__ uint64_t s_warp[SCAN_THREADS / 32 + 1];
   __shared__ uint64_t s_base;
@@ -76,44 +78,29 @@ project_scan_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint
   __syncthreads();
   const uint32_t tile = s_tile;
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t warp_base = tile * PROJECT_TILE + warp * (32 * SCAN_ITEMS);
-  uint32_t t[SCAN_ITEMS];
+  const uint32_t chunk_base = tile * scan_chunk;
+  // pass A: packed (rows, instances) total of the chunk, then ONE look-back per scan_chunk primitives
+  uint64_t mine = 0;
 #pragma unroll
-  for (int j = 0; j < SCAN_ITEMS; ++j) {
-    const uint32_t p = warp_base + 32 * j + lane;
-    t[j] = (p < n) ? tiles_touched[p] : 0u;
-  }
-  // per item: packed (1 row, t tiles) exclusive prefix inside the warp, in primitive order
-  uint64_t ex[SCAN_ITEMS];
-  uint64_t run = 0;
+  for (int rnd = 0; rnd < scan_rounds; ++rnd) {
+    const uint32_t warp_base = chunk_base + rnd * PROJECT_TILE + warp * (32 * SCAN_ITEMS);
 #pragma unroll
-  for (int j = 0; j < SCAN_ITEMS; ++j) {
-    const uint64_t v = t[j] ? ((1ull << PACK_SHIFT) | (uint64_t)t[j]) : 0ull;
-    uint64_t inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint64_t y = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= (unsigned)o) inc += y;
+    for (int j = 0; j < SCAN_ITEMS; ++j) {
+      const uint32_t p = warp_base + 32 * j + lane;
+      const uint32_t t = (p < n) ? tiles_touched[p] : 0u;
+      mine += t ? ((1ull << PACK_SHIFT) | (uint64_t)t) : 0ull;
     }
-    ex[j] = run + inc - v;
-    run += __shfl_sync(0xffffffffu, inc, 31);
   }
-  if (lane == 0) s_warp[warp] = run;
+  for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+  if (lane == 0) s_warp[warp] = mine;
   __syncthreads();
   if (threadIdx.x < 32) {
-    uint64_t w = (lane < SCAN_THREADS / 32) ? s_warp[lane] : 0ull;
-    uint64_t inc = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint64_t y = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= (unsigned)o) inc += y;
-    }
-    const uint64_t total = __shfl_sync(0xffffffffu, inc, 31);
-    if (lane < SCAN_THREADS / 32) s_warp[lane] = inc - w;
+    uint64_t total = (lane < SCAN_THREADS / 32) ? s_warp[lane] : 0ull;
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
     const uint64_t base = odin_lookback_u64(state, tile, total, status);
     if (lane == 0) {
       s_base = base;
-      if (tile == (n + PROJECT_TILE - 1) / PROJECT_TILE - 1) {  // last tile: totals
+      if (tile == (n + scan_chunk - 1) / scan_chunk - 1) {  // last chunk: totals
         const uint64_t all = base + total;
         const uint64_t rows = all >> PACK_SHIFT, inst = all & PACK_LOW;
         *num_rows = (uint32_t)(rows < capacity ? rows : capacity);
@@ -123,17 +110,55 @@ project_scan_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint
     }
   }
   __syncthreads();
-  const uint64_t base = s_base + s_warp[warp];
+  uint64_t round_base = s_base;
+  // pass B: re-read the chunk (from cache), 2048 primitives per round
+  for (int rnd = 0; rnd < scan_rounds; ++rnd) {
+    if (chunk_base + rnd * PROJECT_TILE >= n) break;  // uniform over the block
+    const uint32_t warp_base = chunk_base + rnd * PROJECT_TILE + warp * (32 * SCAN_ITEMS);
+    uint32_t t[SCAN_ITEMS];
 #pragma unroll
-  for (int j = 0; j < SCAN_ITEMS; ++j) {
-    if (t[j]) {
-      const uint64_t e = base + ex[j];
-      const uint64_t r = e >> PACK_SHIFT;
-      if (r < capacity) {
-        prim_id[r] = warp_base + 32 * j + lane;
-        tile_offset[r] = (uint32_t)(e & PACK_LOW);
+    for (int j = 0; j < SCAN_ITEMS; ++j) {
+      const uint32_t p = warp_base + 32 * j + lane;
+      t[j] = (p < n) ? tiles_touched[p] : 0u;
+    }
+    // per item: packed (1 row, t tiles) exclusive prefix inside the warp, in primitive order
+    uint64_t ex[SCAN_ITEMS];
+    uint64_t run = 0;
+#pragma unroll
+    for (int j = 0; j < SCAN_ITEMS; ++j) {
+      const uint64_t v = t[j] ? ((1ull << PACK_SHIFT) | (uint64_t)t[j]) : 0ull;
+      uint64_t inc = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint64_t y = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= (unsigned)o) inc += y;
+      }
+      ex[j] = run + inc - v;
+      run += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    __syncthreads();  // previous round's readers of s_warp are done
+    if (lane == 0) s_warp[warp] = run;
+    __syncthreads();
+    uint64_t before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < SCAN_THREADS / 32; ++w) {
+      const uint64_t x = s_warp[w];
+      if (w < (int)warp) before += x;
+      total += x;
+    }
+    const uint64_t base = round_base + before;
+#pragma unroll
+    for (int j = 0; j < SCAN_ITEMS; ++j) {
+      if (t[j]) {
+        const uint64_t e = base + ex[j];
+        const uint64_t r = e >> PACK_SHIFT;
+        if (r < capacity) {
+          prim_id[r] = warp_base + 32 * j + lane;
+          tile_offset[r] = (uint32_t)(e & PACK_LOW);
+        }
       }
     }
+    round_base += total;
   }
 }
 
@@ -227,9 +252,11 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   }
   {
     OdinKernelScope ks(ctx, K_PROJECT_SCAN, st);
-    project_scan_kernel<<<(n + PROJECT_TILE - 1) / PROJECT_TILE, SCAN_THREADS, 0, st>>>(
+    const int scan_rounds = scan_rounds_for(n, ctx->sm_count);
+    const uint32_t scan_chunk = PROJECT_TILE * (uint32_t)scan_rounds;
+    project_scan_kernel<<<(n + scan_chunk - 1) / scan_chunk, SCAN_THREADS, 0, st>>>(
         out->tiles_touched, n, out->capacity, out->prim_id, out->tile_offset, out->num_rows, out->num_instances, ticket,
-        state, ctx->d_status);
+        state, ctx->d_status, scan_rounds);
   }
   if (out->capacity == 0) return odin_launch_status();
   const uint32_t blocks_cap = (out->capacity + 127) / 128;

@@ -366,14 +366,35 @@ render_bwd_project_kernel(const float* __restrict__ means, const float* __restri
     float gd[3] = {0.f, 0.f, 0.f};
     const float* shrow = sh + p * (3 * K);
     float* gshrow = g_sh + (size_t)r * (3 * K);
+    if ((3 * K) % 4 == 0) {  // 12 or 48 floats per row: 16-byte loads and stores
+      const float4* sh4 = reinterpret_cast<const float4*>(shrow);
+      float4* gsh4 = reinterpret_cast<float4*>(gshrow);
 #pragma unroll
-    for (int k = 0; k < K; ++k) {
+      for (int i = 0; i < 3 * K / 4; ++i) {
+        const float4 c = sh4[i];
+        const float e[4] = {c.x, c.y, c.z, c.w};
+        float o4[4];
 #pragma unroll
-      for (int ch = 0; ch < 3; ++ch) {
-        gshrow[3 * k + ch] = Y[k] * gch[ch];
-        if (k > 0) {
-          const float wgt = shrow[3 * k + ch] * gch[ch];
-          gd[0] += dY[k][0] * wgt; gd[1] += dY[k][1] * wgt; gd[2] += dY[k][2] * wgt;
+        for (int j = 0; j < 4; ++j) {
+          const int w = 4 * i + j, k = w / 3, ch = w % 3;
+          o4[j] = Y[k] * gch[ch];
+          if (k > 0) {
+            const float wgt = e[j] * gch[ch];
+            gd[0] += dY[k][0] * wgt; gd[1] += dY[k][1] * wgt; gd[2] += dY[k][2] * wgt;
+          }
+        }
+        gsh4[i] = make_float4(o4[0], o4[1], o4[2], o4[3]);
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < K; ++k) {
+#pragma unroll
+        for (int ch = 0; ch < 3; ++ch) {
+          gshrow[3 * k + ch] = Y[k] * gch[ch];
+          if (k > 0) {
+            const float wgt = shrow[3 * k + ch] * gch[ch];
+            gd[0] += dY[k][0] * wgt; gd[1] += dY[k][1] * wgt; gd[2] += dY[k][2] * wgt;
+          }
         }
       }
     }

@@ -12,7 +12,8 @@ constexpr int TS_ITEMS = TOUCHED_TILE / TS_THREADS;  // 8 words of 32 primitives
 __global__ void __launch_bounds__(TS_THREADS)
 touched_set_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint32_t* __restrict__ mask,
                    uint32_t* __restrict__ idx, uint32_t idx_capacity, uint32_t* __restrict__ count, uint32_t* ticket,
-                   uint64_t* state, int* status) {
+                   uint64_t* state, int* status, int scan_rounds) {
+  const uint32_t scan_chunk = TOUCHED_TILE * (uint32_t)scan_rounds;
   __shared__ uint32_t s_tile;
   __shared__ uint32_t s_warp[33];
   __shared__ uint64_t s_base;
@@ -20,52 +21,72 @@ touched_set_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint3
   __syncthreads();
   const uint32_t tile = s_tile;
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t warp_base = tile * TOUCHED_TILE + warp * (32 * TS_ITEMS);
-  uint32_t t[TS_ITEMS];
+  const uint32_t chunk_base = tile * scan_chunk;
+  // pass A: how many touched primitives does this chunk hold (one look-back per scan_chunk primitives keeps the
+  // chain of dependent tiles short; the second pass re-reads the chunk from cache)
+  uint32_t mine = 0;
 #pragma unroll
-  for (int j = 0; j < TS_ITEMS; ++j) {
-    const uint32_t p = warp_base + 32 * j + lane;
-    t[j] = (p < n) ? tiles_touched[p] : 0u;
-  }
-  uint32_t ballots[TS_ITEMS];
-  uint32_t warp_count = 0;
+  for (int rnd = 0; rnd < scan_rounds; ++rnd) {
+    const uint32_t warp_base = chunk_base + rnd * TOUCHED_TILE + warp * (32 * TS_ITEMS);
 #pragma unroll
-  for (int j = 0; j < TS_ITEMS; ++j) {
-    ballots[j] = __ballot_sync(0xffffffffu, t[j] > 0);
-    warp_count += __popc(ballots[j]);
+    for (int j = 0; j < TS_ITEMS; ++j) {
+      const uint32_t p = warp_base + 32 * j + lane;
+      mine += (p < n && tiles_touched[p] > 0) ? 1u : 0u;
+    }
   }
-  // mask words (lane j writes word j of the warp)
-  if (lane < TS_ITEMS) {
-    uint32_t w = 0;
-#pragma unroll
-    for (int j = 0; j < TS_ITEMS; ++j)
-      if (lane == (unsigned)j) w = ballots[j];
-    const uint32_t word = warp_base / 32 + lane;
-    if (word < (n + 31) / 32) mask[word] = w;
-  }
-  // exclusive offsets of the warps inside the block
-  uint32_t total;
-  const uint32_t scan = odin_block_exclusive_sum(lane == 0 ? warp_count : 0u, s_warp, &total);
-  const uint32_t warp_off = __shfl_sync(0xffffffffu, scan, 0);
+  uint32_t chunk_total;
+  odin_block_exclusive_sum(mine, s_warp, &chunk_total);
   if (threadIdx.x < 32) {
-    const uint64_t ex = odin_lookback_u64(state, tile, (uint64_t)total, status);
+    const uint64_t ex = odin_lookback_u64(state, tile, (uint64_t)chunk_total, status);
     if (threadIdx.x == 0) s_base = ex;
   }
   __syncthreads();
-  const uint64_t base = s_base;
-  if (tile == (n + TOUCHED_TILE - 1) / TOUCHED_TILE - 1 && threadIdx.x == 0) {
-    const uint64_t v = base + total;
+  uint64_t base = s_base;
+  if (tile == (n + scan_chunk - 1) / scan_chunk - 1 && threadIdx.x == 0) {
+    const uint64_t v = base + chunk_total;
     *count = (uint32_t)(v < idx_capacity ? v : idx_capacity);
     if (v > idx_capacity) odin_set_error(status, ODIN_ERR_CAPACITY);
   }
-  uint64_t pos = base + warp_off;
+  // pass B: masks and the ascending list, 2048 primitives per round
+  for (int rnd = 0; rnd < scan_rounds; ++rnd) {
+    const uint32_t warp_base = chunk_base + rnd * TOUCHED_TILE + warp * (32 * TS_ITEMS);
+    if (chunk_base + rnd * TOUCHED_TILE >= n) break;  // uniform over the block
+    uint32_t t[TS_ITEMS];
 #pragma unroll
-  for (int j = 0; j < TS_ITEMS; ++j) {
-    if (t[j] > 0) {
-      const uint64_t dst = pos + __popc(ballots[j] & ((1u << lane) - 1u));
-      if (dst < idx_capacity) idx[dst] = warp_base + 32 * j + lane;
+    for (int j = 0; j < TS_ITEMS; ++j) {
+      const uint32_t p = warp_base + 32 * j + lane;
+      t[j] = (p < n) ? tiles_touched[p] : 0u;
     }
-    pos += __popc(ballots[j]);
+    uint32_t ballots[TS_ITEMS];
+    uint32_t warp_count = 0;
+#pragma unroll
+    for (int j = 0; j < TS_ITEMS; ++j) {
+      ballots[j] = __ballot_sync(0xffffffffu, t[j] > 0);
+      warp_count += __popc(ballots[j]);
+    }
+    // mask words (lane j writes word j of the warp)
+    if (lane < TS_ITEMS) {
+      uint32_t w = 0;
+#pragma unroll
+      for (int j = 0; j < TS_ITEMS; ++j)
+        if (lane == (unsigned)j) w = ballots[j];
+      const uint32_t word = warp_base / 32 + lane;
+      if (word < (n + 31) / 32) mask[word] = w;
+    }
+    // exclusive offsets of the warps inside the round
+    uint32_t total;
+    const uint32_t scan = odin_block_exclusive_sum(lane == 0 ? warp_count : 0u, s_warp, &total);
+    const uint32_t warp_off = __shfl_sync(0xffffffffu, scan, 0);
+    uint64_t pos = base + warp_off;
+#pragma unroll
+    for (int j = 0; j < TS_ITEMS; ++j) {
+      if (t[j] > 0) {
+        const uint64_t dst = pos + __popc(ballots[j] & ((1u << lane) - 1u));
+        if (dst < idx_capacity) idx[dst] = warp_base + 32 * j + lane;
+      }
+      pos += __popc(ballots[j]);
+    }
+    base += total;
   }
 }
 
@@ -123,10 +144,12 @@ extern "C" int odin_touched_set(odin_ctx* ctx, const uint32_t* d_tiles_touched, 
   ODIN_CUDA(cudaMemsetAsync(ws, 0, need, st));
   uint32_t* ticket = reinterpret_cast<uint32_t*>(ws);
   uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + 256);
-  const uint32_t grid = (n + TOUCHED_TILE - 1) / TOUCHED_TILE;
+  const int scan_rounds = scan_rounds_for(n, ctx->sm_count);
+  const uint32_t scan_chunk = TOUCHED_TILE * (uint32_t)scan_rounds;
+  const uint32_t grid = (n + scan_chunk - 1) / scan_chunk;
   OdinKernelScope ks(ctx, K_TOUCHED, st);
   touched_set_kernel<<<grid, TS_THREADS, 0, st>>>(d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket, state,
-                                                  ctx->d_status);
+                                                  ctx->d_status, scan_rounds);
   return odin_launch_status();
 }
 
@@ -173,8 +196,10 @@ extern "C" int odin_touched_set_static(const uint32_t* d_tiles_touched, uint32_t
   uint32_t* ticket = reinterpret_cast<uint32_t*>(scratch);
   int* status = d_status ? d_status : reinterpret_cast<int*>(scratch + 64);
   uint64_t* state = reinterpret_cast<uint64_t*>(scratch + TS_STATIC_HEADER);
-  touched_set_kernel<<<tiles, TS_THREADS, 0, st>>>(d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket, state,
-                                                  status);
+  const int scan_rounds = scan_rounds_for(n, 148);  // no context here: sized for a B200
+  const uint32_t scan_chunk = TOUCHED_TILE * (uint32_t)scan_rounds;
+  touched_set_kernel<<<(n + scan_chunk - 1) / scan_chunk, TS_THREADS, 0, st>>>(
+      d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket, state, status, scan_rounds);
   return odin_launch_status();
 }
 
