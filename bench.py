@@ -137,7 +137,7 @@ def run_reference(args, rank):
     import oracle
 
     o32 = oracle.get(np.float32)
-    w = wl.make_workload(args.config)
+    w = wl.make_workload(args.config, city_grid=args.city_grid if args.config == 5 else None)
     n = w.scene.n
     steps, warm = args.steps, args.warmup
     # size the per-step sample so that the whole run stays within ~150 s: a probe on 20k primitives gives the cost
@@ -181,6 +181,9 @@ def main():
     ap.add_argument("--impl", default="odin", choices=["odin", "reference"])
     ap.add_argument("--no-kernel-events", action="store_true", help="do not bracket kernels with CUDA events")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--city-grid", type=int, default=None,
+                    help="config 5 only: a city of GxG blocks at the same density (default 64x64 = 20M primitives); "
+                         "for profiler captures that must stay within a few GB")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "odin" else args.warmup
 
@@ -208,12 +211,14 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
 
-    w = wl.make_workload(args.config)
+    w = wl.make_workload(args.config, city_grid=args.city_grid if args.config == 5 else None)
     scene = w.scene
     n, f = scene.n, scene.floats_per_primitive
     cam0 = w.cameras[0]
     W, H = cam0.width, cam0.height
     row_cap = max(1, int(ROW_CAP_FRAC[args.config] * n))
+    if args.config == 5:  # a smaller city (--city-grid) shows the same absolute number of primitives per view
+        row_cap = min(n, max(row_cap, 1_600_000))
     tr = ViewTrainer(scene, W, H, row_cap, INSTANCE_CAP[args.config], mask_slots=MASK_SLOTS, device=local_rank)
     n_views = min(len(w.cameras), args.steps + args.warmup)
     # rank r starts its replica at view r so that replicas do not all render the same camera at the same time

@@ -42,7 +42,7 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
                        const float* __restrict__ dL, float* __restrict__ g2d, float* __restrict__ state) {
   constexpr int BB = BLEND_TAIL_THREADS;
   __shared__ BlendRow s_rowdata[BB];
-  __shared__ float s_blue[BB];
+  __shared__ float2 s_blue[BB];  // blue, power threshold
   __shared__ uint32_t s_rowid[BB];
   __shared__ float s_acc[BB * 9];
   __shared__ uint32_t s_max;
@@ -89,27 +89,28 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
       row.q1 = conic_o[r];
       s_rowdata[threadIdx.x] = row;
-      s_blue[threadIdx.x] = rgb[3 * (size_t)r + 2];
+      s_blue[threadIdx.x] = make_float2(rgb[3 * (size_t)r + 2], blend_power_cut(alpha_min, row.q1.w));
       s_rowid[threadIdx.x] = r;
     }
     __syncthreads();
     for (int j = cnt - 1; j >= 0; --j) {
       const float4 q0 = s_rowdata[j].q0, q1 = s_rowdata[j].q1;
+      const float2 bp = s_blue[j];
       const float dx = q0.x - fx;
       const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
       const float dy = (q0.y - fy0) - slot2;
       const float power = blend_power(h0, h1, h2, dy);
-      const float G = __expf(power);
-      const float og = q1.w * G;
-      const float alpha = fminf(alpha_max, og);
-      const bool on = (b + j < last) && (power <= 0.f) && (alpha >= alpha_min);
+      const bool on = (b + j < last) && (power <= 0.f) && (power >= bp.y);
       if (__ballot_sync(0xffffffffu, on) == 0) continue;
       float vu = 0.f, vv = 0.f, vA = 0.f, vB = 0.f, vC = 0.f, vo = 0.f, vr = 0.f, vg = 0.f, vb = 0.f;
       if (on) {
+        const float G = __expf(power);
+        const float og = q1.w * G;
+        const float alpha = fminf(alpha_max, og);
         const float inv = __fdividef(1.f, 1.f - alpha);
         const float Tb = T * inv;  // transmittance in front of this row
         const float w = alpha * Tb;
-        const float c0 = q0.z, c1 = q0.w, c2 = s_blue[j];
+        const float c0 = q0.z, c1 = q0.w, c2 = bp.x;
         vr = w * g0; vg = w * g1; vb = w * g2;
         const float dLda = (c0 * Tb - S0 * inv) * g0 + (c1 * Tb - S1 * inv) * g1 + (c2 * Tb - S2 * inv) * g2;
         S0 = fmaf(c0, w, S0); S1 = fmaf(c1, w, S1); S2 = fmaf(c2, w, S2);
@@ -154,14 +155,20 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
                         int n_tiles, float bg0, float bg1, float bg2, float alpha_min, float alpha_max,
                         const float* __restrict__ state,
                         const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
-                        const float* __restrict__ dL, float* __restrict__ g2d) {
+                        const float* __restrict__ dL, float* __restrict__ g2d, uint32_t* __restrict__ ticket) {
   __shared__ BlendRow s_rowdata[BLEND_WARPS][32];
-  __shared__ float s_blue[BLEND_WARPS][32];
+  __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, power threshold
   __shared__ uint32_t s_rowid[BLEND_WARPS][32];
+  __shared__ float4 s_ext[BLEND_WARPS][32];  // box outside of which the row cannot contribute
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int tile = blockIdx.x * BLEND_WARPS + warp;
-  if (tile >= n_tiles) return;  // warps never synchronise with each other
+  // warps never synchronise with each other; each keeps taking tiles from a ticket counter (see the forward kernel)
+  while (true) {
+  int tile = 0;
+  if (lane == 0) tile = (int)atomicAdd(ticket, 1u);
+  tile = __shfl_sync(0xffffffffu, tile, 0);
+  if (tile >= n_tiles) return;
   const int tx = tile % TX, ty = tile / TX;
+  const float tile_x0 = (float)(tx * 16), tile_y0 = (float)(ty * 16);
   const int px = tx * 16 + (int)(lane & 15);
   const int py0 = ty * 16 + (int)(lane >> 4);
   const float fx = (float)px + 0.5f, fy0 = (float)py0 + 0.5f;
@@ -211,31 +218,45 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
       row.q1 = conic_o[r];
       s_rowdata[warp][lane] = row;
-      s_blue[warp][lane] = rgb[3 * (size_t)r + 2];
+      const float cut = blend_power_cut(alpha_min, row.q1.w);
+      s_blue[warp][lane] = make_float2(rgb[3 * (size_t)r + 2], cut);
+      s_ext[warp][lane] = blend_extent(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, cut);
       s_rowid[warp][lane] = r;
     }
     __syncwarp();
     for (int j = cnt - 1; j >= 0; --j) {
+      // warp-uniform: a row whose box misses the tile is not evaluated at all
+      const float4 ext = s_ext[warp][j];
+      if (ext.y < tile_x0 + 0.5f || ext.x > tile_x0 + 15.5f || ext.w < tile_y0 + 0.5f || ext.z > tile_y0 + 15.5f)
+        continue;
       const float4 q0 = s_rowdata[warp][j].q0, q1 = s_rowdata[warp][j].q1;
-      const float blue = s_blue[warp][j];
+      const float blue = s_blue[warp][j].x, pcut = s_blue[warp][j].y;
       const float dx = q0.x - fx;
       const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
       const float dy0 = q0.y - fy0;
       const uint32_t k = b + j;
-      // per-lane sums over its eight pixels; the x-dependent factors are applied once at the end
-      float ar = 0.f, ag = 0.f, ab = 0.f, ao = 0.f, gpsum = 0.f, m1y = 0.f, m2yy = 0.f;
-      bool any = false;
+      // phase 1, straight line: the eight exponents and skip tests are independent and overlap in the pipeline
+      float pw[BLEND_SLOTS];
+      uint32_t pass = 0;
 #pragma unroll
       for (int s = 0; s < BLEND_SLOTS; ++s) {
-        const float dy = dy0 - (float)(2 * s);
-        const float power = blend_power(h0, h1, h2, dy);
-        const float G = __expf(power);
-        const float og = q1.w * G;
-        const float alpha = fminf(alpha_max, og);
-        const bool on = (k < last[s]) && (power <= 0.f) && (alpha >= alpha_min);
-        if (__any_sync(0xffffffffu, on)) {
-          any = true;
-          if (on) {
+        pw[s] = blend_power(h0, h1, h2, dy0 - (float)(2 * s));
+        pass |= (k < last[s] && pw[s] <= 0.f && pw[s] >= pcut) ? (1u << s) : 0u;
+      }
+      const uint32_t hit = __reduce_or_sync(0xffffffffu, pass);  // bit s: some lane of the warp passes in slot s
+      if (hit == 0) continue;
+      // phase 2: per-lane sums over its eight pixels; the x-dependent factors are applied once at the end
+      float ar = 0.f, ag = 0.f, ab = 0.f, ao = 0.f, gpsum = 0.f, m1y = 0.f, m2yy = 0.f;
+#pragma unroll
+      for (int s = 0; s < BLEND_SLOTS; ++s) {
+        if (!(hit >> s & 1u)) continue;
+        {
+          if (pass >> s & 1u) {
+            const float dy = dy0 - (float)(2 * s);
+            const float power = pw[s];
+            const float G = __expf(power);
+            const float og = q1.w * G;
+            const float alpha = fminf(alpha_max, og);
             const float inv = __fdividef(1.f, 1.f - alpha);
             const float Tb = T[s] * inv;  // transmittance in front of this row
             const float w = alpha * Tb;
@@ -256,7 +277,6 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
           }
         }
       }
-      if (!any) continue;  // warp-uniform: `any` was set from warp votes
       const float gd = dx * gpsum;  // sum of dL/dpower * dx
       const float vu = -(q1.x * gd + q1.y * m1y);
       const float vv = -(q1.z * m1y + q1.y * gd);
@@ -268,6 +288,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       if (lane == 1) atomicAdd(dst + 8, ab);
     }
     __syncwarp();
+  }
   }
 }
 
@@ -437,6 +458,8 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
   }
   const int n_tiles = TX * TY;
   float* state = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + blend_ws_flags_bytes(n_tiles));
+  uint32_t* ticket = reinterpret_cast<uint32_t*>(ws) + 1;
+  ODIN_CUDA(cudaMemsetAsync(ticket, 0, 4, st));
   {
     OdinKernelScope ks(ctx, K_BWD_TAIL, st);
     render_bwd_tail_kernel<<<n_tiles, BLEND_TAIL_THREADS, 0, st>>>(
@@ -446,10 +469,13 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
   }
   {
     OdinKernelScope ks(ctx, K_BWD_BLEND, st);
-    render_bwd_blend_kernel<<<(n_tiles + BLEND_WARPS - 1) / BLEND_WARPS, BLEND_THREADS, 0, st>>>(
+    const int blocks_all = (n_tiles + BLEND_WARPS - 1) / BLEND_WARPS;
+    const int blocks = blocks_all < ctx->sm_count * 8 ? blocks_all : ctx->sm_count * 8;  // resident warps pull tiles
+    render_bwd_blend_kernel<<<blocks, BLEND_THREADS, 0, st>>>(
         reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
         reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0], cam->bg[1],
-        cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, state, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d);
+        cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, state, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d,
+        ticket);
   }
   const CamParams cp = odin_cam_params(cam, ctx->cfg);
   const uint32_t blocks_cap = (proj->capacity + 127) / 128;

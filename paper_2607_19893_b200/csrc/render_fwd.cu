@@ -11,16 +11,25 @@ __global__ void __launch_bounds__(BLEND_THREADS)
 render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
                   const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX, int n_tiles,
                   float bg0, float bg1, float bg2, float alpha_min, float alpha_max, float t_min, float* __restrict__ out,
-                  float* __restrict__ final_T, uint32_t* __restrict__ n_contrib, uint32_t* __restrict__ tile_more) {
+                  float* __restrict__ final_T, uint32_t* __restrict__ n_contrib, uint32_t* __restrict__ tile_more,
+                  uint32_t* __restrict__ ticket) {
   __shared__ BlendRow s_row[BLEND_WARPS][32];
-  __shared__ float s_blue[BLEND_WARPS][32];
+  __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, power threshold
+  __shared__ float4 s_ext[BLEND_WARPS][32];   // box outside of which the row cannot contribute
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int tile = blockIdx.x * BLEND_WARPS + warp;
-  if (tile >= n_tiles) return;  // warps never synchronise with each other
+  // Warps never synchronise with each other.  Each one keeps taking tiles from a ticket counter until none is left:
+  // lists differ in length by orders of magnitude between tiles, and a fixed tile-to-warp map would leave most of the
+  // GPU idle while the longest ones finish.
+  while (true) {
+  int tile = 0;
+  if (lane == 0) tile = (int)atomicAdd(ticket, 1u);
+  tile = __shfl_sync(0xffffffffu, tile, 0);
+  if (tile >= n_tiles) return;
   const int tx = tile % TX, ty = tile / TX;
   const int px = tx * 16 + (int)(lane & 15);
   const int py0 = ty * 16 + (int)(lane >> 4);
   const float fx = (float)px + 0.5f, fy0 = (float)py0 + 0.5f;
+  const float tile_x0 = (float)(tx * 16), tile_y0 = (float)(ty * 16);
   const uint2 rg = ranges[tile];
   const uint32_t start = rg.x;
   const uint32_t end = min(rg.y, rg.x + BLEND_HEAD);
@@ -45,23 +54,39 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
       row.q1 = conic_o[r];
       s_row[warp][lane] = row;
-      s_blue[warp][lane] = rgb[3 * (size_t)r + 2];
+      const float cut = blend_power_cut(alpha_min, row.q1.w);
+      s_blue[warp][lane] = make_float2(rgb[3 * (size_t)r + 2], cut);
+      s_ext[warp][lane] = blend_extent(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, cut);
     }
     __syncwarp();
     const int cnt = (int)min(32u, end - b);
     for (int j = 0; j < cnt; ++j) {
+      // warp-uniform: a row whose box misses the tile is not evaluated at all
+      const float4 ext = s_ext[warp][j];
+      if (ext.y < tile_x0 + 0.5f || ext.x > tile_x0 + 15.5f || ext.w < tile_y0 + 0.5f || ext.z > tile_y0 + 15.5f)
+        continue;
       const float4 q0 = s_row[warp][j].q0, q1 = s_row[warp][j].q1;
-      const float blue = s_blue[warp][j];
+      const float blue = s_blue[warp][j].x, pcut = s_blue[warp][j].y;
       const float dx = q0.x - fx;
       const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
       const float dy0 = q0.y - fy0;
       const uint32_t ord = (b - start) + j + 1;
+      // phase 1, straight line: the eight exponents and skip tests are independent and overlap in the pipeline
+      float power[BLEND_SLOTS];
+      uint32_t pass = 0;
 #pragma unroll
       for (int s = 0; s < BLEND_SLOTS; ++s) {
-        const float dy = dy0 - (float)(2 * s);
-        const float power = blend_power(h0, h1, h2, dy);
-        const float alpha = fminf(alpha_max, q1.w * __expf(power));
-        if ((live >> s & 1u) && power <= 0.f && alpha >= alpha_min) {
+        power[s] = blend_power(h0, h1, h2, dy0 - (float)(2 * s));
+        pass |= (power[s] <= 0.f && power[s] >= pcut) ? (1u << s) : 0u;
+      }
+      pass &= live;
+      // phase 2: ex2 and the blend, only for slots in which some lane passes
+      const uint32_t hit = __reduce_or_sync(0xffffffffu, pass);  // bit s: some lane of the warp passes in slot s
+#pragma unroll
+      for (int s = 0; s < BLEND_SLOTS; ++s) {
+        if (!(hit >> s & 1u)) continue;
+        if (pass >> s & 1u) {
+          const float alpha = fminf(alpha_max, q1.w * __expf(power[s]));
           const float Tn = T[s] * (1.f - alpha);
           if (Tn < t_min) {
             live &= ~(1u << s);
@@ -93,6 +118,8 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
       n_contrib[pix] = last[s] | ((more && !(live >> s & 1u)) ? BLEND_DONE_BIT : 0u);
     }
   }
+  __syncwarp();  // the staging arrays are reused by the next tile
+  }
 }
 
 // Tail: one block of 256 threads per tile that the head kernel left unfinished, one pixel per thread, rows staged 256
@@ -106,7 +133,7 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
   const int tile = blockIdx.x;
   if (!tile_more[tile]) return;
   __shared__ BlendRow s_row[BLEND_TAIL_THREADS];
-  __shared__ float s_blue[BLEND_TAIL_THREADS];
+  __shared__ float2 s_blue[BLEND_TAIL_THREADS];  // blue, power threshold
   const int tx = tile % TX, ty = tile / TX;
   const int lx = threadIdx.x & 15, ly = threadIdx.x >> 4;
   const int px = tx * 16 + lx, py = ty * 16 + ly;
@@ -137,7 +164,7 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
       row.q1 = conic_o[r];
       s_row[threadIdx.x] = row;
-      s_blue[threadIdx.x] = rgb[3 * (size_t)r + 2];
+      s_blue[threadIdx.x] = make_float2(rgb[3 * (size_t)r + 2], blend_power_cut(alpha_min, row.q1.w));
     }
     __syncthreads();
     const int cnt = (int)min((uint32_t)BLEND_TAIL_THREADS, end - b);
@@ -148,13 +175,13 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
         const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
         const float dy = (q0.y - fy0) - slot2;
         const float power = blend_power(h0, h1, h2, dy);
-        if (power > 0.f) continue;
+        const float2 bp = s_blue[j];
+        if (!(power <= 0.f && power >= bp.y)) continue;
         const float alpha = fminf(alpha_max, q1.w * __expf(power));
-        if (alpha < alpha_min) continue;
         const float Tn = T * (1.f - alpha);
         if (Tn < t_min) { done = true; break; }
         const float w = alpha * T;
-        C0 = fmaf(q0.z, w, C0); C1 = fmaf(q0.w, w, C1); C2 = fmaf(s_blue[j], w, C2);
+        C0 = fmaf(q0.z, w, C0); C1 = fmaf(q0.w, w, C1); C2 = fmaf(bp.x, w, C2);
         T = Tn;
         last = (b - start) + j + 1;
       }
@@ -214,14 +241,19 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
   const int TX = (cam->width + 15) / 16, TY = (cam->height + 15) / 16;
   const int n_tiles = TX * TY;
   if (!ws || !odin_aligned(ws, 256) || ws_bytes < blend_ws_flags_bytes(n_tiles)) return ODIN_ERR_WORKSPACE;
-  uint32_t* tile_more = reinterpret_cast<uint32_t*>(ws);
+  uint32_t* ticket = reinterpret_cast<uint32_t*>(ws);
+  uint32_t* tile_more = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + BLEND_WS_HEADER);
   cudaStream_t st = (cudaStream_t)stream;
+  ODIN_CUDA(cudaMemsetAsync(ticket, 0, 4, st));
   {
     OdinKernelScope ks(ctx, K_FWD, st);
-    render_fwd_kernel<<<(n_tiles + BLEND_WARPS - 1) / BLEND_WARPS, BLEND_THREADS, 0, st>>>(
+    const int blocks_all = (n_tiles + BLEND_WARPS - 1) / BLEND_WARPS;
+    const int blocks = blocks_all < ctx->sm_count * 8 ? blocks_all : ctx->sm_count * 8;  // resident warps pull tiles
+    render_fwd_kernel<<<blocks, BLEND_THREADS, 0, st>>>(
         reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
         reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0], cam->bg[1],
-        cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_more);
+        cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_more,
+        ticket);
   }
   OdinKernelScope ks(ctx, K_FWD_TAIL, st);
   render_fwd_tail_kernel<<<n_tiles, BLEND_TAIL_THREADS, 0, st>>>(

@@ -203,7 +203,7 @@ DEFAULT_LR = np.full(6, 1e-3, dtype=np.float32)
 
 
 def make_workload(cfg: int, n: Optional[int] = None, n_cameras: Optional[int] = None,
-                  resolution: Optional[tuple] = None) -> Workload:
+                  resolution: Optional[tuple] = None, city_grid: Optional[int] = None) -> Workload:
     """Build preset `cfg` (1..5).  `n`, `n_cameras`, `resolution=(W,H)` scale it down for tests;
     focal length scales with the width so the field of view is kept."""
     seed = 1000 * cfg
@@ -247,8 +247,13 @@ def make_workload(cfg: int, n: Optional[int] = None, n_cameras: Optional[int] = 
         return Workload(4, "cfg4_5m_sh3_1920x1080", Scene(3, means, ls, q, lo, sh), cams, 64, DEFAULT_LR.copy(),
                         conflict_window=4, seed_base=seed)
     if cfg == 5:
-        n = n or 20_000_000
         grid, pitch_m = 64, 30.0
+        if city_grid is not None:
+            # a smaller city at the SAME density per block (what a camera sees is unchanged): used for profiler
+            # captures, which must keep only a few GB on the device
+            grid = int(city_grid)
+            n = n or int(round(20_000_000 * (grid / 64.0) ** 2))
+        n = n or 20_000_000
         # per-block Poisson counts, rescaled to sum to n; primitives are stored block by block
         counts = rng.poisson(n / (grid * grid), grid * grid).astype(np.int64)
         diff = n - int(counts.sum())
