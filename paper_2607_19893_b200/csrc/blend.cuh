@@ -14,7 +14,7 @@
 // tail of the whole launch.  The per-pixel state travels through the output images (forward) or a workspace
 // (backward).  Both kernels evaluate dy as (v - (y0 + 0.5)) - 2 s with y0 the first row of the lane's slot pair, so a
 // pixel sees bit-identical power / alpha in either.
-constexpr uint32_t BLEND_HEAD = 512;
+constexpr uint32_t BLEND_HEAD = 256;
 constexpr uint32_t BLEND_DONE_BIT = 0x80000000u;  // in n_contrib while a tile is between the two kernels
 constexpr int BLEND_TAIL_THREADS = 256;
 

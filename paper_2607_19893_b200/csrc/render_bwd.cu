@@ -93,15 +93,29 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
       s_rowid[threadIdx.x] = r;
     }
     __syncthreads();
-    for (int j = cnt - 1; j >= 0; --j) {
+    for (int j4 = cnt - 1; j4 >= 0; j4 -= 4) {
+      // four rows at a time (back to front): exponents and skip tests first, they are independent of each other
+      float pw4[4];
+      bool on4[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int ju = max(j4 - u, 0);
+        const float4 q0 = s_rowdata[ju].q0, q1 = s_rowdata[ju].q1;
+        const float dx = q0.x - fx;
+        const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
+        pw4[u] = blend_power(h0, h1, h2, (q0.y - fy0) - slot2);
+        on4[u] = (j4 - u >= 0) && (b + ju < last) && (pw4[u] <= 0.f) && (pw4[u] >= s_blue[ju].y);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+      const int j = j4 - u;
+      const bool on = on4[u];
+      if (__ballot_sync(0xffffffffu, on) == 0) continue;
       const float4 q0 = s_rowdata[j].q0, q1 = s_rowdata[j].q1;
       const float2 bp = s_blue[j];
       const float dx = q0.x - fx;
-      const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
       const float dy = (q0.y - fy0) - slot2;
-      const float power = blend_power(h0, h1, h2, dy);
-      const bool on = (b + j < last) && (power <= 0.f) && (power >= bp.y);
-      if (__ballot_sync(0xffffffffu, on) == 0) continue;
+      const float power = pw4[u];
       float vu = 0.f, vv = 0.f, vA = 0.f, vB = 0.f, vC = 0.f, vo = 0.f, vr = 0.f, vg = 0.f, vb = 0.f;
       if (on) {
         const float G = __expf(power);
@@ -130,6 +144,7 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
       for (int o = 16; o > 0; o >>= 1) vb += __shfl_xor_sync(0xffffffffu, vb, o);
       if ((lane & 3) == 0) atomicAdd(&s_acc[j * 9 + (lane >> 2)], t8);
       if (lane == 1) atomicAdd(&s_acc[j * 9 + 8], vb);
+      }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < cnt * 9; i += BB) {

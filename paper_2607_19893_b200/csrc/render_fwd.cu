@@ -169,21 +169,37 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
     __syncthreads();
     const int cnt = (int)min((uint32_t)BLEND_TAIL_THREADS, end - b);
     if (!done) {
-      for (int j = 0; j < cnt; ++j) {
-        const float4 q0 = s_row[j].q0, q1 = s_row[j].q1;
-        const float dx = q0.x - fx;
-        const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
-        const float dy = (q0.y - fy0) - slot2;
-        const float power = blend_power(h0, h1, h2, dy);
-        const float2 bp = s_blue[j];
-        if (!(power <= 0.f && power >= bp.y)) continue;
-        const float alpha = fminf(alpha_max, q1.w * __expf(power));
-        const float Tn = T * (1.f - alpha);
-        if (Tn < t_min) { done = true; break; }
-        const float w = alpha * T;
-        C0 = fmaf(q0.z, w, C0); C1 = fmaf(q0.w, w, C1); C2 = fmaf(bp.x, w, C2);
-        T = Tn;
-        last = (b - start) + j + 1;
+      // four rows at a time: their exponents and skip tests are independent (a single pixel per thread has no other
+      // source of instruction-level parallelism), the blends are then applied in order
+      for (int j = 0; j < cnt && !done; j += 4) {
+        float pw[4], opac[4], cr[4], cg[4], cb[4];
+        bool pass[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int ju = min(j + u, cnt - 1);
+          const float4 q0 = s_row[ju].q0, q1 = s_row[ju].q1;
+          const float2 bp = s_blue[ju];
+          const float dx = q0.x - fx;
+          const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
+          pw[u] = blend_power(h0, h1, h2, (q0.y - fy0) - slot2);
+          pass[u] = (j + u < cnt) && pw[u] <= 0.f && pw[u] >= bp.y;
+          opac[u] = q1.w; cr[u] = q0.z; cg[u] = q0.w; cb[u] = bp.x;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (pass[u] && !done) {
+            const float alpha = fminf(alpha_max, opac[u] * __expf(pw[u]));
+            const float Tn = T * (1.f - alpha);
+            if (Tn < t_min) {
+              done = true;
+            } else {
+              const float w = alpha * T;
+              C0 = fmaf(cr[u], w, C0); C1 = fmaf(cg[u], w, C1); C2 = fmaf(cb[u], w, C2);
+              T = Tn;
+              last = (b - start) + j + u + 1;
+            }
+          }
+        }
       }
     }
   }
