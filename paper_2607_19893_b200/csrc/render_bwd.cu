@@ -75,7 +75,9 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
   const uint32_t total = s_max;
   if (total <= BLEND_HEAD) return;  // uniform over the block: the head kernel does the whole tile
   for (int i = threadIdx.x; i < BB * 9; i += BB) s_acc[i] = 0.f;
-  float S0 = T * bg0, S1 = T * bg1, S2 = T * bg2;
+  // Only the suffix colour's product with the pixel's incoming gradient is ever needed, so one scalar is carried:
+  // SG = sum_ch S_ch g_ch with S = sum_{j>k} c_j alpha_j T_j + T_final bg.
+  float SG = T * (bg0 * g0 + bg1 * g1 + bg2 * g2);
   const uint32_t span = total - BLEND_HEAD;
   const int nb = (int)((span + BB - 1) / BB);
   for (int bi = nb - 1; bi >= 0; --bi) {
@@ -126,8 +128,9 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
         const float w = alpha * Tb;
         const float c0 = q0.z, c1 = q0.w, c2 = bp.x;
         vr = w * g0; vg = w * g1; vb = w * g2;
-        const float dLda = (c0 * Tb - S0 * inv) * g0 + (c1 * Tb - S1 * inv) * g1 + (c2 * Tb - S2 * inv) * g2;
-        S0 = fmaf(c0, w, S0); S1 = fmaf(c1, w, S1); S2 = fmaf(c2, w, S2);
+        const float cg = fmaf(c2, g2, fmaf(c1, g1, c0 * g0));
+        const float dLda = Tb * cg - SG * inv;
+        SG = fmaf(w, cg, SG);
         T = Tb;
         if (og <= alpha_max) {
           const float t = G * dLda;
@@ -156,7 +159,7 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
     }
   }
   if (inside) {
-    state[pix] = T; state[plane + pix] = S0; state[2 * plane + pix] = S1; state[3 * plane + pix] = S2;
+    state[pix] = T; state[plane + pix] = SG;
   }
 }
 
@@ -190,7 +193,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
   const uint32_t start = ranges[tile].x;
   const size_t plane = (size_t)W * H;
 
-  float T[BLEND_SLOTS], S0[BLEND_SLOTS], S1[BLEND_SLOTS], S2[BLEND_SLOTS];
+  float T[BLEND_SLOTS], SG[BLEND_SLOTS];  // SG: suffix colour times the pixel's incoming gradient (see the tail kernel)
   float g0[BLEND_SLOTS], g1[BLEND_SLOTS], g2[BLEND_SLOTS];
   uint32_t last[BLEND_SLOTS];
   uint32_t total = 0;
@@ -204,7 +207,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       last[s] = n_contrib[pix];
       g0[s] = dL[pix]; g1[s] = dL[plane + pix]; g2[s] = dL[2 * plane + pix];
     }
-    S0[s] = T[s] * bg0; S1[s] = T[s] * bg1; S2[s] = T[s] * bg2;
+    SG[s] = T[s] * (bg0 * g0[s] + bg1 * g1[s] + bg2 * g2[s]);
     total = max(total, last[s]);
   }
   for (int o = 16; o > 0; o >>= 1) total = max(total, __shfl_xor_sync(0xffffffffu, total, o));
@@ -217,7 +220,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       const int py = py0 + 2 * s;
       if (px < W && py < H) {
         const size_t pix = (size_t)py * W + px;
-        T[s] = state[pix]; S0[s] = state[plane + pix]; S1[s] = state[2 * plane + pix]; S2[s] = state[3 * plane + pix];
+        T[s] = state[pix]; SG[s] = state[plane + pix];
       }
     }
   }
@@ -276,9 +279,9 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
             const float Tb = T[s] * inv;  // transmittance in front of this row
             const float w = alpha * Tb;
             ar = fmaf(w, g0[s], ar); ag = fmaf(w, g1[s], ag); ab = fmaf(w, g2[s], ab);
-            const float dLda = (q0.z * Tb - S0[s] * inv) * g0[s] + (q0.w * Tb - S1[s] * inv) * g1[s] +
-                               (blue * Tb - S2[s] * inv) * g2[s];
-            S0[s] = fmaf(q0.z, w, S0[s]); S1[s] = fmaf(q0.w, w, S1[s]); S2[s] = fmaf(blue, w, S2[s]);
+            const float cg = fmaf(blue, g2[s], fmaf(q0.w, g1[s], q0.z * g0[s]));
+            const float dLda = Tb * cg - SG[s] * inv;
+            SG[s] = fmaf(w, cg, SG[s]);
             T[s] = Tb;
             if (og <= alpha_max) {  // a clamped alpha passes no gradient to opacity or geometry
               const float t = G * dLda;

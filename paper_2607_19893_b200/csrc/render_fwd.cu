@@ -7,7 +7,7 @@
 
 namespace {
 
-__global__ void __launch_bounds__(BLEND_THREADS)
+__global__ void __launch_bounds__(BLEND_THREADS, 7)  // 7 blocks = 28 warps per SM: the kernel is latency-bound
 render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
                   const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX, int n_tiles,
                   float bg0, float bg1, float bg2, float alpha_min, float alpha_max, float t_min, float* __restrict__ out,
