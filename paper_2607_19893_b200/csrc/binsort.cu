@@ -56,6 +56,8 @@ emit_instances_kernel(const uint32_t* __restrict__ tile_offset, const uint32_t* 
   __shared__ ushort4 s_rect[DUP_CHUNK];
   __shared__ uint32_t s_depth[DUP_CHUNK];
   __shared__ uint32_t s_hist[SORT_MAX_PASSES][SORT_RADIX];
+  __shared__ __align__(16) uint16_t s_map[DUP_CHUNK];  // slot of the chunk -> row of the chunk
+  __shared__ uint32_t s_scan[DUP_THREADS / 32];
   const uint32_t V = *num_rows;
   const uint64_t M_all = *num_instances;
   const uint64_t M64 = M_all < capacity ? M_all : capacity;
@@ -84,6 +86,36 @@ emit_instances_kernel(const uint32_t* __restrict__ tile_offset, const uint32_t* 
       s_depth[i] = __float_as_uint(depth[row_lo + i]);
     }
     if (threadIdx.x == 0) s_off[nrows] = (row_hi + 1 < V) ? tile_offset[row_hi + 1] : (uint32_t)M_all;
+    for (int i = threadIdx.x; i < DUP_CHUNK; i += DUP_THREADS) s_map[i] = 0;
+    __syncthreads();
+    // slot -> row of the chunk: every row marks its first slot, an inclusive max-scan fills the rest
+    for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS)
+      s_map[max(s_off[i], c0) - c0] = (uint16_t)i;
+    __syncthreads();
+    {
+      static_assert(DUP_ITEMS == 8, "a thread's slots are one 16-byte word of the map");
+      uint4* map4 = reinterpret_cast<uint4*>(s_map) + threadIdx.x;
+      const uint4 raw = *map4;
+      const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+      uint32_t m[DUP_ITEMS];
+      uint32_t run = 0;
+#pragma unroll
+      for (int k = 0; k < DUP_ITEMS; ++k) {
+        run = max(run, (rw[k >> 1] >> (16 * (k & 1))) & 0xffffu);
+        m[k] = run;
+      }
+      uint32_t inc = run;  // inclusive max over the threads of the warp
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) inc = max(inc, __shfl_up_sync(0xffffffffu, inc, o, 32) * (lane >= (unsigned)o ? 1u : 0u));
+      if (lane == 31) s_scan[threadIdx.x >> 5] = inc;
+      __syncthreads();
+      uint32_t before = __shfl_up_sync(0xffffffffu, inc, 1);
+      if (lane == 0) before = 0;
+      for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) before = max(before, s_scan[w]);
+#pragma unroll
+      for (int k = 0; k < DUP_ITEMS; ++k) m[k] = max(m[k], before);
+      *map4 = make_uint4(m[0] | (m[1] << 16), m[2] | (m[3] << 16), m[4] | (m[5] << 16), m[6] | (m[7] << 16));
+    }
     __syncthreads();
     // depth digits, once per row
     for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS) {
@@ -100,11 +132,7 @@ emit_instances_kernel(const uint32_t* __restrict__ tile_offset, const uint32_t* 
       uint32_t tile = 0xffffffffu;
       uint64_t key = 0;
       if (valid) {
-        uint32_t lo = 0, hi = nrows;  // last j with s_off[j] <= i
-        while (hi - lo > 1) {
-          const uint32_t mid = (lo + hi) >> 1;
-          if (s_off[mid] <= i) lo = mid; else hi = mid;
-        }
+        const uint32_t lo = s_map[i - c0];  // row of the chunk that owns this slot
         const ushort4 rc = s_rect[lo];
         const uint32_t local = i - s_off[lo];
         const uint32_t w = (uint32_t)rc.z - (uint32_t)rc.x;
