@@ -167,9 +167,11 @@ int odin_touched_set_static(const uint32_t* d_tiles_touched, uint32_t n, uint32_
 
 /* Binning and sort.  Emits one (key, value) per (tile, row) pair of the rectangles: key = tile_id << 32 | bit pattern
  * of the float32 depth, tile_id = ty * ceil(width/16) + tx; value = ROW index r (the primitive is proj->prim_id[r]).
- * Sorts by key with a least-significant-digit radix sort (stable: equal keys keep ascending row order) and writes
- * d_tile_ranges [tiles][2] = [first, one past last) position of each tile (an empty tile has first == last).
- * Only the first `capacity` instances are produced when M > capacity (ODIN_ERR_CAPACITY deferred). */
+ * The result is the order of a stable least-significant-digit radix sort by key (equal keys keep ascending row order):
+ * d_vals [capacity] the sorted values, d_keys [capacity] the sorted keys (may be NULL when only the values are wanted:
+ * the later calls read d_vals and d_tile_ranges only), d_tile_ranges [tiles][2] = [first, one past last) position of
+ * each tile (an empty tile has first == last).
+ * When M > capacity only the `capacity` instances of the nearest rows are produced (ODIN_ERR_CAPACITY deferred). */
 int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int width, int height, uint64_t* d_keys, uint32_t* d_vals,
                   uint64_t capacity, uint32_t* d_tile_ranges, void* ws, size_t ws_bytes, void* stream);
 

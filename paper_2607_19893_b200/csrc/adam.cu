@@ -51,7 +51,8 @@ adam_sh_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__
   }
 }
 
-// Geometry block: one thread per row handles mean(3), log scale(3), quaternion(4), opacity(1).
+// Geometry block: four threads per row - mean(3), log scale(3), quaternion(4), opacity(1) - so that a row's twelve
+// gathers are spread over four independent threads instead of queueing in one.
 __global__ void __launch_bounds__(256)
 adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* __restrict__ p_q, float* __restrict__ p_o,
                  float* __restrict__ m_mean, float* __restrict__ m_ls, float4* __restrict__ m_q, float* __restrict__ m_o,
@@ -60,21 +61,25 @@ adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* _
                  const float* __restrict__ g_o, const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count,
                  uint32_t cap, AdamK k) {
   const uint32_t V = min(*count, cap);
-  for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
+  const size_t total = (size_t)V * 4;
+  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+    const uint32_t r = (uint32_t)(e >> 2);
+    const int part = (int)(e & 3);
     const size_t d = idx[r];
+    if (part < 2) {
+      float* __restrict__ p = (part ? p_ls : p_mean) + 3 * d;
+      float* __restrict__ m = (part ? m_ls : m_mean) + 3 * d;
+      float* __restrict__ v = (part ? v_ls : v_mean) + 3 * d;
+      const float* __restrict__ g = (part ? g_ls : g_mean) + 3 * (size_t)r;
+      const float ss = k.step_size[part];
+      float pp[3], mm[3], vv[3], gg[3];
 #pragma unroll
-    for (int i = 0; i < 3; ++i) {
-      float pp = p_mean[3 * d + i], mm = m_mean[3 * d + i], vv = v_mean[3 * d + i];
-      adam_one(pp, mm, vv, g_mean[3 * (size_t)r + i], k.step_size[0], k);
-      p_mean[3 * d + i] = pp; m_mean[3 * d + i] = mm; v_mean[3 * d + i] = vv;
-    }
+      for (int i = 0; i < 3; ++i) { pp[i] = p[i]; mm[i] = m[i]; vv[i] = v[i]; gg[i] = g[i]; }
 #pragma unroll
-    for (int i = 0; i < 3; ++i) {
-      float pp = p_ls[3 * d + i], mm = m_ls[3 * d + i], vv = v_ls[3 * d + i];
-      adam_one(pp, mm, vv, g_ls[3 * (size_t)r + i], k.step_size[1], k);
-      p_ls[3 * d + i] = pp; m_ls[3 * d + i] = mm; v_ls[3 * d + i] = vv;
-    }
-    {
+      for (int i = 0; i < 3; ++i) adam_one(pp[i], mm[i], vv[i], gg[i], ss, k);
+#pragma unroll
+      for (int i = 0; i < 3; ++i) { p[i] = pp[i]; m[i] = mm[i]; v[i] = vv[i]; }
+    } else if (part == 2) {
       float4 pp = p_q[d], mm = m_q[d], vv = v_q[d];
       const float4 gg = g_q[r];
       adam_one(pp.x, mm.x, vv.x, gg.x, k.step_size[2], k);
@@ -82,8 +87,7 @@ adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* _
       adam_one(pp.z, mm.z, vv.z, gg.z, k.step_size[2], k);
       adam_one(pp.w, mm.w, vv.w, gg.w, k.step_size[2], k);
       p_q[d] = pp; m_q[d] = mm; v_q[d] = vv;
-    }
-    {
+    } else {
       float pp = p_o[d], mm = m_o[d], vv = v_o[d];
       adam_one(pp, mm, vv, g_o[r], k.step_size[3], k);
       p_o[d] = pp; m_o[d] = mm; v_o[d] = vv;
@@ -131,7 +135,7 @@ extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m
     default: adam_sh_kernel<48, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
     }
   }
-  size_t gb = ((size_t)cap + 255) / 256;
+  size_t gb = ((size_t)cap * 4 + 255) / 256;
   if (gb > (size_t)ctx->sm_count * 16) gb = (size_t)ctx->sm_count * 16;
   OdinKernelScope ks(ctx, K_ADAM_GEOM, st);
   adam_geom_kernel<<<(unsigned)gb, 256, 0, st>>>(

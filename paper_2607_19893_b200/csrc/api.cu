@@ -71,7 +71,8 @@ extern "C" int odin_poll(odin_ctx* ctx, void* stream) {
 static const char* const kKernelNames[K_COUNT] = {
     "project_cull", "touched_set", "emit_instances", "digit_base", "onesweep_pass", "tile_ranges", "render_fwd", "l1_loss",
     "l1_finish", "zero_rows", "render_bwd_blend", "render_bwd_project", "adam_sh", "adam_geom", "conflict_count",
-    "render_fwd_tail", "render_bwd_tail", "project_scan", "project_rows", "chunk_rows"};
+    "render_fwd_tail", "render_bwd_tail", "project_scan", "project_rows", "chunk_rows", "row_hist",
+    "row_sort_pass", "row_offsets"};
 
 extern "C" int odin_kernel_count(void) { return K_COUNT; }
 
@@ -104,7 +105,7 @@ extern "C" int odin_workspace_bytes(const odin_ctx* ctx, uint32_t n, uint64_t ma
   if (!ctx || !bytes) return ODIN_ERR_NULL;
   size_t b = project_ws_bytes(n);
   const size_t t = touched_ws_bytes(n);
-  const size_t s = binsort_ws_bytes(max_instances);
+  const size_t s = binsort_ws_bytes(max_instances, n);  // a view has at most n rows
   if (t > b) b = t;
   if (s > b) b = s;
   *bytes = b;

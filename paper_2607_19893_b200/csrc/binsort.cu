@@ -1,157 +1,39 @@
-// Tile binning and sort: instance emission (load balanced over instances), digit histograms, a onesweep
-// least-significant-digit radix sort with decoupled look-back (no library sort), and the per-tile ranges.
+// Tile binning and sort.  The order asked for is that of a stable least-significant-digit radix sort of the instance
+// keys tile_id << 32 | depth bits.  All instances of a row share the row's depth, so the passes over the depth digits are
+// taken on the ROWS (several times fewer than the instances): rows are sorted by depth, the instances are emitted in
+// that order (load balanced over instances), and only the passes over the tile-id digits run on the instances.  The
+// result is the very sequence the full-width sort produces: after the depth passes an instance list is ordered by
+// (depth, row, position in the row's rectangle) either way.  Every pass is a onesweep pass with decoupled look-back
+// (no library sort); the per-tile ranges are read off the sorted tile ids.
 #include "common.cuh"
 #include "layout.cuh"
 
 namespace {
 
-// ------------------------------------------------------------------------------------------------ emission
-constexpr int DUP_THREADS = 256;
-constexpr int DUP_ITEMS = 8;
-constexpr int DUP_CHUNK = DUP_THREADS * DUP_ITEMS;  // instances per chunk; a chunk spans at most DUP_CHUNK rows
-
-// Cooperative 256-ary upper bound: first r in [0, V) with off[r] > x (V if none).  All threads must call.
-__device__ __forceinline__ uint32_t block_upper_bound(const uint32_t* __restrict__ off, uint32_t V, uint32_t x) {
-  uint32_t lo = 0, hi = V;
-  while (lo < hi) {
-    const uint32_t span = hi - lo;
-    const uint32_t step = (span + DUP_THREADS - 1) / DUP_THREADS;
-    const uint32_t probe = lo + threadIdx.x * step;
-    const int below = (probe < hi) && (off[probe] <= x);
-    const uint32_t cnt = (uint32_t)__syncthreads_count(below);  // monotone predicate: the first cnt probes are <= x
-    if (cnt == 0) { hi = lo; break; }
-    const uint32_t new_lo = lo + (cnt - 1) * step + 1;
-    const uint32_t new_hi = min(hi, lo + cnt * step);
-    lo = new_lo; hi = new_hi;
-  }
-  return lo;
-}
-
-// Each chunk of DUP_CHUNK consecutive instance slots finds the rows it overlaps, stages their offsets, rectangles and
-// depths in shared memory, and every thread expands its slots: slot i of row r is tile (y0 + k / w, x0 + k % w) with
-// k = i - offset[r], w = x1 - x0.  Keys and values are written fully coalesced.  Digit histograms for the sort are
-// accumulated on the way: depth digits once per row (weighted by the row's slots in the chunk), tile digits per
-// slot with warp aggregation.
-// chunk_row[c] = the row whose slots contain slot c * DUP_CHUNK (one thread per row; a row writes an entry for every
-// chunk boundary that falls inside its slot range, usually none or one).
+// ------------------------------------------------------------------------------------------------ row histograms
+// Digit histograms of the depth bits of all rows, for the SORT_DEPTH_DIGITS row passes (warp-aggregated shared
+// atomics: the high digits of a depth take few distinct values).
 __global__ void __launch_bounds__(256)
-chunk_rows_kernel(const uint32_t* __restrict__ tile_offset, const uint32_t* __restrict__ num_rows,
-                  const uint64_t* __restrict__ num_instances, uint32_t chunks_cap, uint32_t* __restrict__ chunk_row) {
-  const uint32_t V = *num_rows;
-  const uint64_t M_all = *num_instances;
-  for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
-    const uint64_t lo = tile_offset[r];
-    const uint64_t hi = (r + 1 < V) ? (uint64_t)tile_offset[r + 1] : M_all;
-    for (uint64_t c = (lo + DUP_CHUNK - 1) / DUP_CHUNK; c * DUP_CHUNK < hi && c < chunks_cap; ++c) chunk_row[c] = r;
-  }
-}
-
-__global__ void __launch_bounds__(DUP_THREADS)
-emit_instances_kernel(const uint32_t* __restrict__ tile_offset, const uint32_t* __restrict__ chunk_row,
-                      const ushort4* __restrict__ rect,
-                      const float* __restrict__ depth, const uint32_t* __restrict__ num_rows,
-                      const uint64_t* __restrict__ num_instances, uint64_t capacity, int TX, int passes,
-                      uint64_t* __restrict__ keys, uint32_t* __restrict__ vals, uint32_t* __restrict__ hist, int* status) {
-  __shared__ uint32_t s_off[DUP_CHUNK + 1];
-  __shared__ ushort4 s_rect[DUP_CHUNK];
-  __shared__ uint32_t s_depth[DUP_CHUNK];
-  __shared__ uint32_t s_hist[SORT_MAX_PASSES][SORT_RADIX];
-  __shared__ __align__(16) uint16_t s_map[DUP_CHUNK];  // slot of the chunk -> row of the chunk
-  __shared__ uint32_t s_scan[DUP_THREADS / 32];
-  const uint32_t V = *num_rows;
-  const uint64_t M_all = *num_instances;
-  const uint64_t M64 = M_all < capacity ? M_all : capacity;
-  if (blockIdx.x == 0 && threadIdx.x == 0 && M_all > capacity) odin_set_error(status, ODIN_ERR_CAPACITY);
-  const uint32_t M = (uint32_t)(M64 < 0xffffffffull ? M64 : 0xffffffffull);
-  for (int i = threadIdx.x; i < SORT_MAX_PASSES * (int)SORT_RADIX; i += DUP_THREADS) (&s_hist[0][0])[i] = 0;
+row_hist_kernel(const uint32_t* __restrict__ depth_bits, const uint32_t* __restrict__ num_rows, uint32_t* __restrict__ hist) {
+  __shared__ uint32_t s_hist[SORT_DEPTH_DIGITS][SORT_RADIX];
+  for (int i = threadIdx.x; i < SORT_DEPTH_DIGITS * (int)SORT_RADIX; i += 256) (&s_hist[0][0])[i] = 0;
   __syncthreads();
-  const uint32_t chunks = V == 0 ? 0u : (M + DUP_CHUNK - 1) / DUP_CHUNK;
+  const uint32_t V = *num_rows;
   const unsigned lane = threadIdx.x & 31;
-  for (uint32_t chunk = blockIdx.x; chunk < chunks; chunk += gridDim.x) {
-    const uint32_t c0 = chunk * DUP_CHUNK;
-    const uint32_t c1 = (M - c0 < (uint32_t)DUP_CHUNK) ? M : c0 + DUP_CHUNK;
-    // first and last row of the chunk from the chunk -> row table; only the last chunk has to search for its end
-    const uint32_t row_lo = chunk_row[chunk];
-    uint32_t row_hi;
-    if (chunk + 1 < chunks) {
-      const uint32_t rn = chunk_row[chunk + 1];  // row that holds slot c1
-      row_hi = (tile_offset[rn] == c1) ? rn - 1 : rn;
-    } else {
-      row_hi = block_upper_bound(tile_offset, V, c1 - 1) - 1;  // offset[0] = 0, so the bound is >= 1
-    }
-    const uint32_t nrows = row_hi - row_lo + 1;  // <= DUP_CHUNK: every row owns at least one slot
-    for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS) {
-      s_off[i] = tile_offset[row_lo + i];
-      s_rect[i] = rect[row_lo + i];
-      s_depth[i] = __float_as_uint(depth[row_lo + i]);
-    }
-    if (threadIdx.x == 0) s_off[nrows] = (row_hi + 1 < V) ? tile_offset[row_hi + 1] : (uint32_t)M_all;
-    for (int i = threadIdx.x; i < DUP_CHUNK; i += DUP_THREADS) s_map[i] = 0;
-    __syncthreads();
-    // slot -> row of the chunk: every row marks its first slot, an inclusive max-scan fills the rest
-    for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS)
-      s_map[max(s_off[i], c0) - c0] = (uint16_t)i;
-    __syncthreads();
-    {
-      static_assert(DUP_ITEMS == 8, "a thread's slots are one 16-byte word of the map");
-      uint4* map4 = reinterpret_cast<uint4*>(s_map) + threadIdx.x;
-      const uint4 raw = *map4;
-      const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
-      uint32_t m[DUP_ITEMS];
-      uint32_t run = 0;
+  const uint32_t stride = gridDim.x * blockDim.x;
+  for (uint32_t r0 = blockIdx.x * blockDim.x; r0 < V; r0 += stride) {  // uniform trip count inside a warp
+    const uint32_t r = r0 + threadIdx.x;
+    const bool valid = r < V;
+    const uint32_t bits = valid ? depth_bits[r] : 0u;
 #pragma unroll
-      for (int k = 0; k < DUP_ITEMS; ++k) {
-        run = max(run, (rw[k >> 1] >> (16 * (k & 1))) & 0xffffu);
-        m[k] = run;
-      }
-      uint32_t inc = run;  // inclusive max over the threads of the warp
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) inc = max(inc, __shfl_up_sync(0xffffffffu, inc, o, 32) * (lane >= (unsigned)o ? 1u : 0u));
-      if (lane == 31) s_scan[threadIdx.x >> 5] = inc;
-      __syncthreads();
-      uint32_t before = __shfl_up_sync(0xffffffffu, inc, 1);
-      if (lane == 0) before = 0;
-      for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) before = max(before, s_scan[w]);
-#pragma unroll
-      for (int k = 0; k < DUP_ITEMS; ++k) m[k] = max(m[k], before);
-      *map4 = make_uint4(m[0] | (m[1] << 16), m[2] | (m[3] << 16), m[4] | (m[5] << 16), m[6] | (m[7] << 16));
+    for (int d = 0; d < SORT_DEPTH_DIGITS; ++d) {
+      const uint32_t digit = valid ? ((bits >> (SORT_RADIX_BITS * d)) & (SORT_RADIX - 1)) : (SORT_RADIX + lane);
+      const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+      if (valid && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&s_hist[d][digit], (uint32_t)__popc(peers));
     }
-    __syncthreads();
-    // depth digits, once per row
-    for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS) {
-      const uint32_t b = max(s_off[i], c0), e = min(s_off[i + 1], c1);
-      const uint32_t wgt = e - b, bits = s_depth[i];
-#pragma unroll
-      for (int d = 0; d < SORT_DEPTH_DIGITS; ++d)
-        atomicAdd(&s_hist[d][(bits >> (SORT_RADIX_BITS * d)) & (SORT_RADIX - 1)], wgt);
-    }
-#pragma unroll
-    for (int k = 0; k < DUP_ITEMS; ++k) {
-      const uint32_t i = c0 + k * DUP_THREADS + threadIdx.x;
-      const bool valid = i < c1;
-      uint32_t tile = 0xffffffffu;
-      uint64_t key = 0;
-      if (valid) {
-        const uint32_t lo = s_map[i - c0];  // row of the chunk that owns this slot
-        const ushort4 rc = s_rect[lo];
-        const uint32_t local = i - s_off[lo];
-        const uint32_t w = (uint32_t)rc.z - (uint32_t)rc.x;
-        const uint32_t dy = local / w, dx = local - dy * w;
-        tile = ((uint32_t)rc.y + dy) * (uint32_t)TX + (uint32_t)rc.x + dx;
-        key = ((uint64_t)tile << 32) | (uint64_t)s_depth[lo];
-        keys[i] = key;
-        vals[i] = row_lo + lo;
-      }
-      // digits that contain tile bits differ from slot to slot of a row: count them per slot, aggregated per warp
-      for (int d = SORT_DEPTH_DIGITS; d < passes; ++d) {
-        const uint32_t digit = valid ? ((uint32_t)(key >> (SORT_RADIX_BITS * d)) & (SORT_RADIX - 1)) : (SORT_RADIX + lane);
-        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-        if (valid && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&s_hist[d][digit], (uint32_t)__popc(peers));
-      }
-    }
-    __syncthreads();
   }
-  for (int i = threadIdx.x; i < passes * (int)SORT_RADIX; i += DUP_THREADS) {
+  __syncthreads();
+  for (int i = threadIdx.x; i < SORT_DEPTH_DIGITS * (int)SORT_RADIX; i += 256) {
     const uint32_t c = (&s_hist[0][0])[i];
     if (c) atomicAdd(&hist[i], c);
   }
@@ -171,28 +53,40 @@ constexpr int OS_WARPS = OS_THREADS / 32;
 constexpr int OS_ITEMS = SORT_TILE / OS_THREADS;  // 16 keys per thread
 constexpr int OS_DPT = SORT_RADIX / OS_THREADS;   // digits owned by a thread
 constexpr int OS_WINDOW = 2;                      // predecessors fetched per look-back step and digit
+constexpr int OS_BLOCKS = 4;                      // resident blocks per SM
 constexpr uint32_t OS_FLAG_AGG = 1u << 30, OS_FLAG_INC = 2u << 30, OS_VALUE = (1u << 30) - 1;
-constexpr size_t OS_SMEM = (size_t)SORT_TILE * 8 + (size_t)SORT_TILE * 4 + (size_t)OS_WARPS * SORT_RADIX * 4 + 2 * SORT_RADIX * 4 + 16;
+constexpr size_t OS_SMEM = (size_t)SORT_TILE * 4 + (size_t)SORT_TILE * 4 + (size_t)OS_WARPS * SORT_RADIX * 4 + 2 * SORT_RADIX * 4 + 16;
 
-// One pass over one 8-bit digit.  Persistent blocks take 4096-key tiles by ticket.  Per tile: warp-striped loads,
-// per-warp digit ranking with match.any (stable), block digit counts published for look-back, exclusive global digit
-// offsets by a per-digit look-back walk (thread d walks digit d), keys and values exchanged through shared memory so
-// that the global scatter writes runs of consecutive addresses.
-__global__ void __launch_bounds__(OS_THREADS, 3)
-onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in, uint64_t* __restrict__ keys_out,
-                uint32_t* __restrict__ vals_out, const uint64_t* __restrict__ num_instances, uint64_t capacity, int shift,
+// One pass over one 8-bit digit of 32-bit keys.  Persistent blocks take 4096-key tiles by ticket.  Per tile:
+// warp-striped loads, per-warp digit ranking with match.any (stable), block digit counts published for look-back,
+// exclusive global digit offsets by a per-digit look-back walk (thread d walks digit d), keys and values exchanged
+// through shared memory so that the global scatter writes runs of consecutive addresses.
+//   vals_in == nullptr: the values are the positions themselves (first pass over the rows)
+//   keys_out == nullptr: the keys are not needed afterwards (last pass over the rows)
+//   WIDE: the last pass over the instances may also write the full 64-bit key key << 32 | depth_bits[value]
+//   the number of keys is *count32 if given, else min(*count64, capacity)
+template <bool WIDE>
+__global__ void __launch_bounds__(OS_THREADS, OS_BLOCKS)
+onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in, uint32_t* __restrict__ keys_out,
+                uint32_t* __restrict__ vals_out, uint64_t* __restrict__ keys64_out, const uint32_t* __restrict__ depth_bits,
+                const uint32_t* __restrict__ count32, const uint64_t* __restrict__ count64, uint64_t capacity, int shift,
                 const uint32_t* __restrict__ digit_base, uint32_t* states, uint32_t* ticket, int* status) {
   extern __shared__ __align__(16) unsigned char os_smem[];
-  uint64_t* s_keys = reinterpret_cast<uint64_t*>(os_smem);
-  uint32_t* s_vals = reinterpret_cast<uint32_t*>(os_smem + (size_t)SORT_TILE * 8);
-  uint32_t(*s_warp_hist)[SORT_RADIX] = reinterpret_cast<uint32_t(*)[SORT_RADIX]>(os_smem + (size_t)SORT_TILE * 12);
-  uint32_t* s_digit_start = reinterpret_cast<uint32_t*>(os_smem + (size_t)SORT_TILE * 12 + (size_t)OS_WARPS * SORT_RADIX * 4);
+  uint32_t* s_keys = reinterpret_cast<uint32_t*>(os_smem);
+  uint32_t* s_vals = s_keys + SORT_TILE;
+  uint32_t(*s_warp_hist)[SORT_RADIX] = reinterpret_cast<uint32_t(*)[SORT_RADIX]>(s_vals + SORT_TILE);
+  uint32_t* s_digit_start = &s_warp_hist[0][0] + OS_WARPS * SORT_RADIX;
   uint32_t* s_global = s_digit_start + SORT_RADIX;
   uint32_t* s_misc = s_global + SORT_RADIX;  // [0] tile ticket
   __shared__ uint32_t s_scan[33];
 
-  const uint64_t M_all = *num_instances;
-  const uint64_t M64 = M_all < capacity ? M_all : capacity;
+  uint64_t M64;
+  if (count32) {
+    M64 = *count32;
+  } else {
+    const uint64_t M_all = *count64;
+    M64 = M_all < capacity ? M_all : capacity;
+  }
   const uint32_t M = (uint32_t)(M64 < (uint64_t)OS_VALUE ? M64 : (uint64_t)OS_VALUE);
   const uint32_t ntiles = (M + SORT_TILE - 1) / SORT_TILE;
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -200,7 +94,7 @@ onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict
 
   // The keys and values of the NEXT tile are requested as soon as the registers of the current one are free (after
   // the exchange through shared memory), so that their latency overlaps the global scatter of the current tile.
-  uint64_t key[OS_ITEMS];
+  uint32_t key[OS_ITEMS];
   uint32_t val[OS_ITEMS];
   auto load_tile = [&](uint32_t t) {
     const uint32_t wb = t * SORT_TILE + warp * (32 * OS_ITEMS);
@@ -208,8 +102,8 @@ onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict
     for (int j = 0; j < OS_ITEMS; ++j) {
       const uint32_t i = wb + 32 * j + lane;
       const bool in = t < ntiles && i < M;
-      key[j] = in ? keys_in[i] : ~0ull;  // padding sorts to the end of the tile and is never written
-      val[j] = in ? vals_in[i] : 0u;
+      key[j] = in ? keys_in[i] : ~0u;  // padding sorts to the end of the tile and is never written
+      val[j] = in ? (vals_in ? vals_in[i] : i) : 0u;
     }
   };
   if (threadIdx.x == 0) s_misc[0] = atomicAdd(ticket, 1u);
@@ -226,7 +120,7 @@ onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict
     uint32_t pos[OS_ITEMS];
 #pragma unroll
     for (int j = 0; j < OS_ITEMS; ++j) {
-      const uint32_t d = (uint32_t)(key[j] >> shift) & (SORT_RADIX - 1);
+      const uint32_t d = (key[j] >> shift) & (SORT_RADIX - 1);
       const uint32_t peers = __match_any_sync(0xffffffffu, d);
       const int leader = __ffs(peers) - 1;
       uint32_t old = 0;
@@ -322,7 +216,7 @@ onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict
 
 #pragma unroll
     for (int j = 0; j < OS_ITEMS; ++j) {
-      const uint32_t dg = (uint32_t)(key[j] >> shift) & (SORT_RADIX - 1);
+      const uint32_t dg = (key[j] >> shift) & (SORT_RADIX - 1);
       const uint32_t slot = s_digit_start[dg] + s_warp_hist[warp][dg] + pos[j];
       s_keys[slot] = key[j];
       s_vals[slot] = val[j];
@@ -335,11 +229,15 @@ onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict
     for (int j = 0; j < OS_ITEMS; ++j) {
       const uint32_t slot = j * OS_THREADS + threadIdx.x;
       if (slot < tile_count) {
-        const uint64_t k = s_keys[slot];
-        const uint32_t dst = s_global[(uint32_t)(k >> shift) & (SORT_RADIX - 1)] + slot;
+        const uint32_t k = s_keys[slot];
+        const uint32_t dst = s_global[(k >> shift) & (SORT_RADIX - 1)] + slot;
         if (dst < M) {
-          keys_out[dst] = k;
-          vals_out[dst] = s_vals[slot];
+          const uint32_t v = s_vals[slot];
+          if (keys_out) keys_out[dst] = k;
+          vals_out[dst] = v;
+          if (WIDE) {
+            if (keys64_out) keys64_out[dst] = ((uint64_t)k << 32) | (uint64_t)depth_bits[v];
+          }
         }
       }
     }
@@ -348,31 +246,229 @@ onesweep_kernel(const uint64_t* __restrict__ keys_in, const uint32_t* __restrict
   }
 }
 
-// ------------------------------------------------------------------------------------------------ ranges
-__global__ void __launch_bounds__(256)
-tile_ranges_kernel(const uint64_t* __restrict__ keys, const uint64_t* __restrict__ num_instances, uint64_t capacity,
-                   uint32_t n_tiles, uint32_t* __restrict__ ranges) {
-  const uint64_t M_all = *num_instances;
-  const uint64_t M = M_all < capacity ? M_all : capacity;
-  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < M; i += (uint64_t)gridDim.x * blockDim.x) {
-    const uint32_t t = (uint32_t)(keys[i] >> 32);
-    if (t >= n_tiles) continue;
-    if (i == 0) ranges[2 * t] = 0;
-    else {
-      const uint32_t tp = (uint32_t)(keys[i - 1] >> 32);
-      if (tp != t) {
-        ranges[2 * t] = (uint32_t)i;
-        if (tp < n_tiles) ranges[2 * tp + 1] = (uint32_t)i;
-      }
+// ------------------------------------------------------------------------------------------------ sorted offsets
+// sorted_off[i] = number of instances of the rows in front of position i of the depth order: an exclusive scan of the
+// rectangles' tile counts gathered through sorted_row.  2048 positions per block, one decoupled look-back per block,
+// blocks ordered by ticket.
+constexpr int RO_THREADS = 256;
+constexpr int RO_ITEMS = OFFSET_TILE / RO_THREADS;
+
+__global__ void __launch_bounds__(RO_THREADS)
+sorted_offsets_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __restrict__ rect,
+                      const uint32_t* __restrict__ num_rows, uint32_t* __restrict__ sorted_off, uint32_t* ticket,
+                      uint64_t* state, int* status) {
+  __shared__ uint32_t s_tile, s_base;
+  __shared__ uint32_t s_warp[33];
+  const uint32_t V = *num_rows;
+  const uint32_t ntiles = (V + OFFSET_TILE - 1) / OFFSET_TILE;
+  if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
+  __syncthreads();
+  const uint32_t tile = s_tile;
+  if (tile >= ntiles) return;  // uniform over the block; nobody waits for a tile past the end
+  const uint32_t first = tile * OFFSET_TILE + threadIdx.x * RO_ITEMS;
+  uint32_t cnt[RO_ITEMS];
+  uint32_t sum = 0;  // sums are taken modulo 2^32; the true totals fit (M >= 2^32 is an error raised by the projection)
+#pragma unroll
+  for (int k = 0; k < RO_ITEMS; ++k) {
+    cnt[k] = 0;
+    if (first + k < V) {
+      const ushort4 rc = rect[sorted_row[first + k]];
+      cnt[k] = ((uint32_t)rc.z - (uint32_t)rc.x) * ((uint32_t)rc.w - (uint32_t)rc.y);
     }
-    if (i == M - 1) ranges[2 * t + 1] = (uint32_t)M;
+    sum += cnt[k];
+  }
+  uint32_t total;
+  const uint32_t before = odin_block_exclusive_sum(sum, s_warp, &total);
+  if (threadIdx.x < 32) {
+    const uint64_t base = odin_lookback_u64(state, tile, (uint64_t)total, status);
+    if (threadIdx.x == 0) s_base = (uint32_t)base;
+  }
+  __syncthreads();
+  uint32_t run = s_base + before;
+#pragma unroll
+  for (int k = 0; k < RO_ITEMS; ++k) {
+    if (first + k < V) sorted_off[first + k] = run;
+    run += cnt[k];
   }
 }
 
-int sort_passes(int n_tiles) {
+// ------------------------------------------------------------------------------------------------ emission
+constexpr int DUP_THREADS = 256;
+constexpr int DUP_ITEMS = 8;
+constexpr int DUP_CHUNK = DUP_THREADS * DUP_ITEMS;  // instances per chunk; a chunk spans at most DUP_CHUNK rows
+
+// Cooperative 256-ary upper bound: first r in [0, V) with off[r] > x (V if none).  All threads must call.
+__device__ __forceinline__ uint32_t block_upper_bound(const uint32_t* __restrict__ off, uint32_t V, uint32_t x) {
+  uint32_t lo = 0, hi = V;
+  while (lo < hi) {
+    const uint32_t span = hi - lo;
+    const uint32_t step = (span + DUP_THREADS - 1) / DUP_THREADS;
+    const uint32_t probe = lo + threadIdx.x * step;
+    const int below = (probe < hi) && (off[probe] <= x);
+    const uint32_t cnt = (uint32_t)__syncthreads_count(below);  // monotone predicate: the first cnt probes are <= x
+    if (cnt == 0) { hi = lo; break; }
+    const uint32_t new_lo = lo + (cnt - 1) * step + 1;
+    const uint32_t new_hi = min(hi, lo + cnt * step);
+    lo = new_lo; hi = new_hi;
+  }
+  return lo;
+}
+
+// chunk_row[c] = the position (in depth order) of the row whose slots contain slot c * DUP_CHUNK (one thread per
+// position; a row writes an entry for every chunk boundary that falls inside its slot range, usually none or one).
+__global__ void __launch_bounds__(256)
+chunk_rows_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* __restrict__ num_rows,
+                  const uint64_t* __restrict__ num_instances, uint32_t chunks_cap, uint32_t* __restrict__ chunk_row) {
+  const uint32_t V = *num_rows;
+  const uint64_t M_all = *num_instances;
+  for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
+    const uint64_t lo = sorted_off[r];
+    const uint64_t hi = (r + 1 < V) ? (uint64_t)sorted_off[r + 1] : M_all;
+    for (uint64_t c = (lo + DUP_CHUNK - 1) / DUP_CHUNK; c * DUP_CHUNK < hi && c < chunks_cap; ++c) chunk_row[c] = r;
+  }
+}
+
+// Each chunk of DUP_CHUNK consecutive instance slots finds the positions of the depth order it overlaps, stages their
+// offsets, row ids and rectangles in shared memory, and every thread expands its slots: slot i of a row is tile
+// (y0 + k / w, x0 + k % w) with k = i - offset, w = x1 - x0.  Keys (tile ids) and values (row ids) are written fully
+// coalesced.  The histograms of the tile-id digits are accumulated on the way, per slot with warp aggregation.
+__global__ void __launch_bounds__(DUP_THREADS)
+emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* __restrict__ sorted_row,
+                      const uint32_t* __restrict__ chunk_row, const ushort4* __restrict__ rect,
+                      const uint32_t* __restrict__ num_rows, const uint64_t* __restrict__ num_instances, uint64_t capacity,
+                      int TX, int tile_passes, uint32_t* __restrict__ keys, uint32_t* __restrict__ vals,
+                      uint32_t* __restrict__ hist, int* status) {
+  __shared__ uint32_t s_off[DUP_CHUNK + 1];
+  __shared__ ushort4 s_rect[DUP_CHUNK];
+  __shared__ uint32_t s_row[DUP_CHUNK];
+  __shared__ uint32_t s_hist[SORT_MAX_TILE_DIGITS][SORT_RADIX];
+  __shared__ __align__(16) uint16_t s_map[DUP_CHUNK];  // slot of the chunk -> staged row of the chunk
+  __shared__ uint32_t s_scan[DUP_THREADS / 32];
+  const uint32_t V = *num_rows;
+  const uint64_t M_all = *num_instances;
+  const uint64_t M64 = M_all < capacity ? M_all : capacity;
+  if (blockIdx.x == 0 && threadIdx.x == 0 && M_all > capacity) odin_set_error(status, ODIN_ERR_CAPACITY);
+  const uint32_t M = (uint32_t)(M64 < 0xffffffffull ? M64 : 0xffffffffull);
+  for (int i = threadIdx.x; i < SORT_MAX_TILE_DIGITS * (int)SORT_RADIX; i += DUP_THREADS) (&s_hist[0][0])[i] = 0;
+  __syncthreads();
+  const uint32_t chunks = V == 0 ? 0u : (M + DUP_CHUNK - 1) / DUP_CHUNK;
+  const unsigned lane = threadIdx.x & 31;
+  for (uint32_t chunk = blockIdx.x; chunk < chunks; chunk += gridDim.x) {
+    const uint32_t c0 = chunk * DUP_CHUNK;
+    const uint32_t c1 = (M - c0 < (uint32_t)DUP_CHUNK) ? M : c0 + DUP_CHUNK;
+    // first and last position of the chunk from the chunk table; only the last chunk has to search for its end
+    const uint32_t row_lo = chunk_row[chunk];
+    uint32_t row_hi;
+    if (chunk + 1 < chunks) {
+      const uint32_t rn = chunk_row[chunk + 1];  // position that holds slot c1
+      row_hi = (sorted_off[rn] == c1) ? rn - 1 : rn;
+    } else {
+      row_hi = block_upper_bound(sorted_off, V, c1 - 1) - 1;  // offset[0] = 0, so the bound is >= 1
+    }
+    const uint32_t nrows = row_hi - row_lo + 1;  // <= DUP_CHUNK: every row owns at least one slot
+    for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS) {
+      const uint32_t r = sorted_row[row_lo + i];
+      s_off[i] = sorted_off[row_lo + i];
+      s_row[i] = r;
+      s_rect[i] = rect[r];
+    }
+    if (threadIdx.x == 0) s_off[nrows] = (row_hi + 1 < V) ? sorted_off[row_hi + 1] : (uint32_t)M_all;
+    for (int i = threadIdx.x; i < DUP_CHUNK; i += DUP_THREADS) s_map[i] = 0;
+    __syncthreads();
+    // slot -> staged row: every row marks its first slot, an inclusive max-scan fills the rest
+    for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS) s_map[max(s_off[i], c0) - c0] = (uint16_t)i;
+    __syncthreads();
+    {
+      static_assert(DUP_ITEMS == 8, "a thread's slots are one 16-byte word of the map");
+      uint4* map4 = reinterpret_cast<uint4*>(s_map) + threadIdx.x;
+      const uint4 raw = *map4;
+      const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+      uint32_t m[DUP_ITEMS];
+      uint32_t run = 0;
+#pragma unroll
+      for (int k = 0; k < DUP_ITEMS; ++k) {
+        run = max(run, (rw[k >> 1] >> (16 * (k & 1))) & 0xffffu);
+        m[k] = run;
+      }
+      uint32_t inc = run;  // inclusive max over the threads of the warp (values >= 0, so 0 is neutral)
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o, 32);
+        if (lane >= (unsigned)o) inc = max(inc, y);
+      }
+      if (lane == 31) s_scan[threadIdx.x >> 5] = inc;
+      __syncthreads();
+      uint32_t before = __shfl_up_sync(0xffffffffu, inc, 1);
+      if (lane == 0) before = 0;
+      for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) before = max(before, s_scan[w]);
+#pragma unroll
+      for (int k = 0; k < DUP_ITEMS; ++k) m[k] = max(m[k], before);
+      *map4 = make_uint4(m[0] | (m[1] << 16), m[2] | (m[3] << 16), m[4] | (m[5] << 16), m[6] | (m[7] << 16));
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < DUP_ITEMS; ++k) {
+      const uint32_t i = c0 + k * DUP_THREADS + threadIdx.x;
+      const bool valid = i < c1;
+      uint32_t tile = 0;
+      if (valid) {
+        const uint32_t lo = s_map[i - c0];  // staged row that owns this slot
+        const ushort4 rc = s_rect[lo];
+        const uint32_t local = i - s_off[lo];
+        const uint32_t w = (uint32_t)rc.z - (uint32_t)rc.x;
+        const uint32_t dy = local / w, dx = local - dy * w;
+        tile = ((uint32_t)rc.y + dy) * (uint32_t)TX + (uint32_t)rc.x + dx;
+        keys[i] = tile;
+        vals[i] = s_row[lo];
+      }
+      for (int d = 0; d < tile_passes; ++d) {
+        const uint32_t digit = valid ? ((tile >> (SORT_RADIX_BITS * d)) & (SORT_RADIX - 1)) : (SORT_RADIX + lane);
+        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+        if (valid && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&s_hist[d][digit], (uint32_t)__popc(peers));
+      }
+    }
+    __syncthreads();
+  }
+  for (int i = threadIdx.x; i < tile_passes * (int)SORT_RADIX; i += DUP_THREADS) {
+    const uint32_t c = (&s_hist[0][0])[i];
+    if (c) atomicAdd(&hist[i], c);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ ranges
+__global__ void __launch_bounds__(256)
+tile_ranges_kernel(const uint32_t* __restrict__ tile_ids, const uint64_t* __restrict__ num_instances, uint64_t capacity,
+                   uint32_t n_tiles, uint32_t* __restrict__ ranges) {
+  const uint64_t M_all = *num_instances;
+  const uint64_t M = M_all < capacity ? M_all : capacity;
+  // four positions per thread from one 16-byte load (the buffer is padded to a multiple of 256 bytes)
+  for (uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; 4 * q < M; q += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t i0 = 4 * q;
+    const uint4 k4 = reinterpret_cast<const uint4*>(tile_ids)[q];
+    const uint32_t ks[4] = {k4.x, k4.y, k4.z, k4.w};
+    uint32_t tp = i0 ? tile_ids[i0 - 1] : 0xffffffffu;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint64_t i = i0 + j;
+      if (i >= M) break;
+      const uint32_t t = ks[j];
+      if (t < n_tiles) {
+        if (tp != t) {
+          ranges[2 * t] = (uint32_t)i;
+          if (tp < n_tiles) ranges[2 * tp + 1] = (uint32_t)i;
+        }
+        if (i == M - 1) ranges[2 * t + 1] = (uint32_t)M;
+      }
+      tp = t;
+    }
+  }
+}
+
+int tile_digit_passes(uint32_t n_tiles) {
   int tile_bits = 0;
-  while ((1ll << tile_bits) < (long long)n_tiles) ++tile_bits;
-  return (32 + tile_bits + (int)SORT_RADIX_BITS - 1) / (int)SORT_RADIX_BITS;
+  while ((1ull << tile_bits) < (unsigned long long)n_tiles) ++tile_bits;
+  const int p = (tile_bits + (int)SORT_RADIX_BITS - 1) / (int)SORT_RADIX_BITS;
+  return p < 1 ? 1 : p;  // a one-tile image still takes one pass, which moves the emission into the outputs
 }
 
 }  // namespace
@@ -383,65 +479,114 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   if (!ctx || !proj || !d_tile_ranges) return ODIN_ERR_NULL;
   if (width <= 0 || height <= 0 || width > 16384 || height > 16384) return ODIN_ERR_INVALID_ARG;
   if (!proj->num_rows || !proj->num_instances) return ODIN_ERR_NULL;
-  if (capacity >= (1ull << 30)) return ODIN_ERR_INVALID_ARG;
+  if (capacity >= (1ull << 30) || proj->capacity >= (1u << 30)) return ODIN_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const int TX = (width + 15) / 16, TY = (height + 15) / 16;
   const uint32_t n_tiles = (uint32_t)TX * (uint32_t)TY;
   ODIN_CUDA(cudaMemsetAsync(d_tile_ranges, 0, (size_t)n_tiles * 8, st));
   if (capacity == 0 || proj->capacity == 0) return ODIN_OK;
-  if (!d_keys || !d_vals || !proj->tile_offset || !proj->rect || !proj->depth) return ODIN_ERR_NULL;
-  if (!odin_aligned(d_keys, 16) || !odin_aligned(d_vals, 16) || !odin_aligned(proj->rect, 8)) return ODIN_ERR_INVALID_ARG;
-  const BinSortLayout L = binsort_layout(capacity);
+  if (!d_vals || !proj->rect || !proj->depth) return ODIN_ERR_NULL;
+  if ((d_keys && !odin_aligned(d_keys, 16)) || !odin_aligned(d_vals, 16) || !odin_aligned(proj->rect, 8))
+    return ODIN_ERR_INVALID_ARG;
+  const BinSortLayout L = binsort_layout(capacity, proj->capacity);
   if (!ws || !odin_aligned(ws, 256) || ws_bytes < L.total) return ODIN_ERR_WORKSPACE;
   char* base = reinterpret_cast<char*>(ws);
-  const int passes = sort_passes((int)n_tiles);
+  const int tile_passes = tile_digit_passes(n_tiles);
   // zero tickets, histograms and the look-back words of the passes that will run
-  const size_t zero = L.states + (size_t)passes * L.tiles * SORT_RADIX * 4;
+  const size_t zero = L.inst_states + (size_t)tile_passes * L.tiles * SORT_RADIX * 4;
   ODIN_CUDA(cudaMemsetAsync(base, 0, zero, st));
   uint32_t* tickets = reinterpret_cast<uint32_t*>(base + L.header);
   uint32_t* hist = reinterpret_cast<uint32_t*>(base + L.hist);
   uint32_t* dbase = reinterpret_cast<uint32_t*>(base + L.digit_base);
-  uint32_t* states = reinterpret_cast<uint32_t*>(base + L.states);
-  uint64_t* alt_keys = reinterpret_cast<uint64_t*>(base + L.alt_keys);
-  uint32_t* alt_vals = reinterpret_cast<uint32_t*>(base + L.alt_vals);
-  // with an odd number of passes the emission goes to the alternate buffers so that the last pass lands in d_keys
-  uint64_t* kbuf[2] = {d_keys, alt_keys};
-  uint32_t* vbuf[2] = {d_vals, alt_vals};
-  int cur = passes & 1;
-
-  const uint64_t chunks_cap = (capacity + DUP_CHUNK - 1) / DUP_CHUNK;
-  uint32_t grid = (uint32_t)(chunks_cap < (uint64_t)ctx->sm_count * 6 ? chunks_cap : (uint64_t)ctx->sm_count * 6);
+  uint64_t* scan_state = reinterpret_cast<uint64_t*>(base + L.scan_state);
+  uint32_t* row_states = reinterpret_cast<uint32_t*>(base + L.row_states);
+  uint32_t* inst_states = reinterpret_cast<uint32_t*>(base + L.inst_states);
+  uint32_t* row_keys[2] = {reinterpret_cast<uint32_t*>(base + L.row_keys[0]), reinterpret_cast<uint32_t*>(base + L.row_keys[1])};
+  uint32_t* row_vals[2] = {reinterpret_cast<uint32_t*>(base + L.row_vals[0]), reinterpret_cast<uint32_t*>(base + L.row_vals[1])};
+  uint32_t* sorted_off = reinterpret_cast<uint32_t*>(base + L.sorted_off);
+  uint32_t* inst_keys[2] = {reinterpret_cast<uint32_t*>(base + L.inst_keys[0]), reinterpret_cast<uint32_t*>(base + L.inst_keys[1])};
+  uint32_t* inst_vals[2] = {d_vals, reinterpret_cast<uint32_t*>(base + L.alt_vals)};
   uint32_t* chunk_row = reinterpret_cast<uint32_t*>(base + L.chunk_row);
+  const uint32_t* depth_bits = reinterpret_cast<const uint32_t*>(proj->depth);
+  const ushort4* rect = reinterpret_cast<const ushort4*>(proj->rect);
+  const uint32_t sms = (uint32_t)ctx->sm_count;
+  const uint32_t row_blocks = (proj->capacity + 255) / 256;
+
+  // ---- rows by depth
   {
-    OdinKernelScope ks(ctx, K_CHUNK_ROWS, st);
-    const uint32_t rb = (proj->capacity + 255) / 256;
-    chunk_rows_kernel<<<rb < (uint32_t)ctx->sm_count * 8 ? rb : (uint32_t)ctx->sm_count * 8, 256, 0, st>>>(
-        proj->tile_offset, proj->num_rows, proj->num_instances, (uint32_t)chunks_cap, chunk_row);
-  }
-  {
-    OdinKernelScope ks(ctx, K_EMIT, st);
-    emit_instances_kernel<<<grid, DUP_THREADS, 0, st>>>(proj->tile_offset, chunk_row,
-                                                        reinterpret_cast<const ushort4*>(proj->rect),
-                                                        proj->depth, proj->num_rows, proj->num_instances, capacity, TX,
-                                                        passes, kbuf[cur], vbuf[cur], hist, ctx->d_status);
+    OdinKernelScope ks(ctx, K_ROW_HIST, st);
+    row_hist_kernel<<<row_blocks < sms * 8 ? row_blocks : sms * 8, 256, 0, st>>>(depth_bits, proj->num_rows, hist);
   }
   {
     OdinKernelScope ks(ctx, K_DIGIT_BASE, st);
-    digit_base_kernel<<<passes, SORT_RADIX, 0, st>>>(hist, dbase);
+    digit_base_kernel<<<SORT_DEPTH_DIGITS, SORT_RADIX, 0, st>>>(hist, dbase);
   }
-  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OS_SMEM));
-  uint32_t os_grid = L.tiles < (uint32_t)ctx->sm_count * 3 ? L.tiles : (uint32_t)ctx->sm_count * 3;
-  for (int p = 0; p < passes; ++p) {
+  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OS_SMEM));
+  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OS_SMEM));
+  const uint32_t* sorted_row = nullptr;
+  {
+    const uint32_t grid = L.row_tiles < sms * OS_BLOCKS ? L.row_tiles : sms * OS_BLOCKS;
+    const uint32_t* kin = depth_bits;
+    const uint32_t* vin = nullptr;
+    for (int p = 0; p < SORT_DEPTH_DIGITS; ++p) {
+      OdinKernelScope ks(ctx, K_ROW_SORT, st);
+      uint32_t* kout = (p + 1 < SORT_DEPTH_DIGITS) ? row_keys[p & 1] : nullptr;
+      uint32_t* vout = row_vals[p & 1];
+      onesweep_kernel<false><<<grid, OS_THREADS, OS_SMEM, st>>>(
+          kin, vin, kout, vout, nullptr, nullptr, proj->num_rows, nullptr, 0, p * (int)SORT_RADIX_BITS,
+          dbase + p * SORT_RADIX, row_states + (size_t)p * L.row_tiles * SORT_RADIX, tickets + p, ctx->d_status);
+      kin = kout;
+      vin = vout;
+    }
+    sorted_row = vin;
+  }
+  // ---- instances in depth order
+  {
+    OdinKernelScope ks(ctx, K_ROW_OFFSETS, st);
+    sorted_offsets_kernel<<<(proj->capacity + OFFSET_TILE - 1) / OFFSET_TILE, RO_THREADS, 0, st>>>(
+        sorted_row, rect, proj->num_rows, sorted_off, tickets + 8, scan_state, ctx->d_status);
+  }
+  const uint64_t chunks_cap = (capacity + DUP_CHUNK - 1) / DUP_CHUNK;
+  {
+    OdinKernelScope ks(ctx, K_CHUNK_ROWS, st);
+    chunk_rows_kernel<<<row_blocks < sms * 8 ? row_blocks : sms * 8, 256, 0, st>>>(
+        sorted_off, proj->num_rows, proj->num_instances, (uint32_t)chunks_cap, chunk_row);
+  }
+  // the emission goes to the buffers from which `tile_passes` ping-pong steps end in d_vals
+  int cur = tile_passes & 1;
+  uint32_t* tile_hist = hist + SORT_DEPTH_DIGITS * SORT_RADIX;
+  uint32_t* tile_dbase = dbase + SORT_DEPTH_DIGITS * SORT_RADIX;
+  {
+    OdinKernelScope ks(ctx, K_EMIT, st);
+    const uint32_t grid = (uint32_t)(chunks_cap < (uint64_t)sms * 5 ? chunks_cap : (uint64_t)sms * 5);
+    emit_instances_kernel<<<grid, DUP_THREADS, 0, st>>>(sorted_off, sorted_row, chunk_row, rect, proj->num_rows,
+                                                        proj->num_instances, capacity, TX, tile_passes, inst_keys[cur],
+                                                        inst_vals[cur], tile_hist, ctx->d_status);
+  }
+  {
+    OdinKernelScope ks(ctx, K_DIGIT_BASE, st);
+    digit_base_kernel<<<tile_passes, SORT_RADIX, 0, st>>>(tile_hist, tile_dbase);
+  }
+  // ---- instances by tile id
+  const uint32_t os_grid = L.tiles < sms * OS_BLOCKS ? L.tiles : sms * OS_BLOCKS;
+  for (int p = 0; p < tile_passes; ++p) {
     OdinKernelScope ks(ctx, K_ONESWEEP, st);
-    onesweep_kernel<<<os_grid, OS_THREADS, OS_SMEM, st>>>(kbuf[cur], vbuf[cur], kbuf[cur ^ 1], vbuf[cur ^ 1],
-                                                          proj->num_instances, capacity, p * (int)SORT_RADIX_BITS,
-                                                          dbase + p * SORT_RADIX, states + (size_t)p * L.tiles * SORT_RADIX,
-                                                          tickets + p, ctx->d_status);
+    uint32_t* states = inst_states + (size_t)p * L.tiles * SORT_RADIX;
+    if (p + 1 < tile_passes)
+      onesweep_kernel<false><<<os_grid, OS_THREADS, OS_SMEM, st>>>(
+          inst_keys[cur], inst_vals[cur], inst_keys[cur ^ 1], inst_vals[cur ^ 1], nullptr, nullptr, nullptr,
+          proj->num_instances, capacity, p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
+          tickets + SORT_DEPTH_DIGITS + p, ctx->d_status);
+    else
+      onesweep_kernel<true><<<os_grid, OS_THREADS, OS_SMEM, st>>>(
+          inst_keys[cur], inst_vals[cur], inst_keys[cur ^ 1], inst_vals[cur ^ 1], d_keys, depth_bits, nullptr,
+          proj->num_instances, capacity, p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
+          tickets + SORT_DEPTH_DIGITS + p, ctx->d_status);
     cur ^= 1;
   }
   const uint64_t rblocks = (capacity + 255) / 256;
-  const uint32_t rgrid = (uint32_t)(rblocks < (uint64_t)ctx->sm_count * 8 ? rblocks : (uint64_t)ctx->sm_count * 8);
+  const uint32_t rgrid = (uint32_t)(rblocks < (uint64_t)sms * 8 ? rblocks : (uint64_t)sms * 8);
   OdinKernelScope ks(ctx, K_RANGES, st);
-  tile_ranges_kernel<<<rgrid, 256, 0, st>>>(d_keys, proj->num_instances, capacity, n_tiles, d_tile_ranges);
+  tile_ranges_kernel<<<rgrid, 256, 0, st>>>(inst_keys[cur], proj->num_instances, capacity, n_tiles, d_tile_ranges);
   return odin_launch_status();
 }

@@ -123,6 +123,7 @@ class ViewTrainer:
                        B.odin_render_workspace_bytes(self.ctx, self.width, self.height))
         self.ws = z(ws_bytes, torch.uint8)
         self.kernel_launches_per_step = 0
+        self.keep_sorted_keys = False  # view_step: also write the sorted 64-bit keys (only tests look at them)
 
     def close(self) -> None:
         if self.ctx is not None:
@@ -137,9 +138,10 @@ class ViewTrainer:
         B.odin_touched_set(self.ctx, self.proj.tiles_touched, self.n, self.masks[slot], self.idx, self.row_capacity,
                            self.count, self.ws, stream)
 
-    def bin_sort(self, stream=None) -> None:
-        B.odin_bin_sort(self.ctx, self.proj.struct, self.width, self.height, self.keys, self.vals, self.instance_capacity,
-                        self.ranges, self.ws, stream)
+    def bin_sort(self, stream=None, want_keys: bool = True) -> None:
+        """Sorted values and tile ranges; the sorted 64-bit keys too unless want_keys is False (no later stage reads them)."""
+        B.odin_bin_sort(self.ctx, self.proj.struct, self.width, self.height, self.keys if want_keys else None, self.vals,
+                        self.instance_capacity, self.ranges, self.ws, stream)
 
     def render_fwd(self, cam: B.odin_camera, stream=None) -> None:
         B.odin_render_fwd(self.ctx, self.proj.struct, self.vals, self.ranges, cam, self.out, self.final_T, self.n_contrib,
@@ -167,7 +169,7 @@ class ViewTrainer:
         The target image must already be in self.target.  Nothing here synchronises the host."""
         self.project(cam, stream)
         self.touched_set(slot, stream)
-        self.bin_sort(stream)
+        self.bin_sort(stream, want_keys=self.keep_sorted_keys)
         self.render_fwd(cam, stream)
         self.l1_loss(stream)
         self.render_bwd(cam, stream)

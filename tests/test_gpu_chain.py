@@ -19,6 +19,7 @@ def run_chain(oracle32, w, steps, views, window=None):
     n = scene.n
     cam0 = w.cameras[0]
     tr = G.trainer_for(scene, cam0, mask_slots=max(len(views), 1))
+    tr.keep_sorted_keys = True  # the sorted keys are compared below
     p = scene.copy()
     m, v = p.zeros_like(), p.zeros_like()
     masks_o = {}

@@ -225,11 +225,15 @@ def check_bin_sort(oracle32, scene, cam, instance_capacity=None):
     G.load_oracle_projection(tr, po, idx)
     inv = np.full(scene.n, -1, np.int64)
     inv[idx] = np.arange(len(idx))
-    for _ in range(2):
+    for want_keys in (True, True, False):  # twice with the keys (workspace reuse), once without (values only)
         tr.keys.fill_(-1)
-        tr.bin_sort()
+        tr.vals.fill_(-1)
+        tr.bin_sort(want_keys=want_keys)
         G.poll_ok(tr)
-        assert np.array_equal(G.u64(tr.keys)[:m], keys_o)
+        if want_keys:
+            assert np.array_equal(G.u64(tr.keys)[:m], keys_o)
+        else:
+            assert bool((tr.keys == -1).all())
         assert np.array_equal(G.u32(tr.vals)[:m], G.rows_of(inv, vals_o).astype(np.uint32))
         rg = G.u32(tr.ranges)
         assert np.array_equal(rg[:, 1] - rg[:, 0], ranges_o[:, 1] - ranges_o[:, 0])
