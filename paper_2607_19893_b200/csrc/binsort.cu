@@ -4,18 +4,40 @@
 // that order (load balanced over instances), and only the passes over the tile-id digits run on the instances.  The
 // result is the very sequence the full-width sort produces: after the depth passes an instance list is ordered by
 // (depth, row, position in the row's rectangle) either way.  Every pass is a onesweep pass with decoupled look-back
-// (no library sort); the per-tile ranges are read off the sorted tile ids.
+// (no library sort).  The per-tile ranges and the digit histograms of the instance passes come from per-tile instance
+// counts that are accumulated from the rectangles (a difference array over the tile ids), not from the instances.
 #include "common.cuh"
 #include "layout.cuh"
 
 namespace {
 
+// Called by every thread of a 256-thread block after the block's last update of the global histograms.  The block that
+// arrives last of `expected` turns the `digits` 256-bin histograms into exclusive scans (the digit bases of the passes),
+// which saves a launch per histogram kernel.  s_warp: 33 words, s_flag: 1 word of shared memory.
+__device__ __forceinline__ void last_block_digit_bases(const uint32_t* hist, uint32_t* __restrict__ base, int digits,
+                                                       uint32_t* arrivals, uint32_t expected, uint32_t* s_warp,
+                                                       uint32_t* s_flag) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) *s_flag = (atomicAdd(arrivals, 1u) == expected - 1u) ? 1u : 0u;
+  __syncthreads();
+  if (!*s_flag) return;
+  __threadfence();
+  for (int d = 0; d < digits; ++d) {
+    const uint32_t h = ld_volatile_u32(hist + d * SORT_RADIX + threadIdx.x);
+    uint32_t total;
+    base[d * SORT_RADIX + threadIdx.x] = odin_block_exclusive_sum(h, s_warp, &total);
+  }
+}
+
 // ------------------------------------------------------------------------------------------------ row histograms
 // Digit histograms of the depth bits of all rows, for the SORT_DEPTH_DIGITS row passes (warp-aggregated shared
-// atomics: the high digits of a depth take few distinct values).
+// atomics: the high digits of a depth take few distinct values), and their exclusive scans.
 __global__ void __launch_bounds__(256)
-row_hist_kernel(const uint32_t* __restrict__ depth_bits, const uint32_t* __restrict__ num_rows, uint32_t* __restrict__ hist) {
+row_hist_kernel(const uint32_t* __restrict__ depth_bits, const uint32_t* __restrict__ num_rows, uint32_t* __restrict__ hist,
+                uint32_t* __restrict__ base, uint32_t* arrivals) {
   __shared__ uint32_t s_hist[SORT_DEPTH_DIGITS][SORT_RADIX];
+  __shared__ uint32_t s_warp[33], s_flag;
   for (int i = threadIdx.x; i < SORT_DEPTH_DIGITS * (int)SORT_RADIX; i += 256) (&s_hist[0][0])[i] = 0;
   __syncthreads();
   const uint32_t V = *num_rows;
@@ -37,14 +59,7 @@ row_hist_kernel(const uint32_t* __restrict__ depth_bits, const uint32_t* __restr
     const uint32_t c = (&s_hist[0][0])[i];
     if (c) atomicAdd(&hist[i], c);
   }
-}
-
-// exclusive scan of each pass's 256-bin histogram (one block per pass)
-__global__ void __launch_bounds__(SORT_RADIX) digit_base_kernel(const uint32_t* __restrict__ hist, uint32_t* __restrict__ base) {
-  __shared__ uint32_t s_warp[33];
-  uint32_t total;
-  const uint32_t h = hist[blockIdx.x * SORT_RADIX + threadIdx.x];
-  base[blockIdx.x * SORT_RADIX + threadIdx.x] = odin_block_exclusive_sum(h, s_warp, &total);
+  last_block_digit_bases(hist, base, SORT_DEPTH_DIGITS, arrivals, gridDim.x, s_warp, &s_flag);
 }
 
 // ------------------------------------------------------------------------------------------------ onesweep pass
@@ -253,10 +268,20 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
 constexpr int RO_THREADS = 256;
 constexpr int RO_ITEMS = OFFSET_TILE / RO_THREADS;
 
+//
+// The same kernel counts the instances per tile without touching a single instance: one tile row of a rectangle is a
+// run of consecutive tile ids [t0, t1), which adds 1 at t0 and subtracts 1 at t1 in a difference array over the tile
+// ids (global reductions spread over thousands of addresses); tile_scan_kernel integrates it.  Only the first
+// `capacity` instances of the depth order count.
 __global__ void __launch_bounds__(RO_THREADS)
 sorted_offsets_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __restrict__ rect,
-                      const uint32_t* __restrict__ num_rows, uint32_t* __restrict__ sorted_off, uint32_t* ticket,
-                      uint64_t* state, int* status) {
+                      const uint32_t* __restrict__ num_rows, uint32_t capacity, int TX, uint32_t* __restrict__ sorted_off,
+                      uint32_t* __restrict__ tile_diff, uint32_t diff_words, uint32_t* ticket, uint64_t* state,
+                      int* status) {
+  // diff_words != 0: the block first accumulates its part of the difference array in shared memory (`diff_words` =
+  // tiles + 1 words of dynamic shared memory) and adds the non-zero words to the global one at the end: a tile on which
+  // thousands of rectangles pile up would otherwise serialise that many global reductions on one address.
+  extern __shared__ uint32_t s_tdiff[];
   __shared__ uint32_t s_tile, s_base;
   __shared__ uint32_t s_warp[33];
   const uint32_t V = *num_rows;
@@ -265,30 +290,104 @@ sorted_offsets_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __
   __syncthreads();
   const uint32_t tile = s_tile;
   if (tile >= ntiles) return;  // uniform over the block; nobody waits for a tile past the end
+  for (uint32_t i = threadIdx.x; i < diff_words; i += RO_THREADS) s_tdiff[i] = 0;  // (barriers of the scan follow)
   const uint32_t first = tile * OFFSET_TILE + threadIdx.x * RO_ITEMS;
+  ushort4 rc[RO_ITEMS];
   uint32_t cnt[RO_ITEMS];
   uint32_t sum = 0;  // sums are taken modulo 2^32; the true totals fit (M >= 2^32 is an error raised by the projection)
 #pragma unroll
   for (int k = 0; k < RO_ITEMS; ++k) {
-    cnt[k] = 0;
-    if (first + k < V) {
-      const ushort4 rc = rect[sorted_row[first + k]];
-      cnt[k] = ((uint32_t)rc.z - (uint32_t)rc.x) * ((uint32_t)rc.w - (uint32_t)rc.y);
-    }
+    rc[k] = make_ushort4(0, 0, 0, 0);
+    if (first + k < V) rc[k] = rect[sorted_row[first + k]];
+    cnt[k] = ((uint32_t)rc[k].z - (uint32_t)rc[k].x) * ((uint32_t)rc[k].w - (uint32_t)rc[k].y);
     sum += cnt[k];
   }
   uint32_t total;
   const uint32_t before = odin_block_exclusive_sum(sum, s_warp, &total);
   if (threadIdx.x < 32) {
-    const uint64_t base = odin_lookback_u64(state, tile, (uint64_t)total, status);
-    if (threadIdx.x == 0) s_base = (uint32_t)base;
+    const uint64_t b = odin_lookback_u64(state, tile, (uint64_t)total, status);
+    if (threadIdx.x == 0) s_base = (uint32_t)b;
   }
   __syncthreads();
   uint32_t run = s_base + before;
 #pragma unroll
   for (int k = 0; k < RO_ITEMS; ++k) {
     if (first + k < V) sorted_off[first + k] = run;
+    // instances of this row that are emitted: those in front of the capacity
+    uint32_t left = run < capacity ? min(cnt[k], capacity - run) : 0u;
+    const uint32_t w = (uint32_t)rc[k].z - (uint32_t)rc[k].x;
+    for (uint32_t y = rc[k].y; left != 0; ++y) {
+      const uint32_t len = min(w, left);
+      left -= len;
+      const uint32_t t0 = y * (uint32_t)TX + (uint32_t)rc[k].x;
+      uint32_t* diff = diff_words ? s_tdiff : tile_diff;
+      atomicAdd(&diff[t0], 1u);
+      atomicSub(&diff[t0 + len], 1u);
+    }
     run += cnt[k];
+  }
+  if (diff_words) {
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < diff_words; i += RO_THREADS) {
+      const uint32_t d = s_tdiff[i];
+      if (d) atomicAdd(&tile_diff[i], d);
+    }
+  }
+}
+
+// One block.  Integrates the difference array into the instance count of every tile (sums modulo 2^32; every prefix is
+// a true count), writes the tile ranges [first, one past last) as the exclusive scan of the counts, and builds the
+// digit histograms of the instances' tile ids and their exclusive scans (the digit bases of the instance passes).
+constexpr int TS_THREADS = 1024;
+constexpr int TS_ITEMS = 4;
+
+__global__ void __launch_bounds__(TS_THREADS)
+tile_scan_kernel(const uint32_t* __restrict__ tile_diff, uint32_t n_tiles, int tile_passes, uint32_t* __restrict__ ranges,
+                 uint32_t* __restrict__ base) {
+  __shared__ uint32_t s_h[SORT_MAX_TILE_DIGITS][SORT_RADIX];
+  __shared__ uint32_t s_warp[33];
+  for (int i = threadIdx.x; i < SORT_MAX_TILE_DIGITS * (int)SORT_RADIX; i += TS_THREADS) (&s_h[0][0])[i] = 0;
+  __syncthreads();
+  uint32_t carry_count = 0, carry_off = 0;  // count of the tile in front of the batch; instances in front of the batch
+  for (uint32_t b0 = 0; b0 < n_tiles; b0 += TS_THREADS * TS_ITEMS) {
+    const uint32_t t0 = b0 + threadIdx.x * TS_ITEMS;
+    uint32_t c[TS_ITEMS];
+    uint32_t run = 0;
+#pragma unroll
+    for (int k = 0; k < TS_ITEMS; ++k) {
+      run += (t0 + k < n_tiles) ? tile_diff[t0 + k] : 0u;
+      c[k] = run;  // inclusive prefix of the differences inside the thread
+    }
+    uint32_t total;
+    const uint32_t before = carry_count + odin_block_exclusive_sum(run, s_warp, &total);
+    uint32_t mine = 0;
+#pragma unroll
+    for (int k = 0; k < TS_ITEMS; ++k) {
+      c[k] = (t0 + k < n_tiles) ? c[k] + before : 0u;  // instances of tile t0 + k
+      mine += c[k];
+    }
+    carry_count += total;
+    uint32_t total2;
+    uint32_t off = carry_off + odin_block_exclusive_sum(mine, s_warp, &total2);
+    carry_off += total2;
+#pragma unroll
+    for (int k = 0; k < TS_ITEMS; ++k) {
+      const uint32_t t = t0 + k;
+      if (t < n_tiles) {
+        reinterpret_cast<uint2*>(ranges)[t] = make_uint2(off, off + c[k]);
+        if (c[k])
+          for (int d = 0; d < tile_passes; ++d)
+            atomicAdd(&s_h[d][(t >> ((int)SORT_RADIX_BITS * d)) & (SORT_RADIX - 1)], c[k]);
+        off += c[k];
+      }
+    }
+  }
+  __syncthreads();
+  for (int d = 0; d < tile_passes; ++d) {
+    const uint32_t h = threadIdx.x < SORT_RADIX ? s_h[d][threadIdx.x] : 0u;
+    uint32_t total;
+    const uint32_t e = odin_block_exclusive_sum(h, s_warp, &total);
+    if (threadIdx.x < SORT_RADIX) base[d * SORT_RADIX + threadIdx.x] = e;
   }
 }
 
@@ -331,17 +430,15 @@ chunk_rows_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* __res
 // Each chunk of DUP_CHUNK consecutive instance slots finds the positions of the depth order it overlaps, stages their
 // offsets, row ids and rectangles in shared memory, and every thread expands its slots: slot i of a row is tile
 // (y0 + k / w, x0 + k % w) with k = i - offset, w = x1 - x0.  Keys (tile ids) and values (row ids) are written fully
-// coalesced.  The histograms of the tile-id digits are accumulated on the way, per slot with warp aggregation.
+// coalesced.
 __global__ void __launch_bounds__(DUP_THREADS)
 emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* __restrict__ sorted_row,
                       const uint32_t* __restrict__ chunk_row, const ushort4* __restrict__ rect,
                       const uint32_t* __restrict__ num_rows, const uint64_t* __restrict__ num_instances, uint64_t capacity,
-                      int TX, int tile_passes, uint32_t* __restrict__ keys, uint32_t* __restrict__ vals,
-                      uint32_t* __restrict__ hist, int* status) {
+                      int TX, uint32_t* __restrict__ keys, uint32_t* __restrict__ vals, int* status) {
   __shared__ uint32_t s_off[DUP_CHUNK + 1];
   __shared__ ushort4 s_rect[DUP_CHUNK];
   __shared__ uint32_t s_row[DUP_CHUNK];
-  __shared__ uint32_t s_hist[SORT_MAX_TILE_DIGITS][SORT_RADIX];
   __shared__ __align__(16) uint16_t s_map[DUP_CHUNK];  // slot of the chunk -> staged row of the chunk
   __shared__ uint32_t s_scan[DUP_THREADS / 32];
   const uint32_t V = *num_rows;
@@ -349,8 +446,6 @@ emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* _
   const uint64_t M64 = M_all < capacity ? M_all : capacity;
   if (blockIdx.x == 0 && threadIdx.x == 0 && M_all > capacity) odin_set_error(status, ODIN_ERR_CAPACITY);
   const uint32_t M = (uint32_t)(M64 < 0xffffffffull ? M64 : 0xffffffffull);
-  for (int i = threadIdx.x; i < SORT_MAX_TILE_DIGITS * (int)SORT_RADIX; i += DUP_THREADS) (&s_hist[0][0])[i] = 0;
-  __syncthreads();
   const uint32_t chunks = V == 0 ? 0u : (M + DUP_CHUNK - 1) / DUP_CHUNK;
   const unsigned lane = threadIdx.x & 31;
   for (uint32_t chunk = blockIdx.x; chunk < chunks; chunk += gridDim.x) {
@@ -409,58 +504,17 @@ emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* _
 #pragma unroll
     for (int k = 0; k < DUP_ITEMS; ++k) {
       const uint32_t i = c0 + k * DUP_THREADS + threadIdx.x;
-      const bool valid = i < c1;
-      uint32_t tile = 0;
-      if (valid) {
+      if (i < c1) {
         const uint32_t lo = s_map[i - c0];  // staged row that owns this slot
         const ushort4 rc = s_rect[lo];
         const uint32_t local = i - s_off[lo];
         const uint32_t w = (uint32_t)rc.z - (uint32_t)rc.x;
         const uint32_t dy = local / w, dx = local - dy * w;
-        tile = ((uint32_t)rc.y + dy) * (uint32_t)TX + (uint32_t)rc.x + dx;
-        keys[i] = tile;
+        keys[i] = ((uint32_t)rc.y + dy) * (uint32_t)TX + (uint32_t)rc.x + dx;
         vals[i] = s_row[lo];
-      }
-      for (int d = 0; d < tile_passes; ++d) {
-        const uint32_t digit = valid ? ((tile >> (SORT_RADIX_BITS * d)) & (SORT_RADIX - 1)) : (SORT_RADIX + lane);
-        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-        if (valid && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&s_hist[d][digit], (uint32_t)__popc(peers));
       }
     }
     __syncthreads();
-  }
-  for (int i = threadIdx.x; i < tile_passes * (int)SORT_RADIX; i += DUP_THREADS) {
-    const uint32_t c = (&s_hist[0][0])[i];
-    if (c) atomicAdd(&hist[i], c);
-  }
-}
-
-// ------------------------------------------------------------------------------------------------ ranges
-__global__ void __launch_bounds__(256)
-tile_ranges_kernel(const uint32_t* __restrict__ tile_ids, const uint64_t* __restrict__ num_instances, uint64_t capacity,
-                   uint32_t n_tiles, uint32_t* __restrict__ ranges) {
-  const uint64_t M_all = *num_instances;
-  const uint64_t M = M_all < capacity ? M_all : capacity;
-  // four positions per thread from one 16-byte load (the buffer is padded to a multiple of 256 bytes)
-  for (uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; 4 * q < M; q += (uint64_t)gridDim.x * blockDim.x) {
-    const uint64_t i0 = 4 * q;
-    const uint4 k4 = reinterpret_cast<const uint4*>(tile_ids)[q];
-    const uint32_t ks[4] = {k4.x, k4.y, k4.z, k4.w};
-    uint32_t tp = i0 ? tile_ids[i0 - 1] : 0xffffffffu;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint64_t i = i0 + j;
-      if (i >= M) break;
-      const uint32_t t = ks[j];
-      if (t < n_tiles) {
-        if (tp != t) {
-          ranges[2 * t] = (uint32_t)i;
-          if (tp < n_tiles) ranges[2 * tp + 1] = (uint32_t)i;
-        }
-        if (i == M - 1) ranges[2 * t + 1] = (uint32_t)M;
-      }
-      tp = t;
-    }
   }
 }
 
@@ -483,8 +537,11 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   cudaStream_t st = (cudaStream_t)stream;
   const int TX = (width + 15) / 16, TY = (height + 15) / 16;
   const uint32_t n_tiles = (uint32_t)TX * (uint32_t)TY;
-  ODIN_CUDA(cudaMemsetAsync(d_tile_ranges, 0, (size_t)n_tiles * 8, st));
-  if (capacity == 0 || proj->capacity == 0) return ODIN_OK;
+  if (!odin_aligned(d_tile_ranges, 8)) return ODIN_ERR_INVALID_ARG;
+  if (capacity == 0 || proj->capacity == 0) {
+    ODIN_CUDA(cudaMemsetAsync(d_tile_ranges, 0, (size_t)n_tiles * 8, st));
+    return ODIN_OK;
+  }
   if (!d_vals || !proj->rect || !proj->depth) return ODIN_ERR_NULL;
   if ((d_keys && !odin_aligned(d_keys, 16)) || !odin_aligned(d_vals, 16) || !odin_aligned(proj->rect, 8))
     return ODIN_ERR_INVALID_ARG;
@@ -492,12 +549,14 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   if (!ws || !odin_aligned(ws, 256) || ws_bytes < L.total) return ODIN_ERR_WORKSPACE;
   char* base = reinterpret_cast<char*>(ws);
   const int tile_passes = tile_digit_passes(n_tiles);
-  // zero tickets, histograms and the look-back words of the passes that will run
-  const size_t zero = L.inst_states + (size_t)tile_passes * L.tiles * SORT_RADIX * 4;
-  ODIN_CUDA(cudaMemsetAsync(base, 0, zero, st));
+  // zero tickets, histograms, the used part of the difference array and the look-back words of the passes that run
+  ODIN_CUDA(cudaMemsetAsync(base, 0, L.tile_diff + ((size_t)n_tiles + 1) * 4, st));
+  ODIN_CUDA(cudaMemsetAsync(base + L.scan_state, 0,
+                            L.inst_states + (size_t)tile_passes * L.tiles * SORT_RADIX * 4 - L.scan_state, st));
   uint32_t* tickets = reinterpret_cast<uint32_t*>(base + L.header);
   uint32_t* hist = reinterpret_cast<uint32_t*>(base + L.hist);
   uint32_t* dbase = reinterpret_cast<uint32_t*>(base + L.digit_base);
+  uint32_t* tile_diff = reinterpret_cast<uint32_t*>(base + L.tile_diff);
   uint64_t* scan_state = reinterpret_cast<uint64_t*>(base + L.scan_state);
   uint32_t* row_states = reinterpret_cast<uint32_t*>(base + L.row_states);
   uint32_t* inst_states = reinterpret_cast<uint32_t*>(base + L.inst_states);
@@ -515,11 +574,8 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   // ---- rows by depth
   {
     OdinKernelScope ks(ctx, K_ROW_HIST, st);
-    row_hist_kernel<<<row_blocks < sms * 8 ? row_blocks : sms * 8, 256, 0, st>>>(depth_bits, proj->num_rows, hist);
-  }
-  {
-    OdinKernelScope ks(ctx, K_DIGIT_BASE, st);
-    digit_base_kernel<<<SORT_DEPTH_DIGITS, SORT_RADIX, 0, st>>>(hist, dbase);
+    row_hist_kernel<<<row_blocks < sms * 4 ? row_blocks : sms * 4, 256, 0, st>>>(depth_bits, proj->num_rows, hist, dbase,
+                                                                                 tickets + 9);
   }
   ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OS_SMEM));
   ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OS_SMEM));
@@ -541,10 +597,20 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     sorted_row = vin;
   }
   // ---- instances in depth order
+  uint32_t* tile_dbase = dbase + SORT_DEPTH_DIGITS * SORT_RADIX;
   {
     OdinKernelScope ks(ctx, K_ROW_OFFSETS, st);
-    sorted_offsets_kernel<<<(proj->capacity + OFFSET_TILE - 1) / OFFSET_TILE, RO_THREADS, 0, st>>>(
-        sorted_row, rect, proj->num_rows, sorted_off, tickets + 8, scan_state, ctx->d_status);
+    // shared-memory staging of the difference array for images of up to 40,000 tiles (e.g. 4096 x 2304)
+    const uint32_t diff_words = n_tiles + 1 <= 40001u ? n_tiles + 1 : 0u;
+    const size_t diff_smem = (size_t)diff_words * 4;
+    ODIN_CUDA(cudaFuncSetAttribute(sorted_offsets_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 40001 * 4));
+    sorted_offsets_kernel<<<(proj->capacity + OFFSET_TILE - 1) / OFFSET_TILE, RO_THREADS, diff_smem, st>>>(
+        sorted_row, rect, proj->num_rows, (uint32_t)capacity, TX, sorted_off, tile_diff, diff_words, tickets + 8,
+        scan_state, ctx->d_status);
+  }
+  {
+    OdinKernelScope ks(ctx, K_RANGES, st);
+    tile_scan_kernel<<<1, TS_THREADS, 0, st>>>(tile_diff, n_tiles, tile_passes, d_tile_ranges, tile_dbase);
   }
   const uint64_t chunks_cap = (capacity + DUP_CHUNK - 1) / DUP_CHUNK;
   {
@@ -554,18 +620,12 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   }
   // the emission goes to the buffers from which `tile_passes` ping-pong steps end in d_vals
   int cur = tile_passes & 1;
-  uint32_t* tile_hist = hist + SORT_DEPTH_DIGITS * SORT_RADIX;
-  uint32_t* tile_dbase = dbase + SORT_DEPTH_DIGITS * SORT_RADIX;
   {
     OdinKernelScope ks(ctx, K_EMIT, st);
     const uint32_t grid = (uint32_t)(chunks_cap < (uint64_t)sms * 5 ? chunks_cap : (uint64_t)sms * 5);
     emit_instances_kernel<<<grid, DUP_THREADS, 0, st>>>(sorted_off, sorted_row, chunk_row, rect, proj->num_rows,
-                                                        proj->num_instances, capacity, TX, tile_passes, inst_keys[cur],
-                                                        inst_vals[cur], tile_hist, ctx->d_status);
-  }
-  {
-    OdinKernelScope ks(ctx, K_DIGIT_BASE, st);
-    digit_base_kernel<<<tile_passes, SORT_RADIX, 0, st>>>(tile_hist, tile_dbase);
+                                                        proj->num_instances, capacity, TX, inst_keys[cur], inst_vals[cur],
+                                                        ctx->d_status);
   }
   // ---- instances by tile id
   const uint32_t os_grid = L.tiles < sms * OS_BLOCKS ? L.tiles : sms * OS_BLOCKS;
@@ -577,16 +637,12 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
           inst_keys[cur], inst_vals[cur], inst_keys[cur ^ 1], inst_vals[cur ^ 1], nullptr, nullptr, nullptr,
           proj->num_instances, capacity, p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
           tickets + SORT_DEPTH_DIGITS + p, ctx->d_status);
-    else
+    else  // the sorted tile ids themselves are not needed any more: the ranges came from the tile counts
       onesweep_kernel<true><<<os_grid, OS_THREADS, OS_SMEM, st>>>(
-          inst_keys[cur], inst_vals[cur], inst_keys[cur ^ 1], inst_vals[cur ^ 1], d_keys, depth_bits, nullptr,
+          inst_keys[cur], inst_vals[cur], nullptr, inst_vals[cur ^ 1], d_keys, depth_bits, nullptr,
           proj->num_instances, capacity, p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
           tickets + SORT_DEPTH_DIGITS + p, ctx->d_status);
     cur ^= 1;
   }
-  const uint64_t rblocks = (capacity + 255) / 256;
-  const uint32_t rgrid = (uint32_t)(rblocks < (uint64_t)sms * 8 ? rblocks : (uint64_t)sms * 8);
-  OdinKernelScope ks(ctx, K_RANGES, st);
-  tile_ranges_kernel<<<rgrid, 256, 0, st>>>(inst_keys[cur], proj->num_instances, capacity, n_tiles, d_tile_ranges);
   return odin_launch_status();
 }

@@ -38,6 +38,8 @@ struct BinSortLayout {
   size_t header;       // tickets: u32 [0..3] row passes, [4..6] instance passes, [8] offset scan; 256 B
   size_t hist;         // [SORT_MAX_PASSES][SORT_RADIX] u32 global digit histograms (row digits first)
   size_t digit_base;   // [SORT_MAX_PASSES][SORT_RADIX] u32 exclusive scans of the histograms
+  size_t tile_diff;    // u32[2^20 + 1] difference array of the instance counts over the tile ids (the first
+                       // tiles + 1 words are used and must be zero)
   size_t scan_state;   // u64 per OFFSET_TILE rows: look-back words of the sorted-offset scan
   size_t row_states;   // [SORT_DEPTH_DIGITS][row_tiles][SORT_RADIX] u32 look-back words
   size_t inst_states;  // [SORT_MAX_TILE_DIGITS][tiles][SORT_RADIX] u32 look-back words
@@ -62,6 +64,7 @@ static inline BinSortLayout binsort_layout(uint64_t capacity, uint32_t rows) {
   L.header = o; o += 256;
   L.hist = o; o += ws_align((size_t)SORT_MAX_PASSES * SORT_RADIX * 4);
   L.digit_base = o; o += ws_align((size_t)SORT_MAX_PASSES * SORT_RADIX * 4);
+  L.tile_diff = o; o += ws_align((((size_t)1 << 20) + 1) * 4);
   L.scan_state = o; o += ws_align(((size_t)rows + OFFSET_TILE - 1) / OFFSET_TILE * 8 + 8);
   L.row_states = o; o += ws_align((size_t)SORT_DEPTH_DIGITS * L.row_tiles * SORT_RADIX * 4);
   L.inst_states = o; o += ws_align((size_t)SORT_MAX_TILE_DIGITS * L.tiles * SORT_RADIX * 4);
