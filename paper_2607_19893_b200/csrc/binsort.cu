@@ -65,12 +65,16 @@ row_hist_kernel(const uint32_t* __restrict__ depth_bits, const uint32_t* __restr
 // ------------------------------------------------------------------------------------------------ onesweep pass
 constexpr int OS_THREADS = 256;
 constexpr int OS_WARPS = OS_THREADS / 32;
-constexpr int OS_ITEMS = SORT_TILE / OS_THREADS;  // 16 keys per thread
+constexpr int OS_INST_ITEMS = SORT_TILE / OS_THREADS;     // 16 keys per thread in the passes over the instances
+constexpr int OS_ROW_ITEMS = ROW_SORT_TILE / OS_THREADS;  // 4 in the passes over the rows
 constexpr int OS_DPT = SORT_RADIX / OS_THREADS;   // digits owned by a thread
-constexpr int OS_WINDOW = 2;                      // predecessors fetched per look-back step and digit
+constexpr int OS_INST_WINDOW = 2;                 // predecessors fetched per look-back step and digit (instances)
+constexpr int OS_ROW_WINDOW = 8;                  // ... and in the passes over the rows
 constexpr int OS_BLOCKS = 4;                      // resident blocks per SM
 constexpr uint32_t OS_FLAG_AGG = 1u << 30, OS_FLAG_INC = 2u << 30, OS_VALUE = (1u << 30) - 1;
-constexpr size_t OS_SMEM = (size_t)SORT_TILE * 4 + (size_t)SORT_TILE * 4 + (size_t)OS_WARPS * SORT_RADIX * 4 + 2 * SORT_RADIX * 4 + 16;
+constexpr size_t os_smem_bytes(int items) {
+  return (size_t)items * OS_THREADS * 8 + (size_t)OS_WARPS * SORT_RADIX * 4 + 2 * SORT_RADIX * 4 + 16;
+}
 
 // One pass over one 8-bit digit of 32-bit keys.  Persistent blocks take 4096-key tiles by ticket.  Per tile:
 // warp-striped loads, per-warp digit ranking with match.any (stable), block digit counts published for look-back,
@@ -80,7 +84,9 @@ constexpr size_t OS_SMEM = (size_t)SORT_TILE * 4 + (size_t)SORT_TILE * 4 + (size
 //   keys_out == nullptr: the keys are not needed afterwards (last pass over the rows)
 //   WIDE: the last pass over the instances may also write the full 64-bit key key << 32 | depth_bits[value]
 //   the number of keys is *count32 if given, else min(*count64, capacity)
-template <bool WIDE>
+//   ITEMS keys per thread, ITEMS * 256 per tile: 16 for the instances; 4 for the rows, of which there are so few that a
+//   pass is one wave of blocks and its duration is the latency of one tile, mostly the ITEMS-long ranking chain
+template <bool WIDE, int ITEMS, int WINDOW>
 __global__ void __launch_bounds__(OS_THREADS, OS_BLOCKS)
 onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in, uint32_t* __restrict__ keys_out,
                 uint32_t* __restrict__ vals_out, uint64_t* __restrict__ keys64_out, const uint32_t* __restrict__ depth_bits,
@@ -88,8 +94,9 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
                 const uint32_t* __restrict__ digit_base, uint32_t* states, uint32_t* ticket, int* status) {
   extern __shared__ __align__(16) unsigned char os_smem[];
   uint32_t* s_keys = reinterpret_cast<uint32_t*>(os_smem);
-  uint32_t* s_vals = s_keys + SORT_TILE;
-  uint32_t(*s_warp_hist)[SORT_RADIX] = reinterpret_cast<uint32_t(*)[SORT_RADIX]>(s_vals + SORT_TILE);
+  constexpr uint32_t TILE = (uint32_t)ITEMS * OS_THREADS;
+  uint32_t* s_vals = s_keys + TILE;
+  uint32_t(*s_warp_hist)[SORT_RADIX] = reinterpret_cast<uint32_t(*)[SORT_RADIX]>(s_vals + TILE);
   uint32_t* s_digit_start = &s_warp_hist[0][0] + OS_WARPS * SORT_RADIX;
   uint32_t* s_global = s_digit_start + SORT_RADIX;
   uint32_t* s_misc = s_global + SORT_RADIX;  // [0] tile ticket
@@ -103,18 +110,18 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
     M64 = M_all < capacity ? M_all : capacity;
   }
   const uint32_t M = (uint32_t)(M64 < (uint64_t)OS_VALUE ? M64 : (uint64_t)OS_VALUE);
-  const uint32_t ntiles = (M + SORT_TILE - 1) / SORT_TILE;
+  const uint32_t ntiles = (M + TILE - 1) / TILE;
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t lt_mask = (1u << lane) - 1u;
 
   // The keys and values of the NEXT tile are requested as soon as the registers of the current one are free (after
   // the exchange through shared memory), so that their latency overlaps the global scatter of the current tile.
-  uint32_t key[OS_ITEMS];
-  uint32_t val[OS_ITEMS];
+  uint32_t key[ITEMS];
+  uint32_t val[ITEMS];
   auto load_tile = [&](uint32_t t) {
-    const uint32_t wb = t * SORT_TILE + warp * (32 * OS_ITEMS);
+    const uint32_t wb = t * TILE + warp * (32 * ITEMS);
 #pragma unroll
-    for (int j = 0; j < OS_ITEMS; ++j) {
+    for (int j = 0; j < ITEMS; ++j) {
       const uint32_t i = wb + 32 * j + lane;
       const bool in = t < ntiles && i < M;
       key[j] = in ? keys_in[i] : ~0u;  // padding sorts to the end of the tile and is never written
@@ -129,12 +136,12 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
   while (tile < ntiles) {
     for (int i = threadIdx.x; i < OS_WARPS * (int)SORT_RADIX; i += OS_THREADS) (&s_warp_hist[0][0])[i] = 0;
     __syncthreads();
-    const uint32_t tile_base = tile * SORT_TILE;
-    const uint32_t tile_count = min((uint32_t)SORT_TILE, M - tile_base);
+    const uint32_t tile_base = tile * TILE;
+    const uint32_t tile_count = min(TILE, M - tile_base);
 
-    uint32_t pos[OS_ITEMS];
+    uint32_t pos[ITEMS];
 #pragma unroll
-    for (int j = 0; j < OS_ITEMS; ++j) {
+    for (int j = 0; j < ITEMS; ++j) {
       const uint32_t d = (key[j] >> shift) & (SORT_RADIX - 1);
       const uint32_t peers = __match_any_sync(0xffffffffu, d);
       const int leader = __ffs(peers) - 1;
@@ -188,13 +195,13 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
       while (busy) {
         busy = false;
         bool stalled = true;  // cleared as soon as any predecessor word is consumed
-        // a window of OS_WINDOW predecessors per digit is fetched at once: the walk is a chain of dependent L2 round
+        // a window of WINDOW predecessors per digit is fetched at once: the walk is a chain of dependent L2 round
         // trips, and when a launch starts every resident tile has hundreds of aggregates in front of it
-        uint32_t s[OS_DPT][OS_WINDOW];
+        uint32_t s[OS_DPT][WINDOW];
 #pragma unroll
         for (int q = 0; q < OS_DPT; ++q)
 #pragma unroll
-          for (int k = 0; k < OS_WINDOW; ++k)
+          for (int k = 0; k < WINDOW; ++k)
             s[q][k] = (t[q] - k >= 0)
                           ? ld_volatile_u32(states + (size_t)(t[q] - k) * SORT_RADIX + threadIdx.x + q * OS_THREADS)
                           : 0u;
@@ -202,7 +209,7 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
         for (int q = 0; q < OS_DPT; ++q) {
           if (t[q] < 0) continue;
 #pragma unroll
-          for (int k = 0; k < OS_WINDOW; ++k) {
+          for (int k = 0; k < WINDOW; ++k) {
             if (t[q] < 0) break;
             const uint32_t flag = s[q][k] >> 30;
             if (flag == 0) break;  // not published yet: use what precedes it, come back
@@ -230,7 +237,7 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
     __syncthreads();
 
 #pragma unroll
-    for (int j = 0; j < OS_ITEMS; ++j) {
+    for (int j = 0; j < ITEMS; ++j) {
       const uint32_t dg = (key[j] >> shift) & (SORT_RADIX - 1);
       const uint32_t slot = s_digit_start[dg] + s_warp_hist[warp][dg] + pos[j];
       s_keys[slot] = key[j];
@@ -241,7 +248,7 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
     const uint32_t next = s_misc[0];
     load_tile(next);  // in flight while the current tile is written out
 #pragma unroll
-    for (int j = 0; j < OS_ITEMS; ++j) {
+    for (int j = 0; j < ITEMS; ++j) {
       const uint32_t slot = j * OS_THREADS + threadIdx.x;
       if (slot < tile_count) {
         const uint32_t k = s_keys[slot];
@@ -577,8 +584,11 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     row_hist_kernel<<<row_blocks < sms * 4 ? row_blocks : sms * 4, 256, 0, st>>>(depth_bits, proj->num_rows, hist, dbase,
                                                                                  tickets + 9);
   }
-  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OS_SMEM));
-  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OS_SMEM));
+  constexpr size_t OS_SMEM = os_smem_bytes(OS_INST_ITEMS), OS_ROW_SMEM = os_smem_bytes(OS_ROW_ITEMS);
+  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<false, OS_INST_ITEMS, OS_INST_WINDOW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)OS_SMEM));
+  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<true, OS_INST_ITEMS, OS_INST_WINDOW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)OS_SMEM));
   const uint32_t* sorted_row = nullptr;
   {
     const uint32_t grid = L.row_tiles < sms * OS_BLOCKS ? L.row_tiles : sms * OS_BLOCKS;
@@ -588,7 +598,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
       OdinKernelScope ks(ctx, K_ROW_SORT, st);
       uint32_t* kout = (p + 1 < SORT_DEPTH_DIGITS) ? row_keys[p & 1] : nullptr;
       uint32_t* vout = row_vals[p & 1];
-      onesweep_kernel<false><<<grid, OS_THREADS, OS_SMEM, st>>>(
+      onesweep_kernel<false, OS_ROW_ITEMS, OS_ROW_WINDOW><<<grid, OS_THREADS, OS_ROW_SMEM, st>>>(
           kin, vin, kout, vout, nullptr, nullptr, proj->num_rows, nullptr, 0, p * (int)SORT_RADIX_BITS,
           dbase + p * SORT_RADIX, row_states + (size_t)p * L.row_tiles * SORT_RADIX, tickets + p, ctx->d_status);
       kin = kout;
@@ -633,12 +643,12 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     OdinKernelScope ks(ctx, K_ONESWEEP, st);
     uint32_t* states = inst_states + (size_t)p * L.tiles * SORT_RADIX;
     if (p + 1 < tile_passes)
-      onesweep_kernel<false><<<os_grid, OS_THREADS, OS_SMEM, st>>>(
+      onesweep_kernel<false, OS_INST_ITEMS, OS_INST_WINDOW><<<os_grid, OS_THREADS, OS_SMEM, st>>>(
           inst_keys[cur], inst_vals[cur], inst_keys[cur ^ 1], inst_vals[cur ^ 1], nullptr, nullptr, nullptr,
           proj->num_instances, capacity, p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
           tickets + SORT_DEPTH_DIGITS + p, ctx->d_status);
     else  // the sorted tile ids themselves are not needed any more: the ranges came from the tile counts
-      onesweep_kernel<true><<<os_grid, OS_THREADS, OS_SMEM, st>>>(
+      onesweep_kernel<true, OS_INST_ITEMS, OS_INST_WINDOW><<<os_grid, OS_THREADS, OS_SMEM, st>>>(
           inst_keys[cur], inst_vals[cur], nullptr, inst_vals[cur ^ 1], d_keys, depth_bits, nullptr,
           proj->num_instances, capacity, p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
           tickets + SORT_DEPTH_DIGITS + p, ctx->d_status);
