@@ -137,9 +137,9 @@ def kernel_bytes(n, f, v, m, m_proc, p, t, tile_passes, n_pairs):
     b = algorithmic_bytes(n, f, v, m, m_proc, p, t, 0, n_pairs)
     b.pop("total")
     b["row_sort"] = 4 * v + 4 * 16 * v - 8 * v
-    b["emit_instances"] = 4 * v + 16 * v + 8 * m
-    b["onesweep_pass"] = tile_passes * 16 * m
-    b["tile_ranges"] = 12 * t
+    b["emit_instances"] = 4 * v + 16 * v + 8 * m + 12 * t  # offsets + emission; the tile scan rides in the emission
+    b["onesweep_pass"] = tile_passes * 16 * m - 4 * m       # the last pass writes the values only
+    b.pop("tile_ranges")
     b["total"] = float(sum(b.values()))
     return b
 
@@ -356,7 +356,7 @@ def main():
         # kernels that split one stage (head + tail of the blend, the three projection kernels, ...) are judged
         # together: the stage's algorithmic work over the summed time of its kernels in one step
         stage_of = {"render_fwd_tail": "render_fwd", "render_bwd_tail": "render_bwd_blend", "project_cull": "project",
-                    "project_scan": "project", "project_rows": "project", "chunk_rows": "emit_instances",
+                    "project_scan": "project", "project_rows": "project",
                     "adam_sh": "adam", "adam_geom": "adam", "l1_finish": "l1_loss",
                     "zero_rows": "render_bwd_blend", "row_hist": "row_sort", "row_sort_pass": "row_sort",
                     "row_offsets": "emit_instances"}

@@ -274,17 +274,22 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
 // blocks ordered by ticket.
 constexpr int RO_THREADS = 256;
 constexpr int RO_ITEMS = OFFSET_TILE / RO_THREADS;
+// the instances are emitted in chunks of DUP_CHUNK consecutive slots (emit_instances_kernel)
+constexpr int DUP_THREADS = 256;
+constexpr int DUP_ITEMS = 8;
+constexpr int DUP_CHUNK = DUP_THREADS * DUP_ITEMS;  // a chunk spans at most DUP_CHUNK rows
 
 //
 // The same kernel counts the instances per tile without touching a single instance: one tile row of a rectangle is a
 // run of consecutive tile ids [t0, t1), which adds 1 at t0 and subtracts 1 at t1 in a difference array over the tile
-// ids (global reductions spread over thousands of addresses); tile_scan_kernel integrates it.  Only the first
-// `capacity` instances of the depth order count.
+// ids; tile_scan_block integrates it.  Only the first `capacity` instances of the depth order count.
+// It also fills chunk_row[c] = the position (in depth order) of the row whose slots contain slot c * DUP_CHUNK: a row
+// writes an entry for every chunk boundary that falls inside its slot range (usually none or one).
 __global__ void __launch_bounds__(RO_THREADS)
 sorted_offsets_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __restrict__ rect,
                       const uint32_t* __restrict__ num_rows, uint32_t capacity, int TX, uint32_t* __restrict__ sorted_off,
-                      uint32_t* __restrict__ tile_diff, uint32_t diff_words, uint32_t* ticket, uint64_t* state,
-                      int* status) {
+                      uint32_t* __restrict__ chunk_row, uint32_t chunks_cap, uint32_t* __restrict__ tile_diff,
+                      uint32_t diff_words, uint32_t* ticket, uint64_t* state, int* status) {
   // diff_words != 0: the block first accumulates its part of the difference array in shared memory (`diff_words` =
   // tiles + 1 words of dynamic shared memory) and adds the non-zero words to the global one at the end: a tile on which
   // thousands of rectangles pile up would otherwise serialise that many global reductions on one address.
@@ -319,7 +324,12 @@ sorted_offsets_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __
   uint32_t run = s_base + before;
 #pragma unroll
   for (int k = 0; k < RO_ITEMS; ++k) {
-    if (first + k < V) sorted_off[first + k] = run;
+    if (first + k < V) {
+      sorted_off[first + k] = run;
+      const uint64_t hi = (uint64_t)run + cnt[k];
+      for (uint64_t c = ((uint64_t)run + DUP_CHUNK - 1) / DUP_CHUNK; c * DUP_CHUNK < hi && c < chunks_cap; ++c)
+        chunk_row[c] = first + k;
+    }
     // instances of this row that are emitted: those in front of the capacity
     uint32_t left = run < capacity ? min(cnt[k], capacity - run) : 0u;
     const uint32_t w = (uint32_t)rc[k].z - (uint32_t)rc[k].x;
@@ -342,21 +352,21 @@ sorted_offsets_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __
   }
 }
 
-// One block.  Integrates the difference array into the instance count of every tile (sums modulo 2^32; every prefix is
-// a true count), writes the tile ranges [first, one past last) as the exclusive scan of the counts, and builds the
-// digit histograms of the instances' tile ids and their exclusive scans (the digit bases of the instance passes).
-constexpr int TS_THREADS = 1024;
+// Run by ONE block (all of its threads).  Integrates the difference array into the instance count of every tile (sums
+// modulo 2^32; every prefix is a true count), writes the tile ranges [first, one past last) as the exclusive scan of
+// the counts, and builds the digit histograms of the instances' tile ids and their exclusive scans (the digit bases of
+// the instance passes).  Needs blockDim.x >= 256.
 constexpr int TS_ITEMS = 4;
 
-__global__ void __launch_bounds__(TS_THREADS)
-tile_scan_kernel(const uint32_t* __restrict__ tile_diff, uint32_t n_tiles, int tile_passes, uint32_t* __restrict__ ranges,
-                 uint32_t* __restrict__ base) {
+__device__ __forceinline__ void tile_scan_block(const uint32_t* __restrict__ tile_diff, uint32_t n_tiles, int tile_passes,
+                                                uint32_t* __restrict__ ranges, uint32_t* __restrict__ base) {
   __shared__ uint32_t s_h[SORT_MAX_TILE_DIGITS][SORT_RADIX];
   __shared__ uint32_t s_warp[33];
-  for (int i = threadIdx.x; i < SORT_MAX_TILE_DIGITS * (int)SORT_RADIX; i += TS_THREADS) (&s_h[0][0])[i] = 0;
+  const unsigned lane = threadIdx.x & 31;
+  for (int i = threadIdx.x; i < SORT_MAX_TILE_DIGITS * (int)SORT_RADIX; i += blockDim.x) (&s_h[0][0])[i] = 0;
   __syncthreads();
   uint32_t carry_count = 0, carry_off = 0;  // count of the tile in front of the batch; instances in front of the batch
-  for (uint32_t b0 = 0; b0 < n_tiles; b0 += TS_THREADS * TS_ITEMS) {
+  for (uint32_t b0 = 0; b0 < n_tiles; b0 += blockDim.x * TS_ITEMS) {
     const uint32_t t0 = b0 + threadIdx.x * TS_ITEMS;
     uint32_t c[TS_ITEMS];
     uint32_t run = 0;
@@ -382,10 +392,22 @@ tile_scan_kernel(const uint32_t* __restrict__ tile_diff, uint32_t n_tiles, int t
       const uint32_t t = t0 + k;
       if (t < n_tiles) {
         reinterpret_cast<uint2*>(ranges)[t] = make_uint2(off, off + c[k]);
-        if (c[k])
-          for (int d = 0; d < tile_passes; ++d)
-            atomicAdd(&s_h[d][(t >> ((int)SORT_RADIX_BITS * d)) & (SORT_RADIX - 1)], c[k]);
+        if (c[k]) atomicAdd(&s_h[0][t & (SORT_RADIX - 1)], c[k]);
         off += c[k];
+      }
+    }
+    // higher digits: the 128 consecutive tiles of a warp share the digit unless they straddle a multiple of 256 (or
+    // 65536), so the warp adds its sum once instead of 128 times to the same word
+    for (int d = 1; d < tile_passes; ++d) {
+      const int shift = (int)SORT_RADIX_BITS * d;
+      const uint32_t first = __shfl_sync(0xffffffffu, t0, 0), last = __shfl_sync(0xffffffffu, t0 + TS_ITEMS - 1, 31);
+      if ((first >> shift) == (last >> shift)) {
+        const uint32_t sum = __reduce_add_sync(0xffffffffu, mine);
+        if (lane == 0 && sum) atomicAdd(&s_h[d][(first >> shift) & (SORT_RADIX - 1)], sum);
+      } else {
+#pragma unroll
+        for (int k = 0; k < TS_ITEMS; ++k)
+          if (c[k]) atomicAdd(&s_h[d][((t0 + k) >> shift) & (SORT_RADIX - 1)], c[k]);
       }
     }
   }
@@ -399,9 +421,6 @@ tile_scan_kernel(const uint32_t* __restrict__ tile_diff, uint32_t n_tiles, int t
 }
 
 // ------------------------------------------------------------------------------------------------ emission
-constexpr int DUP_THREADS = 256;
-constexpr int DUP_ITEMS = 8;
-constexpr int DUP_CHUNK = DUP_THREADS * DUP_ITEMS;  // instances per chunk; a chunk spans at most DUP_CHUNK rows
 
 // Cooperative 256-ary upper bound: first r in [0, V) with off[r] > x (V if none).  All threads must call.
 __device__ __forceinline__ uint32_t block_upper_bound(const uint32_t* __restrict__ off, uint32_t V, uint32_t x) {
@@ -420,29 +439,23 @@ __device__ __forceinline__ uint32_t block_upper_bound(const uint32_t* __restrict
   return lo;
 }
 
-// chunk_row[c] = the position (in depth order) of the row whose slots contain slot c * DUP_CHUNK (one thread per
-// position; a row writes an entry for every chunk boundary that falls inside its slot range, usually none or one).
-__global__ void __launch_bounds__(256)
-chunk_rows_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* __restrict__ num_rows,
-                  const uint64_t* __restrict__ num_instances, uint32_t chunks_cap, uint32_t* __restrict__ chunk_row) {
-  const uint32_t V = *num_rows;
-  const uint64_t M_all = *num_instances;
-  for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
-    const uint64_t lo = sorted_off[r];
-    const uint64_t hi = (r + 1 < V) ? (uint64_t)sorted_off[r + 1] : M_all;
-    for (uint64_t c = (lo + DUP_CHUNK - 1) / DUP_CHUNK; c * DUP_CHUNK < hi && c < chunks_cap; ++c) chunk_row[c] = r;
-  }
-}
-
 // Each chunk of DUP_CHUNK consecutive instance slots finds the positions of the depth order it overlaps, stages their
 // offsets, row ids and rectangles in shared memory, and every thread expands its slots: slot i of a row is tile
 // (y0 + k / w, x0 + k % w) with k = i - offset, w = x1 - x0.  Keys (tile ids) and values (row ids) are written fully
-// coalesced.
+// coalesced.  The last block of the grid does something else at the same time: the scan over the tiles (ranges and
+// digit bases), which is one block's work and would otherwise be a launch of its own on the critical path.
 __global__ void __launch_bounds__(DUP_THREADS)
 emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* __restrict__ sorted_row,
                       const uint32_t* __restrict__ chunk_row, const ushort4* __restrict__ rect,
                       const uint32_t* __restrict__ num_rows, const uint64_t* __restrict__ num_instances, uint64_t capacity,
-                      int TX, uint32_t* __restrict__ keys, uint32_t* __restrict__ vals, int* status) {
+                      int TX, uint32_t* __restrict__ keys, uint32_t* __restrict__ vals, int* status,
+                      const uint32_t* __restrict__ tile_diff, uint32_t n_tiles, int tile_passes,
+                      uint32_t* __restrict__ ranges, uint32_t* __restrict__ tile_dbase) {
+  if (blockIdx.x == 0) {  // block 0: it is scheduled first
+    tile_scan_block(tile_diff, n_tiles, tile_passes, ranges, tile_dbase);
+    return;
+  }
+  const uint32_t emit_blocks = gridDim.x - 1, emit_block = blockIdx.x - 1;
   __shared__ uint32_t s_off[DUP_CHUNK + 1];
   __shared__ ushort4 s_rect[DUP_CHUNK];
   __shared__ uint32_t s_row[DUP_CHUNK];
@@ -451,11 +464,11 @@ emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* _
   const uint32_t V = *num_rows;
   const uint64_t M_all = *num_instances;
   const uint64_t M64 = M_all < capacity ? M_all : capacity;
-  if (blockIdx.x == 0 && threadIdx.x == 0 && M_all > capacity) odin_set_error(status, ODIN_ERR_CAPACITY);
+  if (emit_block == 0 && threadIdx.x == 0 && M_all > capacity) odin_set_error(status, ODIN_ERR_CAPACITY);
   const uint32_t M = (uint32_t)(M64 < 0xffffffffull ? M64 : 0xffffffffull);
   const uint32_t chunks = V == 0 ? 0u : (M + DUP_CHUNK - 1) / DUP_CHUNK;
   const unsigned lane = threadIdx.x & 31;
-  for (uint32_t chunk = blockIdx.x; chunk < chunks; chunk += gridDim.x) {
+  for (uint32_t chunk = emit_block; chunk < chunks; chunk += emit_blocks) {
     const uint32_t c0 = chunk * DUP_CHUNK;
     const uint32_t c1 = (M - c0 < (uint32_t)DUP_CHUNK) ? M : c0 + DUP_CHUNK;
     // first and last position of the chunk from the chunk table; only the last chunk has to search for its end
@@ -581,7 +594,8 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   // ---- rows by depth
   {
     OdinKernelScope ks(ctx, K_ROW_HIST, st);
-    row_hist_kernel<<<row_blocks < sms * 4 ? row_blocks : sms * 4, 256, 0, st>>>(depth_bits, proj->num_rows, hist, dbase,
+    // one block per SM at most: every block ends with 1024 global reductions onto the same 1024 words
+    row_hist_kernel<<<row_blocks < sms ? row_blocks : sms, 256, 0, st>>>(depth_bits, proj->num_rows, hist, dbase,
                                                                                  tickets + 9);
   }
   constexpr size_t OS_SMEM = os_smem_bytes(OS_INST_ITEMS), OS_ROW_SMEM = os_smem_bytes(OS_ROW_ITEMS);
@@ -608,6 +622,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   }
   // ---- instances in depth order
   uint32_t* tile_dbase = dbase + SORT_DEPTH_DIGITS * SORT_RADIX;
+  const uint64_t chunks_cap = (capacity + DUP_CHUNK - 1) / DUP_CHUNK;
   {
     OdinKernelScope ks(ctx, K_ROW_OFFSETS, st);
     // shared-memory staging of the difference array for images of up to 40,000 tiles (e.g. 4096 x 2304)
@@ -615,27 +630,18 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     const size_t diff_smem = (size_t)diff_words * 4;
     ODIN_CUDA(cudaFuncSetAttribute(sorted_offsets_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 40001 * 4));
     sorted_offsets_kernel<<<(proj->capacity + OFFSET_TILE - 1) / OFFSET_TILE, RO_THREADS, diff_smem, st>>>(
-        sorted_row, rect, proj->num_rows, (uint32_t)capacity, TX, sorted_off, tile_diff, diff_words, tickets + 8,
-        scan_state, ctx->d_status);
-  }
-  {
-    OdinKernelScope ks(ctx, K_RANGES, st);
-    tile_scan_kernel<<<1, TS_THREADS, 0, st>>>(tile_diff, n_tiles, tile_passes, d_tile_ranges, tile_dbase);
-  }
-  const uint64_t chunks_cap = (capacity + DUP_CHUNK - 1) / DUP_CHUNK;
-  {
-    OdinKernelScope ks(ctx, K_CHUNK_ROWS, st);
-    chunk_rows_kernel<<<row_blocks < sms * 8 ? row_blocks : sms * 8, 256, 0, st>>>(
-        sorted_off, proj->num_rows, proj->num_instances, (uint32_t)chunks_cap, chunk_row);
+        sorted_row, rect, proj->num_rows, (uint32_t)capacity, TX, sorted_off, chunk_row, (uint32_t)chunks_cap, tile_diff,
+        diff_words, tickets + 8, scan_state, ctx->d_status);
   }
   // the emission goes to the buffers from which `tile_passes` ping-pong steps end in d_vals
   int cur = tile_passes & 1;
   {
     OdinKernelScope ks(ctx, K_EMIT, st);
-    const uint32_t grid = (uint32_t)(chunks_cap < (uint64_t)sms * 5 ? chunks_cap : (uint64_t)sms * 5);
+    const uint32_t grid = (uint32_t)(chunks_cap < (uint64_t)sms * 5 - 1 ? chunks_cap : (uint64_t)sms * 5 - 1) + 1;
     emit_instances_kernel<<<grid, DUP_THREADS, 0, st>>>(sorted_off, sorted_row, chunk_row, rect, proj->num_rows,
                                                         proj->num_instances, capacity, TX, inst_keys[cur], inst_vals[cur],
-                                                        ctx->d_status);
+                                                        ctx->d_status, tile_diff, n_tiles, tile_passes, d_tile_ranges,
+                                                        tile_dbase);
   }
   // ---- instances by tile id
   const uint32_t os_grid = L.tiles < sms * OS_BLOCKS ? L.tiles : sms * OS_BLOCKS;
