@@ -38,6 +38,12 @@ MASK_SLOTS = CONFLICT_WINDOW + 1
 # Blend kernels are bound by plain fp32 ALU work.  Peak = SMs x 128 fp32 lanes x 2 (fma) x max SM clock.
 ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 FLOPS_PER_PAIR = {"render_fwd": 25.0, "render_bwd_blend": 75.0}
+# DRAM traffic (read + write, bytes per view) of the kernels of a stage, from the ncu capture of one view step that
+# profiles/view_step_kernels_cfg3.txt summarises; only that workload was captured
+NCU_TRAFFIC = {"cfg3_1m_sh3_1600x1066": {
+    "render_bwd_blend": 45.2e6 + 34.9e6, "render_fwd": 9.7e6 + 8.4e6, "onesweep_pass": 119.8e6 + 94.5e6,
+    "adam": 425.6e6 + 195.8e6, "emit_instances": 31.6e6 + 3.9e6, "row_sort": 1.3e6 + 4 * 2.7e6,
+    "project": 40.0e6 + 4.0e6 + 128.7e6, "render_bwd_project": 167.6e6, "touched_set": 4.0e6, "l1_loss": 41.1e6}}
 
 
 def measured_peaks():
@@ -144,6 +150,28 @@ def kernel_bytes(n, f, v, m, m_proc, p, t, tile_passes, n_pairs):
     return b
 
 
+# ---- replicas: the only multi-rank logic of this bench (no collective on the data path) ---------------------------
+def replica_view(step: int, rank: int, n_views: int) -> int:
+    """Rank r starts its replica at view r so that replicas do not all render the same camera at the same time."""
+    return (step + rank) % n_views
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    """The slowest rank's time: every multi-rank number is the maximum over the ranks."""
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(steps: int, world: int, seconds: float) -> float:
+    """Views per second of the whole job: every rank processed `steps` views in (at most) `seconds`."""
+    return world * steps / seconds
+
+
 def run_reference(args, rank):
     """The oracle as it stands, on the host cores, on the same workload (rank 0 only)."""
     if rank != 0:
@@ -235,8 +263,7 @@ def main():
         row_cap = min(n, max(row_cap, 1_600_000))
     tr = ViewTrainer(scene, W, H, row_cap, INSTANCE_CAP[args.config], mask_slots=MASK_SLOTS, device=local_rank)
     n_views = min(len(w.cameras), args.steps + args.warmup)
-    # rank r starts its replica at view r so that replicas do not all render the same camera at the same time
-    view_of = lambda s: (s + rank) % n_views  # noqa: E731
+    view_of = lambda s: replica_view(s, rank, n_views)  # noqa: E731
     cams = [B.make_camera(c) for c in w.cameras[:n_views]]
     host_targets = [torch.from_numpy(w.target(i)).pin_memory() for i in range(n_views)]
     bank = torch.stack([t.to(dev) for t in host_targets])
@@ -292,11 +319,8 @@ def main():
         st = tr.poll()
         if st != B.ODIN_OK:
             raise SystemExit(f"profiled run failed: {B.status_string(st)}")
-    t_max = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_max, op=dist.ReduceOp.MAX)
-    ms = float(t_max.item())
-    value = world * args.steps / (ms * 1e-3)
+    ms = max_over_ranks(ms, world, dev)
+    value = whole_job_value(args.steps, world, ms * 1e-3)
 
     # workload counters of the last view (device side), for the byte model
     v_last = int(tr.count.item())
@@ -330,10 +354,7 @@ def main():
         torch.cuda.synchronize()
     barrier()
     e2e_s = time.perf_counter() - t0
-    e2e_t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
-    e2e_value = world * args.steps / float(e2e_t.item())
+    e2e_value = whole_job_value(args.steps, world, max_over_ranks(e2e_s, world, dev))
     st = tr.poll()
     if st != B.ODIN_OK:
         raise SystemExit(f"end-to-end run failed: {B.status_string(st)}")
@@ -380,6 +401,8 @@ def main():
             roofline = {"kernel": top, "kernels": members, "bound": "hbm", "achieved": ach, "peak": peak_gbs,
                         "unit": "GB/s", "frac": ach / peak_gbs, "traffic": None, "peak_source": peak_src,
                         "note": "algorithmic bytes of the stage per view over the summed time of its launches"}
+        roofline["traffic"] = NCU_TRAFFIC.get(w.name, {}).get(top)
+        roofline["algorithmic_bytes"] = bytes_kernels.get(top)
     step_gbs = bytes_model["total"] / (ms * 1e-3 / args.steps) / 1e9
 
     line = {

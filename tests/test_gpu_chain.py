@@ -11,14 +11,16 @@ import gpu_util as G
 pytestmark = pytest.mark.gpu
 
 
-def run_chain(oracle32, w, steps, views, window=None):
+def run_chain(oracle32, w, steps, views, window=None, row_capacity=None, instance_capacity=None):
     """Runs `steps` views on both sides from the same start.  Both sides see the same parameters at every step
     because the oracle is re-synchronised from the device after each comparison (so one fragile decision cannot
     cascade); every step is compared on its own."""
     scene = w.scene
     n = scene.n
     cam0 = w.cameras[0]
-    tr = G.trainer_for(scene, cam0, mask_slots=max(len(views), 1))
+    tr = G.trainer_for(scene, cam0, row_capacity=row_capacity, instance_capacity=instance_capacity,
+                       mask_slots=max(len(views), 1))
+    rng = np.random.default_rng(7)
     tr.keep_sorted_keys = True  # the sorted keys are compared below
     p = scene.copy()
     m, v = p.zeros_like(), p.zeros_like()
@@ -61,12 +63,17 @@ def run_chain(oracle32, w, steps, views, window=None):
         assert abs(float(tr.loss.item()) - o["loss"]) < 1e-5
         # updated state: compare the touched rows of params, m, v
         idx = o["idx"].astype(np.int64)
-        dev_state = [t.cpu().numpy() for s_ in (tr.params, tr.m, tr.v) for t in s_.tensors()]
         host_state = [a for s_ in (p, m, v) for a in (s_.means, s_.log_scales, s_.quats, s_.opacity_logit, s_.sh)]
+        dev_tensors = [t for s_ in (tr.params, tr.m, tr.v) for t in s_.tensors()]
         un = np.setdiff1d(np.arange(n), idx)
-        for d, h in zip(dev_state, host_state):
+        if len(un) > 2_000_000:  # the largest scenes: a seeded sample of the untouched rows
+            un = np.sort(rng.choice(un, 2_000_000, replace=False))
+        un_dev, idx_dev = torch.from_numpy(un).to(dev), torch.from_numpy(idx).to(dev)
+        for t, h in zip(dev_tensors, host_state):
             # untouched rows identical to the oracle's (which never changed them)
-            assert np.array_equal(d[un].view(np.uint32), h[un].view(np.uint32))
+            assert np.array_equal(t[un_dev].cpu().numpy().view(np.uint32), h[un].view(np.uint32))
+        dev_rows = [t[idx_dev].cpu().numpy() for t in dev_tensors]    # the touched rows, in row order
+        host_rows = [h[idx] for h in host_state]
         # gradient rows: every word inside the bar derived from the un-cancelled term sums (see gpu_util)
         _, g2d_abs = oracle32.render_bwd_blend(o["proj"], o["vals"], o["ranges"], cam, o["final_T"], o["n_contrib"],
                                                o["dL_dout"], want_abs=True)
@@ -83,13 +90,13 @@ def run_chain(oracle32, w, steps, views, window=None):
         assert agree.mean() > 0.9, agree.mean()
 
         def as_rows(st):
-            return np.concatenate([st[0][idx], st[1][idx], st[2][idx], st[3][idx][:, None],
-                                   st[4][idx].reshape(len(idx), -1)], axis=1).astype(np.float64)
+            return np.concatenate([st[0], st[1], st[2], st[3][:, None], st[4].reshape(len(idx), -1)],
+                                  axis=1).astype(np.float64)
 
         g_abs = np.abs(rows)
-        dp, hp = as_rows(dev_state[0:5]), as_rows(host_state[0:5])
-        dm, hm = as_rows(dev_state[5:10]), as_rows(host_state[5:10])
-        dv, hv = as_rows(dev_state[10:15]), as_rows(host_state[10:15])
+        dp, hp = as_rows(dev_rows[0:5]), as_rows(host_rows[0:5])
+        dm, hm = as_rows(dev_rows[5:10]), as_rows(host_rows[5:10])
+        dv, hv = as_rows(dev_rows[10:15]), as_rows(host_rows[10:15])
         assert np.all(np.abs(dm - hm)[agree] <= (1e-3 * (1 - w.beta1) * g_abs + 1e-6 * np.abs(hm) + 1e-30)[agree])
         assert np.all(np.abs(dv - hv)[agree] <= (2.1e-3 * (1 - w.beta2) * g_abs ** 2 + 1e-6 * np.abs(hv) + 1e-30)[agree])
         assert np.all(np.abs(dp - hp)[agree] <= 1e-3 * np.abs(hp)[agree] + 1e-5)
@@ -132,3 +139,23 @@ def test_chain_unbounded_scene_scaled(oracle32):
 def test_chain_city_scaled(oracle32):
     w = wl.make_workload(5, n=300_000, n_cameras=4, resolution=(480, 270))
     run_chain(oracle32, w, steps=2, views=[0, 1])
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# The two workloads bench.py times, at full size and with the capacities it launches with.  Two consecutive steps, so
+# the second one runs on non-zero Adam moments.  The oracle computes every output (a full view of these sizes takes
+# it seconds); untouched rows of the 20 M scene are compared on a seeded sample of 2 M rows.
+def test_chain_cfg3_full_size_as_benchmarked(oracle32):
+    import bench
+
+    w = wl.make_workload(3)
+    run_chain(oracle32, w, steps=2, views=[0, 1], row_capacity=int(bench.ROW_CAP_FRAC[3] * w.scene.n),
+              instance_capacity=bench.INSTANCE_CAP[3])
+
+
+def test_chain_cfg5_full_size_as_benchmarked(oracle32):
+    import bench
+
+    w = wl.make_workload(5)
+    row_cap = min(w.scene.n, max(int(bench.ROW_CAP_FRAC[5] * w.scene.n), 1_600_000))
+    run_chain(oracle32, w, steps=2, views=[0, 1], row_capacity=row_cap, instance_capacity=bench.INSTANCE_CAP[5])
