@@ -498,6 +498,42 @@ void render_bwd_blend(const Real* xy, const Real* conic_o, const Real* rgb, cons
 }
 
 // ---------------------------------------------------------------------------------------------
+// Realized active set C_i (Sec. 2.1, Table 1: the primitives that actually take part in the view's
+// computation, known only after it has executed; Theta >= G_i >= C_i).  Reading: a primitive is
+// realized-active when it is blended into at least one pixel, i.e. it passes the skip tests inside
+// that pixel's n_contrib prefix - exactly the (pixel, primitive) pairs the backward differentiates.
+// active [n] receives 0 / 1.
+template <class Real>
+void realized_active(const Real* xy, const Real* conic_o, const uint32_t* vals, const uint32_t* ranges,
+                     const CameraD& camd, const Config& cfg, const uint32_t* n_contrib, int64_t n, uint8_t* active) {
+  const Cam<Real> cam = make_cam<Real>(camd, cfg.tile);
+  const int W = cam.W, H = cam.H;
+  const Real amin = (Real)cfg.alpha_min, amax = (Real)cfg.alpha_max;
+  for (int64_t i = 0; i < n; ++i) active[i] = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int t = 0; t < cam.TX * cam.TY; ++t) {
+    const int tx = t % cam.TX, ty = t / cam.TX;
+    const uint32_t start = ranges[2 * t];
+    for (int j = ty * cfg.tile; j < std::min(H, (ty + 1) * cfg.tile); ++j)
+      for (int i = tx * cfg.tile; i < std::min(W, (tx + 1) * cfg.tile); ++i) {
+        const size_t pix = (size_t)j * W + i;
+        const Real px = (Real)i + (Real)0.5, py = (Real)j + (Real)0.5;
+        for (uint32_t k = start; k < start + n_contrib[pix]; ++k) {
+          const uint32_t p = vals[k];
+          const Real dx = xy[2 * p] - px, dy = xy[2 * p + 1] - py;
+          const Real A = conic_o[4 * p], B = conic_o[4 * p + 1], Cc = conic_o[4 * p + 2], o = conic_o[4 * p + 3];
+          const Real power = -(Real)0.5 * (A * dx * dx + Cc * dy * dy) - B * dx * dy;
+          if (power > 0) continue;
+          const Real alpha = std::min(amax, o * std::exp(power));
+          if (alpha < amin) continue;
+#pragma omp atomic write
+          active[p] = 1;
+        }
+      }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Backward of the projection, per touched primitive (row r <-> primitive idx[r]).  Branch decisions
 // (Jacobian clamp, colour clamp) are frozen at their forward values.  Output rows [V, F] with
 // F = 11 + 3K ordered mean(3), log_scale(3), quat(4), opacity logit(1), sh[K][3].

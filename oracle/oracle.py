@@ -29,6 +29,14 @@ def _p(a: Optional[np.ndarray]):
     return None if a is None else a.ctypes.data_as(C.c_void_p)
 
 
+def ids_to_mask(idx, n: int) -> np.ndarray:
+    """Bitmask over primitive ids: bit (p & 31) of word (p >> 5)."""
+    mask = np.zeros((n + 31) // 32, np.uint32)
+    i = np.asarray(idx, np.int64)
+    np.bitwise_or.at(mask, i >> 5, np.left_shift(np.uint32(1), (i & 31).astype(np.uint32)))
+    return mask
+
+
 def _cam(cam) -> np.ndarray:
     a = cam.as_f64() if hasattr(cam, "as_f64") else np.asarray(cam, dtype=np.float64)
     assert a.shape == (23,)
@@ -194,6 +202,65 @@ class Oracle:
         a = np.ascontiguousarray(idx_a, np.uint32)
         b = np.ascontiguousarray(idx_b, np.uint32)
         return int(self.lib.oracle_conflict_count(_p(a), C.c_uint32(a.shape[0]), _p(b), C.c_uint32(b.shape[0])))
+
+    # ------------------------------------------------------------------ realized scopes, evidence, hazards
+    def realized_active(self, proj: Projected, vals, ranges, cam, n_contrib):
+        """Realized active set C_i (Sec. 2.1): primitives blended into at least one pixel.  Returns (mask words,
+        ascending primitive ids)."""
+        n = proj.depth.shape[0]
+        active = np.zeros(n, np.uint8)
+        self._f("oracle_realized_active")(
+            _p(self._a(proj.xy)), _p(self._a(proj.conic_o)), _p(np.ascontiguousarray(vals, np.uint32)),
+            _p(np.ascontiguousarray(ranges, np.uint32)), _p(_cam(cam)), _p(self.cfg),
+            _p(np.ascontiguousarray(n_contrib, np.uint32)), C.c_int64(n), _p(active))
+        idx = np.flatnonzero(active).astype(np.uint32)
+        return ids_to_mask(idx, n), idx
+
+    @staticmethod
+    def gradient_evidence(g2d_dense, active_idx, rows=None, touched_idx=None):
+        """Gradient evidence g(p) of the active primitives (Sec. 2.1 g_U(p); Sec. 4.3 gradient gate) and its mean over
+        the active set.  Default reading: Euclidean norm of the gradient with respect to the projected centre (u, v),
+        the first two of the nine compositing words.  With `rows` ([V, F] final gradient rows of the touched primitives
+        `touched_idx`): Euclidean norm of the whole parameter-gradient row instead."""
+        a = np.asarray(active_idx, np.int64)
+        if rows is None:
+            g = np.asarray(g2d_dense, np.float64)[a, :2]
+        else:
+            pos = np.searchsorted(np.asarray(touched_idx, np.int64), a)
+            g = np.asarray(rows, np.float64)[pos]
+        ev = np.sqrt((g * g).sum(axis=1))
+        return ev, (float(ev.sum() / len(a)) if len(a) else 0.0)
+
+    @staticmethod
+    def hazard_sets(r_a, w_a, r_b, w_b):
+        """The three primitive-state hazards of Sec. 4.3 for producer A and consumer B, as ascending id arrays."""
+        r_a, w_a, r_b, w_b = (np.unique(np.asarray(x, np.int64)) for x in (r_a, w_a, r_b, w_b))
+        waw = np.intersect1d(w_b, w_a)
+        raw = np.intersect1d(np.setdiff1d(r_b, w_b), w_a)
+        war = np.intersect1d(w_b, np.setdiff1d(r_a, w_a))
+        return waw, raw, war
+
+    @classmethod
+    def delayed_read_gate(cls, r_a, w_a, r_b, w_b, active_a, evidence_a, tau):
+        """Throughput-first admission of Sec. 4.3: D+ = C_RAW+(A, B); rho = |D+| / |R+(B)|; every delayed primitive
+        needs producer evidence (membership in C_A) no larger than tau times the mean evidence over C_A."""
+        _, delayed, _ = cls.hazard_sets(r_a, w_a, r_b, w_b)
+        n_rb = len(np.unique(np.asarray(r_b, np.int64)))
+        active_a = np.asarray(active_a, np.int64)
+        evidence_a = np.asarray(evidence_a, np.float64)
+        mean = float(evidence_a.sum() / len(active_a)) if len(active_a) else 0.0
+        pos = np.searchsorted(active_a, delayed)
+        pos_ok = pos < len(active_a)
+        has = np.zeros(len(delayed), bool)
+        has[pos_ok] = active_a[pos[pos_ok]] == delayed[pos_ok]
+        passes = np.zeros(len(delayed), bool)
+        passes[has] = evidence_a[pos[has]] <= tau * mean
+        out = dict(n_delayed=len(delayed), n_read_b=n_rb, n_with_evidence=int(has.sum()), n_pass=int(passes.sum()),
+                   mean=mean)
+        out["rho"] = len(delayed) / n_rb if n_rb else None
+        out["admitted"] = bool(n_rb > 0 and len(delayed) / n_rb <= tau and len(active_a) > 0 and has.all()
+                               and passes.all())
+        return out
 
     def sh_basis(self, degree: int, x: float, y: float, z: float) -> np.ndarray:
         out = np.zeros(16, self.dtype)

@@ -51,6 +51,11 @@ Config cfg_from(const double* c) {
     render_bwd_blend<Real>(xy, conic_o, rgb, vals, ranges, cam_from(cam), cfg_from(cfg), final_T, n_contrib, dL_dout,  \
                            n, g2d, g2d_abs);                                                                           \
   }                                                                                                                    \
+  extern "C" void oracle_realized_active_##SUF(const Real* xy, const Real* conic_o, const uint32_t* vals,              \
+                                               const uint32_t* ranges, const double* cam, const double* cfg,           \
+                                               const uint32_t* n_contrib, int64_t n, uint8_t* active) {                \
+    realized_active<Real>(xy, conic_o, vals, ranges, cam_from(cam), cfg_from(cfg), n_contrib, n, active);              \
+  }                                                                                                                    \
   extern "C" void oracle_render_bwd_project_##SUF(int sh_degree, const Real* means, const Real* log_scales,           \
                                                   const Real* quats, const Real* opacity_logit, const Real* sh,        \
                                                   const double* cam, const double* cfg, const uint32_t* idx,           \

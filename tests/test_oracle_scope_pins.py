@@ -1,0 +1,168 @@
+"""Pins of the oracle's realized active set, gradient evidence, hazard sets and delayed-read gate (Sec. 2.1, Sec. 4.3)
+against brute force, closed forms, invariants and a hand-worked example (no GPU)."""
+import os
+
+import numpy as np
+
+from paper_2607_19893_b200 import workloads as wl
+from test_oracle_project_pins import cam_identity, one_splat
+from test_oracle_render_pins import stack_scenes
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+
+
+def read_golden(name):
+    sets = {}
+    with open(os.path.join(GOLDEN, name)) as fh:
+        for line in fh:
+            if line.startswith("#") or "=" not in line:
+                continue
+            k, v = line.split("=")
+            sets[k.strip()] = v.split()
+    return sets
+
+
+# ------------------------------------------------------------------------------- realized active set
+def brute_force_active(f, cam):
+    """Independent restatement: walk every pixel's list front to back with the compositing rule and record who blends."""
+    p = f["proj"]
+    tx = (cam.width + 15) // 16
+    alpha_min, alpha_max, t_min = 1.0 / 255.0, 0.99, 1e-4   # the method's constants
+    active, fragile = set(), False
+    for j in range(cam.height):
+        for i in range(cam.width):
+            s, e = f["ranges"][(j // 16) * tx + i // 16]
+            T = 1.0
+            for k in range(s, e):
+                q = int(f["vals"][k])
+                d = p.xy[q] - (i + 0.5, j + 0.5)
+                A, B, Cc, o = p.conic_o[q]
+                power = -0.5 * (A * d[0] * d[0] + Cc * d[1] * d[1]) - B * d[0] * d[1]
+                if power > 0:
+                    continue
+                alpha = min(alpha_max, o * np.exp(power))
+                if alpha < alpha_min:
+                    continue
+                if T * (1 - alpha) < t_min:
+                    break
+                active.add(q)
+                T *= 1 - alpha
+    return active
+
+
+def test_realized_active_matches_bruteforce_and_is_nested(oracle64):
+    w = wl.make_workload(1)
+    cam = w.cameras[0]
+    f = oracle64.view_forward(w.scene, cam)
+    mask, idx = oracle64.realized_active(f["proj"], f["vals"], f["ranges"], cam, f["n_contrib"])
+    want = brute_force_active(f, cam)
+    assert set(idx.tolist()) == want
+    # Theta >= G_i >= C_i (Sec. 2.1), ascending list, mask = the same set
+    assert set(idx.tolist()) <= set(f["idx"].tolist()) <= set(range(w.scene.n))
+    assert np.all(np.diff(idx.astype(np.int64)) > 0)
+    bits = np.unpackbits(mask.view(np.uint8), bitorder="little")[: w.scene.n]
+    assert np.array_equal(np.flatnonzero(bits), idx)
+    # a primitive is active exactly when the colour gradient has a non-zero un-cancelled term sum for unit dL
+    ones = np.ones_like(f["out"])
+    _, g_abs = oracle64.render_bwd_blend(f["proj"], f["vals"], f["ranges"], cam, f["final_T"], f["n_contrib"], ones,
+                                         want_abs=True)
+    assert np.array_equal(np.flatnonzero(g_abs[:, 6] > 0), idx)
+
+
+def test_occluded_primitive_is_touched_but_not_active(oracle64):
+    """Four wide, almost opaque splats in front of a tiny one on the same axis: after two of them the transmittance is
+    1e-4 and the third would push it below the stop threshold, so every pixel the tiny splat could reach stops before
+    it.  The tiny splat is in the candidate scope (it covers a tile) but not in the realized one.  Without the
+    occluders it is active."""
+    cam = cam_identity(64, 64, 64.0)
+    fronts = [one_splat((0.0, 0.0, 2.0 + 0.1 * k), (0.0, 0.0, 0.0), (1, 0, 0, 0), logit=12.0) for k in range(4)]
+    behind = one_splat((0.0, 0.0, 4.0), (-4.5, -4.5, -4.5), (1, 0, 0, 0), logit=2.0)
+    scene = stack_scenes(fronts + [behind])
+    f = oracle64.view_forward(scene, cam)
+    assert 4 in f["idx"]                                        # touched: geometry locality sees it
+    _, idx = oracle64.realized_active(f["proj"], f["vals"], f["ranges"], cam, f["n_contrib"])
+    assert 4 not in idx and {0, 1} <= set(idx.tolist())
+    assert f["n_contrib"][32, 32] == 2                          # the centre pixel stops at the third occluder
+    f2 = oracle64.view_forward(behind, cam)
+    _, idx2 = oracle64.realized_active(f2["proj"], f2["vals"], f2["ranges"], cam, f2["n_contrib"])
+    assert idx2.tolist() == [0]
+
+
+# ------------------------------------------------------------------------------- gradient evidence
+def test_gradient_evidence_norms_mean_and_linearity(oracle64):
+    g2d = np.zeros((6, 9))
+    g2d[1, :2] = (3.0, 4.0)
+    g2d[2, :2] = (-6.0, 8.0)
+    g2d[4, :2] = (0.0, 0.0)
+    g2d[:, 2:] = 7.0                                            # the other words do not enter the default evidence
+    ev, mean = oracle64.gradient_evidence(g2d, [1, 2, 4])
+    assert np.allclose(ev, (5.0, 10.0, 0.0)) and mean == 5.0
+    ev2, mean2 = oracle64.gradient_evidence(-2.5 * g2d, [1, 2, 4])
+    assert np.allclose(ev2, 2.5 * ev) and np.isclose(mean2, 2.5 * mean)
+    ev0, mean0 = oracle64.gradient_evidence(g2d, [])
+    assert len(ev0) == 0 and mean0 == 0.0
+    # whole-row variant: rows of the touched primitives [2, 4, 5]; active [2, 5]
+    rows = np.array([[1.0, 2.0, 2.0], [9.0, 9.0, 9.0], [0.0, 3.0, 4.0]])
+    evr, meanr = oracle64.gradient_evidence(None, [2, 5], rows=rows, touched_idx=[2, 4, 5])
+    assert np.allclose(evr, (3.0, 5.0)) and meanr == 4.0
+
+
+def test_gradient_evidence_scales_with_the_loss_on_a_rendered_view(oracle64):
+    w = wl.make_workload(1)
+    cam = w.cameras[0]
+    f = oracle64.view_forward(w.scene, cam)
+    _, dl = oracle64.l1_loss(f["out"], w.target(0).astype(np.float64))
+    g = oracle64.render_bwd_blend(f["proj"], f["vals"], f["ranges"], cam, f["final_T"], f["n_contrib"], dl)
+    g3 = oracle64.render_bwd_blend(f["proj"], f["vals"], f["ranges"], cam, f["final_T"], f["n_contrib"], 3.0 * dl)
+    _, idx = oracle64.realized_active(f["proj"], f["vals"], f["ranges"], cam, f["n_contrib"])
+    ev, mean = oracle64.gradient_evidence(g, idx)
+    ev3, mean3 = oracle64.gradient_evidence(g3, idx)
+    assert np.allclose(ev3, 3 * ev, rtol=1e-12) and np.isclose(mean3, 3 * mean)
+    # primitives outside the active set received no gradient at all
+    inactive = np.setdiff1d(np.arange(w.scene.n), idx)
+    assert not g[inactive].any()
+
+
+# ------------------------------------------------------------------------------- hazards
+def test_hazard_sets_hand_example_and_algebra(oracle64):
+    s = {k: np.array([int(x) for x in v]) for k, v in read_golden("hazard_sets_example.txt").items()}
+    waw, raw, war = oracle64.hazard_sets(s["R_A"], s["W_A"], s["R_B"], s["W_B"])
+    assert waw.tolist() == [4, 6] and raw.tolist() == [8] and war.tolist() == [5]
+    assert (len(waw), len(raw), len(war)) == (int(s["n_WAW"][0]), int(s["n_RAW"][0]), int(s["n_WAR"][0]))
+    rng = np.random.default_rng(11)
+    for _ in range(20):
+        n = 400
+        w_a = rng.choice(n, rng.integers(0, 200), replace=False)
+        r_a = np.union1d(w_a, rng.choice(n, rng.integers(0, 100), replace=False))      # W+ is inside R+
+        w_b = rng.choice(n, rng.integers(0, 200), replace=False)
+        r_b = np.union1d(w_b, rng.choice(n, rng.integers(0, 100), replace=False))
+        waw, raw, war = oracle64.hazard_sets(r_a, w_a, r_b, w_b)
+        A_r, A_w, B_r, B_w = set(r_a.tolist()), set(w_a.tolist()), set(r_b.tolist()), set(w_b.tolist())
+        assert set(waw.tolist()) == B_w & A_w
+        assert set(raw.tolist()) == (B_r - B_w) & A_w
+        assert set(war.tolist()) == B_w & (A_r - A_w)
+        # RAW and WAW partition R+(B) & W+(A); the three sets are pairwise disjoint
+        assert len(raw) + len(waw) == len(B_r & A_w)
+        assert not (set(raw.tolist()) & set(waw.tolist())) and not (set(war.tolist()) & set(waw.tolist()))
+        assert len(waw) == oracle64.conflict_count(np.sort(w_a).astype(np.uint32), np.sort(w_b).astype(np.uint32))
+        # this build's pipeline declares R+ = W+: then only WAW can be non-empty
+        _, raw0, war0 = oracle64.hazard_sets(w_a, w_a, w_b, w_b)
+        assert len(raw0) == 0 and len(war0) == 0
+
+
+def test_delayed_read_gate_hand_example(oracle64):
+    g = read_golden("delayed_read_gate_example.txt")
+    ints = lambda k: np.array([int(x) for x in g[k]])  # noqa: E731
+    ev = np.array([float(x) for x in g["evidence_A"]])
+    for case in ("1", "2", "3", "4"):
+        out = oracle64.delayed_read_gate(ints("R_A"), ints("W_A"), ints("R_B" + case), ints("W_B" + case), ints("C_A"), ev,
+                                         float(g["tau" + case][0]))
+        assert out["n_delayed"] == int(g["n_delayed" + case][0])
+        assert out["n_with_evidence"] == int(g["n_with_evidence" + case][0])
+        assert out["n_pass"] == int(g["n_pass" + case][0])
+        assert np.isclose(out["rho"], float(g["rho" + case][0]))
+        assert out["admitted"] == (g["admitted" + case][0] == "yes")
+    assert np.isclose(out["mean"], float(g["mean_A"][0]))
+    # an empty consumer read scope has no delayed-read admission to perform
+    out = oracle64.delayed_read_gate(ints("R_A"), ints("W_A"), [], [], ints("C_A"), ev, 1.0)
+    assert out["rho"] is None and not out["admitted"] and out["n_delayed"] == 0
