@@ -195,11 +195,13 @@ int odin_l1_loss(odin_ctx* ctx, const float* d_rgb, const float* d_target, int w
  * inverse, the EWA projection, the Jacobian (clamp frozen), Sigma = M M^T, scale = exp(log scale), the rotation and
  * the quaternion normalisation, the pixel centre, the SH colour (clamped channels pass nothing; the direction term
  * reaches the mean) and the sigmoid.  grad_rows: compact rows (row r <-> proj->prim_id[r]) in the layout of
- * odin_scene with n >= V. */
+ * odin_scene with n >= V.
+ * d_row_active [capacity] (bytes, may be NULL): 1 for every row that was blended into at least one pixel - the
+ * realized active set C_i of Sec. 2.1, observed where the paper observes it, after the backward pass - else 0. */
 int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odin_camera* cam, const odin_projected* proj,
                     const uint32_t* d_vals, const uint32_t* d_tile_ranges, const float* d_final_T,
                     const uint32_t* d_n_contrib, const float* d_dL_drgb, float* d_grad2d, odin_scene* grad_rows,
-                    void* ws, size_t ws_bytes, void* stream);
+                    uint8_t* d_row_active, void* ws, size_t ws_bytes, void* stream);
 
 /* Optimizer update (phase U) restricted to the touched rows: for every r < *d_count and every scalar theta of
  * primitive d_idx[r] with gradient g: m = b1 m + (1-b1) g; v = b2 v + (1-b2) g^2;
@@ -215,6 +217,46 @@ int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m, odin_scen
  * d_masks [n_masks][mask_stride_words]; d_pairs [n_pairs][2] view slots; d_counts [n_pairs] (overwritten). */
 int odin_conflict_count(odin_ctx* ctx, const uint32_t* d_masks, uint32_t n_masks, uint32_t mask_stride_words,
                         uint32_t n_prims, const uint32_t* d_pairs, uint32_t n_pairs, uint64_t* d_counts, void* stream);
+
+/* ---- realized scope, gradient evidence and admission arithmetic (Sec. 2.1 Table 1, Sec. 4.3) -------------------- */
+
+/* Realized active set C_i and gradient evidence g(p) of a view (Sec. 2.1: Theta >= G_i >= C_i; g_U(p) = per-primitive
+ * gradient magnitude of the active primitives).  From the row flags of odin_render_bwd:
+ * d_mask [ceil(n/32)] bit per primitive id (overwritten); d_idx: ascending primitive ids of the active rows (first
+ * idx_capacity; more defers ODIN_ERR_CAPACITY); d_count [1]; d_evidence [idx_capacity] parallel to d_idx;
+ * d_evidence_sum [1] (double) = sum of the evidence over C_i (mean = sum / count).
+ * evidence_mode 0: Euclidean norm of the gradient with respect to the projected centre, sqrt(g_u^2 + g_v^2) of
+ * d_grad2d (the quantity point-based pipelines accumulate per primitive); 1: Euclidean norm of the whole gradient row
+ * (grad_rows, required in this mode).  The paper says "after the pipeline's normal gradient scaling" without fixing
+ * the norm; both readings are offered.  n = number of primitives of the pool. */
+int odin_active_set(odin_ctx* ctx, const odin_projected* proj, const uint8_t* d_row_active, const float* d_grad2d,
+                    const odin_scene* grad_rows, int evidence_mode, uint32_t n, uint32_t* d_mask, uint32_t* d_idx,
+                    uint32_t idx_capacity, uint32_t* d_count, float* d_evidence, double* d_evidence_sum, void* ws,
+                    size_t ws_bytes, void* stream);
+
+/* Unit unions (Sec. 2.1: R^+(U), W^+(U), C_U are unions over the views of a task unit): d_out [stride_words] = OR of
+ * the masks d_masks[d_members[k]], k < n_members (zero words for n_members = 0). */
+int odin_mask_union(odin_ctx* ctx, const uint32_t* d_masks, uint32_t n_masks, uint32_t mask_stride_words,
+                    uint32_t n_prims, const uint32_t* d_members, uint32_t n_members, uint32_t* d_out, void* stream);
+
+/* The three primitive-state hazards of the quality-first path (Sec. 4.3) for pairs (A, B) = (producer, consumer):
+ *   WAW = W(B) & W(A);  RAW = (R(B) \ W(B)) & W(A);  WAR = W(B) & (R(A) \ W(A)).
+ * d_read_masks, d_write_masks [n_masks][mask_stride_words]: the conservative scopes R^+, W^+ of each unit;
+ * d_pairs [n_pairs][2] = (A, B); d_counts [n_pairs][4] (overwritten) = (#WAW, #RAW, #WAR, #R^+(B)). */
+int odin_hazard_count(odin_ctx* ctx, const uint32_t* d_read_masks, const uint32_t* d_write_masks, uint32_t n_masks,
+                      uint32_t mask_stride_words, uint32_t n_prims, const uint32_t* d_pairs, uint32_t n_pairs,
+                      uint64_t* d_counts, void* stream);
+
+/* Evidence for the throughput-first admission (Sec. 4.3).  Delayed-read set D^+ = C_RAW^+(A, B) =
+ * (R(B) \ W(B)) & W(A).  A delayed primitive has producer evidence when it is in C_A; it passes the gradient gate
+ * when g_A(p) <= tau * mean of g_A over C_A.  Inputs: the three masks [ceil(n_prims/32)], A's active list, evidence,
+ * count and evidence sum as written by odin_active_set.  d_gate [4] (overwritten) = (#D^+, #(D^+ & C_A), #passing the
+ * gate, #R^+(B)).  The caller admits the delayed read iff #R^+(B) > 0, #D^+ / #R^+(B) <= tau, C_A is not empty and
+ * all three first counts are equal. */
+int odin_delayed_read_gate(odin_ctx* ctx, const uint32_t* d_read_b, const uint32_t* d_write_b, const uint32_t* d_write_a,
+                           uint32_t n_prims, const uint32_t* d_active_idx_a, const float* d_evidence_a,
+                           const uint32_t* d_active_count_a, const double* d_evidence_sum_a, uint32_t active_capacity_a,
+                           float tau, uint64_t* d_gate, void* stream);
 
 #ifdef __cplusplus
 }

@@ -27,7 +27,8 @@ EXPORTS = [
     "odin_create", "odin_destroy", "odin_status_string", "odin_poll", "odin_workspace_bytes", "odin_project",
     "odin_touched_set", "odin_bin_sort", "odin_render_fwd", "odin_l1_loss", "odin_render_bwd", "odin_sparse_adam",
     "odin_conflict_count", "odin_kernel_count", "odin_kernel_name", "odin_profile_enable", "odin_profile_collect",
-    "odin_touched_set_static", "odin_render_workspace_bytes",
+    "odin_touched_set_static", "odin_render_workspace_bytes", "odin_active_set", "odin_mask_union", "odin_hazard_count",
+    "odin_delayed_read_gate",
 ]
 
 
@@ -89,11 +90,16 @@ def lib() -> C.CDLL:
                                       C.c_size_t, vp]
         L.odin_l1_loss.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
         L.odin_render_bwd.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_camera), C.POINTER(odin_projected), vp, vp,
-                                      vp, vp, vp, vp, C.POINTER(odin_scene), vp, C.c_size_t, vp]
+                                      vp, vp, vp, vp, C.POINTER(odin_scene), vp, vp, C.c_size_t, vp]
         L.odin_sparse_adam.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_scene), C.POINTER(odin_scene),
                                        C.POINTER(odin_scene), vp, vp, C.POINTER(f32), f32, f32, f32, u32, vp]
         L.odin_conflict_count.argtypes = [vp, vp, u32, u32, u32, vp, u32, vp, vp]
         L.odin_touched_set_static.argtypes = [vp, u32, vp, vp, u32, vp, vp, vp]
+        L.odin_active_set.argtypes = [vp, C.POINTER(odin_projected), vp, vp, C.POINTER(odin_scene), i32, u32, vp, vp, u32,
+                                      vp, vp, vp, vp, C.c_size_t, vp]
+        L.odin_mask_union.argtypes = [vp, vp, u32, u32, u32, vp, u32, vp, vp]
+        L.odin_hazard_count.argtypes = [vp, vp, vp, u32, u32, u32, vp, u32, vp, vp]
+        L.odin_delayed_read_gate.argtypes = [vp, vp, vp, vp, u32, vp, vp, vp, vp, u32, f32, vp, vp]
         L.odin_kernel_count.argtypes = []
         L.odin_kernel_name.argtypes = [i32]
         L.odin_profile_enable.argtypes = [vp, i32]
@@ -219,10 +225,11 @@ def odin_l1_loss(ctx, d_rgb, d_target, width: int, height: int, d_loss, d_dL_drg
 
 
 def odin_render_bwd(ctx, scene: odin_scene, cam: odin_camera, proj: odin_projected, d_vals, d_tile_ranges, d_final_T,
-                    d_n_contrib, d_dL_drgb, d_grad2d, grad_rows: odin_scene, ws, stream=None) -> None:
+                    d_n_contrib, d_dL_drgb, d_grad2d, grad_rows: odin_scene, d_row_active, ws, stream=None) -> None:
     _check(lib().odin_render_bwd(ctx, C.byref(scene), C.byref(cam), C.byref(proj), _ptr(d_vals), _ptr(d_tile_ranges),
                                  _ptr(d_final_T), _ptr(d_n_contrib), _ptr(d_dL_drgb), _ptr(d_grad2d), C.byref(grad_rows),
-                                 _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+                                 _ptr(d_row_active), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                 _stream(stream)),
            "odin_render_bwd")
 
 
@@ -238,6 +245,45 @@ def odin_conflict_count(ctx, d_masks, n_masks: int, mask_stride_words: int, n_pr
                         stream=None) -> None:
     _check(lib().odin_conflict_count(ctx, _ptr(d_masks), int(n_masks), int(mask_stride_words), int(n_prims), _ptr(d_pairs),
                                      int(n_pairs), _ptr(d_counts), _stream(stream)), "odin_conflict_count")
+
+
+def odin_active_set(ctx, proj: odin_projected, d_row_active, d_grad2d, grad_rows: Optional[odin_scene],
+                    evidence_mode: int, n: int, d_mask, d_idx, idx_capacity: int, d_count, d_evidence, d_evidence_sum, ws,
+                    stream=None) -> None:
+    _check(lib().odin_active_set(ctx, C.byref(proj), _ptr(d_row_active), _ptr(d_grad2d),
+                                 None if grad_rows is None else C.byref(grad_rows), int(evidence_mode), int(n),
+                                 _ptr(d_mask), _ptr(d_idx), int(idx_capacity), _ptr(d_count), _ptr(d_evidence),
+                                 _ptr(d_evidence_sum), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                 _stream(stream)), "odin_active_set")
+
+
+def odin_mask_union(ctx, d_masks, n_masks: int, mask_stride_words: int, n_prims: int, d_members, n_members: int, d_out,
+                    stream=None) -> None:
+    _check(lib().odin_mask_union(ctx, _ptr(d_masks), int(n_masks), int(mask_stride_words), int(n_prims), _ptr(d_members),
+                                 int(n_members), _ptr(d_out), _stream(stream)), "odin_mask_union")
+
+
+def odin_hazard_count(ctx, d_read_masks, d_write_masks, n_masks: int, mask_stride_words: int, n_prims: int, d_pairs,
+                      n_pairs: int, d_counts, stream=None) -> None:
+    _check(lib().odin_hazard_count(ctx, _ptr(d_read_masks), _ptr(d_write_masks), int(n_masks), int(mask_stride_words),
+                                   int(n_prims), _ptr(d_pairs), int(n_pairs), _ptr(d_counts), _stream(stream)),
+           "odin_hazard_count")
+
+
+def odin_delayed_read_gate(ctx, d_read_b, d_write_b, d_write_a, n_prims: int, d_active_idx_a, d_evidence_a,
+                           d_active_count_a, d_evidence_sum_a, active_capacity_a: int, tau: float, d_gate,
+                           stream=None) -> None:
+    _check(lib().odin_delayed_read_gate(ctx, _ptr(d_read_b), _ptr(d_write_b), _ptr(d_write_a), int(n_prims),
+                                        _ptr(d_active_idx_a), _ptr(d_evidence_a), _ptr(d_active_count_a),
+                                        _ptr(d_evidence_sum_a), int(active_capacity_a), float(tau), _ptr(d_gate),
+                                        _stream(stream)), "odin_delayed_read_gate")
+
+
+def admit_delayed_read(gate, active_count_a: int, tau: float) -> bool:
+    """The admission rule of Sec. 4.3 from the four counts of odin_delayed_read_gate (#D+, #(D+ & C_A), #pass, #R+(B))."""
+    n_delayed, n_with, n_pass, n_read_b = (int(x) for x in gate)
+    return bool(n_read_b > 0 and n_delayed <= tau * n_read_b and active_count_a > 0 and n_with == n_delayed
+                and n_pass == n_delayed)
 
 
 def odin_kernel_count() -> int:

@@ -14,7 +14,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libodin.so")
 OBJ_DIR = os.path.join(HERE, "build")
 
-SOURCES = ["api.cu", "project.cu", "touched.cu", "binsort.cu", "render_fwd.cu", "render_bwd.cu", "adam.cu"]
+SOURCES = ["api.cu", "project.cu", "touched.cu", "binsort.cu", "render_fwd.cu", "render_bwd.cu", "adam.cu", "scope.cu"]
 # Integer decisions (radius, tile rectangle) are taken from float results in project.cu: keep plain IEEE
 # multiply/add there so that they do not depend on fused multiply-add contraction.
 EXTRA = {"project.cu": ["-fmad=false"]}

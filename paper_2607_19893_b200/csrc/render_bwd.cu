@@ -6,10 +6,14 @@
 
 namespace {
 
-__global__ void zero_rows_kernel(float* __restrict__ g2d, const uint32_t* __restrict__ num_rows, uint32_t capacity) {
+__global__ void zero_rows_kernel(float* __restrict__ g2d, uint8_t* __restrict__ row_active,
+                                 const uint32_t* __restrict__ num_rows, uint32_t capacity) {
   const uint32_t V = min(*num_rows, capacity);
   const size_t count = (size_t)V * 9;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x) g2d[i] = 0.f;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x) {
+    g2d[i] = 0.f;
+    if (row_active && i < V) row_active[i] = 0;
+  }
 }
 
 // Sums eight values across the warp with 9 shuffles: at each of the first three steps a lane hands half of its
@@ -39,7 +43,8 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
                        const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
                        float bg0, float bg1, float bg2, float alpha_min, float alpha_max,
                        const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
-                       const float* __restrict__ dL, float* __restrict__ g2d, float* __restrict__ state) {
+                       const float* __restrict__ dL, float* __restrict__ g2d, float* __restrict__ state,
+                       uint8_t* __restrict__ row_active) {
   constexpr int BB = BLEND_TAIL_THREADS;
   __shared__ BlendRow s_rowdata[BB];
   __shared__ float2 s_blue[BB];  // blue, power threshold
@@ -113,6 +118,7 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
       const int j = j4 - u;
       const bool on = on4[u];
       if (__ballot_sync(0xffffffffu, on) == 0) continue;
+      if (row_active && lane == 0) row_active[s_rowid[j]] = 1;  // realized-active: blended into at least one pixel
       const float4 q0 = s_rowdata[j].q0, q1 = s_rowdata[j].q1;
       const float2 bp = s_blue[j];
       const float dx = q0.x - fx;
@@ -173,7 +179,8 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
                         int n_tiles, float bg0, float bg1, float bg2, float alpha_min, float alpha_max,
                         const float* __restrict__ state,
                         const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
-                        const float* __restrict__ dL, float* __restrict__ g2d, uint32_t* __restrict__ ticket) {
+                        const float* __restrict__ dL, float* __restrict__ g2d, uint32_t* __restrict__ ticket,
+                        uint8_t* __restrict__ row_active) {
   __shared__ BlendRow s_rowdata[BLEND_WARPS][32];
   __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, power threshold
   __shared__ uint32_t s_rowid[BLEND_WARPS][32];
@@ -263,6 +270,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       }
       const uint32_t hit = __reduce_or_sync(0xffffffffu, pass);  // bit s: some lane of the warp passes in slot s
       if (hit == 0) continue;
+      if (row_active && lane == 0) row_active[s_rowid[warp][j]] = 1;  // realized-active (see the tail kernel)
       // phase 2: per-lane sums over its eight pixels; the x-dependent factors are applied once at the end
       float ar = 0.f, ag = 0.f, ab = 0.f, ao = 0.f, gpsum = 0.f, m1y = 0.f, m2yy = 0.f;
 #pragma unroll
@@ -452,7 +460,7 @@ render_bwd_project_kernel(const float* __restrict__ means, const float* __restri
 extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odin_camera* cam, const odin_projected* proj,
                                const uint32_t* d_vals, const uint32_t* d_tile_ranges, const float* d_final_T,
                                const uint32_t* d_n_contrib, const float* d_dL_drgb, float* d_grad2d, odin_scene* grad_rows,
-                               void* ws, size_t ws_bytes, void* stream) {
+                               uint8_t* d_row_active, void* ws, size_t ws_bytes, void* stream) {
   if (!ctx || !proj || !grad_rows) return ODIN_ERR_NULL;
   int rc = odin_check_scene(scene);
   if (rc != ODIN_OK) return rc;
@@ -472,7 +480,7 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
   const uint32_t zgrid = (uint32_t)ctx->sm_count * 8;
   {
     OdinKernelScope ks(ctx, K_ZERO_ROWS, st);
-    zero_rows_kernel<<<zgrid, 256, 0, st>>>(d_grad2d, proj->num_rows, proj->capacity);
+    zero_rows_kernel<<<zgrid, 256, 0, st>>>(d_grad2d, d_row_active, proj->num_rows, proj->capacity);
   }
   const int n_tiles = TX * TY;
   float* state = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + blend_ws_flags_bytes(n_tiles));
@@ -483,7 +491,7 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
     render_bwd_tail_kernel<<<n_tiles, BLEND_TAIL_THREADS, 0, st>>>(
         reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
         reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
-        ctx->cfg.alpha_min, ctx->cfg.alpha_max, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d, state);
+        ctx->cfg.alpha_min, ctx->cfg.alpha_max, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d, state, d_row_active);
   }
   {
     OdinKernelScope ks(ctx, K_BWD_BLEND, st);
@@ -493,7 +501,7 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
         reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
         reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0], cam->bg[1],
         cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, state, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d,
-        ticket);
+        ticket, d_row_active);
   }
   const CamParams cp = odin_cam_params(cam, ctx->cfg);
   const uint32_t blocks_cap = (proj->capacity + 127) / 128;

@@ -119,6 +119,13 @@ class ViewTrainer:
         self.masks = z((self.mask_slots, max(self.mask_stride, 4)), torch.int32)
         self.idx = z(max(self.row_capacity, 1), torch.int32)
         self.count = z(1, torch.int32)
+        # realized active set of the last view (Sec. 2.1 C_i) and its gradient evidence
+        self.row_active = z(max(self.row_capacity, 1), torch.uint8)
+        self.active_masks = z((self.mask_slots, max(self.mask_stride, 4)), torch.int32)
+        self.active_idx = z(max(self.row_capacity, 1), torch.int32)
+        self.active_count = z(1, torch.int32)
+        self.evidence = z(max(self.row_capacity, 1), torch.float32)
+        self.evidence_sum = z(1, torch.float64)
         ws_bytes = max(B.odin_workspace_bytes(self.ctx, self.n, self.instance_capacity),
                        B.odin_render_workspace_bytes(self.ctx, self.width, self.height))
         self.ws = z(ws_bytes, torch.uint8)
@@ -152,7 +159,13 @@ class ViewTrainer:
 
     def render_bwd(self, cam: B.odin_camera, stream=None) -> None:
         B.odin_render_bwd(self.ctx, self.params.struct, cam, self.proj.struct, self.vals, self.ranges, self.final_T,
-                          self.n_contrib, self.dL, self.grad2d, self.grads.struct, self.ws, stream)
+                          self.n_contrib, self.dL, self.grad2d, self.grads.struct, self.row_active, self.ws, stream)
+
+    def active_set(self, slot: int = 0, evidence_mode: int = 0, stream=None) -> None:
+        """Realized active set of the view whose backward pass ran last: mask (slot), list, count, evidence, sum."""
+        B.odin_active_set(self.ctx, self.proj.struct, self.row_active, self.grad2d, self.grads.struct, evidence_mode,
+                          self.n, self.active_masks[slot], self.active_idx, self.row_capacity, self.active_count,
+                          self.evidence, self.evidence_sum, self.ws, stream)
 
     def sparse_adam(self, lr, beta1, beta2, eps, step: int, stream=None) -> None:
         B.odin_sparse_adam(self.ctx, self.params.struct, self.m.struct, self.v.struct, self.grads.struct, self.idx,

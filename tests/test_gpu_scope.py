@@ -1,0 +1,257 @@
+"""Parity of the realized active set, gradient evidence, unit unions, hazard counts and the delayed-read gate
+(Sec. 2.1 Table 1, Sec. 4.3) through the C ABI against the oracle (needs a GPU)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_19893_b200 import binding as B
+from paper_2607_19893_b200 import workloads as wl
+
+import gpu_util as G
+from test_gpu_stages import load_sorted, oracle_view, faint_scene
+
+pytestmark = pytest.mark.gpu
+
+
+def mask_ids(words, n):
+    return np.flatnonzero(np.unpackbits(np.ascontiguousarray(words).view(np.uint8), bitorder="little")[:n])
+
+
+# ------------------------------------------------------------------------------------------------ active set
+def check_active_set(oracle32, scene, cam, seed=0):
+    n = scene.n
+    f, inv = oracle_view(oracle32, scene, cam)
+    rng = np.random.default_rng(seed)
+    dl = rng.uniform(-1, 1, f["out"].shape).astype(np.float32)
+    robust = f["pix_margin"] > 2e-5
+    dl[:, ~robust] = 0  # see test_gpu_stages.check_backward
+    g2d_o, g2d_abs = oracle32.render_bwd_blend(f["proj"], f["vals"], f["ranges"], cam, f["final_T"], f["n_contrib"], dl,
+                                               want_abs=True)
+    rows_o = oracle32.render_bwd_project(scene, cam, f["idx"], g2d_o, f["proj"].clamp_flags).astype(np.float64)
+    _, active_o = oracle32.realized_active(f["proj"], f["vals"], f["ranges"], cam, f["n_contrib"])
+    # what is certain: activity through pixels whose decisions are all robust
+    nc_sure = f["n_contrib"].copy()
+    nc_sure[~robust] = 0
+    _, active_sure = oracle32.realized_active(f["proj"], f["vals"], f["ranges"], cam, nc_sure)
+    # what may differ: primitives inside the walked prefix of a fragile pixel
+    tx = (cam.width + 15) // 16
+    maybe = set()
+    for j, i in np.argwhere(~robust):
+        s = f["ranges"][(j // 16) * tx + i // 16, 0]
+        maybe |= set(f["vals"][s:s + f["n_contrib"][j, i]].tolist())
+
+    v = len(f["idx"])
+    tr = G.trainer_for(scene, cam, row_capacity=max(v, 1), instance_capacity=len(f["vals"]) + 1)
+    load_sorted(tr, f, inv)
+    tr.final_T.copy_(torch.from_numpy(f["final_T"]).to(tr.device))
+    tr.n_contrib.copy_(torch.from_numpy(f["n_contrib"].view(np.int32)).to(tr.device))
+    tr.dL.copy_(torch.from_numpy(dl).to(tr.device))
+    for mode in (0, 1, 0):
+        tr.render_bwd(B.make_camera(cam))
+        tr.active_set(slot=0, evidence_mode=mode)
+        G.poll_ok(tr)
+        cnt = int(tr.active_count.item())
+        idx = G.u32(tr.active_idx)[:cnt]
+        # list, mask and flags describe the same set; ascending primitive ids
+        assert np.all(np.diff(idx.astype(np.int64)) > 0)
+        assert np.array_equal(mask_ids(G.u32(tr.active_masks[0]), n), idx)
+        flags = tr.row_active.cpu().numpy()[:v].astype(bool)
+        assert np.array_equal(f["idx"][flags], idx)
+        # against the oracle: certain members present, nothing beyond what a fragile pixel can explain
+        dev, want = set(idx.tolist()), set(active_o.tolist())
+        assert set(active_sure.tolist()) <= dev
+        assert (dev ^ want) <= maybe
+        assert len(dev ^ want) <= max(2, int((~robust).sum()))
+        assert dev <= set(f["idx"].tolist())  # C_i inside G_i
+        # evidence of the primitives both sides call active
+        both = np.array(sorted(dev & want), np.int64)
+        ev_dev = tr.evidence.cpu().numpy()[:cnt].astype(np.float64)
+        ev_dev_both = ev_dev[np.searchsorted(idx, both)]
+        if mode == 0:
+            ev_o, _ = oracle32.gradient_evidence(g2d_o, both)
+            b = G.grad2d_bound(g2d_o[both, :2], g2d_abs[both, :2])
+            tol = np.sqrt((b * b).sum(axis=1)) + 1e-6 * ev_o
+        else:
+            ev_o, _ = oracle32.gradient_evidence(None, both, rows=rows_o, touched_idx=f["idx"])
+            bound = G.rows_bound(oracle32, scene, cam, f["idx"], f["proj"].clamp_flags, rows_o, g2d_o, g2d_abs)
+            pos = np.searchsorted(f["idx"].astype(np.int64), both)
+            tol = 10 * np.sqrt((bound[pos] ** 2).sum(axis=1)) + 1e-6 * ev_o
+        assert np.all(np.abs(ev_dev_both - ev_o) <= tol), np.abs(ev_dev_both - ev_o).max()
+        assert ev_o.max() > 1e-4
+        # the sum is the sum of the listed evidence
+        assert float(tr.evidence_sum.item()) == pytest.approx(float(ev_dev.sum()), rel=1e-12, abs=1e-30)
+    tr.close()
+    return len(active_o), v
+
+
+def test_active_set_cfg1(oracle32):
+    w = wl.make_workload(1)
+    check_active_set(oracle32, w.scene, w.cameras[0])
+
+
+def test_active_set_cfg2_many_occluded(oracle32):
+    w = wl.make_workload(2, n=30_000)
+    na, v = check_active_set(oracle32, w.scene, w.cameras[3], seed=2)
+    assert na < v  # some touched primitives never blend: the realized scope is strictly inside the candidate scope
+
+
+def test_active_set_long_lists_head_and_tail_kernels(oracle32):
+    s, cam = faint_scene(n=12_000)
+    check_active_set(oracle32, s, cam, seed=4)
+
+
+def test_active_set_capacity_and_empty_view(oracle32):
+    w = wl.make_workload(1)
+    cam = w.cameras[0]
+    f, inv = oracle_view(oracle32, w.scene, cam)
+    v = len(f["idx"])
+    tr = G.trainer_for(w.scene, cam, row_capacity=v, instance_capacity=len(f["vals"]) + 1)
+    load_sorted(tr, f, inv)
+    tr.final_T.copy_(torch.from_numpy(f["final_T"]).to(tr.device))
+    tr.n_contrib.copy_(torch.from_numpy(f["n_contrib"].view(np.int32)).to(tr.device))
+    tr.render_bwd(B.make_camera(cam))
+    # a list capacity smaller than the set: truncated list, deferred error, nothing written past the capacity
+    small = torch.full((64,), -1, dtype=torch.int32, device=tr.device)
+    ev = torch.full((64,), -1.0, dtype=torch.float32, device=tr.device)
+    B.odin_active_set(tr.ctx, tr.proj.struct, tr.row_active, tr.grad2d, None, 0, tr.n, tr.active_masks[0], small, 50,
+                      tr.active_count, ev, tr.evidence_sum, tr.ws)
+    assert tr.poll() == B.ODIN_ERR_CAPACITY
+    assert int(tr.active_count.item()) == 50
+    got = small.cpu().numpy()
+    assert np.all(got[50:] == -1) and np.all(np.diff(got[:50]) > 0) and np.all(ev.cpu().numpy()[50:] == -1.0)
+    # no rows at all
+    tr.proj.num_rows.zero_()
+    tr.active_set()
+    G.poll_ok(tr)
+    assert int(tr.active_count.item()) == 0 and float(tr.evidence_sum.item()) == 0.0
+    assert not G.u32(tr.active_masks[0]).any()
+    tr.close()
+
+
+def test_active_set_after_a_whole_view_step(oracle32):
+    w = wl.make_workload(2, n=40_000)
+    tr = G.trainer_for(w.scene, w.cameras[0], mask_slots=2)
+    for s, view in enumerate((1, 5)):
+        tr.target.copy_(torch.from_numpy(w.target(view)).to(tr.device))
+        tr.view_step(B.make_camera(w.cameras[view]), s + 1, w.lr, w.beta1, w.beta2, w.eps, slot=s)
+        tr.active_set(slot=s)
+        G.poll_ok(tr)
+        touched, active = G.u32(tr.masks[s]), G.u32(tr.active_masks[s])
+        assert not (active & ~touched).any()                       # C_i inside G_i, word by word
+        cnt = int(tr.active_count.item())
+        assert 0 < cnt <= int(tr.count.item())
+        assert cnt == int(np.unpackbits(active.view(np.uint8)).sum())
+    tr.close()
+
+
+# ------------------------------------------------------------------------------------------------ unions, hazards, gate
+def random_scopes(rng, n, units):
+    """Per unit: write scope inside read scope (Sec. 2.1: W+ inside R+)."""
+    reads, writes = [], []
+    for _ in range(units):
+        w = np.sort(rng.choice(n, rng.integers(0, n // 2 + 1), replace=False))
+        r = np.union1d(w, rng.choice(n, rng.integers(0, n // 3 + 1), replace=False))
+        reads.append(r); writes.append(w)
+    return reads, writes
+
+
+def to_device_masks(id_lists, n, dev):
+    from oracle.oracle import ids_to_mask
+    words = (n + 31) // 32
+    stride = (words + 3) // 4 * 4
+    m = np.zeros((len(id_lists), stride), np.uint32)
+    for k, ids in enumerate(id_lists):
+        m[k, :words] = ids_to_mask(ids, n)
+    return torch.from_numpy(m.view(np.int32)).to(dev), stride
+
+
+@pytest.mark.parametrize("n", [1, 31, 4097, 250_003])
+def test_hazard_counts_and_unions_match_the_set_algebra(oracle32, n):
+    rng = np.random.default_rng(n)
+    dev = torch.device("cuda", 0)
+    ctx = B.odin_create(0)
+    units = 5
+    reads, writes = random_scopes(rng, n, units)
+    d_r, stride = to_device_masks(reads, n, dev)
+    d_w, _ = to_device_masks(writes, n, dev)
+    pairs = np.array([(a, b) for a in range(units) for b in range(units)], np.uint32)
+    d_pairs = torch.from_numpy(pairs.view(np.int32)).to(dev)
+    d_counts = torch.full((len(pairs), 4), -1, dtype=torch.int64, device=dev)
+    B.odin_hazard_count(ctx, d_r, d_w, units, stride, n, d_pairs, len(pairs), d_counts)
+    assert B.odin_poll(ctx) == B.ODIN_OK
+    got = d_counts.cpu().numpy()
+    for (a, b), g in zip(pairs, got):
+        waw, raw, war = oracle32.hazard_sets(reads[a], writes[a], reads[b], writes[b])
+        assert g.tolist() == [len(waw), len(raw), len(war), len(reads[b])]
+    # the pipeline of this repository declares R+ = W+: RAW and WAR vanish, WAW is the conflict count
+    B.odin_hazard_count(ctx, d_w, d_w, units, stride, n, d_pairs, len(pairs), d_counts)
+    d_cc = torch.zeros(len(pairs), dtype=torch.int64, device=dev)
+    B.odin_conflict_count(ctx, d_w, units, stride, n, d_pairs, len(pairs), d_cc)
+    assert B.odin_poll(ctx) == B.ODIN_OK
+    got = d_counts.cpu().numpy()
+    assert not got[:, 1:3].any() and np.array_equal(got[:, 0], d_cc.cpu().numpy())
+    # unit unions: R+(U) = union over the views of the unit
+    members = np.array([0, 2, 3], np.uint32)
+    d_out = torch.full((stride,), -1, dtype=torch.int32, device=dev)
+    B.odin_mask_union(ctx, d_r, units, stride, n, torch.from_numpy(members.view(np.int32)).to(dev), 3, d_out)
+    assert B.odin_poll(ctx) == B.ODIN_OK
+    want = np.union1d(np.union1d(reads[0], reads[2]), reads[3])
+    assert np.array_equal(mask_ids(G.u32(d_out), n), want)
+    assert not G.u32(d_out)[(n + 31) // 32:].any()
+    B.odin_mask_union(ctx, d_r, units, stride, n, None, 0, d_out)      # the union over no view is empty
+    assert B.odin_poll(ctx) == B.ODIN_OK and not G.u32(d_out).any()
+    # a pair naming a unit that does not exist is reported and counts nothing
+    bad = torch.tensor([[0, units]], dtype=torch.int32, device=dev)
+    B.odin_hazard_count(ctx, d_r, d_w, units, stride, n, bad, 1, d_counts)
+    assert B.odin_poll(ctx) == B.ODIN_ERR_INVALID_ARG
+    B.odin_destroy(ctx)
+
+
+def run_gate(ctx, dev, n, r_b, w_b, w_a, active_a, ev_a, tau, capacity=None):
+    d_m, stride = to_device_masks([r_b, w_b, w_a], n, dev)
+    cap = len(active_a) if capacity is None else capacity
+    d_idx = torch.from_numpy(np.asarray(active_a, np.int32)).to(dev) if len(active_a) else torch.zeros(1, dtype=torch.int32, device=dev)
+    d_ev = torch.from_numpy(np.asarray(ev_a, np.float32)).to(dev) if len(active_a) else torch.zeros(1, device=dev)
+    d_cnt = torch.tensor([len(active_a)], dtype=torch.int32, device=dev)
+    d_sum = torch.tensor([float(np.asarray(ev_a, np.float32).astype(np.float64).sum())], dtype=torch.float64, device=dev)
+    d_gate = torch.full((4,), -1, dtype=torch.int64, device=dev)
+    B.odin_delayed_read_gate(ctx, d_m[0], d_m[1], d_m[2], n, d_idx, d_ev, d_cnt, d_sum, cap, tau, d_gate)
+    assert B.odin_poll(ctx) == B.ODIN_OK
+    return d_gate.cpu().numpy()
+
+
+def test_delayed_read_gate_hand_example(oracle32):
+    from test_oracle_scope_pins import read_golden
+    g = read_golden("delayed_read_gate_example.txt")
+    ints = lambda k: np.array([int(x) for x in g[k]])  # noqa: E731
+    ev = np.array([float(x) for x in g["evidence_A"]], np.float32)
+    dev = torch.device("cuda", 0)
+    ctx = B.odin_create(0)
+    for case in "1234":
+        tau = float(g["tau" + case][0])
+        gate = run_gate(ctx, dev, 32, ints("R_B" + case), ints("W_B" + case), ints("W_A"), ints("C_A"), ev, tau)
+        assert gate.tolist() == [int(g["n_delayed" + case][0]), int(g["n_with_evidence" + case][0]),
+                                 int(g["n_pass" + case][0]), len(ints("R_B" + case))]
+        assert B.admit_delayed_read(gate, len(ints("C_A")), tau) == (g["admitted" + case][0] == "yes")
+    B.odin_destroy(ctx)
+
+
+@pytest.mark.parametrize("n", [33, 5000, 300_001])
+def test_delayed_read_gate_random_scopes(oracle32, n):
+    rng = np.random.default_rng(3 * n)
+    dev = torch.device("cuda", 0)
+    ctx = B.odin_create(0)
+    for trial in range(6):
+        (r_a, r_b), (w_a, w_b) = random_scopes(rng, n, 2)
+        # A's realized set: most of its write scope (so some delayed primitives lack evidence), heavy-tailed evidence
+        active_a = np.sort(rng.choice(w_a, int(0.8 * len(w_a)), replace=False)) if len(w_a) else w_a
+        ev_a = rng.lognormal(-2.0, 1.5, len(active_a)).astype(np.float32)
+        tau = float(np.float32(rng.choice([0.05, 0.2, 0.5, 1.0])))
+        want = oracle32.delayed_read_gate(r_a, w_a, r_b, w_b, active_a, ev_a, tau)
+        gate = run_gate(ctx, dev, n, r_b, w_b, w_a, active_a, ev_a, tau)
+        assert gate.tolist() == [want["n_delayed"], want["n_with_evidence"], want["n_pass"], want["n_read_b"]], trial
+        assert B.admit_delayed_read(gate, len(active_a), tau) == want["admitted"]
+    # with R+ = W+ nothing is ever delayed
+    gate = run_gate(ctx, dev, n, w_b, w_b, w_a, active_a, ev_a, 0.2)
+    assert gate[0] == 0 and gate[1] == 0
+    B.odin_destroy(ctx)
