@@ -338,6 +338,46 @@ def main():
     tile_passes = max(1, (max(int(np.ceil(np.log2(max(tx * ty, 1)))), 0) + 7) // 8)
     bytes_kernels = kernel_bytes(n, f, v_last, m_last, m_proc, W * H, tx * ty, tile_passes, n_pairs_last)
 
+    # ---- scope calls beyond the view step (realized active set, hazard counts): timed on their own --------------
+    scope = None
+    if rank == 0:
+        reps = 20
+        last_slot = (total_steps - 1) % MASK_SLOTS
+        hz_pairs = torch.tensor([(a, last_slot) for a in range(MASK_SLOTS) if a != last_slot], dtype=torch.int32,
+                                device=dev)
+        hz_counts = torch.zeros((len(hz_pairs), 4), dtype=torch.int64, device=dev)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        tr.track_active = True                                           # one more view with the row flags on
+        step(total_steps - 1, bank[view_of(total_steps - 1)])
+        tr.active_set(slot=last_slot, stream=stream)                     # warm
+        B.odin_hazard_count(tr.ctx, tr.masks, tr.masks, MASK_SLOTS, tr.masks.shape[1], n, hz_pairs, len(hz_pairs),
+                            hz_counts, stream)
+        torch.cuda.synchronize()
+        ev[0].record(stream)
+        for _ in range(reps):
+            tr.active_set(slot=last_slot, stream=stream)
+        ev[1].record(stream)
+        for _ in range(reps):
+            B.odin_hazard_count(tr.ctx, tr.masks, tr.masks, MASK_SLOTS, tr.masks.shape[1], n, hz_pairs, len(hz_pairs),
+                                hz_counts, stream)
+        ev[2].record(stream)
+        torch.cuda.synchronize()
+        tr.track_active = False
+        n_active = int(tr.active_count.item())
+        t_as, t_hz = ev[0].elapsed_time(ev[1]) / reps, ev[1].elapsed_time(ev[2]) / reps
+        b_as = v_last * (1 + 4) + n_active * (8 + 4 + 4) + n / 8      # flags, ids, (g_u, g_v), list + evidence, mask
+        b_hz = len(hz_pairs) * 4 * n / 8                                # four masks per pair
+        peak_gbs_, _ = measured_peaks()
+        scope = {"active_set": {"ms": t_as, "active": n_active, "algorithmic_bytes": b_as,
+                                "frac_of_measured_hbm": b_as / (t_as * 1e-3) / 1e9 / peak_gbs_},
+                 "hazard_count": {"ms": t_hz, "pairs": int(len(hz_pairs)), "algorithmic_bytes": b_hz,
+                                  "frac_of_measured_hbm": b_hz / (t_hz * 1e-3) / 1e9 / peak_gbs_},
+                 "note": "not part of `value`: the realized active set and the hazard counts of Sec. 4.3 for the last "
+                         "view against the views before it, each averaged over 20 calls"}
+        st = tr.poll()
+        if st != B.ODIN_OK:
+            raise SystemExit(f"scope calls failed: {B.status_string(st)}")
+
     # ---- end-to-end run: host target in, loss / V / counts out, every step --------------------------------------
     h_loss = torch.zeros(1, dtype=torch.float32).pin_memory()
     h_count = torch.zeros(1, dtype=torch.int32).pin_memory()
@@ -424,6 +464,7 @@ def main():
                      "frac_of_measured_implementation_bytes":
                          bytes_kernels["total"] / (ms * 1e-3 / args.steps) / 1e9 / peak_gbs},
         "kernels": shares,
+        "scope_calls": scope,
     }
 
     # ---- the oracle on the host cores, bounded sample -----------------------------------------------------------

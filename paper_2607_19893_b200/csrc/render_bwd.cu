@@ -173,6 +173,10 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
 // pixels, the colour and opacity gradients and three moments of dL/dpower (sum, sum*dy, sum*dy^2); dx is constant per
 // lane, so the conic / centre gradients follow from the moments with a handful of operations per row instead of per
 // pixel.  One transposing warp reduction and nine global atomics per (tile, row) that contributed.
+// TRACK: also flag the rows that contributed (realized active set).  A separate instantiation because this loop is
+// sensitive to anything added to it: the flag store costs ~5 % of the kernel, and callers who do not ask for the flags
+// do not pay for it.
+template <bool TRACK>
 __global__ void __launch_bounds__(BLEND_THREADS)
 render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
                         const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
@@ -270,7 +274,6 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       }
       const uint32_t hit = __reduce_or_sync(0xffffffffu, pass);  // bit s: some lane of the warp passes in slot s
       if (hit == 0) continue;
-      if (row_active && lane == 0) row_active[s_rowid[warp][j]] = 1;  // realized-active (see the tail kernel)
       // phase 2: per-lane sums over its eight pixels; the x-dependent factors are applied once at the end
       float ar = 0.f, ag = 0.f, ab = 0.f, ao = 0.f, gpsum = 0.f, m1y = 0.f, m2yy = 0.f;
 #pragma unroll
@@ -309,9 +312,13 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       const float vA = -0.5f * dx * gd, vB = -dx * m1y, vC = -0.5f * m2yy;
       const float t8 = warp_transpose_sum8(vu, vv, vA, vB, vC, ao, ar, ag, lane);
       for (int o = 16; o > 0; o >>= 1) ab += __shfl_xor_sync(0xffffffffu, ab, o);
-      float* dst = g2d + (size_t)s_rowid[warp][j] * 9;
+      const uint32_t rid = s_rowid[warp][j];
+      float* dst = g2d + (size_t)rid * 9;
       if ((lane & 3) == 0) atomicAdd(dst + (lane >> 2), t8);
       if (lane == 1) atomicAdd(dst + 8, ab);
+      if (TRACK) {
+        if (lane == 2) row_active[rid] = 1;  // realized-active: blended into at least one pixel
+      }
     }
     __syncwarp();
   }
@@ -497,11 +504,15 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
     OdinKernelScope ks(ctx, K_BWD_BLEND, st);
     const int blocks_all = (n_tiles + BLEND_WARPS - 1) / BLEND_WARPS;
     const int blocks = blocks_all < ctx->sm_count * 8 ? blocks_all : ctx->sm_count * 8;  // resident warps pull tiles
-    render_bwd_blend_kernel<<<blocks, BLEND_THREADS, 0, st>>>(
-        reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
-        reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0], cam->bg[1],
-        cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, state, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d,
-        ticket, d_row_active);
+#define LAUNCH_BLEND(TRACK)                                                                                             \
+  render_bwd_blend_kernel<TRACK><<<blocks, BLEND_THREADS, 0, st>>>(                                                     \
+      reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb,       \
+      d_vals, reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0],          \
+      cam->bg[1], cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, state, d_final_T, d_n_contrib, d_dL_drgb,         \
+      d_grad2d, ticket, d_row_active)
+    if (d_row_active) LAUNCH_BLEND(true);
+    else LAUNCH_BLEND(false);
+#undef LAUNCH_BLEND
   }
   const CamParams cp = odin_cam_params(cam, ctx->cfg);
   const uint32_t blocks_cap = (proj->capacity + 127) / 128;

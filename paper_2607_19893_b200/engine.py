@@ -131,6 +131,7 @@ class ViewTrainer:
         self.ws = z(ws_bytes, torch.uint8)
         self.kernel_launches_per_step = 0
         self.keep_sorted_keys = False  # view_step: also write the sorted 64-bit keys (only tests look at them)
+        self.track_active = False      # render_bwd: also flag the rows that contributed (needed by active_set)
 
     def close(self) -> None:
         if self.ctx is not None:
@@ -159,10 +160,14 @@ class ViewTrainer:
 
     def render_bwd(self, cam: B.odin_camera, stream=None) -> None:
         B.odin_render_bwd(self.ctx, self.params.struct, cam, self.proj.struct, self.vals, self.ranges, self.final_T,
-                          self.n_contrib, self.dL, self.grad2d, self.grads.struct, self.row_active, self.ws, stream)
+                          self.n_contrib, self.dL, self.grad2d, self.grads.struct,
+                          self.row_active if self.track_active else None, self.ws, stream)
 
     def active_set(self, slot: int = 0, evidence_mode: int = 0, stream=None) -> None:
-        """Realized active set of the view whose backward pass ran last: mask (slot), list, count, evidence, sum."""
+        """Realized active set of the view whose backward pass ran last (with track_active set): mask (slot), list,
+        count, evidence, sum."""
+        if not self.track_active:
+            raise RuntimeError("active_set needs the row flags of render_bwd: set track_active before the backward pass")
         B.odin_active_set(self.ctx, self.proj.struct, self.row_active, self.grad2d, self.grads.struct, evidence_mode,
                           self.n, self.active_masks[slot], self.active_idx, self.row_capacity, self.active_count,
                           self.evidence, self.evidence_sum, self.ws, stream)

@@ -22,6 +22,7 @@ def run_chain(oracle32, w, steps, views, window=None, row_capacity=None, instanc
                        mask_slots=max(len(views), 1))
     rng = np.random.default_rng(7)
     tr.keep_sorted_keys = True  # the sorted keys are compared below
+    tr.track_active = True      # ... and the realized active set
     p = scene.copy()
     m, v = p.zeros_like(), p.zeros_like()
     masks_o = {}
@@ -57,6 +58,18 @@ def run_chain(oracle32, w, steps, views, window=None, row_capacity=None, instanc
             assert np.array_equal(rg[:, 1] - rg[:, 0], o["ranges"][:, 1] - o["ranges"][:, 0])
             # keys: tile ids are exact; depth bits come from the GPU projection (may differ in the last bit)
             assert np.array_equal(G.u64(tr.keys)[:mm] >> np.uint64(32), o["keys"] >> np.uint64(32))
+        # realized active set of the view (row flags of the backward pass): inside the touched set; against the oracle
+        # it may differ only by primitives whose activity hangs on a fragile pixel decision
+        tr.active_set(slot=slot)
+        G.poll_ok(tr)
+        n_act = int(tr.active_count.item())
+        act_dev = G.u32(tr.active_idx)[:n_act]
+        assert not (G.u32(tr.active_masks[slot]) & ~G.u32(tr.masks[slot])).any()
+        if not differs.any():
+            _, act_o = oracle32.realized_active(o["proj"], o["vals"], o["ranges"], cam, o["n_contrib"])
+            n_fragile_pix = int((o["pix_margin"] <= 2e-5).sum())
+            assert len(np.setxor1d(act_dev, act_o)) <= max(4, n_fragile_pix)
+            assert len(act_o) > 0
         robust = o["pix_margin"] > 1e-3
         out = tr.out.cpu().numpy()
         assert np.abs(out - o["out"])[:, robust].max() < 1e-4

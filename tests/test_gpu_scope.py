@@ -42,6 +42,7 @@ def check_active_set(oracle32, scene, cam, seed=0):
 
     v = len(f["idx"])
     tr = G.trainer_for(scene, cam, row_capacity=max(v, 1), instance_capacity=len(f["vals"]) + 1)
+    tr.track_active = True
     load_sorted(tr, f, inv)
     tr.final_T.copy_(torch.from_numpy(f["final_T"]).to(tr.device))
     tr.n_contrib.copy_(torch.from_numpy(f["n_contrib"].view(np.int32)).to(tr.device))
@@ -106,6 +107,7 @@ def test_active_set_capacity_and_empty_view(oracle32):
     f, inv = oracle_view(oracle32, w.scene, cam)
     v = len(f["idx"])
     tr = G.trainer_for(w.scene, cam, row_capacity=v, instance_capacity=len(f["vals"]) + 1)
+    tr.track_active = True
     load_sorted(tr, f, inv)
     tr.final_T.copy_(torch.from_numpy(f["final_T"]).to(tr.device))
     tr.n_contrib.copy_(torch.from_numpy(f["n_contrib"].view(np.int32)).to(tr.device))
@@ -131,6 +133,9 @@ def test_active_set_capacity_and_empty_view(oracle32):
 def test_active_set_after_a_whole_view_step(oracle32):
     w = wl.make_workload(2, n=40_000)
     tr = G.trainer_for(w.scene, w.cameras[0], mask_slots=2)
+    with pytest.raises(RuntimeError):
+        tr.active_set()                                             # the flags have to be asked for first
+    tr.track_active = True
     for s, view in enumerate((1, 5)):
         tr.target.copy_(torch.from_numpy(w.target(view)).to(tr.device))
         tr.view_step(B.make_camera(w.cameras[view]), s + 1, w.lr, w.beta1, w.beta2, w.eps, slot=s)
