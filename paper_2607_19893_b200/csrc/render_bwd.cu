@@ -177,7 +177,7 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
 // sensitive to anything added to it: the flag store costs ~5 % of the kernel, and callers who do not ask for the flags
 // do not pay for it.
 template <bool TRACK>
-__global__ void __launch_bounds__(BLEND_THREADS)
+__global__ void __launch_bounds__(BLEND_THREADS, 5)
 render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
                         const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
                         int n_tiles, float bg0, float bg1, float bg2, float alpha_min, float alpha_max,
