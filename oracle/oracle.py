@@ -262,6 +262,42 @@ class Oracle:
                                and passes.all())
         return out
 
+    # ------------------------------------------------------------------ relative locality graph from counts (Sec. 4.1, 4.2)
+    @staticmethod
+    def rlg_weights(sizes, pairs, counts) -> np.ndarray:
+        """Eq. (1) with the per-view primitive sets in the place of the track sets (the computation-based RLG of
+        Sec. 4.1): w_ij = |P_i & P_j| / |P_i | P_j|, 0 when the union is empty.  One float32 division per pair."""
+        sizes = np.asarray(sizes, np.int64)
+        pairs = np.asarray(pairs, np.int64).reshape(-1, 2)
+        inter = np.asarray(counts, np.int64)
+        union = sizes[pairs[:, 0]] + sizes[pairs[:, 1]] - inter
+        w = np.zeros(len(pairs), np.float32)
+        nz = union > 0
+        w[nz] = inter[nz].astype(np.float32) / union[nz].astype(np.float32)
+        return w
+
+    @staticmethod
+    def rlg_topk(weights, k: int) -> np.ndarray:
+        """Neighbour retention of Sec. 4.1: every item keeps its k strongest neighbours (larger weight first, lower
+        index first among equals, zero weights are not edges); the graph is undirected, so an edge stays when either
+        end keeps it.  Dropped edges read as w = 0."""
+        w = np.array(weights, np.float32, copy=True)
+        n = w.shape[0]
+        np.fill_diagonal(w, 0)
+        keep = np.zeros((n, n), bool)
+        for i in range(n):
+            order = sorted((j for j in range(n) if j != i and w[i, j] > 0), key=lambda j: (-w[i, j], j))
+            keep[i, order[:k]] = True
+        keep |= keep.T
+        return np.where(keep, w, np.float32(0))
+
+    @staticmethod
+    def sds_scores(weights, prev_unit, candidates) -> np.ndarray:
+        """Eq. (2): s(v | U_prev) = sum over u in U_prev of w_uv, for every candidate v."""
+        w = np.asarray(weights, np.float64)
+        prev_unit = np.asarray(prev_unit, np.int64)
+        return np.array([w[prev_unit, v].sum() for v in np.asarray(candidates, np.int64)], np.float64)
+
     def sh_basis(self, degree: int, x: float, y: float, z: float) -> np.ndarray:
         out = np.zeros(16, self.dtype)
         ct = C.c_float if self.dtype == np.float32 else C.c_double

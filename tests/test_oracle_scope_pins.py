@@ -166,3 +166,61 @@ def test_delayed_read_gate_hand_example(oracle64):
     # an empty consumer read scope has no delayed-read admission to perform
     out = oracle64.delayed_read_gate(ints("R_A"), ints("W_A"), [], [], ints("C_A"), ev, 1.0)
     assert out["rho"] is None and not out["admitted"] and out["n_delayed"] == 0
+
+
+# ------------------------------------------------------------------------------- relative locality graph from counts
+def dense_from_pairs(n, pairs, w):
+    m = np.zeros((n, n), np.float32)
+    for (a, b), x in zip(pairs, w):
+        m[a, b] = m[b, a] = x
+    return m
+
+
+def test_rlg_weights_topk_and_sds_scores_hand_example(oracle64):
+    g = read_golden("rlg_example.txt")
+    sizes = np.array([int(x) for x in g["sizes"]])
+    pairs = np.array([int(x) for x in g["pairs"]]).reshape(-1, 2)
+    counts = np.array([int(x) for x in g["counts"]])
+    w = oracle64.rlg_weights(sizes, pairs, counts)
+    assert np.allclose(w, [float(x) for x in g["weights"]], rtol=1e-6)
+    full = dense_from_pairs(4, pairs, w)
+    top1 = oracle64.rlg_topk(full, 1)
+    edges = {tuple(e) for e in np.array([int(x) for x in g["top1_edges"]]).reshape(-1, 2).tolist()}
+    assert {(a, b) for a in range(4) for b in range(a + 1, 4) if top1[a, b] > 0} == edges
+    assert np.array_equal(top1, top1.T) and not np.diag(top1).any()
+    prev, cand = [int(x) for x in g["prev_unit"]], [int(x) for x in g["candidates"]]
+    assert np.allclose(oracle64.sds_scores(full, prev, cand), [float(x) for x in g["scores_full"]], rtol=1e-6)
+    assert np.allclose(oracle64.sds_scores(top1, prev, cand), [float(x) for x in g["scores_top1"]], rtol=1e-6)
+
+
+def test_rlg_weights_are_jaccard_of_the_sets_and_topk_is_monotone(oracle64):
+    rng = np.random.default_rng(21)
+    n, views = 3000, 9
+    sets = [set(rng.choice(n, rng.integers(0, 1500), replace=False).tolist()) for _ in range(views)]
+    sets[4] = set()
+    pairs = np.array([(a, b) for a in range(views) for b in range(a + 1, views)])
+    counts = np.array([len(sets[a] & sets[b]) for a, b in pairs])
+    sizes = np.array([len(s) for s in sets])
+    w = oracle64.rlg_weights(sizes, pairs, counts)
+    for (a, b), x in zip(pairs, w):
+        u = len(sets[a] | sets[b])
+        assert np.isclose(x, len(sets[a] & sets[b]) / u if u else 0.0, rtol=1e-6)
+        assert 0.0 <= x <= 1.0
+    full = dense_from_pairs(views, pairs, w)
+    prev_edges = -1
+    for k in range(0, views):
+        g = oracle64.rlg_topk(full, k)
+        assert np.array_equal(g, g.T)
+        assert np.all((g == 0) | (g == full))                       # retention only removes edges
+        deg_kept = [(np.argsort(-full[i], kind="stable")[:k]) for i in range(views)]
+        for i in range(views):                                      # every item still sees its own k strongest
+            for j in deg_kept[i]:
+                if full[i, j] > 0:
+                    assert g[i, j] == full[i, j]
+        edges = int((g > 0).sum())
+        assert edges >= prev_edges
+        prev_edges = edges
+    assert np.array_equal(oracle64.rlg_topk(full, views), full)     # k >= degree keeps everything
+    # Eq. (2) is additive over the previous unit
+    s01 = oracle64.sds_scores(full, [0, 1], [5, 6, 7])
+    assert np.allclose(s01, oracle64.sds_scores(full, [0], [5, 6, 7]) + oracle64.sds_scores(full, [1], [5, 6, 7]))
