@@ -258,6 +258,28 @@ int odin_delayed_read_gate(odin_ctx* ctx, const uint32_t* d_read_b, const uint32
                            const uint32_t* d_active_count_a, const double* d_evidence_sum_a, uint32_t active_capacity_a,
                            float tau, uint64_t* d_gate, void* stream);
 
+/* ---- relative locality graph from the measured scopes (Sec. 4.1 Eq. (1), Sec. 4.2 Eq. (2)) ------------------------
+ * The paper builds its ahead-of-time graph from SfM tracks and says that realized activity can refresh the scores
+ * later; these calls evaluate the same formulas on the per-view primitive sets this library produces (the
+ * computation-based graph of Sec. 4.1): set sizes from odin_touched_set / odin_active_set, intersections from
+ * odin_conflict_count / odin_hazard_count. */
+
+/* Eq. (1): d_weights [n_pairs] = d_counts[i] / (d_sizes[a] + d_sizes[b] - d_counts[i]) for pair i = (a, b), 0 when the
+ * union is empty (one float32 division).  d_counts [n_pairs] u64 intersection sizes, d_sizes [n_views] set sizes. */
+int odin_rlg_weights(odin_ctx* ctx, const uint64_t* d_counts, const uint32_t* d_sizes, const uint32_t* d_pairs,
+                     uint32_t n_pairs, uint32_t n_views, float* d_weights, void* stream);
+
+/* Neighbour retention: every item keeps its k strongest neighbours (larger weight first, lower index first among equal
+ * weights; zero weights are not edges); the graph is undirected, so an edge stays when either end keeps it.
+ * d_weights, d_retained [n_views][n_views] row major (distinct buffers; d_weights symmetric); dropped edges and the
+ * diagonal are written as 0.  ws: n_views^2 bytes.  n_views <= 32768. */
+int odin_rlg_topk(odin_ctx* ctx, const float* d_weights, uint32_t n_views, uint32_t k, float* d_retained, void* ws,
+                  size_t ws_bytes, void* stream);
+
+/* Eq. (2): d_scores[c] = sum over u in the previous unit of w[u][v], v = d_candidates[c] (fp32 accumulation). */
+int odin_sds_scores(odin_ctx* ctx, const float* d_weights, uint32_t n_views, const uint32_t* d_prev_unit, uint32_t n_prev,
+                    const uint32_t* d_candidates, uint32_t n_candidates, float* d_scores, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -28,7 +28,7 @@ EXPORTS = [
     "odin_touched_set", "odin_bin_sort", "odin_render_fwd", "odin_l1_loss", "odin_render_bwd", "odin_sparse_adam",
     "odin_conflict_count", "odin_kernel_count", "odin_kernel_name", "odin_profile_enable", "odin_profile_collect",
     "odin_touched_set_static", "odin_render_workspace_bytes", "odin_active_set", "odin_mask_union", "odin_hazard_count",
-    "odin_delayed_read_gate",
+    "odin_delayed_read_gate", "odin_rlg_weights", "odin_rlg_topk", "odin_sds_scores",
 ]
 
 
@@ -100,6 +100,9 @@ def lib() -> C.CDLL:
         L.odin_mask_union.argtypes = [vp, vp, u32, u32, u32, vp, u32, vp, vp]
         L.odin_hazard_count.argtypes = [vp, vp, vp, u32, u32, u32, vp, u32, vp, vp]
         L.odin_delayed_read_gate.argtypes = [vp, vp, vp, vp, u32, vp, vp, vp, vp, u32, f32, vp, vp]
+        L.odin_rlg_weights.argtypes = [vp, vp, vp, vp, u32, u32, vp, vp]
+        L.odin_rlg_topk.argtypes = [vp, vp, u32, u32, vp, vp, C.c_size_t, vp]
+        L.odin_sds_scores.argtypes = [vp, vp, u32, vp, u32, vp, u32, vp, vp]
         L.odin_kernel_count.argtypes = []
         L.odin_kernel_name.argtypes = [i32]
         L.odin_profile_enable.argtypes = [vp, i32]
@@ -277,6 +280,22 @@ def odin_delayed_read_gate(ctx, d_read_b, d_write_b, d_write_a, n_prims: int, d_
                                         _ptr(d_active_idx_a), _ptr(d_evidence_a), _ptr(d_active_count_a),
                                         _ptr(d_evidence_sum_a), int(active_capacity_a), float(tau), _ptr(d_gate),
                                         _stream(stream)), "odin_delayed_read_gate")
+
+
+def odin_rlg_weights(ctx, d_counts, d_sizes, d_pairs, n_pairs: int, n_views: int, d_weights, stream=None) -> None:
+    _check(lib().odin_rlg_weights(ctx, _ptr(d_counts), _ptr(d_sizes), _ptr(d_pairs), int(n_pairs), int(n_views),
+                                  _ptr(d_weights), _stream(stream)), "odin_rlg_weights")
+
+
+def odin_rlg_topk(ctx, d_weights, n_views: int, k: int, d_retained, ws, stream=None) -> None:
+    _check(lib().odin_rlg_topk(ctx, _ptr(d_weights), int(n_views), int(k), _ptr(d_retained), _ptr(ws),
+                               0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)), "odin_rlg_topk")
+
+
+def odin_sds_scores(ctx, d_weights, n_views: int, d_prev_unit, n_prev: int, d_candidates, n_candidates: int, d_scores,
+                    stream=None) -> None:
+    _check(lib().odin_sds_scores(ctx, _ptr(d_weights), int(n_views), _ptr(d_prev_unit), int(n_prev), _ptr(d_candidates),
+                                 int(n_candidates), _ptr(d_scores), _stream(stream)), "odin_sds_scores")
 
 
 def admit_delayed_read(gate, active_count_a: int, tau: float) -> bool:

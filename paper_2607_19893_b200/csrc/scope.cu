@@ -191,7 +191,125 @@ delayed_read_gate_kernel(const uint32_t* __restrict__ read_b, const uint32_t* __
   block_add4(n_delayed, n_with, n_pass, nrb, gate);
 }
 
+// ------------------------------------------------------------------------------------------------ locality graph
+// Eq. (1) on per-view primitive sets: one float32 division per pair.
+__global__ void rlg_weights_kernel(const unsigned long long* __restrict__ counts, const uint32_t* __restrict__ sizes,
+                                   const uint32_t* __restrict__ pairs, uint32_t n_pairs, uint32_t n_views,
+                                   float* __restrict__ weights, int* status) {
+  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n_pairs; i += gridDim.x * blockDim.x) {
+    const uint32_t a = pairs[2 * i], b = pairs[2 * i + 1];
+    float w = 0.f;
+    if (a < n_views && b < n_views) {
+      const unsigned long long inter = counts[i];
+      const unsigned long long uni = (unsigned long long)sizes[a] + sizes[b] - inter;
+      if (uni > 0) w = (float)inter / (float)uni;
+    } else {
+      odin_set_error(status, ODIN_ERR_INVALID_ARG);
+    }
+    weights[i] = w;
+  }
+}
+
+// Neighbour retention.  keep[i][j] = 1 when j is among the k strongest neighbours of i (larger weight first, lower index
+// first among equals, zero weights are not edges).  One block per item i, thread j ranks w_ij by counting who beats it.
+__global__ void rlg_rank_kernel(const float* __restrict__ w, uint32_t n, uint32_t k, uint8_t* __restrict__ keep) {
+  const uint32_t i = blockIdx.x;
+  for (uint32_t j = threadIdx.x; j < n; j += blockDim.x) {
+    const float x = (j == i) ? 0.f : w[(size_t)i * n + j];
+    uint32_t rank = 0;
+    if (x > 0.f)
+      for (uint32_t q = 0; q < n; ++q) {
+        if (q == i) continue;
+        const float y = w[(size_t)i * n + q];
+        rank += (y > x || (y == x && q < j)) ? 1u : 0u;
+      }
+    keep[(size_t)i * n + j] = (x > 0.f && rank < k) ? 1 : 0;
+  }
+}
+
+// The graph is undirected: an edge stays when either end keeps it; dropped edges and the diagonal read as 0.
+__global__ void rlg_retain_kernel(const float* __restrict__ w, const uint8_t* __restrict__ keep, uint32_t n,
+                                  float* __restrict__ out) {
+  const size_t total = (size_t)n * n;
+  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+    const uint32_t i = (uint32_t)(e / n), j = (uint32_t)(e % n);
+    out[e] = (i != j && (keep[e] || keep[(size_t)j * n + i])) ? w[e] : 0.f;
+  }
+}
+
+// Eq. (2): one block per candidate v, threads stride over the previous unit.
+__global__ void __launch_bounds__(128)
+sds_scores_kernel(const float* __restrict__ w, uint32_t n, const uint32_t* __restrict__ prev, uint32_t n_prev,
+                  const uint32_t* __restrict__ cand, float* __restrict__ scores, int* status) {
+  __shared__ float s[4];
+  const uint32_t v = cand[blockIdx.x];
+  float acc = 0.f;
+  if (v < n) {
+    for (uint32_t q = threadIdx.x; q < n_prev; q += 128) {
+      const uint32_t u = prev[q];
+      if (u < n) acc += w[(size_t)u * n + v];
+      else odin_set_error(status, ODIN_ERR_INVALID_ARG);
+    }
+  } else if (threadIdx.x == 0) {
+    odin_set_error(status, ODIN_ERR_INVALID_ARG);
+  }
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) s[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) scores[blockIdx.x] = s[0] + s[1] + s[2] + s[3];
+}
+
 }  // namespace
+
+extern "C" int odin_rlg_weights(odin_ctx* ctx, const uint64_t* d_counts, const uint32_t* d_sizes, const uint32_t* d_pairs,
+                                uint32_t n_pairs, uint32_t n_views, float* d_weights, void* stream) {
+  if (!ctx) return ODIN_ERR_NULL;
+  if (n_pairs == 0) return ODIN_OK;
+  if (!d_counts || !d_sizes || !d_pairs || !d_weights) return ODIN_ERR_NULL;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint32_t grid = (n_pairs + 255) / 256;
+  if (grid > (uint32_t)ctx->sm_count * 8) grid = (uint32_t)ctx->sm_count * 8;
+  OdinKernelScope ks(ctx, K_RLG, st);
+  rlg_weights_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const unsigned long long*>(d_counts), d_sizes, d_pairs,
+                                          n_pairs, n_views, d_weights, ctx->d_status);
+  return odin_launch_status();
+}
+
+extern "C" int odin_rlg_topk(odin_ctx* ctx, const float* d_weights, uint32_t n_views, uint32_t k, float* d_retained,
+                             void* ws, size_t ws_bytes, void* stream) {
+  if (!ctx) return ODIN_ERR_NULL;
+  if (n_views == 0) return ODIN_OK;
+  if (n_views > 32768) return ODIN_ERR_INVALID_ARG;
+  if (!d_weights || !d_retained) return ODIN_ERR_NULL;
+  if (d_weights == d_retained) return ODIN_ERR_INVALID_ARG;
+  const size_t need = (size_t)n_views * n_views;
+  if (!ws || ws_bytes < need) return ODIN_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint8_t* keep = reinterpret_cast<uint8_t*>(ws);
+  {
+    OdinKernelScope ks(ctx, K_RLG, st);
+    rlg_rank_kernel<<<n_views, 128, 0, st>>>(d_weights, n_views, k, keep);
+  }
+  size_t grid = (need + 255) / 256;
+  if (grid > (size_t)ctx->sm_count * 8) grid = (size_t)ctx->sm_count * 8;
+  OdinKernelScope ks(ctx, K_RLG, st);
+  rlg_retain_kernel<<<(unsigned)grid, 256, 0, st>>>(d_weights, keep, n_views, d_retained);
+  return odin_launch_status();
+}
+
+extern "C" int odin_sds_scores(odin_ctx* ctx, const float* d_weights, uint32_t n_views, const uint32_t* d_prev_unit,
+                               uint32_t n_prev, const uint32_t* d_candidates, uint32_t n_candidates, float* d_scores,
+                               void* stream) {
+  if (!ctx) return ODIN_ERR_NULL;
+  if (n_candidates == 0) return ODIN_OK;
+  if (!d_weights || !d_candidates || !d_scores || (n_prev > 0 && !d_prev_unit)) return ODIN_ERR_NULL;
+  if (n_views == 0) return ODIN_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  OdinKernelScope ks(ctx, K_RLG, st);
+  sds_scores_kernel<<<n_candidates, 128, 0, st>>>(d_weights, n_views, d_prev_unit, n_prev, d_candidates, d_scores,
+                                                 ctx->d_status);
+  return odin_launch_status();
+}
 
 extern "C" int odin_active_set(odin_ctx* ctx, const odin_projected* proj, const uint8_t* d_row_active,
                                const float* d_grad2d, const odin_scene* grad_rows, int evidence_mode, uint32_t n,

@@ -212,6 +212,67 @@ def test_hazard_counts_and_unions_match_the_set_algebra(oracle32, n):
     B.odin_destroy(ctx)
 
 
+# ------------------------------------------------------------------------------------------------ locality graph
+def test_locality_graph_from_the_masks_of_rendered_views(oracle32):
+    """Eq. (1) on the touched sets of eight rendered views (sizes and intersections measured by the library), top-k
+    retention, Eq. (2) scores: weights and retained edges bit exact, scores to fp32 summation order."""
+    w = wl.make_workload(2, n=60_000)
+    views = 8
+    tr = G.trainer_for(w.scene, w.cameras[0], mask_slots=views)
+    sizes = torch.zeros(views, dtype=torch.int32, device=tr.device)
+    sets = []
+    for v in range(views):
+        tr.project(B.make_camera(w.cameras[v]))
+        tr.touched_set(slot=v)
+        sizes[v:v + 1].copy_(tr.count)
+        G.poll_ok(tr)
+        sets.append(G.u32(tr.idx)[: int(tr.count.item())].copy())
+    pairs = np.array([(a, b) for a in range(views) for b in range(a + 1, views)], np.uint32)
+    d_pairs = torch.from_numpy(pairs.view(np.int32)).to(tr.device)
+    d_counts = torch.zeros(len(pairs), dtype=torch.int64, device=tr.device)
+    tr.conflict_count(d_pairs, len(pairs), d_counts)
+    d_w = torch.full((len(pairs),), -1.0, dtype=torch.float32, device=tr.device)
+    B.odin_rlg_weights(tr.ctx, d_counts, sizes, d_pairs, len(pairs), views, d_w)
+    G.poll_ok(tr)
+    counts_o = np.array([oracle32.conflict_count(sets[a], sets[b]) for a, b in pairs])
+    want_w = oracle32.rlg_weights([len(s) for s in sets], pairs, counts_o)
+    assert np.array_equal(d_w.cpu().numpy(), want_w) and want_w.max() > 0.05
+    full = np.zeros((views, views), np.float32)
+    for (a, b), x in zip(pairs, want_w):
+        full[a, b] = full[b, a] = x
+    d_full = torch.from_numpy(full).to(tr.device)
+    d_ret = torch.full((views, views), -1.0, dtype=torch.float32, device=tr.device)
+    ws = torch.zeros(views * views, dtype=torch.uint8, device=tr.device)
+    prev = torch.tensor([0, 3, 5], dtype=torch.int32, device=tr.device)
+    cand = torch.tensor([1, 2, 4, 6, 7], dtype=torch.int32, device=tr.device)
+    d_s = torch.zeros(5, dtype=torch.float32, device=tr.device)
+    for k in (0, 1, 2, 3, 7, 100):
+        B.odin_rlg_topk(tr.ctx, d_full, views, k, d_ret, ws)
+        G.poll_ok(tr)
+        want = oracle32.rlg_topk(full, k)
+        assert np.array_equal(d_ret.cpu().numpy(), want)
+        B.odin_sds_scores(tr.ctx, d_ret, views, prev, 3, cand, 5, d_s)
+        G.poll_ok(tr)
+        assert np.allclose(d_s.cpu().numpy(), oracle32.sds_scores(want, [0, 3, 5], [1, 2, 4, 6, 7]), rtol=1e-6, atol=1e-7)
+    # equal weights: the lower index wins the last retained place
+    tie = np.zeros((4, 4), np.float32)
+    tie[0, 1] = tie[1, 0] = tie[0, 2] = tie[2, 0] = tie[0, 3] = tie[3, 0] = 0.25
+    tie[2, 3] = tie[3, 2] = 0.5
+    d_tie = torch.from_numpy(tie).to(tr.device)
+    d_ret4 = torch.zeros((4, 4), dtype=torch.float32, device=tr.device)
+    B.odin_rlg_topk(tr.ctx, d_tie, 4, 1, d_ret4, ws)
+    G.poll_ok(tr)
+    # item 0 keeps 1 (first of three equals), item 1 keeps 0, items 2 and 3 keep each other: {0,2} and {0,3} are dropped
+    got = d_ret4.cpu().numpy()
+    assert np.array_equal(got, oracle32.rlg_topk(tie, 1))
+    assert got[0, 1] == 0.25 and got[0, 2] == 0 and got[0, 3] == 0 and got[2, 3] == 0.5
+    # a pair that names a view that does not exist is reported
+    bad = torch.tensor([[0, views]], dtype=torch.int32, device=tr.device)
+    B.odin_rlg_weights(tr.ctx, d_counts, sizes, bad, 1, views, d_w)
+    assert tr.poll() == B.ODIN_ERR_INVALID_ARG
+    tr.close()
+
+
 def run_gate(ctx, dev, n, r_b, w_b, w_a, active_a, ev_a, tau, capacity=None):
     d_m, stride = to_device_masks([r_b, w_b, w_a], n, dev)
     cap = len(active_a) if capacity is None else capacity
