@@ -43,6 +43,7 @@ struct Config {
   double radius_sigmas = 3.0;      // screen-space extent in standard deviations
   double jac_clamp = 1.3;          // guard on t_x/t_z, t_y/t_z inside the projection Jacobian
   int tile = 16;
+  int binning = 0;                 // 0: rectangle of the radius; 1: additionally cut to the extent of alpha >= alpha_min
 };
 
 struct CameraD {
@@ -249,6 +250,35 @@ void project(int64_t n, int sh_degree, const Real* means, const Real* log_scales
     int x1 = (int)std::min<Real>((Real)cam.TX, std::max<Real>(0, fx1));
     int y0 = (int)std::min<Real>((Real)cam.TY, std::max<Real>(0, fy0));
     int y1 = (int)std::min<Real>((Real)cam.TY, std::max<Real>(0, fy1));
+    const Real opac = 1 / (1 + std::exp(-opacity_logit[p]));
+    if (cfg.binning == 1) {
+      // Optimised-pipeline variant (Sec. 5: pipelines with tighter kernels keep the same primitive-id namespace): the
+      // rectangle is cut to the axis-aligned extent of the region where alpha = opac * exp(-q/2) can reach alpha_min,
+      // q = d^T Sigma'^-1 d <= k = 2 ln(opac / alpha_min), whose half extents are sqrt(k Sigma'_xx), sqrt(k Sigma'_yy).
+      // No pixel outside it passes the skip test, so images and gradients are those of the plain rectangle.  The
+      // extent is widened by 1e-4 relative + 1e-3 pixels against rounding of the per-pixel test.
+      const Real amin = (Real)cfg.alpha_min;
+      mg = std::min(mg, std::abs(opac - amin) / amin);
+      if (!(opac >= amin)) {
+        x1 = x0;  // never reaches alpha_min anywhere
+      } else {
+        const Real k = 2 * std::log(opac / amin);
+        const Real ex = std::sqrt(k * g.a) * (Real)1.0001 + (Real)1e-3, ey = std::sqrt(k * g.c) * (Real)1.0001 + (Real)1e-3;
+        // tiles that hold a pixel centre (i + 0.5) within [u - ex, u + ex]
+        const Real e[4] = {(u - ex - (Real)0.5) / tile, (u + ex - (Real)0.5) / tile, (v - ey - (Real)0.5) / tile,
+                           (v + ey - (Real)0.5) / tile};
+        const int tx0 = (int)std::min<Real>((Real)cam.TX, std::max<Real>(0, std::floor(e[0])));
+        const int tx1 = (int)std::min<Real>((Real)cam.TX, std::max<Real>(0, std::floor(e[1]) + 1));
+        const int ty0 = (int)std::min<Real>((Real)cam.TY, std::max<Real>(0, std::floor(e[2])));
+        const int ty1 = (int)std::min<Real>((Real)cam.TY, std::max<Real>(0, std::floor(e[3]) + 1));
+        x0 = std::max(x0, tx0); x1 = std::max(x0, std::min(x1, tx1));
+        y0 = std::max(y0, ty0); y1 = std::max(y0, std::min(y1, ty1));
+        for (int i = 0; i < 4; ++i) {
+          Real f = e[i] - std::floor(e[i]);
+          mg = std::min(mg, std::min(f, 1 - f) / std::max<Real>(1, std::abs(e[i])));
+        }
+      }
+    }
     // decision margins: radius rounding and the four rectangle edges (in units of one tile)
     {
       Real fr = rr - std::floor(rr);
@@ -270,7 +300,7 @@ void project(int64_t n, int sh_degree, const Real* means, const Real* log_scales
     rect[4 * p] = x0; rect[4 * p + 1] = y0; rect[4 * p + 2] = x1; rect[4 * p + 3] = y1;
     xy[2 * p] = u; xy[2 * p + 1] = v; depth[p] = g.t[2];
     conic_o[4 * p] = A; conic_o[4 * p + 1] = B; conic_o[4 * p + 2] = C;
-    conic_o[4 * p + 3] = 1 / (1 + std::exp(-opacity_logit[p]));
+    conic_o[4 * p + 3] = opac;
     // view-dependent colour
     Real d[3] = {means[3 * p] - cam.pos[0], means[3 * p + 1] - cam.pos[1], means[3 * p + 2] - cam.pos[2]};
     Real len = std::sqrt(d[0] * d[0] + d[1] * d[1] + d[2] * d[2]);

@@ -13,7 +13,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = os.path.join(_HERE, "liboracle.so")
 _SRC = [os.path.join(_HERE, "oracle_capi.cpp"), os.path.join(_HERE, "odin_oracle.hpp")]
 
-DEFAULT_CFG = np.array([1.0 / 255.0, 0.99, 1e-4, 0.3, 3.0, 1.3, 16.0], dtype=np.float64)
+# alpha_min, alpha_max, t_min, dilation, radius_sigmas, jac_clamp, tile, binning (0 plain rectangle, 1 tight extent)
+DEFAULT_CFG = np.array([1.0 / 255.0, 0.99, 1e-4, 0.3, 3.0, 1.3, 16.0, 0.0], dtype=np.float64)
 
 
 def build(force: bool = False) -> str:

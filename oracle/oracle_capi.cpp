@@ -19,7 +19,7 @@ Config cfg_from(const double* c) {
   Config k;
   if (c) {
     k.alpha_min = c[0]; k.alpha_max = c[1]; k.t_min = c[2]; k.dilation = c[3];
-    k.radius_sigmas = c[4]; k.jac_clamp = c[5]; k.tile = (int)c[6];
+    k.radius_sigmas = c[4]; k.jac_clamp = c[5]; k.tile = (int)c[6]; k.binning = (int)c[7];
   }
   return k;
 }
