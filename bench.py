@@ -223,6 +223,9 @@ def main():
     ap.add_argument("--impl", default="odin", choices=["odin", "reference"])
     ap.add_argument("--no-kernel-events", action="store_true", help="do not bracket kernels with CUDA events")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--binning", type=int, default=0, choices=[0, 1],
+                    help="0: tile rectangle of the radius (the method as published, the default and the headline); "
+                         "1: tight-extent rectangles (same image and gradients, fewer instances)")
     ap.add_argument("--city-grid", type=int, default=None,
                     help="config 5 only: a city of GxG blocks at the same density (default 64x64 = 20M primitives); "
                          "for profiler captures that must stay within a few GB")
@@ -261,7 +264,8 @@ def main():
     row_cap = max(1, int(ROW_CAP_FRAC[args.config] * n))
     if args.config == 5:  # a smaller city (--city-grid) shows the same absolute number of primitives per view
         row_cap = min(n, max(row_cap, 1_600_000))
-    tr = ViewTrainer(scene, W, H, row_cap, INSTANCE_CAP[args.config], mask_slots=MASK_SLOTS, device=local_rank)
+    tr = ViewTrainer(scene, W, H, row_cap, INSTANCE_CAP[args.config], mask_slots=MASK_SLOTS, device=local_rank,
+                     cfg=B.default_config(binning=args.binning))
     n_views = min(len(w.cameras), args.steps + args.warmup)
     view_of = lambda s: replica_view(s, rank, n_views)  # noqa: E731
     cams = [B.make_camera(c) for c in w.cameras[:n_views]]
@@ -451,7 +455,7 @@ def main():
         "data": "synthetic",
         "config": {"workload": w.name, "primitives": n, "floats_per_primitive": f, "image": [W, H], "views": n_views,
                    "visible_last_view": v_last, "instances_last_view": m_last, "traversed_last_view": m_proc,
-                   "conflict_window": CONFLICT_WINDOW, "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   "conflict_window": CONFLICT_WINDOW, "binning": args.binning, "parallelism": "replicas only" if world > 1 else "1 gpu",
                    "l2": "no flush: parameters + moments + instance buffers exceed the 126 MB L2 between uses"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches),

@@ -46,7 +46,7 @@ typedef enum {
 
 typedef struct odin_ctx odin_ctx; /* opaque: device ordinal, configuration, deferred-status word */
 
-/* Renderer constants.  Defaults (pass NULL to odin_create): 1/255, 0.99, 1e-4, 0.3, 3, 1.3, 16. */
+/* Renderer constants.  Defaults (pass NULL to odin_create): 1/255, 0.99, 1e-4, 0.3, 3, 1.3, 16, 0. */
 typedef struct {
   float alpha_min;     /* a contribution with alpha below this is skipped */
   float alpha_max;     /* alpha clamp */
@@ -55,6 +55,11 @@ typedef struct {
   float radius_sigmas; /* screen extent in standard deviations of the major axis */
   float jac_clamp;     /* t_x/t_z and t_y/t_z are clamped to +-jac_clamp * (half image / focal) inside the Jacobian */
   int tile;            /* tile edge in pixels; only 16 is supported */
+  int binning;         /* 0: tile rectangle of the radius (the method as published).  1: the rectangle is additionally cut
+                          to the axis-aligned extent of the region where opacity * exp(-q/2) can reach alpha_min
+                          (half extents sqrt(2 ln(opacity/alpha_min) * Sigma'_xx), ..._yy; a primitive whose opacity is
+                          below alpha_min gets no tile).  An optimised-pipeline variant in the sense of Sec. 5: the
+                          primitive ids, the image and the gradients are unchanged, the instance lists are shorter. */
 } odin_config;
 
 /* Pinhole camera (host struct).  w2c is the row-major 3x4 world-to-camera matrix [R|t]; camera axes are x right,

@@ -40,7 +40,12 @@ class OdinError(RuntimeError):
 
 class odin_config(C.Structure):
     _fields_ = [("alpha_min", C.c_float), ("alpha_max", C.c_float), ("t_min", C.c_float), ("dilation", C.c_float),
-                ("radius_sigmas", C.c_float), ("jac_clamp", C.c_float), ("tile", C.c_int)]
+                ("radius_sigmas", C.c_float), ("jac_clamp", C.c_float), ("tile", C.c_int), ("binning", C.c_int)]
+
+
+def default_config(binning: int = 0) -> odin_config:
+    """The renderer constants of the method; binning 1 selects the tight-extent tile rectangles."""
+    return odin_config(1.0 / 255.0, 0.99, 1e-4, 0.3, 3.0, 1.3, 16, int(binning))
 
 
 class odin_camera(C.Structure):

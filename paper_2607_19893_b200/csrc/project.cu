@@ -18,12 +18,24 @@ struct Footprint {
   uint32_t tiles;
 };
 
+// How the tile rectangle is chosen.  binning 0: the rectangle of the radius.  binning 1 (an optimised-pipeline variant
+// in the sense of Sec. 5: same primitive ids, same image): additionally cut to the axis-aligned extent of the region in
+// which alpha = opacity * exp(-q / 2) can reach alpha_min, q = d^T Sigma'^-1 d <= k = 2 ln(opacity / alpha_min), whose
+// half extents are sqrt(k Sigma'_xx), sqrt(k Sigma'_yy) (widened by 1e-4 relative + 1e-3 pixels).  No pixel outside it
+// passes the skip test of the blend kernels, so the instances that disappear never contributed.
+struct BinRule {
+  float dilation, radius_sigmas, alpha_min;
+  int binning;
+};
+
 // Conic, radius and tile rectangle of one primitive.  Plain IEEE arithmetic (this file is compiled without fused
 // multiply-add contraction): the integer results must not depend on which kernel evaluates them.
-__device__ __forceinline__ Footprint project_footprint(const CamParams& cam, float dilation, float radius_sigmas,
+__device__ __forceinline__ Footprint project_footprint(const CamParams& cam, const BinRule& rule,
                                                       const float* __restrict__ means,
                                                       const float* __restrict__ log_scales,
-                                                      const float4* __restrict__ quats, size_t p) {
+                                                      const float4* __restrict__ quats,
+                                                      const float* __restrict__ opacity_logit, size_t p) {
+  const float dilation = rule.dilation, radius_sigmas = rule.radius_sigmas;
   Footprint f;
   f.tiles = 0; f.u = f.v = f.depth = f.cA = f.cB = f.cC = 0.f; f.rad = f.x0 = f.y0 = f.x1 = f.y1 = 0;
   SplatGeom g;
@@ -44,6 +56,22 @@ __device__ __forceinline__ Footprint project_footprint(const CamParams& cam, flo
   f.x1 = (int)fminf(ftx, fmaxf(0.f, ceilf((f.u + radf) / 16.f)));
   f.y0 = (int)fminf(fty, fmaxf(0.f, floorf((f.v - radf) / 16.f)));
   f.y1 = (int)fminf(fty, fmaxf(0.f, ceilf((f.v + radf) / 16.f)));
+  if (rule.binning == 1) {
+    const float opac = 1.f / (1.f + expf(-opacity_logit[p]));
+    if (!(opac >= rule.alpha_min)) {
+      f.x1 = f.x0;  // never reaches alpha_min anywhere
+    } else {
+      const float k = 2.f * logf(opac / rule.alpha_min);
+      const float ex = sqrtf(k * g.a) * 1.0001f + 1e-3f, ey = sqrtf(k * g.c) * 1.0001f + 1e-3f;
+      // tiles that hold a pixel centre (i + 0.5) within [u - ex, u + ex]
+      const int tx0 = (int)fminf(ftx, fmaxf(0.f, floorf((f.u - ex - 0.5f) / 16.f)));
+      const int tx1 = (int)fminf(ftx, fmaxf(0.f, floorf((f.u + ex - 0.5f) / 16.f) + 1.f));
+      const int ty0 = (int)fminf(fty, fmaxf(0.f, floorf((f.v - ey - 0.5f) / 16.f)));
+      const int ty1 = (int)fminf(fty, fmaxf(0.f, floorf((f.v + ey - 0.5f) / 16.f) + 1.f));
+      f.x0 = max(f.x0, tx0); f.x1 = max(f.x0, min(f.x1, tx1));
+      f.y0 = max(f.y0, ty0); f.y1 = max(f.y0, min(f.y1, ty1));
+    }
+  }
   f.tiles = (uint32_t)(f.x1 - f.x0) * (uint32_t)(f.y1 - f.y0);
   f.rad = (int)fminf(radf, 2.0e9f);
   return f;
@@ -51,10 +79,11 @@ __device__ __forceinline__ Footprint project_footprint(const CamParams& cam, flo
 
 __global__ void __launch_bounds__(256)
 project_cull_kernel(const float* __restrict__ means, const float* __restrict__ log_scales, const float4* __restrict__ quats,
-                    uint32_t n, CamParams cam, float dilation, float radius_sigmas, uint32_t* __restrict__ tiles_touched) {
+                    const float* __restrict__ opacity_logit, uint32_t n, CamParams cam, BinRule rule,
+                    uint32_t* __restrict__ tiles_touched) {
   const uint32_t p = blockIdx.x * 256u + threadIdx.x;
   if (p >= n) return;
-  tiles_touched[p] = project_footprint(cam, dilation, radius_sigmas, means, log_scales, quats, p).tiles;
+  tiles_touched[p] = project_footprint(cam, rule, means, log_scales, quats, opacity_logit, p).tiles;
 }
 
 // packed look-back value: rows in the upper 28 bits, tile instances in the lower 34 bits
@@ -165,13 +194,13 @@ project_scan_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint
 template <int DEG>
 __global__ void __launch_bounds__(128)
 project_rows_kernel(const float* __restrict__ means, const float* __restrict__ log_scales, const float4* __restrict__ quats,
-                    const float* __restrict__ opacity_logit, const float* __restrict__ sh, CamParams cam, float dilation,
-                    float radius_sigmas, odin_projected out) {
+                    const float* __restrict__ opacity_logit, const float* __restrict__ sh, CamParams cam, BinRule rule,
+                    odin_projected out) {
   constexpr int K = (DEG + 1) * (DEG + 1);
   const uint32_t V = min(*out.num_rows, out.capacity);
   for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
     const size_t p = out.prim_id[r];
-    const Footprint f = project_footprint(cam, dilation, radius_sigmas, means, log_scales, quats, p);
+    const Footprint f = project_footprint(cam, rule, means, log_scales, quats, opacity_logit, p);
     reinterpret_cast<float2*>(out.xy)[r] = make_float2(f.u, f.v);
     out.depth[r] = f.depth;
     const float o = 1.f / (1.f + expf(-opacity_logit[p]));
@@ -245,10 +274,11 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + 256);
   const CamParams cp = odin_cam_params(cam, ctx->cfg);
   const float4* q4 = reinterpret_cast<const float4*>(scene->quats);
+  const BinRule rule = {ctx->cfg.dilation, ctx->cfg.radius_sigmas, ctx->cfg.alpha_min, ctx->cfg.binning};
   {
     OdinKernelScope ks(ctx, K_PROJECT, st);
-    project_cull_kernel<<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4, n, cp, ctx->cfg.dilation,
-                                                         ctx->cfg.radius_sigmas, out->tiles_touched);
+    project_cull_kernel<<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit, n, cp,
+                                                         rule, out->tiles_touched);
   }
   {
     OdinKernelScope ks(ctx, K_PROJECT_SCAN, st);
@@ -264,7 +294,7 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   OdinKernelScope ks(ctx, K_PROJECT_ROWS, st);
 #define LAUNCH(D)                                                                                                      \
   project_rows_kernel<D><<<grid, 128, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit, scene->sh, cp, \
-                                               ctx->cfg.dilation, ctx->cfg.radius_sigmas, *out)
+                                               rule, *out)
   switch (scene->sh_degree) {
     case 0: LAUNCH(0); break;
     case 1: LAUNCH(1); break;

@@ -88,10 +88,10 @@ class ViewTrainer:
     """Owns every device buffer of the view step and enqueues the seven calls (plus the loss) on one stream."""
 
     def __init__(self, scene, width: int, height: int, row_capacity: int, instance_capacity: int, mask_slots: int = 1,
-                 device: int = 0):
+                 device: int = 0, cfg: Optional[B.odin_config] = None):
         self.device = torch.device("cuda", device)
         torch.cuda.set_device(self.device)
-        self.ctx = B.odin_create(device)
+        self.ctx = B.odin_create(device, cfg)
         self.n, self.sh_degree = scene.means.shape[0], scene.sh_degree
         self.width, self.height = int(width), int(height)
         self.tx, self.ty = (width + 15) // 16, (height + 15) // 16

@@ -11,7 +11,7 @@ import gpu_util as G
 pytestmark = pytest.mark.gpu
 
 
-def run_chain(oracle32, w, steps, views, window=None, row_capacity=None, instance_capacity=None):
+def run_chain(oracle32, w, steps, views, window=None, row_capacity=None, instance_capacity=None, cfg=None):
     """Runs `steps` views on both sides from the same start.  Both sides see the same parameters at every step
     because the oracle is re-synchronised from the device after each comparison (so one fragile decision cannot
     cascade); every step is compared on its own."""
@@ -19,7 +19,7 @@ def run_chain(oracle32, w, steps, views, window=None, row_capacity=None, instanc
     n = scene.n
     cam0 = w.cameras[0]
     tr = G.trainer_for(scene, cam0, row_capacity=row_capacity, instance_capacity=instance_capacity,
-                       mask_slots=max(len(views), 1))
+                       mask_slots=max(len(views), 1), cfg=cfg)
     rng = np.random.default_rng(7)
     tr.keep_sorted_keys = True  # the sorted keys are compared below
     tr.track_active = True      # ... and the realized active set
@@ -152,6 +152,27 @@ def test_chain_unbounded_scene_scaled(oracle32):
 def test_chain_city_scaled(oracle32):
     w = wl.make_workload(5, n=300_000, n_cameras=4, resolution=(480, 270))
     run_chain(oracle32, w, steps=2, views=[0, 1])
+
+
+def test_chain_tight_extent_binning(oracle32):
+    """The whole step with binning = 1 against the oracle in the same mode (every check of run_chain), and against
+    the plain mode: fewer instances, the same image."""
+    from test_gpu_stages import tight_oracle
+
+    w = wl.make_workload(3, n=100_000, n_cameras=4, resolution=(400, 267))
+    run_chain(tight_oracle(), w, steps=3, views=[0, 1, 2], cfg=B.default_config(binning=1))
+    cam = w.cameras[1]
+    outs, m = [], []
+    for binning in (0, 1):
+        tr = G.trainer_for(w.scene, cam, cfg=B.default_config(binning=binning))
+        tr.target.copy_(torch.from_numpy(w.target(1)).to(tr.device))
+        tr.view_step(B.make_camera(cam), 1, w.lr, w.beta1, w.beta2, w.eps, update=False)
+        G.poll_ok(tr)
+        outs.append(tr.out.cpu().numpy())
+        m.append(int(tr.proj.num_instances.item()))
+        tr.close()
+    assert m[1] < 0.8 * m[0]
+    assert np.array_equal(outs[0], outs[1])  # the same pairs blend in the same order: bitwise the same image
 
 
 # ---------------------------------------------------------------------------------------------------------------

@@ -139,8 +139,8 @@ def test_sparse_adam_stage(oracle32, sh_degree, n, v):
 
 
 # ------------------------------------------------------------------------------------------------ projection
-def check_projection(oracle32, scene, cam, row_capacity=None):
-    tr = G.trainer_for(scene, cam, row_capacity=row_capacity)
+def check_projection(oracle32, scene, cam, row_capacity=None, cfg=None):
+    tr = G.trainer_for(scene, cam, row_capacity=row_capacity, cfg=cfg)
     ccam = B.make_camera(cam)
     po = oracle32.project(scene, cam)
     for _ in range(2):
@@ -201,6 +201,26 @@ def test_project_other_sh_degrees(oracle32, deg):
     k = (deg + 1) ** 2
     s2 = wl.Scene(deg, s.means, s.log_scales, s.quats, s.opacity_logit, np.ascontiguousarray(s.sh[:, :k]))
     check_projection(oracle32, s2, w.cameras[1])
+
+
+def tight_oracle():
+    import oracle
+    from oracle.oracle import DEFAULT_CFG
+    cfg = DEFAULT_CFG.copy()
+    cfg[7] = 1
+    return oracle.Oracle(np.float32, cfg=cfg)
+
+
+def test_project_tight_extent_binning(oracle32):
+    """binning = 1: the rectangles (and with them tiles_touched, rows, offsets) are those of the oracle's tight rule."""
+    ot = tight_oracle()
+    w = wl.make_workload(3, n=200_000, resolution=(800, 533))
+    v_tight = check_projection(ot, w.scene, w.cameras[2], cfg=B.default_config(binning=1))
+    po, pt = oracle32.project(w.scene, w.cameras[2]), ot.project(w.scene, w.cameras[2])
+    assert v_tight <= int((po.tiles_touched > 0).sum())
+    assert int(pt.tiles_touched.sum()) < 0.8 * int(po.tiles_touched.sum())
+    w2 = wl.make_workload(2, n=50_000)
+    check_projection(ot, w2.scene, w2.cameras[6], cfg=B.default_config(binning=1))
 
 
 def test_project_row_capacity_overflow(oracle32):
