@@ -30,6 +30,13 @@ struct BinRule {
 
 // Conic, radius and tile rectangle of one primitive.  Plain IEEE arithmetic (this file is compiled without fused
 // multiply-add contraction): the integer results must not depend on which kernel evaluates them.
+// PRETEST (the counting kernel, where most primitives end up with no tile): a primitive in front of the camera whose
+// centre lies farther from the image than a bound on its radius cannot touch a tile, and the bound needs neither the
+// quaternion nor the covariance.  With T = J W (W a rotation) the projected covariance satisfies
+// lambda_max(T Sigma T^T) <= |J|_F^2 s_max^2, |J|_F^2 <= (fx/z)^2 (1 + limx^2) + (fy/z)^2 (1 + limy^2), and the radius
+// formula adds at most sqrt(0.1) to the larger eigenvalue; the bound is then widened by 1 % + 2 pixels, far beyond
+// rounding.  Only primitives for which the exact rectangle is certainly empty leave here, so the result is unchanged.
+template <bool PRETEST = false>
 __device__ __forceinline__ Footprint project_footprint(const CamParams& cam, const BinRule& rule,
                                                       const float* __restrict__ means,
                                                       const float* __restrict__ log_scales,
@@ -42,6 +49,15 @@ __device__ __forceinline__ Footprint project_footprint(const CamParams& cam, con
   odin_camera_space(cam, means[3 * p], means[3 * p + 1], means[3 * p + 2], g.t);
   if (!(g.t[2] > cam.znear && g.t[2] < cam.zfar)) return f;
   const float ls[3] = {log_scales[3 * p], log_scales[3 * p + 1], log_scales[3 * p + 2]};
+  if (PRETEST) {
+    const float iz = 1.f / g.t[2];
+    const float uc = cam.fx * g.t[0] * iz + cam.cx, vc = cam.fy * g.t[1] * iz + cam.cy;
+    const float smax = expf(fmaxf(ls[0], fmaxf(ls[1], ls[2])));
+    const float jx = cam.fx * iz, jy = cam.fy * iz;
+    const float jn2 = jx * jx * (1.f + cam.limx * cam.limx) + jy * jy * (1.f + cam.limy * cam.limy);
+    const float rb = radius_sigmas * sqrtf(jn2 * smax * smax + dilation + 0.32f) * 1.01f + 2.f;
+    if (uc + rb < 0.f || uc - rb > 16.f * (float)cam.TX || vc + rb < 0.f || vc - rb > 16.f * (float)cam.TY) return f;
+  }
   odin_splat_geometry(cam, dilation, ls, quats[p], g);
   if (!(g.det > 0.f)) return f;
   f.cA = g.c / g.det; f.cB = -g.b / g.det; f.cC = g.a / g.det;
@@ -83,7 +99,7 @@ project_cull_kernel(const float* __restrict__ means, const float* __restrict__ l
                     uint32_t* __restrict__ tiles_touched) {
   const uint32_t p = blockIdx.x * 256u + threadIdx.x;
   if (p >= n) return;
-  tiles_touched[p] = project_footprint(cam, rule, means, log_scales, quats, opacity_logit, p).tiles;
+  tiles_touched[p] = project_footprint<true>(cam, rule, means, log_scales, quats, opacity_logit, p).tiles;
 }
 
 // packed look-back value: rows in the upper 28 bits, tile instances in the lower 34 bits

@@ -7,8 +7,12 @@ namespace {
 constexpr int TS_THREADS = 256;
 constexpr int TS_ITEMS = TOUCHED_TILE / TS_THREADS;  // 8 words of 32 primitives per warp
 
-// Each warp owns 256 consecutive primitives = 8 mask words; load j of lane l is primitive warp_base + 32 j + l, so one
-// ballot is one mask word and ranks inside the warp follow the primitive order.
+// A block takes `scan_rounds` x 2048 consecutive primitives by ticket; each of its eight warps owns a contiguous eighth
+// of them.  Load q of lane l is primitive span_base + 32 q + l, so one ballot is one mask word and ranks inside the
+// warp follow the primitive order.  The ballots are kept (word q in lane q % 32), so the list is written after the
+// look-back without reading the counts a second time.
+constexpr int TS_MAX_ROUNDS = 8;
+
 __global__ void __launch_bounds__(TS_THREADS)
 touched_set_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint32_t* __restrict__ mask,
                    uint32_t* __restrict__ idx, uint32_t idx_capacity, uint32_t* __restrict__ count, uint32_t* ticket,
@@ -21,72 +25,48 @@ touched_set_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint3
   __syncthreads();
   const uint32_t tile = s_tile;
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t chunk_base = tile * scan_chunk;
-  // pass A: how many touched primitives does this chunk hold (one look-back per scan_chunk primitives keeps the
-  // chain of dependent tiles short; the second pass re-reads the chunk from cache)
-  uint32_t mine = 0;
-#pragma unroll
-  for (int rnd = 0; rnd < scan_rounds; ++rnd) {
-    const uint32_t warp_base = chunk_base + rnd * TOUCHED_TILE + warp * (32 * TS_ITEMS);
-#pragma unroll
-    for (int j = 0; j < TS_ITEMS; ++j) {
-      const uint32_t p = warp_base + 32 * j + lane;
-      mine += (p < n && tiles_touched[p] > 0) ? 1u : 0u;
-    }
+  const int words = scan_rounds * TS_ITEMS;  // mask words (ballots) per warp: 8 .. 64
+  const uint32_t span_base = tile * scan_chunk + warp * (uint32_t)words * 32u;
+  const uint32_t n_words = (n + 31) / 32;
+  // pass A: ballots of the warp's span; word q stays in lane q % 32 of keep[q / 32]
+  uint32_t keep[TS_MAX_ROUNDS * TS_ITEMS / 32] = {0u, 0u};
+  uint32_t warp_count = 0;
+#pragma unroll 8
+  for (int q = 0; q < words; ++q) {
+    const uint32_t p = span_base + 32u * (uint32_t)q + lane;
+    const uint32_t bal = __ballot_sync(0xffffffffu, p < n && tiles_touched[p] > 0);
+    warp_count += __popc(bal);
+    if (lane == (unsigned)(q & 31)) keep[q >> 5] = bal;
+  }
+  // the mask words of the span: 32 consecutive words per store
+  for (int h = 0; h * 32 < words; ++h) {
+    const uint32_t word = span_base / 32 + h * 32 + lane;
+    if ((int)(h * 32 + lane) < words && word < n_words) mask[word] = keep[h];
   }
   uint32_t chunk_total;
-  odin_block_exclusive_sum(mine, s_warp, &chunk_total);
+  const uint32_t scan = odin_block_exclusive_sum(lane == 0 ? warp_count : 0u, s_warp, &chunk_total);
+  const uint32_t warp_off = __shfl_sync(0xffffffffu, scan, 0);
   if (threadIdx.x < 32) {
     const uint64_t ex = odin_lookback_u64(state, tile, (uint64_t)chunk_total, status);
     if (threadIdx.x == 0) s_base = ex;
   }
   __syncthreads();
-  uint64_t base = s_base;
+  const uint64_t base = s_base;
   if (tile == (n + scan_chunk - 1) / scan_chunk - 1 && threadIdx.x == 0) {
     const uint64_t v = base + chunk_total;
     *count = (uint32_t)(v < idx_capacity ? v : idx_capacity);
     if (v > idx_capacity) odin_set_error(status, ODIN_ERR_CAPACITY);
   }
-  // pass B: masks and the ascending list, 2048 primitives per round
-  for (int rnd = 0; rnd < scan_rounds; ++rnd) {
-    const uint32_t warp_base = chunk_base + rnd * TOUCHED_TILE + warp * (32 * TS_ITEMS);
-    if (chunk_base + rnd * TOUCHED_TILE >= n) break;  // uniform over the block
-    uint32_t t[TS_ITEMS];
-#pragma unroll
-    for (int j = 0; j < TS_ITEMS; ++j) {
-      const uint32_t p = warp_base + 32 * j + lane;
-      t[j] = (p < n) ? tiles_touched[p] : 0u;
+  // pass B: the ascending list from the kept ballots
+  uint64_t pos = base + warp_off;
+  const uint32_t lt = (1u << lane) - 1u;
+  for (int q = 0; q < words; ++q) {
+    const uint32_t bal = __shfl_sync(0xffffffffu, keep[q >> 5], q & 31);
+    if (bal >> lane & 1u) {
+      const uint64_t dst = pos + __popc(bal & lt);
+      if (dst < idx_capacity) idx[dst] = span_base + 32u * (uint32_t)q + lane;
     }
-    uint32_t ballots[TS_ITEMS];
-    uint32_t warp_count = 0;
-#pragma unroll
-    for (int j = 0; j < TS_ITEMS; ++j) {
-      ballots[j] = __ballot_sync(0xffffffffu, t[j] > 0);
-      warp_count += __popc(ballots[j]);
-    }
-    // mask words (lane j writes word j of the warp)
-    if (lane < TS_ITEMS) {
-      uint32_t w = 0;
-#pragma unroll
-      for (int j = 0; j < TS_ITEMS; ++j)
-        if (lane == (unsigned)j) w = ballots[j];
-      const uint32_t word = warp_base / 32 + lane;
-      if (word < (n + 31) / 32) mask[word] = w;
-    }
-    // exclusive offsets of the warps inside the round
-    uint32_t total;
-    const uint32_t scan = odin_block_exclusive_sum(lane == 0 ? warp_count : 0u, s_warp, &total);
-    const uint32_t warp_off = __shfl_sync(0xffffffffu, scan, 0);
-    uint64_t pos = base + warp_off;
-#pragma unroll
-    for (int j = 0; j < TS_ITEMS; ++j) {
-      if (t[j] > 0) {
-        const uint64_t dst = pos + __popc(ballots[j] & ((1u << lane) - 1u));
-        if (dst < idx_capacity) idx[dst] = warp_base + 32 * j + lane;
-      }
-      pos += __popc(ballots[j]);
-    }
-    base += total;
+    pos += __popc(bal);
   }
 }
 
