@@ -171,6 +171,8 @@ project_scan_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint
     uint64_t run = 0;
 #pragma unroll
     for (int j = 0; j < SCAN_ITEMS; ++j) {
+      ex[j] = run;
+      if (__ballot_sync(0xffffffffu, t[j] != 0) == 0) continue;  // 32 culled primitives in a row: nothing to scan
       const uint64_t v = t[j] ? ((1ull << PACK_SHIFT) | (uint64_t)t[j]) : 0ull;
       uint64_t inc = v;
 #pragma unroll
