@@ -6,8 +6,9 @@ sparse Adam -> conflict counts) on seeded synthetic scenes.
 
 One JSON line on stdout (rank 0).  `value` = views/s with every input resident in HBM; `e2e` = the same step driven
 with HOST inputs (the view's target image copied from pinned memory, loss / V / conflict counts read back) inside the
-timed region.  `roofline` describes the kernel with the largest share of the step, timed with CUDA events on the launch
-stream inside the timed region; `step_hbm` gives the whole step's algorithmic bytes against the measured HBM peak.
+timed region (the copy of the next view's target overlaps the current view's kernels).  `roofline` describes the stage
+with the largest share of the step, timed with CUDA events around every launch in a second pass over the same steps;
+`step_hbm` gives the whole step's algorithmic bytes against the measured HBM peak.
 The path does not shard (one view step is one GPU's work): with --gpus N every rank runs an independent replica.
 """
 from __future__ import annotations
@@ -383,26 +384,28 @@ def main():
             raise SystemExit(f"scope calls failed: {B.status_string(st)}")
 
     # ---- end-to-end run: host target in, loss / V / counts out, every step --------------------------------------
-    h_loss = torch.zeros(1, dtype=torch.float32).pin_memory()
-    h_count = torch.zeros(1, dtype=torch.int32).pin_memory()
-    h_counts = torch.zeros(max(CONFLICT_WINDOW, 1), dtype=torch.int64).pin_memory()
-    staging = torch.empty_like(bank[0])
+    # The public call for host-resident targets (engine.ViewTrainer.train_from_host): two staging buffers, the copy of
+    # the next view's target overlaps the current view's kernels, and the host waits for the results of the previous
+    # view while the current one runs.  Every step still has its own host-to-device copy and its own device-to-host
+    # read inside the timed region.
+    results = []
+    tr.prepare_host_io(d_counts.numel())  # one-time allocations stay outside the timed region
     barrier()
     t0 = time.perf_counter()
-    for s in range(args.warmup, total_steps):
-        staging.copy_(host_targets[view_of(s)], non_blocking=True)
-        step(s, staging)
-        h_loss.copy_(tr.loss, non_blocking=True)
-        h_count.copy_(tr.count, non_blocking=True)
-        h_counts.copy_(d_counts, non_blocking=True)
-        torch.cuda.synchronize()
+    tr.train_from_host(range(args.warmup, total_steps), cam_of=lambda s: cams[view_of(s)],
+                       host_target_of=lambda s: host_targets[view_of(s)], lr=w.lr, beta1=w.beta1, beta2=w.beta2,
+                       eps=w.eps, slot_of=lambda s: s % MASK_SLOTS,
+                       pairs_of=lambda s: (d_pairs[s], len(pair_lists[s])), d_counts=d_counts,
+                       on_result=lambda s, loss, touched, counts: results.append((s, loss, touched)))
+    torch.cuda.synchronize()
     barrier()
     e2e_s = time.perf_counter() - t0
     e2e_value = whole_job_value(args.steps, world, max_over_ranks(e2e_s, world, dev))
     st = tr.poll()
     if st != B.ODIN_OK:
         raise SystemExit(f"end-to-end run failed: {B.status_string(st)}")
-    h2d = int(staging.numel() * 4)
+    assert len(results) == args.steps and all(np.isfinite(r[1]) and r[2] > 0 for r in results)
+    h2d = int(bank[0].numel() * 4)
     d2h = int(4 + 4 + 8 * max(CONFLICT_WINDOW, 1))
 
     clocks = sampler.stop(t_begin, t_end) if sampler else None

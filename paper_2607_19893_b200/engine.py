@@ -196,5 +196,78 @@ class ViewTrainer:
         if n_pairs:
             self.conflict_count(d_pairs, n_pairs, d_counts, stream)
 
+    def prepare_host_io(self, n_counts: int = 0):
+        """Staging buffers, pinned result slots, copy stream and events of train_from_host (allocated once)."""
+        io = getattr(self, "_host_io", None)
+        if io is None or io["n_counts"] < n_counts:
+            io = {
+                "n_counts": n_counts,
+                "copy_stream": torch.cuda.Stream(device=self.device),
+                "staging": [torch.empty_like(self.target) for _ in range(2)],
+                "h_loss": [torch.zeros(1, dtype=torch.float32).pin_memory() for _ in range(2)],
+                "h_count": [torch.zeros(1, dtype=torch.int32).pin_memory() for _ in range(2)],
+                "h_counts": [torch.zeros(max(n_counts, 1), dtype=torch.int64).pin_memory() for _ in range(2)],
+                "copied": [torch.cuda.Event() for _ in range(2)],
+                "consumed": [torch.cuda.Event() for _ in range(2)],
+                "done": [torch.cuda.Event() for _ in range(2)],
+            }
+            self._host_io = io
+        return io
+
+    def train_from_host(self, steps, cam_of, host_target_of, lr, beta1: float, beta2: float, eps: float,
+                        slot_of=lambda s: 0, pairs_of=None, d_counts=None, on_result=None) -> None:
+        """Training views whose targets live in pinned HOST memory.  For every step s in `steps`: the target
+        host_target_of(s) is copied to the device, the view cam_of(s) is stepped, and the loss, the number of touched
+        primitives and (if pairs_of is given) the conflict counts are read back into pinned memory and handed to
+        on_result(s, loss, touched, counts).  Two staging buffers and a copy stream: the copy of the next target
+        overlaps the current view's kernels, and the host waits for the results of the previous view while the current
+        one runs.  Marshalling only: every kernel is the library's."""
+        steps = list(steps)
+        n_counts = 0 if d_counts is None else d_counts.numel()
+        io = self.prepare_host_io(n_counts)
+        if not steps:
+            return
+        stream = torch.cuda.current_stream()
+        copy_stream, staging = io["copy_stream"], io["staging"]
+        h_loss, h_count, h_counts = io["h_loss"], io["h_count"], io["h_counts"]
+        copied, consumed, done = io["copied"], io["consumed"], io["done"]
+        saved_target = self.target
+
+        def enqueue_copy(i):
+            k = i & 1
+            with torch.cuda.stream(copy_stream):
+                copy_stream.wait_event(consumed[k])  # the step that read this buffer last has finished
+                staging[k].copy_(host_target_of(steps[i]), non_blocking=True)
+                copied[k].record(copy_stream)
+
+        def deliver(i):
+            k = i & 1
+            done[k].synchronize()
+            if on_result is not None:
+                on_result(steps[i], float(h_loss[k][0]), int(h_count[k][0]), h_counts[k][:n_counts].clone())
+
+        for k in range(2):
+            consumed[k].record(stream)
+        enqueue_copy(0)
+        for i, s in enumerate(steps):
+            k = i & 1
+            if i + 1 < len(steps):
+                enqueue_copy(i + 1)
+            stream.wait_event(copied[k])
+            self.target = staging[k]
+            pairs = pairs_of(s) if pairs_of is not None else None
+            self.view_step(cam_of(s), s + 1, lr, beta1, beta2, eps, slot=slot_of(s), d_pairs=pairs[0] if pairs else None,
+                           n_pairs=pairs[1] if pairs else 0, d_counts=d_counts, stream=stream)
+            consumed[k].record(stream)
+            h_loss[k].copy_(self.loss, non_blocking=True)
+            h_count[k].copy_(self.count, non_blocking=True)
+            if n_counts:
+                h_counts[k][:n_counts].copy_(d_counts, non_blocking=True)
+            done[k].record(stream)
+            if i > 0:
+                deliver(i - 1)
+        deliver(len(steps) - 1)
+        self.target = saved_target
+
     def poll(self, stream=None) -> int:
         return B.odin_poll(self.ctx, stream)

@@ -154,6 +154,39 @@ def test_chain_city_scaled(oracle32):
     run_chain(oracle32, w, steps=2, views=[0, 1])
 
 
+def test_train_from_host_equals_the_plain_loop():
+    """The double-buffered host-target loop is marshalling only: the same kernels on the same inputs, so losses, counts
+    and the trained parameters are bitwise those of the plain loop (atomics aside: compared with a tolerance)."""
+    w = wl.make_workload(2, n=30_000)
+    steps = list(range(6))
+    cams = [B.make_camera(c) for c in w.cameras]
+    host_targets = [torch.from_numpy(w.target(v)).pin_memory() for v in range(len(w.cameras))]
+    a = G.trainer_for(w.scene, w.cameras[0], mask_slots=3)
+    b = G.trainer_for(w.scene, w.cameras[0], mask_slots=3)
+    pairs = torch.tensor([[0, 1], [1, 2]], dtype=torch.int32, device=a.device)
+    counts_a = torch.zeros(2, dtype=torch.int64, device=a.device)
+    counts_b = torch.zeros(2, dtype=torch.int64, device=b.device)
+    got = []
+    a.train_from_host(steps, cam_of=lambda s: cams[s % 8], host_target_of=lambda s: host_targets[s % 8], lr=w.lr,
+                      beta1=w.beta1, beta2=w.beta2, eps=w.eps, slot_of=lambda s: s % 3,
+                      pairs_of=lambda s: (pairs, 2), d_counts=counts_a,
+                      on_result=lambda s, loss, touched, counts: got.append((s, loss, touched, counts.tolist())))
+    G.poll_ok(a)
+    want = []
+    for s in steps:
+        b.target.copy_(host_targets[s % 8].to(b.device))
+        b.view_step(cams[s % 8], s + 1, w.lr, w.beta1, w.beta2, w.eps, slot=s % 3, d_pairs=pairs, n_pairs=2,
+                    d_counts=counts_b)
+        G.poll_ok(b)
+        want.append((s, float(b.loss.item()), int(b.count.item()), counts_b.cpu().tolist()))
+    assert [g[0] for g in got] == steps
+    for g, x in zip(got, want):
+        assert g[2] == x[2] and g[3] == x[3] and abs(g[1] - x[1]) < 1e-6
+    for ta, tb in zip(a.params.tensors(), b.params.tensors()):
+        assert torch.allclose(ta, tb, rtol=1e-4, atol=1e-6)
+    a.close(); b.close()
+
+
 def test_chain_tight_extent_binning(oracle32):
     """The whole step with binning = 1 against the oracle in the same mode (every check of run_chain), and against
     the plain mode: fewer instances, the same image."""
