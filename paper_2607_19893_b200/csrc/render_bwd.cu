@@ -341,6 +341,24 @@ render_bwd_project_kernel(const float* __restrict__ means, const float* __restri
     const float* gg = g2d + (size_t)r * 9;
     const float gu = gg[0], gv = gg[1], gA = gg[2], gB = gg[3], gC = gg[4], go = gg[5];
     const float grgb[3] = {gg[6], gg[7], gg[8]};
+    // The chain rule is linear in these nine words.  Most touched rows never blend into a pixel (they are occluded)
+    // and arrive with all nine at zero: their gradient row is zero and needs neither the scene nor any arithmetic.
+    if (gu == 0.f && gv == 0.f && gA == 0.f && gB == 0.f && gC == 0.f && go == 0.f && grgb[0] == 0.f && grgb[1] == 0.f &&
+        grgb[2] == 0.f) {
+#pragma unroll
+      for (int j = 0; j < 3; ++j) { g_means[3 * (size_t)r + j] = 0.f; g_ls[3 * (size_t)r + j] = 0.f; }
+      g_quats[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+      g_opac[r] = 0.f;
+      float* out = g_sh + (size_t)r * (3 * K);
+      if ((3 * K) % 4 == 0) {
+#pragma unroll
+        for (int i = 0; i < 3 * K / 4; ++i) reinterpret_cast<float4*>(out)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 3 * K; ++i) out[i] = 0.f;
+      }
+      continue;
+    }
     const float mx = means[3 * p], my = means[3 * p + 1], mz = means[3 * p + 2];
     SplatGeom g;
     odin_camera_space(cam, mx, my, mz, g.t);
