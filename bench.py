@@ -479,13 +479,17 @@ def main():
         import oracle
 
         o32 = oracle.get(np.float32)
-        n_sample_views = 1 if n >= 1_000_000 else (2 if n >= 100_000 else 8)
         p = scene.copy()
         m_, v_ = p.zeros_like(), p.zeros_like()
         t0 = time.perf_counter()
-        for s in range(n_sample_views):
+        n_sample_views = 0
+        while n_sample_views < 16:  # whole views until about ten seconds of CPU work are on the clock
+            s = n_sample_views
             o32.view_step(p, m_, v_, w.cameras[s % len(w.cameras)], w.target(s % len(w.cameras)), w.lr, w.beta1, w.beta2,
                           w.eps, s + 1)
+            n_sample_views += 1
+            if time.perf_counter() - t0 > 10.0:
+                break
         dt = time.perf_counter() - t0
         line["cpu_baseline"] = {"value": n_sample_views / dt, "unit": UNIT, "cores": o32.num_threads(), "kind": "oracle",
                                 "sample": f"{n_sample_views} full view step(s) of the same workload"}
