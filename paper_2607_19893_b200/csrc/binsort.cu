@@ -70,7 +70,7 @@ constexpr int OS_ROW_ITEMS = ROW_SORT_TILE / OS_THREADS;  // 4 in the passes ove
 constexpr int OS_DPT = SORT_RADIX / OS_THREADS;   // digits owned by a thread
 constexpr int OS_INST_WINDOW = 2;                 // predecessors fetched per look-back step and digit (instances)
 constexpr int OS_ROW_WINDOW = 8;                  // ... and in the passes over the rows
-constexpr int OS_BLOCKS = 4;                      // resident blocks per SM
+constexpr int OS_BLOCKS = 4;                    // resident blocks per SM
 constexpr uint32_t OS_FLAG_AGG = 1u << 30, OS_FLAG_INC = 2u << 30, OS_VALUE = (1u << 30) - 1;
 constexpr size_t os_smem_bytes(int items) {
   return (size_t)items * OS_THREADS * 8 + (size_t)OS_WARPS * SORT_RADIX * 4 + 2 * SORT_RADIX * 4 + 16;

@@ -280,6 +280,21 @@ def test_bin_sort_many_tiles_six_passes(oracle32):
     assert m > 500_000
 
 
+def test_bin_sort_image_of_73728_tiles(oracle32):
+    """8192 x 2304 pixels = 512 x 144 tiles: three passes over the tile-id digits, and more tiles than the
+    shared-memory staging of the per-tile counts holds (the counts then go straight to global memory)."""
+    w = wl.make_workload(3, n=20_000, resolution=(8192, 2304))
+    cam = w.cameras[5]
+    assert ((cam.width + 15) // 16) * ((cam.height + 15) // 16) == 73728
+    m = check_bin_sort(oracle32, w.scene, cam)
+    assert m > 1_000_000
+
+
+def test_bin_sort_image_of_one_tile(oracle32):
+    w = wl.make_workload(1, resolution=(16, 16))
+    check_bin_sort(oracle32, w.scene, w.cameras[0])
+
+
 def test_bin_sort_equal_depth_ties(oracle32):
     # many identical splats: identical keys, order decided by the row index alone
     w = wl.make_workload(1)
