@@ -42,9 +42,9 @@ FLOPS_PER_PAIR = {"render_fwd": 25.0, "render_bwd_blend": 75.0}
 # DRAM traffic (read + write, bytes per view) of the kernels of a stage, from the ncu capture of one view step that
 # profiles/view_step_kernels_cfg3.txt summarises; only that workload was captured
 NCU_TRAFFIC = {"cfg3_1m_sh3_1600x1066": {
-    "render_bwd_blend": 45.2e6 + 34.9e6, "render_fwd": 9.7e6 + 8.4e6, "onesweep_pass": 119.8e6 + 94.5e6,
-    "adam": 425.6e6 + 195.8e6, "emit_instances": 31.6e6 + 3.9e6, "row_sort": 1.3e6 + 4 * 2.7e6,
-    "project": 40.0e6 + 4.0e6 + 128.7e6, "render_bwd_project": 167.6e6, "touched_set": 4.0e6, "l1_loss": 41.1e6}}
+    "render_bwd_blend": 45.3e6 + 34.9e6, "render_fwd": 9.7e6 + 8.4e6, "onesweep_pass": 123.0e6 + 95.1e6,
+    "adam": 425.4e6 + 196.6e6, "emit_instances": 32.1e6 + 3.9e6, "row_sort": 1.3e6 + 1.5e6 + 2.7e6 + 2.7e6 + 2.6e6,
+    "project": 39.4e6 + 4.0e6 + 128.5e6, "render_bwd_project": 40.4e6, "touched_set": 4.0e6, "l1_loss": 41.3e6}}
 
 
 def measured_peaks():

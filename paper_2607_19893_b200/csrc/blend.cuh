@@ -65,9 +65,3 @@ __device__ __forceinline__ float4 blend_extent(float u, float v, float A, float 
   const float ey = sqrtf(k * A / det) * 1.0001f + 1e-3f;
   return make_float4(u - ex, u + ex, v - ey, v + ey);
 }
-
-// Slots (pairs of pixel rows 2 s, 2 s + 1 of the tile whose first row is y0) that the box [y_lo, y_hi] can reach.
-__device__ __forceinline__ void blend_slot_range(float y_lo, float y_hi, float y0, int* s_lo, int* s_hi) {
-  *s_lo = max(0, (int)ceilf((y_lo - y0 - 1.5f) * 0.5f));
-  *s_hi = min(BLEND_SLOTS - 1, (int)floorf((y_hi - y0 - 0.5f) * 0.5f));
-}
