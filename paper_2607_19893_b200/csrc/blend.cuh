@@ -48,20 +48,33 @@ __device__ __forceinline__ float blend_power(float h0, float h1, float h2, float
 // additional test power <= 0 can never meet.
 __device__ __forceinline__ float blend_power_cut(float alpha_min, float opacity) { return logf(alpha_min / opacity); }
 
-// Box (x_lo, x_hi, y_lo, y_hi) in pixel-centre coordinates outside of which a row cannot pass the skip test.  The set
-// power >= cut is the ellipse A dx^2 + 2 B dx dy + C dy^2 <= k with k = -2 cut; its half extents are
-// sqrt(k C / det) in x and sqrt(k A / det) in y, det = A C - B^2.  The box is widened by 1e-4 relative + 1e-3 pixels,
-// far more than the rounding of the per-pixel test, so skipping by it never changes a result.  Computed once per row
-// by the lane that stages it; all lanes then take warp-uniform decisions from it (skip the row, restrict the slots).
-__device__ __forceinline__ float4 blend_extent(float u, float v, float A, float B, float C, float cut) {
-  const float k = fmaxf(-2.f * cut, 0.f);
-  const float det = A * C - B * B;
-  if (!(det > 0.f) || !(k < 3.0e38f)) {  // degenerate conic: no bound; cut = +inf (opacity 0) also lands here
-    const float big = 3.0e38f;
-    return (cut > 0.f) ? make_float4(big, -big, big, -big) : make_float4(-big, big, -big, big);
+// Can the row pass the skip test at any pixel of the tile whose first pixel centre is (x_lo, y_lo)?  The set
+// power >= cut is the ellipse q(dx, dy) = A dx^2 + 2 B dx dy + C dy^2 <= k, k = -2 cut, around the row's centre (u, v);
+// the pixel centres of the tile lie in the rectangle [x_lo, x_lo + 15] x [y_lo, y_lo + 15].  q is convex, so its
+// minimum over the rectangle is 0 if the centre lies inside and otherwise sits on one of the four edges, where it is
+// the clamped one-dimensional minimiser.  The bound is widened by 1e-4 relative + 1e-3 + 2e-6 of the largest term any
+// pixel of the tile can see (the rounding of this evaluation and of the per-pixel exponent is a few ulp of that term),
+// so a row it rejects fails the per-pixel test everywhere in the tile and skipping it never changes a result.
+// Evaluated once per (tile, row) by the thread that stages the row; anything that is not a proper ellipse is kept.
+__device__ __forceinline__ bool blend_reaches_tile(float u, float v, float A, float B, float C, float cut, float x_lo,
+                                                   float y_lo) {
+  if (!(cut <= 0.f)) return false;  // opacity below alpha_min (cut > 0), zero (+inf) or not a number: nothing passes
+  const float dxl = x_lo - u, dxh = dxl + 15.f, dyl = y_lo - v, dyh = dyl + 15.f;
+  if (dxl <= 0.f && dxh >= 0.f && dyl <= 0.f && dyh >= 0.f) return true;
+  if (!(A * C - B * B > 0.f) || !(A > 1e-30f) || !(C > 1e-30f) || !(A < 1e30f) || !(C < 1e30f)) return true;
+  const float iA = __fdividef(1.f, A), iC = __fdividef(1.f, C);
+  float qmin;
+  {
+    const float t0 = fminf(fmaxf(-B * dxl * iC, dyl), dyh), t1 = fminf(fmaxf(-B * dxh * iC, dyl), dyh);
+    const float q0 = fmaf(t0, fmaf(C, t0, 2.f * B * dxl), A * dxl * dxl);
+    const float q1 = fmaf(t1, fmaf(C, t1, 2.f * B * dxh), A * dxh * dxh);
+    const float s0 = fminf(fmaxf(-B * dyl * iA, dxl), dxh), s1 = fminf(fmaxf(-B * dyh * iA, dxl), dxh);
+    const float q2 = fmaf(s0, fmaf(A, s0, 2.f * B * dyl), C * dyl * dyl);
+    const float q3 = fmaf(s1, fmaf(A, s1, 2.f * B * dyh), C * dyh * dyh);
+    qmin = fminf(fminf(q0, q1), fminf(q2, q3));
   }
-  if (cut > 0.f) return make_float4(3.0e38f, -3.0e38f, 3.0e38f, -3.0e38f);  // opacity below alpha_min: never passes
-  const float ex = sqrtf(k * C / det) * 1.0001f + 1e-3f;
-  const float ey = sqrtf(k * A / det) * 1.0001f + 1e-3f;
-  return make_float4(u - ex, u + ex, v - ey, v + ey);
+  const float mx = fmaxf(fabsf(dxl), fabsf(dxh)), my = fmaxf(fabsf(dyl), fabsf(dyh));
+  const float big = A * mx * mx + 2.f * fabsf(B) * mx * my + C * my * my;
+  const float bound = fmaf(-2.f * cut, 1.0001f, 1e-3f + 2e-6f * big);
+  return !(qmin > bound);
 }

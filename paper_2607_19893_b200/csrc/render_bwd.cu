@@ -49,10 +49,13 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
   __shared__ BlendRow s_rowdata[BB];
   __shared__ float2 s_blue[BB];  // blue, power threshold
   __shared__ uint32_t s_rowid[BB];
+  __shared__ uint32_t s_ord[BB];
+  __shared__ uint32_t s_wcnt[BB / 32];
   __shared__ float s_acc[BB * 9];
   __shared__ uint32_t s_max;
   const int tile = blockIdx.x;
   const int tx = tile % TX, ty = tile / TX;
+  const float tile_x0 = (float)(tx * 16) + 0.5f, tile_y0 = (float)(ty * 16) + 0.5f;
   const int lx = threadIdx.x & 15, ly = threadIdx.x >> 4;
   const int px = tx * 16 + lx, py = ty * 16 + ly;
   const bool inside = px < W && py < H;
@@ -87,17 +90,35 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
   const int nb = (int)((span + BB - 1) / BB);
   for (int bi = nb - 1; bi >= 0; --bi) {
     const uint32_t b = BLEND_HEAD + (uint32_t)bi * BB;
-    const int cnt = (int)min((uint32_t)BB, total - b);
-    __syncthreads();
-    if ((int)threadIdx.x < cnt) {
-      const uint32_t r = vals[start + b + threadIdx.x];
+    const int staged = (int)min((uint32_t)BB, total - b);
+    // stage up to 256 entries and keep, in list order, only the rows whose ellipse reaches the tile
+    BlendRow row;
+    float2 bp = make_float2(0.f, 0.f);
+    uint32_t r = 0;
+    bool reach = false;
+    if ((int)threadIdx.x < staged) {
+      r = vals[start + b + threadIdx.x];
       const float2 c = xy[r];
-      BlendRow row;
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
       row.q1 = conic_o[r];
-      s_rowdata[threadIdx.x] = row;
-      s_blue[threadIdx.x] = make_float2(rgb[3 * (size_t)r + 2], blend_power_cut(alpha_min, row.q1.w));
-      s_rowid[threadIdx.x] = r;
+      bp = make_float2(rgb[3 * (size_t)r + 2], blend_power_cut(alpha_min, row.q1.w));
+      reach = blend_reaches_tile(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, bp.y, tile_x0, tile_y0);
+    }
+    const uint32_t wm = __ballot_sync(0xffffffffu, reach);
+    if (lane == 0) s_wcnt[threadIdx.x >> 5] = __popc(wm);
+    __syncthreads();  // also: the flush of the previous batch is complete
+    int cnt = 0, pos = __popc(wm & ((1u << lane) - 1u));
+#pragma unroll
+    for (int w = 0; w < BB / 32; ++w) {
+      const int c = (int)s_wcnt[w];
+      if (w < (int)(threadIdx.x >> 5)) pos += c;
+      cnt += c;
+    }
+    if (reach) {
+      s_rowdata[pos] = row;
+      s_blue[pos] = bp;
+      s_rowid[pos] = r;
+      s_ord[pos] = b + threadIdx.x;  // 0-based position in the tile's list
     }
     __syncthreads();
     for (int j4 = cnt - 1; j4 >= 0; j4 -= 4) {
@@ -111,7 +132,7 @@ render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
         const float dx = q0.x - fx;
         const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
         pw4[u] = blend_power(h0, h1, h2, (q0.y - fy0) - slot2);
-        on4[u] = (j4 - u >= 0) && (b + ju < last) && (pw4[u] <= 0.f) && (pw4[u] >= s_blue[ju].y);
+        on4[u] = (j4 - u >= 0) && (s_ord[ju] < last) && (pw4[u] <= 0.f) && (pw4[u] >= s_blue[ju].y);
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -188,7 +209,6 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
   __shared__ BlendRow s_rowdata[BLEND_WARPS][32];
   __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, power threshold
   __shared__ uint32_t s_rowid[BLEND_WARPS][32];
-  __shared__ float4 s_ext[BLEND_WARPS][32];  // box outside of which the row cannot contribute
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   // warps never synchronise with each other; each keeps taking tiles from a ticket counter (see the forward kernel)
   while (true) {
@@ -240,6 +260,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
   for (int bi = nb - 1; bi >= 0; --bi) {
     const uint32_t b = (uint32_t)bi * 32;
     const int cnt = (int)min(32u, total - b);
+    bool reach = false;
     if ((int)lane < cnt) {
       const uint32_t r = vals[start + b + lane];
       const float2 c = xy[r];
@@ -249,15 +270,15 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       s_rowdata[warp][lane] = row;
       const float cut = blend_power_cut(alpha_min, row.q1.w);
       s_blue[warp][lane] = make_float2(rgb[3 * (size_t)r + 2], cut);
-      s_ext[warp][lane] = blend_extent(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, cut);
       s_rowid[warp][lane] = r;
+      reach = blend_reaches_tile(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, cut, tile_x0 + 0.5f, tile_y0 + 0.5f);
     }
+    // warp-uniform: only the rows whose ellipse reaches the tile are evaluated, back to front
+    uint32_t rows = __ballot_sync(0xffffffffu, reach);
     __syncwarp();
-    for (int j = cnt - 1; j >= 0; --j) {
-      // warp-uniform: a row whose box misses the tile is not evaluated at all
-      const float4 ext = s_ext[warp][j];
-      if (ext.y < tile_x0 + 0.5f || ext.x > tile_x0 + 15.5f || ext.w < tile_y0 + 0.5f || ext.z > tile_y0 + 15.5f)
-        continue;
+    while (rows) {
+      const int j = 31 - __clz(rows);
+      rows ^= 1u << j;
       const float4 q0 = s_rowdata[warp][j].q0, q1 = s_rowdata[warp][j].q1;
       const float blue = s_blue[warp][j].x, pcut = s_blue[warp][j].y;
       const float dx = q0.x - fx;

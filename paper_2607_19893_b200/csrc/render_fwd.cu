@@ -15,7 +15,6 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
                   uint32_t* __restrict__ ticket) {
   __shared__ BlendRow s_row[BLEND_WARPS][32];
   __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, power threshold
-  __shared__ float4 s_ext[BLEND_WARPS][32];   // box outside of which the row cannot contribute
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   // Warps never synchronise with each other.  Each one keeps taking tiles from a ticket counter until none is left:
   // lists differ in length by orders of magnitude between tiles, and a fixed tile-to-warp map would leave most of the
@@ -47,6 +46,7 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
   for (uint32_t b = start; b < end; b += 32) {
     if (!__any_sync(0xffffffffu, live != 0)) break;
     const uint32_t i = b + lane;
+    bool reach = false;
     if (i < end) {
       const uint32_t r = vals[i];
       const float2 c = xy[r];
@@ -56,15 +56,14 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
       s_row[warp][lane] = row;
       const float cut = blend_power_cut(alpha_min, row.q1.w);
       s_blue[warp][lane] = make_float2(rgb[3 * (size_t)r + 2], cut);
-      s_ext[warp][lane] = blend_extent(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, cut);
+      reach = blend_reaches_tile(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, cut, tile_x0 + 0.5f, tile_y0 + 0.5f);
     }
+    // warp-uniform: only the rows whose ellipse reaches the tile are evaluated, in list order
+    uint32_t rows = __ballot_sync(0xffffffffu, reach);
     __syncwarp();
-    const int cnt = (int)min(32u, end - b);
-    for (int j = 0; j < cnt; ++j) {
-      // warp-uniform: a row whose box misses the tile is not evaluated at all
-      const float4 ext = s_ext[warp][j];
-      if (ext.y < tile_x0 + 0.5f || ext.x > tile_x0 + 15.5f || ext.w < tile_y0 + 0.5f || ext.z > tile_y0 + 15.5f)
-        continue;
+    while (rows) {
+      const int j = __ffs(rows) - 1;
+      rows &= rows - 1;
       const float4 q0 = s_row[warp][j].q0, q1 = s_row[warp][j].q1;
       const float blue = s_blue[warp][j].x, pcut = s_blue[warp][j].y;
       const float dx = q0.x - fx;
@@ -134,6 +133,8 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
   if (!tile_more[tile]) return;
   __shared__ BlendRow s_row[BLEND_TAIL_THREADS];
   __shared__ float2 s_blue[BLEND_TAIL_THREADS];  // blue, power threshold
+  __shared__ uint32_t s_ord[BLEND_TAIL_THREADS];  // 1-based position of the row in the tile's list
+  __shared__ uint32_t s_wcnt[BLEND_TAIL_THREADS / 32];
   const int tx = tile % TX, ty = tile / TX;
   const int lx = threadIdx.x & 15, ly = threadIdx.x >> 4;
   const int px = tx * 16 + lx, py = ty * 16 + ly;
@@ -154,20 +155,39 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
     last = nc & ~BLEND_DONE_BIT;
     done = (nc & BLEND_DONE_BIT) != 0;
   }
+  const float tile_x0 = (float)(tx * 16) + 0.5f, tile_y0 = (float)(ty * 16) + 0.5f;
+  const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (uint32_t b = start + BLEND_HEAD; b < end; b += BLEND_TAIL_THREADS) {
     if (__syncthreads_count(done) == BLEND_TAIL_THREADS) break;
+    // stage 256 entries and keep, in list order, only the rows whose ellipse reaches the tile
     const uint32_t i = b + threadIdx.x;
+    BlendRow row;
+    float2 bp = make_float2(0.f, 0.f);
+    bool reach = false;
     if (i < end) {
       const uint32_t r = vals[i];
       const float2 c = xy[r];
-      BlendRow row;
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
       row.q1 = conic_o[r];
-      s_row[threadIdx.x] = row;
-      s_blue[threadIdx.x] = make_float2(rgb[3 * (size_t)r + 2], blend_power_cut(alpha_min, row.q1.w));
+      bp = make_float2(rgb[3 * (size_t)r + 2], blend_power_cut(alpha_min, row.q1.w));
+      reach = blend_reaches_tile(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, bp.y, tile_x0, tile_y0);
+    }
+    const uint32_t wm = __ballot_sync(0xffffffffu, reach);
+    if (lane == 0) s_wcnt[warp] = __popc(wm);
+    __syncthreads();
+    int cnt = 0, pos = __popc(wm & ((1u << lane) - 1u));
+#pragma unroll
+    for (int w = 0; w < BLEND_TAIL_THREADS / 32; ++w) {
+      const int c = (int)s_wcnt[w];
+      if (w < (int)warp) pos += c;
+      cnt += c;
+    }
+    if (reach) {
+      s_row[pos] = row;
+      s_blue[pos] = bp;
+      s_ord[pos] = i - start + 1;
     }
     __syncthreads();
-    const int cnt = (int)min((uint32_t)BLEND_TAIL_THREADS, end - b);
     if (!done) {
       // four rows at a time: their exponents and skip tests are independent (a single pixel per thread has no other
       // source of instruction-level parallelism), the blends are then applied in order
@@ -196,7 +216,7 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
               const float w = alpha * T;
               C0 = fmaf(cr[u], w, C0); C1 = fmaf(cg[u], w, C1); C2 = fmaf(cb[u], w, C2);
               T = Tn;
-              last = (b - start) + j + u + 1;
+              last = s_ord[j + u];
             }
           }
         }
