@@ -118,9 +118,14 @@ int odin_poll(odin_ctx* ctx, void* stream);
  * `max_instances` instance capacity. */
 int odin_workspace_bytes(const odin_ctx* ctx, uint32_t n, uint64_t max_instances, size_t* bytes);
 
-/* Workspace size for odin_render_fwd / odin_render_bwd on a width x height image (per-tile flags and 16 bytes per
- * pixel of hand-over state for tiles with long lists).  The same workspace may serve all five calls if it is at least
- * as large as both sizes. */
+/* Minimum workspace size for odin_render_fwd / odin_render_bwd on a width x height image.  The forward call leaves in
+ * it, for every tile whose list is longer than 256 entries, one record (8 KB: transmittance and colour still to come of
+ * the tile's 256 pixels) per further 256 entries that it walks; the backward call of the same view replays the
+ * segments of such lists independently from these records, so it must be given the SAME workspace, unmodified in
+ * between.  The minimum size holds 2 x tiles + 4096 records; a larger workspace is used in full.  If a view needs more
+ * records than fit, the image is still complete, ODIN_ERR_CAPACITY is deferred by the forward call and the gradients
+ * of the affected tiles are approximate.  The same workspace may serve all five calls if it is at least as large as
+ * both sizes (odin_project / odin_touched_set / odin_bin_sort of the NEXT view may overwrite it). */
 int odin_render_workspace_bytes(const odin_ctx* ctx, int width, int height, size_t* bytes);
 
 /* Launch accounting and optional per-kernel timing (the coarse phase profile the paper's scheduler consumes, Sec. 4.2,
@@ -202,7 +207,8 @@ int odin_l1_loss(odin_ctx* ctx, const float* d_rgb, const float* d_target, int w
  * reaches the mean) and the sigmoid.  grad_rows: compact rows (row r <-> proj->prim_id[r]) in the layout of
  * odin_scene with n >= V.
  * d_row_active [capacity] (bytes, may be NULL): 1 for every row that was blended into at least one pixel - the
- * realized active set C_i of Sec. 2.1, observed where the paper observes it, after the backward pass - else 0. */
+ * realized active set C_i of Sec. 2.1, observed where the paper observes it, after the backward pass - else 0.
+ * ws: the workspace the odin_render_fwd call of this view used, unmodified since (see odin_render_workspace_bytes). */
 int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odin_camera* cam, const odin_projected* proj,
                     const uint32_t* d_vals, const uint32_t* d_tile_ranges, const float* d_final_T,
                     const uint32_t* d_n_contrib, const float* d_dL_drgb, float* d_grad2d, odin_scene* grad_rows,

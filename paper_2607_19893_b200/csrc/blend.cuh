@@ -9,23 +9,74 @@
 #pragma once
 #include "common.cuh"
 
-// Long lists.  A tile whose pixels are still live after BLEND_HEAD list entries is finished by a second kernel that
-// gives the tile eight warps (one pixel per thread): a single warp walking a list of thousands of entries would be the
-// tail of the whole launch.  The per-pixel state travels through the output images (forward) or a workspace
-// (backward).  Both kernels evaluate dy as (v - (y0 + 0.5)) - 2 s with y0 the first row of the lane's slot pair, so a
-// pixel sees bit-identical power / alpha in either.
+// Long lists.  Forward: a tile whose pixels are still live after BLEND_HEAD list entries is finished by a second kernel
+// that gives the tile eight warps (one pixel per thread): a single warp walking a list of thousands of entries would be
+// the tail of the whole launch.  The per-pixel state travels through the output images.  Both kernels evaluate dy as
+// (v - (y0 + 0.5)) - 2 s with y0 the first row of the lane's slot pair, so a pixel sees bit-identical power / alpha in
+// either.
+// Backward: the list of a tile is cut into SEGMENTS of BLEND_HEAD entries that are replayed independently, one warp
+// each, all in one launch.  What a segment needs is the state of every pixel at its END: the transmittance and the
+// colour still to come behind it.  The forward tail kernel leaves exactly that in the workspace: for every BLEND_HEAD
+// entries it walks it takes a segment slot from a counter and stores, for its 256 pixels, the transmittance before
+// those entries and the colour they added; when the tile is finished it walks its slots from the last to the first
+// and replaces "colour added" by the running sum "colour still to come" (summed from the back, small terms first, as
+// the sequential replay would: a difference final colour - colour so far would lose the small suffixes of nearly
+// saturated pixels to rounding).  So the backward pass has no sequential tail at all, and the workspace of
+// odin_render_bwd must be the one the odin_render_fwd of the same view used.
 constexpr uint32_t BLEND_HEAD = 256;
-constexpr uint32_t BLEND_DONE_BIT = 0x80000000u;  // in n_contrib while a tile is between the two kernels
+constexpr uint32_t BLEND_DONE_BIT = 0x80000000u;  // in n_contrib while a tile is between the two forward kernels
 constexpr int BLEND_TAIL_THREADS = 256;
 
-// Workspace of the render calls:
-//   [256 B: tile tickets of the forward ([0]) and backward ([1]) head kernels][tile flags u32 x tiles | 256-aligned]
-//   [T, S0, S1, S2 planes, fp32 x pixels each]
+// Workspace of the render calls (every region 256-byte aligned):
+//   [256 B: u32 [0] tile ticket of the forward head kernel, [1] work ticket of the backward kernel, [2] segments taken]
+//   [tile_first: u32 x tiles   forward head: 1 = the tail kernel must continue; forward tail: 1 + slot of the tile's
+//                              segment that starts at entry BLEND_HEAD (0 = none)]
+//   [seg_tile: uint2 x S       (tile, k): the slot holds the state before entry k * BLEND_HEAD of that tile]
+//   [seg_link: uint2 x S       1 + slot of the same tile's segment k + 1, of segment k - 1 (0 = none)]
+//   [ckpt: BlendRecord x 256 x S   per pixel (thread t = 16 * row + column of the tile): T, colour to come (3)]
+// S, the number of segment slots, follows from the size of the workspace the caller passes; the minimum size holds
+// 2 x tiles + 4096 of them.
 constexpr size_t BLEND_WS_HEADER = 256;
-static inline size_t blend_ws_flags_bytes(int n_tiles) { return BLEND_WS_HEADER + ((size_t)n_tiles * 4 + 255) / 256 * 256; }
+// The colour is kept in double: the backward pass needs its product with the pixel's incoming gradient, a sum over
+// the three channels that cancels when the gradient's signs differ (an L1 loss: +-1/N), and a float colour would
+// make that product wrong in its leading digits for every row of the segment at once.
+struct BlendRecord {
+  float T, pad;
+  double S0, S1, S2;
+};
+static_assert(sizeof(BlendRecord) == 32, "record layout");
+constexpr size_t BLEND_SEG_BYTES = 8 + 8 + 256 * sizeof(BlendRecord);
+struct BlendWs {
+  size_t tile_first, seg_tile, seg_link, ckpt, total;
+  uint32_t segments;
+};
+static inline size_t blend_align(size_t x) { return (x + 255) / 256 * 256; }
+static inline size_t blend_ws_flags_bytes(int n_tiles) { return BLEND_WS_HEADER + blend_align((size_t)n_tiles * 4); }
+static inline BlendWs blend_ws_layout(int n_tiles, uint32_t segments) {
+  BlendWs L;
+  L.segments = segments;
+  L.tile_first = BLEND_WS_HEADER;
+  L.seg_tile = L.tile_first + blend_align((size_t)n_tiles * 4);
+  L.seg_link = L.seg_tile + blend_align((size_t)segments * 8);
+  L.ckpt = L.seg_link + blend_align((size_t)segments * 8);
+  L.total = L.ckpt + (size_t)segments * 256 * sizeof(BlendRecord);
+  return L;
+}
+static inline uint32_t blend_min_segments(int n_tiles) { return 2u * (uint32_t)n_tiles + 4096u; }
 static inline size_t blend_ws_bytes(int width, int height) {
   const int n_tiles = ((width + 15) / 16) * ((height + 15) / 16);
-  return blend_ws_flags_bytes(n_tiles) + (size_t)16 * width * height;
+  return blend_ws_layout(n_tiles, blend_min_segments(n_tiles)).total;
+}
+// the largest number of segment slots whose layout fits into ws_bytes (at least the minimum, which the caller checked)
+static inline uint32_t blend_ws_segments(int n_tiles, size_t ws_bytes) {
+  uint32_t s = blend_min_segments(n_tiles);
+  const size_t fixed = blend_ws_layout(n_tiles, 0).total + 3 * 256;
+  if (ws_bytes > fixed) {
+    const size_t fit = (ws_bytes - fixed) / BLEND_SEG_BYTES;
+    if (fit > s) s = (uint32_t)(fit < 0x7fffffffu ? fit : 0x7fffffffu);
+  }
+  while (blend_ws_layout(n_tiles, s).total > ws_bytes && s > blend_min_segments(n_tiles)) --s;
+  return s;
 }
 
 constexpr int BLEND_SLOTS = 8;          // pixels per lane

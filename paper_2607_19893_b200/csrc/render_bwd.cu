@@ -1,5 +1,5 @@
-// Backward phase: (a) per-tile back-to-front replay of the compositing, one warp per tile, per-lane accumulation over
-// eight pixels, one transposing warp reduction and one global atomic per (tile, row, word);
+// Backward phase: (a) back-to-front replay of the compositing, one warp per segment of a tile's list, per-lane
+// accumulation over eight pixels, one transposing warp reduction and one global atomic per (segment, row, word);
 // (b) per-row chain rule through the projection into compact gradient rows.
 #include "blend.cuh"
 #include "geom.cuh"
@@ -34,166 +34,14 @@ __device__ __forceinline__ float warp_transpose_sum8(float a0, float a1, float a
   return d;
 }
 
-// Tail of long lists (runs first): tiles in which some pixel used more than BLEND_HEAD entries get a block of 256
-// threads, one pixel per thread, that walks entries [BLEND_HEAD, total) back to front, 256 at a time, reduces the
-// nine words over each warp and over the block in shared memory, issues one global atomic per (tile, row, word) and
-// leaves every pixel's transmittance and suffix colour in `state` for the head kernel.
-__global__ void __launch_bounds__(BLEND_TAIL_THREADS)
-render_bwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
-                       const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
-                       float bg0, float bg1, float bg2, float alpha_min, float alpha_max,
-                       const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
-                       const float* __restrict__ dL, float* __restrict__ g2d, float* __restrict__ state,
-                       uint8_t* __restrict__ row_active) {
-  constexpr int BB = BLEND_TAIL_THREADS;
-  __shared__ BlendRow s_rowdata[BB];
-  __shared__ float2 s_blue[BB];  // blue, power threshold
-  __shared__ uint32_t s_rowid[BB];
-  __shared__ uint32_t s_ord[BB];
-  __shared__ uint32_t s_wcnt[BB / 32];
-  __shared__ float s_acc[BB * 9];
-  __shared__ uint32_t s_max;
-  const int tile = blockIdx.x;
-  const int tx = tile % TX, ty = tile / TX;
-  const float tile_x0 = (float)(tx * 16) + 0.5f, tile_y0 = (float)(ty * 16) + 0.5f;
-  const int lx = threadIdx.x & 15, ly = threadIdx.x >> 4;
-  const int px = tx * 16 + lx, py = ty * 16 + ly;
-  const bool inside = px < W && py < H;
-  const unsigned lane = threadIdx.x & 31;
-  const float fx = (float)px + 0.5f;
-  const float fy0 = (float)(ty * 16 + (ly & 1)) + 0.5f;
-  const float slot2 = (float)(2 * (ly >> 1));
-  const uint32_t start = ranges[tile].x;
-  const size_t pix = (size_t)py * W + px, plane = (size_t)W * H;
-  float T = 1.f, g0 = 0.f, g1 = 0.f, g2 = 0.f;
-  uint32_t last = 0;
-  if (inside) {
-    T = final_T[pix];
-    last = n_contrib[pix];
-    g0 = dL[pix]; g1 = dL[plane + pix]; g2 = dL[2 * plane + pix];
-  }
-  if (threadIdx.x == 0) s_max = 0;
-  __syncthreads();
-  {
-    uint32_t m = last;
-    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
-    if (lane == 0 && m) atomicMax(&s_max, m);
-  }
-  __syncthreads();
-  const uint32_t total = s_max;
-  if (total <= BLEND_HEAD) return;  // uniform over the block: the head kernel does the whole tile
-  for (int i = threadIdx.x; i < BB * 9; i += BB) s_acc[i] = 0.f;
-  // Only the suffix colour's product with the pixel's incoming gradient is ever needed, so one scalar is carried:
-  // SG = sum_ch S_ch g_ch with S = sum_{j>k} c_j alpha_j T_j + T_final bg.
-  float SG = T * (bg0 * g0 + bg1 * g1 + bg2 * g2);
-  const uint32_t span = total - BLEND_HEAD;
-  const int nb = (int)((span + BB - 1) / BB);
-  for (int bi = nb - 1; bi >= 0; --bi) {
-    const uint32_t b = BLEND_HEAD + (uint32_t)bi * BB;
-    const int staged = (int)min((uint32_t)BB, total - b);
-    // stage up to 256 entries and keep, in list order, only the rows whose ellipse reaches the tile
-    BlendRow row;
-    float2 bp = make_float2(0.f, 0.f);
-    uint32_t r = 0;
-    bool reach = false;
-    if ((int)threadIdx.x < staged) {
-      r = vals[start + b + threadIdx.x];
-      const float2 c = xy[r];
-      row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
-      row.q1 = conic_o[r];
-      bp = make_float2(rgb[3 * (size_t)r + 2], blend_power_cut(alpha_min, row.q1.w));
-      reach = blend_reaches_tile(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, bp.y, tile_x0, tile_y0);
-    }
-    const uint32_t wm = __ballot_sync(0xffffffffu, reach);
-    if (lane == 0) s_wcnt[threadIdx.x >> 5] = __popc(wm);
-    __syncthreads();  // also: the flush of the previous batch is complete
-    int cnt = 0, pos = __popc(wm & ((1u << lane) - 1u));
-#pragma unroll
-    for (int w = 0; w < BB / 32; ++w) {
-      const int c = (int)s_wcnt[w];
-      if (w < (int)(threadIdx.x >> 5)) pos += c;
-      cnt += c;
-    }
-    if (reach) {
-      s_rowdata[pos] = row;
-      s_blue[pos] = bp;
-      s_rowid[pos] = r;
-      s_ord[pos] = b + threadIdx.x;  // 0-based position in the tile's list
-    }
-    __syncthreads();
-    for (int j4 = cnt - 1; j4 >= 0; j4 -= 4) {
-      // four rows at a time (back to front): exponents and skip tests first, they are independent of each other
-      float pw4[4];
-      bool on4[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int ju = max(j4 - u, 0);
-        const float4 q0 = s_rowdata[ju].q0, q1 = s_rowdata[ju].q1;
-        const float dx = q0.x - fx;
-        const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
-        pw4[u] = blend_power(h0, h1, h2, (q0.y - fy0) - slot2);
-        on4[u] = (j4 - u >= 0) && (s_ord[ju] < last) && (pw4[u] <= 0.f) && (pw4[u] >= s_blue[ju].y);
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-      const int j = j4 - u;
-      const bool on = on4[u];
-      if (__ballot_sync(0xffffffffu, on) == 0) continue;
-      if (row_active && lane == 0) row_active[s_rowid[j]] = 1;  // realized-active: blended into at least one pixel
-      const float4 q0 = s_rowdata[j].q0, q1 = s_rowdata[j].q1;
-      const float2 bp = s_blue[j];
-      const float dx = q0.x - fx;
-      const float dy = (q0.y - fy0) - slot2;
-      const float power = pw4[u];
-      float vu = 0.f, vv = 0.f, vA = 0.f, vB = 0.f, vC = 0.f, vo = 0.f, vr = 0.f, vg = 0.f, vb = 0.f;
-      if (on) {
-        const float G = __expf(power);
-        const float og = q1.w * G;
-        const float alpha = fminf(alpha_max, og);
-        const float inv = __fdividef(1.f, 1.f - alpha);
-        const float Tb = T * inv;  // transmittance in front of this row
-        const float w = alpha * Tb;
-        const float c0 = q0.z, c1 = q0.w, c2 = bp.x;
-        vr = w * g0; vg = w * g1; vb = w * g2;
-        const float cg = fmaf(c2, g2, fmaf(c1, g1, c0 * g0));
-        const float dLda = Tb * cg - SG * inv;
-        SG = fmaf(w, cg, SG);
-        T = Tb;
-        if (og <= alpha_max) {
-          const float t = G * dLda;
-          const float gp = q1.w * t;
-          vu = -(q1.x * dx + q1.y * dy) * gp;
-          vv = -(q1.z * dy + q1.y * dx) * gp;
-          vA = -0.5f * dx * dx * gp;
-          vB = -dx * dy * gp;
-          vC = -0.5f * dy * dy * gp;
-          vo = t;
-        }
-      }
-      const float t8 = warp_transpose_sum8(vu, vv, vA, vB, vC, vo, vr, vg, lane);
-      for (int o = 16; o > 0; o >>= 1) vb += __shfl_xor_sync(0xffffffffu, vb, o);
-      if ((lane & 3) == 0) atomicAdd(&s_acc[j * 9 + (lane >> 2)], t8);
-      if (lane == 1) atomicAdd(&s_acc[j * 9 + 8], vb);
-      }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < cnt * 9; i += BB) {
-      const float v = s_acc[i];
-      if (v != 0.f) {
-        atomicAdd(&g2d[(size_t)s_rowid[i / 9] * 9 + (i % 9)], v);
-        s_acc[i] = 0.f;
-      }
-    }
-  }
-  if (inside) {
-    state[pix] = T; state[plane + pix] = SG;
-  }
-}
-
-// One warp per tile, eight pixels per lane (blend.cuh).  For every row of the list the lane accumulates, over its own
-// pixels, the colour and opacity gradients and three moments of dL/dpower (sum, sum*dy, sum*dy^2); dx is constant per
-// lane, so the conic / centre gradients follow from the moments with a handful of operations per row instead of per
-// pixel.  One transposing warp reduction and nine global atomics per (tile, row) that contributed.
+// One warp per SEGMENT of a tile's list (BLEND_HEAD entries), eight pixels per lane (blend.cuh).  Segment 0 of every
+// tile is a work item; the later segments are the ones the forward tail kernel recorded, together with the state of
+// every pixel at the segment's start.  A segment is replayed back to front from the state at its END: that of the
+// next segment's record, or the final state of the pixel when nothing behind the segment contributed.  For every row
+// the lane accumulates, over its own pixels, the colour and opacity gradients and three moments of dL/dpower (sum,
+// sum*dy, sum*dy^2); dx is constant per lane, so the conic / centre gradients follow from the moments with a handful
+// of operations per row instead of per pixel.  One transposing warp reduction and nine global atomics per (segment,
+// row) that contributed.
 // TRACK: also flag the rows that contributed (realized active set).  A separate instantiation because this loop is
 // sensitive to anything added to it: the flag store costs ~5 % of the kernel, and callers who do not ask for the flags
 // do not pay for it.
@@ -202,7 +50,9 @@ __global__ void __launch_bounds__(BLEND_THREADS, 5)
 render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
                         const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
                         int n_tiles, float bg0, float bg1, float bg2, float alpha_min, float alpha_max,
-                        const float* __restrict__ state,
+                        const uint32_t* __restrict__ tile_first, const uint32_t* __restrict__ seg_count,
+                        const uint2* __restrict__ seg_tile, const uint2* __restrict__ seg_link,
+                        const BlendRecord* __restrict__ ckpt, uint32_t seg_cap,
                         const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
                         const float* __restrict__ dL, float* __restrict__ g2d, uint32_t* __restrict__ ticket,
                         uint8_t* __restrict__ row_active) {
@@ -210,12 +60,27 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
   __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, power threshold
   __shared__ uint32_t s_rowid[BLEND_WARPS][32];
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // warps never synchronise with each other; each keeps taking tiles from a ticket counter (see the forward kernel)
+  const uint32_t n_seg = min(*seg_count, seg_cap);
+  // warps never synchronise with each other; each keeps taking work items from a ticket counter (see the forward
+  // kernel).  The recorded segments come first: they are full-length, the segments 0 of most tiles are not.
   while (true) {
-  int tile = 0;
-  if (lane == 0) tile = (int)atomicAdd(ticket, 1u);
-  tile = __shfl_sync(0xffffffffu, tile, 0);
-  if (tile >= n_tiles) return;
+  uint32_t item = 0;
+  if (lane == 0) item = atomicAdd(ticket, 1u);
+  item = __shfl_sync(0xffffffffu, item, 0);
+  int tile;
+  uint32_t seg = 0, next;
+  if (item < n_seg) {
+    const uint2 st = seg_tile[item];
+    tile = (int)st.x; seg = st.y; next = seg_link[item].x;
+  } else {
+    if (item - n_seg >= (uint32_t)n_tiles) return;
+    tile = (int)(item - n_seg);
+    next = tile_first[tile];
+  }
+  // a workspace that is not the forward call's own must not lead anywhere: records are checked before use
+  if ((uint32_t)tile >= (uint32_t)n_tiles || seg >= (1u << 23)) continue;
+  if (next > seg_cap) next = 0;
+  const uint32_t seg_base = seg * BLEND_HEAD;
   const int tx = tile % TX, ty = tile / TX;
   const float tile_x0 = (float)(tx * 16), tile_y0 = (float)(ty * 16);
   const int px = tx * 16 + (int)(lane & 15);
@@ -224,7 +89,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
   const uint32_t start = ranges[tile].x;
   const size_t plane = (size_t)W * H;
 
-  float T[BLEND_SLOTS], SG[BLEND_SLOTS];  // SG: suffix colour times the pixel's incoming gradient (see the tail kernel)
+  float T[BLEND_SLOTS], SG[BLEND_SLOTS];  // SG: colour still to come times the pixel's incoming gradient
   float g0[BLEND_SLOTS], g1[BLEND_SLOTS], g2[BLEND_SLOTS];
   uint32_t last[BLEND_SLOTS];
   uint32_t total = 0;
@@ -238,23 +103,31 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       last[s] = n_contrib[pix];
       g0[s] = dL[pix]; g1[s] = dL[plane + pix]; g2[s] = dL[2 * plane + pix];
     }
+    // Only the product of the colour to come with the pixel's incoming gradient is ever needed, so one scalar is
+    // carried: SG = sum_ch S_ch g_ch with S = sum_{j>k} c_j alpha_j T_j + T_final bg.
     SG[s] = T[s] * (bg0 * g0[s] + bg1 * g1[s] + bg2 * g2[s]);
     total = max(total, last[s]);
   }
   for (int o = 16; o > 0; o >>= 1) total = max(total, __shfl_xor_sync(0xffffffffu, total, o));
-  // `total` = list entries any pixel of the tile used.  Entries beyond BLEND_HEAD were already walked by the tail
-  // kernel, which left every pixel's transmittance and suffix colour in the workspace.
-  if (total > BLEND_HEAD) {
-    total = BLEND_HEAD;
+  // `total` = list entries any pixel of the tile used
+  if (total <= seg_base) continue;  // nothing in this segment contributed
+  if (total > seg_base + BLEND_HEAD) {
+    // rows behind this segment contributed: start from the state the forward pass recorded at the segment's end
+    total = seg_base + BLEND_HEAD;
+    // next == 0: the record is missing (the segment slots ran out, which the forward call reported, or n_contrib is
+    // not the forward pass's own); the final state stands in, exact for the pixels that end inside this segment
+    if (next != 0) {
+      const BlendRecord* ck = ckpt + (size_t)(next - 1) * 256 + lane;
 #pragma unroll
-    for (int s = 0; s < BLEND_SLOTS; ++s) {
-      const int py = py0 + 2 * s;
-      if (px < W && py < H) {
-        const size_t pix = (size_t)py * W + px;
-        T[s] = state[pix]; SG[s] = state[plane + pix];
+      for (int s = 0; s < BLEND_SLOTS; ++s) {
+        const BlendRecord c = ck[32 * s];  // pixel (row 2 s + lane / 16, column lane % 16) = thread 32 s + lane of the tail
+        T[s] = c.T;
+        SG[s] = (float)fma(c.S2, (double)g2[s], fma(c.S1, (double)g1[s], c.S0 * (double)g0[s]));
       }
     }
   }
+  total -= seg_base;  // entries of this segment to walk
+  const uint32_t seg_start = start + seg_base;
   // walk the remaining entries back to front, 32 at a time
   const int nb = (int)((total + 31) / 32);
   for (int bi = nb - 1; bi >= 0; --bi) {
@@ -262,7 +135,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
     const int cnt = (int)min(32u, total - b);
     bool reach = false;
     if ((int)lane < cnt) {
-      const uint32_t r = vals[start + b + lane];
+      const uint32_t r = vals[seg_start + b + lane];
       const float2 c = xy[r];
       BlendRow row;
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
@@ -284,7 +157,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       const float dx = q0.x - fx;
       const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
       const float dy0 = q0.y - fy0;
-      const uint32_t k = b + j;
+      const uint32_t k = seg_base + b + j;
       // phase 1, straight line: the eight exponents and skip tests are independent and overlap in the pipeline
       float pw[BLEND_SLOTS];
       uint32_t pass = 0;
@@ -529,26 +402,24 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
     zero_rows_kernel<<<zgrid, 256, 0, st>>>(d_grad2d, d_row_active, proj->num_rows, proj->capacity);
   }
   const int n_tiles = TX * TY;
-  float* state = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + blend_ws_flags_bytes(n_tiles));
-  uint32_t* ticket = reinterpret_cast<uint32_t*>(ws) + 1;
+  const BlendWs L = blend_ws_layout(n_tiles, blend_ws_segments(n_tiles, ws_bytes));
+  char* base = reinterpret_cast<char*>(ws);
+  uint32_t* header = reinterpret_cast<uint32_t*>(base);
+  uint32_t* ticket = header + 1;
   ODIN_CUDA(cudaMemsetAsync(ticket, 0, 4, st));
   {
-    OdinKernelScope ks(ctx, K_BWD_TAIL, st);
-    render_bwd_tail_kernel<<<n_tiles, BLEND_TAIL_THREADS, 0, st>>>(
-        reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
-        reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
-        ctx->cfg.alpha_min, ctx->cfg.alpha_max, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d, state, d_row_active);
-  }
-  {
     OdinKernelScope ks(ctx, K_BWD_BLEND, st);
-    const int blocks_all = (n_tiles + BLEND_WARPS - 1) / BLEND_WARPS;
-    const int blocks = blocks_all < ctx->sm_count * 8 ? blocks_all : ctx->sm_count * 8;  // resident warps pull tiles
+    const size_t blocks_all = ((size_t)n_tiles + L.segments + BLEND_WARPS - 1) / BLEND_WARPS;
+    const int blocks = blocks_all < (size_t)ctx->sm_count * 8 ? (int)blocks_all : ctx->sm_count * 8;  // resident warps pull work
 #define LAUNCH_BLEND(TRACK)                                                                                             \
   render_bwd_blend_kernel<TRACK><<<blocks, BLEND_THREADS, 0, st>>>(                                                     \
       reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb,       \
       d_vals, reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0],          \
-      cam->bg[1], cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, state, d_final_T, d_n_contrib, d_dL_drgb,         \
-      d_grad2d, ticket, d_row_active)
+      cam->bg[1], cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max,                                                   \
+      reinterpret_cast<const uint32_t*>(base + L.tile_first), header + 2,                                               \
+      reinterpret_cast<const uint2*>(base + L.seg_tile), reinterpret_cast<const uint2*>(base + L.seg_link),             \
+      reinterpret_cast<const BlendRecord*>(base + L.ckpt), L.segments, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d, ticket,  \
+      d_row_active)
     if (d_row_active) LAUNCH_BLEND(true);
     else LAUNCH_BLEND(false);
 #undef LAUNCH_BLEND

@@ -123,18 +123,23 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
 
 // Tail: one block of 256 threads per tile that the head kernel left unfinished, one pixel per thread, rows staged 256
 // at a time.  Thread t handles column t % 16 and row t / 16 = 2 s + (row inside the slot pair), as in the head kernel.
-__global__ void __launch_bounds__(BLEND_TAIL_THREADS)
+// For every batch the block takes a segment slot and stores there, per pixel, the transmittance before the batch and
+// the colour the batch added; when the tile is finished the stored colours are summed from the last record to the
+// first into "colour still to come" (see blend.cuh): the backward pass starts its segments from these records.
+__global__ void __launch_bounds__(BLEND_TAIL_THREADS, 3)
 render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const float* __restrict__ rgb,
                        const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
                        float bg0, float bg1, float bg2, float alpha_min, float alpha_max, float t_min,
                        float* __restrict__ out, float* __restrict__ final_T, uint32_t* __restrict__ n_contrib,
-                       const uint32_t* __restrict__ tile_more) {
+                       uint32_t* __restrict__ tile_first, uint32_t* __restrict__ seg_count, uint2* __restrict__ seg_tile,
+                       uint2* __restrict__ seg_link, BlendRecord* __restrict__ ckpt, uint32_t seg_cap, int* status) {
   const int tile = blockIdx.x;
-  if (!tile_more[tile]) return;
+  if (!tile_first[tile]) return;
   __shared__ BlendRow s_row[BLEND_TAIL_THREADS];
   __shared__ float2 s_blue[BLEND_TAIL_THREADS];  // blue, power threshold
   __shared__ uint32_t s_ord[BLEND_TAIL_THREADS];  // 1-based position of the row in the tile's list
   __shared__ uint32_t s_wcnt[BLEND_TAIL_THREADS / 32];
+  __shared__ uint32_t s_slot;
   const int tx = tile % TX, ty = tile / TX;
   const int lx = threadIdx.x & 15, ly = threadIdx.x >> 4;
   const int px = tx * 16 + lx, py = ty * 16 + ly;
@@ -157,7 +162,9 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
   }
   const float tile_x0 = (float)(tx * 16) + 0.5f, tile_y0 = (float)(ty * 16) + 0.5f;
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (uint32_t b = start + BLEND_HEAD; b < end; b += BLEND_TAIL_THREADS) {
+  uint32_t first_slot = 0, prev_slot = 0;  // 1 + slot; 0 = none
+  uint32_t k = 1;                          // segment index: the batch starts at list entry k * BLEND_HEAD
+  for (uint32_t b = start + BLEND_HEAD; b < end; b += BLEND_TAIL_THREADS, ++k) {
     if (__syncthreads_count(done) == BLEND_TAIL_THREADS) break;
     // stage 256 entries and keep, in list order, only the rows whose ellipse reaches the tile
     const uint32_t i = b + threadIdx.x;
@@ -174,7 +181,25 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
     }
     const uint32_t wm = __ballot_sync(0xffffffffu, reach);
     if (lane == 0) s_wcnt[warp] = __popc(wm);
+    if (threadIdx.x == 0) s_slot = atomicAdd(seg_count, 1u);
     __syncthreads();
+    // the record of segment k: the transmittance before entry k * BLEND_HEAD (where the backward replay of segment
+    // k - 1 begins) and, once the batch is done, the colour its entries added
+    const uint32_t slot = s_slot;
+    const bool have = slot < seg_cap;
+    if (have) {
+      if (threadIdx.x == 0) {
+        seg_tile[slot] = make_uint2((uint32_t)tile, k);
+        seg_link[slot] = make_uint2(0u, prev_slot);
+        if (prev_slot) seg_link[prev_slot - 1].x = slot + 1;
+      }
+      if (!first_slot) first_slot = slot + 1;
+      prev_slot = slot + 1;
+    } else if (threadIdx.x == 0) {
+      odin_set_error(status, ODIN_ERR_CAPACITY);  // the backward pass will miss this tile's later segments
+    }
+    const float T_start = T;
+    double D0 = 0.0, D1 = 0.0, D2 = 0.0;
     int cnt = 0, pos = __popc(wm & ((1u << lane) - 1u));
 #pragma unroll
     for (int w = 0; w < BLEND_TAIL_THREADS / 32; ++w) {
@@ -214,13 +239,22 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
               done = true;
             } else {
               const float w = alpha * T;
+              // the image keeps its one sequential sum per pixel (so it does not depend on where the batches fall);
+              // the per-batch sums, in double, only feed the records
               C0 = fmaf(cr[u], w, C0); C1 = fmaf(cg[u], w, C1); C2 = fmaf(cb[u], w, C2);
+              const double wd = (double)w;
+              D0 = fma((double)cr[u], wd, D0); D1 = fma((double)cg[u], wd, D1); D2 = fma((double)cb[u], wd, D2);
               T = Tn;
               last = s_ord[j + u];
             }
           }
         }
       }
+    }
+    if (have) {
+      BlendRecord rec;
+      rec.T = T_start; rec.pad = 0.f; rec.S0 = D0; rec.S1 = D1; rec.S2 = D2;
+      ckpt[(size_t)slot * BLEND_TAIL_THREADS + threadIdx.x] = rec;
     }
   }
   if (inside) {
@@ -229,6 +263,17 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
     out[2 * plane + pix] = C2 + T * bg2;
     final_T[pix] = T;
     n_contrib[pix] = last;
+  }
+  // colour added by a segment -> colour still to come at its start, summed from the tile's last record to its first
+  // (each thread rewrites its own words; the links were written by thread 0 before barriers every thread has passed)
+  __syncthreads();
+  if (threadIdx.x == 0) tile_first[tile] = first_slot;
+  double S0 = (double)T * (double)bg0, S1 = (double)T * (double)bg1, S2 = (double)T * (double)bg2;
+  for (uint32_t s1 = prev_slot; s1 != 0;) {
+    BlendRecord* c = ckpt + (size_t)(s1 - 1) * BLEND_TAIL_THREADS + threadIdx.x;
+    S0 += c->S0; S1 += c->S1; S2 += c->S2;
+    c->S0 = S0; c->S1 = S1; c->S2 = S2;
+    s1 = seg_link[s1 - 1].y;
   }
 }
 
@@ -276,11 +321,13 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
     return ODIN_ERR_INVALID_ARG;
   const int TX = (cam->width + 15) / 16, TY = (cam->height + 15) / 16;
   const int n_tiles = TX * TY;
-  if (!ws || !odin_aligned(ws, 256) || ws_bytes < blend_ws_flags_bytes(n_tiles)) return ODIN_ERR_WORKSPACE;
-  uint32_t* ticket = reinterpret_cast<uint32_t*>(ws);
-  uint32_t* tile_more = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + BLEND_WS_HEADER);
+  if (!ws || !odin_aligned(ws, 256) || ws_bytes < blend_ws_bytes(cam->width, cam->height)) return ODIN_ERR_WORKSPACE;
+  const BlendWs L = blend_ws_layout(n_tiles, blend_ws_segments(n_tiles, ws_bytes));
+  char* base = reinterpret_cast<char*>(ws);
+  uint32_t* header = reinterpret_cast<uint32_t*>(base);
+  uint32_t* tile_first = reinterpret_cast<uint32_t*>(base + L.tile_first);
   cudaStream_t st = (cudaStream_t)stream;
-  ODIN_CUDA(cudaMemsetAsync(ticket, 0, 4, st));
+  ODIN_CUDA(cudaMemsetAsync(header, 0, 16, st));  // tile ticket, work ticket of the backward pass, segments taken
   {
     OdinKernelScope ks(ctx, K_FWD, st);
     const int blocks_all = (n_tiles + BLEND_WARPS - 1) / BLEND_WARPS;
@@ -288,14 +335,16 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
     render_fwd_kernel<<<blocks, BLEND_THREADS, 0, st>>>(
         reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
         reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0], cam->bg[1],
-        cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_more,
-        ticket);
+        cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_first,
+        header);
   }
   OdinKernelScope ks(ctx, K_FWD_TAIL, st);
   render_fwd_tail_kernel<<<n_tiles, BLEND_TAIL_THREADS, 0, st>>>(
       reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
       reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
-      ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_more);
+      ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_first, header + 2,
+      reinterpret_cast<uint2*>(base + L.seg_tile), reinterpret_cast<uint2*>(base + L.seg_link),
+      reinterpret_cast<BlendRecord*>(base + L.ckpt), L.segments, ctx->d_status);
   return odin_launch_status();
 }
 

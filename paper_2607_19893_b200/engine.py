@@ -88,7 +88,7 @@ class ViewTrainer:
     """Owns every device buffer of the view step and enqueues the seven calls (plus the loss) on one stream."""
 
     def __init__(self, scene, width: int, height: int, row_capacity: int, instance_capacity: int, mask_slots: int = 1,
-                 device: int = 0, cfg: Optional[B.odin_config] = None):
+                 device: int = 0, cfg: Optional[B.odin_config] = None, extra_render_records: int = 0):
         self.device = torch.device("cuda", device)
         torch.cuda.set_device(self.device)
         self.ctx = B.odin_create(device, cfg)
@@ -126,9 +126,12 @@ class ViewTrainer:
         self.active_count = z(1, torch.int32)
         self.evidence = z(max(self.row_capacity, 1), torch.float32)
         self.evidence_sum = z(1, torch.float64)
-        ws_bytes = max(B.odin_workspace_bytes(self.ctx, self.n, self.instance_capacity),
-                       B.odin_render_workspace_bytes(self.ctx, self.width, self.height))
-        self.ws = z(ws_bytes, torch.uint8)
+        self.ws = z(B.odin_workspace_bytes(self.ctx, self.n, self.instance_capacity), torch.uint8)
+        # The render workspace is a buffer of its own: the forward pass leaves per-pixel records for long lists in it
+        # that the backward pass of the same view reads, so nothing else may write there in between.  Every 8,208
+        # bytes beyond the minimum hold one more record (a further 256 list entries of one tile).
+        self.render_ws = z(B.odin_render_workspace_bytes(self.ctx, self.width, self.height)
+                           + 8208 * int(extra_render_records), torch.uint8)
         self.kernel_launches_per_step = 0
         self.keep_sorted_keys = False  # view_step: also write the sorted 64-bit keys (only tests look at them)
         self.track_active = False      # render_bwd: also flag the rows that contributed (needed by active_set)
@@ -153,7 +156,7 @@ class ViewTrainer:
 
     def render_fwd(self, cam: B.odin_camera, stream=None) -> None:
         B.odin_render_fwd(self.ctx, self.proj.struct, self.vals, self.ranges, cam, self.out, self.final_T, self.n_contrib,
-                          self.ws, stream)
+                          self.render_ws, stream)
 
     def l1_loss(self, stream=None) -> None:
         B.odin_l1_loss(self.ctx, self.out, self.target, self.width, self.height, self.loss, self.dL, stream)
@@ -161,7 +164,7 @@ class ViewTrainer:
     def render_bwd(self, cam: B.odin_camera, stream=None) -> None:
         B.odin_render_bwd(self.ctx, self.params.struct, cam, self.proj.struct, self.vals, self.ranges, self.final_T,
                           self.n_contrib, self.dL, self.grad2d, self.grads.struct,
-                          self.row_active if self.track_active else None, self.ws, stream)
+                          self.row_active if self.track_active else None, self.render_ws, stream)
 
     def active_set(self, slot: int = 0, evidence_mode: int = 0, stream=None) -> None:
         """Realized active set of the view whose backward pass ran last (with track_active set): mask (slot), list,

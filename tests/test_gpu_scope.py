@@ -44,6 +44,7 @@ def check_active_set(oracle32, scene, cam, seed=0):
     tr = G.trainer_for(scene, cam, row_capacity=max(v, 1), instance_capacity=len(f["vals"]) + 1)
     tr.track_active = True
     load_sorted(tr, f, inv)
+    tr.render_fwd(B.make_camera(cam))  # the backward pass starts long lists from the states this leaves in the workspace
     tr.final_T.copy_(torch.from_numpy(f["final_T"]).to(tr.device))
     tr.n_contrib.copy_(torch.from_numpy(f["n_contrib"].view(np.int32)).to(tr.device))
     tr.dL.copy_(torch.from_numpy(dl).to(tr.device))
@@ -109,6 +110,7 @@ def test_active_set_capacity_and_empty_view(oracle32):
     tr = G.trainer_for(w.scene, cam, row_capacity=v, instance_capacity=len(f["vals"]) + 1)
     tr.track_active = True
     load_sorted(tr, f, inv)
+    tr.render_fwd(B.make_camera(cam))  # the backward pass starts long lists from the states this leaves in the workspace
     tr.final_T.copy_(torch.from_numpy(f["final_T"]).to(tr.device))
     tr.n_contrib.copy_(torch.from_numpy(f["n_contrib"].view(np.int32)).to(tr.device))
     tr.render_bwd(B.make_camera(cam))

@@ -417,6 +417,9 @@ def check_backward(oracle32, scene, cam, seed=0, min_robust=1 - 2e-3):
     v = len(f["idx"])
     tr = G.trainer_for(scene, cam, row_capacity=max(v, 1), instance_capacity=len(f["vals"]) + 1)
     load_sorted(tr, f, inv)
+    # the backward pass starts the later segments of long lists from the per-pixel states the forward pass leaves in
+    # the workspace; everything else it reads is the oracle's
+    tr.render_fwd(B.make_camera(cam))
     tr.final_T.copy_(torch.from_numpy(f["final_T"]).to(tr.device))
     tr.n_contrib.copy_(torch.from_numpy(f["n_contrib"].view(np.int32)).to(tr.device))
     tr.dL.copy_(torch.from_numpy(dl).to(tr.device))
