@@ -42,9 +42,47 @@ FLOPS_PER_PAIR = {"render_fwd": 25.0, "render_bwd_blend": 75.0}
 # DRAM traffic (read + write, bytes per view) of the kernels of a stage, from the ncu capture of one view step that
 # profiles/view_step_kernels_cfg3.txt summarises; only that workload was captured
 NCU_TRAFFIC = {"cfg3_1m_sh3_1600x1066": {
-    "render_bwd_blend": 45.3e6 + 34.9e6, "render_fwd": 9.7e6 + 8.4e6, "onesweep_pass": 123.0e6 + 95.1e6,
-    "adam": 425.4e6 + 196.6e6, "emit_instances": 32.1e6 + 3.9e6, "row_sort": 1.3e6 + 1.5e6 + 2.7e6 + 2.7e6 + 2.6e6,
-    "project": 39.4e6 + 4.0e6 + 128.5e6, "render_bwd_project": 40.4e6, "touched_set": 4.0e6, "l1_loss": 41.3e6}}
+    "render_bwd_blend": 48.3e6, "render_fwd": 9.6e6 + 8.4e6, "onesweep_pass": 120.4e6 + 95.1e6,
+    "adam": 425.1e6 + 196.0e6, "emit_instances": 32.6e6 + 3.9e6, "row_sort": 1.3e6 + 1.5e6 + 2.7e6 + 2.7e6 + 2.7e6,
+    "project": 39.4e6 + 4.0e6 + 128.4e6, "render_bwd_project": 40.1e6, "touched_set": 4.0e6, "l1_loss": 41.1e6}}
+
+
+def evaluated_entries(tr, tile_max, alpha_min):
+    """Of the list entries the blend kernels walk (tile_max per tile), the number whose ellipse reaches the tile's
+    pixel centres: only for those is the per-pixel arithmetic evaluated, so only those count as work in the ALU
+    roofline of the blend stages.  Measurement code (torch, outside every timed region): the same convex-quadratic
+    minimum over the tile's rectangle that the kernels take when they stage a row, without their rounding slack."""
+    import torch
+
+    counts = tile_max.flatten()
+    n_t = counts.numel()
+    total = int(counts.sum().item())
+    if total == 0:
+        return 0
+    dev = counts.device
+    tiles = torch.repeat_interleave(torch.arange(n_t, device=dev), counts)
+    first = torch.cumsum(counts, 0) - counts
+    pos = tr.ranges.view(n_t, 2)[:, 0].to(torch.int64)[tiles] + (torch.arange(total, device=dev) - first[tiles])
+    rows = tr.vals[pos].to(torch.int64)
+    u, v = tr.proj.xy[rows, 0].double(), tr.proj.xy[rows, 1].double()
+    co = tr.proj.conic_opacity[rows].double()
+    a, b, c, op = co[:, 0], co[:, 1], co[:, 2], co[:, 3]
+    k = 2.0 * torch.log(torch.clamp(op, min=1e-300) / alpha_min)
+    xl = (tiles % tr.tx).double() * 16 + 0.5 - u
+    yl = torch.div(tiles, tr.tx, rounding_mode="floor").double() * 16 + 0.5 - v
+    xh, yh = xl + 15, yl + 15
+    inside = (xl <= 0) & (xh >= 0) & (yl <= 0) & (yh >= 0)
+
+    def q(dx, dy):
+        return a * dx * dx + 2 * b * dx * dy + c * dy * dy
+
+    qmin = torch.full_like(u, float("inf"))
+    for dx in (xl, xh):
+        qmin = torch.minimum(qmin, q(dx, torch.minimum(torch.maximum(-b * dx / c, yl), yh)))
+    for dy in (yl, yh):
+        qmin = torch.minimum(qmin, q(torch.minimum(torch.maximum(-b * dy / a, xl), xh), dy))
+    reach = (k >= 0) & (inside | (qmin <= k))
+    return int(reach.sum().item())
 
 
 def measured_peaks():
@@ -336,7 +374,8 @@ def main():
     pad[:H, :W] = ncon
     tile_max = pad.view(ty, 16, tx, 16).amax(dim=(1, 3)).to(torch.int64)
     m_proc = int(tile_max.sum().item())           # list entries the backward pass walks
-    pairs_bwd = 256 * m_proc
+    m_eval = evaluated_entries(tr, tile_max, float(B.default_config().alpha_min))  # ... of which the ellipse reaches the tile
+    pairs_bwd = 256 * m_eval
     passes = (32 + max(int(np.ceil(np.log2(max(tx * ty, 1)))), 0) + 7) // 8  # 8-bit digits
     n_pairs_last = len(pair_lists[-1])
     bytes_model = algorithmic_bytes(n, f, v_last, m_last, m_proc, W * H, tx * ty, passes, n_pairs_last)
@@ -423,7 +462,7 @@ def main():
                   for k, (t, c) in prof.items() if c}
         # kernels that split one stage (head + tail of the blend, the three projection kernels, ...) are judged
         # together: the stage's algorithmic work over the summed time of its kernels in one step
-        stage_of = {"render_fwd_tail": "render_fwd", "render_bwd_tail": "render_bwd_blend", "project_cull": "project",
+        stage_of = {"render_fwd_tail": "render_fwd", "project_cull": "project",
                     "project_scan": "project", "project_rows": "project",
                     "adam_sh": "adam", "adam_geom": "adam", "l1_finish": "l1_loss",
                     "zero_rows": "render_bwd_blend", "row_hist": "row_sort", "row_sort_pass": "row_sort",
@@ -441,8 +480,10 @@ def main():
             ach = flops / t_stage / 1e12
             roofline = {"kernel": top, "kernels": members, "bound": "alu", "achieved": ach, "peak": ALU_PEAK_TFLOPS,
                         "unit": "TFLOP/s", "frac": ach / ALU_PEAK_TFLOPS, "traffic": None,
-                        "note": f"{FLOPS_PER_PAIR[top]:.0f} flop x {pairs_bwd} (pixel,row) pairs per view; peak = "
-                                "148 SM x 128 lanes x 2 x 1.965 GHz"}
+                        "note": f"{FLOPS_PER_PAIR[top]:.0f} flop x {pairs_bwd} (pixel,row) pairs per view = 256 x the "
+                                f"{m_eval} walked list entries whose ellipse reaches their tile (of {m_proc} walked: "
+                                "the others are rejected when the row is staged); peak = 148 SM x 128 lanes x 2 x "
+                                "1.965 GHz"}
         else:
             ach = bytes_kernels[top] / t_stage / 1e9
             roofline = {"kernel": top, "kernels": members, "bound": "hbm", "achieved": ach, "peak": peak_gbs,
@@ -457,7 +498,7 @@ def main():
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": w.name, "primitives": n, "floats_per_primitive": f, "image": [W, H], "views": n_views,
-                   "visible_last_view": v_last, "instances_last_view": m_last, "traversed_last_view": m_proc,
+                   "visible_last_view": v_last, "instances_last_view": m_last, "traversed_last_view": m_proc, "evaluated_last_view": m_eval,
                    "conflict_window": CONFLICT_WINDOW, "binning": args.binning, "parallelism": "replicas only" if world > 1 else "1 gpu",
                    "l2": "no flush: parameters + moments + instance buffers exceed the 126 MB L2 between uses"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
