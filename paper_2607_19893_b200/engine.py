@@ -213,6 +213,12 @@ class ViewTrainer:
                 "copied": [torch.cuda.Event() for _ in range(2)],
                 "consumed": [torch.cuda.Event() for _ in range(2)],
                 "done": [torch.cuda.Event() for _ in range(2)],
+                # the results of a step are read back on a stream of their own, from device slots of the step's parity,
+                # so that the compute stream carries kernels only and the next step need not wait for the read
+                "read_stream": torch.cuda.Stream(device=self.device),
+                "d_loss": [torch.zeros_like(self.loss) for _ in range(2)],
+                "d_count": [torch.zeros_like(self.count) for _ in range(2)],
+                "d_counts": [torch.zeros(max(n_counts, 1), dtype=torch.int64, device=self.device) for _ in range(2)],
             }
             self._host_io = io
         return io
@@ -223,8 +229,10 @@ class ViewTrainer:
         host_target_of(s) is copied to the device, the view cam_of(s) is stepped, and the loss, the number of touched
         primitives and (if pairs_of is given) the conflict counts are read back into pinned memory and handed to
         on_result(s, loss, touched, counts).  Two staging buffers and a copy stream: the copy of the next target
-        overlaps the current view's kernels, and the host waits for the results of the previous view while the current
-        one runs.  Marshalling only: every kernel is the library's."""
+        overlaps the current view's kernels, the results are read back on a third stream from device slots that
+        alternate with the step, and the host waits for the results of the previous view while the current one runs.
+        Afterwards self.loss, self.count and d_counts hold the last step's results.  Marshalling only: every kernel
+        is the library's."""
         steps = list(steps)
         n_counts = 0 if d_counts is None else d_counts.numel()
         io = self.prepare_host_io(n_counts)
@@ -234,7 +242,8 @@ class ViewTrainer:
         copy_stream, staging = io["copy_stream"], io["staging"]
         h_loss, h_count, h_counts = io["h_loss"], io["h_count"], io["h_counts"]
         copied, consumed, done = io["copied"], io["consumed"], io["done"]
-        saved_target = self.target
+        read_stream = io["read_stream"]
+        saved_target, saved_loss, saved_count = self.target, self.loss, self.count
 
         def enqueue_copy(i):
             k = i & 1
@@ -257,20 +266,29 @@ class ViewTrainer:
             if i + 1 < len(steps):
                 enqueue_copy(i + 1)
             stream.wait_event(copied[k])
-            self.target = staging[k]
+            self.target, self.loss, self.count = staging[k], io["d_loss"][k], io["d_count"][k]
+            step_counts = io["d_counts"][k][:n_counts] if n_counts else None
             pairs = pairs_of(s) if pairs_of is not None else None
             self.view_step(cam_of(s), s + 1, lr, beta1, beta2, eps, slot=slot_of(s), d_pairs=pairs[0] if pairs else None,
-                           n_pairs=pairs[1] if pairs else 0, d_counts=d_counts, stream=stream)
+                           n_pairs=pairs[1] if pairs else 0, d_counts=step_counts, stream=stream)
             consumed[k].record(stream)
-            h_loss[k].copy_(self.loss, non_blocking=True)
-            h_count[k].copy_(self.count, non_blocking=True)
-            if n_counts:
-                h_counts[k][:n_counts].copy_(d_counts, non_blocking=True)
-            done[k].record(stream)
+            with torch.cuda.stream(read_stream):
+                read_stream.wait_event(consumed[k])
+                h_loss[k].copy_(self.loss, non_blocking=True)
+                h_count[k].copy_(self.count, non_blocking=True)
+                if n_counts:
+                    h_counts[k][:n_counts].copy_(step_counts, non_blocking=True)
+                done[k].record(read_stream)
             if i > 0:
-                deliver(i - 1)
+                deliver(i - 1)  # also: the slots of parity k ^ 1 are free again before step i + 1 writes them
         deliver(len(steps) - 1)
-        self.target = saved_target
+        # leave the trainer as the plain loop would: its own buffers hold the last step's results
+        k = (len(steps) - 1) & 1
+        saved_loss.copy_(io["d_loss"][k])
+        saved_count.copy_(io["d_count"][k])
+        if n_counts:
+            d_counts.view(-1)[:n_counts].copy_(io["d_counts"][k][:n_counts])
+        self.target, self.loss, self.count = saved_target, saved_loss, saved_count
 
     def poll(self, stream=None) -> int:
         return B.odin_poll(self.ctx, stream)
