@@ -6,10 +6,11 @@ from paper_2607_19893_b200 import binding as B
 from paper_2607_19893_b200.engine import ViewTrainer
 
 
-def trainer_for(scene, cam, row_capacity=None, instance_capacity=None, mask_slots=1, cfg=None):
+def trainer_for(scene, cam, row_capacity=None, instance_capacity=None, mask_slots=1, cfg=None, extra_render_records=0):
     n = scene.means.shape[0]
     return ViewTrainer(scene, cam.width, cam.height, row_capacity if row_capacity is not None else n,
-                       instance_capacity if instance_capacity is not None else max(64 * n, 1 << 16), mask_slots, cfg=cfg)
+                       instance_capacity if instance_capacity is not None else max(64 * n, 1 << 16), mask_slots, cfg=cfg,
+                       extra_render_records=extra_render_records)
 
 
 def compact_from_oracle(proj, idx):

@@ -340,12 +340,13 @@ def load_sorted(tr, f, inv):
     tr.ranges.copy_(torch.from_numpy(f["ranges"].view(np.int32)).to(tr.device))
 
 
-def check_forward(oracle32, scene, cam, min_robust=1 - 2e-3):
+def check_forward(oracle32, scene, cam, min_robust=1 - 2e-3, extra_render_records=0, expect_status=B.ODIN_OK):
     f, inv = oracle_view(oracle32, scene, cam)
-    tr = G.trainer_for(scene, cam, row_capacity=max(len(f["idx"]), 1), instance_capacity=len(f["vals"]) + 1)
+    tr = G.trainer_for(scene, cam, row_capacity=max(len(f["idx"]), 1), instance_capacity=len(f["vals"]) + 1,
+                       extra_render_records=extra_render_records)
     load_sorted(tr, f, inv)
     tr.render_fwd(B.make_camera(cam))
-    G.poll_ok(tr)
+    assert tr.poll() == expect_status
     out = tr.out.cpu().numpy()
     ft = tr.final_T.cpu().numpy()
     nc = G.u32(tr.n_contrib)
@@ -401,7 +402,7 @@ def test_l1_loss(oracle32):
 
 
 # ------------------------------------------------------------------------------------------------ backward
-def check_backward(oracle32, scene, cam, seed=0, min_robust=1 - 2e-3):
+def check_backward(oracle32, scene, cam, seed=0, min_robust=1 - 2e-3, extra_render_records=0):
     f, inv = oracle_view(oracle32, scene, cam)
     rng = np.random.default_rng(seed)
     dl = rng.uniform(-1, 1, f["out"].shape).astype(np.float32)
@@ -415,7 +416,8 @@ def check_backward(oracle32, scene, cam, seed=0, min_robust=1 - 2e-3):
                                                want_abs=True)
     rows_o = oracle32.render_bwd_project(scene, cam, f["idx"], g2d_o, f["proj"].clamp_flags).astype(np.float64)
     v = len(f["idx"])
-    tr = G.trainer_for(scene, cam, row_capacity=max(v, 1), instance_capacity=len(f["vals"]) + 1)
+    tr = G.trainer_for(scene, cam, row_capacity=max(v, 1), instance_capacity=len(f["vals"]) + 1,
+                       extra_render_records=extra_render_records)
     load_sorted(tr, f, inv)
     # the backward pass starts the later segments of long lists from the per-pixel states the forward pass leaves in
     # the workspace; everything else it reads is the oracle's
@@ -499,3 +501,36 @@ def test_render_fwd_mixed_short_and_long_lists(oracle32):
     lens = f["ranges"][:, 1] - f["ranges"][:, 0]
     assert lens.min() < 512 < lens.max()
     check_backward(oracle32, s, cam, seed=13, min_robust=0.98)
+
+
+def one_tile_scene_with_a_list_of_a_million(n_faint=1_060_000, n_solid=48, seed=21):
+    """A 16x16 image (one tile) in front of which lie a million splats too faint to pass the alpha threshold, and a
+    few ordinary ones behind them: the forward pass has to walk the whole list before anything blends, more than 4,100
+    batches of 256 entries, each of which takes a segment record."""
+    rng = np.random.default_rng(seed)
+    n = n_faint + n_solid
+    means = np.zeros((n, 3), np.float32)
+    means[:, :2] = rng.uniform(-0.08, 0.08, (n, 2))
+    means[:n_faint, 2] = rng.uniform(2.0, 4.0, n_faint)
+    means[n_faint:, 2] = rng.uniform(5.0, 6.0, n_solid)
+    log_scales = np.full((n, 3), np.log(0.05), np.float32) + 0.2 * rng.standard_normal((n, 3)).astype(np.float32)
+    quats = rng.standard_normal((n, 4)).astype(np.float32)
+    opacity_logit = np.full(n, np.log(0.003 / 0.997), np.float32)       # 0.003 < 1/255: never blends
+    opacity_logit[n_faint:] = rng.uniform(-2.0, 0.0, n_solid).astype(np.float32)
+    sh = rng.uniform(-1.0, 2.0, (n, 1, 3)).astype(np.float32)
+    scene = wl.Scene(0, means, log_scales, quats, opacity_logit, sh)
+    w2c = np.concatenate([np.eye(3), np.zeros((3, 1))], axis=1)
+    cam = wl.Camera(16, 16, 64.0, 64.0, 8.0, 8.0, 0.2, 1.0e9, w2c, np.array([0.3, 0.1, 0.5]))
+    return scene, cam
+
+
+def test_render_more_segments_than_the_minimum_workspace_records(oracle32):
+    s, cam = one_tile_scene_with_a_list_of_a_million()
+    # the minimum render workspace of a one-tile image holds 2 + 4096 records: the image is still exact, the forward
+    # call reports that the backward pass will lack records
+    f = check_forward(oracle32, s, cam, expect_status=B.ODIN_ERR_CAPACITY)
+    assert f["n_contrib"].max() > 1_050_000 and len(f["vals"]) > 1_050_000
+    # with room for the ~4,140 records: no error, and the backward pass (one warp per segment, 4,140 of them for the one
+    # tile, all but the last without a single contribution) meets the same bar as everywhere else
+    check_forward(oracle32, s, cam, extra_render_records=256)
+    check_backward(oracle32, s, cam, seed=22, extra_render_records=256)
