@@ -464,7 +464,7 @@ def main():
         # together: the stage's algorithmic work over the summed time of its kernels in one step
         stage_of = {"render_fwd_tail": "render_fwd", "project_cull": "project",
                     "project_scan": "project", "project_rows": "project",
-                    "adam_sh": "adam", "adam_geom": "adam", "l1_finish": "l1_loss",
+                    "adam_sh": "adam", "adam_geom": "adam",
                     "zero_rows": "render_bwd_blend", "row_hist": "row_sort", "row_sort_pass": "row_sort",
                     "row_offsets": "emit_instances"}
         stage_ms = {}

@@ -71,7 +71,7 @@ extern "C" int odin_poll(odin_ctx* ctx, void* stream) {
 
 static const char* const kKernelNames[K_COUNT] = {
     "project_cull", "touched_set", "emit_instances", "onesweep_pass", "render_fwd", "l1_loss",
-    "l1_finish", "zero_rows", "render_bwd_blend", "render_bwd_project", "adam_sh", "adam_geom", "conflict_count",
+    "zero_rows", "render_bwd_blend", "render_bwd_project", "adam_sh", "adam_geom", "conflict_count",
     "render_fwd_tail", "project_scan", "project_rows", "row_hist",
     "row_sort_pass", "row_offsets", "active_set", "mask_union", "hazard_count", "delayed_read_gate",
     "locality_graph"};

@@ -9,7 +9,7 @@
 
 // Kernel ids for launch counting and optional per-kernel CUDA-event timing.
 enum OdinKernelId {
-  K_PROJECT = 0, K_TOUCHED, K_EMIT, K_ONESWEEP, K_FWD, K_L1, K_L1_FINISH, K_ZERO_ROWS,
+  K_PROJECT = 0, K_TOUCHED, K_EMIT, K_ONESWEEP, K_FWD, K_L1, K_ZERO_ROWS,
   K_BWD_BLEND, K_BWD_PROJECT, K_ADAM_SH, K_ADAM_GEOM, K_CONFLICT, K_FWD_TAIL, K_PROJECT_SCAN,
   K_PROJECT_ROWS, K_ROW_HIST, K_ROW_SORT, K_ROW_OFFSETS, K_ACTIVE_SET, K_MASK_UNION, K_HAZARD,
   K_GATE, K_RLG, K_COUNT

@@ -281,7 +281,7 @@ constexpr int LB = 256;
 
 __global__ void __launch_bounds__(LB)
 l1_loss_kernel(const float* __restrict__ out, const float* __restrict__ target, size_t count, float inv, double* loss_acc,
-               float* __restrict__ dL) {
+               float* __restrict__ dL, double inv_count, float* __restrict__ loss) {
   float acc = 0.f;
   for (size_t i = (size_t)blockIdx.x * LB + threadIdx.x; i < count; i += (size_t)gridDim.x * LB) {
     const float d = out[i] - target[i];
@@ -296,10 +296,15 @@ l1_loss_kernel(const float* __restrict__ out, const float* __restrict__ target, 
     double t = 0;
     for (int i = 0; i < LB / 32; ++i) t += (double)s[i];
     atomicAdd(loss_acc, t);
+    // the block that arrives last turns the sum into the mean (no second launch)
+    __threadfence();
+    uint32_t* arrivals = reinterpret_cast<uint32_t*>(loss_acc + 1);
+    if (atomicAdd(arrivals, 1u) == gridDim.x - 1u) {
+      __threadfence();
+      *loss = (float)(atomicAdd(loss_acc, 0.0) * inv_count);
+    }
   }
 }
-
-__global__ void l1_finish_kernel(const double* acc, double inv, float* loss) { *loss = (float)(*acc * inv); }
 
 }  // namespace
 
@@ -354,16 +359,14 @@ extern "C" int odin_l1_loss(odin_ctx* ctx, const float* d_rgb, const float* d_ta
   if (width <= 0 || height <= 0) return ODIN_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t count = (size_t)3 * width * height;
-  // the accumulator lives behind the status word in the context's device block
+  // the accumulator (8 bytes) and the arrival counter of the blocks (4 bytes behind it) live behind the status word in
+  // the context's device block
   double* acc = reinterpret_cast<double*>(reinterpret_cast<char*>(ctx->d_status) + 64);
-  ODIN_CUDA(cudaMemsetAsync(acc, 0, 8, st));
+  ODIN_CUDA(cudaMemsetAsync(acc, 0, 16, st));
   size_t blocks = (count + LB - 1) / LB;
   if (blocks > (size_t)ctx->sm_count * 8) blocks = (size_t)ctx->sm_count * 8;
-  {
-    OdinKernelScope ks(ctx, K_L1, st);
-    l1_loss_kernel<<<(unsigned)blocks, LB, 0, st>>>(d_rgb, d_target, count, (float)(1.0 / (double)count), acc, d_dL_drgb);
-  }
-  OdinKernelScope ks(ctx, K_L1_FINISH, st);
-  l1_finish_kernel<<<1, 1, 0, st>>>(acc, 1.0 / (double)count, d_loss);
+  OdinKernelScope ks(ctx, K_L1, st);
+  l1_loss_kernel<<<(unsigned)blocks, LB, 0, st>>>(d_rgb, d_target, count, (float)(1.0 / (double)count), acc, d_dL_drgb,
+                                                  1.0 / (double)count, d_loss);
   return odin_launch_status();
 }
