@@ -156,7 +156,9 @@ def conflict_pairs(step: int):
 
 
 def algorithmic_bytes(n, f, v, m, m_proc, p, t, passes, n_pairs):
-    """Bytes one view has to move, per stage (fp32; F floats per primitive)."""
+    """Bytes one view of the METHOD has to move, per stage (fp32; f floats per primitive, v visible rows, m instances,
+    m_proc walked list entries, p pixels, t tiles): every array a stage must read or write counted once, the sort as
+    `passes` 8-bit passes over 12-byte instances (8-byte key + 4-byte value, read and written)."""
     f4 = 4 * f
     b = {
         "project": 12 * n + (f4 - 12) * v + 4 * n + 61 * v,

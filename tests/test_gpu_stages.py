@@ -493,6 +493,28 @@ def test_render_bwd_lists_longer_than_the_head(oracle32):
     check_backward(oracle32, s, cam, seed=11, min_robust=0.98)
 
 
+def test_render_bwd_with_a_workspace_that_is_not_the_forward_pass_s(oracle32):
+    """The backward pass reads segment records from the render workspace.  A workspace that holds something else
+    (here: every byte 0xff, then every byte 0) must not lead it outside its buffers: every record is checked before
+    use, the call completes, and what it computes without usable records is finite (exact wherever a list ends within
+    its first 256 entries)."""
+    s, cam = faint_scene(n=12_000, seed=10)
+    f, inv = oracle_view(oracle32, s, cam)
+    v = len(f["idx"])
+    tr = G.trainer_for(s, cam, row_capacity=v, instance_capacity=len(f["vals"]) + 1)
+    load_sorted(tr, f, inv)
+    tr.render_fwd(B.make_camera(cam))
+    G.poll_ok(tr)
+    tr.dL.fill_(1.0 / 3.0)
+    for byte in (0xFF, 0x00):
+        tr.render_ws.fill_(byte)
+        tr.render_bwd(B.make_camera(cam))
+        G.poll_ok(tr)
+        assert torch.isfinite(tr.grad2d[:v]).all()
+        assert torch.isfinite(torch.from_numpy(tr.grads.rows_as_matrix(v))).all()
+    tr.close()
+
+
 def test_render_fwd_mixed_short_and_long_lists(oracle32):
     # half of the image crowded with faint splats (tail kernel), the other half nearly empty (head kernel only)
     s, cam = faint_scene(n=16_000, seed=12)
