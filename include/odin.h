@@ -189,7 +189,10 @@ int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int width, int heig
  * power = -(A dx^2 + C dy^2)/2 - B dx dy; skip if power > 0; alpha = min(alpha_max, opacity * exp(power)); skip if
  * alpha < alpha_min; stop if T (1 - alpha) < t_min; colour += rgb * alpha * T; T *= 1 - alpha.
  * d_rgb [3][H][W] = colour + T * bg (planar, not clamped); d_final_T [H][W]; d_n_contrib [H][W] = 1 + list offset of the
- * last row that contributed (0 if none). */
+ * last row that contributed (0 if none).
+ * ws (at least odin_render_workspace_bytes, 256-byte aligned): scratch, and the records that odin_render_bwd of the
+ * same view reads (see odin_render_workspace_bytes); ODIN_ERR_CAPACITY is deferred when they do not all fit (the
+ * outputs of this call are complete in any case). */
 int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const uint32_t* d_vals, const uint32_t* d_tile_ranges,
                     const odin_camera* cam, float* d_rgb, float* d_final_T, uint32_t* d_n_contrib, void* ws, size_t ws_bytes,
                     void* stream);
