@@ -50,12 +50,16 @@ __device__ __forceinline__ Footprint project_footprint(const CamParams& cam, con
   if (!(g.t[2] > cam.znear && g.t[2] < cam.zfar)) return f;
   const float ls[3] = {log_scales[3 * p], log_scales[3 * p + 1], log_scales[3 * p + 2]};
   if (PRETEST) {
-    const float iz = 1.f / g.t[2];
+    // hardware approximations (relative error ~1e-6) are enough here: the bound carries 1 % + 2 pixels of slack, and
+    // most primitives of a large scene leave at this test
+    const float iz = __fdividef(1.f, g.t[2]);
     const float uc = cam.fx * g.t[0] * iz + cam.cx, vc = cam.fy * g.t[1] * iz + cam.cy;
-    const float smax = expf(fmaxf(ls[0], fmaxf(ls[1], ls[2])));
+    const float smax = __expf(fmaxf(ls[0], fmaxf(ls[1], ls[2])));
     const float jx = cam.fx * iz, jy = cam.fy * iz;
     const float jn2 = jx * jx * (1.f + cam.limx * cam.limx) + jy * jy * (1.f + cam.limy * cam.limy);
-    const float rb = radius_sigmas * sqrtf(jn2 * smax * smax + dilation + 0.32f) * 1.01f + 2.f;
+    float root;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(root) : "f"(jn2 * smax * smax + dilation + 0.32f));
+    const float rb = radius_sigmas * root * 1.01f + 2.f;
     if (uc + rb < 0.f || uc - rb > 16.f * (float)cam.TX || vc + rb < 0.f || vc - rb > 16.f * (float)cam.TY) return f;
   }
   odin_splat_geometry(cam, dilation, ls, quats[p], g);
