@@ -211,20 +211,25 @@ int odin_l1_loss(odin_ctx* ctx, const float* d_rgb, const float* d_target, int w
  * odin_scene with n >= V.
  * d_row_active [capacity] (bytes, may be NULL): 1 for every row that was blended into at least one pixel - the
  * realized active set C_i of Sec. 2.1, observed where the paper observes it, after the backward pass - else 0.
+ * d_row_zero [capacity] (bytes, may be NULL): if given, a row whose nine words of d_grad2d are all zero (it never
+ * blended: most touched rows are occluded) is NOT written to grad_rows; d_row_zero[r] = 1 says so instead, 0 marks the
+ * rows that were written.  odin_sparse_adam takes the same flags and reads no gradient for the flagged rows.
  * ws: the workspace the odin_render_fwd call of this view used, unmodified since (see odin_render_workspace_bytes). */
 int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odin_camera* cam, const odin_projected* proj,
                     const uint32_t* d_vals, const uint32_t* d_tile_ranges, const float* d_final_T,
                     const uint32_t* d_n_contrib, const float* d_dL_drgb, float* d_grad2d, odin_scene* grad_rows,
-                    uint8_t* d_row_active, void* ws, size_t ws_bytes, void* stream);
+                    uint8_t* d_row_active, uint8_t* d_row_zero, void* ws, size_t ws_bytes, void* stream);
 
 /* Optimizer update (phase U) restricted to the touched rows: for every r < *d_count and every scalar theta of
  * primitive d_idx[r] with gradient g: m = b1 m + (1-b1) g; v = b2 v + (1-b2) g^2;
  * theta -= lr_group / (1 - b1^step) * m / (sqrt(v) / sqrt(1 - b2^step) + eps).  step is the global 1-based step.
  * lr: mean, log scale, quaternion, opacity, SH degree 0, SH degrees >= 1.  Rows that are not listed are neither read
- * nor written.  d_idx must be strictly ascending (as produced by odin_touched_set / odin_project). */
+ * nor written.  d_idx must be strictly ascending (as produced by odin_touched_set / odin_project).
+ * d_row_zero [rows] (bytes, may be NULL): the flags of odin_render_bwd; a flagged row's gradient is taken as zero
+ * without reading grad_rows (its moments still decay and its parameters still move, exactly as with a row of zeros). */
 int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m, odin_scene* v, const odin_scene* grad_rows,
-                     const uint32_t* d_idx, const uint32_t* d_count, const float lr[6], float beta1, float beta2,
-                     float eps, uint32_t step, void* stream);
+                     const uint8_t* d_row_zero, const uint32_t* d_idx, const uint32_t* d_count, const float lr[6],
+                     float beta1, float beta2, float eps, uint32_t step, void* stream);
 
 /* Conflict counts (Sec. 4.3): for each listed pair (a, b) of views, |W^+(a) & W^+(b)| = popcount of the AND of their
  * touched bitmasks, the size of C_WAW^+ (C_RAW^+ and C_WAR^+ are empty because R^+ = W^+ here).

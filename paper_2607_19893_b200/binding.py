@@ -95,9 +95,9 @@ def lib() -> C.CDLL:
                                       C.c_size_t, vp]
         L.odin_l1_loss.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
         L.odin_render_bwd.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_camera), C.POINTER(odin_projected), vp, vp,
-                                      vp, vp, vp, vp, C.POINTER(odin_scene), vp, vp, C.c_size_t, vp]
+                                      vp, vp, vp, vp, C.POINTER(odin_scene), vp, vp, vp, C.c_size_t, vp]
         L.odin_sparse_adam.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_scene), C.POINTER(odin_scene),
-                                       C.POINTER(odin_scene), vp, vp, C.POINTER(f32), f32, f32, f32, u32, vp]
+                                       C.POINTER(odin_scene), vp, vp, vp, C.POINTER(f32), f32, f32, f32, u32, vp]
         L.odin_conflict_count.argtypes = [vp, vp, u32, u32, u32, vp, u32, vp, vp]
         L.odin_touched_set_static.argtypes = [vp, u32, vp, vp, u32, vp, vp, vp]
         L.odin_active_set.argtypes = [vp, C.POINTER(odin_projected), vp, vp, C.POINTER(odin_scene), i32, u32, vp, vp, u32,
@@ -233,19 +233,20 @@ def odin_l1_loss(ctx, d_rgb, d_target, width: int, height: int, d_loss, d_dL_drg
 
 
 def odin_render_bwd(ctx, scene: odin_scene, cam: odin_camera, proj: odin_projected, d_vals, d_tile_ranges, d_final_T,
-                    d_n_contrib, d_dL_drgb, d_grad2d, grad_rows: odin_scene, d_row_active, ws, stream=None) -> None:
+                    d_n_contrib, d_dL_drgb, d_grad2d, grad_rows: odin_scene, d_row_active, d_row_zero, ws,
+                    stream=None) -> None:
     _check(lib().odin_render_bwd(ctx, C.byref(scene), C.byref(cam), C.byref(proj), _ptr(d_vals), _ptr(d_tile_ranges),
                                  _ptr(d_final_T), _ptr(d_n_contrib), _ptr(d_dL_drgb), _ptr(d_grad2d), C.byref(grad_rows),
-                                 _ptr(d_row_active), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
-                                 _stream(stream)),
+                                 _ptr(d_row_active), _ptr(d_row_zero), _ptr(ws),
+                                 0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
            "odin_render_bwd")
 
 
-def odin_sparse_adam(ctx, params: odin_scene, m: odin_scene, v: odin_scene, grad_rows: odin_scene, d_idx, d_count,
-                     lr: Sequence[float], beta1: float, beta2: float, eps: float, step: int, stream=None) -> None:
+def odin_sparse_adam(ctx, params: odin_scene, m: odin_scene, v: odin_scene, grad_rows: odin_scene, d_row_zero, d_idx,
+                     d_count, lr: Sequence[float], beta1: float, beta2: float, eps: float, step: int, stream=None) -> None:
     lr_arr = (C.c_float * 6)(*[float(x) for x in lr])
-    _check(lib().odin_sparse_adam(ctx, C.byref(params), C.byref(m), C.byref(v), C.byref(grad_rows), _ptr(d_idx),
-                                  _ptr(d_count), lr_arr, float(beta1), float(beta2), float(eps), int(step),
+    _check(lib().odin_sparse_adam(ctx, C.byref(params), C.byref(m), C.byref(v), C.byref(grad_rows), _ptr(d_row_zero),
+                                  _ptr(d_idx), _ptr(d_count), lr_arr, float(beta1), float(beta2), float(eps), int(step),
                                   _stream(stream)), "odin_sparse_adam")
 
 

@@ -31,7 +31,8 @@ __device__ __forceinline__ void adam_one(float& th, float& m, float& v, float g,
 template <int ROWF, int VEC>
 __global__ void __launch_bounds__(256)
 adam_sh_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v, const float* __restrict__ g,
-               const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count, uint32_t cap, AdamK k) {
+               const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count, uint32_t cap, AdamK k,
+               const uint8_t* __restrict__ row_zero) {
   constexpr int EPR = ROWF / VEC;  // elements per row
   const uint32_t V = min(*count, cap);
   const size_t total = (size_t)V * EPR;
@@ -39,8 +40,9 @@ adam_sh_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__
     const uint32_t r = (uint32_t)(e / EPR);
     const uint32_t j = (uint32_t)(e - (size_t)r * EPR);
     const size_t dst = (size_t)idx[r] * ROWF + (size_t)j * VEC;
+    const bool zero = row_zero && row_zero[r];  // the gradient row was not written: it is zero
     if (VEC == 4) {
-      const float4 gg = reinterpret_cast<const float4*>(g)[e];
+      const float4 gg = zero ? make_float4(0.f, 0.f, 0.f, 0.f) : reinterpret_cast<const float4*>(g)[e];
       float4 pp = *reinterpret_cast<float4*>(p + dst), mm = *reinterpret_cast<float4*>(m + dst),
              vv = *reinterpret_cast<float4*>(v + dst);
       // floats 0..2 of a row are the degree-0 coefficients (group 4); the rest group 5
@@ -54,7 +56,7 @@ adam_sh_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__
       *reinterpret_cast<float4*>(v + dst) = vv;
     } else {
       float pp = p[dst], mm = m[dst], vv = v[dst];
-      adam_one(pp, mm, vv, g[e], k.step_size[j < 3 ? 4 : 5], k);
+      adam_one(pp, mm, vv, zero ? 0.f : g[e], k.step_size[j < 3 ? 4 : 5], k);
       p[dst] = pp; m[dst] = mm; v[dst] = vv;
     }
   }
@@ -68,13 +70,14 @@ adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* _
                  float* __restrict__ v_mean, float* __restrict__ v_ls, float4* __restrict__ v_q, float* __restrict__ v_o,
                  const float* __restrict__ g_mean, const float* __restrict__ g_ls, const float4* __restrict__ g_q,
                  const float* __restrict__ g_o, const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count,
-                 uint32_t cap, AdamK k) {
+                 uint32_t cap, AdamK k, const uint8_t* __restrict__ row_zero) {
   const uint32_t V = min(*count, cap);
   const size_t total = (size_t)V * 4;
   for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
     const uint32_t r = (uint32_t)(e >> 2);
     const int part = (int)(e & 3);
     const size_t d = idx[r];
+    const bool zero = row_zero && row_zero[r];  // the gradient row was not written: it is zero
     if (part < 2) {
       float* __restrict__ p = (part ? p_ls : p_mean) + 3 * d;
       float* __restrict__ m = (part ? m_ls : m_mean) + 3 * d;
@@ -83,14 +86,14 @@ adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* _
       const float ss = k.step_size[part];
       float pp[3], mm[3], vv[3], gg[3];
 #pragma unroll
-      for (int i = 0; i < 3; ++i) { pp[i] = p[i]; mm[i] = m[i]; vv[i] = v[i]; gg[i] = g[i]; }
+      for (int i = 0; i < 3; ++i) { pp[i] = p[i]; mm[i] = m[i]; vv[i] = v[i]; gg[i] = zero ? 0.f : g[i]; }
 #pragma unroll
       for (int i = 0; i < 3; ++i) adam_one(pp[i], mm[i], vv[i], gg[i], ss, k);
 #pragma unroll
       for (int i = 0; i < 3; ++i) { p[i] = pp[i]; m[i] = mm[i]; v[i] = vv[i]; }
     } else if (part == 2) {
       float4 pp = p_q[d], mm = m_q[d], vv = v_q[d];
-      const float4 gg = g_q[r];
+      const float4 gg = zero ? make_float4(0.f, 0.f, 0.f, 0.f) : g_q[r];
       adam_one(pp.x, mm.x, vv.x, gg.x, k.step_size[2], k);
       adam_one(pp.y, mm.y, vv.y, gg.y, k.step_size[2], k);
       adam_one(pp.z, mm.z, vv.z, gg.z, k.step_size[2], k);
@@ -98,7 +101,7 @@ adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* _
       p_q[d] = pp; m_q[d] = mm; v_q[d] = vv;
     } else {
       float pp = p_o[d], mm = m_o[d], vv = v_o[d];
-      adam_one(pp, mm, vv, g_o[r], k.step_size[3], k);
+      adam_one(pp, mm, vv, zero ? 0.f : g_o[r], k.step_size[3], k);
       p_o[d] = pp; m_o[d] = mm; v_o[d] = vv;
     }
   }
@@ -107,8 +110,9 @@ adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* _
 }  // namespace
 
 extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m, odin_scene* v,
-                                const odin_scene* grad_rows, const uint32_t* d_idx, const uint32_t* d_count,
-                                const float lr[6], float beta1, float beta2, float eps, uint32_t step, void* stream) {
+                                const odin_scene* grad_rows, const uint8_t* d_row_zero, const uint32_t* d_idx,
+                                const uint32_t* d_count, const float lr[6], float beta1, float beta2, float eps,
+                                uint32_t step, void* stream) {
   if (!ctx || !lr || !d_count) return ODIN_ERR_NULL;
   int rc = odin_check_scene(params);
   if (rc == ODIN_OK) rc = odin_check_scene(m);
@@ -138,10 +142,10 @@ extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m
   {
     OdinKernelScope ks(ctx, K_ADAM_SH, st);
     switch (params->sh_degree) {
-    case 0: adam_sh_kernel<3, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
-    case 1: adam_sh_kernel<12, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
-    case 2: adam_sh_kernel<27, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
-    default: adam_sh_kernel<48, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k); break;
+    case 0: adam_sh_kernel<3, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero); break;
+    case 1: adam_sh_kernel<12, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero); break;
+    case 2: adam_sh_kernel<27, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero); break;
+    default: adam_sh_kernel<48, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero); break;
     }
   }
   size_t gb = ((size_t)cap * 4 + 255) / 256;
@@ -151,6 +155,6 @@ extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m
       params->means, params->log_scales, reinterpret_cast<float4*>(params->quats), params->opacity_logit, m->means,
       m->log_scales, reinterpret_cast<float4*>(m->quats), m->opacity_logit, v->means, v->log_scales,
       reinterpret_cast<float4*>(v->quats), v->opacity_logit, grad_rows->means, grad_rows->log_scales,
-      reinterpret_cast<const float4*>(grad_rows->quats), grad_rows->opacity_logit, d_idx, d_count, cap, k);
+      reinterpret_cast<const float4*>(grad_rows->quats), grad_rows->opacity_logit, d_idx, d_count, cap, k, d_row_zero);
   return odin_launch_status();
 }

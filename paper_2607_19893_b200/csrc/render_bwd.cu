@@ -227,7 +227,8 @@ render_bwd_project_kernel(const float* __restrict__ means, const float* __restri
                           const float* __restrict__ sh, CamParams cam, float dilation, const uint32_t* __restrict__ prim_id,
                           const uint8_t* __restrict__ clamp_flags, const uint32_t* __restrict__ num_rows, uint32_t capacity,
                           const float* __restrict__ g2d, float* __restrict__ g_means, float* __restrict__ g_ls,
-                          float4* __restrict__ g_quats, float* __restrict__ g_opac, float* __restrict__ g_sh) {
+                          float4* __restrict__ g_quats, float* __restrict__ g_opac, float* __restrict__ g_sh,
+                          uint8_t* __restrict__ row_zero) {
   constexpr int K = (DEG + 1) * (DEG + 1);
   const uint32_t V = min(*num_rows, capacity);
   for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
@@ -239,6 +240,10 @@ render_bwd_project_kernel(const float* __restrict__ means, const float* __restri
     // and arrive with all nine at zero: their gradient row is zero and needs neither the scene nor any arithmetic.
     if (gu == 0.f && gv == 0.f && gA == 0.f && gB == 0.f && gC == 0.f && go == 0.f && grgb[0] == 0.f && grgb[1] == 0.f &&
         grgb[2] == 0.f) {
+      if (row_zero) {  // the caller takes a flag instead of a row of zeros (the optimizer then reads no gradient for it)
+        row_zero[r] = 1;
+        continue;
+      }
 #pragma unroll
       for (int j = 0; j < 3; ++j) { g_means[3 * (size_t)r + j] = 0.f; g_ls[3 * (size_t)r + j] = 0.f; }
       g_quats[r] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -253,6 +258,7 @@ render_bwd_project_kernel(const float* __restrict__ means, const float* __restri
       }
       continue;
     }
+    if (row_zero) row_zero[r] = 0;
     const float mx = means[3 * p], my = means[3 * p + 1], mz = means[3 * p + 2];
     SplatGeom g;
     odin_camera_space(cam, mx, my, mz, g.t);
@@ -379,7 +385,7 @@ render_bwd_project_kernel(const float* __restrict__ means, const float* __restri
 extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odin_camera* cam, const odin_projected* proj,
                                const uint32_t* d_vals, const uint32_t* d_tile_ranges, const float* d_final_T,
                                const uint32_t* d_n_contrib, const float* d_dL_drgb, float* d_grad2d, odin_scene* grad_rows,
-                               uint8_t* d_row_active, void* ws, size_t ws_bytes, void* stream) {
+                               uint8_t* d_row_active, uint8_t* d_row_zero, void* ws, size_t ws_bytes, void* stream) {
   if (!ctx || !proj || !grad_rows) return ODIN_ERR_NULL;
   int rc = odin_check_scene(scene);
   if (rc != ODIN_OK) return rc;
@@ -432,7 +438,7 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
       scene->means, scene->log_scales, reinterpret_cast<const float4*>(scene->quats), scene->opacity_logit, scene->sh,  \
       cp, ctx->cfg.dilation, proj->prim_id, proj->clamp_flags, proj->num_rows, proj->capacity, d_grad2d,                \
       grad_rows->means, grad_rows->log_scales, reinterpret_cast<float4*>(grad_rows->quats), grad_rows->opacity_logit,    \
-      grad_rows->sh)
+      grad_rows->sh, d_row_zero)
   OdinKernelScope ks(ctx, K_BWD_PROJECT, st);
   switch (scene->sh_degree) {
     case 0: LAUNCH(0); break;

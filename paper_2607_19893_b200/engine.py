@@ -135,6 +135,9 @@ class ViewTrainer:
         self.kernel_launches_per_step = 0
         self.keep_sorted_keys = False  # view_step: also write the sorted 64-bit keys (only tests look at them)
         self.track_active = False      # render_bwd: also flag the rows that contributed (needed by active_set)
+        self.skip_zero_rows = True     # render_bwd flags zero gradient rows instead of writing them; Adam takes the flags
+        self.row_zero = z(max(self.row_capacity, 1), torch.uint8)
+        self._row_zero_in_use = None   # the flags the last render_bwd wrote (None: every row was written)
 
     def close(self) -> None:
         if self.ctx is not None:
@@ -162,9 +165,20 @@ class ViewTrainer:
         B.odin_l1_loss(self.ctx, self.out, self.target, self.width, self.height, self.loss, self.dL, stream)
 
     def render_bwd(self, cam: B.odin_camera, stream=None) -> None:
+        # rows whose gradient is zero (never blended: most touched rows) are flagged instead of written, unless the
+        # realized active set is tracked (its evidence reads the gradient rows)
+        self._row_zero_in_use = self.row_zero if (self.skip_zero_rows and not self.track_active) else None
         B.odin_render_bwd(self.ctx, self.params.struct, cam, self.proj.struct, self.vals, self.ranges, self.final_T,
                           self.n_contrib, self.dL, self.grad2d, self.grads.struct,
-                          self.row_active if self.track_active else None, self.render_ws, stream)
+                          self.row_active if self.track_active else None, self._row_zero_in_use, self.render_ws, stream)
+
+    def gradient_rows(self, v: int) -> np.ndarray:
+        """The first v gradient rows as one matrix (see DeviceScene.rows_as_matrix), the rows that the backward pass
+        flagged as zero instead of writing them filled in with zeros."""
+        rows = self.grads.rows_as_matrix(v)
+        if self._row_zero_in_use is not None:
+            rows[self._row_zero_in_use[:v].cpu().numpy().astype(bool)] = 0
+        return rows
 
     def active_set(self, slot: int = 0, evidence_mode: int = 0, stream=None) -> None:
         """Realized active set of the view whose backward pass ran last (with track_active set): mask (slot), list,
@@ -176,8 +190,8 @@ class ViewTrainer:
                           self.evidence, self.evidence_sum, self.ws, stream)
 
     def sparse_adam(self, lr, beta1, beta2, eps, step: int, stream=None) -> None:
-        B.odin_sparse_adam(self.ctx, self.params.struct, self.m.struct, self.v.struct, self.grads.struct, self.idx,
-                           self.count, lr, beta1, beta2, eps, step, stream)
+        B.odin_sparse_adam(self.ctx, self.params.struct, self.m.struct, self.v.struct, self.grads.struct,
+                           self._row_zero_in_use, self.idx, self.count, lr, beta1, beta2, eps, step, stream)
 
     def conflict_count(self, d_pairs, n_pairs: int, d_counts, stream=None) -> None:
         B.odin_conflict_count(self.ctx, self.masks, self.mask_slots, self.masks.shape[1], self.n, d_pairs, n_pairs,

@@ -54,7 +54,7 @@ def test_null_context_is_rejected_without_a_device(lib):
     assert lib.odin_render_workspace_bytes(null, 64, 64, C.byref(sz)) == B.ODIN_ERR_NULL
     assert lib.odin_render_fwd(null, None, None, None, None, None, None, None, None, 0, None) == B.ODIN_ERR_NULL
     assert lib.odin_l1_loss(null, None, None, 1, 1, None, None, None) == B.ODIN_ERR_NULL
-    assert lib.odin_render_bwd(null, None, None, None, None, None, None, None, None, None, None, None, None, 0,
+    assert lib.odin_render_bwd(null, None, None, None, None, None, None, None, None, None, None, None, None, None, 0,
                                None) == B.ODIN_ERR_NULL
     assert lib.odin_active_set(null, None, None, None, None, 0, 0, None, None, 0, None, None, None, None, 0,
                                None) == B.ODIN_ERR_NULL
@@ -65,7 +65,8 @@ def test_null_context_is_rejected_without_a_device(lib):
     assert lib.odin_rlg_weights(null, None, None, None, 0, 0, None, None) == B.ODIN_ERR_NULL
     assert lib.odin_rlg_topk(null, None, 0, 0, None, None, 0, None) == B.ODIN_ERR_NULL
     assert lib.odin_sds_scores(null, None, 0, None, 0, None, 0, None, None) == B.ODIN_ERR_NULL
-    assert lib.odin_sparse_adam(null, None, None, None, None, None, None, None, 0.9, 0.999, 1e-8, 1, None) == B.ODIN_ERR_NULL
+    assert lib.odin_sparse_adam(null, None, None, None, None, None, None, None, None, 0.9, 0.999, 1e-8, 1,
+                                None) == B.ODIN_ERR_NULL
     assert lib.odin_conflict_count(null, None, 0, 0, 0, None, 0, None, None) == B.ODIN_ERR_NULL
 
 

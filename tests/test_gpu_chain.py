@@ -91,7 +91,7 @@ def run_chain(oracle32, w, steps, views, window=None, row_capacity=None, instanc
         _, g2d_abs = oracle32.render_bwd_blend(o["proj"], o["vals"], o["ranges"], cam, o["final_T"], o["n_contrib"],
                                                o["dL_dout"], want_abs=True)
         rows = o["rows"].astype(np.float64)
-        rows_dev = tr.grads.rows_as_matrix(len(idx)).astype(np.float64)
+        rows_dev = tr.gradient_rows(len(idx)).astype(np.float64)
         if not differs.any():
             bound = G.rows_bound(oracle32, pre, cam, o["idx"], o["proj"].clamp_flags, rows, o["g2d"], g2d_abs)
             # the chained run also carries the device's own projection and pixel rounding into the gradients
