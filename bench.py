@@ -42,9 +42,9 @@ FLOPS_PER_PAIR = {"render_fwd": 25.0, "render_bwd_blend": 75.0}
 # DRAM traffic (read + write, bytes per view) of the kernels of a stage, from the ncu capture of one view step that
 # profiles/view_step_kernels_cfg3.txt summarises; only that workload was captured
 NCU_TRAFFIC = {"cfg3_1m_sh3_1600x1066": {
-    "render_bwd_blend": 48.3e6, "render_fwd": 9.6e6 + 8.4e6, "onesweep_pass": 120.4e6 + 95.1e6,
-    "adam": 425.1e6 + 196.0e6, "emit_instances": 32.6e6 + 3.9e6, "row_sort": 1.3e6 + 1.5e6 + 2.7e6 + 2.7e6 + 2.7e6,
-    "project": 39.4e6 + 4.0e6 + 128.4e6, "render_bwd_project": 40.1e6, "touched_set": 4.0e6, "l1_loss": 41.1e6}}
+    "render_bwd_blend": 49.1e6, "render_fwd": 9.6e6 + 8.4e6, "onesweep_pass": 119.9e6 + 95.0e6,
+    "adam": 366.1e6 + 185.6e6, "emit_instances": 31.5e6 + 3.9e6, "row_sort": 1.3e6 + 1.5e6 + 2.7e6 + 2.7e6 + 2.7e6,
+    "project": 39.4e6 + 4.0e6 + 128.5e6, "render_bwd_project": 18.9e6, "touched_set": 4.0e6, "l1_loss": 41.1e6}}
 
 
 def evaluated_entries(tr, tile_max, alpha_min):
