@@ -281,9 +281,18 @@ constexpr int LB = 256;
 
 __global__ void __launch_bounds__(LB)
 l1_loss_kernel(const float* __restrict__ out, const float* __restrict__ target, size_t count, float inv, double* loss_acc,
-               float* __restrict__ dL, double inv_count, float* __restrict__ loss) {
+               float* __restrict__ dL, double inv_count, float* __restrict__ loss, size_t vec4) {
+  // vec4: number of leading float4 groups (0 when the three images are not 16-byte aligned); the rest one by one
   float acc = 0.f;
-  for (size_t i = (size_t)blockIdx.x * LB + threadIdx.x; i < count; i += (size_t)gridDim.x * LB) {
+  const size_t tid = (size_t)blockIdx.x * LB + threadIdx.x, stride = (size_t)gridDim.x * LB;
+  for (size_t i = tid; i < vec4; i += stride) {
+    const float4 a = reinterpret_cast<const float4*>(out)[i], b = reinterpret_cast<const float4*>(target)[i];
+    const float d0 = a.x - b.x, d1 = a.y - b.y, d2 = a.z - b.z, d3 = a.w - b.w;
+    acc += (fabsf(d0) + fabsf(d1)) + (fabsf(d2) + fabsf(d3));
+    reinterpret_cast<float4*>(dL)[i] = make_float4(d0 > 0.f ? inv : (d0 < 0.f ? -inv : 0.f), d1 > 0.f ? inv : (d1 < 0.f ? -inv : 0.f),
+                                                   d2 > 0.f ? inv : (d2 < 0.f ? -inv : 0.f), d3 > 0.f ? inv : (d3 < 0.f ? -inv : 0.f));
+  }
+  for (size_t i = vec4 * 4 + tid; i < count; i += stride) {
     const float d = out[i] - target[i];
     acc += fabsf(d);
     dL[i] = d > 0.f ? inv : (d < 0.f ? -inv : 0.f);
@@ -363,10 +372,12 @@ extern "C" int odin_l1_loss(odin_ctx* ctx, const float* d_rgb, const float* d_ta
   // the context's device block
   double* acc = reinterpret_cast<double*>(reinterpret_cast<char*>(ctx->d_status) + 64);
   ODIN_CUDA(cudaMemsetAsync(acc, 0, 16, st));
-  size_t blocks = (count + LB - 1) / LB;
+  const bool aligned = odin_aligned(d_rgb, 16) && odin_aligned(d_target, 16) && odin_aligned(d_dL_drgb, 16);
+  const size_t vec4 = aligned ? count / 4 : 0;
+  size_t blocks = (count / 4 + LB - 1) / LB + 1;
   if (blocks > (size_t)ctx->sm_count * 8) blocks = (size_t)ctx->sm_count * 8;
   OdinKernelScope ks(ctx, K_L1, st);
   l1_loss_kernel<<<(unsigned)blocks, LB, 0, st>>>(d_rgb, d_target, count, (float)(1.0 / (double)count), acc, d_dL_drgb,
-                                                  1.0 / (double)count, d_loss);
+                                                  1.0 / (double)count, d_loss, vec4);
   return odin_launch_status();
 }

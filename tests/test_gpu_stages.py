@@ -407,6 +407,17 @@ def test_l1_loss(oracle32):
     assert B.odin_poll(ctx) == B.ODIN_OK
     assert abs(float(d_loss.item()) - loss_o) < 1e-6 * max(1.0, loss_o)
     assert np.array_equal(d_g.cpu().numpy(), g_o)
+    # images that start 4 bytes into their allocations (no 16-byte alignment): the element-wise path
+    count = out.size
+    bufs = [torch.zeros(count + 1, device=dev) for _ in range(3)]
+    m_out, m_tgt, m_g = (b[1:] for b in bufs)
+    m_out.copy_(d_out.flatten())
+    m_tgt.copy_(d_tgt.flatten())
+    d_loss.zero_()
+    B.odin_l1_loss(ctx, m_out, m_tgt, w_, h_, d_loss, m_g)
+    assert B.odin_poll(ctx) == B.ODIN_OK
+    assert abs(float(d_loss.item()) - loss_o) < 1e-6 * max(1.0, loss_o)
+    assert np.array_equal(m_g.cpu().numpy().reshape(g_o.shape), g_o)
     B.odin_destroy(ctx)
 
 
