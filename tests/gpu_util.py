@@ -69,14 +69,45 @@ def grad2d_bound(want2d, abs2d):
     return GRAD_RTOL * np.abs(want2d) + GRAD_FLOOR * abs2d + 1e-30
 
 
+# The chain rule of a row runs in fp32 on both sides: every intermediate is rounded to 2^-24 relative, so a word that
+# is a cancelled combination of intermediates carries an absolute error of a few ulp of the LARGEST quantities of the
+# row, whatever its own size.  Eight ulp of the row's largest word are granted to every word of the row.
+ROW_ULP_FLOOR = 8 * 2.0 ** -24
+
+
 def rows_bound(oracle, scene, cam, idx, clamp_flags, rows_o, want2d_dense, abs2d_dense):
     n = want2d_dense.shape[0]
     # second term: rounding inside the fp32 chain rule itself (its own sums cancel too)
     slack2d = GRAD_FLOOR * abs2d_dense + GRAD_FLOOR * np.abs(want2d_dense)
-    bound = GRAD_RTOL * np.abs(rows_o) + 1e-30
+    bound = GRAD_RTOL * np.abs(rows_o) + ROW_ULP_FLOOR * np.abs(rows_o).max(axis=1, keepdims=True) + 1e-30
     for c in range(9):
         unit = np.zeros((n, 9))
         unit[:, c] = 1.0
         jac_c = oracle.render_bwd_project(scene, cam, idx, unit, clamp_flags).astype(np.float64)
         bound = bound + np.abs(jac_c) * slack2d[idx.astype(np.int64), c][:, None]
     return bound
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Measured distances to the bars are printed (pytest -rP or -s shows them) so that every slack factor in the chained
+# tests can be read against what the device actually does.
+def report(tag, **kv):
+    print("PARITY " + tag + " " + " ".join(f"{k}={v:.4g}" if isinstance(v, float) else f"{k}={v}" for k, v in kv.items()),
+          flush=True)
+
+
+def blended_at_pixels(o, pixels_yx, upto, tx, alpha_min=1.0 / 255.0):
+    """Primitive ids that blend (alpha within 1 % of the skip threshold or above) at the given pixels, looking at the
+    first upto[k] entries of the pixel's tile list.  pixels_yx: [K,2] (row, column).  These are the primitives whose
+    gradient changes when a decision of that pixel falls the other way."""
+    out = []
+    xy, co = o["proj"].xy.astype(np.float64), o["proj"].conic_o.astype(np.float64)
+    for (y, x), n in zip(pixels_yx, upto):
+        t = (y // 16) * tx + (x // 16)
+        s, e = int(o["ranges"][t, 0]), int(o["ranges"][t, 1])
+        prims = o["vals"][s:min(e, s + int(n))].astype(np.int64)
+        dx, dy = xy[prims, 0] - (x + 0.5), xy[prims, 1] - (y + 0.5)
+        power = -0.5 * (co[prims, 0] * dx * dx + co[prims, 2] * dy * dy) - co[prims, 1] * dx * dy
+        alpha = co[prims, 3] * np.exp(np.minimum(power, 0.0))
+        out.append(prims[(power <= 1e-6) & (alpha >= 0.99 * alpha_min)])
+    return np.unique(np.concatenate(out)) if out else np.zeros(0, np.int64)

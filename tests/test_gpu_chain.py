@@ -7,151 +7,302 @@ from paper_2607_19893_b200 import binding as B
 from paper_2607_19893_b200 import workloads as wl
 
 import gpu_util as G
+from oracle import oracle as oracle_mod
 
 pytestmark = pytest.mark.gpu
 
 
-def run_chain(oracle32, w, steps, views, window=None, row_capacity=None, instance_capacity=None, cfg=None):
+# Bars of the chained run (every factor is derived below or measured and printed per step, see G.report):
+#  * integer outputs: bit exact once the primitives whose tile count differs from the oracle's are taken out of both
+#    sides; such a primitive must sit within FRAGILE_PRIM (2e-6 relative, ~30 float ulps) of a projection decision.
+#  * pixels: 1e-4 absolute wherever the oracle's decision margin exceeds PIX_MARGIN (the others, "fragile", must be
+#    fewer than max_fragile = 2e-3 of the pixels); every pixel outside the tiles of a differing primitive within 5e-3;
+#    those tiles must be fewer than 2 % of the image.
+#  * gradient rows: G.rows_bound (1e-3 relative + 1e-5 of the un-cancelled term sums, pushed through the oracle's own
+#    Jacobian) times ROWS_SLACK for every word of every primitive that does not sit on a fragile pixel.  The chained
+#    run carries the device's own projection (conic, centre, colour: each a few ulp from the oracle's) into every
+#    term, which the stage-isolated bound does not contain (a strongly anisotropic splat amplifies an ulp of its
+#    scales into 1e-4 of its conic); ROWS_SLACK = 8 is about 2x the largest ratio measured on the five presets (4.3,
+#    one word of 5e7 at preset 5; printed as rows_worst).
+#  * Adam: every touched word of params / m / v against the oracle's Adam applied to the DEVICE's gradient rows, 2e-5
+#    relative (the stage-isolated bar), and against the oracle's own chained result wherever the two gradients agree to
+#    1e-3 relative (the benchmark spec's 1e-3 relative, 1e-5 absolute floor).
+FRAGILE_PRIM = 2e-6
+PIX_MARGIN = 2e-5
+ROWS_SLACK = 8.0
+
+
+def window_pairs(step, window, slots):
+    """Mask slots compared after `step`: the current view against the (up to) `window` views before it."""
+    cur = step % slots
+    return [(cur, (step - j) % slots) for j in range(1, min(window, step) + 1)]
+
+
+def run_chain(oracle32, w, steps, views, window=None, row_capacity=None, instance_capacity=None, cfg=None, tag="chain",
+              max_fragile=2e-3):
     """Runs `steps` views on both sides from the same start.  Both sides see the same parameters at every step
     because the oracle is re-synchronised from the device after each comparison (so one fragile decision cannot
-    cascade); every step is compared on its own."""
+    cascade); every step is compared on its own.  window = k: every view's touched mask is compared, inside the step,
+    with the masks of the k views before it as they were when produced; None: all pairs over the latest masks at the
+    end."""
     scene = w.scene
     n = scene.n
     cam0 = w.cameras[0]
+    slots = (window + 1) if window else max(len(views), 1)
     tr = G.trainer_for(scene, cam0, row_capacity=row_capacity, instance_capacity=instance_capacity,
-                       mask_slots=max(len(views), 1), cfg=cfg)
+                       mask_slots=slots, cfg=cfg)
     rng = np.random.default_rng(7)
     tr.keep_sorted_keys = True  # the sorted keys are compared below
     tr.track_active = True      # ... and the realized active set
     p = scene.copy()
     m, v = p.zeros_like(), p.zeros_like()
-    masks_o = {}
+    masks_o, differs_at = {}, {}
     dev = tr.device
-    n_fragile = 0
+    tx = tr.tx
+    d_counts = torch.zeros(max(window or 1, 1), dtype=torch.int64, device=dev)
     for s in range(steps):
         view = views[s % len(views)]
         cam = w.cameras[view]
         tgt = w.target(view)
-        pre = p.copy()  # parameters this view was rendered with
-        o = oracle32.view_step(p, m, v, cam, tgt, w.lr, w.beta1, w.beta2, w.eps, s + 1)
         tr.target.copy_(torch.from_numpy(tgt).to(dev))
-        slot = s % len(views)
-        tr.view_step(B.make_camera(cam), s + 1, w.lr, w.beta1, w.beta2, w.eps, slot=slot)
+        slot = s % slots
+        pairs = window_pairs(s, window, slots) if window else []
+        d_pairs = torch.tensor(pairs if pairs else [(0, 0)], dtype=torch.int32, device=dev)
+        tr.view_step(B.make_camera(cam), s + 1, w.lr, w.beta1, w.beta2, w.eps, slot=slot, d_pairs=d_pairs,
+                     n_pairs=len(pairs), d_counts=d_counts)
         G.poll_ok(tr)
-        # integer decisions of the projection may legitimately differ only on primitives that sit within a few
-        # float ulps of a threshold; when none differs, every integer output of the chain must be bit exact
-        fragile_prims = o["proj"].margin < 2e-6
-        tt_dev = G.u32(tr.proj.tiles_touched)[:n]
-        differs = tt_dev != o["proj"].tiles_touched
-        assert not (differs & ~fragile_prims).any()
-        n_fragile += int(differs.sum())
         vdev = int(tr.count.item())
-        if not differs.any():
-            # identical projected decisions: integer outputs are bit exact through the whole chain
-            assert vdev == len(o["idx"])
-            assert np.array_equal(G.u32(tr.idx)[:vdev], o["idx"])
-            assert np.array_equal(G.u32(tr.masks[slot])[: len(o["mask"])], o["mask"])
-            assert np.array_equal(G.u32(tr.proj.prim_id)[:vdev], o["idx"])
-            mm = len(o["keys"])
-            assert int(tr.proj.num_instances.item()) == mm
-            rg = G.u32(tr.ranges)
-            assert np.array_equal(rg[:, 1] - rg[:, 0], o["ranges"][:, 1] - o["ranges"][:, 0])
-            # keys: tile ids are exact; depth bits come from the GPU projection (may differ in the last bit)
-            assert np.array_equal(G.u64(tr.keys)[:mm] >> np.uint64(32), o["keys"] >> np.uint64(32))
-        # realized active set of the view (row flags of the backward pass): inside the touched set; against the oracle
-        # it may differ only by primitives whose activity hangs on a fragile pixel decision
+        idx_dev = G.u32(tr.idx)[:vdev]
+        names = ("means", "log_scales", "quats", "opacity_logit", "sh")
+        # the state this view starts from: all of it for the parameters, the device's touched rows of the moments
+        pre = p.copy()
+        pre_rows = [wl.Scene(scene.sh_degree, *(np.ascontiguousarray(getattr(st, nm)[idx_dev]) for nm in names))
+                    for st in (p, m, v)]
+        o = oracle32.view_step(p, m, v, cam, tgt, w.lr, w.beta1, w.beta2, w.eps, s + 1)
+        # ---- integer outputs.  Tile counts may differ only on primitives within a few ulp of a projection decision;
+        # with those primitives removed from both sides every integer output of the chain is bit exact.
+        tt_dev = G.u32(tr.proj.tiles_touched)[:n]
+        tt_o = o["proj"].tiles_touched
+        differs = tt_dev != tt_o
+        assert not (differs & ~(o["proj"].margin < FRAGILE_PRIM)).any()
+        D = np.flatnonzero(differs)
+        differs_at[s] = len(D)
+        keep = ~differs
+        assert vdev == int(np.count_nonzero(tt_dev)) and np.array_equal(idx_dev, np.flatnonzero(tt_dev))
+        assert np.array_equal(idx_dev[keep[idx_dev]], o["idx"][keep[o["idx"]]])
+        assert np.array_equal(G.u32(tr.proj.prim_id)[:vdev], idx_dev)
+        d_mask = oracle_mod.ids_to_mask(D, n)
+        assert not ((G.u32(tr.masks[slot])[: len(o["mask"])] ^ o["mask"]) & ~d_mask).any()
+        mm_dev, mm_o = int(tr.proj.num_instances.item()), len(o["keys"])
+        assert mm_dev - int(tt_dev[D].sum()) == mm_o - int(tt_o[D].sum())
+        keys_dev = G.u64(tr.keys)[:mm_dev]
+        prims_dev = idx_dev[G.u32(tr.vals)[:mm_dev]]
+        tiles_dev = (keys_dev >> np.uint64(32)).astype(np.int64)
+        # the device's list is a valid stable sort of its own keys: keys ascend, equal keys keep ascending primitive
+        # order, the low word is the bit pattern of the device's own depth, the ranges cut it at the tile changes
+        assert np.all(keys_dev[1:] >= keys_dev[:-1])
+        assert np.all((keys_dev[1:] > keys_dev[:-1]) | (prims_dev[1:] > prims_dev[:-1]))
+        depth_bits = G.u32(tr.proj.depth)[:vdev]
+        assert np.array_equal((keys_dev & np.uint64(0xFFFFFFFF)).astype(np.uint32), depth_bits[G.u32(tr.vals)[:mm_dev]])
+        rg = G.u32(tr.ranges).astype(np.int64)
+        lens = rg[:, 1] - rg[:, 0]
+        assert lens.min() >= 0 and int(lens.sum()) == mm_dev
+        assert np.array_equal(np.repeat(np.arange(len(rg)), lens), tiles_dev)
+        assert np.array_equal(rg[lens > 0, 0], (np.cumsum(lens) - lens)[lens > 0])
+        # ... and holds exactly the oracle's (tile, primitive) pairs.  (The order inside a tile follows the device's
+        # own depth bits, which may differ from the oracle's in the last place.)
+        tiles_o = (o["keys"] >> np.uint64(32)).astype(np.int64)
+        same_depth = len(D) == 0 and np.array_equal(depth_bits, o["proj"].depth[o["idx"]].view(np.uint32))
+        if same_depth:  # identical decisions and depth bits: the sorted sequence is the oracle's, position by position
+            assert np.array_equal(keys_dev, o["keys"]) and np.array_equal(prims_dev, o["vals"])
+        else:
+            pairs_dev = np.sort((tiles_dev << 32 | prims_dev.astype(np.int64))[keep[prims_dev]])
+            pairs_o = np.sort((tiles_o << 32 | o["vals"].astype(np.int64))[keep[o["vals"]]])
+            assert np.array_equal(pairs_dev, pairs_o)
+            del pairs_dev, pairs_o
+        if pairs:
+            want = np.array([oracle32.conflict_count(o["idx"], masks_o[b]) for _, b in pairs], np.int64)
+            got = G.u64(d_counts)[: len(pairs)].astype(np.int64)
+            slack = np.array([len(D) + differs_at[s - j] for j in range(1, len(pairs) + 1)])
+            assert np.all(np.abs(got - want) <= slack), (got, want, slack)
+        masks_o[slot] = o["idx"]
+        # ---- what a differing primitive can reach: the tiles of its rectangle on either side, the pixels in them and
+        # every primitive listed there
+        aff_pix = np.zeros(o["final_T"].shape, bool)
+        aff_prims = np.zeros(n, bool)
+        if len(D):
+            rect_dev = tr.proj.rect.cpu().numpy().view(np.uint16)[:vdev]
+            tile_hit = np.zeros(len(rg), bool)
+            grid = tile_hit.reshape(-1, tx)
+            for pr in D:  # the tiles that one side lists for the primitive and the other does not
+                cover = np.zeros((2,) + grid.shape, bool)
+                if tt_o[pr]:
+                    x0, y0, x1, y1 = o["proj"].rect[pr]
+                    cover[0, y0:y1, x0:x1] = True
+                if tt_dev[pr]:
+                    x0, y0, x1, y1 = rect_dev[np.searchsorted(idx_dev, pr)].astype(np.int64)
+                    cover[1, y0:y1, x0:x1] = True
+                grid |= cover[0] ^ cover[1]
+            aff_pix = np.repeat(np.repeat(grid, 16, axis=0), 16, axis=1)[: aff_pix.shape[0], : aff_pix.shape[1]]
+            aff_prims[o["vals"][tile_hit[tiles_o]]] = True
+            aff_prims[D] = True
+        # ---- fragile pixels: a decision within PIX_MARGIN of its threshold may fall the other way on the device; the
+        # primitives in the walked prefix of such a pixel's list are exempt from the gradient comparison
+        ncon_dev = G.u32(tr.n_contrib)
+        robust = (o["pix_margin"] > PIX_MARGIN) & ~aff_pix
+        fragile_yx = np.argwhere(~robust & ~aff_pix)
+        upto = np.maximum(o["n_contrib"], ncon_dev)[tuple(fragile_yx.T)] + 1 if len(fragile_yx) else []
+        frag_prims = np.zeros(n, bool)
+        frag_prims[G.blended_at_pixels(o, fragile_yx, upto, tx)] = True
+        exempt = frag_prims | aff_prims
+        # ---- realized active set (row flags of the backward pass): inside the touched set; it differs from the
+        # oracle's only by primitives on fragile pixels or in the tiles of a differing primitive
         tr.active_set(slot=slot)
         G.poll_ok(tr)
         n_act = int(tr.active_count.item())
         act_dev = G.u32(tr.active_idx)[:n_act]
         assert not (G.u32(tr.active_masks[slot]) & ~G.u32(tr.masks[slot])).any()
-        if not differs.any():
-            _, act_o = oracle32.realized_active(o["proj"], o["vals"], o["ranges"], cam, o["n_contrib"])
-            n_fragile_pix = int((o["pix_margin"] <= 2e-5).sum())
-            assert len(np.setxor1d(act_dev, act_o)) <= max(4, n_fragile_pix)
-            assert len(act_o) > 0
-        robust = o["pix_margin"] > 1e-3
+        _, act_o = oracle32.realized_active(o["proj"], o["vals"], o["ranges"], cam, o["n_contrib"])
+        act_diff = np.setxor1d(act_dev, act_o)
+        assert exempt[act_diff].all(), (len(act_diff), int((~exempt[act_diff]).sum()))
+        assert len(act_o) > 0
+        # ---- pixels and loss
         out = tr.out.cpu().numpy()
-        assert np.abs(out - o["out"])[:, robust].max() < 1e-4
+        pix_err = np.abs(out - o["out"])
+        fragile_frac = float((o["pix_margin"] <= PIX_MARGIN).mean())
+        assert fragile_frac <= max_fragile and aff_pix.mean() <= 0.02, (fragile_frac, float(aff_pix.mean()), len(D))
+        assert pix_err[:, robust].max() < 1e-4
+        assert np.array_equal(ncon_dev[robust], o["n_contrib"][robust])
+        assert pix_err[:, ~aff_pix].max() < 5e-3
         assert abs(float(tr.loss.item()) - o["loss"]) < 1e-5
-        # updated state: compare the touched rows of params, m, v
+        # ---- gradient rows
         idx = o["idx"].astype(np.int64)
-        host_state = [a for s_ in (p, m, v) for a in (s_.means, s_.log_scales, s_.quats, s_.opacity_logit, s_.sh)]
-        dev_tensors = [t for s_ in (tr.params, tr.m, tr.v) for t in s_.tensors()]
-        un = np.setdiff1d(np.arange(n), idx)
-        if len(un) > 2_000_000:  # the largest scenes: a seeded sample of the untouched rows
-            un = np.sort(rng.choice(un, 2_000_000, replace=False))
-        un_dev, idx_dev = torch.from_numpy(un).to(dev), torch.from_numpy(idx).to(dev)
-        for t, h in zip(dev_tensors, host_state):
-            # untouched rows identical to the oracle's (which never changed them)
-            assert np.array_equal(t[un_dev].cpu().numpy().view(np.uint32), h[un].view(np.uint32))
-        dev_rows = [t[idx_dev].cpu().numpy() for t in dev_tensors]    # the touched rows, in row order
-        host_rows = [h[idx] for h in host_state]
-        # gradient rows: every word inside the bar derived from the un-cancelled term sums (see gpu_util)
+        sel = keep[idx]                      # rows of primitives both sides list
+        rows_of_dev = np.searchsorted(idx_dev, idx[sel])
         _, g2d_abs = oracle32.render_bwd_blend(o["proj"], o["vals"], o["ranges"], cam, o["final_T"], o["n_contrib"],
                                                o["dL_dout"], want_abs=True)
-        rows = o["rows"].astype(np.float64)
-        rows_dev = tr.gradient_rows(len(idx)).astype(np.float64)
-        if not differs.any():
-            bound = G.rows_bound(oracle32, pre, cam, o["idx"], o["proj"].clamp_flags, rows, o["g2d"], g2d_abs)
-            # the chained run also carries the device's own projection and pixel rounding into the gradients
-            assert (np.abs(rows_dev - rows) <= 4 * bound).mean() > 0.9999
-        # Adam state and parameters.  With eps = 1e-15 a first Adam step is ~ lr * sign(g), so a gradient word that is
-        # rounding noise (a cancelled sum) can legitimately move its parameter the other way: compare m, v and the
-        # parameters wherever the two gradients agree to 1e-3 relative, and require that to be the bulk of the words.
+        rows = o["rows"].astype(np.float64)[sel]
+        rows_dev = tr.gradient_rows(vdev).astype(np.float64)[rows_of_dev]
+        bound = G.rows_bound(oracle32, pre, cam, o["idx"], o["proj"].clamp_flags, o["rows"].astype(np.float64), o["g2d"],
+                             g2d_abs)[sel]
+        err = np.abs(rows_dev - rows)
+        checked = ~exempt[idx[sel]]
+        ratio = (err / bound)[checked]
+        plain = (err <= 1e-3 * np.abs(rows) + 1e-5)[checked]
+        rel_only = (err <= 1e-3 * np.abs(rows))[checked]
+        wr, wc = np.unravel_index(np.argmax(np.where(checked[:, None], err / bound, 0)), err.shape)
+        G.report(f"{tag}[step {s}] rows", over_1x=float((ratio > 1).mean()), over_4x=float((ratio > 4).mean()),
+                 over_10x=float((ratio > 10).mean()), worst=float(ratio.max()), worst_col=int(wc),
+                 worst_oracle=float(rows[wr, wc]), worst_dev=float(rows_dev[wr, wc]), worst_bound=float(bound[wr, wc]),
+                 worst_row_absmax=float(np.abs(rows[wr]).max()))
+        assert ratio.max() <= ROWS_SLACK, ratio.max()
+        assert plain.all()  # the loss gradient is +-1/(3HW): north_star's plain bar holds for every word
+        # ---- Adam, every touched word: the oracle's update applied to the device's own gradient rows
+        qa, qm, qv = pre_rows  # compact: row r of these belongs to primitive idx_dev[r]
+        g_dev_rows = tr.gradient_rows(vdev).astype(np.float32)
+        # the first moment is a sum of two terms that may cancel: its error is judged against the terms
+        k3 = 3 * scene.sh_k
+        m_terms = dict(zip(names, (w.beta1 * np.abs(getattr(qm, nm)).astype(np.float64) for nm in names)))
+        g_parts = dict(means=g_dev_rows[:, 0:3], log_scales=g_dev_rows[:, 3:6], quats=g_dev_rows[:, 6:10],
+                       opacity_logit=g_dev_rows[:, 10], sh=g_dev_rows[:, 11:11 + k3].reshape(vdev, scene.sh_k, 3))
+        oracle32.sparse_adam(qa, qm, qv, g_dev_rows, np.arange(vdev, dtype=np.uint32), w.lr, w.beta1, w.beta2, w.eps,
+                             s + 1)
+        idx_dev_t = torch.from_numpy(idx_dev.astype(np.int64)).to(dev)
+        worst_adam = 0.0
+        for s_dev, s_q, kind in ((tr.params, qa, "p"), (tr.m, qm, "m"), (tr.v, qv, "v")):
+            for t, name in zip(s_dev.tensors(), names):
+                got = t[idx_dev_t].cpu().numpy().astype(np.float64)
+                want = getattr(s_q, name).astype(np.float64)
+                tol = 2e-5 * np.abs(want) + 1e-30
+                if kind == "p":  # the update itself is bounded by ~lr: compare on the scale of the step as well
+                    tol = tol + 2e-5 * float(w.lr.max())
+                if kind == "m":
+                    tol = tol + 2e-5 * (m_terms[name] + (1 - w.beta1) * np.abs(g_parts[name]).astype(np.float64))
+                worst_adam = max(worst_adam, float((np.abs(got - want) / tol).max()))
+        assert worst_adam <= 1.0, worst_adam
+        # ---- untouched rows identical to the oracle's (which never changed them)
+        host_state = [a for s_ in (p, m, v) for a in (s_.means, s_.log_scales, s_.quats, s_.opacity_logit, s_.sh)]
+        dev_tensors = [t for s_ in (tr.params, tr.m, tr.v) for t in s_.tensors()]
+        touched_either = np.zeros(n, bool)
+        touched_either[idx] = True
+        touched_either[idx_dev] = True
+        un = np.flatnonzero(~touched_either)
+        if len(un) > 2_000_000:  # the largest scenes: a seeded sample of the untouched rows
+            un = np.sort(rng.choice(un, 2_000_000, replace=False))
+        un_dev = torch.from_numpy(un).to(dev)
+        for t, h in zip(dev_tensors, host_state):
+            assert np.array_equal(t[un_dev].cpu().numpy().view(np.uint32), h[un].view(np.uint32))
+        # ---- chained state against the oracle's own, wherever the two gradients agree to 1e-3 relative.  With
+        # eps = 1e-15 a first Adam step is ~ lr * sign(g), so a gradient word that is rounding noise (a cancelled sum)
+        # may move its parameter the other way; those words are covered by the check above.
+        both = idx[sel]
+        both_dev = torch.from_numpy(both).to(dev)
         agree = np.abs(rows_dev - rows) <= 1e-3 * np.abs(rows)
-        assert agree.mean() > 0.9, agree.mean()
 
-        def as_rows(st):
-            return np.concatenate([st[0], st[1], st[2], st[3][:, None], st[4].reshape(len(idx), -1)],
+        def as_rows(parts):
+            return np.concatenate([parts[0], parts[1], parts[2], parts[3][:, None], parts[4].reshape(len(both), -1)],
                                   axis=1).astype(np.float64)
 
         g_abs = np.abs(rows)
-        dp, hp = as_rows(dev_rows[0:5]), as_rows(host_rows[0:5])
-        dm, hm = as_rows(dev_rows[5:10]), as_rows(host_rows[5:10])
-        dv, hv = as_rows(dev_rows[10:15]), as_rows(host_rows[10:15])
+        dp, dm, dv = (as_rows([t[both_dev].cpu().numpy() for t in st.tensors()]) for st in (tr.params, tr.m, tr.v))
+        hp, hm, hv = (as_rows([getattr(st, nm)[both] for nm in names]) for st in (p, m, v))
         assert np.all(np.abs(dm - hm)[agree] <= (1e-3 * (1 - w.beta1) * g_abs + 1e-6 * np.abs(hm) + 1e-30)[agree])
         assert np.all(np.abs(dv - hv)[agree] <= (2.1e-3 * (1 - w.beta2) * g_abs ** 2 + 1e-6 * np.abs(hv) + 1e-30)[agree])
         assert np.all(np.abs(dp - hp)[agree] <= 1e-3 * np.abs(hp)[agree] + 1e-5)
-        masks_o[slot] = o["idx"]
+        G.report(f"{tag}[step {s}]", V=vdev, M=mm_dev, differing_prims=len(D), fragile_prims_within_2e6=int(
+                 (o["proj"].margin < FRAGILE_PRIM).sum()), same_depth_bits=bool(same_depth),
+                 affected_tiles_pixels=int(aff_pix.sum()), robust_pixels=float(robust.mean()), fragile_pixels=fragile_frac,
+                 pix_err_robust=float(pix_err[:, robust].max()), pix_err_all=float(pix_err[:, ~aff_pix].max()),
+                 active_o=len(act_o), active_diff=len(act_diff), rows_checked=float(checked.mean()),
+                 rows_within_1x=float((ratio <= 1).mean()), rows_within_2x=float((ratio <= 2).mean()),
+                 rows_worst=float(ratio.max()), plain_bar=float(plain.mean()), rel_1e3_no_floor=float(rel_only.mean()),
+                 grads_agree=float(agree.mean()), adam_worst_of_2e5=worst_adam)
         # re-synchronise the oracle's state from the device
         for s_dev, s_host in ((tr.params, p), (tr.m, m), (tr.v, v)):
             for t, a in zip(s_dev.tensors(), (s_host.means, s_host.log_scales, s_host.quats, s_host.opacity_logit, s_host.sh)):
                 a[...] = t.cpu().numpy()
-    # conflict counts over the latest mask of every view slot
-    slots = sorted(masks_o)
-    pairs = np.array([(a, b) for a in slots for b in slots if a < b], np.uint32).reshape(-1, 2)
-    if len(pairs):
-        d_pairs = torch.from_numpy(pairs.view(np.int32)).to(dev)
-        d_counts = torch.zeros(len(pairs), dtype=torch.int64, device=dev)
-        tr.conflict_count(d_pairs, len(pairs), d_counts)
-        G.poll_ok(tr)
-        want = np.array([oracle32.conflict_count(masks_o[a], masks_o[b]) for a, b in pairs], np.uint64)
-        got = G.u64(d_counts)
-        if n_fragile == 0:
-            assert np.array_equal(got, want)
-        else:
-            assert np.all(np.abs(got.astype(np.int64) - want.astype(np.int64)) <= n_fragile)
+    if window is None:
+        # conflict counts over the latest mask of every view slot
+        used = sorted(masks_o)
+        pairs = np.array([(a, b) for a in used for b in used if a < b], np.uint32).reshape(-1, 2)
+        if len(pairs):
+            d_pairs = torch.from_numpy(pairs.view(np.int32)).to(dev)
+            d_counts = torch.zeros(len(pairs), dtype=torch.int64, device=dev)
+            tr.conflict_count(d_pairs, len(pairs), d_counts)
+            G.poll_ok(tr)
+            want = np.array([oracle32.conflict_count(masks_o[a], masks_o[b]) for a, b in pairs], np.int64)
+            got = G.u64(d_counts).astype(np.int64)
+            last = {sl: max(st for st in differs_at if st % slots == sl) for sl in used}
+            slack = np.array([differs_at[last[a]] + differs_at[last[b]] for a, b in pairs])
+            assert np.all(np.abs(got - want) <= slack), (got, want, slack)
     tr.close()
 
 
 def test_chain_cfg1_one_step(oracle32):
-    run_chain(oracle32, wl.make_workload(1), steps=1, views=[0])
+    run_chain(oracle32, wl.make_workload(1), steps=1, views=[0], tag="cfg1")
 
 
 def test_chain_cfg2_ten_steps_all_pairs(oracle32):
     # 100k splats, 8 orbit views, 10 steps cycling the views, then the 28 pairwise intersection counts
-    run_chain(oracle32, wl.make_workload(2), steps=10, views=list(range(8)))
+    run_chain(oracle32, wl.make_workload(2), steps=10, views=list(range(8)), tag="cfg2")
 
 
 def test_chain_unbounded_scene_scaled(oracle32):
     w = wl.make_workload(3, n=100_000, n_cameras=4, resolution=(400, 267))
-    run_chain(oracle32, w, steps=3, views=[0, 1, 2])
+    run_chain(oracle32, w, steps=3, views=[0, 1, 2], tag="cfg3_scaled")
+
+
+def test_chain_cfg4_scaled_with_the_window_of_four(oracle32):
+    """Preset 4 (larger splats, 1080p aspect, conflict counts against the previous 4 views) at a size the oracle
+    finishes in seconds: 7 steps over 7 cameras, so the window is full from step 4 on and a mask slot is reused."""
+    w = wl.make_workload(4, n=250_000, n_cameras=8, resolution=(960, 540))
+    assert w.conflict_window == 4
+    run_chain(oracle32, w, steps=7, views=list(range(7)), window=w.conflict_window, tag="cfg4_scaled")
 
 
 def test_chain_city_scaled(oracle32):
     w = wl.make_workload(5, n=300_000, n_cameras=4, resolution=(480, 270))
-    run_chain(oracle32, w, steps=2, views=[0, 1])
+    run_chain(oracle32, w, steps=2, views=[0, 1], tag="cfg5_scaled")
 
 
 def test_train_from_host_equals_the_plain_loop():
@@ -193,7 +344,7 @@ def test_chain_tight_extent_binning(oracle32):
     from test_gpu_stages import tight_oracle
 
     w = wl.make_workload(3, n=100_000, n_cameras=4, resolution=(400, 267))
-    run_chain(tight_oracle(), w, steps=3, views=[0, 1, 2], cfg=B.default_config(binning=1))
+    run_chain(tight_oracle(), w, steps=3, views=[0, 1, 2], cfg=B.default_config(binning=1), tag="cfg3_scaled_binning1")
     cam = w.cameras[1]
     outs, m = [], []
     for binning in (0, 1):
@@ -217,7 +368,17 @@ def test_chain_cfg3_full_size_as_benchmarked(oracle32):
 
     w = wl.make_workload(3)
     run_chain(oracle32, w, steps=2, views=[0, 1], row_capacity=int(bench.ROW_CAP_FRAC[3] * w.scene.n),
-              instance_capacity=bench.INSTANCE_CAP[3])
+              instance_capacity=bench.INSTANCE_CAP[3], tag="cfg3_full")
+
+
+def test_chain_cfg4_full_size_one_step(oracle32):
+    """Preset 4 at full size (5 M primitives, 1080p, 2.7e8 instances; the oracle's stable sort of them takes minutes),
+    one step with the capacities bench.py launches it with."""
+    import bench
+
+    w = wl.make_workload(4)
+    run_chain(oracle32, w, steps=1, views=[0], window=w.conflict_window, row_capacity=int(bench.ROW_CAP_FRAC[4] * w.scene.n),
+              instance_capacity=bench.INSTANCE_CAP[4], tag="cfg4_full")
 
 
 def test_chain_cfg5_full_size_as_benchmarked(oracle32):
@@ -225,4 +386,5 @@ def test_chain_cfg5_full_size_as_benchmarked(oracle32):
 
     w = wl.make_workload(5)
     row_cap = min(w.scene.n, max(int(bench.ROW_CAP_FRAC[5] * w.scene.n), 1_600_000))
-    run_chain(oracle32, w, steps=2, views=[0, 1], row_capacity=row_cap, instance_capacity=bench.INSTANCE_CAP[5])
+    run_chain(oracle32, w, steps=2, views=[0, 1], row_capacity=row_cap, instance_capacity=bench.INSTANCE_CAP[5],
+              tag="cfg5_full")

@@ -458,12 +458,14 @@ def check_backward(oracle32, scene, cam, seed=0, min_robust=1 - 2e-3, extra_rend
         bound = G.rows_bound(oracle32, scene, cam, f["idx"], f["proj"].clamp_flags, rows_o, g2d_o, g2d_abs)
         err = np.abs(rows - rows_o)
         bad = err > bound
-        # the bound does not see cancellation INSIDE a Jacobian entry (e.g. the conic-to-covariance step of a nearly
-        # degenerate conic), where oracle and device both round in fp32: allow 1e-4 of the words up to 10x the bound
-        assert bad.mean() < 1e-4 and not (err > 10 * bound).any(), (
-            int(bad.sum()), np.argwhere(bad)[:5], err[bad][:5], rows_o[bad][:5], bound[bad][:5])
-        # most words are not cancelled sums and meet the plain bar: 1e-3 relative with a 1e-5 absolute floor
         plain = err <= 1e-3 * np.abs(rows_o) + 1e-5
+        G.report("bwd_stage rows", words=err.size, over_1x=float(bad.mean()), worst=float((err / bound).max()),
+                 plain_bar=float(plain.mean()), rows_absmax=float(np.abs(rows_o).max()))
+        # every word inside the bar (it includes a few ulp of the row's largest word for the cancellation inside a
+        # Jacobian entry, e.g. the conic-to-covariance step of a nearly degenerate conic)
+        assert not bad.any(), (int(bad.sum()), np.argwhere(bad)[:5], err[bad][:5], rows_o[bad][:5], bound[bad][:5])
+        # with an incoming gradient of O(1) per pixel (not the 1/(3HW) of a real loss) the words are sums of hundreds
+        # of O(1) terms; those that are not cancelled sums also meet the plain bar: 1e-3 relative, 1e-5 absolute floor
         assert plain.mean() > 0.999, plain.mean()
     tr.close()
 
