@@ -114,6 +114,14 @@ const char* odin_status_string(int status);
  * clears it. */
 int odin_poll(odin_ctx* ctx, void* stream);
 
+/* Number of unsuccessful polls after which a device-side wait of this context's later calls gives up (the look-back of
+ * the prefix scans and of the radix sort waits for a word another thread block publishes).  Default 2^22, far beyond
+ * anything a healthy launch needs.  A wait that gives up defers ODIN_ERR_TIMEOUT, the kernel carries on with clamped
+ * addresses and returns; the outputs of that call are then invalid but nothing is written outside the caller's
+ * buffers.  0 makes a wait give up the first time it finds its predecessor unpublished: for diagnostics and tests of
+ * the timeout path.  polls in [0, 2^30]. */
+int odin_set_wait_limit(odin_ctx* ctx, int polls);
+
 /* Workspace size sufficient for odin_project, odin_touched_set and odin_bin_sort with at most n primitives and
  * `max_instances` instance capacity. */
 int odin_workspace_bytes(const odin_ctx* ctx, uint32_t n, uint64_t max_instances, size_t* bytes);
@@ -168,8 +176,12 @@ int odin_touched_set(odin_ctx* ctx, const uint32_t* d_tiles_touched, uint32_t n,
  *  - n may be at most 33,554,432 (2^25) primitives; a larger n returns ODIN_ERR_INVALID_ARG and nothing is launched.
  *  - d_status (device int, may be NULL) is where a deferred ODIN_ERR_CAPACITY / ODIN_ERR_TIMEOUT is written (only if it
  *    holds 0, so clear it beforehand); with NULL those conditions are dropped (outputs are still truncated safely).
- *  - The first call on each device also looks up the array's device address; make that first call before any stream
- *    capture begins.
+ *  - The first call on each device also looks up the array's device address, which may make the CUDA runtime load the
+ *    library's device code onto that GPU (that is when the array itself comes into being, and the runtime may
+ *    synchronise the device while it does so).  Treat the first call per device as a warm-up: make it during
+ *    start-up, before the phase in which nothing may allocate begins and before any stream capture.
+ *  - The block size is chosen for the 148 SMs of a B200 (there is no context to ask); on another GPU the result is the
+ *    same, only the split of the work differs.
  *  - Every call on a device shares the one array.  The call clears the part it uses, but two calls whose kernels
  *    overlap on the GPU (different streams, different host threads) race on it: serialise them. */
 int odin_touched_set_static(const uint32_t* d_tiles_touched, uint32_t n, uint32_t* d_mask, uint32_t* d_idx,
@@ -246,8 +258,8 @@ int odin_conflict_count(odin_ctx* ctx, const uint32_t* d_masks, uint32_t n_masks
  * d_evidence_sum [1] (double) = sum of the evidence over C_i (mean = sum / count).
  * evidence_mode 0: Euclidean norm of the gradient with respect to the projected centre, sqrt(g_u^2 + g_v^2) of
  * d_grad2d (the quantity point-based pipelines accumulate per primitive); 1: Euclidean norm of the whole gradient row
- * (grad_rows, required in this mode).  The paper says "after the pipeline's normal gradient scaling" without fixing
- * the norm; both readings are offered.  n = number of primitives of the pool. */
+ * (grad_rows, required in this mode).  Sec. 2.1 / Sec. 4.3 leave the norm of g(p) open, so both readings are
+ * offered.  n = number of primitives of the pool. */
 int odin_active_set(odin_ctx* ctx, const odin_projected* proj, const uint8_t* d_row_active, const float* d_grad2d,
                     const odin_scene* grad_rows, int evidence_mode, uint32_t n, uint32_t* d_mask, uint32_t* d_idx,
                     uint32_t idx_capacity, uint32_t* d_count, float* d_evidence, double* d_evidence_sum, void* ws,

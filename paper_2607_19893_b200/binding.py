@@ -28,7 +28,7 @@ EXPORTS = [
     "odin_touched_set", "odin_bin_sort", "odin_render_fwd", "odin_l1_loss", "odin_render_bwd", "odin_sparse_adam",
     "odin_conflict_count", "odin_kernel_count", "odin_kernel_name", "odin_profile_enable", "odin_profile_collect",
     "odin_touched_set_static", "odin_render_workspace_bytes", "odin_active_set", "odin_mask_union", "odin_hazard_count",
-    "odin_delayed_read_gate", "odin_rlg_weights", "odin_rlg_topk", "odin_sds_scores",
+    "odin_delayed_read_gate", "odin_rlg_weights", "odin_rlg_topk", "odin_sds_scores", "odin_set_wait_limit",
 ]
 
 
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
         L.odin_create.argtypes = [C.POINTER(vp), i32, C.POINTER(odin_config)]
         L.odin_destroy.argtypes = [vp]
         L.odin_poll.argtypes = [vp, vp]
+        L.odin_set_wait_limit.argtypes = [vp, i32]
         L.odin_workspace_bytes.argtypes = [vp, u32, u64, C.POINTER(C.c_size_t)]
         L.odin_project.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_camera), C.POINTER(odin_projected), vp,
                                    C.c_size_t, vp]
@@ -180,6 +181,10 @@ def odin_destroy(ctx) -> None:
 def odin_poll(ctx, stream=None) -> int:
     """Synchronises the stream and returns the deferred device-side status (0 = ok) without raising."""
     return int(lib().odin_poll(ctx, _stream(stream)))
+
+
+def odin_set_wait_limit(ctx, polls: int) -> None:
+    _check(lib().odin_set_wait_limit(ctx, int(polls)), "odin_set_wait_limit")
 
 
 def odin_workspace_bytes(ctx, n: int, max_instances: int) -> int:
@@ -302,13 +307,6 @@ def odin_sds_scores(ctx, d_weights, n_views: int, d_prev_unit, n_prev: int, d_ca
                     stream=None) -> None:
     _check(lib().odin_sds_scores(ctx, _ptr(d_weights), int(n_views), _ptr(d_prev_unit), int(n_prev), _ptr(d_candidates),
                                  int(n_candidates), _ptr(d_scores), _stream(stream)), "odin_sds_scores")
-
-
-def admit_delayed_read(gate, active_count_a: int, tau: float) -> bool:
-    """The admission rule of Sec. 4.3 from the four counts of odin_delayed_read_gate (#D+, #(D+ & C_A), #pass, #R+(B))."""
-    n_delayed, n_with, n_pass, n_read_b = (int(x) for x in gate)
-    return bool(n_read_b > 0 and n_delayed <= tau * n_read_b and active_count_a > 0 and n_with == n_delayed
-                and n_pass == n_delayed)
 
 
 def odin_kernel_count() -> int:

@@ -32,14 +32,16 @@ template <int ROWF, int VEC>
 __global__ void __launch_bounds__(256)
 adam_sh_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v, const float* __restrict__ g,
                const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count, uint32_t cap, AdamK k,
-               const uint8_t* __restrict__ row_zero) {
+               const uint8_t* __restrict__ row_zero, uint32_t n_prims) {
   constexpr int EPR = ROWF / VEC;  // elements per row
   const uint32_t V = min(*count, cap);
   const size_t total = (size_t)V * EPR;
   for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
     const uint32_t r = (uint32_t)(e / EPR);
     const uint32_t j = (uint32_t)(e - (size_t)r * EPR);
-    const size_t dst = (size_t)idx[r] * ROWF + (size_t)j * VEC;
+    const uint32_t prim = idx[r];
+    if (prim >= n_prims) continue;  // an index list that is not a view's own (e.g. after a timed-out scan): no write
+    const size_t dst = (size_t)prim * ROWF + (size_t)j * VEC;
     const bool zero = row_zero && row_zero[r];  // the gradient row was not written: it is zero
     if (VEC == 4) {
       const float4 gg = zero ? make_float4(0.f, 0.f, 0.f, 0.f) : reinterpret_cast<const float4*>(g)[e];
@@ -70,13 +72,14 @@ adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* _
                  float* __restrict__ v_mean, float* __restrict__ v_ls, float4* __restrict__ v_q, float* __restrict__ v_o,
                  const float* __restrict__ g_mean, const float* __restrict__ g_ls, const float4* __restrict__ g_q,
                  const float* __restrict__ g_o, const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count,
-                 uint32_t cap, AdamK k, const uint8_t* __restrict__ row_zero) {
+                 uint32_t cap, AdamK k, const uint8_t* __restrict__ row_zero, uint32_t n_prims) {
   const uint32_t V = min(*count, cap);
   const size_t total = (size_t)V * 4;
   for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
     const uint32_t r = (uint32_t)(e >> 2);
     const int part = (int)(e & 3);
     const size_t d = idx[r];
+    if (d >= n_prims) continue;
     const bool zero = row_zero && row_zero[r];  // the gradient row was not written: it is zero
     if (part < 2) {
       float* __restrict__ p = (part ? p_ls : p_mean) + 3 * d;
@@ -142,10 +145,10 @@ extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m
   {
     OdinKernelScope ks(ctx, K_ADAM_SH, st);
     switch (params->sh_degree) {
-    case 0: adam_sh_kernel<3, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero); break;
-    case 1: adam_sh_kernel<12, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero); break;
-    case 2: adam_sh_kernel<27, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero); break;
-    default: adam_sh_kernel<48, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero); break;
+    case 0: adam_sh_kernel<3, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n); break;
+    case 1: adam_sh_kernel<12, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n); break;
+    case 2: adam_sh_kernel<27, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n); break;
+    default: adam_sh_kernel<48, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n); break;
     }
   }
   size_t gb = ((size_t)cap * 4 + 255) / 256;
@@ -155,6 +158,7 @@ extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m
       params->means, params->log_scales, reinterpret_cast<float4*>(params->quats), params->opacity_logit, m->means,
       m->log_scales, reinterpret_cast<float4*>(m->quats), m->opacity_logit, v->means, v->log_scales,
       reinterpret_cast<float4*>(v->quats), v->opacity_logit, grad_rows->means, grad_rows->log_scales,
-      reinterpret_cast<const float4*>(grad_rows->quats), grad_rows->opacity_logit, d_idx, d_count, cap, k, d_row_zero);
+      reinterpret_cast<const float4*>(grad_rows->quats), grad_rows->opacity_logit, d_idx, d_count, cap, k, d_row_zero,
+      params->n);
   return odin_launch_status();
 }

@@ -30,6 +30,7 @@ extern "C" int odin_create(odin_ctx** out, int device, const odin_config* cfg) {
     return ODIN_ERR_CUDA;
   }
   ctx->sm_count = prop.multiProcessorCount;
+  ctx->spin_limit = ODIN_DEFAULT_SPIN_LIMIT;
   *ctx->h_status = 0;
   *out = ctx;
   return ODIN_OK;
@@ -41,6 +42,13 @@ extern "C" int odin_destroy(odin_ctx* ctx) {
   cudaFreeHost(ctx->h_status);
   for (cudaEvent_t e : ctx->prof.events) cudaEventDestroy(e);
   delete ctx;
+  return ODIN_OK;
+}
+
+extern "C" int odin_set_wait_limit(odin_ctx* ctx, int polls) {
+  if (!ctx) return ODIN_ERR_NULL;
+  if (polls < 0 || polls > (1 << 30)) return ODIN_ERR_INVALID_ARG;
+  ctx->spin_limit = polls;
   return ODIN_OK;
 }
 

@@ -91,7 +91,8 @@ __global__ void __launch_bounds__(OS_THREADS, OS_BLOCKS)
 onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in, uint32_t* __restrict__ keys_out,
                 uint32_t* __restrict__ vals_out, uint64_t* __restrict__ keys64_out, const uint32_t* __restrict__ depth_bits,
                 const uint32_t* __restrict__ count32, const uint64_t* __restrict__ count64, uint64_t capacity, int shift,
-                const uint32_t* __restrict__ digit_base, uint32_t* states, uint32_t* ticket, int* status) {
+                const uint32_t* __restrict__ digit_base, uint32_t* states, uint32_t* ticket, int* status,
+                int spin_limit, uint32_t depth_rows) {
   extern __shared__ __align__(16) unsigned char os_smem[];
   uint32_t* s_keys = reinterpret_cast<uint32_t*>(os_smem);
   constexpr uint32_t TILE = (uint32_t)ITEMS * OS_THREADS;
@@ -221,7 +222,7 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
         }
         if (busy && stalled) {
           __nanosleep(32);
-          if (++spins > ODIN_SPIN_LIMIT) { odin_set_error(status, ODIN_ERR_TIMEOUT); break; }
+          if (++spins > spin_limit) { odin_set_error(status, ODIN_ERR_TIMEOUT); break; }
         }
       }
 #pragma unroll
@@ -258,7 +259,9 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
           if (keys_out) keys_out[dst] = k;
           vals_out[dst] = v;
           if (WIDE) {
-            if (keys64_out) keys64_out[dst] = ((uint64_t)k << 32) | (uint64_t)depth_bits[v];
+            // (depth_rows: length of depth_bits; the clamp only matters for a list that an earlier timed-out pass left
+            // partly unwritten)
+            if (keys64_out) keys64_out[dst] = ((uint64_t)k << 32) | (uint64_t)depth_bits[min(v, depth_rows - 1)];
           }
         }
       }
@@ -289,7 +292,7 @@ __global__ void __launch_bounds__(RO_THREADS)
 sorted_offsets_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __restrict__ rect,
                       const uint32_t* __restrict__ num_rows, uint32_t capacity, int TX, uint32_t* __restrict__ sorted_off,
                       uint32_t* __restrict__ chunk_row, uint32_t chunks_cap, uint32_t* __restrict__ tile_diff,
-                      uint32_t diff_words, uint32_t* ticket, uint64_t* state, int* status) {
+                      uint32_t diff_words, uint32_t* ticket, uint64_t* state, int* status, int spin_limit) {
   // diff_words != 0: the block first accumulates its part of the difference array in shared memory (`diff_words` =
   // tiles + 1 words of dynamic shared memory) and adds the non-zero words to the global one at the end: a tile on which
   // thousands of rectangles pile up would otherwise serialise that many global reductions on one address.
@@ -310,14 +313,16 @@ sorted_offsets_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __
 #pragma unroll
   for (int k = 0; k < RO_ITEMS; ++k) {
     rc[k] = make_ushort4(0, 0, 0, 0);
-    if (first + k < V) rc[k] = rect[sorted_row[first + k]];
+    // (a row id is clamped to the rows of this view: it stays in range even if a pass of the row sort gave up and left
+    // part of its output unwritten)
+    if (first + k < V) rc[k] = rect[min(sorted_row[first + k], V - 1)];
     cnt[k] = ((uint32_t)rc[k].z - (uint32_t)rc[k].x) * ((uint32_t)rc[k].w - (uint32_t)rc[k].y);
     sum += cnt[k];
   }
   uint32_t total;
   const uint32_t before = odin_block_exclusive_sum(sum, s_warp, &total);
   if (threadIdx.x < 32) {
-    const uint64_t b = odin_lookback_u64(state, tile, (uint64_t)total, status);
+    const uint64_t b = odin_lookback_u64(state, tile, (uint64_t)total, status, spin_limit);
     if (threadIdx.x == 0) s_base = (uint32_t)b;
   }
   __syncthreads();
@@ -359,7 +364,7 @@ sorted_offsets_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __
 constexpr int TS_ITEMS = 4;
 
 __device__ __forceinline__ void tile_scan_block(const uint32_t* __restrict__ tile_diff, uint32_t n_tiles, int tile_passes,
-                                                uint32_t* __restrict__ ranges, uint32_t* __restrict__ base) {
+                                                uint32_t* __restrict__ ranges, uint32_t* __restrict__ base, uint32_t cap) {
   __shared__ uint32_t s_h[SORT_MAX_TILE_DIGITS][SORT_RADIX];
   __shared__ uint32_t s_warp[33];
   const unsigned lane = threadIdx.x & 31;
@@ -391,7 +396,8 @@ __device__ __forceinline__ void tile_scan_block(const uint32_t* __restrict__ til
     for (int k = 0; k < TS_ITEMS; ++k) {
       const uint32_t t = t0 + k;
       if (t < n_tiles) {
-        reinterpret_cast<uint2*>(ranges)[t] = make_uint2(off, off + c[k]);
+        // never beyond the instance capacity (the counts already respect it unless a look-back gave up)
+        reinterpret_cast<uint2*>(ranges)[t] = make_uint2(min(off, cap), min(off + c[k], cap));
         if (c[k]) atomicAdd(&s_h[0][t & (SORT_RADIX - 1)], c[k]);
         off += c[k];
       }
@@ -452,7 +458,8 @@ emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* _
                       const uint32_t* __restrict__ tile_diff, uint32_t n_tiles, int tile_passes,
                       uint32_t* __restrict__ ranges, uint32_t* __restrict__ tile_dbase) {
   if (blockIdx.x == 0) {  // block 0: it is scheduled first
-    tile_scan_block(tile_diff, n_tiles, tile_passes, ranges, tile_dbase);
+    tile_scan_block(tile_diff, n_tiles, tile_passes, ranges, tile_dbase,
+                    (uint32_t)(capacity < 0xffffffffull ? capacity : 0xffffffffull));
     return;
   }
   const uint32_t emit_blocks = gridDim.x - 1, emit_block = blockIdx.x - 1;
@@ -472,17 +479,20 @@ emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* _
     const uint32_t c0 = chunk * DUP_CHUNK;
     const uint32_t c1 = (M - c0 < (uint32_t)DUP_CHUNK) ? M : c0 + DUP_CHUNK;
     // first and last position of the chunk from the chunk table; only the last chunk has to search for its end
-    const uint32_t row_lo = chunk_row[chunk];
+    // (every index taken from the tables is clamped: if a look-back gave up, parts of them were never written, and
+    // the emission must still stay inside its buffers; with intact tables the clamps change nothing)
+    const uint32_t row_lo = min(chunk_row[chunk], V - 1);
     uint32_t row_hi;
     if (chunk + 1 < chunks) {
-      const uint32_t rn = chunk_row[chunk + 1];  // position that holds slot c1
-      row_hi = (sorted_off[rn] == c1) ? rn - 1 : rn;
+      const uint32_t rn = min(chunk_row[chunk + 1], V - 1);  // position that holds slot c1
+      row_hi = (sorted_off[rn] == c1 && rn > 0) ? rn - 1 : rn;
     } else {
-      row_hi = block_upper_bound(sorted_off, V, c1 - 1) - 1;  // offset[0] = 0, so the bound is >= 1
+      row_hi = max(block_upper_bound(sorted_off, V, c1 - 1), 1u) - 1;  // offset[0] = 0, so the bound is >= 1
     }
+    row_hi = min(max(row_hi, row_lo), row_lo + (uint32_t)DUP_CHUNK - 1);
     const uint32_t nrows = row_hi - row_lo + 1;  // <= DUP_CHUNK: every row owns at least one slot
     for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS) {
-      const uint32_t r = sorted_row[row_lo + i];
+      const uint32_t r = min(sorted_row[row_lo + i], V - 1);
       s_off[i] = sorted_off[row_lo + i];
       s_row[i] = r;
       s_rect[i] = rect[r];
@@ -491,7 +501,8 @@ emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* _
     for (int i = threadIdx.x; i < DUP_CHUNK; i += DUP_THREADS) s_map[i] = 0;
     __syncthreads();
     // slot -> staged row: every row marks its first slot, an inclusive max-scan fills the rest
-    for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS) s_map[max(s_off[i], c0) - c0] = (uint16_t)i;
+    for (uint32_t i = threadIdx.x; i < nrows; i += DUP_THREADS)
+      s_map[min(max(s_off[i], c0) - c0, (uint32_t)DUP_CHUNK - 1)] = (uint16_t)i;
     __syncthreads();
     {
       static_assert(DUP_ITEMS == 8, "a thread's slots are one 16-byte word of the map");
@@ -614,7 +625,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
       uint32_t* vout = row_vals[p & 1];
       onesweep_kernel<false, OS_ROW_ITEMS, OS_ROW_WINDOW><<<grid, OS_THREADS, OS_ROW_SMEM, st>>>(
           kin, vin, kout, vout, nullptr, nullptr, proj->num_rows, nullptr, 0, p * (int)SORT_RADIX_BITS,
-          dbase + p * SORT_RADIX, row_states + (size_t)p * L.row_tiles * SORT_RADIX, tickets + p, ctx->d_status);
+          dbase + p * SORT_RADIX, row_states + (size_t)p * L.row_tiles * SORT_RADIX, tickets + p, ctx->d_status, ctx->spin_limit, proj->capacity);
       kin = kout;
       vin = vout;
     }
@@ -631,7 +642,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     ODIN_CUDA(cudaFuncSetAttribute(sorted_offsets_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 40001 * 4));
     sorted_offsets_kernel<<<(proj->capacity + OFFSET_TILE - 1) / OFFSET_TILE, RO_THREADS, diff_smem, st>>>(
         sorted_row, rect, proj->num_rows, (uint32_t)capacity, TX, sorted_off, chunk_row, (uint32_t)chunks_cap, tile_diff,
-        diff_words, tickets + 8, scan_state, ctx->d_status);
+        diff_words, tickets + 8, scan_state, ctx->d_status, ctx->spin_limit);
   }
   // the emission goes to the buffers from which `tile_passes` ping-pong steps end in d_vals
   int cur = tile_passes & 1;
@@ -652,12 +663,12 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
       onesweep_kernel<false, OS_INST_ITEMS, OS_INST_WINDOW><<<os_grid, OS_THREADS, OS_SMEM, st>>>(
           inst_keys[cur], inst_vals[cur], inst_keys[cur ^ 1], inst_vals[cur ^ 1], nullptr, nullptr, nullptr,
           proj->num_instances, capacity, p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
-          tickets + SORT_DEPTH_DIGITS + p, ctx->d_status);
+          tickets + SORT_DEPTH_DIGITS + p, ctx->d_status, ctx->spin_limit, proj->capacity);
     else  // the sorted tile ids themselves are not needed any more: the ranges came from the tile counts
       onesweep_kernel<true, OS_INST_ITEMS, OS_INST_WINDOW><<<os_grid, OS_THREADS, OS_SMEM, st>>>(
           inst_keys[cur], inst_vals[cur], nullptr, inst_vals[cur ^ 1], d_keys, depth_bits, nullptr,
           proj->num_instances, capacity, p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
-          tickets + SORT_DEPTH_DIGITS + p, ctx->d_status);
+          tickets + SORT_DEPTH_DIGITS + p, ctx->d_status, ctx->spin_limit, proj->capacity);
     cur ^= 1;
   }
   return odin_launch_status();

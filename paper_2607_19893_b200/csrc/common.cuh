@@ -29,6 +29,7 @@ struct odin_ctx {
   odin_config cfg;
   int* d_status;  // first deferred device-side error (0 = none)
   int* h_status;  // pinned mirror read by odin_poll
+  int spin_limit; // polls after which a device-side wait gives up (odin_set_wait_limit)
   OdinProf prof;
 };
 
@@ -75,9 +76,10 @@ __device__ __forceinline__ void odin_set_error(int* status, int code) { atomicCA
 // Decoupled look-back for single-pass prefix sums.  A tile publishes first its own aggregate, then its inclusive
 // prefix; a later tile walks backwards over its predecessors, adding aggregates until it meets an inclusive prefix.
 // Tiles take their index from an atomic ticket, so every predecessor of a running tile has already started.
-// Every wait is bounded: after ODIN_SPIN_LIMIT polls the walker records ODIN_ERR_TIMEOUT and carries on with what
-// it has (callers clamp every address they derive from the result).
-#define ODIN_SPIN_LIMIT (1 << 22)
+// Every wait is bounded: after `spin_limit` unsuccessful polls (a kernel argument; ODIN_DEFAULT_SPIN_LIMIT unless the
+// context was told otherwise) the walker records ODIN_ERR_TIMEOUT and carries on with what it has (callers clamp every
+// address they derive from the result).
+constexpr int ODIN_DEFAULT_SPIN_LIMIT = 1 << 22;
 
 constexpr uint64_t LB64_FLAG_SHIFT = 62;
 constexpr uint64_t LB64_AGG = 1ull << LB64_FLAG_SHIFT;
@@ -104,7 +106,8 @@ __device__ __forceinline__ void st_volatile_u32(uint32_t* p, uint32_t v) {
 // Called by ONE warp of the tile (all 32 lanes).  state[] has one 64-bit word per tile, zero before the launch.
 // Returns the exclusive prefix (sum of the aggregates of tiles 0..tile-1) in every lane and publishes this tile's
 // inclusive prefix.  `aggregate` must fit 62 bits; two packed counters are fine as long as neither overflows its field.
-__device__ __forceinline__ uint64_t odin_lookback_u64(uint64_t* state, uint32_t tile, uint64_t aggregate, int* status) {
+__device__ __forceinline__ uint64_t odin_lookback_u64(uint64_t* state, uint32_t tile, uint64_t aggregate, int* status,
+                                                      int spin_limit) {
   const unsigned lane = threadIdx.x & 31;
   if (tile == 0) {
     if (lane == 0) st_volatile_u64(&state[0], LB64_INC | aggregate);
@@ -135,7 +138,7 @@ __device__ __forceinline__ uint64_t odin_lookback_u64(uint64_t* state, uint32_t 
       look -= first_invalid;
     } else {
       __nanosleep(64);
-      if (++spins > ODIN_SPIN_LIMIT) {
+      if (++spins > spin_limit) {
         if (lane == 0) odin_set_error(status, ODIN_ERR_TIMEOUT);
         break;
       }

@@ -118,18 +118,25 @@ __global__ void __launch_bounds__(SCAN_THREADS)
 project_scan_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint32_t capacity,
                     uint32_t* __restrict__ prim_id, uint32_t* __restrict__ tile_offset, uint32_t* __restrict__ num_rows,
                     uint64_t* __restrict__ num_instances, uint32_t* ticket, uint64_t* state, int* status,
-                    int scan_rounds) {
+                    int scan_rounds, int spin_limit) {
   const uint32_t scan_chunk = PROJECT_TILE * (uint32_t)scan_rounds;
   __shared__ uint32_t s_tile;
   __shared__ uint64_t s_warp[SCAN_THREADS / 32 + 1];
+  __shared__ uint64_t s_inst[SCAN_THREADS / 32];
   __shared__ uint64_t s_base;
+  unsigned long long* exact_instances = reinterpret_cast<unsigned long long*>(ticket + 2);  // zeroed with the ticket
   if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
   __syncthreads();
   const uint32_t tile = s_tile;
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t chunk_base = tile * scan_chunk;
-  // pass A: packed (rows, instances) total of the chunk, then ONE look-back per scan_chunk primitives
-  uint64_t mine = 0;
+  // pass A: packed (rows, instances) total of the chunk, then ONE look-back per scan_chunk primitives.  The instance
+  // field holds 34 bits, a chunk can reach 2^14 primitives x 2^20 tiles and there are up to 2^14 chunks, so the packed
+  // sums can carry into the row field when the view has 2^32 instances or more (an error by definition).  That case
+  // is caught on a counter of its own: every chunk adds its exact instance count (kept apart in 64 bits, the packed
+  // copy saturated) to a 64-bit total, and whoever sees that total reach 2^32 reports ODIN_ERR_CAPACITY.  The outputs
+  // of such a view are meaningless but every write stays inside the caller's capacities (the row guard below).
+  uint64_t mine = 0, mine_inst = 0;
 #pragma unroll
   for (int rnd = 0; rnd < scan_rounds; ++rnd) {
     const uint32_t warp_base = chunk_base + rnd * PROJECT_TILE + warp * (32 * SCAN_ITEMS);
@@ -137,16 +144,29 @@ project_scan_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint
     for (int j = 0; j < SCAN_ITEMS; ++j) {
       const uint32_t p = warp_base + 32 * j + lane;
       const uint32_t t = (p < n) ? tiles_touched[p] : 0u;
-      mine += t ? ((1ull << PACK_SHIFT) | (uint64_t)t) : 0ull;
+      mine += t ? (1ull << PACK_SHIFT) : 0ull;
+      mine_inst += t;
     }
   }
-  for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
-  if (lane == 0) s_warp[warp] = mine;
+  for (int o = 16; o > 0; o >>= 1) {
+    mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    mine_inst += __shfl_xor_sync(0xffffffffu, mine_inst, o);
+  }
+  if (lane == 0) { s_warp[warp] = mine; s_inst[warp] = mine_inst; }
   __syncthreads();
   if (threadIdx.x < 32) {
     uint64_t total = (lane < SCAN_THREADS / 32) ? s_warp[lane] : 0ull;
-    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-    const uint64_t base = odin_lookback_u64(state, tile, total, status);
+    uint64_t total_inst = (lane < SCAN_THREADS / 32) ? s_inst[lane] : 0ull;
+    for (int o = 16; o > 0; o >>= 1) {
+      total += __shfl_xor_sync(0xffffffffu, total, o);
+      total_inst += __shfl_xor_sync(0xffffffffu, total_inst, o);
+    }
+    if (lane == 0 && total_inst != 0) {
+      const unsigned long long before = atomicAdd(exact_instances, (unsigned long long)total_inst);
+      if (before + total_inst >= (1ull << 32)) odin_set_error(status, ODIN_ERR_CAPACITY);
+    }
+    total |= total_inst < (1ull << 32) ? total_inst : ((1ull << 32) - 1);
+    const uint64_t base = odin_lookback_u64(state, tile, total, status, spin_limit);
     if (lane == 0) {
       s_base = base;
       if (tile == (n + scan_chunk - 1) / scan_chunk - 1) {  // last chunk: totals
@@ -217,11 +237,11 @@ template <int DEG>
 __global__ void __launch_bounds__(128)
 project_rows_kernel(const float* __restrict__ means, const float* __restrict__ log_scales, const float4* __restrict__ quats,
                     const float* __restrict__ opacity_logit, const float* __restrict__ sh, CamParams cam, BinRule rule,
-                    odin_projected out) {
+                    odin_projected out, uint32_t n) {
   constexpr int K = (DEG + 1) * (DEG + 1);
   const uint32_t V = min(*out.num_rows, out.capacity);
   for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
-    const size_t p = out.prim_id[r];
+    const size_t p = min(out.prim_id[r], n - 1);  // in range even if the scan gave up and left part of the map unwritten
     const Footprint f = project_footprint(cam, rule, means, log_scales, quats, opacity_logit, p);
     reinterpret_cast<float2*>(out.xy)[r] = make_float2(f.u, f.v);
     out.depth[r] = f.depth;
@@ -308,7 +328,7 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
     const uint32_t scan_chunk = PROJECT_TILE * (uint32_t)scan_rounds;
     project_scan_kernel<<<(n + scan_chunk - 1) / scan_chunk, SCAN_THREADS, 0, st>>>(
         out->tiles_touched, n, out->capacity, out->prim_id, out->tile_offset, out->num_rows, out->num_instances, ticket,
-        state, ctx->d_status, scan_rounds);
+        state, ctx->d_status, scan_rounds, ctx->spin_limit);
   }
   if (out->capacity == 0) return odin_launch_status();
   const uint32_t blocks_cap = (out->capacity + 127) / 128;
@@ -316,7 +336,7 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   OdinKernelScope ks(ctx, K_PROJECT_ROWS, st);
 #define LAUNCH(D)                                                                                                      \
   project_rows_kernel<D><<<grid, 128, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit, scene->sh, cp, \
-                                               rule, *out)
+                                               rule, *out, n)
   switch (scene->sh_degree) {
     case 0: LAUNCH(0); break;
     case 1: LAUNCH(1); break;

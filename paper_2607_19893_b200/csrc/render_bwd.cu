@@ -55,7 +55,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
                         const BlendRecord* __restrict__ ckpt, uint32_t seg_cap,
                         const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
                         const float* __restrict__ dL, float* __restrict__ g2d, uint32_t* __restrict__ ticket,
-                        uint8_t* __restrict__ row_active) {
+                        uint8_t* __restrict__ row_active, uint32_t row_cap) {
   __shared__ BlendRow s_rowdata[BLEND_WARPS][32];
   __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, power threshold
   __shared__ uint32_t s_rowid[BLEND_WARPS][32];
@@ -135,7 +135,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
     const int cnt = (int)min(32u, total - b);
     bool reach = false;
     if ((int)lane < cnt) {
-      const uint32_t r = vals[seg_start + b + lane];
+      const uint32_t r = min(vals[seg_start + b + lane], row_cap - 1);  // in range whatever the list holds
       const float2 c = xy[r];
       BlendRow row;
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
@@ -228,11 +228,11 @@ render_bwd_project_kernel(const float* __restrict__ means, const float* __restri
                           const uint8_t* __restrict__ clamp_flags, const uint32_t* __restrict__ num_rows, uint32_t capacity,
                           const float* __restrict__ g2d, float* __restrict__ g_means, float* __restrict__ g_ls,
                           float4* __restrict__ g_quats, float* __restrict__ g_opac, float* __restrict__ g_sh,
-                          uint8_t* __restrict__ row_zero) {
+                          uint8_t* __restrict__ row_zero, uint32_t n) {
   constexpr int K = (DEG + 1) * (DEG + 1);
   const uint32_t V = min(*num_rows, capacity);
   for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
-    const size_t p = prim_id[r];
+    const size_t p = min(prim_id[r], n - 1);
     const float* gg = g2d + (size_t)r * 9;
     const float gu = gg[0], gv = gg[1], gA = gg[2], gB = gg[3], gC = gg[4], go = gg[5];
     const float grgb[3] = {gg[6], gg[7], gg[8]};
@@ -425,7 +425,7 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
       reinterpret_cast<const uint32_t*>(base + L.tile_first), header + 2,                                               \
       reinterpret_cast<const uint2*>(base + L.seg_tile), reinterpret_cast<const uint2*>(base + L.seg_link),             \
       reinterpret_cast<const BlendRecord*>(base + L.ckpt), L.segments, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d, ticket,  \
-      d_row_active)
+      d_row_active, proj->capacity)
     if (d_row_active) LAUNCH_BLEND(true);
     else LAUNCH_BLEND(false);
 #undef LAUNCH_BLEND
@@ -438,7 +438,7 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
       scene->means, scene->log_scales, reinterpret_cast<const float4*>(scene->quats), scene->opacity_logit, scene->sh,  \
       cp, ctx->cfg.dilation, proj->prim_id, proj->clamp_flags, proj->num_rows, proj->capacity, d_grad2d,                \
       grad_rows->means, grad_rows->log_scales, reinterpret_cast<float4*>(grad_rows->quats), grad_rows->opacity_logit,    \
-      grad_rows->sh, d_row_zero)
+      grad_rows->sh, d_row_zero, scene->n)
   OdinKernelScope ks(ctx, K_BWD_PROJECT, st);
   switch (scene->sh_degree) {
     case 0: LAUNCH(0); break;

@@ -12,7 +12,7 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
                   const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX, int n_tiles,
                   float bg0, float bg1, float bg2, float alpha_min, float alpha_max, float t_min, float* __restrict__ out,
                   float* __restrict__ final_T, uint32_t* __restrict__ n_contrib, uint32_t* __restrict__ tile_more,
-                  uint32_t* __restrict__ ticket) {
+                  uint32_t* __restrict__ ticket, uint32_t row_cap) {
   __shared__ BlendRow s_row[BLEND_WARPS][32];
   __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, power threshold
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -48,7 +48,7 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
     const uint32_t i = b + lane;
     bool reach = false;
     if (i < end) {
-      const uint32_t r = vals[i];
+      const uint32_t r = min(vals[i], row_cap - 1);  // in range whatever the list holds (e.g. after a timed-out sort)
       const float2 c = xy[r];
       BlendRow row;
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
@@ -132,7 +132,8 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
                        float bg0, float bg1, float bg2, float alpha_min, float alpha_max, float t_min,
                        float* __restrict__ out, float* __restrict__ final_T, uint32_t* __restrict__ n_contrib,
                        uint32_t* __restrict__ tile_first, uint32_t* __restrict__ seg_count, uint2* __restrict__ seg_tile,
-                       uint2* __restrict__ seg_link, BlendRecord* __restrict__ ckpt, uint32_t seg_cap, int* status) {
+                       uint2* __restrict__ seg_link, BlendRecord* __restrict__ ckpt, uint32_t seg_cap, int* status,
+                       uint32_t row_cap) {
   const int tile = blockIdx.x;
   if (!tile_first[tile]) return;
   __shared__ BlendRow s_row[BLEND_TAIL_THREADS];
@@ -172,7 +173,7 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
     float2 bp = make_float2(0.f, 0.f);
     bool reach = false;
     if (i < end) {
-      const uint32_t r = vals[i];
+      const uint32_t r = min(vals[i], row_cap - 1);
       const float2 c = xy[r];
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
       row.q1 = conic_o[r];
@@ -350,7 +351,7 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
         reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
         reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0], cam->bg[1],
         cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_first,
-        header);
+        header, proj->capacity);
   }
   OdinKernelScope ks(ctx, K_FWD_TAIL, st);
   render_fwd_tail_kernel<<<n_tiles, BLEND_TAIL_THREADS, 0, st>>>(
@@ -358,7 +359,7 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
       reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
       ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_first, header + 2,
       reinterpret_cast<uint2*>(base + L.seg_tile), reinterpret_cast<uint2*>(base + L.seg_link),
-      reinterpret_cast<BlendRecord*>(base + L.ckpt), L.segments, ctx->d_status);
+      reinterpret_cast<BlendRecord*>(base + L.ckpt), L.segments, ctx->d_status, proj->capacity);
   return odin_launch_status();
 }
 

@@ -28,7 +28,8 @@ active_set_kernel(const uint8_t* __restrict__ row_active, const uint32_t* __rest
                   const uint32_t* __restrict__ num_rows, uint32_t row_capacity, const float* __restrict__ grad2d,
                   GradRows rows, int evidence_mode, uint32_t* __restrict__ mask, uint32_t* __restrict__ idx,
                   uint32_t idx_capacity, uint32_t* __restrict__ count, float* __restrict__ evidence,
-                  double* __restrict__ evidence_sum, uint32_t* ticket, uint64_t* state, int* status) {
+                  double* __restrict__ evidence_sum, uint32_t* ticket, uint64_t* state, int* status, int spin_limit,
+                  uint32_t n_prims) {
   __shared__ uint32_t s_tile, s_base;
   __shared__ uint32_t s_warp[33];
   __shared__ double s_sum[AS_THREADS / 32];
@@ -46,7 +47,7 @@ active_set_kernel(const uint8_t* __restrict__ row_active, const uint32_t* __rest
   uint32_t total;
   const uint32_t before = odin_block_exclusive_sum(mine, s_warp, &total);
   if (threadIdx.x < 32) {
-    const uint64_t b = odin_lookback_u64(state, tile, (uint64_t)total, status);
+    const uint64_t b = odin_lookback_u64(state, tile, (uint64_t)total, status, spin_limit);
     if (threadIdx.x == 0) {
       s_base = (uint32_t)b;
       if (tile == ntiles - 1) {  // last tile: totals
@@ -64,6 +65,7 @@ active_set_kernel(const uint8_t* __restrict__ row_active, const uint32_t* __rest
     if (!(flags >> k & 1u)) continue;
     const uint32_t r = first + k;
     const uint32_t p = prim_id[r];
+    if (p >= n_prims) { ++pos; continue; }  // a row map that is not this view's own (e.g. after a timed-out scan)
     float ev;
     if (evidence_mode == 0) {
       const float gu = grad2d[(size_t)r * 9], gv = grad2d[(size_t)r * 9 + 1];
@@ -349,7 +351,7 @@ extern "C" int odin_active_set(odin_ctx* ctx, const odin_projected* proj, const 
   OdinKernelScope ks(ctx, K_ACTIVE_SET, st);
   active_set_kernel<<<tiles, AS_THREADS, 0, st>>>(d_row_active, proj->prim_id, proj->num_rows, proj->capacity, d_grad2d,
                                                  rows, evidence_mode, d_mask, d_idx, idx_capacity, d_count, d_evidence,
-                                                 d_evidence_sum, ticket, state, ctx->d_status);
+                                                 d_evidence_sum, ticket, state, ctx->d_status, ctx->spin_limit, n);
   return odin_launch_status();
 }
 

@@ -1,4 +1,6 @@
 // Touched-set bitmask + ascending index list (single pass, decoupled look-back) and pairwise intersection counts.
+#include <atomic>
+
 #include "common.cuh"
 #include "layout.cuh"
 
@@ -16,7 +18,7 @@ constexpr int TS_MAX_ROUNDS = 8;
 __global__ void __launch_bounds__(TS_THREADS)
 touched_set_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint32_t* __restrict__ mask,
                    uint32_t* __restrict__ idx, uint32_t idx_capacity, uint32_t* __restrict__ count, uint32_t* ticket,
-                   uint64_t* state, int* status, int scan_rounds) {
+                   uint64_t* state, int* status, int scan_rounds, int spin_limit) {
   const uint32_t scan_chunk = TOUCHED_TILE * (uint32_t)scan_rounds;
   __shared__ uint32_t s_tile;
   __shared__ uint32_t s_warp[33];
@@ -47,7 +49,7 @@ touched_set_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint3
   const uint32_t scan = odin_block_exclusive_sum(lane == 0 ? warp_count : 0u, s_warp, &chunk_total);
   const uint32_t warp_off = __shfl_sync(0xffffffffu, scan, 0);
   if (threadIdx.x < 32) {
-    const uint64_t ex = odin_lookback_u64(state, tile, (uint64_t)chunk_total, status);
+    const uint64_t ex = odin_lookback_u64(state, tile, (uint64_t)chunk_total, status, spin_limit);
     if (threadIdx.x == 0) s_base = ex;
   }
   __syncthreads();
@@ -129,7 +131,7 @@ extern "C" int odin_touched_set(odin_ctx* ctx, const uint32_t* d_tiles_touched, 
   const uint32_t grid = (n + scan_chunk - 1) / scan_chunk;
   OdinKernelScope ks(ctx, K_TOUCHED, st);
   touched_set_kernel<<<grid, TS_THREADS, 0, st>>>(d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket, state,
-                                                  ctx->d_status, scan_rounds);
+                                                  ctx->d_status, scan_rounds, ctx->spin_limit);
   return odin_launch_status();
 }
 
@@ -146,9 +148,10 @@ constexpr size_t TS_STATIC_BYTES = TS_STATIC_HEADER + (size_t)(TS_STATIC_MAX_N /
 static __device__ __align__(256) unsigned char g_touched_static_scratch[TS_STATIC_BYTES];
 
 // In host code the array's name is only a handle for the runtime, not a device address, so the address is asked for
-// once per device (with that device current) and cached.
+// once per device (with that device current) and cached.  The cache entries are atomics: two host threads that make
+// the first call on a device at the same time both look the address up and store the same value.
 constexpr int TS_STATIC_MAX_DEVICES = 64;
-static unsigned char* g_touched_static_ptr[TS_STATIC_MAX_DEVICES] = {};
+static std::atomic<unsigned char*> g_touched_static_ptr[TS_STATIC_MAX_DEVICES];
 
 extern "C" int odin_touched_set_static(const uint32_t* d_tiles_touched, uint32_t n, uint32_t* d_mask, uint32_t* d_idx,
                                        uint32_t idx_capacity, uint32_t* d_count, int* d_status, void* stream) {
@@ -163,23 +166,27 @@ extern "C" int odin_touched_set_static(const uint32_t* d_tiles_touched, uint32_t
   int device = -1;
   ODIN_CUDA(cudaGetDevice(&device));
   if (device < 0 || device >= TS_STATIC_MAX_DEVICES) return ODIN_ERR_UNSUPPORTED;
-  if (!g_touched_static_ptr[device]) {  // first call on this device: resolve the array's device address
+  unsigned char* scratch = g_touched_static_ptr[device].load(std::memory_order_acquire);
+  if (!scratch) {  // first call on this device: resolve the array's device address (this may load the module)
     void* p = nullptr;
     ODIN_CUDA(cudaGetSymbolAddress(&p, g_touched_static_scratch));
     if (!p) return ODIN_ERR_CUDA;
-    g_touched_static_ptr[device] = static_cast<unsigned char*>(p);
+    scratch = static_cast<unsigned char*>(p);
+    g_touched_static_ptr[device].store(scratch, std::memory_order_release);
   }
-  unsigned char* scratch = g_touched_static_ptr[device];
   const uint32_t tiles = (n + TOUCHED_TILE - 1) / TOUCHED_TILE;
   // the array keeps whatever the previous call left: the ticket, the sink and the look-back words must start at zero
   ODIN_CUDA(cudaMemsetAsync(scratch, 0, TS_STATIC_HEADER + (size_t)tiles * 8, st));
   uint32_t* ticket = reinterpret_cast<uint32_t*>(scratch);
   int* status = d_status ? d_status : reinterpret_cast<int*>(scratch + 64);
   uint64_t* state = reinterpret_cast<uint64_t*>(scratch + TS_STATIC_HEADER);
-  const int scan_rounds = scan_rounds_for(n, 148);  // no context here: sized for a B200
+  // no context here, so the SM count is not looked up: the block size is chosen for the 148 SMs of a B200 (any other
+  // count only changes how many blocks share the work, never the result)
+  const int scan_rounds = scan_rounds_for(n, 148);
   const uint32_t scan_chunk = TOUCHED_TILE * (uint32_t)scan_rounds;
   touched_set_kernel<<<(n + scan_chunk - 1) / scan_chunk, TS_THREADS, 0, st>>>(
-      d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket, state, status, scan_rounds);
+      d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket, state, status, scan_rounds,
+      ODIN_DEFAULT_SPIN_LIMIT);
   return odin_launch_status();
 }
 

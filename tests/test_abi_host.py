@@ -46,6 +46,7 @@ def test_null_context_is_rejected_without_a_device(lib):
     null = C.c_void_p(None)
     assert lib.odin_destroy(null) == B.ODIN_ERR_NULL
     assert lib.odin_poll(null, None) == B.ODIN_ERR_NULL
+    assert lib.odin_set_wait_limit(null, 0) == B.ODIN_ERR_NULL
     sz = C.c_size_t(0)
     assert lib.odin_workspace_bytes(null, 10, 10, C.byref(sz)) == B.ODIN_ERR_NULL
     assert lib.odin_project(null, None, None, None, None, 0, None) == B.ODIN_ERR_NULL

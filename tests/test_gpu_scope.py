@@ -275,6 +275,15 @@ def test_locality_graph_from_the_masks_of_rendered_views(oracle32):
     tr.close()
 
 
+def admit_delayed_read(gate, active_count_a, tau):
+    """The admission rule of Sec. 4.3 as the caller evaluates it from the four counts of odin_delayed_read_gate
+    (#D+, #(D+ & C_A), #passing, #R+(B)): rho = #D+ / #R+(B) <= tau, C_A not empty, every delayed primitive has
+    evidence and passes the gate."""
+    n_delayed, n_with, n_pass, n_read_b = (int(x) for x in gate)
+    return bool(n_read_b > 0 and n_delayed <= tau * n_read_b and active_count_a > 0 and n_with == n_delayed
+                and n_pass == n_delayed)
+
+
 def run_gate(ctx, dev, n, r_b, w_b, w_a, active_a, ev_a, tau, capacity=None):
     d_m, stride = to_device_masks([r_b, w_b, w_a], n, dev)
     cap = len(active_a) if capacity is None else capacity
@@ -300,7 +309,7 @@ def test_delayed_read_gate_hand_example(oracle32):
         gate = run_gate(ctx, dev, 32, ints("R_B" + case), ints("W_B" + case), ints("W_A"), ints("C_A"), ev, tau)
         assert gate.tolist() == [int(g["n_delayed" + case][0]), int(g["n_with_evidence" + case][0]),
                                  int(g["n_pass" + case][0]), len(ints("R_B" + case))]
-        assert B.admit_delayed_read(gate, len(ints("C_A")), tau) == (g["admitted" + case][0] == "yes")
+        assert admit_delayed_read(gate, len(ints("C_A")), tau) == (g["admitted" + case][0] == "yes")
     B.odin_destroy(ctx)
 
 
@@ -318,7 +327,7 @@ def test_delayed_read_gate_random_scopes(oracle32, n):
         want = oracle32.delayed_read_gate(r_a, w_a, r_b, w_b, active_a, ev_a, tau)
         gate = run_gate(ctx, dev, n, r_b, w_b, w_a, active_a, ev_a, tau)
         assert gate.tolist() == [want["n_delayed"], want["n_with_evidence"], want["n_pass"], want["n_read_b"]], trial
-        assert B.admit_delayed_read(gate, len(active_a), tau) == want["admitted"]
+        assert admit_delayed_read(gate, len(active_a), tau) == want["admitted"]
     # with R+ = W+ nothing is ever delayed
     gate = run_gate(ctx, dev, n, w_b, w_b, w_a, active_a, ev_a, 0.2)
     assert gate[0] == 0 and gate[1] == 0

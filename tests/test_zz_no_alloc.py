@@ -64,6 +64,54 @@ def test_static_touched_set_matches_workspace_version_twice():
     B.odin_destroy(ctx)
 
 
+def test_static_touched_set_leaves_free_device_memory_unchanged():
+    """The point of the entry point: after the warm-up call (which may make the runtime load the library's device code)
+    a call allocates nothing, so the free device memory reported by the runtime is the same before and after it."""
+    dev = torch.device("cuda", 0)
+    n = 3_000_017
+    rng = np.random.default_rng(78)
+    tt = ((rng.random(n) < 0.2) * 3).astype(np.uint32)
+    d_tt = torch.from_numpy(tt.view(np.int32)).to(dev)
+    d_mask = torch.zeros((n + 31) // 32, dtype=torch.int32, device=dev)
+    d_idx = torch.zeros(n, dtype=torch.int32, device=dev)
+    d_count = torch.zeros(1, dtype=torch.int32, device=dev)
+    B.odin_touched_set_static(d_tt, n, d_mask, d_idx, n, d_count, None)  # warm-up: first call on the device
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info(dev)
+    for _ in range(3):
+        B.odin_touched_set_static(d_tt, n, d_mask, d_idx, n, d_count, None)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info(dev)
+    assert free_after == free_before
+    assert int(d_count.item()) == int(np.count_nonzero(tt))
+
+
+def test_static_touched_set_at_its_size_limit_and_without_a_status_word():
+    dev = torch.device("cuda", 0)
+    ctx = B.odin_create(0)
+    n = 1 << 25  # the largest size: the whole fixed array is in use
+    ws = torch.zeros(B.odin_workspace_bytes(ctx, n, 0), dtype=torch.uint8, device=dev)
+    rng = np.random.default_rng(79)
+    tt = (rng.random(n) < 0.03).astype(np.uint32)
+    tt[-1] = 9  # the very last primitive
+    (mask_a, idx_a, cnt_a, st_a), (mask_b, idx_b, cnt_b, st_b) = run_both(ctx, ws, tt, idx_capacity=1_200_000)
+    assert st_a == st_b == B.ODIN_OK and cnt_a == cnt_b == int(np.count_nonzero(tt))
+    assert np.array_equal(mask_a, mask_b) and np.array_equal(idx_a, idx_b)
+    assert idx_b[cnt_b - 1] == n - 1
+    B.odin_destroy(ctx)
+    # no status word (NULL): an overflowing list is still cut at the capacity, the condition goes to the internal sink
+    tt = np.ones(70_000, np.uint32)
+    d_tt = torch.from_numpy(tt.view(np.int32)).to(dev)
+    d_mask = torch.zeros((len(tt) + 31) // 32, dtype=torch.int32, device=dev)
+    d_idx = torch.full((1000 + 64,), -1, dtype=torch.int32, device=dev)
+    d_count = torch.zeros(1, dtype=torch.int32, device=dev)
+    B.odin_touched_set_static(d_tt, len(tt), d_mask, d_idx[:1000], 1000, d_count, None)
+    torch.cuda.synchronize()
+    assert int(d_count.item()) == 1000
+    assert np.array_equal(d_idx[:1000].cpu().numpy(), np.arange(1000)) and (d_idx[1000:] == -1).all()
+    assert (d_mask.cpu().numpy().view(np.uint32)[: 70_000 // 32] == 0xFFFFFFFF).all()
+
+
 def test_static_touched_set_limits_and_empty_input():
     dev = torch.device("cuda", 0)
     d_count = torch.full((1,), 9, dtype=torch.int32, device=dev)
