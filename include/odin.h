@@ -46,7 +46,7 @@ typedef enum {
 
 typedef struct odin_ctx odin_ctx; /* opaque: device ordinal, configuration, deferred-status word */
 
-/* Renderer constants.  Defaults (pass NULL to odin_create): 1/255, 0.99, 1e-4, 0.3, 3, 1.3, 16, 0. */
+/* Renderer constants.  Defaults (pass NULL to odin_create): 1/255, 0.99, 1e-4, 0.3, 3, 1.3, 16, 0, 0. */
 typedef struct {
   float alpha_min;     /* a contribution with alpha below this is skipped */
   float alpha_max;     /* alpha clamp */
@@ -60,6 +60,10 @@ typedef struct {
                           (half extents sqrt(2 ln(opacity/alpha_min) * Sigma'_xx), ..._yy; a primitive whose opacity is
                           below alpha_min gets no tile).  An optimised-pipeline variant in the sense of Sec. 5: the
                           primitive ids, the image and the gradients are unchanged, the instance lists are shorter. */
+  int instance_sort;   /* how odin_bin_sort orders the (tile, row) instances; the result is the same either way.
+                          0: counting scatter (per-chunk tile counts from the rectangles, every instance written once, to
+                          its final place) for images of up to 768 x 40,000 tiles (per row / in all), radix passes beyond;
+                          1: always radix passes over the instances (tile-id digits, onesweep). */
 } odin_config;
 
 /* Pinhole camera (host struct).  w2c is the row-major 3x4 world-to-camera matrix [R|t]; camera axes are x right,
@@ -125,6 +129,13 @@ int odin_set_wait_limit(odin_ctx* ctx, int polls);
 /* Workspace size sufficient for odin_project, odin_touched_set and odin_bin_sort with at most n primitives and
  * `max_instances` instance capacity. */
 int odin_workspace_bytes(const odin_ctx* ctx, uint32_t n, uint64_t max_instances, size_t* bytes);
+
+/* Workspace size sufficient for odin_bin_sort on a width x height image with at most `row_capacity` visible rows
+ * (odin_projected.capacity) and `max_instances` instance capacity: the counting scatter needs one counter per (2048
+ * sorted rows, tile) and no instance buffers; the radix passes need three instance-sized buffers.  odin_bin_sort takes
+ * the counting scatter whenever the image qualifies and the workspace it is given is at least this large. */
+int odin_bin_sort_workspace_bytes(const odin_ctx* ctx, uint32_t row_capacity, uint64_t max_instances, int width, int height,
+                                  size_t* bytes);
 
 /* Minimum workspace size for odin_render_fwd / odin_render_bwd on a width x height image.  The forward call leaves in
  * it, for every tile whose list is longer than 256 entries, one record (8 KB: transmittance and colour still to come of

@@ -29,6 +29,7 @@ EXPORTS = [
     "odin_conflict_count", "odin_kernel_count", "odin_kernel_name", "odin_profile_enable", "odin_profile_collect",
     "odin_touched_set_static", "odin_render_workspace_bytes", "odin_active_set", "odin_mask_union", "odin_hazard_count",
     "odin_delayed_read_gate", "odin_rlg_weights", "odin_rlg_topk", "odin_sds_scores", "odin_set_wait_limit",
+    "odin_bin_sort_workspace_bytes",
 ]
 
 
@@ -40,12 +41,14 @@ class OdinError(RuntimeError):
 
 class odin_config(C.Structure):
     _fields_ = [("alpha_min", C.c_float), ("alpha_max", C.c_float), ("t_min", C.c_float), ("dilation", C.c_float),
-                ("radius_sigmas", C.c_float), ("jac_clamp", C.c_float), ("tile", C.c_int), ("binning", C.c_int)]
+                ("radius_sigmas", C.c_float), ("jac_clamp", C.c_float), ("tile", C.c_int), ("binning", C.c_int),
+                ("instance_sort", C.c_int)]
 
 
-def default_config(binning: int = 0) -> odin_config:
-    """The renderer constants of the method; binning 1 selects the tight-extent tile rectangles."""
-    return odin_config(1.0 / 255.0, 0.99, 1e-4, 0.3, 3.0, 1.3, 16, int(binning))
+def default_config(binning: int = 0, instance_sort: int = 0) -> odin_config:
+    """The renderer constants of the method; binning 1 selects the tight-extent tile rectangles, instance_sort 1 the
+    radix passes over the instances in place of the counting scatter."""
+    return odin_config(1.0 / 255.0, 0.99, 1e-4, 0.3, 3.0, 1.3, 16, int(binning), int(instance_sort))
 
 
 class odin_camera(C.Structure):
@@ -87,6 +90,7 @@ def lib() -> C.CDLL:
         L.odin_poll.argtypes = [vp, vp]
         L.odin_set_wait_limit.argtypes = [vp, i32]
         L.odin_workspace_bytes.argtypes = [vp, u32, u64, C.POINTER(C.c_size_t)]
+        L.odin_bin_sort_workspace_bytes.argtypes = [vp, u32, u64, i32, i32, C.POINTER(C.c_size_t)]
         L.odin_project.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_camera), C.POINTER(odin_projected), vp,
                                    C.c_size_t, vp]
         L.odin_touched_set.argtypes = [vp, vp, u32, vp, vp, u32, vp, vp, C.c_size_t, vp]
@@ -181,6 +185,13 @@ def odin_destroy(ctx) -> None:
 def odin_poll(ctx, stream=None) -> int:
     """Synchronises the stream and returns the deferred device-side status (0 = ok) without raising."""
     return int(lib().odin_poll(ctx, _stream(stream)))
+
+
+def odin_bin_sort_workspace_bytes(ctx, row_capacity: int, max_instances: int, width: int, height: int) -> int:
+    b = C.c_size_t(0)
+    _check(lib().odin_bin_sort_workspace_bytes(ctx, int(row_capacity), int(max_instances), int(width), int(height),
+                                               C.byref(b)), "odin_bin_sort_workspace_bytes")
+    return int(b.value)
 
 
 def odin_set_wait_limit(ctx, polls: int) -> None:

@@ -7,10 +7,11 @@
 extern "C" int odin_create(odin_ctx** out, int device, const odin_config* cfg) {
   if (!out) return ODIN_ERR_NULL;
   *out = nullptr;
-  odin_config c = {1.0f / 255.0f, 0.99f, 1e-4f, 0.3f, 3.0f, 1.3f, 16, 0};
+  odin_config c = {1.0f / 255.0f, 0.99f, 1e-4f, 0.3f, 3.0f, 1.3f, 16, 0, 0};
   if (cfg) c = *cfg;
   if (c.tile != 16) return ODIN_ERR_UNSUPPORTED;
   if (c.binning != 0 && c.binning != 1) return ODIN_ERR_INVALID_ARG;
+  if (c.instance_sort != 0 && c.instance_sort != 1) return ODIN_ERR_INVALID_ARG;
   if (!(c.alpha_min > 0) || !(c.alpha_max < 1) || !(c.alpha_max > c.alpha_min) || !(c.t_min > 0) || !(c.dilation >= 0) ||
       !(c.radius_sigmas > 0) || !(c.jac_clamp > 0))
     return ODIN_ERR_INVALID_ARG;
@@ -82,7 +83,7 @@ static const char* const kKernelNames[K_COUNT] = {
     "zero_rows", "render_bwd_blend", "render_bwd_project", "adam_sh", "adam_geom", "conflict_count",
     "render_fwd_tail", "project_scan", "project_rows", "row_hist",
     "row_sort_pass", "row_offsets", "active_set", "mask_union", "hazard_count", "delayed_read_gate",
-    "locality_graph"};
+    "locality_graph", "tile_bases"};
 
 extern "C" int odin_kernel_count(void) { return K_COUNT; }
 

@@ -549,6 +549,319 @@ emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* _
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------ counting scatter
+// The instances never need a sort of their own.  With the rows in depth order, the list of a tile is the subsequence of
+// rows whose rectangle covers it, so the final position of an instance is
+//     first position of the tile + instances of the tile in earlier chunks of rows + rank of the row inside its chunk,
+// and all three are cheap: the rectangles give the per-(chunk, tile) counts through a difference array (one block per
+// chunk of OFFSET_TILE sorted rows), a scan over the chunks and one over the tiles give the first positions, and the
+// rank inside a chunk comes out of a bit matrix (tile x row) in shared memory in which set bits are read off in row
+// order.  Three launches that together move 8V + 4M bytes plus the counters, against emission + two radix passes over
+// 8-byte instances.
+
+// One block per chunk, blocks ordered by ticket (one look-back for the running instance offset, which is only needed
+// for the capacity rule: the instances in front of `capacity` in depth order are the ones that exist).  Writes the
+// rectangles in depth order and the chunk's instance count for every tile.
+__global__ void __launch_bounds__(RO_THREADS)
+chunk_counts_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __restrict__ rect,
+                    const uint32_t* __restrict__ num_rows, uint32_t capacity, int TX, uint32_t n_tiles, uint32_t tiles_pad,
+                    uint32_t* __restrict__ sorted_off, ushort4* __restrict__ sorted_rect, uint32_t* __restrict__ counts,
+                    uint32_t* ticket, uint64_t* state, int* status, int spin_limit) {
+  extern __shared__ __align__(16) uint32_t s_tdiff[];  // tiles_pad + 8 words
+  __shared__ uint32_t s_tile, s_base;
+  __shared__ uint32_t s_warp[33];
+  const uint32_t V = *num_rows;
+  const uint32_t ntiles = (V + OFFSET_TILE - 1) / OFFSET_TILE;
+  if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
+  __syncthreads();
+  const uint32_t tile = s_tile;
+  if (tile >= ntiles) return;  // uniform over the block; nobody waits for a chunk past the end
+  for (uint32_t i = threadIdx.x; i < tiles_pad + 8; i += RO_THREADS) s_tdiff[i] = 0;  // (barriers of the scan follow)
+  const uint32_t first = tile * OFFSET_TILE + threadIdx.x * RO_ITEMS;
+  ushort4 rc[RO_ITEMS];
+  uint32_t cnt[RO_ITEMS];
+  uint32_t sum = 0;
+#pragma unroll
+  for (int k = 0; k < RO_ITEMS; ++k) {
+    rc[k] = make_ushort4(0, 0, 0, 0);
+    if (first + k < V) rc[k] = rect[min(sorted_row[first + k], V - 1)];
+    cnt[k] = ((uint32_t)rc[k].z - (uint32_t)rc[k].x) * ((uint32_t)rc[k].w - (uint32_t)rc[k].y);
+    sum += cnt[k];
+  }
+  uint32_t total;
+  const uint32_t before = odin_block_exclusive_sum(sum, s_warp, &total);
+  if (threadIdx.x < 32) {
+    const uint64_t b = odin_lookback_u64(state, tile, (uint64_t)total, status, spin_limit);
+    if (threadIdx.x == 0) s_base = (uint32_t)b;
+  }
+  __syncthreads();
+  uint32_t run = s_base + before;
+#pragma unroll
+  for (int k = 0; k < RO_ITEMS; ++k) {
+    if (first + k < V) {
+      sorted_off[first + k] = run;
+      sorted_rect[first + k] = rc[k];
+    }
+    uint32_t left = run < capacity ? min(cnt[k], capacity - run) : 0u;
+    const uint32_t w = (uint32_t)rc[k].z - (uint32_t)rc[k].x;
+    for (uint32_t y = rc[k].y; left != 0; ++y) {
+      const uint32_t len = min(w, left);
+      left -= len;
+      const uint32_t t0 = min(y * (uint32_t)TX + (uint32_t)rc[k].x, n_tiles);  // (clamps: see emit_instances_kernel)
+      atomicAdd(&s_tdiff[t0], 1u);
+      atomicSub(&s_tdiff[min(t0 + len, n_tiles)], 1u);
+    }
+    run += cnt[k];
+  }
+  __syncthreads();
+  // integrate the difference array: instances of every tile in this chunk
+  uint32_t* __restrict__ out = counts + (size_t)tile * tiles_pad;
+  uint32_t carry = 0;
+  for (uint32_t b0 = 0; b0 < n_tiles; b0 += RO_THREADS * 4) {
+    const uint32_t t0 = b0 + threadIdx.x * 4;
+    uint4 d = make_uint4(0, 0, 0, 0);
+    if (t0 < n_tiles) d = *reinterpret_cast<const uint4*>(s_tdiff + t0);  // padded: words past n_tiles are zero or unused
+    const uint32_t c0 = d.x, c1 = c0 + d.y, c2 = c1 + d.z, c3 = c2 + d.w;
+    uint32_t tot;
+    const uint32_t base = carry + odin_block_exclusive_sum(c3, s_warp, &tot);
+    if (t0 + 3 < n_tiles) {
+      *reinterpret_cast<uint4*>(out + t0) = make_uint4(c0 + base, c1 + base, c2 + base, c3 + base);
+    } else {
+      if (t0 < n_tiles) out[t0] = c0 + base;
+      if (t0 + 1 < n_tiles) out[t0 + 1] = c1 + base;
+      if (t0 + 2 < n_tiles) out[t0 + 2] = c2 + base;
+    }
+    carry += tot;
+  }
+}
+
+// counts[c][t] -> exclusive prefix over the chunks c; tile totals; tile ranges.  A block owns 32 tiles; its eight warps
+// split the chunks (each warp sums its share, the shares are combined in shared memory, then each warp rewrites its
+// share), so the chains of dependent loads are an eighth as long.  The block that arrives last scans the tile totals
+// into the ranges.
+constexpr int TB_THREADS = 256;
+constexpr int TB_PARTS = TB_THREADS / 32;
+
+__global__ void __launch_bounds__(TB_THREADS)
+tile_bases_kernel(uint32_t* __restrict__ counts, uint32_t tiles_pad, uint32_t n_tiles, const uint32_t* __restrict__ num_rows,
+                  const uint64_t* __restrict__ num_instances, uint64_t capacity, uint32_t* tile_total,
+                  uint32_t* __restrict__ ranges, uint32_t* arrivals, int* status) {
+  __shared__ uint32_t s_part[TB_PARTS][32];
+  __shared__ uint32_t s_warp[33];
+  __shared__ uint32_t s_flag;
+  const uint32_t V = *num_rows;
+  const uint32_t nchunks = (V + OFFSET_TILE - 1) / OFFSET_TILE;
+  const unsigned lane = threadIdx.x & 31, part = threadIdx.x >> 5;
+  const uint32_t t = blockIdx.x * 32 + lane;
+  const uint32_t per = (nchunks + TB_PARTS - 1) / TB_PARTS;
+  const uint32_t c_lo = min(part * per, nchunks), c_hi = min(c_lo + per, nchunks);
+  uint32_t* __restrict__ col = counts + t;
+  uint32_t mine = 0;
+  if (t < n_tiles) {
+    uint32_t c = c_lo;
+    for (; c + 8 <= c_hi; c += 8) {
+      uint32_t v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = col[(size_t)(c + i) * tiles_pad];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) mine += v[i];
+    }
+    for (; c < c_hi; ++c) mine += col[(size_t)c * tiles_pad];
+  }
+  s_part[part][lane] = mine;
+  __syncthreads();
+  uint32_t acc = 0, all = 0;
+#pragma unroll
+  for (int q = 0; q < TB_PARTS; ++q) {
+    const uint32_t x = s_part[q][lane];
+    if (q < (int)part) acc += x;
+    all += x;
+  }
+  if (t < n_tiles) {
+    if (part == 0) tile_total[t] = all;
+    uint32_t c = c_lo;
+    for (; c + 8 <= c_hi; c += 8) {
+      uint32_t v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = col[(size_t)(c + i) * tiles_pad];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { col[(size_t)(c + i) * tiles_pad] = acc; acc += v[i]; }
+    }
+    for (; c < c_hi; ++c) {
+      const uint32_t v = col[(size_t)c * tiles_pad];
+      col[(size_t)c * tiles_pad] = acc;
+      acc += v;
+    }
+  }
+  // the block that arrives last turns the tile totals into the tile ranges
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_flag = (atomicAdd(arrivals, 1u) == gridDim.x - 1u) ? 1u : 0u;
+  __syncthreads();
+  if (!s_flag) return;
+  __threadfence();
+  if (threadIdx.x == 0 && *num_instances > capacity) odin_set_error(status, ODIN_ERR_CAPACITY);
+  const uint32_t cap = (uint32_t)(capacity < 0xffffffffull ? capacity : 0xffffffffull);
+  uint32_t carry = 0;
+  for (uint32_t b0 = 0; b0 < n_tiles; b0 += TB_THREADS * 4) {
+    const uint32_t t0 = b0 + threadIdx.x * 4;
+    uint32_t c[4], sum = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      c[k] = (t0 + k < n_tiles) ? ld_volatile_u32(tile_total + t0 + k) : 0u;
+      sum += c[k];
+    }
+    uint32_t tot;
+    uint32_t off = carry + odin_block_exclusive_sum(sum, s_warp, &tot);
+    carry += tot;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (t0 + k < n_tiles) reinterpret_cast<uint2*>(ranges)[t0 + k] = make_uint2(min(off, cap), min(off + c[k], cap));
+      off += c[k];
+    }
+  }
+}
+
+// Writes every instance to its final place.  A work item is (chunk of OFFSET_TILE sorted rows, band of `band_rows` tile
+// rows); blocks loop over the items.  The rows of the chunk whose rectangle meets the band are compacted in order,
+// then handled SC_SUB at a time: every such row sets its bit in the bit vector of each tile it covers inside the band
+// (word-major bit matrix [SC_SUB / 32][tiles of the band]), and every tile reads its bits off in order, which is the
+// depth order, and writes the row ids behind the position it has reached.
+constexpr int SC_THREADS = 256;
+constexpr int SC_ITEMS = OFFSET_TILE / SC_THREADS;
+constexpr int SC_SUB = 256;
+constexpr int SC_WORDS = SC_SUB / 32;
+constexpr uint32_t SC_BAND_TILES = SCATTER_MAX_TX;  // tiles of a band: band_rows * TX <= this
+constexpr size_t SC_SMEM = (size_t)OFFSET_TILE * (8 + 4 + 4) + (size_t)SC_WORDS * SC_BAND_TILES * 4 + SC_BAND_TILES * 4;
+
+template <bool WIDE>
+__global__ void __launch_bounds__(SC_THREADS)
+scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const uint32_t* __restrict__ sorted_row,
+                         const uint32_t* __restrict__ sorted_off, const uint32_t* __restrict__ num_rows,
+                         const uint64_t* __restrict__ num_instances, uint32_t capacity, int TX, int TY, int band_rows,
+                         const uint32_t* __restrict__ counts, uint32_t tiles_pad, const uint2* __restrict__ ranges,
+                         uint32_t* __restrict__ vals, uint64_t* __restrict__ keys64,
+                         const uint32_t* __restrict__ depth_bits) {
+  extern __shared__ __align__(16) unsigned char sc_smem[];
+  ushort4* s_prect = reinterpret_cast<ushort4*>(sc_smem);                    // [OFFSET_TILE] rectangles of the rows kept
+  uint32_t* s_prow = reinterpret_cast<uint32_t*>(s_prect + OFFSET_TILE);     // [OFFSET_TILE] their row ids
+  uint32_t* s_plim = s_prow + OFFSET_TILE;                                   // [OFFSET_TILE] instances they may emit
+  uint32_t* s_bits = s_plim + OFFSET_TILE;                                   // [SC_WORDS][band tiles]
+  uint32_t* s_pos = s_bits + SC_WORDS * SC_BAND_TILES;                       // [band tiles] next position of the tile
+  __shared__ uint32_t s_warp[33];
+  const uint32_t V = *num_rows;
+  const uint32_t nchunks = (V + OFFSET_TILE - 1) / OFFSET_TILE;
+  const uint32_t nbands = ((uint32_t)TY + band_rows - 1) / band_rows;
+  const uint32_t items = nchunks * nbands;
+  const bool cut = *num_instances > (uint64_t)capacity;  // only then can a row be denied some of its instances
+  for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
+    const uint32_t chunk = item / nbands, band = item - chunk * nbands;  // neighbouring blocks share a chunk's rows
+    const uint32_t by0 = band * band_rows, by1 = min((uint32_t)TY, by0 + band_rows);
+    const uint32_t band_tiles = (by1 - by0) * (uint32_t)TX;
+    const uint32_t first = chunk * OFFSET_TILE + threadIdx.x * SC_ITEMS;
+    ushort4 rc[SC_ITEMS];
+    uint32_t keep = 0;
+#pragma unroll
+    for (int k = 0; k < SC_ITEMS; ++k) {
+      rc[k] = make_ushort4(0, 0, 0, 0);
+      if (first + k < V) {
+        rc[k] = sorted_rect[first + k];
+        if ((uint32_t)rc[k].y < by1 && (uint32_t)rc[k].w > by0 && rc[k].z > rc[k].x) keep |= 1u << k;
+      }
+    }
+    uint32_t npass;
+    uint32_t p = odin_block_exclusive_sum((uint32_t)__popc(keep), s_warp, &npass);  // (its barriers also fence the reuse
+    if (npass == 0) continue;                                                      //  of the arrays below; uniform)
+#pragma unroll
+    for (int k = 0; k < SC_ITEMS; ++k) {
+      if (keep >> k & 1u) {
+        s_prect[p] = rc[k];
+        s_prow[p] = min(sorted_row[first + k], V - 1);
+        uint32_t lim = 0xffffffffu;
+        if (cut) {
+          const uint32_t off = sorted_off[first + k];
+          lim = off < capacity ? capacity - off : 0u;
+        }
+        s_plim[p] = lim;
+        ++p;
+      }
+    }
+    for (uint32_t t = threadIdx.x; t < band_tiles; t += SC_THREADS) {
+      const uint32_t tile = by0 * (uint32_t)TX + t;
+      s_pos[t] = ranges[tile].x + counts[(size_t)chunk * tiles_pad + tile];
+    }
+    __syncthreads();
+    for (uint32_t sub = 0; sub < npass; sub += SC_SUB) {
+      for (uint32_t i = threadIdx.x; i < SC_WORDS * band_tiles; i += SC_THREADS) s_bits[i] = 0;
+      __syncthreads();
+      {
+        // A row covers anything from one tile to the whole band.  A lane sets the bits of a small row by itself; the
+        // large rows of a warp are then taken one at a time by all 32 lanes (one tile per lane and step), so that a
+        // splat that fills the band costs the warp a few dozen steps instead of one lane several hundred.
+        const uint32_t j = sub + threadIdx.x;
+        const unsigned lane = threadIdx.x & 31;
+        uint32_t* word = s_bits + (threadIdx.x >> 5) * band_tiles;  // the warp's 32 rows are the bits of these words
+        uint32_t rx = 0, ry = 0, w = 1, lim = 0, ya = 0, yb = 0, x1 = 0;
+        if (j < npass) {
+          const ushort4 r = s_prect[j];
+          rx = r.x; ry = r.y; w = (uint32_t)r.z - (uint32_t)r.x; lim = s_plim[j];
+          ya = max((uint32_t)r.y, by0); yb = min((uint32_t)r.w, by1);
+          x1 = min((uint32_t)r.z, (uint32_t)TX);
+        }
+        const uint32_t wb = x1 > rx ? x1 - rx : 0u, cells = (yb > ya ? yb - ya : 0u) * wb;
+        const bool large = cells > 16;
+        if (!large && cells != 0) {
+          const uint32_t bit = 1u << lane;
+          for (uint32_t y = ya; y < yb; ++y) {
+            const uint32_t k0 = (y - ry) * w;  // index of the instance inside the row's rectangle, row major
+            uint32_t* line = word + (y - by0) * (uint32_t)TX;
+            for (uint32_t x = rx; x < x1; ++x)
+              if (k0 + (x - rx) < lim) atomicOr(line + x, bit);  // other lanes of the warp may hold the same tile
+          }
+        }
+        uint32_t todo = __ballot_sync(0xffffffffu, large);
+        __syncwarp();
+        while (todo) {
+          const int src = __ffs(todo) - 1;
+          todo &= todo - 1;
+          const uint32_t q_rx = __shfl_sync(0xffffffffu, rx, src), q_ry = __shfl_sync(0xffffffffu, ry, src);
+          const uint32_t q_w = __shfl_sync(0xffffffffu, w, src), q_lim = __shfl_sync(0xffffffffu, lim, src);
+          const uint32_t q_ya = __shfl_sync(0xffffffffu, ya, src), q_wb = __shfl_sync(0xffffffffu, wb, src);
+          const uint32_t q_cells = __shfl_sync(0xffffffffu, cells, src);
+          const uint32_t bit = 1u << src;
+          for (uint32_t c = lane; c < q_cells; c += 32) {  // distinct tiles per lane: no two lanes share a word here
+            const uint32_t dy = c / q_wb, dx = c - dy * q_wb;
+            const uint32_t y = q_ya + dy;
+            if ((y - q_ry) * q_w + dx < q_lim) word[(y - by0) * (uint32_t)TX + q_rx + dx] |= bit;
+          }
+          __syncwarp();
+        }
+      }
+      __syncthreads();
+      for (uint32_t t = threadIdx.x; t < band_tiles; t += SC_THREADS) {
+        uint32_t pos = s_pos[t];
+#pragma unroll
+        for (int wd = 0; wd < SC_WORDS; ++wd) {
+          uint32_t bits = s_bits[wd * band_tiles + t];
+          while (bits) {
+            const int b = __ffs(bits) - 1;
+            bits &= bits - 1;
+            const uint32_t row = s_prow[sub + wd * 32 + b];
+            if (pos < capacity) {
+              vals[pos] = row;
+              if (WIDE) keys64[pos] = ((uint64_t)(by0 * (uint32_t)TX + t) << 32) | (uint64_t)depth_bits[row];
+            }
+            ++pos;
+          }
+        }
+        s_pos[t] = pos;
+      }
+      __syncthreads();
+    }
+  }
+}
+
 int tile_digit_passes(uint32_t n_tiles) {
   int tile_bits = 0;
   while ((1ull << tile_bits) < (unsigned long long)n_tiles) ++tile_bits;
@@ -557,6 +870,17 @@ int tile_digit_passes(uint32_t n_tiles) {
 }
 
 }  // namespace
+
+extern "C" int odin_bin_sort_workspace_bytes(const odin_ctx* ctx, uint32_t row_capacity, uint64_t max_instances, int width,
+                                            int height, size_t* bytes) {
+  if (!ctx || !bytes) return ODIN_ERR_NULL;
+  if (width <= 0 || height <= 0 || width > 16384 || height > 16384) return ODIN_ERR_INVALID_ARG;
+  const int TX = (width + 15) / 16, TY = (height + 15) / 16;
+  const uint32_t n_tiles = (uint32_t)TX * (uint32_t)TY;
+  if (ctx->cfg.instance_sort != 1 && scatter_eligible(TX, n_tiles)) *bytes = scatter_layout(row_capacity, n_tiles).total;
+  else *bytes = binsort_ws_bytes(max_instances, row_capacity);
+  return ODIN_OK;
+}
 
 extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int width, int height, uint64_t* d_keys,
                              uint32_t* d_vals, uint64_t capacity, uint32_t* d_tile_ranges, void* ws, size_t ws_bytes,
@@ -576,27 +900,37 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   if (!d_vals || !proj->rect || !proj->depth) return ODIN_ERR_NULL;
   if ((d_keys && !odin_aligned(d_keys, 16)) || !odin_aligned(d_vals, 16) || !odin_aligned(proj->rect, 8))
     return ODIN_ERR_INVALID_ARG;
+  const bool scatter = ctx->cfg.instance_sort != 1 && scatter_eligible(TX, n_tiles);
+  const ScatterLayout F = scatter_layout(proj->capacity, n_tiles);
   const BinSortLayout L = binsort_layout(capacity, proj->capacity);
-  if (!ws || !odin_aligned(ws, 256) || ws_bytes < L.total) return ODIN_ERR_WORKSPACE;
+  const bool use_scatter = scatter && ws && ws_bytes >= F.total;
+  if (!ws || !odin_aligned(ws, 256) || (!use_scatter && ws_bytes < L.total)) return ODIN_ERR_WORKSPACE;
   char* base = reinterpret_cast<char*>(ws);
   const int tile_passes = tile_digit_passes(n_tiles);
-  // zero tickets, histograms, the used part of the difference array and the look-back words of the passes that run
-  ODIN_CUDA(cudaMemsetAsync(base, 0, L.tile_diff + ((size_t)n_tiles + 1) * 4, st));
-  ODIN_CUDA(cudaMemsetAsync(base + L.scan_state, 0,
-                            L.inst_states + (size_t)tile_passes * L.tiles * SORT_RADIX * 4 - L.scan_state, st));
-  uint32_t* tickets = reinterpret_cast<uint32_t*>(base + L.header);
-  uint32_t* hist = reinterpret_cast<uint32_t*>(base + L.hist);
-  uint32_t* dbase = reinterpret_cast<uint32_t*>(base + L.digit_base);
-  uint32_t* tile_diff = reinterpret_cast<uint32_t*>(base + L.tile_diff);
-  uint64_t* scan_state = reinterpret_cast<uint64_t*>(base + L.scan_state);
-  uint32_t* row_states = reinterpret_cast<uint32_t*>(base + L.row_states);
-  uint32_t* inst_states = reinterpret_cast<uint32_t*>(base + L.inst_states);
-  uint32_t* row_keys[2] = {reinterpret_cast<uint32_t*>(base + L.row_keys[0]), reinterpret_cast<uint32_t*>(base + L.row_keys[1])};
-  uint32_t* row_vals[2] = {reinterpret_cast<uint32_t*>(base + L.row_vals[0]), reinterpret_cast<uint32_t*>(base + L.row_vals[1])};
-  uint32_t* sorted_off = reinterpret_cast<uint32_t*>(base + L.sorted_off);
-  uint32_t* inst_keys[2] = {reinterpret_cast<uint32_t*>(base + L.inst_keys[0]), reinterpret_cast<uint32_t*>(base + L.inst_keys[1])};
-  uint32_t* inst_vals[2] = {d_vals, reinterpret_cast<uint32_t*>(base + L.alt_vals)};
-  uint32_t* chunk_row = reinterpret_cast<uint32_t*>(base + L.chunk_row);
+  // the regions both paths share (tickets, row histograms, look-back words of the row passes, ping-pong row buffers)
+  const size_t o_hist = use_scatter ? F.hist : L.hist, o_dbase = use_scatter ? F.digit_base : L.digit_base;
+  const size_t o_scan = use_scatter ? F.scan_state : L.scan_state, o_rstates = use_scatter ? F.row_states : L.row_states;
+  const uint32_t row_tiles = use_scatter ? F.row_tiles : L.row_tiles;
+  if (use_scatter) {
+    // zero tickets, histograms and the look-back words of the offset scan and of the row passes
+    ODIN_CUDA(cudaMemsetAsync(base, 0, F.row_keys[0], st));
+  } else {
+    // zero tickets, histograms, the used part of the difference array and the look-back words of the passes that run
+    ODIN_CUDA(cudaMemsetAsync(base, 0, L.tile_diff + ((size_t)n_tiles + 1) * 4, st));
+    ODIN_CUDA(cudaMemsetAsync(base + L.scan_state, 0,
+                              L.inst_states + (size_t)tile_passes * L.tiles * SORT_RADIX * 4 - L.scan_state, st));
+  }
+  uint32_t* tickets = reinterpret_cast<uint32_t*>(base);
+  uint32_t* hist = reinterpret_cast<uint32_t*>(base + o_hist);
+  uint32_t* dbase = reinterpret_cast<uint32_t*>(base + o_dbase);
+  uint64_t* scan_state = reinterpret_cast<uint64_t*>(base + o_scan);
+  uint32_t* row_states = reinterpret_cast<uint32_t*>(base + o_rstates);
+  uint32_t* row_keys[2], *row_vals[2];
+  for (int b = 0; b < 2; ++b) {
+    row_keys[b] = reinterpret_cast<uint32_t*>(base + (use_scatter ? F.row_keys[b] : L.row_keys[b]));
+    row_vals[b] = reinterpret_cast<uint32_t*>(base + (use_scatter ? F.row_vals[b] : L.row_vals[b]));
+  }
+  uint32_t* sorted_off = reinterpret_cast<uint32_t*>(base + (use_scatter ? F.sorted_off : L.sorted_off));
   const uint32_t* depth_bits = reinterpret_cast<const uint32_t*>(proj->depth);
   const ushort4* rect = reinterpret_cast<const ushort4*>(proj->rect);
   const uint32_t sms = (uint32_t)ctx->sm_count;
@@ -610,13 +944,9 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
                                                                                  tickets + 9);
   }
   constexpr size_t OS_SMEM = os_smem_bytes(OS_INST_ITEMS), OS_ROW_SMEM = os_smem_bytes(OS_ROW_ITEMS);
-  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<false, OS_INST_ITEMS, OS_INST_WINDOW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)OS_SMEM));
-  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<true, OS_INST_ITEMS, OS_INST_WINDOW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)OS_SMEM));
   const uint32_t* sorted_row = nullptr;
   {
-    const uint32_t grid = L.row_tiles < sms * OS_BLOCKS ? L.row_tiles : sms * OS_BLOCKS;
+    const uint32_t grid = row_tiles < sms * OS_BLOCKS ? row_tiles : sms * OS_BLOCKS;
     const uint32_t* kin = depth_bits;
     const uint32_t* vin = nullptr;
     for (int p = 0; p < SORT_DEPTH_DIGITS; ++p) {
@@ -625,12 +955,62 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
       uint32_t* vout = row_vals[p & 1];
       onesweep_kernel<false, OS_ROW_ITEMS, OS_ROW_WINDOW><<<grid, OS_THREADS, OS_ROW_SMEM, st>>>(
           kin, vin, kout, vout, nullptr, nullptr, proj->num_rows, nullptr, 0, p * (int)SORT_RADIX_BITS,
-          dbase + p * SORT_RADIX, row_states + (size_t)p * L.row_tiles * SORT_RADIX, tickets + p, ctx->d_status, ctx->spin_limit, proj->capacity);
+          dbase + p * SORT_RADIX, row_states + (size_t)p * row_tiles * SORT_RADIX, tickets + p, ctx->d_status,
+          ctx->spin_limit, proj->capacity);
       kin = kout;
       vin = vout;
     }
     sorted_row = vin;
   }
+  if (use_scatter) {
+    // ---- instances straight to their final places
+    ushort4* sorted_rect = reinterpret_cast<ushort4*>(base + F.sorted_rect);
+    uint32_t* tile_total = reinterpret_cast<uint32_t*>(base + F.tile_total);
+    uint32_t* counts = reinterpret_cast<uint32_t*>(base + F.counts);
+    const uint32_t cap32 = (uint32_t)capacity;
+    {
+      OdinKernelScope ks(ctx, K_ROW_OFFSETS, st);
+      const size_t smem = ((size_t)F.tiles_pad + 8) * 4;
+      ODIN_CUDA(cudaFuncSetAttribute(chunk_counts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)(((size_t)SCATTER_MAX_TILES + 64 + 8) * 4)));
+      chunk_counts_kernel<<<F.chunks, RO_THREADS, smem, st>>>(sorted_row, rect, proj->num_rows, cap32, TX, n_tiles,
+                                                             F.tiles_pad, sorted_off, sorted_rect, counts, tickets + 8,
+                                                             scan_state, ctx->d_status, ctx->spin_limit);
+    }
+    {
+      OdinKernelScope ks(ctx, K_TILE_BASES, st);
+      tile_bases_kernel<<<(n_tiles + 31) / 32, TB_THREADS, 0, st>>>(counts, F.tiles_pad, n_tiles, proj->num_rows,
+                                                                   proj->num_instances, capacity, tile_total,
+                                                                   d_tile_ranges, tickets + 10, ctx->d_status);
+    }
+    {
+      OdinKernelScope ks(ctx, K_EMIT, st);
+      int band_rows = (int)(SC_BAND_TILES / (uint32_t)TX);
+      if (band_rows > TY) band_rows = TY;
+      const uint64_t items_cap = (uint64_t)F.chunks * (((uint32_t)TY + band_rows - 1) / band_rows);
+      const uint32_t grid = (uint32_t)(items_cap < (uint64_t)sms * 3 ? items_cap : (uint64_t)sms * 3);
+      ODIN_CUDA(cudaFuncSetAttribute(scatter_instances_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM));
+      ODIN_CUDA(cudaFuncSetAttribute(scatter_instances_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM));
+      if (d_keys)
+        scatter_instances_kernel<true><<<grid, SC_THREADS, SC_SMEM, st>>>(
+            sorted_rect, sorted_row, sorted_off, proj->num_rows, proj->num_instances, cap32, TX, TY, band_rows, counts,
+            F.tiles_pad, reinterpret_cast<const uint2*>(d_tile_ranges), d_vals, d_keys, depth_bits);
+      else
+        scatter_instances_kernel<false><<<grid, SC_THREADS, SC_SMEM, st>>>(
+            sorted_rect, sorted_row, sorted_off, proj->num_rows, proj->num_instances, cap32, TX, TY, band_rows, counts,
+            F.tiles_pad, reinterpret_cast<const uint2*>(d_tile_ranges), d_vals, nullptr, depth_bits);
+    }
+    return odin_launch_status();
+  }
+  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<false, OS_INST_ITEMS, OS_INST_WINDOW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)OS_SMEM));
+  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<true, OS_INST_ITEMS, OS_INST_WINDOW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)OS_SMEM));
+  uint32_t* tile_diff = reinterpret_cast<uint32_t*>(base + L.tile_diff);
+  uint32_t* inst_states = reinterpret_cast<uint32_t*>(base + L.inst_states);
+  uint32_t* inst_keys[2] = {reinterpret_cast<uint32_t*>(base + L.inst_keys[0]), reinterpret_cast<uint32_t*>(base + L.inst_keys[1])};
+  uint32_t* inst_vals[2] = {d_vals, reinterpret_cast<uint32_t*>(base + L.alt_vals)};
+  uint32_t* chunk_row = reinterpret_cast<uint32_t*>(base + L.chunk_row);
   // ---- instances in depth order
   uint32_t* tile_dbase = dbase + SORT_DEPTH_DIGITS * SORT_RADIX;
   const uint64_t chunks_cap = (capacity + DUP_CHUNK - 1) / DUP_CHUNK;

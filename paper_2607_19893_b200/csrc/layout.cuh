@@ -79,3 +79,47 @@ static inline BinSortLayout binsort_layout(uint64_t capacity, uint32_t rows) {
   return L;
 }
 static inline size_t binsort_ws_bytes(uint64_t capacity, uint32_t rows) { return binsort_layout(capacity, rows).total; }
+
+// Counting scatter of the instances (the default for ordinary image sizes): the rows are sorted by depth as above, then
+// every chunk of OFFSET_TILE sorted rows counts its instances per tile, a scan over the chunks turns the counts into the
+// first position of every (chunk, tile) pair, and the instances are written straight to their final places: no pass
+// over the instances at all.  Needs one counter per (chunk, tile): images of up to SCATTER_MAX_TILES tiles.
+constexpr uint32_t SCATTER_MAX_TX = 768;        // tiles per image row the emission's shared-memory bit matrix can hold
+constexpr uint32_t SCATTER_MAX_TILES = 40000;   // tiles whose difference array fits into one block's shared memory
+struct ScatterLayout {
+  size_t header;       // as in BinSortLayout; [10] arrival counter of the tile-base kernel
+  size_t hist, digit_base;  // row digits only
+  size_t scan_state, row_states;
+  size_t row_keys[2], row_vals[2];
+  size_t sorted_off;   // u32[rows + 1]
+  size_t sorted_rect;  // ushort4[rows] rectangles in depth order
+  size_t tile_total;   // u32[tiles]
+  size_t counts;       // u32[chunks][tiles_pad]: instances of the tile in the chunk, then their exclusive prefix over the chunks
+  size_t total;
+  uint32_t row_tiles, chunks, tiles_pad;
+};
+static inline ScatterLayout scatter_layout(uint32_t rows, uint32_t n_tiles) {
+  ScatterLayout L;
+  L.row_tiles = (rows + ROW_SORT_TILE - 1) / ROW_SORT_TILE;
+  if (L.row_tiles == 0) L.row_tiles = 1;
+  L.chunks = (rows + OFFSET_TILE - 1) / OFFSET_TILE;
+  if (L.chunks == 0) L.chunks = 1;
+  L.tiles_pad = (n_tiles + 63) / 64 * 64;
+  size_t o = 0;
+  L.header = o; o += 256;
+  L.hist = o; o += ws_align((size_t)SORT_DEPTH_DIGITS * SORT_RADIX * 4);
+  L.digit_base = o; o += ws_align((size_t)SORT_DEPTH_DIGITS * SORT_RADIX * 4);
+  L.scan_state = o; o += ws_align((size_t)L.chunks * 8 + 8);
+  L.row_states = o; o += ws_align((size_t)SORT_DEPTH_DIGITS * L.row_tiles * SORT_RADIX * 4);
+  for (int b = 0; b < 2; ++b) { L.row_keys[b] = o; o += ws_align((size_t)rows * 4); }
+  for (int b = 0; b < 2; ++b) { L.row_vals[b] = o; o += ws_align((size_t)rows * 4); }
+  L.sorted_off = o; o += ws_align((size_t)rows * 4 + 4);
+  L.sorted_rect = o; o += ws_align((size_t)rows * 8);
+  L.tile_total = o; o += ws_align((size_t)n_tiles * 4);
+  L.counts = o; o += ws_align((size_t)L.chunks * L.tiles_pad * 4);
+  L.total = o;
+  return L;
+}
+static inline bool scatter_eligible(int TX, uint32_t n_tiles) {
+  return (uint32_t)TX <= SCATTER_MAX_TX && n_tiles <= SCATTER_MAX_TILES;
+}

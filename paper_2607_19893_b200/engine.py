@@ -126,7 +126,11 @@ class ViewTrainer:
         self.active_count = z(1, torch.int32)
         self.evidence = z(max(self.row_capacity, 1), torch.float32)
         self.evidence_sum = z(1, torch.float64)
-        self.ws = z(B.odin_workspace_bytes(self.ctx, self.n, self.instance_capacity), torch.uint8)
+        # one workspace for odin_project / odin_touched_set (sized by the pool) and odin_bin_sort (sized by the rows and,
+        # if the image is too large for the counting scatter, by the instances)
+        self.ws = z(max(B.odin_workspace_bytes(self.ctx, self.n, 0),
+                        B.odin_bin_sort_workspace_bytes(self.ctx, self.row_capacity, self.instance_capacity, self.width,
+                                                        self.height)), torch.uint8)
         # The render workspace is a buffer of its own: the forward pass leaves per-pixel records for long lists in it
         # that the backward pass of the same view reads, so nothing else may write there in between.  Every 8,208
         # bytes beyond the minimum hold one more record (a further 256 list entries of one tile).

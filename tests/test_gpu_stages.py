@@ -244,13 +244,18 @@ def test_project_row_capacity_overflow(oracle32):
 
 
 # ------------------------------------------------------------------------------------------------ bin / sort
-def check_bin_sort(oracle32, scene, cam, instance_capacity=None):
+# instance_sort 0: the counting scatter (radix passes only for images beyond its tile limits); 1: always the radix passes
+SORT_PATHS = [0, 1]
+
+
+def check_bin_sort(oracle32, scene, cam, instance_capacity=None, instance_sort=0):
     po = oracle32.project(scene, cam)
     mask, idx = oracle32.touched_set(po.tiles_touched)
     keys_o, vals_o, ranges_o = oracle32.bin_sort(po, cam)
     m = len(keys_o)
     tr = G.trainer_for(scene, cam, row_capacity=max(len(idx), 1),
-                       instance_capacity=instance_capacity if instance_capacity is not None else m + 17)
+                       instance_capacity=instance_capacity if instance_capacity is not None else m + 17,
+                       cfg=B.default_config(instance_sort=instance_sort))
     G.load_oracle_projection(tr, po, idx)
     inv = np.full(scene.n, -1, np.int64)
     inv[idx] = np.arange(len(idx))
@@ -272,21 +277,32 @@ def check_bin_sort(oracle32, scene, cam, instance_capacity=None):
     return m
 
 
-def test_bin_sort_cfg1(oracle32):
+@pytest.mark.parametrize("path", SORT_PATHS)
+def test_bin_sort_cfg1(oracle32, path):
     w = wl.make_workload(1)
-    check_bin_sort(oracle32, w.scene, w.cameras[0])
+    check_bin_sort(oracle32, w.scene, w.cameras[0], instance_sort=path)
 
 
-def test_bin_sort_cfg2(oracle32):
+@pytest.mark.parametrize("path", SORT_PATHS)
+def test_bin_sort_cfg2(oracle32, path):
     w = wl.make_workload(2)
-    m = check_bin_sort(oracle32, w.scene, w.cameras[2])
-    assert m > 3 * 4096  # several sort tiles and a ragged tail
+    m = check_bin_sort(oracle32, w.scene, w.cameras[2], instance_sort=path)
+    assert m > 3 * 4096  # several sort tiles / chunks of rows and a ragged tail
 
 
-def test_bin_sort_many_tiles_six_passes(oracle32):
+@pytest.mark.parametrize("path", SORT_PATHS)
+def test_bin_sort_many_tiles_six_passes(oracle32, path):
     w = wl.make_workload(3, n=120_000)  # 6700 tiles -> 13 tile bits -> 6 digit passes, ~1.2M instances
-    m = check_bin_sort(oracle32, w.scene, w.cameras[7])
+    m = check_bin_sort(oracle32, w.scene, w.cameras[7], instance_sort=path)
     assert m > 500_000
+
+
+def test_bin_sort_large_splats_many_rows_per_band(oracle32):
+    """Preset 4's large splats at 960 x 540: a chunk of 2048 sorted rows puts hundreds of rows into every band of tile
+    rows (several sub-batches of the scatter's bit matrix), and rectangles span many bands."""
+    w = wl.make_workload(4, n=150_000, n_cameras=4, resolution=(960, 540))
+    m = check_bin_sort(oracle32, w.scene, w.cameras[1])
+    assert m > 1_500_000
 
 
 def test_bin_sort_image_of_73728_tiles(oracle32):
@@ -299,38 +315,65 @@ def test_bin_sort_image_of_73728_tiles(oracle32):
     assert m > 1_000_000
 
 
-def test_bin_sort_image_of_one_tile(oracle32):
+@pytest.mark.parametrize("path", SORT_PATHS)
+def test_bin_sort_image_of_one_tile(oracle32, path):
     w = wl.make_workload(1, resolution=(16, 16))
-    check_bin_sort(oracle32, w.scene, w.cameras[0])
+    check_bin_sort(oracle32, w.scene, w.cameras[0], instance_sort=path)
 
 
-def test_bin_sort_equal_depth_ties(oracle32):
+@pytest.mark.parametrize("path", SORT_PATHS)
+def test_bin_sort_equal_depth_ties(oracle32, path):
     # many identical splats: identical keys, order decided by the row index alone
     w = wl.make_workload(1)
     s = w.scene
     rep = lambda a: np.ascontiguousarray(np.repeat(a[:3], 3000, axis=0))  # noqa: E731
     s2 = wl.Scene(0, rep(s.means), rep(s.log_scales), rep(s.quats), rep(s.opacity_logit), rep(s.sh))
-    check_bin_sort(oracle32, s2, w.cameras[0])
+    check_bin_sort(oracle32, s2, w.cameras[0], instance_sort=path)
 
 
-def test_bin_sort_empty_view(oracle32):
+@pytest.mark.parametrize("path", SORT_PATHS)
+def test_bin_sort_empty_view(oracle32, path):
     w = wl.make_workload(1)
     s = w.scene.copy()
     s.means[:, 2] = -5.0  # everything behind the camera
-    check_bin_sort(oracle32, s, w.cameras[0])
+    check_bin_sort(oracle32, s, w.cameras[0], instance_sort=path)
 
 
-def test_bin_sort_instance_capacity_overflow(oracle32):
+@pytest.mark.parametrize("path", SORT_PATHS)
+def test_bin_sort_instance_capacity_overflow(oracle32, path):
+    """More instances than the caller's capacity: the instances of the nearest rows are kept (the first `capacity` of
+    the depth order, a row's rectangle in row-major order), sorted; nothing is written beyond the capacity."""
     w = wl.make_workload(1)
     cam = w.cameras[0]
     po = oracle32.project(w.scene, cam)
     mask, idx = oracle32.touched_set(po.tiles_touched)
-    tr = G.trainer_for(w.scene, cam, instance_capacity=1000)
+    cap = 1000
+    tr = G.trainer_for(w.scene, cam, instance_capacity=cap + 64, cfg=B.default_config(instance_sort=path))
+    tr.instance_capacity = cap  # the buffers are 64 entries longer than the capacity the call is told
     G.load_oracle_projection(tr, po, idx)
+    tr.keys.fill_(-1)
+    tr.vals.fill_(-1)
     tr.bin_sort()
     assert tr.poll() == B.ODIN_ERR_CAPACITY
-    keys = G.u64(tr.keys)[:1000]
-    assert np.all(np.diff(keys.astype(np.int64)) >= 0)  # the first 1000 instances, sorted; nothing out of bounds
+    assert bool((tr.keys[cap:] == -1).all()) and bool((tr.vals[cap:] == -1).all())
+    # expected: emission order = rows by (depth bits, row), each rectangle row major; keep the first `cap`; stable sort
+    bits = po.depth[idx].astype(np.float32).view(np.uint32)
+    order = np.lexsort((np.arange(len(idx)), bits))
+    tx = tr.tx
+    tiles, rows = [], []
+    for r in order:
+        x0, y0, x1, y1 = po.rect[idx[r]]
+        for yy in range(y0, y1):
+            for xx in range(x0, x1):
+                tiles.append(yy * tx + xx)
+                rows.append(r)
+    tiles, rows = np.array(tiles[:cap], np.int64), np.array(rows[:cap], np.int64)
+    final = np.argsort(tiles, kind="stable")
+    keys = G.u64(tr.keys)[:cap]
+    assert np.array_equal(G.u32(tr.vals)[:cap], rows[final].astype(np.uint32))
+    assert np.array_equal(keys, (tiles[final].astype(np.uint64) << np.uint64(32)) | bits[rows[final]].astype(np.uint64))
+    rg = G.u32(tr.ranges).astype(np.int64)
+    assert np.array_equal(rg[:, 1] - rg[:, 0], np.bincount(tiles, minlength=len(rg)))
     tr.close()
 
 
