@@ -137,6 +137,13 @@ int odin_workspace_bytes(const odin_ctx* ctx, uint32_t n, uint64_t max_instances
 int odin_bin_sort_workspace_bytes(const odin_ctx* ctx, uint32_t row_capacity, uint64_t max_instances, int width, int height,
                                   size_t* bytes);
 
+/* Changes odin_config.instance_sort for the later odin_bin_sort calls of this context (0 or 1, see odin_config).  The
+ * counting scatter wins when rectangles cover many tiles (it never moves an instance twice), the radix passes when they
+ * cover a handful (their cost per instance does not depend on how the instances are spread over the image); a caller
+ * can time one view either way during warm-up and keep the faster.  A workspace sized by odin_bin_sort_workspace_bytes
+ * under one mode may be too small for the other: size it for both if the mode is going to change. */
+int odin_set_instance_sort(odin_ctx* ctx, int mode);
+
 /* Minimum workspace size for odin_render_fwd / odin_render_bwd on a width x height image.  The forward call leaves in
  * it, for every tile whose list is longer than 256 entries, one record (8 KB: transmittance and colour still to come of
  * the tile's 256 pixels) per further 256 entries that it walks; the backward call of the same view replays the
@@ -157,6 +164,18 @@ int odin_kernel_count(void);
 const char* odin_kernel_name(int id);
 int odin_profile_enable(odin_ctx* ctx, int on);
 int odin_profile_collect(odin_ctx* ctx, void* stream, float* h_ms, uint64_t* h_launches);
+
+/* Measurement aids (not part of the view step; bench.py uses them for its roofline figures).
+ * odin_measure_fp32_peak: runs a kernel of independent fp32 fused multiply-add chains on every SM, synchronises, and
+ * writes the sustained rate in TFLOP/s (2 flop per multiply-add) to the HOST float *h_tflops: the denominator for the
+ * compositing kernels, which are bound by plain ALU work.
+ * odin_count_blend_pairs: d_counts [2] (device, overwritten) = number of (pixel, list entry) pairs inside the pixels'
+ * walked prefixes (d_n_contrib of odin_render_fwd), and how many of them blend (pass the skip tests): the work the
+ * method itself defines for the two compositing passes of the view. */
+int odin_measure_fp32_peak(odin_ctx* ctx, void* stream, float* h_tflops);
+int odin_count_blend_pairs(odin_ctx* ctx, const odin_projected* proj, const uint32_t* d_vals,
+                           const uint32_t* d_tile_ranges, const odin_camera* cam, const uint32_t* d_n_contrib,
+                           uint64_t* d_counts, void* stream);
 
 /* ---- the seven calls of the view step ------------------------------------------------------------------------ */
 

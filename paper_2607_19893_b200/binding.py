@@ -29,7 +29,7 @@ EXPORTS = [
     "odin_conflict_count", "odin_kernel_count", "odin_kernel_name", "odin_profile_enable", "odin_profile_collect",
     "odin_touched_set_static", "odin_render_workspace_bytes", "odin_active_set", "odin_mask_union", "odin_hazard_count",
     "odin_delayed_read_gate", "odin_rlg_weights", "odin_rlg_topk", "odin_sds_scores", "odin_set_wait_limit",
-    "odin_bin_sort_workspace_bytes",
+    "odin_bin_sort_workspace_bytes", "odin_set_instance_sort", "odin_measure_fp32_peak", "odin_count_blend_pairs",
 ]
 
 
@@ -89,6 +89,9 @@ def lib() -> C.CDLL:
         L.odin_destroy.argtypes = [vp]
         L.odin_poll.argtypes = [vp, vp]
         L.odin_set_wait_limit.argtypes = [vp, i32]
+        L.odin_set_instance_sort.argtypes = [vp, i32]
+        L.odin_measure_fp32_peak.argtypes = [vp, vp, C.POINTER(C.c_float)]
+        L.odin_count_blend_pairs.argtypes = [vp, C.POINTER(odin_projected), vp, vp, C.POINTER(odin_camera), vp, vp, vp]
         L.odin_workspace_bytes.argtypes = [vp, u32, u64, C.POINTER(C.c_size_t)]
         L.odin_bin_sort_workspace_bytes.argtypes = [vp, u32, u64, i32, i32, C.POINTER(C.c_size_t)]
         L.odin_project.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_camera), C.POINTER(odin_projected), vp,
@@ -192,6 +195,23 @@ def odin_bin_sort_workspace_bytes(ctx, row_capacity: int, max_instances: int, wi
     _check(lib().odin_bin_sort_workspace_bytes(ctx, int(row_capacity), int(max_instances), int(width), int(height),
                                                C.byref(b)), "odin_bin_sort_workspace_bytes")
     return int(b.value)
+
+
+def odin_measure_fp32_peak(ctx, stream=None) -> float:
+    """Sustained fp32 multiply-add rate of the device in TFLOP/s (synchronises)."""
+    t = C.c_float(0.0)
+    _check(lib().odin_measure_fp32_peak(ctx, _stream(stream), C.byref(t)), "odin_measure_fp32_peak")
+    return float(t.value)
+
+
+def odin_count_blend_pairs(ctx, proj: odin_projected, d_vals, d_tile_ranges, cam: odin_camera, d_n_contrib, d_counts,
+                           stream=None) -> None:
+    _check(lib().odin_count_blend_pairs(ctx, C.byref(proj), _ptr(d_vals), _ptr(d_tile_ranges), C.byref(cam),
+                                        _ptr(d_n_contrib), _ptr(d_counts), _stream(stream)), "odin_count_blend_pairs")
+
+
+def odin_set_instance_sort(ctx, mode: int) -> None:
+    _check(lib().odin_set_instance_sort(ctx, int(mode)), "odin_set_instance_sort")
 
 
 def odin_set_wait_limit(ctx, polls: int) -> None:

@@ -53,6 +53,13 @@ extern "C" int odin_set_wait_limit(odin_ctx* ctx, int polls) {
   return ODIN_OK;
 }
 
+extern "C" int odin_set_instance_sort(odin_ctx* ctx, int mode) {
+  if (!ctx) return ODIN_ERR_NULL;
+  if (mode != 0 && mode != 1) return ODIN_ERR_INVALID_ARG;
+  ctx->cfg.instance_sort = mode;
+  return ODIN_OK;
+}
+
 extern "C" const char* odin_status_string(int s) {
   switch (s) {
     case ODIN_OK: return "ok";
@@ -110,6 +117,51 @@ extern "C" int odin_profile_collect(odin_ctx* ctx, void* stream, float* h_ms, ui
   }
   p.used = 0;
   return ODIN_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Measurement aid: the fp32 multiply-add rate this GPU sustains, the denominator for the kernels that are bound by
+// plain ALU work (the two compositing kernels).  Every thread runs eight independent chains of fused multiply-adds.
+namespace {
+constexpr int FMA_CHAINS = 8;
+__global__ void __launch_bounds__(256) fp32_peak_kernel(float* sink, int iters, float a, float b) {
+  float x[FMA_CHAINS];
+#pragma unroll
+  for (int k = 0; k < FMA_CHAINS; ++k) x[k] = (float)(threadIdx.x + k) * 1e-3f;
+  for (int i = 0; i < iters; ++i) {
+#pragma unroll
+    for (int k = 0; k < FMA_CHAINS; ++k) x[k] = fmaf(x[k], a, b);
+  }
+  float s = 0.f;
+#pragma unroll
+  for (int k = 0; k < FMA_CHAINS; ++k) s += x[k];
+  if (s == 123.456f) sink[0] = s;  // keeps the chains alive; practically never true
+}
+}  // namespace
+
+extern "C" int odin_measure_fp32_peak(odin_ctx* ctx, void* stream, float* h_tflops) {
+  if (!ctx || !h_tflops) return ODIN_ERR_NULL;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* sink = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->d_status) + 128);
+  const int iters = 1 << 14, blocks = ctx->sm_count * 8;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  ODIN_CUDA(cudaEventCreate(&e0));
+  if (cudaEventCreate(&e1) != cudaSuccess) { cudaEventDestroy(e0); return ODIN_ERR_CUDA; }
+  float best_ms = 0.f;
+  for (int rep = 0; rep < 4; ++rep) {  // the first repetition warms up
+    cudaEventRecord(e0, st);
+    fp32_peak_kernel<<<blocks, 256, 0, st>>>(sink, iters, 0.999f, 1e-3f);
+    cudaEventRecord(e1, st);
+    if (cudaEventSynchronize(e1) != cudaSuccess) { cudaEventDestroy(e0); cudaEventDestroy(e1); return ODIN_ERR_CUDA; }
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, e0, e1);
+    if (rep > 0 && (best_ms == 0.f || ms < best_ms)) best_ms = ms;
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  const double flops = 2.0 * FMA_CHAINS * (double)iters * 256.0 * (double)blocks;
+  *h_tflops = best_ms > 0.f ? (float)(flops / (best_ms * 1e-3) / 1e12) : 0.f;
+  return odin_launch_status();
 }
 
 extern "C" int odin_workspace_bytes(const odin_ctx* ctx, uint32_t n, uint64_t max_instances, size_t* bytes) {

@@ -278,6 +278,43 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
   }
 }
 
+// Measurement aid (not part of the view step): how many (pixel, list entry) pairs the compositing of a view consists
+// of.  One block per tile, one pixel per thread, the same tests as the forward kernels.  counts[0]: pairs inside the
+// pixel's walked prefix (entries up to the last one that contributed to the pixel); counts[1]: those that blend (pass
+// the skip tests): the pairs the backward pass differentiates.
+__global__ void __launch_bounds__(256)
+count_pairs_kernel(const float2* __restrict__ xy, const float4* __restrict__ conic_o, const uint32_t* __restrict__ vals,
+                   const uint2* __restrict__ ranges, int W, int H, int TX, float alpha_min, float alpha_max,
+                   const uint32_t* __restrict__ n_contrib, uint32_t row_cap, unsigned long long* __restrict__ counts) {
+  const int tile = blockIdx.x;
+  const int px = (tile % TX) * 16 + (int)(threadIdx.x & 15), py = (tile / TX) * 16 + (int)(threadIdx.x >> 4);
+  unsigned long long walked = 0, blended = 0;
+  if (px < W && py < H) {
+    const uint32_t start = ranges[tile].x;
+    const uint32_t n = min(n_contrib[(size_t)py * W + px], ranges[tile].y - start);
+    const float fx = (float)px + 0.5f, fy = (float)py + 0.5f;
+    walked = n;
+    for (uint32_t k = 0; k < n; ++k) {
+      const uint32_t r = min(vals[start + k], row_cap - 1);
+      const float2 c = xy[r];
+      const float4 q = conic_o[r];
+      const float dx = c.x - fx, dy = c.y - fy;
+      const float power = -0.5f * (q.x * dx * dx + q.z * dy * dy) - q.y * dx * dy;
+      if (power > 0.f) continue;
+      if (fminf(alpha_max, q.w * __expf(power)) < alpha_min) continue;
+      ++blended;
+    }
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    walked += __shfl_xor_sync(0xffffffffu, walked, o);
+    blended += __shfl_xor_sync(0xffffffffu, blended, o);
+  }
+  if ((threadIdx.x & 31) == 0 && walked) {
+    atomicAdd(&counts[0], walked);
+    atomicAdd(&counts[1], blended);
+  }
+}
+
 constexpr int LB = 256;
 
 __global__ void __launch_bounds__(LB)
@@ -360,6 +397,24 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
       ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_first, header + 2,
       reinterpret_cast<uint2*>(base + L.seg_tile), reinterpret_cast<uint2*>(base + L.seg_link),
       reinterpret_cast<BlendRecord*>(base + L.ckpt), L.segments, ctx->d_status, proj->capacity);
+  return odin_launch_status();
+}
+
+extern "C" int odin_count_blend_pairs(odin_ctx* ctx, const odin_projected* proj, const uint32_t* d_vals,
+                                      const uint32_t* d_tile_ranges, const odin_camera* cam, const uint32_t* d_n_contrib,
+                                      uint64_t* d_counts, void* stream) {
+  if (!ctx || !proj || !d_tile_ranges || !d_n_contrib || !d_counts) return ODIN_ERR_NULL;
+  const int rc = odin_check_camera(cam);
+  if (rc != ODIN_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  ODIN_CUDA(cudaMemsetAsync(d_counts, 0, 16, st));
+  if (proj->capacity == 0) return ODIN_OK;
+  if (!proj->xy || !proj->conic_opacity || !d_vals) return ODIN_ERR_NULL;
+  const int TX = (cam->width + 15) / 16, TY = (cam->height + 15) / 16;
+  count_pairs_kernel<<<TX * TY, 256, 0, st>>>(
+      reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), d_vals,
+      reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, ctx->cfg.alpha_min, ctx->cfg.alpha_max,
+      d_n_contrib, proj->capacity, reinterpret_cast<unsigned long long*>(d_counts));
   return odin_launch_status();
 }
 

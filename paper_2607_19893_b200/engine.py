@@ -128,9 +128,13 @@ class ViewTrainer:
         self.evidence_sum = z(1, torch.float64)
         # one workspace for odin_project / odin_touched_set (sized by the pool) and odin_bin_sort (sized by the rows and,
         # if the image is too large for the counting scatter, by the instances)
-        self.ws = z(max(B.odin_workspace_bytes(self.ctx, self.n, 0),
-                        B.odin_bin_sort_workspace_bytes(self.ctx, self.row_capacity, self.instance_capacity, self.width,
-                                                        self.height)), torch.uint8)
+        sort_ws = []
+        for mode in (0, 1):  # sized for either way of ordering the instances (see choose_instance_sort)
+            B.odin_set_instance_sort(self.ctx, mode)
+            sort_ws.append(B.odin_bin_sort_workspace_bytes(self.ctx, self.row_capacity, self.instance_capacity, self.width,
+                                                           self.height))
+        B.odin_set_instance_sort(self.ctx, 0 if cfg is None else int(cfg.instance_sort))
+        self.ws = z(max(B.odin_workspace_bytes(self.ctx, self.n, 0), *sort_ws), torch.uint8)
         # The render workspace is a buffer of its own: the forward pass leaves per-pixel records for long lists in it
         # that the backward pass of the same view reads, so nothing else may write there in between.  Every 8,208
         # bytes beyond the minimum hold one more record (a further 256 list entries of one tile).
@@ -160,6 +164,28 @@ class ViewTrainer:
         """Sorted values and tile ranges; the sorted 64-bit keys too unless want_keys is False (no later stage reads them)."""
         B.odin_bin_sort(self.ctx, self.proj.struct, self.width, self.height, self.keys if want_keys else None, self.vals,
                         self.instance_capacity, self.ranges, self.ws, stream)
+
+    def choose_instance_sort(self, cam: B.odin_camera, reps: int = 3) -> int:
+        """Warm-up calibration: times odin_bin_sort on the CURRENT projection both ways (CUDA events, a few repetitions)
+        and keeps the faster for the later views.  Synchronises the device; call it outside any timed region, after at
+        least one odin_project.  Returns the mode kept."""
+        stream = torch.cuda.current_stream()
+        best = None
+        for mode in (0, 1):
+            B.odin_set_instance_sort(self.ctx, mode)
+            self.bin_sort(want_keys=False)  # warm
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            ev[0].record(stream)
+            for _ in range(reps):
+                self.bin_sort(want_keys=False)
+            ev[1].record(stream)
+            torch.cuda.synchronize()
+            ms = ev[0].elapsed_time(ev[1]) / reps
+            if best is None or ms < best[1]:
+                best = (mode, ms)
+        B.odin_set_instance_sort(self.ctx, best[0])
+        self.instance_sort = best[0]
+        return best[0]
 
     def render_fwd(self, cam: B.odin_camera, stream=None) -> None:
         B.odin_render_fwd(self.ctx, self.proj.struct, self.vals, self.ranges, cam, self.out, self.final_T, self.n_contrib,
