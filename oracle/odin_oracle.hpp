@@ -43,7 +43,8 @@ struct Config {
   double radius_sigmas = 3.0;      // screen-space extent in standard deviations
   double jac_clamp = 1.3;          // guard on t_x/t_z, t_y/t_z inside the projection Jacobian
   int tile = 16;
-  int binning = 0;                 // 0: rectangle of the radius; 1: additionally cut to the extent of alpha >= alpha_min
+  int binning = 0;                 // 0: rectangle of the radius; 1: additionally cut to the extent of alpha >= alpha_min;
+                                   // 2: only the tiles of that rectangle which the region alpha >= alpha_min reaches
 };
 
 struct CameraD {
@@ -317,6 +318,103 @@ void project(int64_t n, int sh_degree, const Real* means, const Real* log_scales
       rgb[3 * p + ch] = acc;
     }
     clamp_flags[p] = flags;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Exact binning (binning = 2; an optimised-pipeline variant in the sense of Sec. 5: same primitive ids, same image).
+// A primitive keeps a tile of its rectangle only if some pixel of the tile can pass the skip test, i.e. if the region
+// alpha = opac * exp(-q/2) >= alpha_min, the ellipse q(d) = A dx^2 + 2 B dx dy + C dy^2 <= k with k = 2 ln(opac /
+// alpha_min) around the centre, reaches the rectangle spanned by the tile's 16 x 16 pixel centres.  q is convex, so
+// its minimum over that rectangle is 0 when the centre lies inside and otherwise sits on one of the four edges, at the
+// clamped minimiser of the one-dimensional restriction.  The tile is kept iff  min q <= k (1 + 1e-4) + 1e-3 +
+// 2e-6 * (largest value q takes on the rectangle's corners, by absolute terms): the slack covers the rounding of this
+// evaluation and of the per-pixel test, so a dropped tile holds no pixel that passes.  The tiles a primitive keeps in
+// one tile row are reported as the span from the first to the last tile of the row that passes (the set is an
+// interval, the ellipse being convex).  *margin receives the relative distance of the decision to its threshold.
+template <class Real>
+bool tile_reached(Real u, Real v, Real A, Real B, Real C, Real opac, const Config& cfg, int tx, int ty, Real* margin) {
+  const Real amin = (Real)cfg.alpha_min;
+  if (!(opac >= amin)) { if (margin) *margin = std::abs(opac - amin) / amin; return false; }
+  const Real k = 2 * std::log(opac / amin);
+  const Real T = (Real)cfg.tile;
+  const Real xl = (Real)tx * T + (Real)0.5 - u, xh = xl + (T - 1);
+  const Real yl = (Real)ty * T + (Real)0.5 - v, yh = yl + (T - 1);
+  auto q = [&](Real dx, Real dy) { return A * dx * dx + 2 * B * dx * dy + C * dy * dy; };
+  auto clampv = [](Real x, Real lo, Real hi) { return std::min(std::max(x, lo), hi); };
+  Real qmin;
+  if (xl <= 0 && xh >= 0 && yl <= 0 && yh >= 0) {
+    qmin = 0;
+  } else {
+    // edges x = xl, x = xh: minimise over dy; edges y = yl, y = yh: minimise over dx
+    const Real q0 = q(xl, clampv(-B * xl / C, yl, yh)), q1 = q(xh, clampv(-B * xh / C, yl, yh));
+    const Real q2 = q(clampv(-B * yl / A, xl, xh), yl), q3 = q(clampv(-B * yh / A, xl, xh), yh);
+    qmin = std::min(std::min(q0, q1), std::min(q2, q3));
+  }
+  const Real mx = std::max(std::abs(xl), std::abs(xh)), my = std::max(std::abs(yl), std::abs(yh));
+  const Real big = A * mx * mx + 2 * std::abs(B) * mx * my + C * my * my;
+  const Real bound = k * (Real)1.0001 + (Real)1e-3 + (Real)2e-6 * big;
+  if (margin) *margin = std::abs(qmin - bound) / std::max<Real>(bound, 1);
+  return qmin <= bound;
+}
+
+// Spans of the kept tiles for every (primitive, tile row of its rectangle).  span_ptr [n + 1]: prefix of the
+// rectangles' heights; span_x [2 * span_ptr[n]]: first and one-past-last kept tile of each tile row (equal = none).
+// tiles_touched is replaced by the number of kept tiles; margin is lowered to the closest tile decision.
+template <class Real>
+void tile_spans(int64_t n, const Real* xy, const Real* conic_o, const int32_t* rect, const Config& cfg,
+                const int64_t* span_ptr, int32_t* span_x, uint32_t* tiles_touched, Real* margin) {
+#pragma omp parallel for schedule(dynamic, 256)
+  for (int64_t p = 0; p < n; ++p) {
+    if (tiles_touched[p] == 0) continue;
+    const int x0 = rect[4 * p], y0 = rect[4 * p + 1], x1 = rect[4 * p + 2], y1 = rect[4 * p + 3];
+    uint32_t kept = 0;
+    Real mg = margin[p];
+    for (int ty = y0; ty < y1; ++ty) {
+      int first = x1, last = x0 - 1;
+      for (int tx = x0; tx < x1; ++tx) {
+        Real m1;
+        if (tile_reached(xy[2 * p], xy[2 * p + 1], conic_o[4 * p], conic_o[4 * p + 1], conic_o[4 * p + 2],
+                         conic_o[4 * p + 3], cfg, tx, ty, &m1)) {
+          first = std::min(first, tx);
+          last = std::max(last, tx);
+        }
+        mg = std::min(mg, m1);
+      }
+      int32_t* sp = span_x + 2 * (span_ptr[p] + (ty - y0));
+      if (last >= first) { sp[0] = first; sp[1] = last + 1; kept += (uint32_t)(last + 1 - first); }
+      else { sp[0] = x0; sp[1] = x0; }
+    }
+    tiles_touched[p] = kept;
+    margin[p] = mg;
+  }
+}
+
+// Binning and sort from spans: as bin_sort, the instances of a primitive being the kept tiles of its rectangle in
+// row-major order.
+inline void bin_sort_spans(int64_t n, const float* depth32, const int32_t* rect, const uint32_t* tiles_touched,
+                           const int64_t* span_ptr, const int32_t* span_x, int TX, int TY, uint64_t* keys, uint32_t* vals,
+                           uint32_t* ranges) {
+  std::vector<std::pair<uint64_t, uint32_t>> kv;
+  uint64_t M = 0;
+  for (int64_t p = 0; p < n; ++p) M += tiles_touched[p];
+  kv.reserve(M);
+  for (int64_t p = 0; p < n; ++p) {
+    if (tiles_touched[p] == 0) continue;
+    uint32_t bits;
+    std::memcpy(&bits, &depth32[p], 4);
+    for (int ty = rect[4 * p + 1]; ty < rect[4 * p + 3]; ++ty) {
+      const int32_t* sp = span_x + 2 * (span_ptr[p] + (ty - rect[4 * p + 1]));
+      for (int tx = sp[0]; tx < sp[1]; ++tx) kv.emplace_back(((uint64_t)(uint32_t)(ty * TX + tx) << 32) | bits, (uint32_t)p);
+    }
+  }
+  std::stable_sort(kv.begin(), kv.end(), [](const auto& a, const auto& b) { return a.first < b.first; });
+  for (uint64_t i = 0; i < M; ++i) { keys[i] = kv[i].first; vals[i] = kv[i].second; }
+  uint64_t pos = 0;
+  for (int t = 0; t < TX * TY; ++t) {
+    ranges[2 * t] = (uint32_t)pos;
+    while (pos < M && (uint32_t)(keys[pos] >> 32) == (uint32_t)t) ++pos;
+    ranges[2 * t + 1] = (uint32_t)pos;
   }
 }
 

@@ -13,7 +13,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = os.path.join(_HERE, "liboracle.so")
 _SRC = [os.path.join(_HERE, "oracle_capi.cpp"), os.path.join(_HERE, "odin_oracle.hpp")]
 
-# alpha_min, alpha_max, t_min, dilation, radius_sigmas, jac_clamp, tile, binning (0 plain rectangle, 1 tight extent)
+# alpha_min, alpha_max, t_min, dilation, radius_sigmas, jac_clamp, tile, binning (0 plain rectangle, 1 tight extent,
+# 2 exact: only the tiles the region alpha >= alpha_min reaches)
 DEFAULT_CFG = np.array([1.0 / 255.0, 0.99, 1e-4, 0.3, 3.0, 1.3, 16.0, 0.0], dtype=np.float64)
 
 
@@ -57,6 +58,8 @@ class Projected:
     tiles_touched: np.ndarray  # [N] uint32
     clamp_flags: np.ndarray  # [N] uint8, bit ch set when colour channel ch was clamped at 0
     margin: np.ndarray  # [N] relative distance to the nearest decision threshold
+    span_ptr: Optional[np.ndarray] = None  # binning 2: [N+1] prefix of the rectangles' heights (tile rows)
+    span_x: Optional[np.ndarray] = None  # binning 2: [span_ptr[N], 2] first / one-past-last kept tile of each tile row
 
 
 class Oracle:
@@ -110,7 +113,25 @@ class Oracle:
             _p(out.xy), _p(out.depth), _p(out.conic_o), _p(out.rgb), _p(out.radius), _p(out.rect),
             _p(out.tiles_touched), _p(out.clamp_flags), _p(out.margin),
         )
+        if int(self.cfg[7]) == 2:
+            # exact binning: of every rectangle only the tiles the region alpha >= alpha_min reaches; a primitive that
+            # keeps no tile is not visible
+            h = np.where(out.tiles_touched > 0, out.rect[:, 3] - out.rect[:, 1], 0).astype(np.int64)
+            out.span_ptr = np.concatenate([[0], np.cumsum(h)]).astype(np.int64)
+            out.span_x = np.zeros((int(out.span_ptr[-1]), 2), np.int32)
+            self._f("oracle_tile_spans")(C.c_int64(n), _p(out.xy), _p(out.conic_o), _p(out.rect), _p(self.cfg),
+                                         _p(out.span_ptr), _p(out.span_x), _p(out.tiles_touched), _p(out.margin))
+            gone = out.tiles_touched == 0
+            for a in (out.xy, out.depth, out.conic_o, out.rgb, out.radius, out.rect, out.clamp_flags):
+                a[gone] = 0
         return out
+
+    def tile_reached(self, u, v, conic_o, tx: int, ty: int) -> bool:
+        """The exact-binning rule for one (primitive, tile) pair: can a pixel of the tile pass the skip test?"""
+        ct = C.c_float if self.dtype == np.float32 else C.c_double
+        a, b, c, o = (float(x) for x in conic_o)
+        return bool(self._f("oracle_tile_reached")(ct(u), ct(v), ct(a), ct(b), ct(c), ct(o), _p(self.cfg), C.c_int(tx),
+                                                   C.c_int(ty)))
 
     def touched_set(self, tiles_touched: np.ndarray):
         tt = np.ascontiguousarray(tiles_touched, dtype=np.uint32)
@@ -130,6 +151,11 @@ class Oracle:
         ranges = np.zeros((tx * ty, 2), np.uint32)
         d32 = np.ascontiguousarray(proj.depth, dtype=np.float32)
         rect = np.ascontiguousarray(proj.rect, dtype=np.int32)
+        if proj.span_ptr is not None:
+            self.lib.oracle_bin_sort_spans(C.c_int64(n), _p(d32), _p(rect), _p(tt), _p(proj.span_ptr),
+                                           _p(np.ascontiguousarray(proj.span_x, np.int32)), C.c_int(tx), C.c_int(ty),
+                                           _p(keys), _p(vals), _p(ranges))
+            return keys, vals, ranges
         self.lib.oracle_bin_sort(C.c_int64(n), _p(d32), _p(rect), _p(tt), C.c_int(tx), C.c_int(ty), _p(keys), _p(vals),
                                  _p(ranges))
         return keys, vals, ranges

@@ -74,6 +74,15 @@ Config cfg_from(const double* c) {
   }                                                                                                                    \
   extern "C" void oracle_sh_basis_##SUF(int degree, Real x, Real y, Real z, Real* Y) {                                \
     sh_basis<Real>(degree, x, y, z, Y);                                                                                \
+  }                                                                                                                    \
+  extern "C" void oracle_tile_spans_##SUF(int64_t n, const Real* xy, const Real* conic_o, const int32_t* rect,        \
+                                          const double* cfg, const int64_t* span_ptr, int32_t* span_x,                 \
+                                          uint32_t* tiles_touched, Real* margin) {                                     \
+    tile_spans<Real>(n, xy, conic_o, rect, cfg_from(cfg), span_ptr, span_x, tiles_touched, margin);                    \
+  }                                                                                                                    \
+  extern "C" int oracle_tile_reached_##SUF(Real u, Real v, Real A, Real B, Real C, Real opac, const double* cfg,      \
+                                           int tx, int ty) {                                                           \
+    return tile_reached<Real>(u, v, A, B, C, opac, cfg_from(cfg), tx, ty, (Real*)nullptr) ? 1 : 0;                     \
   }
 
 ORACLE_DEFINE(f32, float)
@@ -88,6 +97,11 @@ extern "C" uint64_t oracle_count_instances(int64_t n, const uint32_t* tiles_touc
 extern "C" void oracle_bin_sort(int64_t n, const float* depth32, const int32_t* rect, const uint32_t* tiles_touched,
                                 int TX, int TY, uint64_t* keys, uint32_t* vals, uint32_t* ranges) {
   bin_sort(n, depth32, rect, tiles_touched, TX, TY, keys, vals, ranges);
+}
+extern "C" void oracle_bin_sort_spans(int64_t n, const float* depth32, const int32_t* rect, const uint32_t* tiles_touched,
+                                      const int64_t* span_ptr, const int32_t* span_x, int TX, int TY, uint64_t* keys,
+                                      uint32_t* vals, uint32_t* ranges) {
+  bin_sort_spans(n, depth32, rect, tiles_touched, span_ptr, span_x, TX, TY, keys, vals, ranges);
 }
 extern "C" uint64_t oracle_conflict_count(const uint32_t* idx_a, uint32_t na, const uint32_t* idx_b, uint32_t nb) {
   return conflict_count(idx_a, na, idx_b, nb);
