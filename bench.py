@@ -317,7 +317,7 @@ def run_config(args, cfg_id, steps, warmup, rank, local_rank, world, want_cpu_ba
     sampler = ClockSampler(local_rank) if rank == 0 else None  # started early: nvidia-smi takes a while to come up
     for s in range(warmup):
         step(s, bank[view_of(s)])
-        if s == 0 and args.instance_sort < 0:
+        if s == 0 and args.instance_sort < 0 and args.binning != 2:  # (exact binning exists in the scatter only)
             # warm-up calibration: order the instances of this first view both ways, keep the faster (outside the timed
             # region; the choice is reported in `config`)
             tr.choose_instance_sort(cams[view_of(0)])
@@ -571,9 +571,10 @@ def main():
     ap.add_argument("--impl", default="odin", choices=["odin", "reference"])
     ap.add_argument("--no-kernel-events", action="store_true", help="do not bracket kernels with CUDA events")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--binning", type=int, default=0, choices=[0, 1],
+    ap.add_argument("--binning", type=int, default=0, choices=[0, 1, 2],
                     help="0: tile rectangle of the radius (the method as published, the default and the headline); "
-                         "1: tight-extent rectangles (same image and gradients, fewer instances)")
+                         "1: tight-extent rectangles; 2: exact binning, only the tiles the splat's alpha >= alpha_min "
+                         "region reaches (both: same image and gradients, fewer instances)")
     ap.add_argument("--instance-sort", type=int, default=-1, choices=[-1, 0, 1],
                     help="how odin_bin_sort orders the instances: 0 counting scatter, 1 radix passes, -1 (default) the "
                          "faster of the two on the first warm-up view")

@@ -59,7 +59,16 @@ typedef struct {
                           to the axis-aligned extent of the region where opacity * exp(-q/2) can reach alpha_min
                           (half extents sqrt(2 ln(opacity/alpha_min) * Sigma'_xx), ..._yy; a primitive whose opacity is
                           below alpha_min gets no tile).  An optimised-pipeline variant in the sense of Sec. 5: the
-                          primitive ids, the image and the gradients are unchanged, the instance lists are shorter. */
+                          primitive ids, the image and the gradients are unchanged, the instance lists are shorter.
+                          2: exact binning.  The rectangle stays that of the radius, but a primitive keeps only those of
+                          its tiles that the region opacity * exp(-q/2) >= alpha_min reaches: the minimum of the conic's
+                          quadratic form q over the rectangle of the tile's 16 x 16 pixel centres is at most
+                          2 ln(opacity / alpha_min) (widened for rounding: a dropped tile holds no pixel that passes the
+                          skip test).  The kept tiles of a tile row are one span; tiles_touched counts the kept tiles, a
+                          primitive that keeps none is not visible, and odin_bin_sort recomputes the spans from the
+                          rows (xy, conic_opacity, rect).  Same image, gradients and realized active set; about half
+                          the instances on scenes of large splats.  Needs the counting scatter (instance_sort 0 on an
+                          image within its limits); otherwise odin_bin_sort returns ODIN_ERR_UNSUPPORTED. */
   int instance_sort;   /* how odin_bin_sort orders the (tile, row) instances; the result is the same either way.
                           0: counting scatter (per-chunk tile counts from the rectangles, every instance written once, to
                           its final place) for images of up to 768 x 40,000 tiles (per row / in all), radix passes beyond;

@@ -10,7 +10,7 @@ extern "C" int odin_create(odin_ctx** out, int device, const odin_config* cfg) {
   odin_config c = {1.0f / 255.0f, 0.99f, 1e-4f, 0.3f, 3.0f, 1.3f, 16, 0, 0};
   if (cfg) c = *cfg;
   if (c.tile != 16) return ODIN_ERR_UNSUPPORTED;
-  if (c.binning != 0 && c.binning != 1) return ODIN_ERR_INVALID_ARG;
+  if (c.binning < 0 || c.binning > 2) return ODIN_ERR_INVALID_ARG;
   if (c.instance_sort != 0 && c.instance_sort != 1) return ODIN_ERR_INVALID_ARG;
   if (!(c.alpha_min > 0) || !(c.alpha_max < 1) || !(c.alpha_max > c.alpha_min) || !(c.t_min > 0) || !(c.dilation >= 0) ||
       !(c.radius_sigmas > 0) || !(c.jac_clamp > 0))

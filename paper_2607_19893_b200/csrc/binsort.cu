@@ -8,6 +8,7 @@
 // counts that are accumulated from the rectangles (a difference array over the tile ids), not from the instances.
 #include "common.cuh"
 #include "layout.cuh"
+#include "tilespan.cuh"
 
 namespace {
 
@@ -563,11 +564,18 @@ emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* _
 // One block per chunk, blocks ordered by ticket (one look-back for the running instance offset, which is only needed
 // for the capacity rule: the instances in front of `capacity` in depth order are the ones that exist).  Writes the
 // rectangles in depth order and the chunk's instance count for every tile.
-__global__ void __launch_bounds__(RO_THREADS)
+// EXACT (binning 2): a row's instances are the kept spans of its rectangle's tile rows (tilespan.cuh), recomputed here
+// from the row's centre, conic and opacity, which are also written out in depth order for the scatter kernel.
+// THREADS x ITEMS = OFFSET_TILE rows per block: 256 x 8 for the plain rectangles, 1024 x 2 when the spans have to be
+// computed (that is several hundred instructions per tile row of every rectangle: more warps per chunk)
+template <bool EXACT, int THREADS, int ITEMS>
+__global__ void __launch_bounds__(THREADS)
 chunk_counts_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __restrict__ rect,
-                    const uint32_t* __restrict__ num_rows, uint32_t capacity, int TX, uint32_t n_tiles, uint32_t tiles_pad,
-                    uint32_t* __restrict__ sorted_off, ushort4* __restrict__ sorted_rect, uint32_t* __restrict__ counts,
-                    uint32_t* ticket, uint64_t* state, int* status, int spin_limit) {
+                    const float2* __restrict__ xy, const float4* __restrict__ conic_o, float alpha_min,
+                    const uint32_t* __restrict__ num_rows, const uint64_t* __restrict__ num_instances, uint32_t capacity,
+                    int TX, uint32_t n_tiles, uint32_t tiles_pad, uint32_t* __restrict__ sorted_off,
+                    ushort4* __restrict__ sorted_rect, float4* __restrict__ sorted_geo4, float2* __restrict__ sorted_geo2,
+                    uint32_t* __restrict__ counts, uint32_t* ticket, uint64_t* state, int* status, int spin_limit) {
   extern __shared__ __align__(16) uint32_t s_tdiff[];  // tiles_pad + 8 words
   __shared__ uint32_t s_tile, s_base;
   __shared__ uint32_t s_warp[33];
@@ -577,16 +585,74 @@ chunk_counts_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __re
   __syncthreads();
   const uint32_t tile = s_tile;
   if (tile >= ntiles) return;  // uniform over the block; nobody waits for a chunk past the end
-  for (uint32_t i = threadIdx.x; i < tiles_pad + 8; i += RO_THREADS) s_tdiff[i] = 0;  // (barriers of the scan follow)
-  const uint32_t first = tile * OFFSET_TILE + threadIdx.x * RO_ITEMS;
-  ushort4 rc[RO_ITEMS];
-  uint32_t cnt[RO_ITEMS];
+  for (uint32_t i = threadIdx.x; i < tiles_pad + 8; i += THREADS) s_tdiff[i] = 0;
+  __syncthreads();
+  // only when the view has more instances than the caller's capacity can a row be denied some of its instances (those
+  // at or behind `capacity` in depth order); otherwise the counts do not depend on the running offset
+  const bool cut = *num_instances > (uint64_t)capacity;
+  const uint32_t first = tile * OFFSET_TILE + threadIdx.x * ITEMS;
+  ushort4 rc[ITEMS];
+  uint32_t cnt[ITEMS];
   uint32_t sum = 0;
+  // adds the run of tiles [t0, t0 + len) to the difference array
+  auto add_run = [&](uint32_t t0, uint32_t len) {
+    t0 = min(t0, n_tiles);  // (clamps: see emit_instances_kernel)
+    atomicAdd(&s_tdiff[t0], 1u);
+    atomicSub(&s_tdiff[min(t0 + len, n_tiles)], 1u);
+  };
 #pragma unroll
-  for (int k = 0; k < RO_ITEMS; ++k) {
+  for (int k = 0; k < ITEMS; ++k) {
     rc[k] = make_ushort4(0, 0, 0, 0);
-    if (first + k < V) rc[k] = rect[min(sorted_row[first + k], V - 1)];
-    cnt[k] = ((uint32_t)rc[k].z - (uint32_t)rc[k].x) * ((uint32_t)rc[k].w - (uint32_t)rc[k].y);
+    cnt[k] = 0;
+    SpanConic e;
+    e.k = -1.f;
+    if (first + k < V) {
+      const uint32_t r = min(sorted_row[first + k], V - 1);
+      rc[k] = rect[r];
+      if (EXACT) {
+        const float2 c = xy[r];
+        const float4 q = conic_o[r];
+        e = odin_span_conic(c.x, c.y, q.x, q.y, q.z, q.w, alpha_min);
+        sorted_geo4[first + k] = make_float4(e.u, e.v, e.A, e.B);
+        sorted_geo2[first + k] = make_float2(e.C, e.k);
+      } else {
+        cnt[k] = ((uint32_t)rc[k].z - (uint32_t)rc[k].x) * ((uint32_t)rc[k].w - (uint32_t)rc[k].y);
+      }
+    }
+    if (EXACT) {
+      // a lane walks the tile rows of a low rectangle by itself; the tall rectangles of the warp are walked by all 32
+      // lanes together (one tile row per lane and step)
+      const int h = (int)rc[k].w - (int)rc[k].y;
+      const bool tall = h > 4;
+      if (h > 0 && !tall)
+        for (int y = rc[k].y; y < (int)rc[k].w; ++y) {
+          int xa, xb;
+          odin_row_span(e, y, rc[k].x, rc[k].z, xa, xb);
+          if (xb > xa) {
+            cnt[k] += (uint32_t)(xb - xa);
+            if (!cut) add_run((uint32_t)y * (uint32_t)TX + (uint32_t)xa, (uint32_t)(xb - xa));
+          }
+        }
+      uint32_t todo = __ballot_sync(0xffffffffu, tall);
+      while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const SpanConic q = odin_span_conic_bcast(e, src);
+        const int qx0 = __shfl_sync(0xffffffffu, (int)rc[k].x, src), qy0 = __shfl_sync(0xffffffffu, (int)rc[k].y, src);
+        const int qx1 = __shfl_sync(0xffffffffu, (int)rc[k].z, src), qy1 = __shfl_sync(0xffffffffu, (int)rc[k].w, src);
+        uint32_t kept = 0;
+        for (int y = qy0 + (int)(threadIdx.x & 31); y < qy1; y += 32) {
+          int xa, xb;
+          odin_row_span(q, y, qx0, qx1, xa, xb);
+          if (xb > xa) {
+            kept += (uint32_t)(xb - xa);
+            if (!cut) add_run((uint32_t)y * (uint32_t)TX + (uint32_t)xa, (uint32_t)(xb - xa));
+          }
+        }
+        kept = __reduce_add_sync(0xffffffffu, kept);
+        if ((int)(threadIdx.x & 31) == src) cnt[k] = kept;
+      }
+    }
     sum += cnt[k];
   }
   uint32_t total;
@@ -598,19 +664,33 @@ chunk_counts_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __re
   __syncthreads();
   uint32_t run = s_base + before;
 #pragma unroll
-  for (int k = 0; k < RO_ITEMS; ++k) {
+  for (int k = 0; k < ITEMS; ++k) {
     if (first + k < V) {
       sorted_off[first + k] = run;
       sorted_rect[first + k] = rc[k];
     }
-    uint32_t left = run < capacity ? min(cnt[k], capacity - run) : 0u;
-    const uint32_t w = (uint32_t)rc[k].z - (uint32_t)rc[k].x;
-    for (uint32_t y = rc[k].y; left != 0; ++y) {
-      const uint32_t len = min(w, left);
-      left -= len;
-      const uint32_t t0 = min(y * (uint32_t)TX + (uint32_t)rc[k].x, n_tiles);  // (clamps: see emit_instances_kernel)
-      atomicAdd(&s_tdiff[t0], 1u);
-      atomicSub(&s_tdiff[min(t0 + len, n_tiles)], 1u);
+    if (!EXACT || cut) {
+      // the instances of the row that exist: those in front of `capacity`, its tiles taken in row-major order
+      uint32_t left = run < capacity ? min(cnt[k], capacity - run) : 0u;
+      const uint32_t w = (uint32_t)rc[k].z - (uint32_t)rc[k].x;
+      SpanConic e;
+      if (EXACT && left != 0) {
+        const float4 g4 = sorted_geo4[first + k];  // written above by this thread
+        const float2 g2 = sorted_geo2[first + k];
+        e.u = g4.x; e.v = g4.y; e.A = g4.z; e.B = g4.w; e.C = g2.x; e.k = g2.y;
+      }
+      for (uint32_t y = rc[k].y; left != 0 && y < (uint32_t)rc[k].w; ++y) {
+        uint32_t x0 = rc[k].x, len = w;
+        if (EXACT) {
+          int xa, xb;
+          odin_row_span(e, (int)y, rc[k].x, rc[k].z, xa, xb);
+          x0 = (uint32_t)xa; len = (uint32_t)(xb - xa);
+          if (len == 0) continue;
+        }
+        len = min(len, left);
+        left -= len;
+        add_run(y * (uint32_t)TX + x0, len);
+      }
     }
     run += cnt[k];
   }
@@ -618,7 +698,7 @@ chunk_counts_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __re
   // integrate the difference array: instances of every tile in this chunk
   uint32_t* __restrict__ out = counts + (size_t)tile * tiles_pad;
   uint32_t carry = 0;
-  for (uint32_t b0 = 0; b0 < n_tiles; b0 += RO_THREADS * 4) {
+  for (uint32_t b0 = 0; b0 < n_tiles; b0 += THREADS * 4) {
     const uint32_t t0 = b0 + threadIdx.x * 4;
     uint4 d = make_uint4(0, 0, 0, 0);
     if (t0 < n_tiles) d = *reinterpret_cast<const uint4*>(s_tdiff + t0);  // padded: words past n_tiles are zero or unused
@@ -733,11 +813,15 @@ constexpr int SC_ITEMS = OFFSET_TILE / SC_THREADS;
 constexpr int SC_SUB = 256;
 constexpr int SC_WORDS = SC_SUB / 32;
 constexpr uint32_t SC_BAND_TILES = SCATTER_MAX_TX;  // tiles of a band: band_rows * TX <= this
-constexpr size_t SC_SMEM = (size_t)OFFSET_TILE * (8 + 4 + 4) + (size_t)SC_WORDS * SC_BAND_TILES * 4 + SC_BAND_TILES * 4;
+constexpr size_t SC_SMEM =
+    (size_t)OFFSET_TILE * (8 + 4 + 4 + 2) + (size_t)SC_WORDS * SC_BAND_TILES * 4 + SC_BAND_TILES * 4;
 
-template <bool WIDE>
+// EXACT (binning 2): the tiles of a row inside a tile row are the kept span (tilespan.cuh), recomputed from the row's
+// centre, conic and threshold as chunk_counts_kernel left them in depth order.
+template <bool WIDE, bool EXACT>
 __global__ void __launch_bounds__(SC_THREADS)
-scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const uint32_t* __restrict__ sorted_row,
+scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const float4* __restrict__ sorted_geo4,
+                         const float2* __restrict__ sorted_geo2, const uint32_t* __restrict__ sorted_row,
                          const uint32_t* __restrict__ sorted_off, const uint32_t* __restrict__ num_rows,
                          const uint64_t* __restrict__ num_instances, uint32_t capacity, int TX, int TY, int band_rows,
                          const uint32_t* __restrict__ counts, uint32_t tiles_pad, const uint2* __restrict__ ranges,
@@ -749,6 +833,7 @@ scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const uint32_t
   uint32_t* s_plim = s_prow + OFFSET_TILE;                                   // [OFFSET_TILE] instances they may emit
   uint32_t* s_bits = s_plim + OFFSET_TILE;                                   // [SC_WORDS][band tiles]
   uint32_t* s_pos = s_bits + SC_WORDS * SC_BAND_TILES;                       // [band tiles] next position of the tile
+  uint16_t* s_pidx = reinterpret_cast<uint16_t*>(s_pos + SC_BAND_TILES);     // [OFFSET_TILE] place of the row in its chunk
   __shared__ uint32_t s_warp[33];
   const uint32_t V = *num_rows;
   const uint32_t nchunks = (V + OFFSET_TILE - 1) / OFFSET_TILE;
@@ -784,6 +869,7 @@ scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const uint32_t
           lim = off < capacity ? capacity - off : 0u;
         }
         s_plim[p] = lim;
+        if (EXACT) s_pidx[p] = (uint16_t)(threadIdx.x * SC_ITEMS + k);
         ++p;
       }
     }
@@ -796,46 +882,62 @@ scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const uint32_t
       for (uint32_t i = threadIdx.x; i < SC_WORDS * band_tiles; i += SC_THREADS) s_bits[i] = 0;
       __syncthreads();
       {
-        // A row covers anything from one tile to the whole band.  A lane sets the bits of a small row by itself; the
-        // large rows of a warp are then taken one at a time by all 32 lanes (one tile per lane and step), so that a
-        // splat that fills the band costs the warp a few dozen steps instead of one lane several hundred.
+        // Tile row by tile row of the band: the tiles of a row of the list inside one tile row are a run [xa, xa + len).
+        // A lane sets the bits of a short run by itself; the long runs of a warp are then taken one at a time by all 32
+        // lanes (one tile per lane and step), so that a splat as wide as the image costs the warp a few steps instead
+        // of one lane a hundred.
         const uint32_t j = sub + threadIdx.x;
         const unsigned lane = threadIdx.x & 31;
         uint32_t* word = s_bits + (threadIdx.x >> 5) * band_tiles;  // the warp's 32 rows are the bits of these words
-        uint32_t rx = 0, ry = 0, w = 1, lim = 0, ya = 0, yb = 0, x1 = 0;
+        uint32_t rx = 0, ry = 0, ry1 = 0, w = 1, lim = 0, x1 = 0;
+        SpanConic e;
+        e.k = -1.f;
         if (j < npass) {
           const ushort4 r = s_prect[j];
-          rx = r.x; ry = r.y; w = (uint32_t)r.z - (uint32_t)r.x; lim = s_plim[j];
-          ya = max((uint32_t)r.y, by0); yb = min((uint32_t)r.w, by1);
+          rx = r.x; ry = r.y; ry1 = r.w; w = (uint32_t)r.z - (uint32_t)r.x; lim = s_plim[j];
           x1 = min((uint32_t)r.z, (uint32_t)TX);
-        }
-        const uint32_t wb = x1 > rx ? x1 - rx : 0u, cells = (yb > ya ? yb - ya : 0u) * wb;
-        const bool large = cells > 16;
-        if (!large && cells != 0) {
-          const uint32_t bit = 1u << lane;
-          for (uint32_t y = ya; y < yb; ++y) {
-            const uint32_t k0 = (y - ry) * w;  // index of the instance inside the row's rectangle, row major
-            uint32_t* line = word + (y - by0) * (uint32_t)TX;
-            for (uint32_t x = rx; x < x1; ++x)
-              if (k0 + (x - rx) < lim) atomicOr(line + x, bit);  // other lanes of the warp may hold the same tile
+          if (EXACT) {
+            const uint32_t gi = chunk * OFFSET_TILE + s_pidx[j];
+            const float4 g4 = sorted_geo4[gi];
+            const float2 g2 = sorted_geo2[gi];
+            e.u = g4.x; e.v = g4.y; e.A = g4.z; e.B = g4.w; e.C = g2.x; e.k = g2.y;
           }
         }
-        uint32_t todo = __ballot_sync(0xffffffffu, large);
-        __syncwarp();
-        while (todo) {
-          const int src = __ffs(todo) - 1;
-          todo &= todo - 1;
-          const uint32_t q_rx = __shfl_sync(0xffffffffu, rx, src), q_ry = __shfl_sync(0xffffffffu, ry, src);
-          const uint32_t q_w = __shfl_sync(0xffffffffu, w, src), q_lim = __shfl_sync(0xffffffffu, lim, src);
-          const uint32_t q_ya = __shfl_sync(0xffffffffu, ya, src), q_wb = __shfl_sync(0xffffffffu, wb, src);
-          const uint32_t q_cells = __shfl_sync(0xffffffffu, cells, src);
-          const uint32_t bit = 1u << src;
-          for (uint32_t c = lane; c < q_cells; c += 32) {  // distinct tiles per lane: no two lanes share a word here
-            const uint32_t dy = c / q_wb, dx = c - dy * q_wb;
-            const uint32_t y = q_ya + dy;
-            if ((y - q_ry) * q_w + dx < q_lim) word[(y - by0) * (uint32_t)TX + q_rx + dx] |= bit;
+        for (uint32_t y = by0; y < by1; ++y) {
+          uint32_t xa = 0, len = 0, k0 = 0;  // the lane's run in this tile row; k0: index of its first instance in the row
+          if (j < npass && y >= ry && y < ry1) {
+            if (EXACT) {
+              int a, b;
+              odin_row_span(e, (int)y, (int)rx, (int)x1, a, b);
+              xa = (uint32_t)a; len = (uint32_t)(b - a);
+              if (cut && len != 0)  // instances of the tile rows above (rare path: the view overflows the capacity)
+                for (uint32_t yy = ry; yy < y; ++yy) {
+                  odin_row_span(e, (int)yy, (int)rx, (int)x1, a, b);
+                  k0 += (uint32_t)(b - a);
+                }
+            } else {
+              xa = rx; len = x1 > rx ? x1 - rx : 0u; k0 = (y - ry) * w;
+            }
           }
+          uint32_t* line = word + (y - by0) * (uint32_t)TX;
+          const bool large = len > 16;
+          if (!large) {
+            const uint32_t bit = 1u << lane;
+            for (uint32_t i = 0; i < len; ++i)
+              if (k0 + i < lim) atomicOr(line + xa + i, bit);  // other lanes of the warp may hold the same tile
+          }
+          uint32_t todo = __ballot_sync(0xffffffffu, large);
           __syncwarp();
+          while (todo) {
+            const int src = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const uint32_t q_xa = __shfl_sync(0xffffffffu, xa, src), q_len = __shfl_sync(0xffffffffu, len, src);
+            const uint32_t q_k0 = __shfl_sync(0xffffffffu, k0, src), q_lim = __shfl_sync(0xffffffffu, lim, src);
+            const uint32_t bit = 1u << src;
+            for (uint32_t c = lane; c < q_len; c += 32)  // distinct tiles per lane: no two lanes share a word here
+              if (q_k0 + c < q_lim) line[q_xa + c] |= bit;
+            __syncwarp();
+          }
         }
       }
       __syncthreads();
@@ -904,6 +1006,9 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   const ScatterLayout F = scatter_layout(proj->capacity, n_tiles);
   const BinSortLayout L = binsort_layout(capacity, proj->capacity);
   const bool use_scatter = scatter && ws && ws_bytes >= F.total;
+  const bool exact = ctx->cfg.binning == 2;
+  if (exact && !use_scatter) return ODIN_ERR_UNSUPPORTED;  // the spans of exact binning exist in the scatter path only
+  if (exact && (!proj->xy || !proj->conic_opacity)) return ODIN_ERR_NULL;
   if (!ws || !odin_aligned(ws, 256) || (!use_scatter && ws_bytes < L.total)) return ODIN_ERR_WORKSPACE;
   char* base = reinterpret_cast<char*>(ws);
   const int tile_passes = tile_digit_passes(n_tiles);
@@ -967,15 +1072,26 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     ushort4* sorted_rect = reinterpret_cast<ushort4*>(base + F.sorted_rect);
     uint32_t* tile_total = reinterpret_cast<uint32_t*>(base + F.tile_total);
     uint32_t* counts = reinterpret_cast<uint32_t*>(base + F.counts);
+    float4* geo4 = reinterpret_cast<float4*>(base + F.sorted_geo4);
+    float2* geo2 = reinterpret_cast<float2*>(base + F.sorted_geo2);
     const uint32_t cap32 = (uint32_t)capacity;
     {
       OdinKernelScope ks(ctx, K_ROW_OFFSETS, st);
       const size_t smem = ((size_t)F.tiles_pad + 8) * 4;
-      ODIN_CUDA(cudaFuncSetAttribute(chunk_counts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)(((size_t)SCATTER_MAX_TILES + 64 + 8) * 4)));
-      chunk_counts_kernel<<<F.chunks, RO_THREADS, smem, st>>>(sorted_row, rect, proj->num_rows, cap32, TX, n_tiles,
-                                                             F.tiles_pad, sorted_off, sorted_rect, counts, tickets + 8,
-                                                             scan_state, ctx->d_status, ctx->spin_limit);
+      const int max_smem = (int)(((size_t)SCATTER_MAX_TILES + 64 + 8) * 4);
+      static_assert(RO_THREADS * RO_ITEMS == (int)OFFSET_TILE && 1024 * 2 == (int)OFFSET_TILE, "rows per chunk");
+      ODIN_CUDA(cudaFuncSetAttribute(chunk_counts_kernel<false, RO_THREADS, RO_ITEMS>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+      ODIN_CUDA(cudaFuncSetAttribute(chunk_counts_kernel<true, 1024, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     max_smem));
+#define LAUNCH_COUNTS(EXACT, THREADS, ITEMS)                                                                           \
+  chunk_counts_kernel<EXACT, THREADS, ITEMS><<<F.chunks, THREADS, smem, st>>>(                                         \
+      sorted_row, rect, reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), \
+      ctx->cfg.alpha_min, proj->num_rows, proj->num_instances, cap32, TX, n_tiles, F.tiles_pad, sorted_off, sorted_rect, \
+      geo4, geo2, counts, tickets + 8, scan_state, ctx->d_status, ctx->spin_limit)
+      if (exact) LAUNCH_COUNTS(true, 1024, 2);
+      else LAUNCH_COUNTS(false, RO_THREADS, RO_ITEMS);
+#undef LAUNCH_COUNTS
     }
     {
       OdinKernelScope ks(ctx, K_TILE_BASES, st);
@@ -993,16 +1109,17 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
       if (band_rows > TY) band_rows = TY;
       const uint64_t items_cap = (uint64_t)F.chunks * (((uint32_t)TY + band_rows - 1) / band_rows);
       const uint32_t grid = (uint32_t)(items_cap < (uint64_t)sms * 3 ? items_cap : (uint64_t)sms * 3);
-      ODIN_CUDA(cudaFuncSetAttribute(scatter_instances_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM));
-      ODIN_CUDA(cudaFuncSetAttribute(scatter_instances_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM));
-      if (d_keys)
-        scatter_instances_kernel<true><<<grid, SC_THREADS, SC_SMEM, st>>>(
-            sorted_rect, sorted_row, sorted_off, proj->num_rows, proj->num_instances, cap32, TX, TY, band_rows, counts,
-            F.tiles_pad, reinterpret_cast<const uint2*>(d_tile_ranges), d_vals, d_keys, depth_bits);
-      else
-        scatter_instances_kernel<false><<<grid, SC_THREADS, SC_SMEM, st>>>(
-            sorted_rect, sorted_row, sorted_off, proj->num_rows, proj->num_instances, cap32, TX, TY, band_rows, counts,
-            F.tiles_pad, reinterpret_cast<const uint2*>(d_tile_ranges), d_vals, nullptr, depth_bits);
+#define LAUNCH_SCATTER(WIDE, EXACT)                                                                                    \
+  do {                                                                                                                 \
+    ODIN_CUDA(cudaFuncSetAttribute(scatter_instances_kernel<WIDE, EXACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
+                                   (int)SC_SMEM));                                                                     \
+    scatter_instances_kernel<WIDE, EXACT><<<grid, SC_THREADS, SC_SMEM, st>>>(                                          \
+        sorted_rect, geo4, geo2, sorted_row, sorted_off, proj->num_rows, proj->num_instances, cap32, TX, TY, band_rows, \
+        counts, F.tiles_pad, reinterpret_cast<const uint2*>(d_tile_ranges), d_vals, d_keys, depth_bits);               \
+  } while (0)
+      if (d_keys) { if (exact) LAUNCH_SCATTER(true, true); else LAUNCH_SCATTER(true, false); }
+      else { if (exact) LAUNCH_SCATTER(false, true); else LAUNCH_SCATTER(false, false); }
+#undef LAUNCH_SCATTER
     }
     return odin_launch_status();
   }

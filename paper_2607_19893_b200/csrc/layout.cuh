@@ -93,6 +93,8 @@ struct ScatterLayout {
   size_t row_keys[2], row_vals[2];
   size_t sorted_off;   // u32[rows + 1]
   size_t sorted_rect;  // ushort4[rows] rectangles in depth order
+  size_t sorted_geo4;  // float4[rows] (u, v, conic A, B) in depth order   } exact binning only: what the span of a
+  size_t sorted_geo2;  // float2[rows] (conic C, 2 ln(opacity / alpha_min)) } tile row is computed from
   size_t tile_total;   // u32[tiles]
   size_t counts;       // u32[chunks][tiles_pad]: instances of the tile in the chunk, then their exclusive prefix over the chunks
   size_t total;
@@ -115,6 +117,8 @@ static inline ScatterLayout scatter_layout(uint32_t rows, uint32_t n_tiles) {
   for (int b = 0; b < 2; ++b) { L.row_vals[b] = o; o += ws_align((size_t)rows * 4); }
   L.sorted_off = o; o += ws_align((size_t)rows * 4 + 4);
   L.sorted_rect = o; o += ws_align((size_t)rows * 8);
+  L.sorted_geo4 = o; o += ws_align((size_t)rows * 16);
+  L.sorted_geo2 = o; o += ws_align((size_t)rows * 8);
   L.tile_total = o; o += ws_align((size_t)n_tiles * 4);
   L.counts = o; o += ws_align((size_t)L.chunks * L.tiles_pad * 4);
   L.total = o;

@@ -9,6 +9,7 @@
 // through a block-wide scan in the first kernel.
 #include "geom.cuh"
 #include "layout.cuh"
+#include "tilespan.cuh"
 
 namespace {
 
@@ -97,13 +98,44 @@ __device__ __forceinline__ Footprint project_footprint(const CamParams& cam, con
   return f;
 }
 
+template <bool EXACT>  // EXACT: binning 2 (a separate instantiation: the default path does not carry its registers)
 __global__ void __launch_bounds__(256)
 project_cull_kernel(const float* __restrict__ means, const float* __restrict__ log_scales, const float4* __restrict__ quats,
                     const float* __restrict__ opacity_logit, uint32_t n, CamParams cam, BinRule rule,
                     uint32_t* __restrict__ tiles_touched) {
   const uint32_t p = blockIdx.x * 256u + threadIdx.x;
-  if (p >= n) return;
-  tiles_touched[p] = project_footprint<true>(cam, rule, means, log_scales, quats, opacity_logit, p).tiles;
+  Footprint f = {};
+  if (p < n) f = project_footprint<true>(cam, rule, means, log_scales, quats, opacity_logit, p);
+  if (EXACT) {
+    // exact binning: of the rectangle only the tiles the splat's alpha >= alpha_min region reaches (tilespan.cuh).  A
+    // lane counts a rectangle of few tile rows by itself; the tall ones of the warp are counted by all 32 lanes together.
+    SpanConic e;
+    e.k = -1.f;
+    if (f.tiles != 0) {
+      const float opac = 1.f / (1.f + expf(-opacity_logit[p]));
+      e = odin_span_conic(f.u, f.v, f.cA, f.cB, f.cC, opac, rule.alpha_min);
+    }
+    const bool tall = f.tiles != 0 && f.y1 - f.y0 > 4;
+    if (f.tiles != 0 && !tall) {
+      uint32_t kept = 0;
+      for (int ty = f.y0; ty < f.y1; ++ty) {
+        int xa, xb;
+        odin_row_span(e, ty, f.x0, f.x1, xa, xb);
+        kept += (uint32_t)(xb - xa);
+      }
+      f.tiles = kept;
+    }
+    uint32_t todo = __ballot_sync(0xffffffffu, tall);
+    while (todo) {
+      const int src = __ffs(todo) - 1;
+      todo &= todo - 1;
+      const SpanConic q = odin_span_conic_bcast(e, src);
+      const uint32_t kept = odin_rect_kept_warp(q, __shfl_sync(0xffffffffu, f.x0, src), __shfl_sync(0xffffffffu, f.y0, src),
+                                                __shfl_sync(0xffffffffu, f.x1, src), __shfl_sync(0xffffffffu, f.y1, src));
+      if ((int)(threadIdx.x & 31) == src) f.tiles = kept;
+    }
+  }
+  if (p < n) tiles_touched[p] = f.tiles;
 }
 
 // packed look-back value: rows in the upper 28 bits, tile instances in the lower 34 bits
@@ -319,8 +351,12 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   const BinRule rule = {ctx->cfg.dilation, ctx->cfg.radius_sigmas, ctx->cfg.alpha_min, ctx->cfg.binning};
   {
     OdinKernelScope ks(ctx, K_PROJECT, st);
-    project_cull_kernel<<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit, n, cp,
-                                                         rule, out->tiles_touched);
+    if (rule.binning == 2)
+      project_cull_kernel<true><<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit,
+                                                                 n, cp, rule, out->tiles_touched);
+    else
+      project_cull_kernel<false><<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4,
+                                                                  scene->opacity_logit, n, cp, rule, out->tiles_touched);
   }
   {
     OdinKernelScope ks(ctx, K_PROJECT_SCAN, st);

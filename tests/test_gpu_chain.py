@@ -359,6 +359,27 @@ def test_chain_tight_extent_binning(oracle32):
     assert np.array_equal(outs[0], outs[1])  # the same pairs blend in the same order: bitwise the same image
 
 
+def test_chain_exact_binning(oracle32):
+    """The whole step with binning = 2 against the oracle in the same mode (every check of run_chain), and against
+    the plain mode: about half the instances, the same image bit for bit."""
+    from test_gpu_stages import exact_oracle
+
+    w = wl.make_workload(3, n=100_000, n_cameras=4, resolution=(400, 267))
+    run_chain(exact_oracle(), w, steps=3, views=[0, 1, 2], cfg=B.default_config(binning=2), tag="cfg3_scaled_binning2")
+    cam = w.cameras[1]
+    outs, m = [], []
+    for binning in (0, 2):
+        tr = G.trainer_for(w.scene, cam, cfg=B.default_config(binning=binning))
+        tr.target.copy_(torch.from_numpy(w.target(1)).to(tr.device))
+        tr.view_step(B.make_camera(cam), 1, w.lr, w.beta1, w.beta2, w.eps, update=False)
+        G.poll_ok(tr)
+        outs.append(tr.out.cpu().numpy())
+        m.append(int(tr.proj.num_instances.item()))
+        tr.close()
+    assert m[1] < 0.7 * m[0]
+    assert np.array_equal(outs[0], outs[1])  # the same pairs blend in the same order: bitwise the same image
+
+
 # ---------------------------------------------------------------------------------------------------------------
 # The two workloads bench.py times, at full size and with the capacities it launches with.  Two consecutive steps, so
 # the second one runs on non-zero Adam moments.  The oracle computes every output (a full view of these sizes takes

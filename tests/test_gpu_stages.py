@@ -232,6 +232,58 @@ def test_project_tight_extent_binning(oracle32):
     check_projection(ot, w2.scene, w2.cameras[6], cfg=B.default_config(binning=1))
 
 
+def exact_oracle():
+    import oracle
+    from oracle.oracle import DEFAULT_CFG
+    cfg = DEFAULT_CFG.copy()
+    cfg[7] = 2
+    return oracle.Oracle(np.float32, cfg=cfg)
+
+
+def test_project_exact_binning(oracle32):
+    """binning = 2: tiles_touched counts the tiles the region alpha >= alpha_min reaches, as the oracle's exact rule has
+    it; primitives that keep no tile leave the touched set."""
+    oe = exact_oracle()
+    w = wl.make_workload(3, n=200_000, resolution=(800, 533))
+    v_exact = check_projection(oe, w.scene, w.cameras[2], cfg=B.default_config(binning=2))
+    po, pe = oracle32.project(w.scene, w.cameras[2]), oe.project(w.scene, w.cameras[2])
+    assert v_exact <= int((po.tiles_touched > 0).sum())
+    assert int(pe.tiles_touched.sum()) < 0.7 * int(po.tiles_touched.sum())
+    w2 = wl.make_workload(4, n=60_000, n_cameras=4, resolution=(960, 540))  # large splats: long spans, the bisection
+    check_projection(oe, w2.scene, w2.cameras[1], cfg=B.default_config(binning=2))
+
+
+def test_bin_sort_exact_binning(oracle32):
+    """binning = 2 through odin_bin_sort: the device recomputes the spans from the rows it is given (here the oracle's)
+    and must produce the oracle's lists.  Its logarithm may differ from the host's in the last place, so a primitive
+    with a tile decision within 1e-5 of the threshold is left out of the comparison on both sides."""
+    oe = exact_oracle()
+    for w, cam_i in ((wl.make_workload(3, n=120_000), 7), (wl.make_workload(4, n=40_000, n_cameras=4, resolution=(960, 540)), 1)):
+        cam = w.cameras[cam_i]
+        po = oe.project(w.scene, cam)
+        mask, idx = oe.touched_set(po.tiles_touched)
+        keys_o, vals_o, ranges_o = oe.bin_sort(po, cam)
+        m = len(keys_o)
+        tr = G.trainer_for(w.scene, cam, row_capacity=max(len(idx), 1), instance_capacity=m + 4096,
+                           cfg=B.default_config(binning=2))
+        G.load_oracle_projection(tr, po, idx)
+        tr.keys.fill_(-1)
+        tr.vals.fill_(-1)
+        tr.bin_sort()
+        G.poll_ok(tr)
+        rg = G.u32(tr.ranges).astype(np.int64)
+        m_dev = int(rg[-1, 1])
+        keys_d, prims_d = G.u64(tr.keys)[:m_dev], idx[G.u32(tr.vals)[:m_dev]]
+        assert np.all(keys_d[1:] >= keys_d[:-1])
+        assert np.array_equal(np.repeat(np.arange(len(rg)), rg[:, 1] - rg[:, 0]), (keys_d >> np.uint64(32)).astype(np.int64))
+        fragile = po.margin < 1e-5
+        keep_d, keep_o = ~fragile[prims_d], ~fragile[vals_o]
+        assert np.array_equal(keys_d[keep_d], keys_o[keep_o]) and np.array_equal(prims_d[keep_d], vals_o[keep_o])
+        G.report("bin_sort exact", M=m, M_dev=m_dev, fragile_prims=int(fragile[idx].sum()), rows=len(idx))
+        assert abs(m_dev - m) <= int(po.tiles_touched[fragile].sum()) and fragile[idx].mean() < 0.01
+        tr.close()
+
+
 def test_project_row_capacity_overflow(oracle32):
     w = wl.make_workload(1)
     tr = G.trainer_for(w.scene, w.cameras[0], row_capacity=100)
