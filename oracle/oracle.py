@@ -289,6 +289,29 @@ class Oracle:
                                and passes.all())
         return out
 
+    # ------------------------------------------------------------------ task units of several views (Sec. 2.1, Sec. 6.1)
+    @staticmethod
+    def accumulate_rows(idx_a, rows_a, idx_b, rows_b):
+        """Gradient rows of a task unit of two views (Sec. 2.1: the unit's scope is the union of its views' scopes;
+        Sec. 6.1 runs two views per unit): the union of the two ascending index lists and, per member, the sum of the
+        rows the views hold for it (a view that did not touch the primitive contributes nothing)."""
+        idx_a, idx_b = np.asarray(idx_a, np.int64), np.asarray(idx_b, np.int64)
+        union = np.union1d(idx_a, idx_b)
+        out = np.zeros((len(union), np.asarray(rows_a).shape[1]), np.float64)
+        out[np.searchsorted(union, idx_a)] += np.asarray(rows_a, np.float64)
+        out[np.searchsorted(union, idx_b)] += np.asarray(rows_b, np.float64)
+        return union.astype(np.uint32), out
+
+    def unit_step(self, params, m, v, cams, targets, lr, beta1, beta2, eps, step):
+        """One task unit of two views: both are rendered and differentiated with the SAME parameters, their gradient
+        rows are accumulated over the union of their touched sets, and one sparse Adam update is applied to the union
+        at the unit's step."""
+        views = [self.view_step(params, m, v, cam, tgt, lr, beta1, beta2, eps, step, update=False)
+                 for cam, tgt in zip(cams, targets)]
+        union, rows = self.accumulate_rows(views[0]["idx"], views[0]["rows"], views[1]["idx"], views[1]["rows"])
+        self.sparse_adam(params, m, v, rows.astype(self.dtype), union, lr, beta1, beta2, eps, step)
+        return dict(views=views, idx=union, rows=rows)
+
     # ------------------------------------------------------------------ relative locality graph from counts (Sec. 4.1, 4.2)
     @staticmethod
     def rlg_weights(sizes, pairs, counts) -> np.ndarray:

@@ -224,3 +224,51 @@ def test_rlg_weights_are_jaccard_of_the_sets_and_topk_is_monotone(oracle64):
     # Eq. (2) is additive over the previous unit
     s01 = oracle64.sds_scores(full, [0, 1], [5, 6, 7])
     assert np.allclose(s01, oracle64.sds_scores(full, [0], [5, 6, 7]) + oracle64.sds_scores(full, [1], [5, 6, 7]))
+
+
+# ------------------------------------------------------------------------------- task units of two views (Sec. 2.1, Sec. 6.1)
+def test_accumulate_rows_hand_example(oracle64):
+    idx_a, idx_b = [1, 4, 7], [0, 4, 9]
+    rows_a = np.array([[1.0, 2.0], [3.0, 4.0], [5.0, 6.0]])
+    rows_b = np.array([[10.0, 20.0], [30.0, 40.0], [50.0, 60.0]])
+    union, rows = oracle64.accumulate_rows(idx_a, rows_a, idx_b, rows_b)
+    assert union.tolist() == [0, 1, 4, 7, 9]
+    assert rows.tolist() == [[10, 20], [1, 2], [33, 44], [5, 6], [50, 60]]
+    u2, r2 = oracle64.accumulate_rows(idx_b, rows_b, idx_a, rows_a)            # symmetric
+    assert np.array_equal(union, u2) and np.array_equal(rows, r2)
+    u3, r3 = oracle64.accumulate_rows(idx_a, rows_a, [], np.zeros((0, 2)))    # an empty view adds nothing
+    assert u3.tolist() == idx_a and np.array_equal(r3, rows_a)
+
+
+def test_unit_step_equals_dense_adam_on_the_summed_gradients(oracle64):
+    """Two views with the same parameters, gradients summed, one update: on the rows of the union this is textbook Adam
+    fed with the sum of the two dense gradients (torch.optim.Adam as the library routine), and no other row moves."""
+    import torch
+
+    from paper_2607_19893_b200 import workloads as wl
+
+    w = wl.make_workload(2, n=400)
+    s = w.scene.astype(np.float64)
+    m, v = s.zeros_like(), s.zeros_like()
+    cams, tgts = [w.cameras[0], w.cameras[3]], [w.target(0).astype(np.float64), w.target(3).astype(np.float64)]
+    before = s.copy()
+    lr = w.lr.astype(np.float64)
+    # dense reference: per-view gradients from the oracle's own backward (pinned by finite differences), summed
+    dense = np.zeros((s.n, s.floats_per_primitive))
+    for cam, tgt in zip(cams, tgts):
+        f = oracle64.view_step(before.copy(), m.copy(), v.copy(), cam, tgt, lr, w.beta1, w.beta2, 1e-8, 1, update=False)
+        dense[f["idx"].astype(np.int64)] += f["rows"]
+    touched = np.flatnonzero(np.abs(dense).sum(axis=1) > 0)
+    flat = lambda sc: np.concatenate([sc.means, sc.log_scales, sc.quats, sc.opacity_logit[:, None],  # noqa: E731
+                                      sc.sh.reshape(sc.n, -1)], axis=1)
+    out = oracle64.unit_step(s, m, v, cams, tgts, lr, w.beta1, w.beta2, 1e-8, 1)
+    union = out["idx"].astype(np.int64)
+    assert set(touched) <= set(union)
+    p_t = torch.tensor(flat(before)[union], dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([p_t], lr=float(lr[0]), betas=(w.beta1, w.beta2), eps=1e-8)
+    p_t.grad = torch.tensor(dense[union], dtype=torch.float64)
+    opt.step()
+    assert np.allclose(flat(s)[union], p_t.detach().numpy(), rtol=1e-12, atol=1e-14)
+    rest = np.setdiff1d(np.arange(s.n), union)
+    assert np.array_equal(flat(s)[rest], flat(before)[rest]) and not flat(m)[rest].any()
+    assert np.abs(flat(s)[union] - flat(before)[union]).max() > 1e-5
