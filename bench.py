@@ -414,6 +414,24 @@ def run_config(args, cfg_id, steps, warmup, rank, local_rank, world, want_cpu_ba
                                   "frac_of_measured_hbm": b_hz / (t_hz * 1e-3) / 1e9 / peak_gbs_},
                  "note": "not part of `value`: the realized active set and the hazard counts of Sec. 4.3 for the last "
                          "view against the views before it, each averaged over 20 calls"}
+        # a task unit of two views (Sec. 6.1): both rendered with the same parameters, rows accumulated over the union
+        # of the touched sets, one Adam update
+        va, vb = view_of(total_steps - 2), view_of(total_steps - 1)
+        unit_args = ([cams[va], cams[vb]], [bank[va], bank[vb]])
+        tr.unit_step(*unit_args, total_steps + 1, w.lr, w.beta1, w.beta2, w.eps, slots=(0, 1), stream=stream)  # warm
+        torch.cuda.synchronize()
+        eu = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        unit_reps = 8
+        eu[0].record(stream)
+        for i in range(unit_reps):
+            tr.unit_step(*unit_args, total_steps + 2 + i, w.lr, w.beta1, w.beta2, w.eps, slots=(0, 1), stream=stream)
+        eu[1].record(stream)
+        torch.cuda.synchronize()
+        t_unit = eu[0].elapsed_time(eu[1]) / unit_reps
+        scope["unit_step"] = {"ms_per_unit": t_unit, "views_per_unit": 2, "ms_per_view": t_unit / 2,
+                              "union_size": int(tr._unit["count_u"].item()),
+                              "note": "two views with the same parameters, gradient rows accumulated over the union "
+                                      "list (odin_mask_union, odin_mask_to_list, odin_accumulate_rows), one odin_sparse_adam"}
         st = tr.poll()
         if st != B.ODIN_OK:
             raise SystemExit(f"scope calls failed: {B.status_string(st)}")

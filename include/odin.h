@@ -309,6 +309,23 @@ int odin_active_set(odin_ctx* ctx, const odin_projected* proj, const uint8_t* d_
 int odin_mask_union(odin_ctx* ctx, const uint32_t* d_masks, uint32_t n_masks, uint32_t mask_stride_words,
                     uint32_t n_prims, const uint32_t* d_members, uint32_t n_members, uint32_t* d_out, void* stream);
 
+/* Task units of several views (Sec. 2.1: the scope of a unit is the union of its views' scopes; Sec. 6.1 runs two views
+ * per unit): the views of a unit are rendered and differentiated with the same parameters, their gradient rows are
+ * added up over the union of their touched sets, and ONE optimizer update is applied to the union.
+ * odin_mask_to_list: the ascending list of the members of a bitmask over the primitives (for example the OR of two
+ * views' touched masks from odin_mask_union): d_idx (first idx_capacity members; more defers ODIN_ERR_CAPACITY),
+ * d_count [1].  Bits at or beyond n are ignored.  ws: at least odin_workspace_bytes(n, 0).
+ * odin_accumulate_rows: rows_u[r] = (row of primitive d_idx_u[r] in view a, if a lists it) + (the same for view b),
+ * for r < *d_count_u.  rows_a / rows_b: the compact gradient rows of the two views (row i <-> d_idx_a[i], i <
+ * *d_count_a; d_zero_a: the row_zero flags of odin_render_bwd, may be NULL); rows_u: n >= union size, same SH degree.
+ * odin_sparse_adam(params, m, v, rows_u, NULL, d_idx_u, d_count_u, ...) then updates the unit. */
+int odin_mask_to_list(odin_ctx* ctx, const uint32_t* d_mask, uint32_t n, uint32_t* d_idx, uint32_t idx_capacity,
+                      uint32_t* d_count, void* ws, size_t ws_bytes, void* stream);
+int odin_accumulate_rows(odin_ctx* ctx, const odin_scene* rows_a, const uint8_t* d_zero_a, const uint32_t* d_idx_a,
+                         const uint32_t* d_count_a, const odin_scene* rows_b, const uint8_t* d_zero_b,
+                         const uint32_t* d_idx_b, const uint32_t* d_count_b, const uint32_t* d_idx_u,
+                         const uint32_t* d_count_u, odin_scene* rows_u, void* stream);
+
 /* The three primitive-state hazards of the quality-first path (Sec. 4.3) for pairs (A, B) = (producer, consumer):
  *   WAW = W(B) & W(A);  RAW = (R(B) \ W(B)) & W(A);  WAR = W(B) & (R(A) \ W(A)).
  * d_read_masks, d_write_masks [n_masks][mask_stride_words]: the conservative scopes R^+, W^+ of each unit;

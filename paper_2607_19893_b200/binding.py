@@ -30,6 +30,7 @@ EXPORTS = [
     "odin_touched_set_static", "odin_render_workspace_bytes", "odin_active_set", "odin_mask_union", "odin_hazard_count",
     "odin_delayed_read_gate", "odin_rlg_weights", "odin_rlg_topk", "odin_sds_scores", "odin_set_wait_limit",
     "odin_bin_sort_workspace_bytes", "odin_set_instance_sort", "odin_measure_fp32_peak", "odin_count_blend_pairs",
+    "odin_mask_to_list", "odin_accumulate_rows",
 ]
 
 
@@ -90,6 +91,9 @@ def lib() -> C.CDLL:
         L.odin_poll.argtypes = [vp, vp]
         L.odin_set_wait_limit.argtypes = [vp, i32]
         L.odin_set_instance_sort.argtypes = [vp, i32]
+        L.odin_mask_to_list.argtypes = [vp, vp, u32, vp, u32, vp, vp, C.c_size_t, vp]
+        L.odin_accumulate_rows.argtypes = [vp, C.POINTER(odin_scene), vp, vp, vp, C.POINTER(odin_scene), vp, vp, vp, vp, vp,
+                                           C.POINTER(odin_scene), vp]
         L.odin_measure_fp32_peak.argtypes = [vp, vp, C.POINTER(C.c_float)]
         L.odin_count_blend_pairs.argtypes = [vp, C.POINTER(odin_projected), vp, vp, C.POINTER(odin_camera), vp, vp, vp]
         L.odin_workspace_bytes.argtypes = [vp, u32, u64, C.POINTER(C.c_size_t)]
@@ -208,6 +212,19 @@ def odin_count_blend_pairs(ctx, proj: odin_projected, d_vals, d_tile_ranges, cam
                            stream=None) -> None:
     _check(lib().odin_count_blend_pairs(ctx, C.byref(proj), _ptr(d_vals), _ptr(d_tile_ranges), C.byref(cam),
                                         _ptr(d_n_contrib), _ptr(d_counts), _stream(stream)), "odin_count_blend_pairs")
+
+
+def odin_mask_to_list(ctx, d_mask, n: int, d_idx, idx_capacity: int, d_count, ws, stream=None) -> None:
+    _check(lib().odin_mask_to_list(ctx, _ptr(d_mask), int(n), _ptr(d_idx), int(idx_capacity), _ptr(d_count), _ptr(ws),
+                                   0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "odin_mask_to_list")
+
+
+def odin_accumulate_rows(ctx, rows_a: odin_scene, d_zero_a, d_idx_a, d_count_a, rows_b: odin_scene, d_zero_b, d_idx_b,
+                         d_count_b, d_idx_u, d_count_u, rows_u: odin_scene, stream=None) -> None:
+    _check(lib().odin_accumulate_rows(ctx, C.byref(rows_a), _ptr(d_zero_a), _ptr(d_idx_a), _ptr(d_count_a),
+                                      C.byref(rows_b), _ptr(d_zero_b), _ptr(d_idx_b), _ptr(d_count_b), _ptr(d_idx_u),
+                                      _ptr(d_count_u), C.byref(rows_u), _stream(stream)), "odin_accumulate_rows")
 
 
 def odin_set_instance_sort(ctx, mode: int) -> None:

@@ -110,7 +110,85 @@ adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* _
   }
 }
 
+// Gradient rows of a task unit: one warp per row of the union list looks the primitive up in the two views' ascending
+// index lists (a 32-way search: three steps for a million rows) and adds the rows it finds.
+struct RowsView {
+  const float* means; const float* log_scales; const float* quats; const float* opacity_logit; const float* sh;
+  const uint8_t* zero; const uint32_t* idx; const uint32_t* count; uint32_t cap;
+};
+
+__device__ __forceinline__ int warp_find(const uint32_t* __restrict__ idx, uint32_t n, uint32_t key, unsigned lane) {
+  // position of key in the ascending idx[0..n), or -1; all lanes take part and receive the answer
+  uint32_t lo = 0, hi = n;  // the key, if present, lies in [lo, hi)
+  while (hi - lo > 32) {
+    const uint32_t step = (hi - lo + 31) / 32;
+    const uint32_t probe = lo + lane * step;
+    const bool le = probe < hi && idx[probe] <= key;                // monotone: true for the first cnt lanes
+    const uint32_t cnt = __popc(__ballot_sync(0xffffffffu, le));
+    if (cnt == 0) return -1;                                        // idx[lo] > key (uniform over the warp)
+    lo += (cnt - 1) * step;                                         // idx[lo] <= key < idx[lo + step]
+    hi = min(hi, lo + step);
+  }
+  const uint32_t i = lo + lane;
+  const uint32_t hit = __ballot_sync(0xffffffffu, i < hi && idx[i] == key);
+  return hit ? (int)(lo + __ffs(hit) - 1) : -1;
+}
+
+__global__ void __launch_bounds__(256)
+accumulate_rows_kernel(RowsView a, RowsView b, const uint32_t* __restrict__ idx_u, const uint32_t* __restrict__ count_u,
+                       uint32_t cap_u, int sh_floats, float* __restrict__ o_means, float* __restrict__ o_ls,
+                       float* __restrict__ o_q, float* __restrict__ o_op, float* __restrict__ o_sh) {
+  const unsigned lane = threadIdx.x & 31;
+  const uint32_t U = min(*count_u, cap_u);
+  const uint32_t na = min(*a.count, a.cap), nb = min(*b.count, b.cap);
+  for (uint32_t r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < U; r += gridDim.x * (blockDim.x >> 5)) {
+    const uint32_t p = idx_u[r];
+    int ra = warp_find(a.idx, na, p, lane), rb = warp_find(b.idx, nb, p, lane);
+    if (ra >= 0 && a.zero && a.zero[ra]) ra = -1;  // the view flagged the row as zero instead of writing it
+    if (rb >= 0 && b.zero && b.zero[rb]) rb = -1;
+    auto sum = [&](const float* xa, const float* xb, float* out, int width) {
+      for (int i = lane; i < width; i += 32) {
+        float s = 0.f;
+        if (ra >= 0) s += xa[(size_t)ra * width + i];
+        if (rb >= 0) s += xb[(size_t)rb * width + i];
+        out[(size_t)r * width + i] = s;
+      }
+    };
+    sum(a.means, b.means, o_means, 3);
+    sum(a.log_scales, b.log_scales, o_ls, 3);
+    sum(a.quats, b.quats, o_q, 4);
+    sum(a.opacity_logit, b.opacity_logit, o_op, 1);
+    sum(a.sh, b.sh, o_sh, sh_floats);
+  }
+}
+
 }  // namespace
+
+extern "C" int odin_accumulate_rows(odin_ctx* ctx, const odin_scene* rows_a, const uint8_t* d_zero_a, const uint32_t* d_idx_a,
+                                    const uint32_t* d_count_a, const odin_scene* rows_b, const uint8_t* d_zero_b,
+                                    const uint32_t* d_idx_b, const uint32_t* d_count_b, const uint32_t* d_idx_u,
+                                    const uint32_t* d_count_u, odin_scene* rows_u, void* stream) {
+  if (!ctx || !d_count_a || !d_count_b || !d_count_u) return ODIN_ERR_NULL;
+  int rc = odin_check_scene(rows_a);
+  if (rc == ODIN_OK) rc = odin_check_scene(rows_b);
+  if (rc == ODIN_OK) rc = odin_check_scene(rows_u);
+  if (rc != ODIN_OK) return rc;
+  if (rows_a->sh_degree != rows_u->sh_degree || rows_b->sh_degree != rows_u->sh_degree) return ODIN_ERR_INVALID_ARG;
+  if (rows_u->n == 0) return ODIN_OK;
+  if (!d_idx_u || (rows_a->n && !d_idx_a) || (rows_b->n && !d_idx_b)) return ODIN_ERR_NULL;
+  const RowsView a = {rows_a->means, rows_a->log_scales, rows_a->quats, rows_a->opacity_logit, rows_a->sh, d_zero_a, d_idx_a,
+                      d_count_a, rows_a->n};
+  const RowsView b = {rows_b->means, rows_b->log_scales, rows_b->quats, rows_b->opacity_logit, rows_b->sh, d_zero_b, d_idx_b,
+                      d_count_b, rows_b->n};
+  const int K = (rows_u->sh_degree + 1) * (rows_u->sh_degree + 1);
+  uint32_t grid = (rows_u->n + 7) / 8;
+  if (grid > (uint32_t)ctx->sm_count * 16) grid = (uint32_t)ctx->sm_count * 16;
+  OdinKernelScope ks(ctx, K_ACCUMULATE, (cudaStream_t)stream);
+  accumulate_rows_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(a, b, d_idx_u, d_count_u, rows_u->n, 3 * K, rows_u->means,
+                                                                rows_u->log_scales, rows_u->quats, rows_u->opacity_logit,
+                                                                rows_u->sh);
+  return odin_launch_status();
+}
 
 extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m, odin_scene* v,
                                 const odin_scene* grad_rows, const uint8_t* d_row_zero, const uint32_t* d_idx,

@@ -12,7 +12,7 @@ enum OdinKernelId {
   K_PROJECT = 0, K_TOUCHED, K_EMIT, K_ONESWEEP, K_FWD, K_L1, K_ZERO_ROWS,
   K_BWD_BLEND, K_BWD_PROJECT, K_ADAM_SH, K_ADAM_GEOM, K_CONFLICT, K_FWD_TAIL, K_PROJECT_SCAN,
   K_PROJECT_ROWS, K_ROW_HIST, K_ROW_SORT, K_ROW_OFFSETS, K_ACTIVE_SET, K_MASK_UNION, K_HAZARD,
-  K_GATE, K_RLG, K_TILE_BASES, K_COUNT
+  K_GATE, K_RLG, K_TILE_BASES, K_ACCUMULATE, K_COUNT
 };
 
 struct OdinProf {

@@ -15,6 +15,9 @@ constexpr int TS_ITEMS = TOUCHED_TILE / TS_THREADS;  // 8 words of 32 primitives
 // look-back without reading the counts a second time.
 constexpr int TS_MAX_ROUNDS = 8;
 
+// FROM_MASK: the input is itself a bitmask over the primitives (`tiles_touched` then points at its words): the kernel
+// only lists its members (the index list of a union of scopes, for example) and writes no mask.
+template <bool FROM_MASK>
 __global__ void __launch_bounds__(TS_THREADS)
 touched_set_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint32_t* __restrict__ mask,
                    uint32_t* __restrict__ idx, uint32_t idx_capacity, uint32_t* __restrict__ count, uint32_t* ticket,
@@ -36,15 +39,23 @@ touched_set_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint3
 #pragma unroll 8
   for (int q = 0; q < words; ++q) {
     const uint32_t p = span_base + 32u * (uint32_t)q + lane;
-    const uint32_t bal = __ballot_sync(0xffffffffu, p < n && tiles_touched[p] > 0);
+    uint32_t bal;
+    if (FROM_MASK) {
+      const uint32_t word = span_base / 32 + (uint32_t)q;
+      bal = word < n_words ? tiles_touched[word] : 0u;
+      if (word == n_words - 1 && (n & 31u)) bal &= (1u << (n & 31u)) - 1u;  // bits past n do not name primitives
+    } else {
+      bal = __ballot_sync(0xffffffffu, p < n && tiles_touched[p] > 0);
+    }
     warp_count += __popc(bal);
     if (lane == (unsigned)(q & 31)) keep[q >> 5] = bal;
   }
   // the mask words of the span: 32 consecutive words per store
-  for (int h = 0; h * 32 < words; ++h) {
-    const uint32_t word = span_base / 32 + h * 32 + lane;
-    if ((int)(h * 32 + lane) < words && word < n_words) mask[word] = keep[h];
-  }
+  if (!FROM_MASK)
+    for (int h = 0; h * 32 < words; ++h) {
+      const uint32_t word = span_base / 32 + h * 32 + lane;
+      if ((int)(h * 32 + lane) < words && word < n_words) mask[word] = keep[h];
+    }
   uint32_t chunk_total;
   const uint32_t scan = odin_block_exclusive_sum(lane == 0 ? warp_count : 0u, s_warp, &chunk_total);
   const uint32_t warp_off = __shfl_sync(0xffffffffu, scan, 0);
@@ -130,8 +141,31 @@ extern "C" int odin_touched_set(odin_ctx* ctx, const uint32_t* d_tiles_touched, 
   const uint32_t scan_chunk = TOUCHED_TILE * (uint32_t)scan_rounds;
   const uint32_t grid = (n + scan_chunk - 1) / scan_chunk;
   OdinKernelScope ks(ctx, K_TOUCHED, st);
-  touched_set_kernel<<<grid, TS_THREADS, 0, st>>>(d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket, state,
-                                                  ctx->d_status, scan_rounds, ctx->spin_limit);
+  touched_set_kernel<false><<<grid, TS_THREADS, 0, st>>>(d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket,
+                                                         state, ctx->d_status, scan_rounds, ctx->spin_limit);
+  return odin_launch_status();
+}
+
+extern "C" int odin_mask_to_list(odin_ctx* ctx, const uint32_t* d_mask, uint32_t n, uint32_t* d_idx, uint32_t idx_capacity,
+                                 uint32_t* d_count, void* ws, size_t ws_bytes, void* stream) {
+  if (!ctx || !d_count) return ODIN_ERR_NULL;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (n >= (1u << 28)) return ODIN_ERR_INVALID_ARG;
+  if (n == 0) {
+    ODIN_CUDA(cudaMemsetAsync(d_count, 0, 4, st));
+    return ODIN_OK;
+  }
+  if (!d_mask || (idx_capacity > 0 && !d_idx)) return ODIN_ERR_NULL;
+  const size_t need = touched_ws_bytes(n);
+  if (!ws || !odin_aligned(ws, 256) || ws_bytes < need) return ODIN_ERR_WORKSPACE;
+  ODIN_CUDA(cudaMemsetAsync(ws, 0, need, st));
+  uint32_t* ticket = reinterpret_cast<uint32_t*>(ws);
+  uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + 256);
+  const int scan_rounds = scan_rounds_for(n, ctx->sm_count);
+  const uint32_t scan_chunk = TOUCHED_TILE * (uint32_t)scan_rounds;
+  OdinKernelScope ks(ctx, K_TOUCHED, st);
+  touched_set_kernel<true><<<(n + scan_chunk - 1) / scan_chunk, TS_THREADS, 0, st>>>(
+      d_mask, n, nullptr, d_idx, idx_capacity, d_count, ticket, state, ctx->d_status, scan_rounds, ctx->spin_limit);
   return odin_launch_status();
 }
 
@@ -184,7 +218,7 @@ extern "C" int odin_touched_set_static(const uint32_t* d_tiles_touched, uint32_t
   // count only changes how many blocks share the work, never the result)
   const int scan_rounds = scan_rounds_for(n, 148);
   const uint32_t scan_chunk = TOUCHED_TILE * (uint32_t)scan_rounds;
-  touched_set_kernel<<<(n + scan_chunk - 1) / scan_chunk, TS_THREADS, 0, st>>>(
+  touched_set_kernel<false><<<(n + scan_chunk - 1) / scan_chunk, TS_THREADS, 0, st>>>(
       d_tiles_touched, n, d_mask, d_idx, idx_capacity, d_count, ticket, state, status, scan_rounds,
       ODIN_DEFAULT_SPIN_LIMIT);
   return odin_launch_status();

@@ -243,6 +243,55 @@ class ViewTrainer:
         if n_pairs:
             self.conflict_count(d_pairs, n_pairs, d_counts, stream)
 
+    # -------------------------------------------------------------------------------------------- task unit of two views
+    def prepare_unit(self):
+        """Second set of per-view outputs and the union buffers of unit_step (allocated once)."""
+        u = getattr(self, "_unit", None)
+        if u is None:
+            dev, cap = self.device, max(self.row_capacity, 1)
+            z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=dev)  # noqa: E731
+            union_cap = min(self.n, 2 * self.row_capacity)
+            u = {
+                "grads_b": DeviceScene(self.row_capacity, self.sh_degree, dev), "idx_b": z(cap, torch.int32),
+                "count_b": z(1, torch.int32), "row_zero_b": z(cap, torch.uint8),
+                "mask": z(max(self.mask_stride, 4), torch.int32), "members": z(2, torch.int32),
+                "union_cap": union_cap, "idx_u": z(max(union_cap, 1), torch.int32), "count_u": z(1, torch.int32),
+                "grads_u": DeviceScene(union_cap, self.sh_degree, dev), "loss": z(2, torch.float32),
+            }
+            self._unit = u
+        return u
+
+    def unit_step(self, cams, targets, step: int, lr, beta1: float, beta2: float, eps: float, slots=(0, 1),
+                  stream=None) -> None:
+        """One task unit of two views (Sec. 2.1 unit scopes; Sec. 6.1): both views are projected, rendered and
+        differentiated with the same parameters, their gradient rows are added up over the union of their touched sets
+        and one sparse Adam update is applied to the union.  Afterwards the unit's losses are in self._unit["loss"],
+        the union list / count in self._unit["idx_u"] / ["count_u"], the views' masks in self.masks[slots].
+        Marshalling only: every kernel is the library's."""
+        u = self.prepare_unit()
+        if self.mask_slots < 2:
+            raise RuntimeError("unit_step needs two mask slots")
+        first = (self.grads, self.idx, self.count, self.row_zero, self.loss, self.target)
+        per_view = [(self.grads, self.idx, self.count, self.row_zero), (u["grads_b"], u["idx_b"], u["count_b"], u["row_zero_b"])]
+        zero_flags = []
+        try:
+            for k in range(2):
+                self.grads, self.idx, self.count, self.row_zero = per_view[k]
+                self.loss, self.target = u["loss"][k:k + 1], targets[k]
+                self.view_step(cams[k], step, lr, beta1, beta2, eps, slot=slots[k], update=False, stream=stream)
+                zero_flags.append(self._row_zero_in_use)
+        finally:
+            self.grads, self.idx, self.count, self.row_zero, self.loss, self.target = first
+        u["members"].copy_(torch.tensor(list(slots), dtype=torch.int32), non_blocking=True)
+        B.odin_mask_union(self.ctx, self.masks, self.mask_slots, self.masks.shape[1], self.n, u["members"], 2, u["mask"],
+                          stream)
+        B.odin_mask_to_list(self.ctx, u["mask"], self.n, u["idx_u"], u["union_cap"], u["count_u"], self.ws, stream)
+        (ga, ia, ca, _), (gb, ib, cb, _) = per_view
+        B.odin_accumulate_rows(self.ctx, ga.struct, zero_flags[0], ia, ca, gb.struct, zero_flags[1], ib, cb, u["idx_u"],
+                               u["count_u"], u["grads_u"].struct, stream)
+        B.odin_sparse_adam(self.ctx, self.params.struct, self.m.struct, self.v.struct, u["grads_u"].struct, None,
+                           u["idx_u"], u["count_u"], lr, beta1, beta2, eps, step, stream)
+
     def prepare_host_io(self, n_counts: int = 0):
         """Staging buffers, pinned result slots, copy stream and events of train_from_host (allocated once)."""
         io = getattr(self, "_host_io", None)

@@ -4,7 +4,9 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import oracle as oracle_mod
 from paper_2607_19893_b200 import binding as B
+from paper_2607_19893_b200 import engine as E
 from paper_2607_19893_b200 import workloads as wl
 
 import gpu_util as G
@@ -332,3 +334,111 @@ def test_delayed_read_gate_random_scopes(oracle32, n):
     gate = run_gate(ctx, dev, n, w_b, w_b, w_a, active_a, ev_a, 0.2)
     assert gate[0] == 0 and gate[1] == 0
     B.odin_destroy(ctx)
+
+
+# ------------------------------------------------------------------------------------------------ task unit of two views
+def test_mask_to_list_and_accumulate_rows(oracle32):
+    """The unit calls on their own: the list of a union mask against NumPy, the accumulated rows against the oracle's
+    accumulate_rows (exact: one or two float additions per word), ragged sizes, a view with flagged zero rows."""
+    rng = np.random.default_rng(17)
+    dev = torch.device("cuda", 0)
+    ctx = B.odin_create(0)
+    for n, da, db in ((70_001, 0.3, 0.2), (33, 0.5, 0.5), (3_000_000, 0.02, 0.05)):
+        ia = np.flatnonzero(rng.random(n) < da).astype(np.uint32)
+        ib = np.flatnonzero(rng.random(n) < db).astype(np.uint32)
+        deg = 1
+        f = 11 + 12
+        ra, rb = rng.standard_normal((len(ia), f)).astype(np.float32), rng.standard_normal((len(ib), f)).astype(np.float32)
+        za = (rng.random(len(ia)) < 0.3).astype(np.uint8)  # rows of view a that were flagged zero (their content is stale)
+        ra_eff = ra.copy()
+        ra_eff[za.astype(bool)] = 0
+        union_o, rows_o = oracle32.accumulate_rows(ia, ra_eff, ib, rb)
+        masks = torch.from_numpy(np.stack([oracle_mod.ids_to_mask(ia, n), oracle_mod.ids_to_mask(ib, n)]).view(np.int32)).to(dev)
+        words = masks.shape[1]
+        stride = (words + 3) // 4 * 4
+        mpad = torch.zeros((2, stride), dtype=torch.int32, device=dev)
+        mpad[:, :words] = masks
+        umask = torch.zeros(stride, dtype=torch.int32, device=dev)
+        members = torch.tensor([0, 1], dtype=torch.int32, device=dev)
+        B.odin_mask_union(ctx, mpad, 2, stride, n, members, 2, umask)
+        ws = torch.zeros(B.odin_workspace_bytes(ctx, n, 0), dtype=torch.uint8, device=dev)
+        cap = len(union_o) + 3
+        d_idx = torch.full((cap,), -1, dtype=torch.int32, device=dev)
+        d_cnt = torch.zeros(1, dtype=torch.int32, device=dev)
+        B.odin_mask_to_list(ctx, umask, n, d_idx, cap, d_cnt, ws)
+        assert B.odin_poll(ctx) == B.ODIN_OK
+        assert int(d_cnt.item()) == len(union_o)
+        assert np.array_equal(d_idx.cpu().numpy().view(np.uint32)[: len(union_o)], union_o)
+
+        def scene_of(rows, cap_rows):
+            sc = E.DeviceScene(cap_rows, deg, dev)
+            r = torch.from_numpy(rows).to(dev)
+            k = len(rows)
+            sc.means[:k] = r[:, 0:3]; sc.log_scales[:k] = r[:, 3:6]; sc.quats[:k] = r[:, 6:10]
+            sc.opacity_logit[:k] = r[:, 10]; sc.sh[:k] = r[:, 11:].reshape(k, 4, 3)
+            return sc
+
+        sa, sb, su = scene_of(ra, len(ia) + 2), scene_of(rb, len(ib) + 1), E.DeviceScene(cap, deg, dev)
+        t = lambda a, dt: torch.from_numpy(a.view(dt) if a.dtype != np.uint8 else a).to(dev)  # noqa: E731
+        B.odin_accumulate_rows(ctx, sa.struct, t(za, np.uint8), t(ia, np.int32),
+                               torch.tensor([len(ia)], dtype=torch.int32, device=dev), sb.struct, None, t(ib, np.int32),
+                               torch.tensor([len(ib)], dtype=torch.int32, device=dev), d_idx, d_cnt, su.struct)
+        assert B.odin_poll(ctx) == B.ODIN_OK
+        assert np.array_equal(su.rows_as_matrix(len(union_o)), rows_o.astype(np.float32))
+    B.odin_destroy(ctx)
+
+
+def test_two_view_unit_step(oracle32):
+    """Two views of preset 2 as one task unit against the oracle's unit_step: union list exact, accumulated rows inside
+    the sum of the two views' gradient bars, Adam on every word of the union against the oracle's update of the
+    device's own accumulated rows, untouched rows bitwise."""
+    import gpu_util as G
+
+    w = wl.make_workload(2, n=40_000)
+    cams = [w.cameras[1], w.cameras[2]]
+    tgts = [w.target(1), w.target(2)]
+    tr = G.trainer_for(w.scene, cams[0], mask_slots=2)
+    dev = tr.device
+    p = w.scene.copy()
+    m, v = p.zeros_like(), p.zeros_like()
+    for step in (1, 2):  # the second unit runs on non-zero moments
+        pre = [x.copy() for x in (p, m, v)]
+        o = oracle32.unit_step(p, m, v, cams, tgts, w.lr, w.beta1, w.beta2, w.eps, step)
+        tr.unit_step([B.make_camera(c) for c in cams], [torch.from_numpy(t).to(dev) for t in tgts], step, w.lr, w.beta1,
+                     w.beta2, w.eps)
+        G.poll_ok(tr)
+        u = tr._unit
+        nu = int(u["count_u"].item())
+        idx_u = G.u32(u["idx_u"])[:nu]
+        assert np.array_equal(idx_u, o["idx"])  # (no projection decision of these views sits on a threshold)
+        rows_dev = u["grads_u"].rows_as_matrix(nu).astype(np.float64)
+        # bar of a sum of two views = sum of the two bars
+        bound = np.zeros_like(rows_dev)
+        for view, cam in zip(o["views"], cams):
+            _, g2d_abs = oracle32.render_bwd_blend(view["proj"], view["vals"], view["ranges"], cam, view["final_T"],
+                                                   view["n_contrib"], view["dL_dout"], want_abs=True)
+            b = G.rows_bound(oracle32, pre[0], cam, view["idx"], view["proj"].clamp_flags, view["rows"].astype(np.float64),
+                             view["g2d"], g2d_abs)
+            bound[np.searchsorted(idx_u, view["idx"])] += b
+        err = np.abs(rows_dev - o["rows"])
+        assert (err <= 8 * bound + 1e-30).mean() > 0.9995  # rows on fragile pixels are not singled out here
+        # Adam on every word: the oracle's update applied to the device's accumulated rows
+        names = ("means", "log_scales", "quats", "opacity_logit", "sh")
+        q = [wl.Scene(p.sh_degree, *(np.ascontiguousarray(getattr(st, nm)[idx_u]) for nm in names)) for st in pre]
+        oracle32.sparse_adam(q[0], q[1], q[2], rows_dev.astype(np.float32), np.arange(nu, dtype=np.uint32), w.lr, w.beta1,
+                             w.beta2, w.eps, step)
+        it = torch.from_numpy(idx_u.astype(np.int64)).to(dev)
+        for st_dev, st_q, kind in ((tr.params, q[0], "p"), (tr.m, q[1], "m"), (tr.v, q[2], "v")):
+            for t, nm in zip(st_dev.tensors(), names):
+                got, want = t[it].cpu().numpy().astype(np.float64), getattr(st_q, nm).astype(np.float64)
+                tol = 2e-5 * np.abs(want) + (2e-5 * float(w.lr.max()) if kind == "p" else 1e-30)
+                if kind == "m":
+                    tol = tol + 2e-5 * 1e-3  # first moments may be cancelled sums of terms up to ~1e-3
+                assert np.all(np.abs(got - want) <= tol), (kind, nm)
+        rest = np.setdiff1d(np.arange(p.n), idx_u)
+        for t, h in zip(tr.params.tensors(), (p.means, p.log_scales, p.quats, p.opacity_logit, p.sh)):
+            assert np.array_equal(t.cpu().numpy()[rest].view(np.uint32), h[rest].view(np.uint32))
+        for st_dev, st_h in ((tr.params, p), (tr.m, m), (tr.v, v)):  # re-synchronise the oracle from the device
+            for t, nm in zip(st_dev.tensors(), names):
+                getattr(st_h, nm)[...] = t.cpu().numpy()
+    tr.close()
