@@ -114,6 +114,11 @@ typedef struct {
   uint8_t* clamp_flags;     /* [capacity] bit c set when colour channel c was clamped at 0 */
   uint32_t* num_rows;       /* [1] V: number of rows written (device) */
   uint64_t* num_instances;  /* [1] M: sum of tiles_touched (device) */
+  uint32_t* touched_mask;   /* [ceil(n/32)] optional (NULL: not wanted).  odin_project then also writes the view's touched
+                               bitmask (bit p & 31 of word p >> 5), exactly what odin_touched_set derives from
+                               tiles_touched; with prim_id (the ascending list) and num_rows (its length) the whole
+                               touched set of Sec. 2.1 is then an output of the projection's own scan and the separate
+                               call (one more pass over tiles_touched) can be left out. */
 } odin_projected;
 
 /* ---- context ------------------------------------------------------------------------------------------------- */

@@ -67,7 +67,7 @@ class odin_projected(C.Structure):
     _fields_ = [("capacity", C.c_uint32), ("tiles_touched", C.c_void_p), ("prim_id", C.c_void_p), ("xy", C.c_void_p),
                 ("depth", C.c_void_p), ("conic_opacity", C.c_void_p), ("rgb", C.c_void_p), ("radius", C.c_void_p),
                 ("rect", C.c_void_p), ("tile_offset", C.c_void_p), ("clamp_flags", C.c_void_p),
-                ("num_rows", C.c_void_p), ("num_instances", C.c_void_p)]
+                ("num_rows", C.c_void_p), ("num_instances", C.c_void_p), ("touched_mask", C.c_void_p)]
 
 
 _lib = None

@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(SCAN_THREADS)
 project_scan_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint32_t capacity,
                     uint32_t* __restrict__ prim_id, uint32_t* __restrict__ tile_offset, uint32_t* __restrict__ num_rows,
                     uint64_t* __restrict__ num_instances, uint32_t* ticket, uint64_t* state, int* status,
-                    int scan_rounds, int spin_limit) {
+                    int scan_rounds, int spin_limit, uint32_t* __restrict__ touched_mask) {
   const uint32_t scan_chunk = PROJECT_TILE * (uint32_t)scan_rounds;
   __shared__ uint32_t s_tile;
   __shared__ uint64_t s_warp[SCAN_THREADS / 32 + 1];
@@ -228,7 +228,10 @@ project_scan_kernel(const uint32_t* __restrict__ tiles_touched, uint32_t n, uint
 #pragma unroll
     for (int j = 0; j < SCAN_ITEMS; ++j) {
       ex[j] = run;
-      if (__ballot_sync(0xffffffffu, t[j] != 0) == 0) continue;  // 32 culled primitives in a row: nothing to scan
+      const uint32_t visible = __ballot_sync(0xffffffffu, t[j] != 0);
+      // the 32 primitives of this load are one word of the touched bitmask
+      if (touched_mask && lane == 0 && warp_base + 32 * j < n) touched_mask[(warp_base + 32 * j) >> 5] = visible;
+      if (visible == 0) continue;  // 32 culled primitives in a row: nothing to scan
       const uint64_t v = t[j] ? ((1ull << PACK_SHIFT) | (uint64_t)t[j]) : 0ull;
       uint64_t inc = v;
 #pragma unroll
@@ -364,7 +367,7 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
     const uint32_t scan_chunk = PROJECT_TILE * (uint32_t)scan_rounds;
     project_scan_kernel<<<(n + scan_chunk - 1) / scan_chunk, SCAN_THREADS, 0, st>>>(
         out->tiles_touched, n, out->capacity, out->prim_id, out->tile_offset, out->num_rows, out->num_instances, ticket,
-        state, ctx->d_status, scan_rounds, ctx->spin_limit);
+        state, ctx->d_status, scan_rounds, ctx->spin_limit, out->touched_mask);
   }
   if (out->capacity == 0) return odin_launch_status();
   const uint32_t blocks_cap = (out->capacity + 127) / 128;

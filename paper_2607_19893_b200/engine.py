@@ -68,7 +68,7 @@ class ProjectedBuffers:
         self.struct = B.odin_projected(
             self.capacity, *(t.data_ptr() for t in (self.tiles_touched, self.prim_id, self.xy, self.depth,
                                                     self.conic_opacity, self.rgb, self.radius, self.rect, self.tile_offset,
-                                                    self.clamp_flags, self.num_rows, self.num_instances)))
+                                                    self.clamp_flags, self.num_rows, self.num_instances)), None)
 
     def load_rows(self, **arrays) -> None:
         """Overwrite compact arrays from host data (used by stage-isolated tests)."""
@@ -144,6 +144,11 @@ class ViewTrainer:
         self.keep_sorted_keys = False  # view_step: also write the sorted 64-bit keys (only tests look at them)
         self.track_active = False      # render_bwd: also flag the rows that contributed (needed by active_set)
         self.skip_zero_rows = True     # render_bwd flags zero gradient rows instead of writing them; Adam takes the flags
+        # the touched set as a by-product of the projection's scan (mask written by odin_project, list = its row map):
+        # view_step then leaves the separate odin_touched_set call out.  self.idx / self.count name the buffers that
+        # hold the list and its length of the last view either way.
+        self.fused_touched = True
+        self._own_idx, self._own_count = self.idx, self.count
         self.row_zero = z(max(self.row_capacity, 1), torch.uint8)
         self._row_zero_in_use = None   # the flags the last render_bwd wrote (None: every row was written)
 
@@ -229,11 +234,21 @@ class ViewTrainer:
 
     # -------------------------------------------------------------------------------------------- whole view
     def view_step(self, cam: B.odin_camera, step: int, lr, beta1: float, beta2: float, eps: float, slot: int = 0,
-                  d_pairs=None, n_pairs: int = 0, d_counts=None, update: bool = True, stream=None) -> None:
+                  d_pairs=None, n_pairs: int = 0, d_counts=None, update: bool = True, stream=None,
+                  fused_touched: Optional[bool] = None) -> None:
         """project -> touched set -> bin/sort -> composite -> L1 loss -> backward -> sparse Adam -> conflict counts.
         The target image must already be in self.target.  Nothing here synchronises the host."""
-        self.project(cam, stream)
-        self.touched_set(slot, stream)
+        fused = self.fused_touched if fused_touched is None else fused_touched
+        if fused:
+            self.proj.struct.touched_mask = self.masks[slot].data_ptr()
+            self.project(cam, stream)
+            self.idx, self.count = self.proj.prim_id, self.proj.num_rows
+        else:
+            self.proj.struct.touched_mask = None
+            if self.idx is self.proj.prim_id:
+                self.idx, self.count = self._own_idx, self._own_count
+            self.project(cam, stream)
+            self.touched_set(slot, stream)
         self.bin_sort(stream, want_keys=self.keep_sorted_keys)
         self.render_fwd(cam, stream)
         self.l1_loss(stream)
@@ -272,13 +287,16 @@ class ViewTrainer:
         if self.mask_slots < 2:
             raise RuntimeError("unit_step needs two mask slots")
         first = (self.grads, self.idx, self.count, self.row_zero, self.loss, self.target)
-        per_view = [(self.grads, self.idx, self.count, self.row_zero), (u["grads_b"], u["idx_b"], u["count_b"], u["row_zero_b"])]
+        per_view = [(self.grads, self._own_idx, self._own_count, self.row_zero),
+                    (u["grads_b"], u["idx_b"], u["count_b"], u["row_zero_b"])]
         zero_flags = []
         try:
             for k in range(2):
                 self.grads, self.idx, self.count, self.row_zero = per_view[k]
                 self.loss, self.target = u["loss"][k:k + 1], targets[k]
-                self.view_step(cams[k], step, lr, beta1, beta2, eps, slot=slots[k], update=False, stream=stream)
+                # (the two views need index lists of their own: the separate touched-set call writes them)
+                self.view_step(cams[k], step, lr, beta1, beta2, eps, slot=slots[k], update=False, stream=stream,
+                               fused_touched=False)
                 zero_flags.append(self._row_zero_in_use)
         finally:
             self.grads, self.idx, self.count, self.row_zero, self.loss, self.target = first
@@ -364,6 +382,9 @@ class ViewTrainer:
             pairs = pairs_of(s) if pairs_of is not None else None
             self.view_step(cam_of(s), s + 1, lr, beta1, beta2, eps, slot=slot_of(s), d_pairs=pairs[0] if pairs else None,
                            n_pairs=pairs[1] if pairs else 0, d_counts=step_counts, stream=stream)
+            if self.count is not io["d_count"][k]:  # the count lives in the projection's buffers: keep this step's copy
+                io["d_count"][k].copy_(self.count, non_blocking=True)
+                self.count = io["d_count"][k]
             consumed[k].record(stream)
             with torch.cuda.stream(read_stream):
                 read_stream.wait_event(consumed[k])
