@@ -5,7 +5,12 @@
 
 namespace {
 
+// A row whose gradient and both moments are zero is left alone: m' = v' = 0 and theta' = theta - step * 0 / (0 + eps) =
+// theta bit for bit (eps > 0), so neither the parameter is read nor anything written.  Most touched rows of a view are
+// occluded (zero gradient), and until a primitive has been active in some view its moments are zero too: for those
+// rows the update costs the two moment reads only.  (skip_idle is off when eps == 0, where 0 / 0 would be the result.)
 struct AdamK {
+  int skip_idle;
   float beta1, beta2, omb1, omb2, eps;
   float step_size[6];  // lr_g / (1 - beta1^t)
   float inv_bc2s;      // 1 / sqrt(1 - beta2^t)
@@ -45,8 +50,11 @@ adam_sh_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__
     const bool zero = row_zero && row_zero[r];  // the gradient row was not written: it is zero
     if (VEC == 4) {
       const float4 gg = zero ? make_float4(0.f, 0.f, 0.f, 0.f) : reinterpret_cast<const float4*>(g)[e];
-      float4 pp = *reinterpret_cast<float4*>(p + dst), mm = *reinterpret_cast<float4*>(m + dst),
-             vv = *reinterpret_cast<float4*>(v + dst);
+      float4 mm = *reinterpret_cast<float4*>(m + dst), vv = *reinterpret_cast<float4*>(v + dst);
+      if (k.skip_idle && gg.x == 0.f && gg.y == 0.f && gg.z == 0.f && gg.w == 0.f && mm.x == 0.f && mm.y == 0.f &&
+          mm.z == 0.f && mm.w == 0.f && vv.x == 0.f && vv.y == 0.f && vv.z == 0.f && vv.w == 0.f)
+        continue;
+      float4 pp = *reinterpret_cast<float4*>(p + dst);
       // floats 0..2 of a row are the degree-0 coefficients (group 4); the rest group 5
       const int f0 = j * 4;
       adam_one(pp.x, mm.x, vv.x, gg.x, k.step_size[f0 + 0 < 3 ? 4 : 5], k);
@@ -57,8 +65,11 @@ adam_sh_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__
       *reinterpret_cast<float4*>(m + dst) = mm;
       *reinterpret_cast<float4*>(v + dst) = vv;
     } else {
-      float pp = p[dst], mm = m[dst], vv = v[dst];
-      adam_one(pp, mm, vv, zero ? 0.f : g[e], k.step_size[j < 3 ? 4 : 5], k);
+      float mm = m[dst], vv = v[dst];
+      const float gg = zero ? 0.f : g[e];
+      if (k.skip_idle && gg == 0.f && mm == 0.f && vv == 0.f) continue;
+      float pp = p[dst];
+      adam_one(pp, mm, vv, gg, k.step_size[j < 3 ? 4 : 5], k);
       p[dst] = pp; m[dst] = mm; v[dst] = vv;
     }
   }
@@ -89,22 +100,34 @@ adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* _
       const float ss = k.step_size[part];
       float pp[3], mm[3], vv[3], gg[3];
 #pragma unroll
-      for (int i = 0; i < 3; ++i) { pp[i] = p[i]; mm[i] = m[i]; vv[i] = v[i]; gg[i] = zero ? 0.f : g[i]; }
+      for (int i = 0; i < 3; ++i) { mm[i] = m[i]; vv[i] = v[i]; gg[i] = zero ? 0.f : g[i]; }
+      if (k.skip_idle && gg[0] == 0.f && gg[1] == 0.f && gg[2] == 0.f && mm[0] == 0.f && mm[1] == 0.f && mm[2] == 0.f &&
+          vv[0] == 0.f && vv[1] == 0.f && vv[2] == 0.f)
+        continue;
+#pragma unroll
+      for (int i = 0; i < 3; ++i) pp[i] = p[i];
 #pragma unroll
       for (int i = 0; i < 3; ++i) adam_one(pp[i], mm[i], vv[i], gg[i], ss, k);
 #pragma unroll
       for (int i = 0; i < 3; ++i) { p[i] = pp[i]; m[i] = mm[i]; v[i] = vv[i]; }
     } else if (part == 2) {
-      float4 pp = p_q[d], mm = m_q[d], vv = v_q[d];
+      float4 mm = m_q[d], vv = v_q[d];
       const float4 gg = zero ? make_float4(0.f, 0.f, 0.f, 0.f) : g_q[r];
+      if (k.skip_idle && gg.x == 0.f && gg.y == 0.f && gg.z == 0.f && gg.w == 0.f && mm.x == 0.f && mm.y == 0.f &&
+          mm.z == 0.f && mm.w == 0.f && vv.x == 0.f && vv.y == 0.f && vv.z == 0.f && vv.w == 0.f)
+        continue;
+      float4 pp = p_q[d];
       adam_one(pp.x, mm.x, vv.x, gg.x, k.step_size[2], k);
       adam_one(pp.y, mm.y, vv.y, gg.y, k.step_size[2], k);
       adam_one(pp.z, mm.z, vv.z, gg.z, k.step_size[2], k);
       adam_one(pp.w, mm.w, vv.w, gg.w, k.step_size[2], k);
       p_q[d] = pp; m_q[d] = mm; v_q[d] = vv;
     } else {
-      float pp = p_o[d], mm = m_o[d], vv = v_o[d];
-      adam_one(pp, mm, vv, zero ? 0.f : g_o[r], k.step_size[3], k);
+      float mm = m_o[d], vv = v_o[d];
+      const float gg = zero ? 0.f : g_o[r];
+      if (k.skip_idle && gg == 0.f && mm == 0.f && vv == 0.f) continue;
+      float pp = p_o[d];
+      adam_one(pp, mm, vv, gg, k.step_size[3], k);
       p_o[d] = pp; m_o[d] = mm; v_o[d] = vv;
     }
   }
@@ -209,6 +232,7 @@ extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m
   if (!d_idx) return ODIN_ERR_NULL;
   AdamK k;
   k.beta1 = beta1; k.beta2 = beta2; k.omb1 = 1.f - beta1; k.omb2 = 1.f - beta2; k.eps = eps;
+  k.skip_idle = eps > 0.f ? 1 : 0;
   const float bc1 = 1.f - (float)pow((double)beta1, (double)step);
   const float bc2s = (float)sqrt(1.0 - pow((double)beta2, (double)step));
   for (int i = 0; i < 6; ++i) k.step_size[i] = lr[i] / bc1;
