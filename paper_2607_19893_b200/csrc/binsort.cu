@@ -814,8 +814,9 @@ constexpr int SC_ITEMS = OFFSET_TILE / SC_THREADS;
 constexpr int SC_SUB = 256;
 constexpr int SC_WORDS = SC_SUB / 32;
 constexpr uint32_t SC_BAND_TILES = SCATTER_MAX_TX;  // tiles of a band: band_rows * TX <= this
-constexpr size_t SC_SMEM =
-    (size_t)OFFSET_TILE * (8 + 4 + 4 + 2) + (size_t)SC_WORDS * SC_BAND_TILES * 4 + SC_BAND_TILES * 4;
+// (the rows kept for a band are staged SC_SUB at a time, straight from the registers that hold the chunk's rectangles:
+// 32 KB of shared memory per block instead of 64, seven resident blocks instead of three)
+constexpr size_t SC_SMEM = (size_t)SC_SUB * (8 + 4 + 4 + 4) + (size_t)SC_WORDS * SC_BAND_TILES * 4 + SC_BAND_TILES * 4;
 
 // EXACT (binning 2): the tiles of a row inside a tile row are the kept span (tilespan.cuh), recomputed from the row's
 // centre, conic and threshold as chunk_counts_kernel left them in depth order.
@@ -829,12 +830,12 @@ scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const float4* 
                          uint32_t* __restrict__ vals, uint64_t* __restrict__ keys64,
                          const uint32_t* __restrict__ depth_bits) {
   extern __shared__ __align__(16) unsigned char sc_smem[];
-  ushort4* s_prect = reinterpret_cast<ushort4*>(sc_smem);                    // [OFFSET_TILE] rectangles of the rows kept
-  uint32_t* s_prow = reinterpret_cast<uint32_t*>(s_prect + OFFSET_TILE);     // [OFFSET_TILE] their row ids
-  uint32_t* s_plim = s_prow + OFFSET_TILE;                                   // [OFFSET_TILE] instances they may emit
-  uint32_t* s_bits = s_plim + OFFSET_TILE;                                   // [SC_WORDS][band tiles]
+  ushort4* s_prect = reinterpret_cast<ushort4*>(sc_smem);                    // [SC_SUB] rectangles of the rows of the batch
+  uint32_t* s_prow = reinterpret_cast<uint32_t*>(s_prect + SC_SUB);          // [SC_SUB] their row ids
+  uint32_t* s_plim = s_prow + SC_SUB;                                        // [SC_SUB] instances they may emit
+  uint32_t* s_pidx = s_plim + SC_SUB;                                        // [SC_SUB] place of the row in its chunk
+  uint32_t* s_bits = s_pidx + SC_SUB;                                        // [SC_WORDS][band tiles]
   uint32_t* s_pos = s_bits + SC_WORDS * SC_BAND_TILES;                       // [band tiles] next position of the tile
-  uint16_t* s_pidx = reinterpret_cast<uint16_t*>(s_pos + SC_BAND_TILES);     // [OFFSET_TILE] place of the row in its chunk
   __shared__ uint32_t s_warp[33];
   const uint32_t V = *num_rows;
   const uint32_t nchunks = (V + OFFSET_TILE - 1) / OFFSET_TILE;
@@ -857,23 +858,8 @@ scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const float4* 
       }
     }
     uint32_t npass;
-    uint32_t p = odin_block_exclusive_sum((uint32_t)__popc(keep), s_warp, &npass);  // (its barriers also fence the reuse
-    if (npass == 0) continue;                                                      //  of the arrays below; uniform)
-#pragma unroll
-    for (int k = 0; k < SC_ITEMS; ++k) {
-      if (keep >> k & 1u) {
-        s_prect[p] = rc[k];
-        s_prow[p] = min(sorted_row[first + k], V - 1);
-        uint32_t lim = 0xffffffffu;
-        if (cut) {
-          const uint32_t off = sorted_off[first + k];
-          lim = off < capacity ? capacity - off : 0u;
-        }
-        s_plim[p] = lim;
-        if (EXACT) s_pidx[p] = (uint16_t)(threadIdx.x * SC_ITEMS + k);
-        ++p;
-      }
-    }
+    const uint32_t p0 = odin_block_exclusive_sum((uint32_t)__popc(keep), s_warp, &npass);  // (its barriers also fence
+    if (npass == 0) continue;                                                             //  the reuse of s_pos; uniform)
     for (uint32_t t = threadIdx.x; t < band_tiles; t += SC_THREADS) {
       const uint32_t tile = by0 * (uint32_t)TX + t;
       s_pos[t] = ranges[tile].x + counts[(size_t)chunk * tiles_pad + tile];
@@ -881,6 +867,28 @@ scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const float4* 
     __syncthreads();
     for (uint32_t sub = 0; sub < npass; sub += SC_SUB) {
       for (uint32_t i = threadIdx.x; i < SC_WORDS * band_tiles; i += SC_THREADS) s_bits[i] = 0;
+      {
+        // stage the rows of this batch: kept row number p0 + (kept rows of the thread in front of it)
+        uint32_t p = p0;
+#pragma unroll
+        for (int k = 0; k < SC_ITEMS; ++k) {
+          if (keep >> k & 1u) {
+            if (p >= sub && p < sub + SC_SUB) {
+              const uint32_t q = p - sub;
+              s_prect[q] = rc[k];
+              s_prow[q] = min(sorted_row[first + k], V - 1);
+              uint32_t lim = 0xffffffffu;
+              if (cut) {
+                const uint32_t off = sorted_off[first + k];
+                lim = off < capacity ? capacity - off : 0u;
+              }
+              s_plim[q] = lim;
+              s_pidx[q] = threadIdx.x * SC_ITEMS + k;
+            }
+            ++p;
+          }
+        }
+      }
       __syncthreads();
       {
         // Tile row by tile row of the band: the tiles of a row of the list inside one tile row are a run [xa, xa + len).
@@ -894,11 +902,11 @@ scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const float4* 
         SpanConic e;
         e.k = -1.f;
         if (j < npass) {
-          const ushort4 r = s_prect[j];
-          rx = r.x; ry = r.y; ry1 = r.w; w = (uint32_t)r.z - (uint32_t)r.x; lim = s_plim[j];
+          const ushort4 r = s_prect[threadIdx.x];
+          rx = r.x; ry = r.y; ry1 = r.w; w = (uint32_t)r.z - (uint32_t)r.x; lim = s_plim[threadIdx.x];
           x1 = min((uint32_t)r.z, (uint32_t)TX);
           if (EXACT) {
-            const uint32_t gi = chunk * OFFSET_TILE + s_pidx[j];
+            const uint32_t gi = chunk * OFFSET_TILE + s_pidx[threadIdx.x];
             const float4 g4 = sorted_geo4[gi];
             const float2 g2 = sorted_geo2[gi];
             e.u = g4.x; e.v = g4.y; e.A = g4.z; e.B = g4.w; e.C = g2.x; e.k = g2.y;
@@ -950,7 +958,7 @@ scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const float4* 
           while (bits) {
             const int b = __ffs(bits) - 1;
             bits &= bits - 1;
-            const uint32_t row = s_prow[sub + wd * 32 + b];
+            const uint32_t row = s_prow[wd * 32 + b];
             if (pos < capacity) {
               vals[pos] = row;
               if (WIDE) keys64[pos] = ((uint64_t)(by0 * (uint32_t)TX + t) << 32) | (uint64_t)depth_bits[row];
@@ -1109,7 +1117,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
       if (band_rows > 2) band_rows = 2;
       if (band_rows > TY) band_rows = TY;
       const uint64_t items_cap = (uint64_t)F.chunks * (((uint32_t)TY + band_rows - 1) / band_rows);
-      const uint32_t grid = (uint32_t)(items_cap < (uint64_t)sms * 3 ? items_cap : (uint64_t)sms * 3);
+      const uint32_t grid = (uint32_t)(items_cap < (uint64_t)sms * 6 ? items_cap : (uint64_t)sms * 6);
 #define LAUNCH_SCATTER(WIDE, EXACT)                                                                                    \
   do {                                                                                                                 \
     ODIN_CUDA(cudaFuncSetAttribute(scatter_instances_kernel<WIDE, EXACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
