@@ -4,8 +4,8 @@
 // One warp owns one tile.  Lane l handles column x = l % 16 and, for slot s = 0..7, row y = 2 s + l / 16: a slot is two
 // adjacent pixel rows of the tile, so "does any lane of the warp touch this row in slot s" is spatially coherent and
 // worth a warp-uniform branch.  Per row of the sorted list the lane computes once
-//     dx = u - x,  h0 = -A dx^2 / 2,  h1 = -B dx,  h2 = -C / 2
-// and per slot only  power = h0 + dy (h1 + h2 dy)  (two fused multiply-adds), alpha = min(alpha_max, o * exp(power)).
+//     dx = u - x,  h0 = sA dx^2 + lo,  h1 = sB dx,  h2 = sC          (see BlendRow)
+// and per slot only  p = h0 + dy (h1 + h2 dy)  (two fused multiply-adds), alpha = min(alpha_max, 2^p).
 #pragma once
 #include "common.cuh"
 
@@ -83,20 +83,47 @@ constexpr int BLEND_SLOTS = 8;          // pixels per lane
 constexpr int BLEND_WARPS = 4;          // tiles per block (warps do not synchronise with each other)
 constexpr int BLEND_THREADS = 32 * BLEND_WARPS;
 
-struct BlendRow {  // one row of the tile's list as staged in shared memory
+// One row of the tile's list as staged in shared memory.  The exponent is evaluated in base 2 with the opacity folded
+// in: with sA = -A log2(e) / 2, sB = -B log2(e), sC = -C log2(e) / 2 and lo = log2(opacity),
+//     p = sA dx^2 + sB dx dy + sC dy^2 + lo = log2(opacity * exp(power)),   alpha = min(alpha_max, 2^p),
+// so a pixel costs two fused multiply-adds, the tests, one ex2 and one min.  The skip test "alpha < alpha_min" is
+// p < log2(alpha_min), a constant of the launch, and "power > 0" is p > lo; a pixel that fails never reaches ex2.  All
+// blend kernels stage rows through blend_stage_row and form p through blend_x_terms / blend_power, so they agree bit
+// for bit on every (pixel, row) pair.  An opacity of 0 gives lo = -inf (nothing passes).
+struct BlendRow {
   float4 q0;       // u, v, r, g
-  float4 q1;       // conic A, B, C, opacity
+  float4 q1;       // sA, sB, sC, lo
 };
+
+constexpr float BLEND_LOG2E = 1.4426950408889634f;
+constexpr float BLEND_LN2 = 0.6931471805599453f;
+
+__device__ __forceinline__ float4 blend_stage_conic(float4 conic_o) {
+  return make_float4(conic_o.x * (-0.5f * BLEND_LOG2E), conic_o.y * (-BLEND_LOG2E), conic_o.z * (-0.5f * BLEND_LOG2E),
+                     log2f(conic_o.w));
+}
+
+// per row and lane: the terms of p that depend on the column only (dx = u - x)
+__device__ __forceinline__ void blend_x_terms(const float4 q1, float dx, float& h0, float& h1, float& h2) {
+  h0 = fmaf(q1.x * dx, dx, q1.w);
+  h1 = q1.y * dx;
+  h2 = q1.z;
+}
 
 __device__ __forceinline__ float blend_power(float h0, float h1, float h2, float dy) {
   return fmaf(dy, fmaf(h2, dy, h1), h0);
 }
 
-// The skip test "alpha = opacity * exp(power) < alpha_min" is taken on the exponent: power < log(alpha_min / opacity).
-// The threshold is computed once per row when it is staged, so a pixel that fails costs two fused multiply-adds and
-// two compares and never reaches ex2; all four blend kernels use this same form so that they agree on every pair.
-// An opacity of 0 gives +inf (nothing passes); an opacity below alpha_min gives a positive threshold, which the
-// additional test power <= 0 can never meet.
+__device__ __forceinline__ bool blend_passes(float p, float lo, float l2amin) { return p <= lo && p >= l2amin; }
+
+__device__ __forceinline__ float blend_ex2(float p) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(p));
+  return y;
+}
+
+// Threshold of the natural exponent, power >= log(alpha_min / opacity), used by the tile test below when a row is
+// staged.  An opacity of 0 gives +inf; an opacity below alpha_min gives a positive threshold (nothing passes).
 __device__ __forceinline__ float blend_power_cut(float alpha_min, float opacity) { return logf(alpha_min / opacity); }
 
 // Can the row pass the skip test at any pixel of the tile whose first pixel centre is (x_lo, y_lo)?  The set

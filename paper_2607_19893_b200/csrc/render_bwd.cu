@@ -57,10 +57,11 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
                         const float* __restrict__ dL, float* __restrict__ g2d, uint32_t* __restrict__ ticket,
                         uint8_t* __restrict__ row_active, uint32_t row_cap) {
   __shared__ BlendRow s_rowdata[BLEND_WARPS][32];
-  __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, power threshold
+  __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, 1 / opacity
   __shared__ uint32_t s_rowid[BLEND_WARPS][32];
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t n_seg = min(*seg_count, seg_cap);
+  const float l2amin = log2f(alpha_min);
   // warps never synchronise with each other; each keeps taking work items from a ticket counter (see the forward
   // kernel).  The recorded segments come first: they are full-length, the segments 0 of most tiles are not.
   while (true) {
@@ -139,12 +140,13 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       const float2 c = xy[r];
       BlendRow row;
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
-      row.q1 = conic_o[r];
+      const float4 co = conic_o[r];
+      row.q1 = blend_stage_conic(co);
       s_rowdata[warp][lane] = row;
-      const float cut = blend_power_cut(alpha_min, row.q1.w);
-      s_blue[warp][lane] = make_float2(rgb[3 * (size_t)r + 2], cut);
+      s_blue[warp][lane] = make_float2(rgb[3 * (size_t)r + 2], 1.f / co.w);
       s_rowid[warp][lane] = r;
-      reach = blend_reaches_tile(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, cut, tile_x0 + 0.5f, tile_y0 + 0.5f);
+      reach = blend_reaches_tile(c.x, c.y, co.x, co.y, co.z, blend_power_cut(alpha_min, co.w), tile_x0 + 0.5f,
+                                 tile_y0 + 0.5f);
     }
     // warp-uniform: only the rows whose ellipse reaches the tile are evaluated, back to front
     uint32_t rows = __ballot_sync(0xffffffffu, reach);
@@ -153,9 +155,10 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       const int j = 31 - __clz(rows);
       rows ^= 1u << j;
       const float4 q0 = s_rowdata[warp][j].q0, q1 = s_rowdata[warp][j].q1;
-      const float blue = s_blue[warp][j].x, pcut = s_blue[warp][j].y;
+      const float blue = s_blue[warp][j].x;
       const float dx = q0.x - fx;
-      const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
+      float h0, h1, h2;
+      blend_x_terms(q1, dx, h0, h1, h2);
       const float dy0 = q0.y - fy0;
       const uint32_t k = seg_base + b + j;
       // phase 1, straight line: the eight exponents and skip tests are independent and overlap in the pipeline
@@ -164,21 +167,19 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
 #pragma unroll
       for (int s = 0; s < BLEND_SLOTS; ++s) {
         pw[s] = blend_power(h0, h1, h2, dy0 - (float)(2 * s));
-        pass |= (k < last[s] && pw[s] <= 0.f && pw[s] >= pcut) ? (1u << s) : 0u;
+        pass |= (k < last[s] && blend_passes(pw[s], q1.w, l2amin)) ? (1u << s) : 0u;
       }
       const uint32_t hit = __reduce_or_sync(0xffffffffu, pass);  // bit s: some lane of the warp passes in slot s
       if (hit == 0) continue;
       // phase 2: per-lane sums over its eight pixels; the x-dependent factors are applied once at the end
-      float ar = 0.f, ag = 0.f, ab = 0.f, ao = 0.f, gpsum = 0.f, m1y = 0.f, m2yy = 0.f;
+      float ar = 0.f, ag = 0.f, ab = 0.f, gpsum = 0.f, m1y = 0.f, m2yy = 0.f;
 #pragma unroll
       for (int s = 0; s < BLEND_SLOTS; ++s) {
         if (!(hit >> s & 1u)) continue;
         {
           if (pass >> s & 1u) {
             const float dy = dy0 - (float)(2 * s);
-            const float power = pw[s];
-            const float G = __expf(power);
-            const float og = q1.w * G;
+            const float og = blend_ex2(pw[s]);  // opacity * exp(power)
             const float alpha = fminf(alpha_max, og);
             const float inv = __fdividef(1.f, 1.f - alpha);
             const float Tb = T[s] * inv;  // transmittance in front of this row
@@ -189,9 +190,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
             SG[s] = fmaf(w, cg, SG[s]);
             T[s] = Tb;
             if (og <= alpha_max) {  // a clamped alpha passes no gradient to opacity or geometry
-              const float t = G * dLda;
-              ao += t;
-              const float gp = q1.w * t;  // dL/dpower
+              const float gp = og * dLda;  // dL/dpower; dL/dopacity is this over the opacity
               gpsum += gp;
               const float gy = gp * dy;
               m1y += gy;
@@ -201,8 +200,10 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
         }
       }
       const float gd = dx * gpsum;  // sum of dL/dpower * dx
-      const float vu = -(q1.x * gd + q1.y * m1y);
-      const float vv = -(q1.z * m1y + q1.y * gd);
+      const float ao = gpsum * s_blue[warp][j].y;
+      // the staged conic is (-A log2(e) / 2, -B log2(e), -C log2(e) / 2): -(A gd + B m1y) = ln 2 (2 sA gd + sB m1y)
+      const float vu = BLEND_LN2 * fmaf(2.f * q1.x, gd, q1.y * m1y);
+      const float vv = BLEND_LN2 * fmaf(2.f * q1.z, m1y, q1.y * gd);
       const float vA = -0.5f * dx * gd, vB = -dx * m1y, vC = -0.5f * m2yy;
       const float t8 = warp_transpose_sum8(vu, vv, vA, vB, vC, ao, ar, ag, lane);
       for (int o = 16; o > 0; o >>= 1) ab += __shfl_xor_sync(0xffffffffu, ab, o);

@@ -1,7 +1,7 @@
 // Rendering phase: front-to-back alpha compositing.  Head kernel: one WARP per 16x16 tile, eight pixels per lane (see
 // blend.cuh), the tile's sorted rows staged 32 at a time through shared memory, warp-ballot early exit once every
 // pixel of the tile has terminated; per row and lane the x-dependent terms are computed once, each pixel costs two
-// fused multiply-adds, one ex2 and the blend.  Tiles still live after BLEND_HEAD entries are finished by the tail
+// fused multiply-adds, one ex2 (the exponent is kept in base 2 with the opacity folded in) and the blend.  Tiles still live after BLEND_HEAD entries are finished by the tail
 // kernel (eight warps per tile, rows staged 256 at a time).  Also the L1 image loss.
 #include "blend.cuh"
 
@@ -14,8 +14,9 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
                   float* __restrict__ final_T, uint32_t* __restrict__ n_contrib, uint32_t* __restrict__ tile_more,
                   uint32_t* __restrict__ ticket, uint32_t row_cap) {
   __shared__ BlendRow s_row[BLEND_WARPS][32];
-  __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, power threshold
+  __shared__ float s_blue[BLEND_WARPS][32];
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float l2amin = log2f(alpha_min);
   // Warps never synchronise with each other.  Each one keeps taking tiles from a ticket counter until none is left:
   // lists differ in length by orders of magnitude between tiles, and a fixed tile-to-warp map would leave most of the
   // GPU idle while the longest ones finish.
@@ -52,11 +53,12 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
       const float2 c = xy[r];
       BlendRow row;
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
-      row.q1 = conic_o[r];
+      const float4 co = conic_o[r];
+      row.q1 = blend_stage_conic(co);
       s_row[warp][lane] = row;
-      const float cut = blend_power_cut(alpha_min, row.q1.w);
-      s_blue[warp][lane] = make_float2(rgb[3 * (size_t)r + 2], cut);
-      reach = blend_reaches_tile(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, cut, tile_x0 + 0.5f, tile_y0 + 0.5f);
+      s_blue[warp][lane] = rgb[3 * (size_t)r + 2];
+      reach = blend_reaches_tile(c.x, c.y, co.x, co.y, co.z, blend_power_cut(alpha_min, co.w), tile_x0 + 0.5f,
+                                 tile_y0 + 0.5f);
     }
     // warp-uniform: only the rows whose ellipse reaches the tile are evaluated, in list order
     uint32_t rows = __ballot_sync(0xffffffffu, reach);
@@ -65,9 +67,9 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
       const int j = __ffs(rows) - 1;
       rows &= rows - 1;
       const float4 q0 = s_row[warp][j].q0, q1 = s_row[warp][j].q1;
-      const float blue = s_blue[warp][j].x, pcut = s_blue[warp][j].y;
-      const float dx = q0.x - fx;
-      const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
+      const float blue = s_blue[warp][j];
+      float h0, h1, h2;
+      blend_x_terms(q1, q0.x - fx, h0, h1, h2);
       const float dy0 = q0.y - fy0;
       const uint32_t ord = (b - start) + j + 1;
       // phase 1, straight line: the eight exponents and skip tests are independent and overlap in the pipeline
@@ -76,7 +78,7 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
 #pragma unroll
       for (int s = 0; s < BLEND_SLOTS; ++s) {
         power[s] = blend_power(h0, h1, h2, dy0 - (float)(2 * s));
-        pass |= (power[s] <= 0.f && power[s] >= pcut) ? (1u << s) : 0u;
+        pass |= blend_passes(power[s], q1.w, l2amin) ? (1u << s) : 0u;
       }
       pass &= live;
       // phase 2: ex2 and the blend, only for slots in which some lane passes
@@ -85,12 +87,12 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
       for (int s = 0; s < BLEND_SLOTS; ++s) {
         if (!(hit >> s & 1u)) continue;
         if (pass >> s & 1u) {
-          const float alpha = fminf(alpha_max, q1.w * __expf(power[s]));
-          const float Tn = T[s] * (1.f - alpha);
+          const float alpha = fminf(alpha_max, blend_ex2(power[s]));
+          const float w = alpha * T[s];
+          const float Tn = T[s] - w;
           if (Tn < t_min) {
             live &= ~(1u << s);
           } else {
-            const float w = alpha * T[s];
             C0[s] = fmaf(q0.z, w, C0[s]); C1[s] = fmaf(q0.w, w, C1[s]); C2[s] = fmaf(blue, w, C2[s]);
             T[s] = Tn;
             last[s] = ord;
@@ -137,7 +139,7 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
   const int tile = blockIdx.x;
   if (!tile_first[tile]) return;
   __shared__ BlendRow s_row[BLEND_TAIL_THREADS];
-  __shared__ float2 s_blue[BLEND_TAIL_THREADS];  // blue, power threshold
+  __shared__ float s_blue[BLEND_TAIL_THREADS];
   __shared__ uint32_t s_ord[BLEND_TAIL_THREADS];  // 1-based position of the row in the tile's list
   __shared__ uint32_t s_wcnt[BLEND_TAIL_THREADS / 32];
   __shared__ uint32_t s_slot;
@@ -148,6 +150,7 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
   const float fx = (float)px + 0.5f;
   const float fy0 = (float)(ty * 16 + (ly & 1)) + 0.5f;
   const float slot2 = (float)(2 * (ly >> 1));
+  const float l2amin = log2f(alpha_min);
   const uint2 rg = ranges[tile];
   const uint32_t start = rg.x, end = rg.y;
   const size_t pix = (size_t)py * W + px, plane = (size_t)W * H;
@@ -170,15 +173,16 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
     // stage 256 entries and keep, in list order, only the rows whose ellipse reaches the tile
     const uint32_t i = b + threadIdx.x;
     BlendRow row;
-    float2 bp = make_float2(0.f, 0.f);
+    float bp = 0.f;
     bool reach = false;
     if (i < end) {
       const uint32_t r = min(vals[i], row_cap - 1);
       const float2 c = xy[r];
       row.q0 = make_float4(c.x, c.y, rgb[3 * (size_t)r], rgb[3 * (size_t)r + 1]);
-      row.q1 = conic_o[r];
-      bp = make_float2(rgb[3 * (size_t)r + 2], blend_power_cut(alpha_min, row.q1.w));
-      reach = blend_reaches_tile(c.x, c.y, row.q1.x, row.q1.y, row.q1.z, bp.y, tile_x0, tile_y0);
+      const float4 co = conic_o[r];
+      row.q1 = blend_stage_conic(co);
+      bp = rgb[3 * (size_t)r + 2];
+      reach = blend_reaches_tile(c.x, c.y, co.x, co.y, co.z, blend_power_cut(alpha_min, co.w), tile_x0, tile_y0);
     }
     const uint32_t wm = __ballot_sync(0xffffffffu, reach);
     if (lane == 0) s_wcnt[warp] = __popc(wm);
@@ -218,28 +222,27 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
       // four rows at a time: their exponents and skip tests are independent (a single pixel per thread has no other
       // source of instruction-level parallelism), the blends are then applied in order
       for (int j = 0; j < cnt && !done; j += 4) {
-        float pw[4], opac[4], cr[4], cg[4], cb[4];
+        float pw[4], cr[4], cg[4], cb[4];
         bool pass[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const int ju = min(j + u, cnt - 1);
           const float4 q0 = s_row[ju].q0, q1 = s_row[ju].q1;
-          const float2 bp = s_blue[ju];
-          const float dx = q0.x - fx;
-          const float h0 = -0.5f * q1.x * dx * dx, h1 = -q1.y * dx, h2 = -0.5f * q1.z;
+          float h0, h1, h2;
+          blend_x_terms(q1, q0.x - fx, h0, h1, h2);
           pw[u] = blend_power(h0, h1, h2, (q0.y - fy0) - slot2);
-          pass[u] = (j + u < cnt) && pw[u] <= 0.f && pw[u] >= bp.y;
-          opac[u] = q1.w; cr[u] = q0.z; cg[u] = q0.w; cb[u] = bp.x;
+          pass[u] = (j + u < cnt) && blend_passes(pw[u], q1.w, l2amin);
+          cr[u] = q0.z; cg[u] = q0.w; cb[u] = s_blue[ju];
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           if (pass[u] && !done) {
-            const float alpha = fminf(alpha_max, opac[u] * __expf(pw[u]));
-            const float Tn = T * (1.f - alpha);
+            const float alpha = fminf(alpha_max, blend_ex2(pw[u]));
+            const float w = alpha * T;
+            const float Tn = T - w;
             if (Tn < t_min) {
               done = true;
             } else {
-              const float w = alpha * T;
               // the image keeps its one sequential sum per pixel (so it does not depend on where the batches fall);
               // the per-batch sums, in double, only feed the records
               C0 = fmaf(cr[u], w, C0); C1 = fmaf(cg[u], w, C1); C2 = fmaf(cb[u], w, C2);

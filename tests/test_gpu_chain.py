@@ -24,6 +24,8 @@ pytestmark = pytest.mark.gpu
 #    term, which the stage-isolated bound does not contain (a strongly anisotropic splat amplifies an ulp of its
 #    scales into 1e-4 of its conic); ROWS_SLACK = 8 is about 2x the largest ratio measured on the five presets (4.3,
 #    one word of 5e7 at preset 5; printed as rows_worst).
+#    A pixel whose L1 gradient sign differs is accepted only where the oracle's value is within 1e-4 of the target
+#    (the gradient is discontinuous there); its primitives are exempt too (fewer than 1e-3 of the robust pixels).
 #  * Adam: every touched word of params / m / v against the oracle's Adam applied to the DEVICE's gradient rows, 2e-5
 #    relative (the stage-isolated bar), and against the oracle's own chained result wherever the two gradients agree to
 #    1e-3 relative (the benchmark spec's 1e-3 relative, 1e-5 absolute floor).
@@ -150,7 +152,17 @@ def run_chain(oracle32, w, steps, views, window=None, row_capacity=None, instanc
         # primitives in the walked prefix of such a pixel's list are exempt from the gradient comparison
         ncon_dev = G.u32(tr.n_contrib)
         robust = (o["pix_margin"] > PIX_MARGIN) & ~aff_pix
-        fragile_yx = np.argwhere(~robust & ~aff_pix)
+        # The L1 gradient is sign(out - target) / (3 H W): discontinuous where a channel meets its target.  A pixel
+        # whose device gradient has the other sign is legitimate only if the oracle's value lies within the pixel bar
+        # (1e-4) of the target there; the primitives blending at such a pixel see a different incoming gradient and are
+        # exempt like those of a fragile pixel.
+        dL_dev = tr.dL.cpu().numpy().reshape(o["dL_dout"].shape)
+        loss_flip = (np.sign(dL_dev) != np.sign(o["dL_dout"]))
+        near_target = np.abs(o["out"] - tgt) < 1e-4
+        assert not (loss_flip & ~near_target)[:, robust].any()
+        loss_flip = loss_flip.any(axis=0)
+        assert loss_flip[robust].mean() <= 1e-3
+        fragile_yx = np.argwhere((~robust | loss_flip) & ~aff_pix)
         upto = np.maximum(o["n_contrib"], ncon_dev)[tuple(fragile_yx.T)] + 1 if len(fragile_yx) else []
         frag_prims = np.zeros(n, bool)
         frag_prims[G.blended_at_pixels(o, fragile_yx, upto, tx)] = True
@@ -251,7 +263,7 @@ def run_chain(oracle32, w, steps, views, window=None, row_capacity=None, instanc
         assert np.all(np.abs(dp - hp)[agree] <= 1e-3 * np.abs(hp)[agree] + 1e-5)
         G.report(f"{tag}[step {s}]", V=vdev, M=mm_dev, differing_prims=len(D), fragile_prims_within_2e6=int(
                  (o["proj"].margin < FRAGILE_PRIM).sum()), same_depth_bits=bool(same_depth),
-                 affected_tiles_pixels=int(aff_pix.sum()), robust_pixels=float(robust.mean()), fragile_pixels=fragile_frac,
+                 affected_tiles_pixels=int(aff_pix.sum()), robust_pixels=float(robust.mean()), fragile_pixels=fragile_frac, loss_sign_flips=int(loss_flip.sum()),
                  pix_err_robust=float(pix_err[:, robust].max()), pix_err_all=float(pix_err[:, ~aff_pix].max()),
                  active_o=len(act_o), active_diff=len(act_diff), rows_checked=float(checked.mean()),
                  rows_within_1x=float((ratio <= 1).mean()), rows_within_2x=float((ratio <= 2).mean()),
