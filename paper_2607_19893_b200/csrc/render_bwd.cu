@@ -161,44 +161,38 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
       blend_x_terms(q1, dx, h0, h1, h2);
       const float dy0 = q0.y - fy0;
       const uint32_t k = seg_base + b + j;
-      // phase 1, straight line: the eight exponents and skip tests are independent and overlap in the pipeline
+      // the eight exponents first (independent, they overlap in the pipeline), then test and differentiate slot by slot;
+      // per-lane sums over its eight pixels, the x-dependent factors are applied once at the end
       float pw[BLEND_SLOTS];
-      uint32_t pass = 0;
 #pragma unroll
-      for (int s = 0; s < BLEND_SLOTS; ++s) {
-        pw[s] = blend_power(h0, h1, h2, dy0 - (float)(2 * s));
-        pass |= (k < last[s] && blend_passes(pw[s], q1.w, l2amin)) ? (1u << s) : 0u;
-      }
-      const uint32_t hit = __reduce_or_sync(0xffffffffu, pass);  // bit s: some lane of the warp passes in slot s
-      if (hit == 0) continue;
-      // phase 2: per-lane sums over its eight pixels; the x-dependent factors are applied once at the end
+      for (int s = 0; s < BLEND_SLOTS; ++s) pw[s] = blend_power(h0, h1, h2, dy0 - (float)(2 * s));
       float ar = 0.f, ag = 0.f, ab = 0.f, gpsum = 0.f, m1y = 0.f, m2yy = 0.f;
+      bool some = false;
 #pragma unroll
       for (int s = 0; s < BLEND_SLOTS; ++s) {
-        if (!(hit >> s & 1u)) continue;
-        {
-          if (pass >> s & 1u) {
-            const float dy = dy0 - (float)(2 * s);
-            const float og = blend_ex2(pw[s]);  // opacity * exp(power)
-            const float alpha = fminf(alpha_max, og);
-            const float inv = __fdividef(1.f, 1.f - alpha);
-            const float Tb = T[s] * inv;  // transmittance in front of this row
-            const float w = alpha * Tb;
-            ar = fmaf(w, g0[s], ar); ag = fmaf(w, g1[s], ag); ab = fmaf(w, g2[s], ab);
-            const float cg = fmaf(blue, g2[s], fmaf(q0.w, g1[s], q0.z * g0[s]));
-            const float dLda = Tb * cg - SG[s] * inv;
-            SG[s] = fmaf(w, cg, SG[s]);
-            T[s] = Tb;
-            if (og <= alpha_max) {  // a clamped alpha passes no gradient to opacity or geometry
-              const float gp = og * dLda;  // dL/dpower; dL/dopacity is this over the opacity
-              gpsum += gp;
-              const float gy = gp * dy;
-              m1y += gy;
-              m2yy = fmaf(gy, dy, m2yy);
-            }
+        if (k < last[s] && blend_passes(pw[s], q1.w, l2amin)) {
+          some = true;
+          const float dy = dy0 - (float)(2 * s);
+          const float og = blend_ex2(pw[s]);  // opacity * exp(power)
+          const float alpha = fminf(alpha_max, og);
+          const float inv = __fdividef(1.f, 1.f - alpha);
+          const float Tb = T[s] * inv;  // transmittance in front of this row
+          const float w = alpha * Tb;
+          ar = fmaf(w, g0[s], ar); ag = fmaf(w, g1[s], ag); ab = fmaf(w, g2[s], ab);
+          const float cg = fmaf(blue, g2[s], fmaf(q0.w, g1[s], q0.z * g0[s]));
+          const float dLda = Tb * cg - SG[s] * inv;
+          SG[s] = fmaf(w, cg, SG[s]);
+          T[s] = Tb;
+          if (og <= alpha_max) {  // a clamped alpha passes no gradient to opacity or geometry
+            const float gp = og * dLda;  // dL/dpower; dL/dopacity is this over the opacity
+            gpsum += gp;
+            const float gy = gp * dy;
+            m1y += gy;
+            m2yy = fmaf(gy, dy, m2yy);
           }
         }
       }
+      if (!__any_sync(0xffffffffu, some)) continue;  // the row blends nowhere in the tile
       const float gd = dx * gpsum;  // sum of dL/dpower * dx
       const float ao = gpsum * s_blue[warp][j].y;
       // the staged conic is (-A log2(e) / 2, -B log2(e), -C log2(e) / 2): -(A gd + B m1y) = ln 2 (2 sA gd + sB m1y)

@@ -72,21 +72,13 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
       blend_x_terms(q1, q0.x - fx, h0, h1, h2);
       const float dy0 = q0.y - fy0;
       const uint32_t ord = (b - start) + j + 1;
-      // phase 1, straight line: the eight exponents and skip tests are independent and overlap in the pipeline
+      // the eight exponents first (independent, they overlap in the pipeline), then test and blend slot by slot
       float power[BLEND_SLOTS];
-      uint32_t pass = 0;
+#pragma unroll
+      for (int s = 0; s < BLEND_SLOTS; ++s) power[s] = blend_power(h0, h1, h2, dy0 - (float)(2 * s));
 #pragma unroll
       for (int s = 0; s < BLEND_SLOTS; ++s) {
-        power[s] = blend_power(h0, h1, h2, dy0 - (float)(2 * s));
-        pass |= blend_passes(power[s], q1.w, l2amin) ? (1u << s) : 0u;
-      }
-      pass &= live;
-      // phase 2: ex2 and the blend, only for slots in which some lane passes
-      const uint32_t hit = __reduce_or_sync(0xffffffffu, pass);  // bit s: some lane of the warp passes in slot s
-#pragma unroll
-      for (int s = 0; s < BLEND_SLOTS; ++s) {
-        if (!(hit >> s & 1u)) continue;
-        if (pass >> s & 1u) {
+        if (blend_passes(power[s], q1.w, l2amin) && (live >> s & 1u)) {
           const float alpha = fminf(alpha_max, blend_ex2(power[s]));
           const float w = alpha * T[s];
           const float Tn = T[s] - w;
