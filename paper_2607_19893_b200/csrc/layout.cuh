@@ -25,9 +25,16 @@ constexpr uint32_t OFFSET_TILE = 2048;                       // rows per look-ba
 
 static inline size_t ws_align(size_t x) { return (x + 255) / 256 * 256; }
 
-// [ticket: 256 B][state: u64 per tile]
-static inline size_t project_ws_bytes(uint32_t n) {
+// [ticket: 256 B][state: u64 per 2048 primitives][packed total per 256 primitives: u64][exact (rows, instances) per
+// chunk of the scan, sized for chunks of 2048: 2 x u64]; the last two are used by scenes too large for the fused kernel
+static inline size_t project_ws_group_offset(uint32_t n) {
   return 256 + ws_align(((size_t)n + PROJECT_TILE - 1) / PROJECT_TILE * 8);
+}
+static inline size_t project_ws_chunk_offset(uint32_t n) {
+  return project_ws_group_offset(n) + ws_align(((size_t)n + 255) / 256 * 8);
+}
+static inline size_t project_ws_bytes(uint32_t n) {
+  return project_ws_chunk_offset(n) + ws_align(((size_t)n + PROJECT_TILE - 1) / PROJECT_TILE * 16);
 }
 static inline size_t touched_ws_bytes(uint32_t n) {
   return 256 + ws_align(((size_t)n + TOUCHED_TILE - 1) / TOUCHED_TILE * 8);

@@ -151,7 +151,8 @@ template <bool EXACT>
 __global__ void __launch_bounds__(256)
 project_cull_kernel(const float* __restrict__ means, const float* __restrict__ log_scales, const float4* __restrict__ quats,
                     const float* __restrict__ opacity_logit, uint32_t n, CamParams cam, BinRule rule,
-                    uint32_t* __restrict__ tiles_touched) {
+                    uint32_t* __restrict__ tiles_touched, unsigned long long* __restrict__ group_total,
+                    unsigned long long* __restrict__ chunk_total, uint32_t groups_per_chunk) {
   const uint32_t p = blockIdx.x * 256u + threadIdx.x;
   Footprint f = {};
   if (p < n) {
@@ -163,6 +164,19 @@ project_cull_kernel(const float* __restrict__ means, const float* __restrict__ l
   }
   if (EXACT) f.tiles = exact_tiles_warp(f, rule, opacity_logit, p);
   if (p < n) tiles_touched[p] = f.tiles;
+  // what the scan needs to start anywhere without waiting: the packed (rows, instances) total of this block's 256
+  // primitives and the exact totals of the chunk of blocks it belongs to, added up by the warps that have something to
+  // add (both zeroed before the launch; no block barrier, so a warp with a long covariance path holds nobody up)
+  const uint32_t rows_w = __popc(__ballot_sync(0xffffffffu, f.tiles != 0));
+  if (rows_w == 0) return;
+  uint32_t inst = f.tiles;  // at most 2^20 per primitive: 2^25 per warp
+  for (int o = 16; o > 0; o >>= 1) inst += __shfl_xor_sync(0xffffffffu, inst, o);
+  if ((threadIdx.x & 31) == 0) {
+    atomicAdd(&group_total[blockIdx.x], ((unsigned long long)rows_w << PACK_SHIFT) | (unsigned long long)inst);
+    const size_t c = blockIdx.x / groups_per_chunk;
+    atomicAdd(&chunk_total[2 * c], (unsigned long long)rows_w);
+    atomicAdd(&chunk_total[2 * c + 1], (unsigned long long)inst);
+  }
 }
 
 // Scan of the tile counts, for small scenes fused with the counting.  A block takes `rounds` x 2048 consecutive
@@ -185,8 +199,9 @@ project_scan_kernel(const float* __restrict__ means, const float* __restrict__ l
                     const float4* __restrict__ quats, const float* __restrict__ opacity_logit, uint32_t n, CamParams cam,
                     BinRule rule, uint32_t* tiles_touched, uint32_t capacity, uint32_t* __restrict__ prim_id,
                     uint32_t* __restrict__ tile_offset, uint32_t* __restrict__ num_rows,
-                    uint64_t* __restrict__ num_instances, uint32_t* ticket, uint64_t* state, int* status, int rounds,
-                    int spin_limit, uint32_t* __restrict__ touched_mask) {
+                    uint64_t* __restrict__ num_instances, uint32_t* ticket, uint64_t* state,
+                    const uint64_t* __restrict__ group_total, const uint64_t* __restrict__ chunk_total, int* status,
+                    int rounds, int spin_limit, uint32_t* __restrict__ touched_mask) {
   __shared__ uint32_t s_tile;
   __shared__ uint64_t s_warp[SCAN_THREADS / 32];
   __shared__ uint64_t s_inst[SCAN_THREADS / 32];
@@ -194,131 +209,161 @@ project_scan_kernel(const float* __restrict__ means, const float* __restrict__ l
   __shared__ uint64_t s_tot[SCAN_MAX_ROUNDS][SCAN_THREADS / 32];  // packed total of (round, warp)
   __shared__ uint32_t s_t[FUSED ? SCAN_ITEMS : 1][SCAN_THREADS];  // fused (one round): tile count of item j of thread t
   __shared__ uint8_t s_list[FUSED ? SCAN_THREADS / 32 : 1][32 * SCAN_ITEMS];  // per warp: survivors as 32 j + lane
-  unsigned long long* exact_instances = reinterpret_cast<unsigned long long*>(ticket + 2);  // zeroed with the ticket
-  if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
-  __syncthreads();
-  const uint32_t tile = s_tile;
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t chunk = PROJECT_TILE * (uint32_t)rounds;
-  const uint32_t chunk_base = tile * chunk;
-
-  // ---- A
-  uint64_t rows_b = 0, inst_b = 0;  // the warp's rows and instances over all rounds (uniform over the warp)
-  int done = 0;                      // rounds that hold primitives (uniform over the block)
-  for (int rnd = 0; rnd < rounds; ++rnd) {
-    if (chunk_base + rnd * PROJECT_TILE >= n) break;  // uniform over the block
-    const uint32_t warp_base = chunk_base + rnd * PROJECT_TILE + warp * (32 * SCAN_ITEMS);
-    uint32_t t[SCAN_ITEMS];
-    if (FUSED) {
-      float ct[SCAN_ITEMS][3];  // mean, then camera-space mean
-#pragma unroll
-      for (int j = 0; j < SCAN_ITEMS; ++j) {
-        const uint32_t p = warp_base + 32 * j + lane;
-        ct[j][0] = ct[j][1] = ct[j][2] = 0.f;
-        if (p < n) {
-          ct[j][0] = means[3 * (size_t)p]; ct[j][1] = means[3 * (size_t)p + 1]; ct[j][2] = means[3 * (size_t)p + 2];
+  int done = 0;  // rounds that hold primitives (uniform over the block)
+  uint32_t tile, chunk_base;
+  if (FUSED) {
+    unsigned long long* exact_instances = reinterpret_cast<unsigned long long*>(ticket + 2);  // zeroed with the ticket
+    if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
+    __syncthreads();
+    tile = s_tile;
+    chunk_base = tile * chunk;
+    // ---- A
+    uint64_t rows_b = 0, inst_b = 0;  // the warp's rows and instances over all rounds (uniform over the warp)
+    for (int rnd = 0; rnd < rounds; ++rnd) {
+      if (chunk_base + rnd * PROJECT_TILE >= n) break;  // uniform over the block
+      const uint32_t warp_base = chunk_base + rnd * PROJECT_TILE + warp * (32 * SCAN_ITEMS);
+      uint32_t t[SCAN_ITEMS];
+      {
+        float ct[SCAN_ITEMS][3];  // mean, then camera-space mean
+  #pragma unroll
+        for (int j = 0; j < SCAN_ITEMS; ++j) {
+          const uint32_t p = warp_base + 32 * j + lane;
+          ct[j][0] = ct[j][1] = ct[j][2] = 0.f;
+          if (p < n) {
+            ct[j][0] = means[3 * (size_t)p]; ct[j][1] = means[3 * (size_t)p + 1]; ct[j][2] = means[3 * (size_t)p + 2];
+          }
+        }
+        uint32_t front = 0;
+  #pragma unroll
+        for (int j = 0; j < SCAN_ITEMS; ++j) {
+          const uint32_t p = warp_base + 32 * j + lane;
+          const float mx = ct[j][0], my = ct[j][1], mz = ct[j][2];
+          odin_camera_space(cam, mx, my, mz, ct[j]);
+          if (p < n && ct[j][2] > cam.znear && ct[j][2] < cam.zfar) front |= 1u << j;
+        }
+        float ls[SCAN_ITEMS][3];
+  #pragma unroll
+        for (int j = 0; j < SCAN_ITEMS; ++j) {
+          const uint32_t p = warp_base + 32 * j + lane;
+          ls[j][0] = ls[j][1] = ls[j][2] = 0.f;
+          if (front >> j & 1u) {
+            ls[j][0] = log_scales[3 * (size_t)p]; ls[j][1] = log_scales[3 * (size_t)p + 1];
+            ls[j][2] = log_scales[3 * (size_t)p + 2];
+          }
+        }
+        uint32_t n_alive = 0;
+  #pragma unroll
+        for (int j = 0; j < SCAN_ITEMS; ++j) {
+          const bool alive = (front >> j & 1u) && cull_survives(cam, rule, ct[j], ls[j][0], ls[j][1], ls[j][2]);
+          const uint32_t b = __ballot_sync(0xffffffffu, alive);
+          if (alive) s_list[warp][n_alive + __popc(b & ((1u << lane) - 1u))] = (uint8_t)(32 * j + lane);
+          n_alive += __popc(b);
+          s_t[j][threadIdx.x] = 0;
+        }
+        __syncwarp();
+        // exact footprints of the survivors, a warp-load at a time
+        for (uint32_t i0 = 0; i0 < n_alive; i0 += 32) {
+          const bool have = i0 + lane < n_alive;
+          const uint32_t q = have ? s_list[warp][i0 + lane] : 0u;
+          const uint32_t p = warp_base + q;
+          Footprint f = {};
+          if (have) f = project_footprint(cam, rule, means, log_scales, quats, opacity_logit, p);
+          if (EXACT) f.tiles = exact_tiles_warp(f, rule, opacity_logit, p);
+          if (have) s_t[q >> 5][warp * 32 + (q & 31)] = f.tiles;
+        }
+        __syncwarp();
+  #pragma unroll
+        for (int j = 0; j < SCAN_ITEMS; ++j) {
+          const uint32_t p = warp_base + 32 * j + lane;
+          t[j] = s_t[j][threadIdx.x];
+          if (p < n) tiles_touched[p] = t[j];
         }
       }
-      uint32_t front = 0;
-#pragma unroll
+      // the warp's packed (rows, instances) total of this round
+      uint32_t rows_w = 0;
+      uint64_t inst_l = 0;
+  #pragma unroll
       for (int j = 0; j < SCAN_ITEMS; ++j) {
-        const uint32_t p = warp_base + 32 * j + lane;
-        const float mx = ct[j][0], my = ct[j][1], mz = ct[j][2];
-        odin_camera_space(cam, mx, my, mz, ct[j]);
-        if (p < n && ct[j][2] > cam.znear && ct[j][2] < cam.zfar) front |= 1u << j;
+        rows_w += __popc(__ballot_sync(0xffffffffu, t[j] != 0));
+        inst_l += t[j];
       }
-      float ls[SCAN_ITEMS][3];
-#pragma unroll
-      for (int j = 0; j < SCAN_ITEMS; ++j) {
-        const uint32_t p = warp_base + 32 * j + lane;
-        ls[j][0] = ls[j][1] = ls[j][2] = 0.f;
-        if (front >> j & 1u) {
-          ls[j][0] = log_scales[3 * (size_t)p]; ls[j][1] = log_scales[3 * (size_t)p + 1];
-          ls[j][2] = log_scales[3 * (size_t)p + 2];
+      for (int o = 16; o > 0; o >>= 1) inst_l += __shfl_xor_sync(0xffffffffu, inst_l, o);
+      if (lane == 0) s_tot[rnd][warp] = ((uint64_t)rows_w << PACK_SHIFT) + inst_l;
+      rows_b += rows_w;
+      inst_b += inst_l;
+      done = rnd + 1;
+    }
+
+    // ---- B.  The instance field of the packed value holds 34 bits and there are up to 2^21 blocks of up to 2^14 x 2^20
+    // instances, so the packed sums can carry into the row field when the view has 2^32 instances or more (an error by
+    // definition).  That case is caught on a counter of its own: every block adds its exact instance count (kept apart
+    // in 64 bits, the packed copy saturated) to a 64-bit total, and whoever sees that total reach 2^32 reports
+    // ODIN_ERR_CAPACITY.  The outputs of such a view are meaningless but every write stays inside the caller's
+    // capacities (the row guard below).
+    if (lane == 0) { s_warp[warp] = rows_b; s_inst[warp] = inst_b; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      uint64_t total = (lane < SCAN_THREADS / 32) ? s_warp[lane] : 0ull;
+      uint64_t total_inst = (lane < SCAN_THREADS / 32) ? s_inst[lane] : 0ull;
+      for (int o = 16; o > 0; o >>= 1) {
+        total += __shfl_xor_sync(0xffffffffu, total, o);
+        total_inst += __shfl_xor_sync(0xffffffffu, total_inst, o);
+      }
+      if (lane == 0 && total_inst != 0) {
+        const unsigned long long seen = atomicAdd(exact_instances, (unsigned long long)total_inst);
+        if (seen + total_inst >= (1ull << 32)) odin_set_error(status, ODIN_ERR_CAPACITY);
+      }
+      total = (total << PACK_SHIFT) | (total_inst < (1ull << 32) ? total_inst : ((1ull << 32) - 1));
+      const uint64_t base = odin_lookback_u64(state, tile, total, status, spin_limit);
+      if (lane == 0) {
+        s_base = base;
+        if (tile == (n + chunk - 1) / chunk - 1) {  // last block: totals
+          const uint64_t all = base + total;
+          const uint64_t rows = all >> PACK_SHIFT, inst = all & PACK_LOW;
+          *num_rows = (uint32_t)(rows < capacity ? rows : capacity);
+          *num_instances = inst;
+          if (rows > capacity || inst >= (1ull << 32)) odin_set_error(status, ODIN_ERR_CAPACITY);
         }
       }
-      uint32_t n_alive = 0;
-#pragma unroll
-      for (int j = 0; j < SCAN_ITEMS; ++j) {
-        const bool alive = (front >> j & 1u) && cull_survives(cam, rule, ct[j], ls[j][0], ls[j][1], ls[j][2]);
-        const uint32_t b = __ballot_sync(0xffffffffu, alive);
-        if (alive) s_list[warp][n_alive + __popc(b & ((1u << lane) - 1u))] = (uint8_t)(32 * j + lane);
-        n_alive += __popc(b);
-        s_t[j][threadIdx.x] = 0;
-      }
-      __syncwarp();
-      // exact footprints of the survivors, a warp-load at a time
-      for (uint32_t i0 = 0; i0 < n_alive; i0 += 32) {
-        const bool have = i0 + lane < n_alive;
-        const uint32_t q = have ? s_list[warp][i0 + lane] : 0u;
-        const uint32_t p = warp_base + q;
-        Footprint f = {};
-        if (have) f = project_footprint(cam, rule, means, log_scales, quats, opacity_logit, p);
-        if (EXACT) f.tiles = exact_tiles_warp(f, rule, opacity_logit, p);
-        if (have) s_t[q >> 5][warp * 32 + (q & 31)] = f.tiles;
-      }
-      __syncwarp();
-#pragma unroll
-      for (int j = 0; j < SCAN_ITEMS; ++j) {
-        const uint32_t p = warp_base + 32 * j + lane;
-        t[j] = s_t[j][threadIdx.x];
-        if (p < n) tiles_touched[p] = t[j];
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < SCAN_ITEMS; ++j) {
-        const uint32_t p = warp_base + 32 * j + lane;
-        t[j] = (p < n) ? tiles_touched[p] : 0u;
-      }
     }
-    // the warp's packed (rows, instances) total of this round
-    uint32_t rows_w = 0;
-    uint64_t inst_l = 0;
-#pragma unroll
-    for (int j = 0; j < SCAN_ITEMS; ++j) {
-      rows_w += __popc(__ballot_sync(0xffffffffu, t[j] != 0));
-      inst_l += t[j];
-    }
-    for (int o = 16; o > 0; o >>= 1) inst_l += __shfl_xor_sync(0xffffffffu, inst_l, o);
-    if (lane == 0) s_tot[rnd][warp] = ((uint64_t)rows_w << PACK_SHIFT) + inst_l;
-    rows_b += rows_w;
-    inst_b += inst_l;
-    done = rnd + 1;
-  }
+    __syncthreads();
 
-  // ---- B.  The instance field of the packed value holds 34 bits and there are up to 2^21 blocks of up to 2^14 x 2^20
-  // instances, so the packed sums can carry into the row field when the view has 2^32 instances or more (an error by
-  // definition).  That case is caught on a counter of its own: every block adds its exact instance count (kept apart
-  // in 64 bits, the packed copy saturated) to a 64-bit total, and whoever sees that total reach 2^32 reports
-  // ODIN_ERR_CAPACITY.  The outputs of such a view are meaningless but every write stays inside the caller's
-  // capacities (the row guard below).
-  if (lane == 0) { s_warp[warp] = rows_b; s_inst[warp] = inst_b; }
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    uint64_t total = (lane < SCAN_THREADS / 32) ? s_warp[lane] : 0ull;
-    uint64_t total_inst = (lane < SCAN_THREADS / 32) ? s_inst[lane] : 0ull;
-    for (int o = 16; o > 0; o >>= 1) {
-      total += __shfl_xor_sync(0xffffffffu, total, o);
-      total_inst += __shfl_xor_sync(0xffffffffu, total_inst, o);
+  } else {
+    // The counting kernel left the packed total of every 256 primitives (one (round, warp) of this kernel) and the exact
+    // totals of every chunk: the block's base is a sum over the chunks in front of it, nothing is waited for.
+    tile = blockIdx.x;
+    chunk_base = tile * chunk;
+    const uint32_t groups = (n + 32 * SCAN_ITEMS - 1) / (32 * SCAN_ITEMS);
+    if (threadIdx.x < (unsigned)rounds * (SCAN_THREADS / 32)) {
+      const uint64_t g = (uint64_t)tile * rounds * (SCAN_THREADS / 32) + threadIdx.x;
+      s_tot[threadIdx.x / (SCAN_THREADS / 32)][threadIdx.x % (SCAN_THREADS / 32)] = g < groups ? group_total[g] : 0ull;
     }
-    if (lane == 0 && total_inst != 0) {
-      const unsigned long long seen = atomicAdd(exact_instances, (unsigned long long)total_inst);
-      if (seen + total_inst >= (1ull << 32)) odin_set_error(status, ODIN_ERR_CAPACITY);
-    }
-    total = (total << PACK_SHIFT) | (total_inst < (1ull << 32) ? total_inst : ((1ull << 32) - 1));
-    const uint64_t base = odin_lookback_u64(state, tile, total, status, spin_limit);
-    if (lane == 0) {
-      s_base = base;
-      if (tile == (n + chunk - 1) / chunk - 1) {  // last block: totals
-        const uint64_t all = base + total;
-        const uint64_t rows = all >> PACK_SHIFT, inst = all & PACK_LOW;
-        *num_rows = (uint32_t)(rows < capacity ? rows : capacity);
-        *num_instances = inst;
-        if (rows > capacity || inst >= (1ull << 32)) odin_set_error(status, ODIN_ERR_CAPACITY);
+    if (warp == 0) {
+      uint64_t rows = 0, inst = 0;
+      for (uint32_t c = lane; c < tile; c += 32) { rows += chunk_total[2 * (size_t)c]; inst += chunk_total[2 * (size_t)c + 1]; }
+      for (int o = 16; o > 0; o >>= 1) {
+        rows += __shfl_xor_sync(0xffffffffu, rows, o);
+        inst += __shfl_xor_sync(0xffffffffu, inst, o);
+      }
+      if (lane == 0) {
+        // 2^32 instances or more are an error by definition: the packed base is saturated so that the row field stays
+        // intact and every write stays inside the caller's capacities (the row guard below)
+        s_base = (rows << PACK_SHIFT) | (inst < (1ull << 32) ? inst : ((1ull << 32) - 1));
+        if (tile == (n + chunk - 1) / chunk - 1) {  // last block: totals
+          rows += chunk_total[2 * (size_t)tile];
+          inst += chunk_total[2 * (size_t)tile + 1];
+          *num_rows = (uint32_t)(rows < capacity ? rows : capacity);
+          *num_instances = inst;
+          if (rows > capacity || inst >= (1ull << 32)) odin_set_error(status, ODIN_ERR_CAPACITY);
+        }
       }
     }
+    __syncthreads();
+    const uint32_t left = n - chunk_base;  // the grid has no block behind the last primitive
+    done = (int)min((uint32_t)rounds, (left + PROJECT_TILE - 1) / PROJECT_TILE);
   }
-  __syncthreads();
 
   // ---- C.  No barrier from here on: the packed prefix of (round, warp) follows from the per-warp totals of A.
   uint64_t base = s_base;
@@ -456,11 +501,13 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   const int rounds = fused ? 1 : scan_rounds_for(n, ctx->sm_count);
   const uint32_t chunk = PROJECT_TILE * (uint32_t)rounds;
   const uint32_t blocks = (n + chunk - 1) / chunk;
+  uint64_t* group_total = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + project_ws_group_offset(n));
+  uint64_t* chunk_total = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + project_ws_chunk_offset(n));
 #define LAUNCH(E, F)                                                                                                   \
   project_scan_kernel<E, F><<<blocks, SCAN_THREADS, 0, st>>>(                                                          \
       scene->means, scene->log_scales, q4, scene->opacity_logit, n, cp, rule, out->tiles_touched, out->capacity,      \
-      out->prim_id, out->tile_offset, out->num_rows, out->num_instances, ticket, state, ctx->d_status, rounds,        \
-      ctx->spin_limit, out->touched_mask)
+      out->prim_id, out->tile_offset, out->num_rows, out->num_instances, ticket, state, group_total, chunk_total,     \
+      ctx->d_status, rounds, ctx->spin_limit, out->touched_mask)
   if (fused) {
     OdinKernelScope ks(ctx, K_PROJECT, st);
     if (rule.binning == 2) LAUNCH(true, true);
@@ -468,12 +515,15 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   } else {
     {
       OdinKernelScope ks(ctx, K_PROJECT, st);
+      const uint32_t gpc = (uint32_t)rounds * (SCAN_THREADS / 32);  // counting blocks per chunk of the scan
+      unsigned long long* ct = reinterpret_cast<unsigned long long*>(chunk_total);
+      unsigned long long* gt = reinterpret_cast<unsigned long long*>(group_total);
       if (rule.binning == 2)
-        project_cull_kernel<true><<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4,
-                                                                   scene->opacity_logit, n, cp, rule, out->tiles_touched);
+        project_cull_kernel<true><<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit,
+                                                                   n, cp, rule, out->tiles_touched, gt, ct, gpc);
       else
-        project_cull_kernel<false><<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4,
-                                                                    scene->opacity_logit, n, cp, rule, out->tiles_touched);
+        project_cull_kernel<false><<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit,
+                                                                    n, cp, rule, out->tiles_touched, gt, ct, gpc);
     }
     OdinKernelScope ks(ctx, K_PROJECT_SCAN, st);
     LAUNCH(false, false);
