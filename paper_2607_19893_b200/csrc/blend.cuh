@@ -28,9 +28,11 @@ constexpr uint32_t BLEND_DONE_BIT = 0x80000000u;  // in n_contrib while a tile i
 constexpr int BLEND_TAIL_THREADS = 256;
 
 // Workspace of the render calls (every region 256-byte aligned):
-//   [256 B: u32 [0] tile ticket of the forward head kernel, [1] work ticket of the backward kernel, [2] segments taken]
+//   [256 B: u32 [0] tile ticket of the forward head kernel, [1] work ticket of the backward kernel, [2] segments taken,
+//           [3] ticket of the forward tail kernel, [4..7] tiles queued for it in each of four classes of list length]
 //   [tile_first: u32 x tiles   forward head: 1 = the tail kernel must continue; forward tail: 1 + slot of the tile's
 //                              segment that starts at entry BLEND_HEAD (0 = none)]
+//   [queue: u32 x 4 x tiles    tiles the forward tail kernel must finish, one region per class, longest lists first]
 //   [seg_tile: uint2 x S       (tile, k): the slot holds the state before entry k * BLEND_HEAD of that tile]
 //   [seg_link: uint2 x S       1 + slot of the same tile's segment k + 1, of segment k - 1 (0 = none)]
 //   [ckpt: BlendRecord x 256 x S   per pixel (thread t = 16 * row + column of the tile): T, colour to come (3)]
@@ -47,7 +49,7 @@ struct BlendRecord {
 static_assert(sizeof(BlendRecord) == 32, "record layout");
 constexpr size_t BLEND_SEG_BYTES = 8 + 8 + 256 * sizeof(BlendRecord);
 struct BlendWs {
-  size_t tile_first, seg_tile, seg_link, ckpt, total;
+  size_t tile_first, queue, seg_tile, seg_link, ckpt, total;
   uint32_t segments;
 };
 static inline size_t blend_align(size_t x) { return (x + 255) / 256 * 256; }
@@ -56,7 +58,8 @@ static inline BlendWs blend_ws_layout(int n_tiles, uint32_t segments) {
   BlendWs L;
   L.segments = segments;
   L.tile_first = BLEND_WS_HEADER;
-  L.seg_tile = L.tile_first + blend_align((size_t)n_tiles * 4);
+  L.queue = L.tile_first + blend_align((size_t)n_tiles * 4);
+  L.seg_tile = L.queue + blend_align((size_t)n_tiles * 16);
   L.seg_link = L.seg_tile + blend_align((size_t)segments * 8);
   L.ckpt = L.seg_link + blend_align((size_t)segments * 8);
   L.total = L.ckpt + (size_t)segments * 256 * sizeof(BlendRecord);

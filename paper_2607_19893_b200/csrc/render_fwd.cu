@@ -12,7 +12,7 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
                   const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX, int n_tiles,
                   float bg0, float bg1, float bg2, float alpha_min, float alpha_max, float t_min, float* __restrict__ out,
                   float* __restrict__ final_T, uint32_t* __restrict__ n_contrib, uint32_t* __restrict__ tile_more,
-                  uint32_t* __restrict__ ticket, uint32_t row_cap) {
+                  uint32_t* __restrict__ ticket, uint32_t row_cap, uint32_t* __restrict__ tail_queue) {
   __shared__ BlendRow s_row[BLEND_WARPS][32];
   __shared__ float s_blue[BLEND_WARPS][32];
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -96,7 +96,14 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
   }
   // the tail kernel takes over when entries remain and some pixel is still live
   const bool more = (rg.y > end) && __any_sync(0xffffffffu, live != 0);
-  if (lane == 0) tile_more[tile] = more ? 1u : 0u;
+  if (lane == 0) {
+    tile_more[tile] = more ? 1u : 0u;
+    if (more) {  // queue of the tail kernel, longest lists first (four classes)
+      const uint32_t len = rg.y - rg.x;
+      const uint32_t cls = len > 8 * BLEND_HEAD ? 0u : (len > 4 * BLEND_HEAD ? 1u : (len > 2 * BLEND_HEAD ? 2u : 3u));
+      tail_queue[cls * (uint32_t)n_tiles + atomicAdd(ticket + 4 + cls, 1u)] = (uint32_t)tile;
+    }
+  }
   const size_t plane = (size_t)W * H;
 #pragma unroll
   for (int s = 0; s < BLEND_SLOTS; ++s) {
@@ -125,14 +132,29 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
                        const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX,
                        float bg0, float bg1, float bg2, float alpha_min, float alpha_max, float t_min,
                        float* __restrict__ out, float* __restrict__ final_T, uint32_t* __restrict__ n_contrib,
-                       uint32_t* __restrict__ tile_first, uint32_t* __restrict__ seg_count, uint2* __restrict__ seg_tile,
+                       uint32_t* __restrict__ tile_first, uint32_t* __restrict__ header,
+                       const uint32_t* __restrict__ tail_queue, int n_tiles, uint2* __restrict__ seg_tile,
                        uint2* __restrict__ seg_link, BlendRecord* __restrict__ ckpt, uint32_t seg_cap, int* status,
                        uint32_t row_cap) {
-  const int tile = blockIdx.x;
-  if (!tile_first[tile]) return;
   __shared__ BlendRow s_row[BLEND_TAIL_THREADS];
+  __shared__ uint32_t s_item;
+  // The duration of this kernel is that of its longest list (a chain of batches), so the blocks take the tiles the head
+  // kernel queued by ticket, the class of the longest lists first.
+  const uint32_t c0 = header[4], c1 = header[5], c2 = header[6], c3 = header[7];
+  while (true) {
+  __syncthreads();  // the previous tile's readers of shared memory are done
+  if (threadIdx.x == 0) s_item = atomicAdd(header + 3, 1u);
+  __syncthreads();
+  uint32_t item = s_item;
+  if (item >= c0 + c1 + c2 + c3) return;
+  uint32_t cls = 0;
+  if (item >= c0) { item -= c0; cls = 1; if (item >= c1) { item -= c1; cls = 2; if (item >= c2) { item -= c2; cls = 3; } } }
+  const int tile = (int)min(tail_queue[cls * (uint32_t)n_tiles + item], (uint32_t)n_tiles - 1);
   __shared__ float s_blue[BLEND_TAIL_THREADS];
   __shared__ uint32_t s_ord[BLEND_TAIL_THREADS];  // 1-based position of the row in the tile's list
+  // the row's colour in double, converted once when the row is staged: the per-batch sums that feed the records are kept
+  // in double, and a conversion per (pixel, row) pair made the conversion unit the limit of tiles with long dense lists
+  __shared__ double s_cd[BLEND_TAIL_THREADS][3];
   __shared__ uint32_t s_wcnt[BLEND_TAIL_THREADS / 32];
   __shared__ uint32_t s_slot;
   const int tx = tile % TX, ty = tile / TX;
@@ -178,7 +200,7 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
     }
     const uint32_t wm = __ballot_sync(0xffffffffu, reach);
     if (lane == 0) s_wcnt[warp] = __popc(wm);
-    if (threadIdx.x == 0) s_slot = atomicAdd(seg_count, 1u);
+    if (threadIdx.x == 0) s_slot = atomicAdd(header + 2, 1u);
     __syncthreads();
     // the record of segment k: the transmittance before entry k * BLEND_HEAD (where the backward replay of segment
     // k - 1 begins) and, once the batch is done, the colour its entries added
@@ -208,6 +230,7 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
       s_row[pos] = row;
       s_blue[pos] = bp;
       s_ord[pos] = i - start + 1;
+      s_cd[pos][0] = (double)row.q0.z; s_cd[pos][1] = (double)row.q0.w; s_cd[pos][2] = (double)bp;
     }
     __syncthreads();
     if (!done) {
@@ -239,7 +262,7 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
               // the per-batch sums, in double, only feed the records
               C0 = fmaf(cr[u], w, C0); C1 = fmaf(cg[u], w, C1); C2 = fmaf(cb[u], w, C2);
               const double wd = (double)w;
-              D0 = fma((double)cr[u], wd, D0); D1 = fma((double)cg[u], wd, D1); D2 = fma((double)cb[u], wd, D2);
+              D0 = fma(s_cd[j + u][0], wd, D0); D1 = fma(s_cd[j + u][1], wd, D1); D2 = fma(s_cd[j + u][2], wd, D2);
               T = Tn;
               last = s_ord[j + u];
             }
@@ -270,6 +293,7 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
     S0 += c->S0; S1 += c->S1; S2 += c->S2;
     c->S0 = S0; c->S1 = S1; c->S2 = S2;
     s1 = seg_link[s1 - 1].y;
+  }
   }
 }
 
@@ -373,8 +397,9 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
   char* base = reinterpret_cast<char*>(ws);
   uint32_t* header = reinterpret_cast<uint32_t*>(base);
   uint32_t* tile_first = reinterpret_cast<uint32_t*>(base + L.tile_first);
+  uint32_t* tail_queue = reinterpret_cast<uint32_t*>(base + L.queue);
   cudaStream_t st = (cudaStream_t)stream;
-  ODIN_CUDA(cudaMemsetAsync(header, 0, 16, st));  // tile ticket, work ticket of the backward pass, segments taken
+  ODIN_CUDA(cudaMemsetAsync(header, 0, 32, st));  // tickets, segments taken, the four class counts of the tail queue
   {
     OdinKernelScope ks(ctx, K_FWD, st);
     const int blocks_all = (n_tiles + BLEND_WARPS - 1) / BLEND_WARPS;
@@ -383,14 +408,15 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
         reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
         reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0], cam->bg[1],
         cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_first,
-        header, proj->capacity);
+        header, proj->capacity, tail_queue);
   }
   OdinKernelScope ks(ctx, K_FWD_TAIL, st);
-  render_fwd_tail_kernel<<<n_tiles, BLEND_TAIL_THREADS, 0, st>>>(
+  const int tail_blocks = n_tiles < ctx->sm_count * 3 ? n_tiles : ctx->sm_count * 3;  // resident blocks pull tiles
+  render_fwd_tail_kernel<<<tail_blocks, BLEND_TAIL_THREADS, 0, st>>>(
       reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
       reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
-      ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_first, header + 2,
-      reinterpret_cast<uint2*>(base + L.seg_tile), reinterpret_cast<uint2*>(base + L.seg_link),
+      ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_first, header,
+      tail_queue, n_tiles, reinterpret_cast<uint2*>(base + L.seg_tile), reinterpret_cast<uint2*>(base + L.seg_link),
       reinterpret_cast<BlendRecord*>(base + L.ckpt), L.segments, ctx->d_status, proj->capacity);
   return odin_launch_status();
 }
