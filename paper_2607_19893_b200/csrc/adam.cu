@@ -84,6 +84,7 @@ adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* _
                  const float* __restrict__ g_mean, const float* __restrict__ g_ls, const float4* __restrict__ g_q,
                  const float* __restrict__ g_o, const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count,
                  uint32_t cap, AdamK k, const uint8_t* __restrict__ row_zero, uint32_t n_prims) {
+  odin_after_predecessor();  // launched behind the SH kernel (which it does not depend on: the two overlap at the seam)
   const uint32_t V = min(*count, cap);
   const size_t total = (size_t)V * 4;
   for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
@@ -256,11 +257,11 @@ extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m
   size_t gb = ((size_t)cap * 4 + 255) / 256;
   if (gb > (size_t)ctx->sm_count * 16) gb = (size_t)ctx->sm_count * 16;
   OdinKernelScope ks(ctx, K_ADAM_GEOM, st);
-  adam_geom_kernel<<<(unsigned)gb, 256, 0, st>>>(
+  ODIN_CUDA(odin_launch(ctx, true, adam_geom_kernel, dim3((unsigned)gb), dim3(256), 0, st,
       params->means, params->log_scales, reinterpret_cast<float4*>(params->quats), params->opacity_logit, m->means,
       m->log_scales, reinterpret_cast<float4*>(m->quats), m->opacity_logit, v->means, v->log_scales,
       reinterpret_cast<float4*>(v->quats), v->opacity_logit, grad_rows->means, grad_rows->log_scales,
       reinterpret_cast<const float4*>(grad_rows->quats), grad_rows->opacity_logit, d_idx, d_count, cap, k, d_row_zero,
-      params->n);
+      params->n));
   return odin_launch_status();
 }

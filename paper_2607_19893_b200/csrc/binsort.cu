@@ -107,6 +107,7 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
                 const uint32_t* __restrict__ count32, const uint64_t* __restrict__ count64, uint64_t capacity, int shift,
                 const uint32_t* __restrict__ digit_base, uint32_t* states, uint32_t* ticket, int* status,
                 int spin_limit, uint32_t depth_rows) {
+  odin_after_predecessor();  // launched behind the histogram / the pass in front
   extern __shared__ __align__(16) unsigned char os_smem[];
   uint32_t* s_keys = reinterpret_cast<uint32_t*>(os_smem);
   constexpr uint32_t TILE = (uint32_t)ITEMS * OS_THREADS;
@@ -309,6 +310,7 @@ sorted_offsets_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __
                       const uint32_t* __restrict__ num_rows, uint32_t capacity, int TX, uint32_t* __restrict__ sorted_off,
                       uint32_t* __restrict__ chunk_row, uint32_t chunks_cap, uint32_t* __restrict__ tile_diff,
                       uint32_t diff_words, uint32_t* ticket, uint64_t* state, int* status, int spin_limit) {
+  odin_after_predecessor();
   // diff_words != 0: the block first accumulates its part of the difference array in shared memory (`diff_words` =
   // tiles + 1 words of dynamic shared memory) and adds the non-zero words to the global one at the end: a tile on which
   // thousands of rectangles pile up would otherwise serialise that many global reductions on one address.
@@ -473,6 +475,7 @@ emit_instances_kernel(const uint32_t* __restrict__ sorted_off, const uint32_t* _
                       int TX, uint32_t* __restrict__ keys, uint32_t* __restrict__ vals, int* status,
                       const uint32_t* __restrict__ tile_diff, uint32_t n_tiles, int tile_passes,
                       uint32_t* __restrict__ ranges, uint32_t* __restrict__ tile_dbase) {
+  odin_after_predecessor();
   if (blockIdx.x == 0) {  // block 0: it is scheduled first
     tile_scan_block(tile_diff, n_tiles, tile_passes, ranges, tile_dbase,
                     (uint32_t)(capacity < 0xffffffffull ? capacity : 0xffffffffull));
@@ -591,6 +594,7 @@ chunk_counts_kernel(const uint32_t* __restrict__ sorted_row, const ushort4* __re
                     int TX, uint32_t n_tiles, uint32_t tiles_pad, uint32_t* __restrict__ sorted_off,
                     ushort4* __restrict__ sorted_rect, float4* __restrict__ sorted_geo4, float2* __restrict__ sorted_geo2,
                     uint32_t* __restrict__ counts, uint32_t* ticket, uint64_t* state, int* status, int spin_limit) {
+  odin_after_predecessor();
   extern __shared__ __align__(16) uint32_t s_tdiff[];  // tiles_pad + 8 words
   __shared__ uint32_t s_tile, s_base;
   __shared__ uint32_t s_warp[33];
@@ -742,6 +746,7 @@ __global__ void __launch_bounds__(TB_THREADS)
 tile_bases_kernel(uint32_t* __restrict__ counts, uint32_t tiles_pad, uint32_t n_tiles, const uint32_t* __restrict__ num_rows,
                   const uint64_t* __restrict__ num_instances, uint64_t capacity, uint32_t* tile_total,
                   uint32_t* __restrict__ ranges, uint32_t* arrivals, int* status) {
+  odin_after_predecessor();
   __shared__ uint32_t s_part[TB_PARTS][32];
   __shared__ uint32_t s_warp[33];
   __shared__ uint32_t s_flag;
@@ -843,6 +848,7 @@ scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const float4* 
                          const uint32_t* __restrict__ counts, uint32_t tiles_pad, const uint2* __restrict__ ranges,
                          uint32_t* __restrict__ vals, uint64_t* __restrict__ keys64,
                          const uint32_t* __restrict__ depth_bits) {
+  odin_after_predecessor();
   extern __shared__ __align__(16) unsigned char sc_smem[];
   ushort4* s_prect = reinterpret_cast<ushort4*>(sc_smem);                    // [SC_SUB] rectangles of the rows of the batch
   uint32_t* s_prow = reinterpret_cast<uint32_t*>(s_prect + SC_SUB);          // [SC_SUB] their row ids
@@ -1081,10 +1087,11 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
       OdinKernelScope ks(ctx, K_ROW_SORT, st);
       uint32_t* kout = (p + 1 < SORT_DEPTH_DIGITS) ? row_keys[p & 1] : nullptr;
       uint32_t* vout = row_vals[p & 1];
-      onesweep_kernel<false, OS_ROW_ITEMS, OS_ROW_WINDOW><<<grid, OS_THREADS, OS_ROW_SMEM, st>>>(
-          kin, vin, kout, vout, nullptr, nullptr, proj->num_rows, nullptr, 0, p * (int)SORT_RADIX_BITS,
-          dbase + p * SORT_RADIX, row_states + (size_t)p * row_tiles * SORT_RADIX, tickets + p, ctx->d_status,
-          ctx->spin_limit, proj->capacity);
+      ODIN_CUDA(odin_launch(ctx, true, onesweep_kernel<false, OS_ROW_ITEMS, OS_ROW_WINDOW>, dim3(grid), dim3(OS_THREADS),
+                            OS_ROW_SMEM, st, kin, vin, kout, vout, nullptr, nullptr, proj->num_rows, nullptr, 0,
+                            p * (int)SORT_RADIX_BITS, dbase + p * SORT_RADIX,
+                            row_states + (size_t)p * row_tiles * SORT_RADIX, tickets + p, ctx->d_status, ctx->spin_limit,
+                            proj->capacity));
       kin = kout;
       vin = vout;
     }
@@ -1108,19 +1115,20 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
       ODIN_CUDA(cudaFuncSetAttribute(chunk_counts_kernel<true, 1024, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      max_smem));
 #define LAUNCH_COUNTS(EXACT, THREADS, ITEMS)                                                                           \
-  chunk_counts_kernel<EXACT, THREADS, ITEMS><<<F.chunks, THREADS, smem, st>>>(                                         \
-      sorted_row, rect, reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), \
-      ctx->cfg.alpha_min, proj->num_rows, proj->num_instances, cap32, TX, n_tiles, F.tiles_pad, sorted_off, sorted_rect, \
-      geo4, geo2, counts, tickets + 8, scan_state, ctx->d_status, ctx->spin_limit)
+  ODIN_CUDA(odin_launch(ctx, true, chunk_counts_kernel<EXACT, THREADS, ITEMS>, dim3(F.chunks), dim3(THREADS), smem, st, \
+                        sorted_row, rect, reinterpret_cast<const float2*>(proj->xy),                                     \
+                        reinterpret_cast<const float4*>(proj->conic_opacity), ctx->cfg.alpha_min, proj->num_rows,        \
+                        proj->num_instances, cap32, TX, n_tiles, F.tiles_pad, sorted_off, sorted_rect, geo4, geo2,       \
+                        counts, tickets + 8, scan_state, ctx->d_status, ctx->spin_limit))
       if (exact) LAUNCH_COUNTS(true, 1024, 2);
       else LAUNCH_COUNTS(false, RO_THREADS, RO_ITEMS);
 #undef LAUNCH_COUNTS
     }
     {
       OdinKernelScope ks(ctx, K_TILE_BASES, st);
-      tile_bases_kernel<<<(n_tiles + 31) / 32, TB_THREADS, 0, st>>>(counts, F.tiles_pad, n_tiles, proj->num_rows,
-                                                                   proj->num_instances, capacity, tile_total,
-                                                                   d_tile_ranges, tickets + 10, ctx->d_status);
+      ODIN_CUDA(odin_launch(ctx, true, tile_bases_kernel, dim3((n_tiles + 31) / 32), dim3(TB_THREADS), 0, st, counts,
+                            F.tiles_pad, n_tiles, proj->num_rows, proj->num_instances, capacity, tile_total,
+                            d_tile_ranges, tickets + 10, ctx->d_status));
     }
     {
       OdinKernelScope ks(ctx, K_EMIT, st);
@@ -1136,9 +1144,10 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   do {                                                                                                                 \
     ODIN_CUDA(cudaFuncSetAttribute(scatter_instances_kernel<WIDE, EXACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
                                    (int)SC_SMEM));                                                                     \
-    scatter_instances_kernel<WIDE, EXACT><<<grid, SC_THREADS, SC_SMEM, st>>>(                                          \
-        sorted_rect, geo4, geo2, sorted_row, sorted_off, proj->num_rows, proj->num_instances, cap32, TX, TY, band_rows, \
-        counts, F.tiles_pad, reinterpret_cast<const uint2*>(d_tile_ranges), d_vals, d_keys, depth_bits);               \
+    ODIN_CUDA(odin_launch(ctx, true, scatter_instances_kernel<WIDE, EXACT>, dim3(grid), dim3(SC_THREADS), SC_SMEM, st,  \
+                          sorted_rect, geo4, geo2, sorted_row, sorted_off, proj->num_rows, proj->num_instances, cap32,  \
+                          TX, TY, band_rows, counts, F.tiles_pad, reinterpret_cast<const uint2*>(d_tile_ranges), d_vals, \
+                          d_keys, depth_bits));                                                                         \
   } while (0)
       if (d_keys) { if (exact) LAUNCH_SCATTER(true, true); else LAUNCH_SCATTER(true, false); }
       else { if (exact) LAUNCH_SCATTER(false, true); else LAUNCH_SCATTER(false, false); }
@@ -1164,19 +1173,19 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     const uint32_t diff_words = n_tiles + 1 <= 40001u ? n_tiles + 1 : 0u;
     const size_t diff_smem = (size_t)diff_words * 4;
     ODIN_CUDA(cudaFuncSetAttribute(sorted_offsets_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 40001 * 4));
-    sorted_offsets_kernel<<<(proj->capacity + OFFSET_TILE - 1) / OFFSET_TILE, RO_THREADS, diff_smem, st>>>(
-        sorted_row, rect, proj->num_rows, (uint32_t)capacity, TX, sorted_off, chunk_row, (uint32_t)chunks_cap, tile_diff,
-        diff_words, tickets + 8, scan_state, ctx->d_status, ctx->spin_limit);
+    ODIN_CUDA(odin_launch(ctx, true, sorted_offsets_kernel, dim3((proj->capacity + OFFSET_TILE - 1) / OFFSET_TILE),
+                          dim3(RO_THREADS), diff_smem, st, sorted_row, rect, proj->num_rows, (uint32_t)capacity, TX,
+                          sorted_off, chunk_row, (uint32_t)chunks_cap, tile_diff, diff_words, tickets + 8, scan_state,
+                          ctx->d_status, ctx->spin_limit));
   }
   // the emission goes to the buffers from which `tile_passes` ping-pong steps end in d_vals
   int cur = tile_passes & 1;
   {
     OdinKernelScope ks(ctx, K_EMIT, st);
     const uint32_t grid = (uint32_t)(chunks_cap < (uint64_t)sms * 5 - 1 ? chunks_cap : (uint64_t)sms * 5 - 1) + 1;
-    emit_instances_kernel<<<grid, DUP_THREADS, 0, st>>>(sorted_off, sorted_row, chunk_row, rect, proj->num_rows,
-                                                        proj->num_instances, capacity, TX, inst_keys[cur], inst_vals[cur],
-                                                        ctx->d_status, tile_diff, n_tiles, tile_passes, d_tile_ranges,
-                                                        tile_dbase);
+    ODIN_CUDA(odin_launch(ctx, true, emit_instances_kernel, dim3(grid), dim3(DUP_THREADS), 0, st, sorted_off, sorted_row,
+                          chunk_row, rect, proj->num_rows, proj->num_instances, capacity, TX, inst_keys[cur], inst_vals[cur],
+                          ctx->d_status, tile_diff, n_tiles, tile_passes, d_tile_ranges, tile_dbase));
   }
   // ---- instances by tile id
   const uint32_t os_grid = L.tiles < sms * OS_BLOCKS ? L.tiles : sms * OS_BLOCKS;
@@ -1184,15 +1193,17 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     OdinKernelScope ks(ctx, K_ONESWEEP, st);
     uint32_t* states = inst_states + (size_t)p * L.tiles * SORT_RADIX;
     if (p + 1 < tile_passes)
-      onesweep_kernel<false, OS_INST_ITEMS, OS_INST_WINDOW><<<os_grid, OS_THREADS, OS_SMEM, st>>>(
-          inst_keys[cur], inst_vals[cur], inst_keys[cur ^ 1], inst_vals[cur ^ 1], nullptr, nullptr, nullptr,
-          proj->num_instances, capacity, p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
-          tickets + SORT_DEPTH_DIGITS + p, ctx->d_status, ctx->spin_limit, proj->capacity);
+      ODIN_CUDA(odin_launch(ctx, true, onesweep_kernel<false, OS_INST_ITEMS, OS_INST_WINDOW>, dim3(os_grid),
+                            dim3(OS_THREADS), OS_SMEM, st, inst_keys[cur], inst_vals[cur], inst_keys[cur ^ 1],
+                            inst_vals[cur ^ 1], nullptr, nullptr, nullptr, proj->num_instances, capacity,
+                            p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
+                            tickets + SORT_DEPTH_DIGITS + p, ctx->d_status, ctx->spin_limit, proj->capacity));
     else  // the sorted tile ids themselves are not needed any more: the ranges came from the tile counts
-      onesweep_kernel<true, OS_INST_ITEMS, OS_INST_WINDOW><<<os_grid, OS_THREADS, OS_SMEM, st>>>(
-          inst_keys[cur], inst_vals[cur], nullptr, inst_vals[cur ^ 1], d_keys, depth_bits, nullptr,
-          proj->num_instances, capacity, p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
-          tickets + SORT_DEPTH_DIGITS + p, ctx->d_status, ctx->spin_limit, proj->capacity);
+      ODIN_CUDA(odin_launch(ctx, true, onesweep_kernel<true, OS_INST_ITEMS, OS_INST_WINDOW>, dim3(os_grid),
+                            dim3(OS_THREADS), OS_SMEM, st, inst_keys[cur], inst_vals[cur], nullptr, inst_vals[cur ^ 1],
+                            d_keys, depth_bits, nullptr, proj->num_instances, capacity, p * (int)SORT_RADIX_BITS,
+                            tile_dbase + p * SORT_RADIX, states, tickets + SORT_DEPTH_DIGITS + p, ctx->d_status,
+                            ctx->spin_limit, proj->capacity));
     cur ^= 1;
   }
   return odin_launch_status();

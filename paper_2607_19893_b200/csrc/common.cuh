@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
 #include <vector>
 
 #include "../../include/odin.h"
@@ -59,6 +60,30 @@ struct OdinKernelScope {
     if (rec) cudaEventRecord(ctx->prof.events[2 * slot + 1], st);
   }
 };
+
+// Programmatic dependent launch.  A kernel that calls odin_after_predecessor() as its first statement may be launched
+// with odin_launch(dependent = true, ...) right behind another kernel of the same call on the same stream: its blocks
+// are then scheduled while the kernel in front drains (once every block of that kernel has started) and wait here
+// until it has completed and its writes are visible, so the ~3.5 us between two dependent launches are not spent idle.
+// Nothing is read or written before the wait, so ordering is exactly that of a plain launch; without a programmatic
+// predecessor both instructions do nothing.  `dependent` must be false unless the operation in front on the stream is
+// a kernel launched by the same call; it is also dropped while per-kernel events are recorded.
+__device__ __forceinline__ void odin_after_predecessor() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+static inline cudaError_t odin_launch(const odin_ctx* ctx, bool dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block,
+                                      size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = grid; lc.blockDim = block; lc.dynamicSmemBytes = smem; lc.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at;
+  lc.numAttrs = (dependent && !ctx->prof.enabled) ? 1 : 0;
+  return cudaLaunchKernelEx(&lc, kernel, std::forward<Args>(args)...);
+}
 
 #define ODIN_CUDA(call)                          \
   do {                                           \

@@ -202,6 +202,7 @@ project_scan_kernel(const float* __restrict__ means, const float* __restrict__ l
                     uint64_t* __restrict__ num_instances, uint32_t* ticket, uint64_t* state,
                     const uint64_t* __restrict__ group_total, const uint64_t* __restrict__ chunk_total, int* status,
                     int rounds, int spin_limit, uint32_t* __restrict__ touched_mask) {
+  odin_after_predecessor();  // not fused: launched behind the counting kernel
   __shared__ uint32_t s_tile;
   __shared__ uint64_t s_warp[SCAN_THREADS / 32];
   __shared__ uint64_t s_inst[SCAN_THREADS / 32];
@@ -413,6 +414,7 @@ __global__ void __launch_bounds__(128)
 project_rows_kernel(const float* __restrict__ means, const float* __restrict__ log_scales, const float4* __restrict__ quats,
                     const float* __restrict__ opacity_logit, const float* __restrict__ sh, CamParams cam, BinRule rule,
                     odin_projected out, uint32_t n) {
+  odin_after_predecessor();
   constexpr int K = (DEG + 1) * (DEG + 1);
   const uint32_t V = min(*out.num_rows, out.capacity);
   for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
@@ -504,10 +506,10 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   uint64_t* group_total = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + project_ws_group_offset(n));
   uint64_t* chunk_total = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + project_ws_chunk_offset(n));
 #define LAUNCH(E, F)                                                                                                   \
-  project_scan_kernel<E, F><<<blocks, SCAN_THREADS, 0, st>>>(                                                          \
-      scene->means, scene->log_scales, q4, scene->opacity_logit, n, cp, rule, out->tiles_touched, out->capacity,      \
-      out->prim_id, out->tile_offset, out->num_rows, out->num_instances, ticket, state, group_total, chunk_total,     \
-      ctx->d_status, rounds, ctx->spin_limit, out->touched_mask)
+  ODIN_CUDA(odin_launch(ctx, !(F), project_scan_kernel<E, F>, dim3(blocks), dim3(SCAN_THREADS), 0, st, scene->means,   \
+                        scene->log_scales, q4, scene->opacity_logit, n, cp, rule, out->tiles_touched, out->capacity,   \
+                        out->prim_id, out->tile_offset, out->num_rows, out->num_instances, ticket, state, group_total, \
+                        chunk_total, ctx->d_status, rounds, ctx->spin_limit, out->touched_mask))
   if (fused) {
     OdinKernelScope ks(ctx, K_PROJECT, st);
     if (rule.binning == 2) LAUNCH(true, true);
@@ -534,8 +536,8 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   const uint32_t grid = blocks_cap < (uint32_t)ctx->sm_count * 16 ? blocks_cap : (uint32_t)ctx->sm_count * 16;
   OdinKernelScope ks(ctx, K_PROJECT_ROWS, st);
 #define LAUNCH(D)                                                                                                      \
-  project_rows_kernel<D><<<grid, 128, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit, scene->sh, cp, \
-                                               rule, *out, n)
+  ODIN_CUDA(odin_launch(ctx, true, project_rows_kernel<D>, dim3(grid), dim3(128), 0, st, scene->means,                 \
+                        scene->log_scales, q4, scene->opacity_logit, scene->sh, cp, rule, *out, n))
   switch (scene->sh_degree) {
     case 0: LAUNCH(0); break;
     case 1: LAUNCH(1); break;

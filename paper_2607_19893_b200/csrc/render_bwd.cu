@@ -56,6 +56,7 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
                         const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
                         const float* __restrict__ dL, float* __restrict__ g2d, uint32_t* __restrict__ ticket,
                         uint8_t* __restrict__ row_active, uint32_t row_cap) {
+  odin_after_predecessor();  // launched behind zero_rows_kernel
   __shared__ BlendRow s_rowdata[BLEND_WARPS][32];
   __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, 1 / opacity
   __shared__ uint32_t s_rowid[BLEND_WARPS][32];
@@ -224,6 +225,7 @@ render_bwd_project_kernel(const float* __restrict__ means, const float* __restri
                           const float* __restrict__ g2d, float* __restrict__ g_means, float* __restrict__ g_ls,
                           float4* __restrict__ g_quats, float* __restrict__ g_opac, float* __restrict__ g_sh,
                           uint8_t* __restrict__ row_zero, uint32_t n) {
+  odin_after_predecessor();
   constexpr int K = (DEG + 1) * (DEG + 1);
   const uint32_t V = min(*num_rows, capacity);
   for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < V; r += gridDim.x * blockDim.x) {
@@ -397,30 +399,30 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
   cudaStream_t st = (cudaStream_t)stream;
   const int TX = (cam->width + 15) / 16, TY = (cam->height + 15) / 16;
   if (!ws || !odin_aligned(ws, 256) || ws_bytes < blend_ws_bytes(cam->width, cam->height)) return ODIN_ERR_WORKSPACE;
-  const uint32_t zgrid = (uint32_t)ctx->sm_count * 8;
-  {
-    OdinKernelScope ks(ctx, K_ZERO_ROWS, st);
-    zero_rows_kernel<<<zgrid, 256, 0, st>>>(d_grad2d, d_row_active, proj->num_rows, proj->capacity);
-  }
   const int n_tiles = TX * TY;
   const BlendWs L = blend_ws_layout(n_tiles, blend_ws_segments(n_tiles, ws_bytes));
   char* base = reinterpret_cast<char*>(ws);
   uint32_t* header = reinterpret_cast<uint32_t*>(base);
   uint32_t* ticket = header + 1;
-  ODIN_CUDA(cudaMemsetAsync(ticket, 0, 4, st));
+  ODIN_CUDA(cudaMemsetAsync(ticket, 0, 4, st));  // in front of all three kernels: they are launched back to back
+  const uint32_t zgrid = (uint32_t)ctx->sm_count * 8;
+  {
+    OdinKernelScope ks(ctx, K_ZERO_ROWS, st);
+    zero_rows_kernel<<<zgrid, 256, 0, st>>>(d_grad2d, d_row_active, proj->num_rows, proj->capacity);
+  }
   {
     OdinKernelScope ks(ctx, K_BWD_BLEND, st);
     const size_t blocks_all = ((size_t)n_tiles + L.segments + BLEND_WARPS - 1) / BLEND_WARPS;
     const int blocks = blocks_all < (size_t)ctx->sm_count * 8 ? (int)blocks_all : ctx->sm_count * 8;  // resident warps pull work
 #define LAUNCH_BLEND(TRACK)                                                                                             \
-  render_bwd_blend_kernel<TRACK><<<blocks, BLEND_THREADS, 0, st>>>(                                                     \
+  ODIN_CUDA(odin_launch(ctx, true, render_bwd_blend_kernel<TRACK>, dim3(blocks), dim3(BLEND_THREADS), 0, st,            \
       reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb,       \
       d_vals, reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0],          \
       cam->bg[1], cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max,                                                   \
       reinterpret_cast<const uint32_t*>(base + L.tile_first), header + 2,                                               \
       reinterpret_cast<const uint2*>(base + L.seg_tile), reinterpret_cast<const uint2*>(base + L.seg_link),             \
       reinterpret_cast<const BlendRecord*>(base + L.ckpt), L.segments, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d, ticket,  \
-      d_row_active, proj->capacity)
+      d_row_active, proj->capacity))
     if (d_row_active) LAUNCH_BLEND(true);
     else LAUNCH_BLEND(false);
 #undef LAUNCH_BLEND
@@ -429,11 +431,11 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
   const uint32_t blocks_cap = (proj->capacity + 127) / 128;
   const uint32_t pgrid = blocks_cap < (uint32_t)ctx->sm_count * 16 ? blocks_cap : (uint32_t)ctx->sm_count * 16;
 #define LAUNCH(D)                                                                                                       \
-  render_bwd_project_kernel<D><<<pgrid, 128, 0, st>>>(                                                                  \
+  ODIN_CUDA(odin_launch(ctx, true, render_bwd_project_kernel<D>, dim3(pgrid), dim3(128), 0, st,                         \
       scene->means, scene->log_scales, reinterpret_cast<const float4*>(scene->quats), scene->opacity_logit, scene->sh,  \
       cp, ctx->cfg.dilation, proj->prim_id, proj->clamp_flags, proj->num_rows, proj->capacity, d_grad2d,                \
       grad_rows->means, grad_rows->log_scales, reinterpret_cast<float4*>(grad_rows->quats), grad_rows->opacity_logit,    \
-      grad_rows->sh, d_row_zero, scene->n)
+      grad_rows->sh, d_row_zero, scene->n))
   OdinKernelScope ks(ctx, K_BWD_PROJECT, st);
   switch (scene->sh_degree) {
     case 0: LAUNCH(0); break;

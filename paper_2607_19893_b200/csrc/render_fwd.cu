@@ -136,6 +136,7 @@ render_fwd_tail_kernel(const float2* __restrict__ xy, const float4* __restrict__
                        const uint32_t* __restrict__ tail_queue, int n_tiles, uint2* __restrict__ seg_tile,
                        uint2* __restrict__ seg_link, BlendRecord* __restrict__ ckpt, uint32_t seg_cap, int* status,
                        uint32_t row_cap) {
+  odin_after_predecessor();  // launched behind the head kernel
   __shared__ BlendRow s_row[BLEND_TAIL_THREADS];
   __shared__ uint32_t s_item;
   // The duration of this kernel is that of its longest list (a chain of batches), so the blocks take the tiles the head
@@ -412,12 +413,12 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
   }
   OdinKernelScope ks(ctx, K_FWD_TAIL, st);
   const int tail_blocks = n_tiles < ctx->sm_count * 3 ? n_tiles : ctx->sm_count * 3;  // resident blocks pull tiles
-  render_fwd_tail_kernel<<<tail_blocks, BLEND_TAIL_THREADS, 0, st>>>(
+  ODIN_CUDA(odin_launch(ctx, true, render_fwd_tail_kernel, dim3(tail_blocks), dim3(BLEND_TAIL_THREADS), 0, st,
       reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
       reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, cam->bg[0], cam->bg[1], cam->bg[2],
       ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_first, header,
       tail_queue, n_tiles, reinterpret_cast<uint2*>(base + L.seg_tile), reinterpret_cast<uint2*>(base + L.seg_link),
-      reinterpret_cast<BlendRecord*>(base + L.ckpt), L.segments, ctx->d_status, proj->capacity);
+      reinterpret_cast<BlendRecord*>(base + L.ckpt), L.segments, ctx->d_status, proj->capacity));
   return odin_launch_status();
 }
 
