@@ -91,8 +91,8 @@ constexpr size_t os_smem_bytes(int items) {
 }
 
 // One pass over one 8-bit digit of 32-bit keys.  Persistent blocks take 4096-key tiles by ticket.  Per tile:
-// warp-striped loads, per-warp digit ranking with match.any (stable), block digit counts published for look-back,
-// exclusive global digit offsets by a per-digit look-back walk (thread d walks digit d), keys and values exchanged
+// warp-striped loads, per-warp digit ranking (stable; match.any, or eight ballots in the passes over the rows), block
+// digit counts published for look-back, exclusive global digit offsets by a per-digit look-back walk (thread d walks digit d), keys and values exchanged
 // through shared memory so that the global scatter writes runs of consecutive addresses.
 //   vals_in == nullptr: the values are the positions themselves (first pass over the rows)
 //   keys_out == nullptr: the keys are not needed afterwards (last pass over the rows)
