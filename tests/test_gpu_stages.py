@@ -284,6 +284,37 @@ def test_bin_sort_exact_binning(oracle32):
         tr.close()
 
 
+def test_project_large_scene_two_kernels(oracle32):
+    """Scenes of more than 2048 x 4 x 148 primitives do not take the fused kernel: a counting kernel (one thread per
+    primitive, leaving packed totals per 256 primitives and exact totals per chunk) and a scan that starts from a sum
+    over the chunks in front of it.  A ragged count just above the limit, both the rectangle rule and exact binning, the
+    touched bitmask as a by-product, and truncation at the row capacity."""
+    n = 2048 * 4 * 148 + 2048 * 3 + 77
+    w = wl.make_workload(5, n=n, n_cameras=4)
+    cam = w.cameras[1]
+    v = check_projection(oracle32, w.scene, cam)
+    assert 0 < v < 0.2 * n
+    check_projection(exact_oracle(), w.scene, cam, cfg=B.default_config(binning=2))
+    # the bitmask written by the scan, and row-capacity truncation, on this path
+    tr = G.trainer_for(w.scene, cam, row_capacity=v // 2)
+    words = (n + 31) // 32
+    mask = torch.full((words + 8,), -1, dtype=torch.int32, device=tr.device)
+    tr.proj.struct.touched_mask = mask[4:].data_ptr()
+    tr.proj.prim_id.fill_(-1)
+    tr.project(B.make_camera(cam))
+    assert tr.poll() == B.ODIN_ERR_CAPACITY
+    assert int(tr.proj.num_rows.item()) == v // 2
+    tt = G.u32(tr.proj.tiles_touched)[:n]
+    want = np.flatnonzero(tt)
+    assert len(want) == v
+    assert np.array_equal(G.u32(tr.proj.prim_id)[: v // 2], want[: v // 2])
+    bits = np.unpackbits(G.u32(mask[4:4 + words]).view(np.uint8), bitorder="little")[:n]
+    assert np.array_equal(bits, (tt > 0).astype(np.uint8))
+    assert (mask[:4] == -1).all() and (mask[4 + words:] == -1).all()
+    tr.proj.struct.touched_mask = None
+    tr.close()
+
+
 def test_project_row_capacity_overflow(oracle32):
     w = wl.make_workload(1)
     tr = G.trainer_for(w.scene, w.cameras[0], row_capacity=100)
