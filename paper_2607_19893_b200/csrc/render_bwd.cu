@@ -55,7 +55,8 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
                         const BlendRecord* __restrict__ ckpt, uint32_t seg_cap,
                         const float* __restrict__ final_T, const uint32_t* __restrict__ n_contrib,
                         const float* __restrict__ dL, float* __restrict__ g2d, uint32_t* __restrict__ ticket,
-                        uint8_t* __restrict__ row_active, uint32_t row_cap) {
+                        uint8_t* __restrict__ row_active, uint32_t row_cap, const uint32_t* __restrict__ bwd_count,
+                        const uint32_t* __restrict__ bwd_queue) {
   odin_after_predecessor();  // launched behind zero_rows_kernel
   __shared__ BlendRow s_rowdata[BLEND_WARPS][32];
   __shared__ float2 s_blue[BLEND_WARPS][32];  // blue, 1 / opacity
@@ -75,8 +76,13 @@ render_bwd_blend_kernel(const float2* __restrict__ xy, const float4* __restrict_
     const uint2 st = seg_tile[item];
     tile = (int)st.x; seg = st.y; next = seg_link[item].x;
   } else {
-    if (item - n_seg >= (uint32_t)n_tiles) return;
-    tile = (int)(item - n_seg);
+    uint32_t pos = item - n_seg;
+    if (pos >= (uint32_t)n_tiles) return;
+    // the tiles in the order the forward pass filed them: classes of walked length, longest first (the class counts
+    // add up to the number of tiles; whatever else the words hold, pos stays below it and the tile is clamped)
+    uint32_t cls = 0;
+    while (cls + 1 < (uint32_t)BLEND_BWD_CLASSES && pos >= bwd_count[cls]) { pos -= bwd_count[cls]; ++cls; }
+    tile = (int)min(bwd_queue[cls * (uint32_t)n_tiles + min(pos, (uint32_t)n_tiles - 1)], (uint32_t)n_tiles - 1);
     next = tile_first[tile];
   }
   // a workspace that is not the forward call's own must not lead anywhere: records are checked before use
@@ -422,7 +428,7 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
       reinterpret_cast<const uint32_t*>(base + L.tile_first), header + 2,                                               \
       reinterpret_cast<const uint2*>(base + L.seg_tile), reinterpret_cast<const uint2*>(base + L.seg_link),             \
       reinterpret_cast<const BlendRecord*>(base + L.ckpt), L.segments, d_final_T, d_n_contrib, d_dL_drgb, d_grad2d, ticket,  \
-      d_row_active, proj->capacity))
+      d_row_active, proj->capacity, header + 8, reinterpret_cast<const uint32_t*>(base + L.bwd_queue)))
     if (d_row_active) LAUNCH_BLEND(true);
     else LAUNCH_BLEND(false);
 #undef LAUNCH_BLEND

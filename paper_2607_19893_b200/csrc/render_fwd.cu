@@ -12,7 +12,8 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
                   const uint32_t* __restrict__ vals, const uint2* __restrict__ ranges, int W, int H, int TX, int n_tiles,
                   float bg0, float bg1, float bg2, float alpha_min, float alpha_max, float t_min, float* __restrict__ out,
                   float* __restrict__ final_T, uint32_t* __restrict__ n_contrib, uint32_t* __restrict__ tile_more,
-                  uint32_t* __restrict__ ticket, uint32_t row_cap, uint32_t* __restrict__ tail_queue) {
+                  uint32_t* __restrict__ ticket, uint32_t row_cap, uint32_t* __restrict__ tail_queue,
+                  uint32_t* __restrict__ bwd_queue) {
   __shared__ BlendRow s_row[BLEND_WARPS][32];
   __shared__ float s_blue[BLEND_WARPS][32];
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -43,6 +44,7 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
     if (px < W && py0 + 2 * s < H) live |= 1u << s;
   }
   const uint32_t inside = live;
+  uint32_t n_eval = 0;  // rows evaluated for this tile: the class of its first segment in the backward pass
 
   for (uint32_t b = start; b < end; b += 32) {
     if (!__any_sync(0xffffffffu, live != 0)) break;
@@ -62,6 +64,7 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
     }
     // warp-uniform: only the rows whose ellipse reaches the tile are evaluated, in list order
     uint32_t rows = __ballot_sync(0xffffffffu, reach);
+    n_eval += __popc(rows);
     __syncwarp();
     while (rows) {
       const int j = __ffs(rows) - 1;
@@ -97,6 +100,8 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
   // the tail kernel takes over when entries remain and some pixel is still live
   const bool more = (rg.y > end) && __any_sync(0xffffffffu, live != 0);
   if (lane == 0) {
+    const uint32_t bc = blend_bwd_class(n_eval);
+    bwd_queue[bc * (uint32_t)n_tiles + atomicAdd(ticket + 8 + bc, 1u)] = (uint32_t)tile;
     tile_more[tile] = more ? 1u : 0u;
     if (more) {  // queue of the tail kernel, longest lists first (four classes)
       const uint32_t len = rg.y - rg.x;
@@ -400,7 +405,7 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
   uint32_t* tile_first = reinterpret_cast<uint32_t*>(base + L.tile_first);
   uint32_t* tail_queue = reinterpret_cast<uint32_t*>(base + L.queue);
   cudaStream_t st = (cudaStream_t)stream;
-  ODIN_CUDA(cudaMemsetAsync(header, 0, 32, st));  // tickets, segments taken, the four class counts of the tail queue
+  ODIN_CUDA(cudaMemsetAsync(header, 0, 96, st));  // tickets, segments taken, the class counts of the two queues
   {
     OdinKernelScope ks(ctx, K_FWD, st);
     const int blocks_all = (n_tiles + BLEND_WARPS - 1) / BLEND_WARPS;
@@ -409,7 +414,7 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
         reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
         reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0], cam->bg[1],
         cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_first,
-        header, proj->capacity, tail_queue);
+        header, proj->capacity, tail_queue, reinterpret_cast<uint32_t*>(base + L.bwd_queue));
   }
   OdinKernelScope ks(ctx, K_FWD_TAIL, st);
   const int tail_blocks = n_tiles < ctx->sm_count * 3 ? n_tiles : ctx->sm_count * 3;  // resident blocks pull tiles
