@@ -847,7 +847,7 @@ scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const float4* 
                          const uint64_t* __restrict__ num_instances, uint32_t capacity, int TX, int TY, int band_rows,
                          const uint32_t* __restrict__ counts, uint32_t tiles_pad, const uint2* __restrict__ ranges,
                          uint32_t* __restrict__ vals, uint64_t* __restrict__ keys64,
-                         const uint32_t* __restrict__ depth_bits) {
+                         const uint32_t* __restrict__ depth_bits, uint32_t* __restrict__ item_ticket) {
   odin_after_predecessor();
   extern __shared__ __align__(16) unsigned char sc_smem[];
   ushort4* s_prect = reinterpret_cast<ushort4*>(sc_smem);                    // [SC_SUB] rectangles of the rows of the batch
@@ -862,7 +862,14 @@ scatter_instances_kernel(const ushort4* __restrict__ sorted_rect, const float4* 
   const uint32_t nbands = ((uint32_t)TY + band_rows - 1) / band_rows;
   const uint32_t items = nchunks * nbands;
   const bool cut = *num_instances > (uint64_t)capacity;  // only then can a row be denied some of its instances
-  for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
+  __shared__ uint32_t s_item;
+  while (true) {
+    // items by ticket (they differ in cost by the number of rows of the chunk that meet the band)
+    __syncthreads();
+    if (threadIdx.x == 0) s_item = atomicAdd(item_ticket, 1u);
+    __syncthreads();
+    const uint32_t item = s_item;
+    if (item >= items) break;
     const uint32_t chunk = item / nbands, band = item - chunk * nbands;  // neighbouring blocks share a chunk's rows
     const uint32_t by0 = band * band_rows, by1 = min((uint32_t)TY, by0 + band_rows);
     const uint32_t band_tiles = (by1 - by0) * (uint32_t)TX;
@@ -1147,7 +1154,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     ODIN_CUDA(odin_launch(ctx, true, scatter_instances_kernel<WIDE, EXACT>, dim3(grid), dim3(SC_THREADS), SC_SMEM, st,  \
                           sorted_rect, geo4, geo2, sorted_row, sorted_off, proj->num_rows, proj->num_instances, cap32,  \
                           TX, TY, band_rows, counts, F.tiles_pad, reinterpret_cast<const uint2*>(d_tile_ranges), d_vals, \
-                          d_keys, depth_bits));                                                                         \
+                          d_keys, depth_bits, tickets + 11));                                                           \
   } while (0)
       if (d_keys) { if (exact) LAUNCH_SCATTER(true, true); else LAUNCH_SCATTER(true, false); }
       else { if (exact) LAUNCH_SCATTER(false, true); else LAUNCH_SCATTER(false, false); }
