@@ -5,9 +5,9 @@
 
 constexpr uint32_t PROJECT_TILE = 2048;   // primitives per look-back tile of the projection scan
 constexpr uint32_t TOUCHED_TILE = 2048;   // primitives per look-back tile of the touched-set kernel
-// The two scan kernels give every block `rounds` x 2048 primitives and one look-back (states are sized for
-// 2048-primitive tiles, which is always enough).  More rounds = a shorter chain of dependent tiles; fewer = more
-// blocks.  Aim at about four blocks per SM, at most 8 rounds.
+// The scan kernels (touched set; projection of scenes too large for its fused kernel) give every block `rounds` x 2048
+// primitives (look-back states are sized for 2048-primitive tiles, which is always enough).  More rounds = fewer
+// dependent tiles / chunk totals to sum; fewer = more blocks.  Aim at about four blocks per SM, at most 8 rounds.
 static inline int scan_rounds_for(uint32_t n, int sm_count) {
   const uint64_t r = (uint64_t)n / ((uint64_t)2048 * (uint64_t)sm_count * 4);
   return r < 1 ? 1 : (r > 8 ? 8 : (int)r);
