@@ -132,6 +132,17 @@ const char* odin_status_string(int status);
  * clears it. */
 int odin_poll(odin_ctx* ctx, void* stream);
 
+/* Chained calls.  Between odin_chain_begin and odin_chain_end the caller promises to enqueue NOTHING but calls of this
+ * library with this context on one stream (no copies, memsets, event waits or kernels of its own in between).  The
+ * library then launches the first kernel of a call as a programmatic dependent of the last kernel of the call before it
+ * (it is scheduled while that one drains and starts with griddepcontrol.wait, so the order of all memory operations is
+ * unchanged) and zeroes its scratch words with a small kernel of the same kind instead of a memset.  Results are those
+ * of unchained calls; only the idle time at the seams between calls goes (about 3 us each).  Calls that enqueue a copy
+ * or memset themselves (odin_poll, the scope calls) are allowed inside a chain and simply interrupt it.  Host-side
+ * state of the context: not thread safe. */
+int odin_chain_begin(odin_ctx* ctx);
+int odin_chain_end(odin_ctx* ctx);
+
 /* Number of unsuccessful polls after which a device-side wait of this context's later calls gives up (the look-back of
  * the prefix scans and of the radix sort waits for a word another thread block publishes).  Default 2^22, far beyond
  * anything a healthy launch needs.  A wait that gives up defers ODIN_ERR_TIMEOUT, the kernel carries on with clamped

@@ -25,7 +25,7 @@ ODIN_ERR_UNSUPPORTED = -7
 
 EXPORTS = [
     "odin_create", "odin_destroy", "odin_status_string", "odin_poll", "odin_workspace_bytes", "odin_project",
-    "odin_touched_set", "odin_bin_sort", "odin_render_fwd", "odin_l1_loss", "odin_render_bwd", "odin_sparse_adam",
+    "odin_touched_set", "odin_bin_sort", "odin_render_fwd", "odin_l1_loss", "odin_chain_begin", "odin_chain_end", "odin_render_bwd", "odin_sparse_adam",
     "odin_conflict_count", "odin_kernel_count", "odin_kernel_name", "odin_profile_enable", "odin_profile_collect",
     "odin_touched_set_static", "odin_render_workspace_bytes", "odin_active_set", "odin_mask_union", "odin_hazard_count",
     "odin_delayed_read_gate", "odin_rlg_weights", "odin_rlg_topk", "odin_sds_scores", "odin_set_wait_limit",
@@ -106,6 +106,8 @@ def lib() -> C.CDLL:
         L.odin_render_fwd.argtypes = [vp, C.POINTER(odin_projected), vp, vp, C.POINTER(odin_camera), vp, vp, vp, vp,
                                       C.c_size_t, vp]
         L.odin_l1_loss.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
+        L.odin_chain_begin.argtypes = [vp]
+        L.odin_chain_end.argtypes = [vp]
         L.odin_render_bwd.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_camera), C.POINTER(odin_projected), vp, vp,
                                       vp, vp, vp, vp, C.POINTER(odin_scene), vp, vp, vp, C.c_size_t, vp]
         L.odin_sparse_adam.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_scene), C.POINTER(odin_scene),
@@ -272,6 +274,14 @@ def odin_render_fwd(ctx, proj: odin_projected, d_vals, d_tile_ranges, cam: odin_
     _check(lib().odin_render_fwd(ctx, C.byref(proj), _ptr(d_vals), _ptr(d_tile_ranges), C.byref(cam), _ptr(d_rgb),
                                  _ptr(d_final_T), _ptr(d_n_contrib), _ptr(ws),
                                  0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)), "odin_render_fwd")
+
+
+def odin_chain_begin(ctx) -> None:
+    _check(lib().odin_chain_begin(ctx), "odin_chain_begin")
+
+
+def odin_chain_end(ctx) -> None:
+    _check(lib().odin_chain_end(ctx), "odin_chain_end")
 
 
 def odin_render_workspace_bytes(ctx, width: int, height: int) -> int:

@@ -38,6 +38,7 @@ __global__ void __launch_bounds__(256)
 adam_sh_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v, const float* __restrict__ g,
                const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count, uint32_t cap, AdamK k,
                const uint8_t* __restrict__ row_zero, uint32_t n_prims) {
+  odin_after_predecessor();
   constexpr int EPR = ROWF / VEC;  // elements per row
   const uint32_t V = min(*count, cap);
   const size_t total = (size_t)V * EPR;
@@ -248,10 +249,10 @@ extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m
   {
     OdinKernelScope ks(ctx, K_ADAM_SH, st);
     switch (params->sh_degree) {
-    case 0: adam_sh_kernel<3, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n); break;
-    case 1: adam_sh_kernel<12, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n); break;
-    case 2: adam_sh_kernel<27, 1><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n); break;
-    default: adam_sh_kernel<48, 4><<<gsh, 256, 0, st>>>(params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n); break;
+    case 0: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<3, 1>, dim3(gsh), dim3(256), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n)); break;
+    case 1: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<12, 4>, dim3(gsh), dim3(256), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n)); break;
+    case 2: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<27, 1>, dim3(gsh), dim3(256), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n)); break;
+    default: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<48, 4>, dim3(gsh), dim3(256), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n)); break;
     }
   }
   size_t gb = ((size_t)cap * 4 + 255) / 256;

@@ -32,6 +32,7 @@ extern "C" int odin_create(odin_ctx** out, int device, const odin_config* cfg) {
   }
   ctx->sm_count = prop.multiProcessorCount;
   ctx->spin_limit = ODIN_DEFAULT_SPIN_LIMIT;
+  ctx->chain = 0;
   *ctx->h_status = 0;
   *out = ctx;
   return ODIN_OK;
@@ -77,6 +78,7 @@ extern "C" const char* odin_status_string(int s) {
 extern "C" int odin_poll(odin_ctx* ctx, void* stream) {
   if (!ctx) return ODIN_ERR_NULL;
   cudaStream_t st = (cudaStream_t)stream;
+  odin_chain_break(ctx);
   ODIN_CUDA(cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
   ODIN_CUDA(cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st));
   ODIN_CUDA(cudaStreamSynchronize(st));
@@ -90,7 +92,19 @@ static const char* const kKernelNames[K_COUNT] = {
     "zero_rows", "render_bwd_blend", "render_bwd_project", "adam_sh", "adam_geom", "conflict_count",
     "render_fwd_tail", "project_scan", "project_rows", "row_hist",
     "row_sort_pass", "row_offsets", "active_set", "mask_union", "hazard_count", "delayed_read_gate",
-    "locality_graph", "tile_bases", "accumulate_rows"};
+    "locality_graph", "tile_bases", "accumulate_rows", "zero_words"};
+
+extern "C" int odin_chain_begin(odin_ctx* ctx) {
+  if (!ctx) return ODIN_ERR_NULL;
+  ctx->chain = 1;
+  return ODIN_OK;
+}
+
+extern "C" int odin_chain_end(odin_ctx* ctx) {
+  if (!ctx) return ODIN_ERR_NULL;
+  ctx->chain = 0;
+  return ODIN_OK;
+}
 
 extern "C" int odin_kernel_count(void) { return K_COUNT; }
 

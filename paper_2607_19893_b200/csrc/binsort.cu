@@ -38,6 +38,7 @@ __device__ __forceinline__ void last_block_digit_bases(const uint32_t* hist, uin
 __global__ void __launch_bounds__(256)
 row_hist_kernel(const uint32_t* __restrict__ depth_bits, const uint32_t* __restrict__ num_rows, uint32_t* __restrict__ hist,
                 uint32_t* __restrict__ base, uint32_t* arrivals) {
+  odin_after_predecessor();
   __shared__ uint32_t s_hist[SORT_DEPTH_DIGITS][SORT_RADIX];
   __shared__ uint32_t s_warp[33], s_flag;
   for (int i = threadIdx.x; i < SORT_DEPTH_DIGITS * (int)SORT_RADIX; i += 256) (&s_hist[0][0])[i] = 0;
@@ -1032,6 +1033,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   const uint32_t n_tiles = (uint32_t)TX * (uint32_t)TY;
   if (!odin_aligned(d_tile_ranges, 8)) return ODIN_ERR_INVALID_ARG;
   if (capacity == 0 || proj->capacity == 0) {
+    odin_chain_break(ctx);
     ODIN_CUDA(cudaMemsetAsync(d_tile_ranges, 0, (size_t)n_tiles * 8, st));
     return ODIN_OK;
   }
@@ -1054,11 +1056,11 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   const uint32_t row_tiles = use_scatter ? F.row_tiles : L.row_tiles;
   if (use_scatter) {
     // zero tickets, histograms and the look-back words of the offset scan and of the row passes
-    ODIN_CUDA(cudaMemsetAsync(base, 0, F.row_keys[0], st));
+    ODIN_CUDA(odin_zero(ctx, base, F.row_keys[0], st));
   } else {
     // zero tickets, histograms, the used part of the difference array and the look-back words of the passes that run
-    ODIN_CUDA(cudaMemsetAsync(base, 0, L.tile_diff + ((size_t)n_tiles + 1) * 4, st));
-    ODIN_CUDA(cudaMemsetAsync(base + L.scan_state, 0,
+    ODIN_CUDA(odin_zero(ctx, base, L.tile_diff + ((size_t)n_tiles + 1) * 4, st));
+    ODIN_CUDA(odin_zero(ctx, base + L.scan_state,
                               L.inst_states + (size_t)tile_passes * L.tiles * SORT_RADIX * 4 - L.scan_state, st));
   }
   uint32_t* tickets = reinterpret_cast<uint32_t*>(base);
@@ -1081,8 +1083,8 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   {
     OdinKernelScope ks(ctx, K_ROW_HIST, st);
     // one block per SM at most: every block ends with 1024 global reductions onto the same 1024 words
-    row_hist_kernel<<<row_blocks < sms * 4 ? row_blocks : sms * 4, 256, 0, st>>>(depth_bits, proj->num_rows, hist, dbase,
-                                                                                 tickets + 9);
+    ODIN_CUDA(odin_launch(ctx, false, row_hist_kernel, dim3(row_blocks < sms * 4 ? row_blocks : sms * 4), dim3(256), 0, st,
+                          depth_bits, proj->num_rows, hist, dbase, tickets + 9));
   }
   constexpr size_t OS_SMEM = os_smem_bytes(OS_INST_ITEMS), OS_ROW_SMEM = os_smem_bytes(OS_ROW_ITEMS);
   const uint32_t* sorted_row = nullptr;

@@ -13,7 +13,7 @@ enum OdinKernelId {
   K_PROJECT = 0, K_TOUCHED, K_EMIT, K_ONESWEEP, K_FWD, K_L1, K_ZERO_ROWS,
   K_BWD_BLEND, K_BWD_PROJECT, K_ADAM_SH, K_ADAM_GEOM, K_CONFLICT, K_FWD_TAIL, K_PROJECT_SCAN,
   K_PROJECT_ROWS, K_ROW_HIST, K_ROW_SORT, K_ROW_OFFSETS, K_ACTIVE_SET, K_MASK_UNION, K_HAZARD,
-  K_GATE, K_RLG, K_TILE_BASES, K_ACCUMULATE, K_COUNT
+  K_GATE, K_RLG, K_TILE_BASES, K_ACCUMULATE, K_ZERO, K_COUNT
 };
 
 struct OdinProf {
@@ -31,6 +31,8 @@ struct odin_ctx {
   int* d_status;  // first deferred device-side error (0 = none)
   int* h_status;  // pinned mirror read by odin_poll
   int spin_limit; // polls after which a device-side wait gives up (odin_set_wait_limit)
+  int chain;      // odin_chain_begin: 0 = off, 1 = on and the next operation is the first (or follows a copy / memset),
+                  // 2 = on and the last operation enqueued was a kernel of this library
   OdinProf prof;
 };
 
@@ -67,13 +69,15 @@ struct OdinKernelScope {
 // until it has completed and its writes are visible, so the ~3.5 us between two dependent launches are not spent idle.
 // Nothing is read or written before the wait, so ordering is exactly that of a plain launch; without a programmatic
 // predecessor both instructions do nothing.  `dependent` must be false unless the operation in front on the stream is
-// a kernel launched by the same call; it is also dropped while per-kernel events are recorded.
+// a kernel launched by the same call (inside a chain, odin_chain_begin, the library keeps track across calls); it is
+// also dropped while per-kernel events are recorded.  EVERY kernel launched through odin_launch calls
+// odin_after_predecessor() first.
 __device__ __forceinline__ void odin_after_predecessor() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 template <typename... KArgs, typename... Args>
-static inline cudaError_t odin_launch(const odin_ctx* ctx, bool dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block,
+static inline cudaError_t odin_launch(odin_ctx* ctx, bool dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block,
                                       size_t smem, cudaStream_t st, Args&&... args) {
   cudaLaunchConfig_t lc = {};
   lc.gridDim = grid; lc.blockDim = block; lc.dynamicSmemBytes = smem; lc.stream = st;
@@ -81,9 +85,34 @@ static inline cudaError_t odin_launch(const odin_ctx* ctx, bool dependent, void 
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at;
-  lc.numAttrs = (dependent && !ctx->prof.enabled) ? 1 : 0;
+  // inside a chain (odin_chain_begin) the kernel in front may belong to the call before this one
+  lc.numAttrs = ((dependent || ctx->chain == 2) && !ctx->prof.enabled) ? 1 : 0;
+  if (ctx->chain) ctx->chain = 2;
   return cudaLaunchKernelEx(&lc, kernel, std::forward<Args>(args)...);
 }
+
+// Zeroing of scratch words at the start of a call.  Outside a chain a memset; inside a chain a small kernel, so that
+// the kernels on both sides of it stay programmatic dependents (a memset between two kernels costs ~2.7 us by itself
+// and the two launch seams around it).  bytes must be a multiple of 4, p 4-byte aligned.
+static __global__ void odin_zero_words_kernel(uint32_t* __restrict__ p, size_t words) {
+  odin_after_predecessor();
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += (size_t)gridDim.x * blockDim.x) p[i] = 0u;
+}
+static inline cudaError_t odin_zero(odin_ctx* ctx, void* p, size_t bytes, cudaStream_t st) {
+  if (bytes == 0) return cudaSuccess;
+  if (!ctx->chain || ctx->prof.enabled || (bytes & 3) || (reinterpret_cast<uintptr_t>(p) & 3)) {
+    if (ctx->chain) ctx->chain = 1;
+    return cudaMemsetAsync(p, 0, bytes, st);
+  }
+  OdinKernelScope ks(ctx, K_ZERO, st);
+  const size_t words = bytes / 4;
+  size_t blocks = (words + 1023) / 1024;
+  if (blocks > 1184) blocks = 1184;
+  return odin_launch(ctx, false, odin_zero_words_kernel, dim3((unsigned)blocks), dim3(256), 0, st,
+                     reinterpret_cast<uint32_t*>(p), words);
+}
+// a copy or memset enqueued by a call inside a chain: the next kernel must not be a dependent of the kernel before it
+static inline void odin_chain_break(odin_ctx* ctx) { if (ctx && ctx->chain) ctx->chain = 1; }
 
 #define ODIN_CUDA(call)                          \
   do {                                           \

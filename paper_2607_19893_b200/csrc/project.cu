@@ -153,6 +153,7 @@ project_cull_kernel(const float* __restrict__ means, const float* __restrict__ l
                     const float* __restrict__ opacity_logit, uint32_t n, CamParams cam, BinRule rule,
                     uint32_t* __restrict__ tiles_touched, unsigned long long* __restrict__ group_total,
                     unsigned long long* __restrict__ chunk_total, uint32_t groups_per_chunk) {
+  odin_after_predecessor();
   const uint32_t p = blockIdx.x * 256u + threadIdx.x;
   Footprint f = {};
   if (p < n) {
@@ -481,6 +482,7 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   cudaStream_t st = (cudaStream_t)stream;
   const uint32_t n = scene->n;
   if (n == 0) {
+    odin_chain_break(ctx);
     ODIN_CUDA(cudaMemsetAsync(out->num_rows, 0, 4, st));
     ODIN_CUDA(cudaMemsetAsync(out->num_instances, 0, 8, st));
     return ODIN_OK;
@@ -488,7 +490,7 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
   if (!out->tiles_touched) return ODIN_ERR_NULL;
   const size_t need = project_ws_bytes(n);
   if (!ws || !odin_aligned(ws, 256) || ws_bytes < need) return ODIN_ERR_WORKSPACE;
-  ODIN_CUDA(cudaMemsetAsync(ws, 0, need, st));
+  ODIN_CUDA(odin_zero(ctx, ws, need, st));
   uint32_t* ticket = reinterpret_cast<uint32_t*>(ws);
   uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + 256);
   const CamParams cp = odin_cam_params(cam, ctx->cfg);
@@ -521,11 +523,13 @@ extern "C" int odin_project(odin_ctx* ctx, const odin_scene* scene, const odin_c
       unsigned long long* ct = reinterpret_cast<unsigned long long*>(chunk_total);
       unsigned long long* gt = reinterpret_cast<unsigned long long*>(group_total);
       if (rule.binning == 2)
-        project_cull_kernel<true><<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit,
-                                                                   n, cp, rule, out->tiles_touched, gt, ct, gpc);
+        ODIN_CUDA(odin_launch(ctx, false, project_cull_kernel<true>, dim3((n + 255) / 256), dim3(256), 0, st, scene->means,
+                              scene->log_scales, q4, scene->opacity_logit,
+                                                                   n, cp, rule, out->tiles_touched, gt, ct, gpc));
       else
-        project_cull_kernel<false><<<(n + 255) / 256, 256, 0, st>>>(scene->means, scene->log_scales, q4, scene->opacity_logit,
-                                                                    n, cp, rule, out->tiles_touched, gt, ct, gpc);
+        ODIN_CUDA(odin_launch(ctx, false, project_cull_kernel<false>, dim3((n + 255) / 256), dim3(256), 0, st, scene->means,
+                              scene->log_scales, q4, scene->opacity_logit,
+                                                                    n, cp, rule, out->tiles_touched, gt, ct, gpc));
     }
     OdinKernelScope ks(ctx, K_PROJECT_SCAN, st);
     LAUNCH(false, false);

@@ -8,6 +8,7 @@ namespace {
 
 __global__ void zero_rows_kernel(float* __restrict__ g2d, uint8_t* __restrict__ row_active,
                                  const uint32_t* __restrict__ num_rows, uint32_t capacity) {
+  odin_after_predecessor();
   const uint32_t V = min(*num_rows, capacity);
   const size_t count = (size_t)V * 9;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x) {
@@ -410,11 +411,12 @@ extern "C" int odin_render_bwd(odin_ctx* ctx, const odin_scene* scene, const odi
   char* base = reinterpret_cast<char*>(ws);
   uint32_t* header = reinterpret_cast<uint32_t*>(base);
   uint32_t* ticket = header + 1;
-  ODIN_CUDA(cudaMemsetAsync(ticket, 0, 4, st));  // in front of all three kernels: they are launched back to back
+  ODIN_CUDA(odin_zero(ctx, ticket, 4, st));  // in front of all three kernels: they are launched back to back
   const uint32_t zgrid = (uint32_t)ctx->sm_count * 8;
   {
     OdinKernelScope ks(ctx, K_ZERO_ROWS, st);
-    zero_rows_kernel<<<zgrid, 256, 0, st>>>(d_grad2d, d_row_active, proj->num_rows, proj->capacity);
+    ODIN_CUDA(odin_launch(ctx, false, zero_rows_kernel, dim3(zgrid), dim3(256), 0, st, d_grad2d, d_row_active, proj->num_rows,
+                          proj->capacity));
   }
   {
     OdinKernelScope ks(ctx, K_BWD_BLEND, st);

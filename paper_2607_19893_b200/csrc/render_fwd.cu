@@ -14,6 +14,7 @@ render_fwd_kernel(const float2* __restrict__ xy, const float4* __restrict__ coni
                   float* __restrict__ final_T, uint32_t* __restrict__ n_contrib, uint32_t* __restrict__ tile_more,
                   uint32_t* __restrict__ ticket, uint32_t row_cap, uint32_t* __restrict__ tail_queue,
                   uint32_t* __restrict__ bwd_queue) {
+  odin_after_predecessor();
   __shared__ BlendRow s_row[BLEND_WARPS][32];
   __shared__ float s_blue[BLEND_WARPS][32];
   const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -345,6 +346,7 @@ constexpr int LB = 256;
 __global__ void __launch_bounds__(LB)
 l1_loss_kernel(const float* __restrict__ out, const float* __restrict__ target, size_t count, float inv, double* loss_acc,
                float* __restrict__ dL, double inv_count, float* __restrict__ loss, size_t vec4) {
+  odin_after_predecessor();
   // vec4: number of leading float4 groups (0 when the three images are not 16-byte aligned); the rest one by one
   float acc = 0.f;
   const size_t tid = (size_t)blockIdx.x * LB + threadIdx.x, stride = (size_t)gridDim.x * LB;
@@ -405,16 +407,16 @@ extern "C" int odin_render_fwd(odin_ctx* ctx, const odin_projected* proj, const 
   uint32_t* tile_first = reinterpret_cast<uint32_t*>(base + L.tile_first);
   uint32_t* tail_queue = reinterpret_cast<uint32_t*>(base + L.queue);
   cudaStream_t st = (cudaStream_t)stream;
-  ODIN_CUDA(cudaMemsetAsync(header, 0, 96, st));  // tickets, segments taken, the class counts of the two queues
+  ODIN_CUDA(odin_zero(ctx, header, 96, st));  // tickets, segments taken, the class counts of the two queues
   {
     OdinKernelScope ks(ctx, K_FWD, st);
     const int blocks_all = (n_tiles + BLEND_WARPS - 1) / BLEND_WARPS;
     const int blocks = blocks_all < ctx->sm_count * 8 ? blocks_all : ctx->sm_count * 8;  // resident warps pull tiles
-    render_fwd_kernel<<<blocks, BLEND_THREADS, 0, st>>>(
+    ODIN_CUDA(odin_launch(ctx, false, render_fwd_kernel, dim3(blocks), dim3(BLEND_THREADS), 0, st,
         reinterpret_cast<const float2*>(proj->xy), reinterpret_cast<const float4*>(proj->conic_opacity), proj->rgb, d_vals,
         reinterpret_cast<const uint2*>(d_tile_ranges), cam->width, cam->height, TX, n_tiles, cam->bg[0], cam->bg[1],
         cam->bg[2], ctx->cfg.alpha_min, ctx->cfg.alpha_max, ctx->cfg.t_min, d_rgb, d_final_T, d_n_contrib, tile_first,
-        header, proj->capacity, tail_queue, reinterpret_cast<uint32_t*>(base + L.bwd_queue));
+        header, proj->capacity, tail_queue, reinterpret_cast<uint32_t*>(base + L.bwd_queue)));
   }
   OdinKernelScope ks(ctx, K_FWD_TAIL, st);
   const int tail_blocks = n_tiles < ctx->sm_count * 3 ? n_tiles : ctx->sm_count * 3;  // resident blocks pull tiles
@@ -434,6 +436,7 @@ extern "C" int odin_count_blend_pairs(odin_ctx* ctx, const odin_projected* proj,
   const int rc = odin_check_camera(cam);
   if (rc != ODIN_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
+  odin_chain_break(ctx);
   ODIN_CUDA(cudaMemsetAsync(d_counts, 0, 16, st));
   if (proj->capacity == 0) return ODIN_OK;
   if (!proj->xy || !proj->conic_opacity || !d_vals) return ODIN_ERR_NULL;
@@ -454,13 +457,13 @@ extern "C" int odin_l1_loss(odin_ctx* ctx, const float* d_rgb, const float* d_ta
   // the accumulator (8 bytes) and the arrival counter of the blocks (4 bytes behind it) live behind the status word in
   // the context's device block
   double* acc = reinterpret_cast<double*>(reinterpret_cast<char*>(ctx->d_status) + 64);
-  ODIN_CUDA(cudaMemsetAsync(acc, 0, 16, st));
+  ODIN_CUDA(odin_zero(ctx, acc, 16, st));
   const bool aligned = odin_aligned(d_rgb, 16) && odin_aligned(d_target, 16) && odin_aligned(d_dL_drgb, 16);
   const size_t vec4 = aligned ? count / 4 : 0;
   size_t blocks = (count / 4 + LB - 1) / LB + 1;
   if (blocks > (size_t)ctx->sm_count * 8) blocks = (size_t)ctx->sm_count * 8;
   OdinKernelScope ks(ctx, K_L1, st);
-  l1_loss_kernel<<<(unsigned)blocks, LB, 0, st>>>(d_rgb, d_target, count, (float)(1.0 / (double)count), acc, d_dL_drgb,
-                                                  1.0 / (double)count, d_loss, vec4);
+  ODIN_CUDA(odin_launch(ctx, false, l1_loss_kernel, dim3((unsigned)blocks), dim3(LB), 0, st, d_rgb, d_target, count, (float)(1.0 / (double)count), acc, d_dL_drgb,
+                                                  1.0 / (double)count, d_loss, vec4));
   return odin_launch_status();
 }

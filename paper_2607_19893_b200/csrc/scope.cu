@@ -321,11 +321,14 @@ extern "C" int odin_active_set(odin_ctx* ctx, const odin_projected* proj, const 
   if (evidence_mode != 0 && evidence_mode != 1) return ODIN_ERR_INVALID_ARG;
   if (n >= (1u << 28)) return ODIN_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
+  odin_chain_break(ctx);
   ODIN_CUDA(cudaMemsetAsync(d_count, 0, 4, st));
+  odin_chain_break(ctx);
   ODIN_CUDA(cudaMemsetAsync(d_evidence_sum, 0, 8, st));
   const uint32_t words = (n + 31) / 32;
   if (words) {
     if (!d_mask) return ODIN_ERR_NULL;
+    odin_chain_break(ctx);
     ODIN_CUDA(cudaMemsetAsync(d_mask, 0, (size_t)words * 4, st));
   }
   if (proj->capacity == 0 || n == 0) return ODIN_OK;
@@ -345,6 +348,7 @@ extern "C" int odin_active_set(odin_ctx* ctx, const odin_projected* proj, const 
   const uint32_t tiles = (proj->capacity + AS_TILE - 1) / AS_TILE;
   const size_t need = 256 + ws_align((size_t)tiles * 8);
   if (!ws || !odin_aligned(ws, 256) || ws_bytes < need) return ODIN_ERR_WORKSPACE;
+  odin_chain_break(ctx);
   ODIN_CUDA(cudaMemsetAsync(ws, 0, need, st));
   uint32_t* ticket = reinterpret_cast<uint32_t*>(ws);
   uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + 256);
@@ -390,6 +394,7 @@ extern "C" int odin_hazard_count(odin_ctx* ctx, const uint32_t* d_read_masks, co
   if (!d_pairs || !d_counts) return ODIN_ERR_NULL;
   if (n_pairs > 65535) return ODIN_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
+  odin_chain_break(ctx);
   ODIN_CUDA(cudaMemsetAsync(d_counts, 0, (size_t)n_pairs * 32, st));
   const uint32_t words = (n_prims + 31) / 32;
   if (words == 0) return ODIN_OK;
@@ -416,6 +421,7 @@ extern "C" int odin_delayed_read_gate(odin_ctx* ctx, const uint32_t* d_read_b, c
   if (!ctx || !d_gate) return ODIN_ERR_NULL;
   if (!(tau >= 0.f && tau <= 1.f)) return ODIN_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
+  odin_chain_break(ctx);
   ODIN_CUDA(cudaMemsetAsync(d_gate, 0, 32, st));
   const uint32_t words = (n_prims + 31) / 32;
   if (words == 0) return ODIN_OK;

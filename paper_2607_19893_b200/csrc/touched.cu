@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(CC_THREADS)
 conflict_count_kernel(const uint32_t* __restrict__ masks, uint32_t stride_words, uint32_t words,
                       const uint32_t* __restrict__ pairs, uint32_t n_masks, unsigned long long* __restrict__ counts,
                       int* status) {
+  odin_after_predecessor();
   const uint32_t pair = blockIdx.y;
   const uint32_t va = pairs[2 * pair], vb = pairs[2 * pair + 1];
   if (va >= n_masks || vb >= n_masks) {  // uniform over the block: a pair naming a missing view counts 0
@@ -128,12 +129,14 @@ extern "C" int odin_touched_set(odin_ctx* ctx, const uint32_t* d_tiles_touched, 
   cudaStream_t st = (cudaStream_t)stream;
   if (n >= (1u << 28)) return ODIN_ERR_INVALID_ARG;
   if (n == 0) {
+    odin_chain_break(ctx);
     ODIN_CUDA(cudaMemsetAsync(d_count, 0, 4, st));
     return ODIN_OK;
   }
   if (!d_tiles_touched || !d_mask || (idx_capacity > 0 && !d_idx)) return ODIN_ERR_NULL;
   const size_t need = touched_ws_bytes(n);
   if (!ws || !odin_aligned(ws, 256) || ws_bytes < need) return ODIN_ERR_WORKSPACE;
+  odin_chain_break(ctx);
   ODIN_CUDA(cudaMemsetAsync(ws, 0, need, st));
   uint32_t* ticket = reinterpret_cast<uint32_t*>(ws);
   uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + 256);
@@ -152,12 +155,14 @@ extern "C" int odin_mask_to_list(odin_ctx* ctx, const uint32_t* d_mask, uint32_t
   cudaStream_t st = (cudaStream_t)stream;
   if (n >= (1u << 28)) return ODIN_ERR_INVALID_ARG;
   if (n == 0) {
+    odin_chain_break(ctx);
     ODIN_CUDA(cudaMemsetAsync(d_count, 0, 4, st));
     return ODIN_OK;
   }
   if (!d_mask || (idx_capacity > 0 && !d_idx)) return ODIN_ERR_NULL;
   const size_t need = touched_ws_bytes(n);
   if (!ws || !odin_aligned(ws, 256) || ws_bytes < need) return ODIN_ERR_WORKSPACE;
+  odin_chain_break(ctx);
   ODIN_CUDA(cudaMemsetAsync(ws, 0, need, st));
   uint32_t* ticket = reinterpret_cast<uint32_t*>(ws);
   uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(ws) + 256);
@@ -232,7 +237,7 @@ extern "C" int odin_conflict_count(odin_ctx* ctx, const uint32_t* d_masks, uint3
   if (!d_pairs || !d_counts) return ODIN_ERR_NULL;
   if (n_pairs > 65535) return ODIN_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
-  ODIN_CUDA(cudaMemsetAsync(d_counts, 0, (size_t)n_pairs * 8, st));
+  ODIN_CUDA(odin_zero(ctx, d_counts, (size_t)n_pairs * 8, st));
   const uint32_t words = (n_prims + 31) / 32;
   if (words == 0) return ODIN_OK;
   if (!d_masks) return ODIN_ERR_NULL;
@@ -243,8 +248,8 @@ extern "C" int odin_conflict_count(odin_ctx* ctx, const uint32_t* d_masks, uint3
   if (gx > cap) gx = cap;
   if (gx == 0) gx = 1;
   OdinKernelScope ks(ctx, K_CONFLICT, st);
-  conflict_count_kernel<<<dim3(gx, n_pairs), CC_THREADS, 0, st>>>(d_masks, mask_stride_words, words, d_pairs, n_masks,
-                                                                 reinterpret_cast<unsigned long long*>(d_counts),
-                                                                 ctx->d_status);
+  ODIN_CUDA(odin_launch(ctx, false, conflict_count_kernel, dim3(gx, n_pairs), dim3(CC_THREADS), 0, st, d_masks,
+                        mask_stride_words, words, d_pairs, n_masks, reinterpret_cast<unsigned long long*>(d_counts),
+                        ctx->d_status));
   return odin_launch_status();
 }

@@ -239,24 +239,30 @@ class ViewTrainer:
         """project -> touched set -> bin/sort -> composite -> L1 loss -> backward -> sparse Adam -> conflict counts.
         The target image must already be in self.target.  Nothing here synchronises the host."""
         fused = self.fused_touched if fused_touched is None else fused_touched
-        if fused:
-            self.proj.struct.touched_mask = self.masks[slot].data_ptr()
-            self.project(cam, stream)
-            self.idx, self.count = self.proj.prim_id, self.proj.num_rows
-        else:
-            self.proj.struct.touched_mask = None
-            if self.idx is self.proj.prim_id:
-                self.idx, self.count = self._own_idx, self._own_count
-            self.project(cam, stream)
-            self.touched_set(slot, stream)
-        self.bin_sort(stream, want_keys=self.keep_sorted_keys)
-        self.render_fwd(cam, stream)
-        self.l1_loss(stream)
-        self.render_bwd(cam, stream)
-        if update:
-            self.sparse_adam(lr, beta1, beta2, eps, step, stream)
-        if n_pairs:
-            self.conflict_count(d_pairs, n_pairs, d_counts, stream)
+        # nothing but this library's calls is enqueued until the end of the step: the calls are chained (the first
+        # kernel of each is launched behind the last kernel of the one before it without an idle seam)
+        B.odin_chain_begin(self.ctx)
+        try:
+            if fused:
+                self.proj.struct.touched_mask = self.masks[slot].data_ptr()
+                self.project(cam, stream)
+                self.idx, self.count = self.proj.prim_id, self.proj.num_rows
+            else:
+                self.proj.struct.touched_mask = None
+                if self.idx is self.proj.prim_id:
+                    self.idx, self.count = self._own_idx, self._own_count
+                self.project(cam, stream)
+                self.touched_set(slot, stream)
+            self.bin_sort(stream, want_keys=self.keep_sorted_keys)
+            self.render_fwd(cam, stream)
+            self.l1_loss(stream)
+            self.render_bwd(cam, stream)
+            if update:
+                self.sparse_adam(lr, beta1, beta2, eps, step, stream)
+            if n_pairs:
+                self.conflict_count(d_pairs, n_pairs, d_counts, stream)
+        finally:
+            B.odin_chain_end(self.ctx)
 
     # -------------------------------------------------------------------------------------------- task unit of two views
     def prepare_unit(self):

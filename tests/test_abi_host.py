@@ -55,6 +55,7 @@ def test_null_context_is_rejected_without_a_device(lib):
     assert lib.odin_render_workspace_bytes(null, 64, 64, C.byref(sz)) == B.ODIN_ERR_NULL
     assert lib.odin_render_fwd(null, None, None, None, None, None, None, None, None, 0, None) == B.ODIN_ERR_NULL
     assert lib.odin_l1_loss(null, None, None, 1, 1, None, None, None) == B.ODIN_ERR_NULL
+    assert lib.odin_chain_begin(null) == B.ODIN_ERR_NULL and lib.odin_chain_end(null) == B.ODIN_ERR_NULL
     assert lib.odin_render_bwd(null, None, None, None, None, None, None, None, None, None, None, None, None, None, 0,
                                None) == B.ODIN_ERR_NULL
     assert lib.odin_active_set(null, None, None, None, None, 0, 0, None, None, 0, None, None, None, None, 0,
