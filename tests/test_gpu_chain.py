@@ -317,6 +317,46 @@ def test_chain_city_scaled(oracle32):
     run_chain(oracle32, w, steps=2, views=[0, 1], tag="cfg5_scaled")
 
 
+def test_chained_calls_equal_unchained_calls(monkeypatch):
+    """odin_chain_begin / odin_chain_end only remove idle time between the calls: a view step whose calls are chained
+    (the default of ViewTrainer.view_step) and one whose calls are not give the same lists, image, counts and conflict
+    counts bit for bit, and the same loss, gradients and parameters up to the order of their atomic sums.  Scenes on
+    both sides of the size at which the projection takes two kernels."""
+    for w in (wl.make_workload(2, n=30_000), wl.make_workload(5, n=2048 * 4 * 148 + 5000, n_cameras=4)):
+        cams = [B.make_camera(c) for c in w.cameras[:3]]
+        a = G.trainer_for(w.scene, w.cameras[0], mask_slots=3, row_capacity=min(w.scene.n, 400_000))
+        b = G.trainer_for(w.scene, w.cameras[0], mask_slots=3, row_capacity=min(w.scene.n, 400_000))
+        pairs = torch.tensor([[0, 1], [1, 2]], dtype=torch.int32, device=a.device)
+        ca = torch.zeros(2, dtype=torch.int64, device=a.device)
+        cb = torch.zeros(2, dtype=torch.int64, device=a.device)
+        for s, cam in enumerate(cams):
+            tgt = torch.from_numpy(w.target(s)).to(a.device)
+            a.target.copy_(tgt)
+            b.target.copy_(tgt)
+            for sa, sb in ((a.params, b.params), (a.m, b.m), (a.v, b.v)):  # the same state on both sides at every step
+                for ta, tb in zip(sa.tensors(), sb.tensors()):
+                    tb.copy_(ta)
+            a.view_step(cam, s + 1, w.lr, w.beta1, w.beta2, w.eps, slot=s, d_pairs=pairs, n_pairs=2, d_counts=ca)
+            with monkeypatch.context() as mp:
+                mp.setattr(B, "odin_chain_begin", lambda ctx: None)
+                b.view_step(cam, s + 1, w.lr, w.beta1, w.beta2, w.eps, slot=s, d_pairs=pairs, n_pairs=2, d_counts=cb)
+            G.poll_ok(a)
+            G.poll_ok(b)
+            v = int(a.count.item())
+            assert v == int(b.count.item()) and v > 0
+            m = int(a.proj.num_instances.item())
+            assert torch.equal(a.ranges, b.ranges) and torch.equal(a.vals[:m], b.vals[:m])
+            assert torch.equal(a.out, b.out) and torch.equal(a.n_contrib, b.n_contrib) and torch.equal(a.final_T, b.final_T)
+            assert torch.equal(a.dL, b.dL) and torch.equal(a.masks[s], b.masks[s]) and torch.equal(ca, cb)
+            assert abs(float(a.loss.item()) - float(b.loss.item())) <= 1e-6 * abs(float(b.loss.item()))
+            ga, gb = a.gradient_rows(v), b.gradient_rows(v)
+            assert np.allclose(ga, gb, rtol=1e-4, atol=1e-9 * max(1.0, float(np.abs(gb).max())))
+            for ta, tb in zip(a.params.tensors(), b.params.tensors()):
+                assert torch.allclose(ta, tb, rtol=1e-5, atol=1e-6)
+        a.close()
+        b.close()
+
+
 def test_train_from_host_equals_the_plain_loop():
     """The double-buffered host-target loop is marshalling only: the same kernels on the same inputs, so losses, counts
     and the trained parameters are bitwise those of the plain loop (atomics aside: compared with a tolerance)."""
