@@ -376,15 +376,14 @@ def run_config(args, cfg_id, steps, warmup, rank, local_rank, world, want_cpu_ba
     sort_mode = int(getattr(tr, "instance_sort", max(args.instance_sort, 0)))
     bytes_kernels = kernel_bytes(n, f, v_last, m_last, m_proc, W * H, tx * ty, tile_passes, n_pairs_last,
                                  scatter=(sort_mode == 0))
-    # Adam leaves a row alone whose gradient and moments are all zero (it then reads the two moments only): count those
-    # rows of the last view (measurement code, outside every timed region; the SH block stands for the row) and charge
-    # them 8F + 5 bytes instead of 28F + 4
+    # Adam skips a row that has no gradient (flagged by the backward pass) and no history (the optimizer's flag of the
+    # primitive is clear) after reading its index and the two flags, in each of its two kernels: count those rows of
+    # the last view (measurement code, outside every timed region) and charge them 12 bytes instead of 28F + 4
     rows_last = tr.idx[:v_last].long()
     flagged = tr.row_zero[:v_last].bool() if tr._row_zero_in_use is not None else torch.zeros(v_last, dtype=torch.bool, device=dev)
-    idle_rows = int((flagged & (tr.m.sh[rows_last].flatten(1) == 0).all(dim=1) & (tr.v.sh[rows_last].flatten(1) == 0).all(dim=1)
-                     & (tr.m.means[rows_last] == 0).all(dim=1)).sum().item())
+    idle_rows = int((flagged & (tr.live[rows_last] == 0)).sum().item())
     bytes_kernels["total"] -= bytes_kernels["adam"]
-    bytes_kernels["adam"] = float(idle_rows * (8 * f + 5) + (v_last - idle_rows) * (28 * f + 4))
+    bytes_kernels["adam"] = float(idle_rows * 12 + (v_last - idle_rows) * (28 * f + 4))
     bytes_kernels["total"] += bytes_kernels["adam"]
     alu_peak = B.odin_measure_fp32_peak(tr.ctx, stream) if rank == 0 else 0.0
 

@@ -298,6 +298,24 @@ int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m, odin_scen
                      const uint8_t* d_row_zero, const uint32_t* d_idx, const uint32_t* d_count, const float lr[6],
                      float beta1, float beta2, float eps, uint32_t step, void* stream);
 
+/* The same update with one byte of optimizer state per primitive that lets it leave untouched history unread (phase U
+ * of Sec. 4.1; most rows a view touches are occluded, receive no gradient and have never received one).
+ * d_live [params->n] (bytes, device, caller-owned, may be NULL = odin_sparse_adam): d_live[p] == 0 promises that
+ * EVERY moment of primitive p, in m and in v, is zero.  A listed row with a zero gradient and d_live == 0 is then
+ * skipped without reading its moments (the result is what the full update gives bit for bit: zero moments stay zero
+ * and theta - step * 0 / (0 + eps) = theta; with eps == 0 nothing is skipped); the call sets d_live[p] = 1 for every
+ * primitive to which it writes moments that may be non-zero, so the promise holds again on return.  The array belongs
+ * with m and v: zero it when they are zeroed, store and restore it with them, and after writing m or v by any other
+ * means call odin_adam_live_refresh (or set every byte to 1, which is always valid).  Not to be shared between two
+ * calls that overlap in time. */
+int odin_sparse_adam_live(odin_ctx* ctx, odin_scene* params, odin_scene* m, odin_scene* v, const odin_scene* grad_rows,
+                          const uint8_t* d_row_zero, const uint32_t* d_idx, const uint32_t* d_count, uint8_t* d_live,
+                          const float lr[6], float beta1, float beta2, float eps, uint32_t step, void* stream);
+
+/* d_live[p] = 1 if any moment of primitive p (any word of its rows in m or v) is non-zero, else 0, for all p < m->n:
+ * the tightest flags that keep the promise of odin_sparse_adam_live.  One pass over both moment pools. */
+int odin_adam_live_refresh(odin_ctx* ctx, const odin_scene* m, const odin_scene* v, uint8_t* d_live, void* stream);
+
 /* Conflict counts (Sec. 4.3): for each listed pair (a, b) of views, |W^+(a) & W^+(b)| = popcount of the AND of their
  * touched bitmasks, the size of C_WAW^+ (C_RAW^+ and C_WAR^+ are empty because R^+ = W^+ here).
  * d_masks [n_masks][mask_stride_words]; d_pairs [n_pairs][2] view slots; d_counts [n_pairs] (overwritten). */

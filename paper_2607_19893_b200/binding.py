@@ -30,7 +30,7 @@ EXPORTS = [
     "odin_touched_set_static", "odin_render_workspace_bytes", "odin_active_set", "odin_mask_union", "odin_hazard_count",
     "odin_delayed_read_gate", "odin_rlg_weights", "odin_rlg_topk", "odin_sds_scores", "odin_set_wait_limit",
     "odin_bin_sort_workspace_bytes", "odin_set_instance_sort", "odin_measure_fp32_peak", "odin_count_blend_pairs",
-    "odin_mask_to_list", "odin_accumulate_rows",
+    "odin_mask_to_list", "odin_accumulate_rows", "odin_sparse_adam_live", "odin_adam_live_refresh",
 ]
 
 
@@ -112,6 +112,9 @@ def lib() -> C.CDLL:
                                       vp, vp, vp, vp, C.POINTER(odin_scene), vp, vp, vp, C.c_size_t, vp]
         L.odin_sparse_adam.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_scene), C.POINTER(odin_scene),
                                        C.POINTER(odin_scene), vp, vp, vp, C.POINTER(f32), f32, f32, f32, u32, vp]
+        L.odin_sparse_adam_live.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_scene), C.POINTER(odin_scene),
+                                            C.POINTER(odin_scene), vp, vp, vp, vp, C.POINTER(f32), f32, f32, f32, u32, vp]
+        L.odin_adam_live_refresh.argtypes = [vp, C.POINTER(odin_scene), C.POINTER(odin_scene), vp, vp]
         L.odin_conflict_count.argtypes = [vp, vp, u32, u32, u32, vp, u32, vp, vp]
         L.odin_touched_set_static.argtypes = [vp, u32, vp, vp, u32, vp, vp, vp]
         L.odin_active_set.argtypes = [vp, C.POINTER(odin_projected), vp, vp, C.POINTER(odin_scene), i32, u32, vp, vp, u32,
@@ -311,6 +314,20 @@ def odin_sparse_adam(ctx, params: odin_scene, m: odin_scene, v: odin_scene, grad
     _check(lib().odin_sparse_adam(ctx, C.byref(params), C.byref(m), C.byref(v), C.byref(grad_rows), _ptr(d_row_zero),
                                   _ptr(d_idx), _ptr(d_count), lr_arr, float(beta1), float(beta2), float(eps), int(step),
                                   _stream(stream)), "odin_sparse_adam")
+
+
+def odin_sparse_adam_live(ctx, params: odin_scene, m: odin_scene, v: odin_scene, grad_rows: odin_scene, d_row_zero, d_idx,
+                          d_count, d_live, lr: Sequence[float], beta1: float, beta2: float, eps: float, step: int,
+                          stream=None) -> None:
+    lr_arr = (C.c_float * 6)(*[float(x) for x in lr])
+    _check(lib().odin_sparse_adam_live(ctx, C.byref(params), C.byref(m), C.byref(v), C.byref(grad_rows), _ptr(d_row_zero),
+                                       _ptr(d_idx), _ptr(d_count), _ptr(d_live), lr_arr, float(beta1), float(beta2),
+                                       float(eps), int(step), _stream(stream)), "odin_sparse_adam_live")
+
+
+def odin_adam_live_refresh(ctx, m: odin_scene, v: odin_scene, d_live, stream=None) -> None:
+    _check(lib().odin_adam_live_refresh(ctx, C.byref(m), C.byref(v), _ptr(d_live), _stream(stream)),
+           "odin_adam_live_refresh")
 
 
 def odin_conflict_count(ctx, d_masks, n_masks: int, mask_stride_words: int, n_prims: int, d_pairs, n_pairs: int, d_counts,

@@ -31,106 +31,165 @@ __device__ __forceinline__ void adam_one(float& th, float& m, float& v, float g,
   th = th - __fdividef(step_size * m, adam_sqrt(v) * k.inv_bc2s + k.eps);
 }
 
-// SH block: ROWF floats per row (3, 12, 27 or 48), processed as VEC-wide elements; element e of the compact
-// gradient block belongs to row e / (ROWF / VEC).
+// Flags of the primitives whose moments may be non-zero (live[p] == 0: every moment of p, in every attribute, is zero).
+// With them a row that has no gradient and no history costs its index and two bytes instead of a read of both moments.
+__device__ __forceinline__ bool adam_cold(const uint8_t* live, size_t prim, const AdamK& k) {
+  return live && k.skip_idle && live[prim] == 0;
+}
+// Called by a thread that is about to write moments that may be non-zero.
+__device__ __forceinline__ void adam_mark_live(uint8_t* live, size_t prim, bool cold, const AdamK& k) {
+  if (live && (cold || !k.skip_idle)) live[prim] = 1;
+}
+
+// Both kernels give a warp 32 consecutive rows of the list at a time.  The warp first looks at the rows themselves
+// (index, row flag, primitive flag: three coalesced or nearly coalesced loads), drops the rows with nothing to do - no
+// gradient and no history, or an index out of range - and leaves the others, in order, in shared memory; the elements
+// of the remaining rows are then spread over the lanes.  Where most rows of a view are occluded a warp so works on full
+// loads of the few rows that matter instead of running the whole chain of dependent loads for one live lane in eight.
+constexpr int ADAM_WARPS = 8;
+
+// returns the number of rows kept; s_prim[i] = primitive, s_info[i] = place in the group | zero << 8 | cold << 9
+__device__ __forceinline__ uint32_t adam_stage_rows(uint32_t grp, uint32_t V, const uint32_t* __restrict__ idx,
+                                                    const uint8_t* __restrict__ row_zero, const uint8_t* live,
+                                                    uint32_t n_prims, const AdamK& k, uint32_t* s_prim, uint32_t* s_info,
+                                                    unsigned lane) {
+  const uint32_t r = grp * 32 + lane;
+  uint32_t prim = 0;
+  bool zero = false, cold = false, act = false;
+  if (r < V) {
+    prim = idx[r];
+    if (prim < n_prims) {  // (an index list that is not a view's own, e.g. after a timed-out scan: no write)
+      zero = row_zero && row_zero[r];  // the gradient row was not written: it is zero
+      // cold: the primitive's flag says that all of its moments are zero, so they are not read.  (A thread of the
+      // other kernel may raise the flag while this one reads it; either value is right here: the moments this kernel
+      // owns are written by nobody else.)
+      cold = adam_cold(live, prim, k);
+      act = !(cold && zero);
+    }
+  }
+  const uint32_t mask = __ballot_sync(0xffffffffu, act);
+  __syncwarp();  // the previous group's entries have been read
+  if (act) {
+    const uint32_t pos = __popc(mask & ((1u << lane) - 1u));
+    s_prim[pos] = prim;
+    s_info[pos] = lane | (zero ? 256u : 0u) | (cold ? 512u : 0u);
+  }
+  __syncwarp();
+  return (uint32_t)__popc(mask);
+}
+
+// SH block: ROWF floats per row (3, 12, 27 or 48), processed as VEC-wide elements.
 template <int ROWF, int VEC>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(ADAM_WARPS * 32)
 adam_sh_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v, const float* __restrict__ g,
                const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count, uint32_t cap, AdamK k,
-               const uint8_t* __restrict__ row_zero, uint32_t n_prims) {
+               const uint8_t* __restrict__ row_zero, uint32_t n_prims, uint8_t* live) {
   odin_after_predecessor();
   constexpr int EPR = ROWF / VEC;  // elements per row
+  __shared__ uint32_t s_prim[ADAM_WARPS][32], s_info[ADAM_WARPS][32];
+  const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t V = min(*count, cap);
-  const size_t total = (size_t)V * EPR;
-  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
-    const uint32_t r = (uint32_t)(e / EPR);
-    const uint32_t j = (uint32_t)(e - (size_t)r * EPR);
-    const uint32_t prim = idx[r];
-    if (prim >= n_prims) continue;  // an index list that is not a view's own (e.g. after a timed-out scan): no write
-    const size_t dst = (size_t)prim * ROWF + (size_t)j * VEC;
-    const bool zero = row_zero && row_zero[r];  // the gradient row was not written: it is zero
-    if (VEC == 4) {
-      const float4 gg = zero ? make_float4(0.f, 0.f, 0.f, 0.f) : reinterpret_cast<const float4*>(g)[e];
-      float4 mm = *reinterpret_cast<float4*>(m + dst), vv = *reinterpret_cast<float4*>(v + dst);
-      if (k.skip_idle && gg.x == 0.f && gg.y == 0.f && gg.z == 0.f && gg.w == 0.f && mm.x == 0.f && mm.y == 0.f &&
-          mm.z == 0.f && mm.w == 0.f && vv.x == 0.f && vv.y == 0.f && vv.z == 0.f && vv.w == 0.f)
-        continue;
-      float4 pp = *reinterpret_cast<float4*>(p + dst);
-      // floats 0..2 of a row are the degree-0 coefficients (group 4); the rest group 5
-      const int f0 = j * 4;
-      adam_one(pp.x, mm.x, vv.x, gg.x, k.step_size[f0 + 0 < 3 ? 4 : 5], k);
-      adam_one(pp.y, mm.y, vv.y, gg.y, k.step_size[f0 + 1 < 3 ? 4 : 5], k);
-      adam_one(pp.z, mm.z, vv.z, gg.z, k.step_size[f0 + 2 < 3 ? 4 : 5], k);
-      adam_one(pp.w, mm.w, vv.w, gg.w, k.step_size[5], k);
-      *reinterpret_cast<float4*>(p + dst) = pp;
-      *reinterpret_cast<float4*>(m + dst) = mm;
-      *reinterpret_cast<float4*>(v + dst) = vv;
-    } else {
-      float mm = m[dst], vv = v[dst];
-      const float gg = zero ? 0.f : g[e];
-      if (k.skip_idle && gg == 0.f && mm == 0.f && vv == 0.f) continue;
-      float pp = p[dst];
-      adam_one(pp, mm, vv, gg, k.step_size[j < 3 ? 4 : 5], k);
-      p[dst] = pp; m[dst] = mm; v[dst] = vv;
+  const uint32_t groups = (V + 31) / 32;
+  // with the primitive flags in use a row that gets this far nearly always has work: its parameters are then fetched
+  // together with the moments instead of after the test on them
+  const bool eager = live != nullptr;
+  for (uint32_t grp = blockIdx.x * ADAM_WARPS + warp; grp < groups; grp += gridDim.x * ADAM_WARPS) {
+    const uint32_t kept = adam_stage_rows(grp, V, idx, row_zero, live, n_prims, k, s_prim[warp], s_info[warp], lane);
+    for (uint32_t q = lane; q < kept * EPR; q += 32) {
+      const uint32_t slot = q / EPR, j = q - slot * EPR;
+      const uint32_t prim = s_prim[warp][slot], info = s_info[warp][slot];
+      const bool zero = info & 256u, cold = info & 512u;
+      const size_t e = (size_t)(grp * 32 + (info & 255u)) * EPR + j;  // element of the compact gradient block
+      const size_t dst = (size_t)prim * ROWF + (size_t)j * VEC;
+      if (VEC == 4) {
+        const float4 gg = zero ? make_float4(0.f, 0.f, 0.f, 0.f) : reinterpret_cast<const float4*>(g)[e];
+        const bool gzero = gg.x == 0.f && gg.y == 0.f && gg.z == 0.f && gg.w == 0.f;
+        if (cold && gzero) continue;
+        float4 mm = make_float4(0.f, 0.f, 0.f, 0.f), vv = mm, pp = mm;
+        if (!cold) { mm = *reinterpret_cast<float4*>(m + dst); vv = *reinterpret_cast<float4*>(v + dst); }
+        if (eager) pp = *reinterpret_cast<float4*>(p + dst);
+        if (k.skip_idle && gzero && mm.x == 0.f && mm.y == 0.f && mm.z == 0.f && mm.w == 0.f && vv.x == 0.f &&
+            vv.y == 0.f && vv.z == 0.f && vv.w == 0.f)
+          continue;
+        adam_mark_live(live, prim, cold, k);
+        if (!eager) pp = *reinterpret_cast<float4*>(p + dst);
+        // floats 0..2 of a row are the degree-0 coefficients (group 4); the rest group 5
+        const int f0 = j * 4;
+        adam_one(pp.x, mm.x, vv.x, gg.x, k.step_size[f0 + 0 < 3 ? 4 : 5], k);
+        adam_one(pp.y, mm.y, vv.y, gg.y, k.step_size[f0 + 1 < 3 ? 4 : 5], k);
+        adam_one(pp.z, mm.z, vv.z, gg.z, k.step_size[f0 + 2 < 3 ? 4 : 5], k);
+        adam_one(pp.w, mm.w, vv.w, gg.w, k.step_size[5], k);
+        *reinterpret_cast<float4*>(p + dst) = pp;
+        *reinterpret_cast<float4*>(m + dst) = mm;
+        *reinterpret_cast<float4*>(v + dst) = vv;
+      } else {
+        const float gg = zero ? 0.f : g[e];
+        if (cold && gg == 0.f) continue;
+        float mm = 0.f, vv = 0.f, pp = 0.f;
+        if (!cold) { mm = m[dst]; vv = v[dst]; }
+        if (eager) pp = p[dst];
+        if (k.skip_idle && gg == 0.f && mm == 0.f && vv == 0.f) continue;
+        adam_mark_live(live, prim, cold, k);
+        if (!eager) pp = p[dst];
+        adam_one(pp, mm, vv, gg, k.step_size[j < 3 ? 4 : 5], k);
+        p[dst] = pp; m[dst] = mm; v[dst] = vv;
+      }
     }
   }
 }
 
-// Geometry block: four threads per row - mean(3), log scale(3), quaternion(4), opacity(1) - so that a row's twelve
-// gathers are spread over four independent threads instead of queueing in one.
-__global__ void __launch_bounds__(256)
-adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float4* __restrict__ p_q, float* __restrict__ p_o,
-                 float* __restrict__ m_mean, float* __restrict__ m_ls, float4* __restrict__ m_q, float* __restrict__ m_o,
-                 float* __restrict__ v_mean, float* __restrict__ v_ls, float4* __restrict__ v_q, float* __restrict__ v_o,
-                 const float* __restrict__ g_mean, const float* __restrict__ g_ls, const float4* __restrict__ g_q,
+// Geometry block: four lanes per row - mean(3), log scale(3), quaternion(4), opacity(1) - on ONE code path (the part
+// selects base pointers and a width), so that the loads of all four parts of eight rows are in flight together; with a
+// branch per part the warp ran three chains of dependent loads one after the other.
+__global__ void __launch_bounds__(ADAM_WARPS * 32)
+adam_geom_kernel(float* __restrict__ p_mean, float* __restrict__ p_ls, float* __restrict__ p_q, float* __restrict__ p_o,
+                 float* __restrict__ m_mean, float* __restrict__ m_ls, float* __restrict__ m_q, float* __restrict__ m_o,
+                 float* __restrict__ v_mean, float* __restrict__ v_ls, float* __restrict__ v_q, float* __restrict__ v_o,
+                 const float* __restrict__ g_mean, const float* __restrict__ g_ls, const float* __restrict__ g_q,
                  const float* __restrict__ g_o, const uint32_t* __restrict__ idx, const uint32_t* __restrict__ count,
-                 uint32_t cap, AdamK k, const uint8_t* __restrict__ row_zero, uint32_t n_prims) {
+                 uint32_t cap, AdamK k, const uint8_t* __restrict__ row_zero, uint32_t n_prims, uint8_t* live) {
   odin_after_predecessor();  // launched behind the SH kernel (which it does not depend on: the two overlap at the seam)
+  __shared__ uint32_t s_prim[ADAM_WARPS][32], s_info[ADAM_WARPS][32];
+  const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t V = min(*count, cap);
-  const size_t total = (size_t)V * 4;
-  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
-    const uint32_t r = (uint32_t)(e >> 2);
-    const int part = (int)(e & 3);
-    const size_t d = idx[r];
-    if (d >= n_prims) continue;
-    const bool zero = row_zero && row_zero[r];  // the gradient row was not written: it is zero
-    if (part < 2) {
-      float* __restrict__ p = (part ? p_ls : p_mean) + 3 * d;
-      float* __restrict__ m = (part ? m_ls : m_mean) + 3 * d;
-      float* __restrict__ v = (part ? v_ls : v_mean) + 3 * d;
-      const float* __restrict__ g = (part ? g_ls : g_mean) + 3 * (size_t)r;
-      const float ss = k.step_size[part];
-      float pp[3], mm[3], vv[3], gg[3];
+  const uint32_t groups = (V + 31) / 32;
+  const bool eager = live != nullptr;  // (see the SH kernel)
+  const int part = (int)(lane & 3);
+  const int width = part < 2 ? 3 : (part == 2 ? 4 : 1);
+  const float ss = k.step_size[part];
+  for (uint32_t grp = blockIdx.x * ADAM_WARPS + warp; grp < groups; grp += gridDim.x * ADAM_WARPS) {
+    const uint32_t kept = adam_stage_rows(grp, V, idx, row_zero, live, n_prims, k, s_prim[warp], s_info[warp], lane);
+    for (uint32_t slot = lane >> 2; slot < kept; slot += 8) {
+      const size_t d = s_prim[warp][slot];
+      const uint32_t info = s_info[warp][slot];
+      const bool zero = info & 256u, cold = info & 512u;
+      const size_t r = (size_t)grp * 32 + (info & 255u);
+      const size_t od = (size_t)width * d, og = (size_t)width * r;
+      float* P = (part == 0 ? p_mean : part == 1 ? p_ls : part == 2 ? p_q : p_o) + od;
+      float* M = (part == 0 ? m_mean : part == 1 ? m_ls : part == 2 ? m_q : m_o) + od;
+      float* Vv = (part == 0 ? v_mean : part == 1 ? v_ls : part == 2 ? v_q : v_o) + od;
+      const float* G = (part == 0 ? g_mean : part == 1 ? g_ls : part == 2 ? g_q : g_o) + og;
+      float pp[4], mm[4], vv[4], gg[4];
+      bool idle = true;
 #pragma unroll
-      for (int i = 0; i < 3; ++i) { mm[i] = m[i]; vv[i] = v[i]; gg[i] = zero ? 0.f : g[i]; }
-      if (k.skip_idle && gg[0] == 0.f && gg[1] == 0.f && gg[2] == 0.f && mm[0] == 0.f && mm[1] == 0.f && mm[2] == 0.f &&
-          vv[0] == 0.f && vv[1] == 0.f && vv[2] == 0.f)
-        continue;
+      for (int i = 0; i < 4; ++i) {
+        const bool on = i < width;
+        mm[i] = (on && !cold) ? M[i] : 0.f;
+        vv[i] = (on && !cold) ? Vv[i] : 0.f;
+        gg[i] = (on && !zero) ? G[i] : 0.f;
+        pp[i] = (on && eager) ? P[i] : 0.f;
+        idle = idle && gg[i] == 0.f && mm[i] == 0.f && vv[i] == 0.f;
+      }
+      if (k.skip_idle && idle) continue;
+      adam_mark_live(live, d, cold, k);
 #pragma unroll
-      for (int i = 0; i < 3; ++i) pp[i] = p[i];
-#pragma unroll
-      for (int i = 0; i < 3; ++i) adam_one(pp[i], mm[i], vv[i], gg[i], ss, k);
-#pragma unroll
-      for (int i = 0; i < 3; ++i) { p[i] = pp[i]; m[i] = mm[i]; v[i] = vv[i]; }
-    } else if (part == 2) {
-      float4 mm = m_q[d], vv = v_q[d];
-      const float4 gg = zero ? make_float4(0.f, 0.f, 0.f, 0.f) : g_q[r];
-      if (k.skip_idle && gg.x == 0.f && gg.y == 0.f && gg.z == 0.f && gg.w == 0.f && mm.x == 0.f && mm.y == 0.f &&
-          mm.z == 0.f && mm.w == 0.f && vv.x == 0.f && vv.y == 0.f && vv.z == 0.f && vv.w == 0.f)
-        continue;
-      float4 pp = p_q[d];
-      adam_one(pp.x, mm.x, vv.x, gg.x, k.step_size[2], k);
-      adam_one(pp.y, mm.y, vv.y, gg.y, k.step_size[2], k);
-      adam_one(pp.z, mm.z, vv.z, gg.z, k.step_size[2], k);
-      adam_one(pp.w, mm.w, vv.w, gg.w, k.step_size[2], k);
-      p_q[d] = pp; m_q[d] = mm; v_q[d] = vv;
-    } else {
-      float mm = m_o[d], vv = v_o[d];
-      const float gg = zero ? 0.f : g_o[r];
-      if (k.skip_idle && gg == 0.f && mm == 0.f && vv == 0.f) continue;
-      float pp = p_o[d];
-      adam_one(pp, mm, vv, gg, k.step_size[3], k);
-      p_o[d] = pp; m_o[d] = mm; v_o[d] = vv;
+      for (int i = 0; i < 4; ++i) {
+        if (i < width) {
+          if (!eager) pp[i] = P[i];
+          adam_one(pp[i], mm[i], vv[i], gg[i], ss, k);
+          P[i] = pp[i]; M[i] = mm[i]; Vv[i] = vv[i];
+        }
+      }
     }
   }
 }
@@ -187,6 +246,13 @@ accumulate_rows_kernel(RowsView a, RowsView b, const uint32_t* __restrict__ idx_
   }
 }
 
+// live[i / width] = 1 for every non-zero word a[i] (the flags are cleared first; one launch per attribute array)
+__global__ void __launch_bounds__(256)
+mark_nonzero_kernel(const float* __restrict__ a, size_t total, uint32_t width, uint8_t* __restrict__ live) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x)
+    if (a[i] != 0.f) live[i / width] = 1;  // (a NaN counts as non-zero)
+}
+
 }  // namespace
 
 extern "C" int odin_accumulate_rows(odin_ctx* ctx, const odin_scene* rows_a, const uint8_t* d_zero_a, const uint32_t* d_idx_a,
@@ -215,10 +281,44 @@ extern "C" int odin_accumulate_rows(odin_ctx* ctx, const odin_scene* rows_a, con
   return odin_launch_status();
 }
 
+extern "C" int odin_adam_live_refresh(odin_ctx* ctx, const odin_scene* m, const odin_scene* v, uint8_t* d_live,
+                                     void* stream) {
+  if (!ctx || !d_live) return ODIN_ERR_NULL;
+  int rc = odin_check_scene(m);
+  if (rc == ODIN_OK) rc = odin_check_scene(v);
+  if (rc != ODIN_OK) return rc;
+  if (m->n != v->n || m->sh_degree != v->sh_degree) return ODIN_ERR_INVALID_ARG;
+  if (m->n == 0) return ODIN_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  odin_chain_break(ctx);
+  ODIN_CUDA(cudaMemsetAsync(d_live, 0, m->n, st));
+  const int K = (m->sh_degree + 1) * (m->sh_degree + 1);
+  for (const odin_scene* s : {m, v}) {
+    const float* arrays[5] = {s->means, s->log_scales, s->quats, s->opacity_logit, s->sh};
+    const uint32_t widths[5] = {3, 3, 4, 1, (uint32_t)(3 * K)};
+    for (int a = 0; a < 5; ++a) {
+      const size_t total = (size_t)m->n * widths[a];
+      size_t blocks = (total + 255) / 256;
+      if (blocks > (size_t)ctx->sm_count * 16) blocks = (size_t)ctx->sm_count * 16;
+      OdinKernelScope ks(ctx, K_ADAM_LIVE, st);
+      mark_nonzero_kernel<<<(unsigned)blocks, 256, 0, st>>>(arrays[a], total, widths[a], d_live);
+    }
+  }
+  return odin_launch_status();
+}
+
 extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m, odin_scene* v,
                                 const odin_scene* grad_rows, const uint8_t* d_row_zero, const uint32_t* d_idx,
                                 const uint32_t* d_count, const float lr[6], float beta1, float beta2, float eps,
                                 uint32_t step, void* stream) {
+  return odin_sparse_adam_live(ctx, params, m, v, grad_rows, d_row_zero, d_idx, d_count, nullptr, lr, beta1, beta2, eps, step,
+                               stream);
+}
+
+extern "C" int odin_sparse_adam_live(odin_ctx* ctx, odin_scene* params, odin_scene* m, odin_scene* v,
+                                     const odin_scene* grad_rows, const uint8_t* d_row_zero, const uint32_t* d_idx,
+                                     const uint32_t* d_count, uint8_t* d_live, const float lr[6], float beta1, float beta2,
+                                     float eps, uint32_t step, void* stream) {
   if (!ctx || !lr || !d_count) return ODIN_ERR_NULL;
   int rc = odin_check_scene(params);
   if (rc == ODIN_OK) rc = odin_check_scene(m);
@@ -242,27 +342,24 @@ extern "C" int odin_sparse_adam(odin_ctx* ctx, odin_scene* params, odin_scene* m
   cudaStream_t st = (cudaStream_t)stream;
   const uint32_t cap = grad_rows->n;
   const int K = (params->sh_degree + 1) * (params->sh_degree + 1);
-  const size_t max_elems = (size_t)cap * (K == 9 ? 27 : (K == 1 ? 3 : 3 * K / 4));
-  size_t blocks = (max_elems + 255) / 256;
+  // a warp per 32 rows of the list
+  size_t blocks = ((size_t)cap + 32 * ADAM_WARPS - 1) / (32 * ADAM_WARPS);
   if (blocks > (size_t)ctx->sm_count * 16) blocks = (size_t)ctx->sm_count * 16;
   const unsigned gsh = (unsigned)blocks;
   {
     OdinKernelScope ks(ctx, K_ADAM_SH, st);
     switch (params->sh_degree) {
-    case 0: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<3, 1>, dim3(gsh), dim3(256), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n)); break;
-    case 1: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<12, 4>, dim3(gsh), dim3(256), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n)); break;
-    case 2: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<27, 1>, dim3(gsh), dim3(256), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n)); break;
-    default: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<48, 4>, dim3(gsh), dim3(256), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n)); break;
+    case 0: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<3, 1>, dim3(gsh), dim3(ADAM_WARPS * 32), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n, d_live)); break;
+    case 1: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<12, 4>, dim3(gsh), dim3(ADAM_WARPS * 32), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n, d_live)); break;
+    case 2: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<27, 1>, dim3(gsh), dim3(ADAM_WARPS * 32), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n, d_live)); break;
+    default: ODIN_CUDA(odin_launch(ctx, false, adam_sh_kernel<48, 4>, dim3(gsh), dim3(ADAM_WARPS * 32), 0, st, params->sh, m->sh, v->sh, grad_rows->sh, d_idx, d_count, cap, k, d_row_zero, params->n, d_live)); break;
     }
   }
-  size_t gb = ((size_t)cap * 4 + 255) / 256;
-  if (gb > (size_t)ctx->sm_count * 16) gb = (size_t)ctx->sm_count * 16;
   OdinKernelScope ks(ctx, K_ADAM_GEOM, st);
-  ODIN_CUDA(odin_launch(ctx, true, adam_geom_kernel, dim3((unsigned)gb), dim3(256), 0, st,
-      params->means, params->log_scales, reinterpret_cast<float4*>(params->quats), params->opacity_logit, m->means,
-      m->log_scales, reinterpret_cast<float4*>(m->quats), m->opacity_logit, v->means, v->log_scales,
-      reinterpret_cast<float4*>(v->quats), v->opacity_logit, grad_rows->means, grad_rows->log_scales,
-      reinterpret_cast<const float4*>(grad_rows->quats), grad_rows->opacity_logit, d_idx, d_count, cap, k, d_row_zero,
-      params->n));
+  ODIN_CUDA(odin_launch(ctx, true, adam_geom_kernel, dim3(gsh), dim3(ADAM_WARPS * 32), 0, st,
+      params->means, params->log_scales, params->quats, params->opacity_logit, m->means, m->log_scales, m->quats,
+      m->opacity_logit, v->means, v->log_scales, v->quats, v->opacity_logit, (const float*)grad_rows->means,
+      (const float*)grad_rows->log_scales, (const float*)grad_rows->quats, (const float*)grad_rows->opacity_logit, d_idx,
+      d_count, cap, k, d_row_zero, params->n, d_live));
   return odin_launch_status();
 }

@@ -92,7 +92,7 @@ static const char* const kKernelNames[K_COUNT] = {
     "zero_rows", "render_bwd_blend", "render_bwd_project", "adam_sh", "adam_geom", "conflict_count",
     "render_fwd_tail", "project_scan", "project_rows", "row_hist",
     "row_sort_pass", "row_offsets", "active_set", "mask_union", "hazard_count", "delayed_read_gate",
-    "locality_graph", "tile_bases", "accumulate_rows", "zero_words"};
+    "locality_graph", "tile_bases", "accumulate_rows", "zero_words", "adam_live_refresh"};
 
 extern "C" int odin_chain_begin(odin_ctx* ctx) {
   if (!ctx) return ODIN_ERR_NULL;

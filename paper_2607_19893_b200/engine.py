@@ -100,6 +100,9 @@ class ViewTrainer:
         self.params = DeviceScene.from_host(scene, dev)
         self.m = DeviceScene(self.n, self.sh_degree, dev)
         self.v = DeviceScene(self.n, self.sh_degree, dev)
+        # one byte per primitive beside the moments: 0 = every moment of the primitive is zero (odin_sparse_adam_live).
+        # Whoever writes self.m / self.v by other means than the optimizer calls calls moments_changed() afterwards.
+        self.live = torch.zeros(max(self.n, 1), dtype=torch.uint8, device=dev)
         self.grads = DeviceScene(self.row_capacity, self.sh_degree, dev)
         self.proj = ProjectedBuffers(self.n, self.row_capacity, dev)
         z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=dev)  # noqa: E731
@@ -225,8 +228,13 @@ class ViewTrainer:
                           self.evidence, self.evidence_sum, self.ws, stream)
 
     def sparse_adam(self, lr, beta1, beta2, eps, step: int, stream=None) -> None:
-        B.odin_sparse_adam(self.ctx, self.params.struct, self.m.struct, self.v.struct, self.grads.struct,
-                           self._row_zero_in_use, self.idx, self.count, lr, beta1, beta2, eps, step, stream)
+        B.odin_sparse_adam_live(self.ctx, self.params.struct, self.m.struct, self.v.struct, self.grads.struct,
+                                self._row_zero_in_use, self.idx, self.count, self.live, lr, beta1, beta2, eps, step,
+                                stream)
+
+    def moments_changed(self, stream=None) -> None:
+        """Recompute the per-primitive flags of the optimizer after self.m / self.v were written from outside."""
+        B.odin_adam_live_refresh(self.ctx, self.m.struct, self.v.struct, self.live, stream)
 
     def conflict_count(self, d_pairs, n_pairs: int, d_counts, stream=None) -> None:
         B.odin_conflict_count(self.ctx, self.masks, self.mask_slots, self.masks.shape[1], self.n, d_pairs, n_pairs,
@@ -313,8 +321,8 @@ class ViewTrainer:
         (ga, ia, ca, _), (gb, ib, cb, _) = per_view
         B.odin_accumulate_rows(self.ctx, ga.struct, zero_flags[0], ia, ca, gb.struct, zero_flags[1], ib, cb, u["idx_u"],
                                u["count_u"], u["grads_u"].struct, stream)
-        B.odin_sparse_adam(self.ctx, self.params.struct, self.m.struct, self.v.struct, u["grads_u"].struct, None,
-                           u["idx_u"], u["count_u"], lr, beta1, beta2, eps, step, stream)
+        B.odin_sparse_adam_live(self.ctx, self.params.struct, self.m.struct, self.v.struct, u["grads_u"].struct, None,
+                                u["idx_u"], u["count_u"], self.live, lr, beta1, beta2, eps, step, stream)
 
     def prepare_host_io(self, n_counts: int = 0):
         """Staging buffers, pinned result slots, copy stream and events of train_from_host (allocated once)."""

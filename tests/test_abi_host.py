@@ -69,6 +69,9 @@ def test_null_context_is_rejected_without_a_device(lib):
     assert lib.odin_sds_scores(null, None, 0, None, 0, None, 0, None, None) == B.ODIN_ERR_NULL
     assert lib.odin_sparse_adam(null, None, None, None, None, None, None, None, None, 0.9, 0.999, 1e-8, 1,
                                 None) == B.ODIN_ERR_NULL
+    assert lib.odin_sparse_adam_live(null, None, None, None, None, None, None, None, None, None, 0.9, 0.999, 1e-8, 1,
+                                     None) == B.ODIN_ERR_NULL
+    assert lib.odin_adam_live_refresh(null, None, None, None, None) == B.ODIN_ERR_NULL
     assert lib.odin_conflict_count(null, None, 0, 0, 0, None, 0, None, None) == B.ODIN_ERR_NULL
 
 

@@ -147,6 +147,64 @@ def test_sparse_adam_stage(oracle32, sh_degree, n, v):
     B.odin_destroy(ctx)
 
 
+@pytest.mark.parametrize("sh_degree,eps", [(3, 1e-15), (0, 1e-8), (2, 0.0)])
+def test_sparse_adam_live_flags(sh_degree, eps):
+    """The update with per-primitive flags equals the update without them bit for bit, over several steps with changing
+    row lists, zero rows (flagged and unflagged) and partially zero rows; the flags keep their promise (a clear flag
+    means zero moments) and the refresh call gives exactly `any moment non-zero`."""
+    rng = np.random.default_rng(11 + sh_degree)
+    n, k = 20_000, (sh_degree + 1) ** 2
+    f = 11 + 3 * k
+    dev = torch.device("cuda", 0)
+    ctx = B.odin_create(0)
+    p0 = wl.Scene(sh_degree, *[rng.standard_normal(s).astype(np.float32) for s in ((n, 3), (n, 3), (n, 4), (n,), (n, k, 3))])
+    sides = []
+    for _ in range(2):
+        sides.append((DeviceScene.from_host(p0, dev), DeviceScene(n, sh_degree, dev), DeviceScene(n, sh_degree, dev)))
+    live = torch.zeros(n, dtype=torch.uint8, device=dev)
+    lr = np.array([1e-3, 2e-3, 5e-4, 1e-2, 3e-3, 1e-4], np.float32)
+
+    def any_moment(m, v):
+        return torch.stack([(t.reshape(n, -1) != 0).any(dim=1) for s in (m, v) for t in s.tensors()]).any(dim=0)
+
+    for step in range(1, 7):
+        v = int(rng.integers(2000, 9000))
+        idx = np.sort(rng.choice(n, v, replace=False)).astype(np.uint32)
+        rows = rng.standard_normal((v, f)).astype(np.float32)
+        kind = rng.random(v)
+        rows[kind < 0.5] = 0                         # no gradient at all ...
+        flagged = kind < 0.3                         # ... most of them flagged, the gradient block then holds NaN
+        part = (kind >= 0.5) & (kind < 0.7)          # gradient in a few words only
+        rows[part] *= (rng.random((int(part.sum()), f)) < 0.05)
+        rows_dev = rows.copy()
+        rows_dev[flagged] = np.nan
+        g = wl.Scene(sh_degree, rows_dev[:, 0:3], rows_dev[:, 3:6], rows_dev[:, 6:10], rows_dev[:, 10],
+                     rows_dev[:, 11:].reshape(v, k, 3))
+        dg = DeviceScene.from_host(g, dev)
+        d_zero = torch.from_numpy(flagged.astype(np.uint8)).to(dev) if step % 3 else None
+        if d_zero is None:                           # every third step without the row flags: zeros are read as zeros
+            dg = DeviceScene.from_host(wl.Scene(sh_degree, rows[:, 0:3], rows[:, 3:6], rows[:, 6:10], rows[:, 10],
+                                                rows[:, 11:].reshape(v, k, 3)), dev)
+        d_idx = torch.from_numpy(idx.view(np.int32)).to(dev)
+        d_count = torch.tensor([v], dtype=torch.int32, device=dev)
+        (pa, ma, va), (pb, mb, vb) = sides
+        B.odin_sparse_adam(ctx, pa.struct, ma.struct, va.struct, dg.struct, d_zero, d_idx, d_count, lr, 0.9, 0.999, eps, step)
+        B.odin_sparse_adam_live(ctx, pb.struct, mb.struct, vb.struct, dg.struct, d_zero, d_idx, d_count, live, lr, 0.9,
+                                0.999, eps, step)
+        assert B.odin_poll(ctx) == B.ODIN_OK
+        for sa, sb in zip(sides[0], sides[1]):
+            for ta, tb in zip(sa.tensors(), sb.tensors()):
+                assert torch.equal(ta.view(torch.int32), tb.view(torch.int32)), step
+        truth = any_moment(mb, vb)
+        assert not bool((truth & (live == 0)).any()), step        # a clear flag promises zero moments
+        if eps > 0:
+            assert int(live.sum().item()) < n                      # and the flags are not trivially all set
+        fresh = torch.full((n,), 7, dtype=torch.uint8, device=dev)
+        B.odin_adam_live_refresh(ctx, mb.struct, vb.struct, fresh)
+        assert torch.equal(fresh.bool(), truth), step
+    B.odin_destroy(ctx)
+
+
 # ------------------------------------------------------------------------------------------------ projection
 def check_projection(oracle32, scene, cam, row_capacity=None, cfg=None):
     tr = G.trainer_for(scene, cam, row_capacity=row_capacity, cfg=cfg)
