@@ -8,14 +8,6 @@
 
 #include "../../include/odin.h"
 
-// Four bytes from global to shared memory without a register in between; the issuing thread waits for its own copies
-// with odin_copy_async_wait, a barrier then shows them to the block.
-__device__ __forceinline__ void odin_copy_async_u32(uint32_t* smem_dst, const uint32_t* gmem_src) {
-  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void odin_copy_async_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-
 // Kernel ids for launch counting and optional per-kernel CUDA-event timing.
 enum OdinKernelId {
   K_PROJECT = 0, K_TOUCHED, K_EMIT, K_ONESWEEP, K_FWD, K_L1, K_ZERO_ROWS,
