@@ -293,7 +293,7 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
 // sorted_off[i] = number of instances of the rows in front of position i of the depth order: an exclusive scan of the
 // rectangles' tile counts gathered through sorted_row.  2048 positions per block, one decoupled look-back per block,
 // blocks ordered by ticket.
-constexpr int RO_THREADS = 256;
+constexpr int RO_THREADS = 1024;
 constexpr int RO_ITEMS = OFFSET_TILE / RO_THREADS;
 // the instances are emitted in chunks of DUP_CHUNK consecutive slots (emit_instances_kernel)
 constexpr int DUP_THREADS = 256;
@@ -1119,7 +1119,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
       const size_t smem = ((size_t)F.tiles_pad + 8) * 4;
       const int max_smem = (int)(((size_t)SCATTER_MAX_TILES + 64 + 8) * 4);
       static_assert(RO_THREADS * RO_ITEMS == (int)OFFSET_TILE && 1024 * 2 == (int)OFFSET_TILE, "rows per chunk");
-      ODIN_CUDA(cudaFuncSetAttribute(chunk_counts_kernel<false, RO_THREADS, RO_ITEMS>,
+      ODIN_CUDA(cudaFuncSetAttribute(chunk_counts_kernel<false, 1024, 2>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
       ODIN_CUDA(cudaFuncSetAttribute(chunk_counts_kernel<true, 1024, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      max_smem));
@@ -1130,7 +1130,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
                         proj->num_instances, cap32, TX, n_tiles, F.tiles_pad, sorted_off, sorted_rect, geo4, geo2,       \
                         counts, tickets + 8, scan_state, ctx->d_status, ctx->spin_limit))
       if (exact) LAUNCH_COUNTS(true, 1024, 2);
-      else LAUNCH_COUNTS(false, RO_THREADS, RO_ITEMS);
+      else LAUNCH_COUNTS(false, 1024, 2);
 #undef LAUNCH_COUNTS
     }
     {
