@@ -77,18 +77,19 @@ __device__ __forceinline__ uint32_t odin_match_digit(uint32_t d) {
 }
 
 // ------------------------------------------------------------------------------------------------ onesweep pass
-constexpr int OS_THREADS = 256;
-constexpr int OS_WARPS = OS_THREADS / 32;
+constexpr int OS_THREADS = 256;                           // threads per block in the passes over the instances
+constexpr int OS_ROW_THREADS = 512;                       // ... and over the rows: one wave of tiles whose duration is the
+                                                          // latency of a tile, so the tile is spread over more threads
+static_assert(OS_THREADS >= (int)SORT_RADIX && OS_ROW_THREADS >= (int)SORT_RADIX, "thread d owns digit d");
 constexpr int OS_INST_ITEMS = SORT_TILE / OS_THREADS;     // 16 keys per thread in the passes over the instances
-constexpr int OS_ROW_ITEMS = ROW_SORT_TILE / OS_THREADS;  // 8 in the passes over the rows (512 / 1024 / 2048 / 4096 keys per
+constexpr int OS_ROW_ITEMS = ROW_SORT_TILE / OS_ROW_THREADS;  // 4 in the passes over the rows (512 / 1024 / 2048 / 4096 keys per
                                                           // tile: 0.074 / 0.070 / 0.064 / 0.065 ms for the four passes at 317 k rows)
-constexpr int OS_DPT = SORT_RADIX / OS_THREADS;   // digits owned by a thread
 constexpr int OS_INST_WINDOW = 2;                 // predecessors fetched per look-back step and digit (instances)
 constexpr int OS_ROW_WINDOW = 8;                  // ... and in the passes over the rows
 constexpr int OS_BLOCKS = 4;                    // resident blocks per SM
 constexpr uint32_t OS_FLAG_AGG = 1u << 30, OS_FLAG_INC = 2u << 30, OS_VALUE = (1u << 30) - 1;
-constexpr size_t os_smem_bytes(int items) {
-  return (size_t)items * OS_THREADS * 8 + (size_t)OS_WARPS * SORT_RADIX * 4 + 2 * SORT_RADIX * 4 + 16;
+constexpr size_t os_smem_bytes(int items, int threads) {
+  return (size_t)items * threads * 8 + (size_t)(threads / 32) * SORT_RADIX * 4 + 2 * SORT_RADIX * 4 + 16;
 }
 
 // One pass over one 8-bit digit of 32-bit keys.  Persistent blocks take 4096-key tiles by ticket.  Per tile:
@@ -101,8 +102,8 @@ constexpr size_t os_smem_bytes(int items) {
 //   the number of keys is *count32 if given, else min(*count64, capacity)
 //   ITEMS keys per thread, ITEMS * 256 per tile: 16 for the instances; 8 for the rows, of which there are so few that a
 //   pass is one wave of blocks and its duration is the latency of one tile, mostly the ITEMS-long ranking chain
-template <bool WIDE, int ITEMS, int WINDOW>
-__global__ void __launch_bounds__(OS_THREADS, OS_BLOCKS)
+template <bool WIDE, int ITEMS, int WINDOW, int THREADS>
+__global__ void __launch_bounds__(THREADS, OS_BLOCKS * OS_THREADS / THREADS)
 onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in, uint32_t* __restrict__ keys_out,
                 uint32_t* __restrict__ vals_out, uint64_t* __restrict__ keys64_out, const uint32_t* __restrict__ depth_bits,
                 const uint32_t* __restrict__ count32, const uint64_t* __restrict__ count64, uint64_t capacity, int shift,
@@ -111,7 +112,10 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
   odin_after_predecessor();  // launched behind the histogram / the pass in front
   extern __shared__ __align__(16) unsigned char os_smem[];
   uint32_t* s_keys = reinterpret_cast<uint32_t*>(os_smem);
-  constexpr uint32_t TILE = (uint32_t)ITEMS * OS_THREADS;
+  constexpr uint32_t TILE = (uint32_t)ITEMS * THREADS;
+  constexpr int OS_WARPS = THREADS / 32;
+  constexpr int OS_DPT = 1;  // thread d owns digit d; the threads beyond the radix own none
+  const bool owner = threadIdx.x < SORT_RADIX;
   uint32_t* s_vals = s_keys + TILE;
   uint32_t(*s_warp_hist)[SORT_RADIX] = reinterpret_cast<uint32_t(*)[SORT_RADIX]>(s_vals + TILE);
   uint32_t* s_digit_start = &s_warp_hist[0][0] + OS_WARPS * SORT_RADIX;
@@ -151,7 +155,7 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
   load_tile(tile);
 
   while (tile < ntiles) {
-    for (int i = threadIdx.x; i < OS_WARPS * (int)SORT_RADIX; i += OS_THREADS) (&s_warp_hist[0][0])[i] = 0;
+    for (int i = threadIdx.x; i < OS_WARPS * (int)SORT_RADIX; i += THREADS) (&s_warp_hist[0][0])[i] = 0;
     __syncthreads();
     const uint32_t tile_base = tile * TILE;
     const uint32_t tile_count = min(TILE, M - tile_base);
@@ -179,16 +183,18 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
     uint32_t cta_count[OS_DPT];
 #pragma unroll
     for (int q = 0; q < OS_DPT; ++q) {
-      const uint32_t d = threadIdx.x + q * OS_THREADS;
+      const uint32_t d = threadIdx.x;
       uint32_t c = 0;
+      if (owner) {
 #pragma unroll
-      for (int w = 0; w < OS_WARPS; ++w) {
-        const uint32_t t = s_warp_hist[w][d];
-        s_warp_hist[w][d] = c;
-        c += t;
+        for (int w = 0; w < OS_WARPS; ++w) {
+          const uint32_t t = s_warp_hist[w][d];
+          s_warp_hist[w][d] = c;
+          c += t;
+        }
+        st_volatile_u32(states + (size_t)tile * SORT_RADIX + d, (tile == 0 ? OS_FLAG_INC : OS_FLAG_AGG) | c);
       }
       cta_count[q] = c;
-      st_volatile_u32(states + (size_t)tile * SORT_RADIX + d, (tile == 0 ? OS_FLAG_INC : OS_FLAG_AGG) | c);
     }
     uint32_t digit_start[OS_DPT];
     {
@@ -197,14 +203,14 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
       for (int q = 0; q < OS_DPT; ++q) {  // digits ascend with q first, so the scans chain
         uint32_t total;
         digit_start[q] = carry + odin_block_exclusive_sum(cta_count[q], s_scan, &total);
-        s_digit_start[threadIdx.x + q * OS_THREADS] = digit_start[q];
+        if (owner) s_digit_start[threadIdx.x] = digit_start[q];
         carry += total;
       }
     }
     uint32_t exclusive[OS_DPT];
 #pragma unroll
     for (int q = 0; q < OS_DPT; ++q) exclusive[q] = 0;
-    if (tile > 0) {
+    if (tile > 0 && owner) {
       // walk back over the predecessors for all owned digits at once
       int64_t t[OS_DPT];
 #pragma unroll
@@ -222,7 +228,7 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
 #pragma unroll
           for (int k = 0; k < WINDOW; ++k)
             s[q][k] = (t[q] - k >= 0)
-                          ? ld_volatile_u32(states + (size_t)(t[q] - k) * SORT_RADIX + threadIdx.x + q * OS_THREADS)
+                          ? ld_volatile_u32(states + (size_t)(t[q] - k) * SORT_RADIX + threadIdx.x)
                           : 0u;
 #pragma unroll
         for (int q = 0; q < OS_DPT; ++q) {
@@ -245,13 +251,13 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
       }
 #pragma unroll
       for (int q = 0; q < OS_DPT; ++q)
-        st_volatile_u32(states + (size_t)tile * SORT_RADIX + threadIdx.x + q * OS_THREADS,
+        st_volatile_u32(states + (size_t)tile * SORT_RADIX + threadIdx.x,
                         OS_FLAG_INC | ((exclusive[q] + cta_count[q]) & OS_VALUE));
     }
 #pragma unroll
     for (int q = 0; q < OS_DPT; ++q) {
-      const uint32_t d = threadIdx.x + q * OS_THREADS;
-      s_global[d] = digit_base[d] + exclusive[q] - digit_start[q];  // + slot index inside the tile = address
+      const uint32_t d = threadIdx.x;
+      if (owner) s_global[d] = digit_base[d] + exclusive[q] - digit_start[q];  // + slot index inside the tile = address
     }
     __syncthreads();
 
@@ -268,7 +274,7 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
     load_tile(next);  // in flight while the current tile is written out
 #pragma unroll
     for (int j = 0; j < ITEMS; ++j) {
-      const uint32_t slot = j * OS_THREADS + threadIdx.x;
+      const uint32_t slot = j * THREADS + threadIdx.x;
       if (slot < tile_count) {
         const uint32_t k = s_keys[slot];
         const uint32_t dst = s_global[(k >> shift) & (SORT_RADIX - 1)] + slot;
@@ -1086,17 +1092,18 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     ODIN_CUDA(odin_launch(ctx, false, row_hist_kernel, dim3(row_blocks < sms * 4 ? row_blocks : sms * 4), dim3(256), 0, st,
                           depth_bits, proj->num_rows, hist, dbase, tickets + 9));
   }
-  constexpr size_t OS_SMEM = os_smem_bytes(OS_INST_ITEMS), OS_ROW_SMEM = os_smem_bytes(OS_ROW_ITEMS);
+  constexpr size_t OS_SMEM = os_smem_bytes(OS_INST_ITEMS, OS_THREADS), OS_ROW_SMEM = os_smem_bytes(OS_ROW_ITEMS, OS_ROW_THREADS);
   const uint32_t* sorted_row = nullptr;
   {
-    const uint32_t grid = row_tiles < sms * OS_BLOCKS ? row_tiles : sms * OS_BLOCKS;
+    const uint32_t row_resident = sms * (OS_BLOCKS * OS_THREADS / OS_ROW_THREADS);
+    const uint32_t grid = row_tiles < row_resident ? row_tiles : row_resident;
     const uint32_t* kin = depth_bits;
     const uint32_t* vin = nullptr;
     for (int p = 0; p < SORT_DEPTH_DIGITS; ++p) {
       OdinKernelScope ks(ctx, K_ROW_SORT, st);
       uint32_t* kout = (p + 1 < SORT_DEPTH_DIGITS) ? row_keys[p & 1] : nullptr;
       uint32_t* vout = row_vals[p & 1];
-      ODIN_CUDA(odin_launch(ctx, true, onesweep_kernel<false, OS_ROW_ITEMS, OS_ROW_WINDOW>, dim3(grid), dim3(OS_THREADS),
+      ODIN_CUDA(odin_launch(ctx, true, onesweep_kernel<false, OS_ROW_ITEMS, OS_ROW_WINDOW, OS_ROW_THREADS>, dim3(grid), dim3(OS_ROW_THREADS),
                             OS_ROW_SMEM, st, kin, vin, kout, vout, nullptr, nullptr, proj->num_rows, nullptr, 0,
                             p * (int)SORT_RADIX_BITS, dbase + p * SORT_RADIX,
                             row_states + (size_t)p * row_tiles * SORT_RADIX, tickets + p, ctx->d_status, ctx->spin_limit,
@@ -1164,9 +1171,9 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     }
     return odin_launch_status();
   }
-  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<false, OS_INST_ITEMS, OS_INST_WINDOW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<false, OS_INST_ITEMS, OS_INST_WINDOW, OS_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)OS_SMEM));
-  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<true, OS_INST_ITEMS, OS_INST_WINDOW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  ODIN_CUDA(cudaFuncSetAttribute(onesweep_kernel<true, OS_INST_ITEMS, OS_INST_WINDOW, OS_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)OS_SMEM));
   uint32_t* tile_diff = reinterpret_cast<uint32_t*>(base + L.tile_diff);
   uint32_t* inst_states = reinterpret_cast<uint32_t*>(base + L.inst_states);
@@ -1202,13 +1209,13 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
     OdinKernelScope ks(ctx, K_ONESWEEP, st);
     uint32_t* states = inst_states + (size_t)p * L.tiles * SORT_RADIX;
     if (p + 1 < tile_passes)
-      ODIN_CUDA(odin_launch(ctx, true, onesweep_kernel<false, OS_INST_ITEMS, OS_INST_WINDOW>, dim3(os_grid),
+      ODIN_CUDA(odin_launch(ctx, true, onesweep_kernel<false, OS_INST_ITEMS, OS_INST_WINDOW, OS_THREADS>, dim3(os_grid),
                             dim3(OS_THREADS), OS_SMEM, st, inst_keys[cur], inst_vals[cur], inst_keys[cur ^ 1],
                             inst_vals[cur ^ 1], nullptr, nullptr, nullptr, proj->num_instances, capacity,
                             p * (int)SORT_RADIX_BITS, tile_dbase + p * SORT_RADIX, states,
                             tickets + SORT_DEPTH_DIGITS + p, ctx->d_status, ctx->spin_limit, proj->capacity));
     else  // the sorted tile ids themselves are not needed any more: the ranges came from the tile counts
-      ODIN_CUDA(odin_launch(ctx, true, onesweep_kernel<true, OS_INST_ITEMS, OS_INST_WINDOW>, dim3(os_grid),
+      ODIN_CUDA(odin_launch(ctx, true, onesweep_kernel<true, OS_INST_ITEMS, OS_INST_WINDOW, OS_THREADS>, dim3(os_grid),
                             dim3(OS_THREADS), OS_SMEM, st, inst_keys[cur], inst_vals[cur], nullptr, inst_vals[cur ^ 1],
                             d_keys, depth_bits, nullptr, proj->num_instances, capacity, p * (int)SORT_RADIX_BITS,
                             tile_dbase + p * SORT_RADIX, states, tickets + SORT_DEPTH_DIGITS + p, ctx->d_status,
