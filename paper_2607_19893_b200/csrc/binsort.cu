@@ -77,7 +77,7 @@ __device__ __forceinline__ uint32_t odin_match_digit(uint32_t d) {
 }
 
 // ------------------------------------------------------------------------------------------------ onesweep pass
-constexpr int OS_THREADS = 256;                           // threads per block in the passes over the instances
+constexpr int OS_THREADS = 512;                           // threads per block in the passes over the instances
 constexpr int OS_ROW_THREADS = 512;                       // ... and over the rows: one wave of tiles whose duration is the
                                                           // latency of a tile, so the tile is spread over more threads
 static_assert(OS_THREADS >= (int)SORT_RADIX && OS_ROW_THREADS >= (int)SORT_RADIX, "thread d owns digit d");
@@ -86,7 +86,7 @@ constexpr int OS_ROW_ITEMS = ROW_SORT_TILE / OS_ROW_THREADS;  // 4 in the passes
                                                           // tile: 0.074 / 0.070 / 0.064 / 0.065 ms for the four passes at 317 k rows)
 constexpr int OS_INST_WINDOW = 2;                 // predecessors fetched per look-back step and digit (instances)
 constexpr int OS_ROW_WINDOW = 8;                  // ... and in the passes over the rows
-constexpr int OS_BLOCKS = 4;                    // resident blocks per SM
+constexpr int OS_RESIDENT = 1024;               // resident threads per SM
 constexpr uint32_t OS_FLAG_AGG = 1u << 30, OS_FLAG_INC = 2u << 30, OS_VALUE = (1u << 30) - 1;
 constexpr size_t os_smem_bytes(int items, int threads) {
   return (size_t)items * threads * 8 + (size_t)(threads / 32) * SORT_RADIX * 4 + 2 * SORT_RADIX * 4 + 16;
@@ -103,7 +103,7 @@ constexpr size_t os_smem_bytes(int items, int threads) {
 //   ITEMS keys per thread, ITEMS * 256 per tile: 16 for the instances; 8 for the rows, of which there are so few that a
 //   pass is one wave of blocks and its duration is the latency of one tile, mostly the ITEMS-long ranking chain
 template <bool WIDE, int ITEMS, int WINDOW, int THREADS>
-__global__ void __launch_bounds__(THREADS, OS_BLOCKS * OS_THREADS / THREADS)
+__global__ void __launch_bounds__(THREADS, OS_RESIDENT / THREADS)
 onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in, uint32_t* __restrict__ keys_out,
                 uint32_t* __restrict__ vals_out, uint64_t* __restrict__ keys64_out, const uint32_t* __restrict__ depth_bits,
                 const uint32_t* __restrict__ count32, const uint64_t* __restrict__ count64, uint64_t capacity, int shift,
@@ -1095,7 +1095,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   constexpr size_t OS_SMEM = os_smem_bytes(OS_INST_ITEMS, OS_THREADS), OS_ROW_SMEM = os_smem_bytes(OS_ROW_ITEMS, OS_ROW_THREADS);
   const uint32_t* sorted_row = nullptr;
   {
-    const uint32_t row_resident = sms * (OS_BLOCKS * OS_THREADS / OS_ROW_THREADS);
+    const uint32_t row_resident = sms * (OS_RESIDENT / OS_ROW_THREADS);
     const uint32_t grid = row_tiles < row_resident ? row_tiles : row_resident;
     const uint32_t* kin = depth_bits;
     const uint32_t* vin = nullptr;
@@ -1204,7 +1204,7 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
                           ctx->d_status, tile_diff, n_tiles, tile_passes, d_tile_ranges, tile_dbase));
   }
   // ---- instances by tile id
-  const uint32_t os_grid = L.tiles < sms * OS_BLOCKS ? L.tiles : sms * OS_BLOCKS;
+  const uint32_t os_grid = L.tiles < sms * (OS_RESIDENT / OS_THREADS) ? L.tiles : sms * (OS_RESIDENT / OS_THREADS);
   for (int p = 0; p < tile_passes; ++p) {
     OdinKernelScope ks(ctx, K_ONESWEEP, st);
     uint32_t* states = inst_states + (size_t)p * L.tiles * SORT_RADIX;
