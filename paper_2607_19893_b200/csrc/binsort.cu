@@ -81,9 +81,9 @@ constexpr int OS_THREADS = 512;                           // threads per block i
 constexpr int OS_ROW_THREADS = 512;                       // ... and over the rows: one wave of tiles whose duration is the
                                                           // latency of a tile, so the tile is spread over more threads
 static_assert(OS_THREADS >= (int)SORT_RADIX && OS_ROW_THREADS >= (int)SORT_RADIX, "thread d owns digit d");
-constexpr int OS_INST_ITEMS = SORT_TILE / OS_THREADS;     // 16 keys per thread in the passes over the instances
-constexpr int OS_ROW_ITEMS = ROW_SORT_TILE / OS_ROW_THREADS;  // 4 in the passes over the rows (512 / 1024 / 2048 / 4096 keys per
-                                                          // tile: 0.074 / 0.070 / 0.064 / 0.065 ms for the four passes at 317 k rows)
+constexpr int OS_INST_ITEMS = SORT_TILE / OS_THREADS;     // 8 keys per thread in the passes over the instances
+constexpr int OS_ROW_ITEMS = ROW_SORT_TILE / OS_ROW_THREADS;  // 4 in the passes over the rows (tiles of 512 / 1024 / 2048 /
+                                                          // 4096 keys on 256 threads: 0.074 / 0.070 / 0.064 / 0.065 ms for the four passes at 317 k rows)
 constexpr int OS_INST_WINDOW = 2;                 // predecessors fetched per look-back step and digit (instances)
 constexpr int OS_ROW_WINDOW = 8;                  // ... and in the passes over the rows
 constexpr int OS_RESIDENT = 1024;               // resident threads per SM
@@ -92,16 +92,18 @@ constexpr size_t os_smem_bytes(int items, int threads) {
   return (size_t)items * threads * 8 + (size_t)(threads / 32) * SORT_RADIX * 4 + 2 * SORT_RADIX * 4 + 16;
 }
 
-// One pass over one 8-bit digit of 32-bit keys.  Persistent blocks take 4096-key tiles by ticket.  Per tile:
-// warp-striped loads, per-warp digit ranking (stable; match.any, or eight ballots in the passes over the rows), block
+// One pass over one 8-bit digit of 32-bit keys.  Persistent blocks take tiles of ITEMS * THREADS keys by ticket.  Per tile:
+// warp-striped loads, per-warp digit ranking (stable; eight ballots per key), block
 // digit counts published for look-back, exclusive global digit offsets by a per-digit look-back walk (thread d walks digit d), keys and values exchanged
 // through shared memory so that the global scatter writes runs of consecutive addresses.
 //   vals_in == nullptr: the values are the positions themselves (first pass over the rows)
 //   keys_out == nullptr: the keys are not needed afterwards (last pass over the rows)
 //   WIDE: the last pass over the instances may also write the full 64-bit key key << 32 | depth_bits[value]
 //   the number of keys is *count32 if given, else min(*count64, capacity)
-//   ITEMS keys per thread, ITEMS * 256 per tile: 16 for the instances; 8 for the rows, of which there are so few that a
-//   pass is one wave of blocks and its duration is the latency of one tile, mostly the ITEMS-long ranking chain
+//   ITEMS keys per thread on THREADS threads: 8 x 512 for the instances, 4 x 512 for the rows, of which there are so few
+//   that a pass is one wave of blocks and its duration is the latency of one tile (with 256 threads per tile the
+//   ITEMS-long ranking chain and the write-out were twice as long: whole step 0.870 -> 0.855 ms at 317 k rows; the two
+//   instance passes at 1.9 M instances 0.084 -> 0.075 ms)
 template <bool WIDE, int ITEMS, int WINDOW, int THREADS>
 __global__ void __launch_bounds__(THREADS, OS_RESIDENT / THREADS)
 onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in, uint32_t* __restrict__ keys_out,
@@ -164,9 +166,9 @@ onesweep_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict
 #pragma unroll
     for (int j = 0; j < ITEMS; ++j) {
       const uint32_t d = (key[j] >> shift) & (SORT_RADIX - 1);
-      // (measured: ballots 0.060 against 0.064 ms for the four row passes at 317 k rows; the instance passes at 1.9 M
-      // instances 0.086 against 0.085 ms, so they keep the single instruction)
-      const uint32_t peers = ITEMS <= 8 ? odin_match_digit(d) : __match_any_sync(0xffffffffu, d);
+      // (measured: ballots 0.060 against 0.064 ms with match.any for the four row passes at 317 k rows; no difference
+      // in the passes over 1.9 M instances)
+      const uint32_t peers = odin_match_digit(d);
       const int leader = __ffs(peers) - 1;
       uint32_t old = 0;
       if ((int)lane == leader) {
