@@ -352,8 +352,29 @@ def test_chained_calls_equal_unchained_calls(monkeypatch):
             assert abs(float(a.loss.item()) - float(b.loss.item())) <= 1e-6 * abs(float(b.loss.item()))
             ga, gb = a.gradient_rows(v), b.gradient_rows(v)
             assert np.allclose(ga, gb, rtol=1e-4, atol=1e-9 * max(1.0, float(np.abs(gb).max())))
-            for ta, tb in zip(a.params.tensors(), b.params.tensors()):
-                assert torch.allclose(ta, tb, rtol=1e-5, atol=1e-6)
+            # Parameters: equal where the gradient is above the noise of the atomic sums.  Adam normalises its step, so an
+            # element whose gradient is itself of the size of that noise (a cancelled sum that comes out as 1e-12 on one
+            # side and -1e-12 or 0 on the other) may move by up to a few learning rates on one side and not on the other:
+            # such elements must be few, their gradients must be noise on both sides, and the move must be of that size.
+            idx = a.idx[:v].long()
+            assert torch.equal(a.idx[:v], b.idx[:v])
+            noise = 16.0 * float(np.abs(ga - gb).max()) + 1e-30
+            cols = 0
+            n_bad = n_all = 0
+            group_lr = [w.lr[0], w.lr[1], w.lr[2], w.lr[3], max(w.lr[4], w.lr[5])]
+            for ta, tb, lr_g in zip(a.params.tensors(), b.params.tensors(), group_lr):
+                rest = torch.ones(ta.shape[0], dtype=torch.bool, device=ta.device)
+                rest[idx] = False
+                assert torch.equal(ta[rest].view(torch.int32), tb[rest].view(torch.int32))  # unlisted: untouched
+                xa, xb = ta[idx].reshape(v, -1).cpu().numpy(), tb[idx].reshape(v, -1).cpu().numpy()
+                width = xa.shape[1]
+                bad = np.abs(xa - xb) > 1e-6 + 1e-5 * np.abs(xb)
+                g_a, g_b = ga[:, cols:cols + width], gb[:, cols:cols + width]
+                assert np.all(np.abs(g_a[bad]) <= noise) and np.all(np.abs(g_b[bad]) <= noise), (s, cols)
+                assert np.all(np.abs(xa - xb)[bad] <= 10.0 * lr_g), (s, cols)
+                n_bad += int(bad.sum()); n_all += bad.size
+                cols += width
+            assert n_bad <= 1e-3 * n_all, (n_bad, n_all)
         a.close()
         b.close()
 
