@@ -12,7 +12,7 @@
 
 namespace {
 
-// Called by every thread of a 256-thread block after the block's last update of the global histograms.  The block that
+// Called by every thread of a block of 256 threads or more after the block's last update of the global histograms.  The block that
 // arrives last of `expected` turns the `digits` 256-bin histograms into exclusive scans (the digit bases of the passes),
 // which saves a launch per histogram kernel.  s_warp: 33 words, s_flag: 1 word of shared memory.
 __device__ __forceinline__ void last_block_digit_bases(const uint32_t* hist, uint32_t* __restrict__ base, int digits,
@@ -25,9 +25,11 @@ __device__ __forceinline__ void last_block_digit_bases(const uint32_t* hist, uin
   if (!*s_flag) return;
   __threadfence();
   for (int d = 0; d < digits; ++d) {
-    const uint32_t h = ld_volatile_u32(hist + d * SORT_RADIX + threadIdx.x);
+    const bool owner = threadIdx.x < SORT_RADIX;  // thread d scans digit d; a larger block's other threads add nothing
+    const uint32_t h = owner ? ld_volatile_u32(hist + d * SORT_RADIX + threadIdx.x) : 0u;
     uint32_t total;
-    base[d * SORT_RADIX + threadIdx.x] = odin_block_exclusive_sum(h, s_warp, &total);
+    const uint32_t e = odin_block_exclusive_sum(h, s_warp, &total);
+    if (owner) base[d * SORT_RADIX + threadIdx.x] = e;
   }
 }
 
@@ -35,13 +37,14 @@ __device__ __forceinline__ void last_block_digit_bases(const uint32_t* hist, uin
 // Digit histograms of the depth bits of all rows, for the SORT_DEPTH_DIGITS row passes, and their exclusive scans.
 // Plain shared atomics: aggregating the equal digits of a warp with match.any first (the high digits of a depth take
 // few distinct values) was slower, 0.023 against 0.016 ms for 317 k rows - the match costs more than the conflicts.
-__global__ void __launch_bounds__(256)
+constexpr int RH_THREADS = 1024;
+__global__ void __launch_bounds__(RH_THREADS)
 row_hist_kernel(const uint32_t* __restrict__ depth_bits, const uint32_t* __restrict__ num_rows, uint32_t* __restrict__ hist,
                 uint32_t* __restrict__ base, uint32_t* arrivals) {
   odin_after_predecessor();
   __shared__ uint32_t s_hist[SORT_DEPTH_DIGITS][SORT_RADIX];
   __shared__ uint32_t s_warp[33], s_flag;
-  for (int i = threadIdx.x; i < SORT_DEPTH_DIGITS * (int)SORT_RADIX; i += 256) (&s_hist[0][0])[i] = 0;
+  for (int i = threadIdx.x; i < SORT_DEPTH_DIGITS * (int)SORT_RADIX; i += RH_THREADS) (&s_hist[0][0])[i] = 0;
   __syncthreads();
   const uint32_t V = *num_rows;
   const unsigned lane = threadIdx.x & 31;
@@ -57,7 +60,7 @@ row_hist_kernel(const uint32_t* __restrict__ depth_bits, const uint32_t* __restr
     }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < SORT_DEPTH_DIGITS * (int)SORT_RADIX; i += 256) {
+  for (int i = threadIdx.x; i < SORT_DEPTH_DIGITS * (int)SORT_RADIX; i += RH_THREADS) {
     const uint32_t c = (&s_hist[0][0])[i];
     if (c) atomicAdd(&hist[i], c);
   }
@@ -1085,13 +1088,13 @@ extern "C" int odin_bin_sort(odin_ctx* ctx, const odin_projected* proj, int widt
   const uint32_t* depth_bits = reinterpret_cast<const uint32_t*>(proj->depth);
   const ushort4* rect = reinterpret_cast<const ushort4*>(proj->rect);
   const uint32_t sms = (uint32_t)ctx->sm_count;
-  const uint32_t row_blocks = (proj->capacity + 255) / 256;
+  const uint32_t row_blocks = (proj->capacity + RH_THREADS - 1) / RH_THREADS;
 
   // ---- rows by depth
   {
     OdinKernelScope ks(ctx, K_ROW_HIST, st);
     // one block per SM at most: every block ends with 1024 global reductions onto the same 1024 words
-    ODIN_CUDA(odin_launch(ctx, false, row_hist_kernel, dim3(row_blocks < sms * 4 ? row_blocks : sms * 4), dim3(256), 0, st,
+    ODIN_CUDA(odin_launch(ctx, false, row_hist_kernel, dim3(row_blocks < sms ? row_blocks : sms), dim3(RH_THREADS), 0, st,
                           depth_bits, proj->num_rows, hist, dbase, tickets + 9));
   }
   constexpr size_t OS_SMEM = os_smem_bytes(OS_INST_ITEMS, OS_THREADS), OS_ROW_SMEM = os_smem_bytes(OS_ROW_ITEMS, OS_ROW_THREADS);
