@@ -88,6 +88,25 @@ def rows_bound(oracle, scene, cam, idx, clamp_flags, rows_o, want2d_dense, abs2d
     return bound
 
 
+def assert_states_close(tensors_a, tensors_b, lr, steps, rtol=1e-4, atol=1e-6, max_fraction=1e-4):
+    """Two runs of the same steps whose only difference is the order of the backward pass's atomic sums.  The optimizer
+    normalises its step by the gradient's own magnitude, so an element whose gradient is a cancelled sum of the size of
+    that rounding noise may move by learning rates in one run and not in the other.  Everything else must agree: at most
+    `max_fraction` of the elements may lie outside rtol / atol, and none by more than the optimizer can move it in
+    `steps` steps."""
+    bad = total = 0
+    worst = 0.0
+    for ta, tb in zip(tensors_a, tensors_b):
+        d = (ta - tb).abs()
+        out = d > atol + rtol * tb.abs()
+        bad += int(out.sum().item())
+        total += d.numel()
+        if bool(out.any()):
+            worst = max(worst, float(d[out].max().item()))
+    assert bad <= max_fraction * total, (bad, total)
+    assert worst <= 10.0 * float(max(lr)) * steps, worst
+
+
 # ---------------------------------------------------------------------------------------------------------------
 # Measured distances to the bars are printed (pytest -rP or -s shows them) so that every slack factor in the chained
 # tests can be read against what the device actually does.

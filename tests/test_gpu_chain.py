@@ -407,8 +407,7 @@ def test_train_from_host_equals_the_plain_loop():
     assert [g[0] for g in got] == steps
     for g, x in zip(got, want):
         assert g[2] == x[2] and g[3] == x[3] and abs(g[1] - x[1]) < 1e-6
-    for ta, tb in zip(a.params.tensors(), b.params.tensors()):
-        assert torch.allclose(ta, tb, rtol=1e-4, atol=1e-6)
+    G.assert_states_close(a.params.tensors(), b.params.tensors(), w.lr, len(steps))
     a.close(); b.close()
 
 

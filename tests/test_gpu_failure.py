@@ -136,6 +136,5 @@ def test_checkpoint_resume_equals_the_uninterrupted_run():
     for x, y in zip(log_a, log_b):
         assert x[2] == y[2] and abs(x[1] - y[1]) < 1e-6
     for group in ("params", "m", "v"):
-        for ta, tc in zip(getattr(a, group).tensors(), getattr(c, group).tensors()):
-            assert torch.allclose(ta, tc, rtol=1e-4, atol=1e-6)
+        G.assert_states_close(getattr(a, group).tensors(), getattr(c, group).tensors(), w.lr, 10)
     a.close(); c.close()
